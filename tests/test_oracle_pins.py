@@ -1,0 +1,340 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself.
+
+P1  a budget equal to the whole residual (or sink+window covering the context) must give dense
+    SDPA, computed here independently (explicit de-paging loop + torch fp64 SDPA).
+P2  tiny inputs: top-k against a full sort, the residual against a set difference, and the
+    estimator averaged over ALL subsets of the residual must equal the exact sums; its variance
+    must equal the finite-population formula for sampling without replacement.
+P3  the (eps, delta) definition (Definition 4.1 of the paper) over 1,000 seeds.
+P4  closed-form budgets (Lemma 4.1, Corollaries D.2, Theorem 4.3) on hand-computable populations.
+P5  Philox4x32-10 against the published known-answer vectors.
+P6  the sampler is uniform over subsets (chi-square) and never selects outside the residual.
+"""
+import itertools
+import math
+import os
+import statistics
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import vattn_oracle as O
+from paper_2510_05688_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def ZQ(x):
+    """Phi^{-1}(1 - x/2) from the Python standard library (not the routine the oracle calls)."""
+    return statistics.NormalDist().inv_cdf(1.0 - 0.5 * x)
+
+
+# ----------------------------------------------------------------------------- helpers (independent of the oracle)
+def depage_loop(case, cache, b, g):
+    """Token-by-token de-paging, written independently of oracle.gather_rows."""
+    vals = case.values(cache).astype(np.float64)
+    n = int(case.seq_lens[b])
+    rows = np.zeros((n, case.head_dim))
+    for i in range(n):
+        rows[i] = vals[int(case.block_table[b, i // 16]), g, i % 16]
+    return rows
+
+
+def torch_sdpa(case, b, h, scale):
+    G = case.num_q_heads // case.num_kv_heads
+    g = h // G
+    K = torch.from_numpy(depage_loop(case, case.k_cache, b, g))
+    V = torch.from_numpy(depage_loop(case, case.v_cache, b, g))
+    q = torch.from_numpy(case.values(case.q)[b, h].astype(np.float64))[None, :]
+    o = torch.nn.functional.scaled_dot_product_attention(q[None, None], K[None, None], V[None, None], scale=scale)
+    return o[0, 0, 0].numpy()
+
+
+def small_case(dtype, seq_lens=(70, 33), Hq=4, Hkv=2, d=32, **kw):
+    args = dict(dtype=dtype, B=len(seq_lens), Hq=Hq, Hkv=Hkv, d=d, seq_lens=list(seq_lens), sink=3,
+                window=5, k=4, eps=0.05, delta=0.05, seed=11, gen_seed=77, rho_v=1.0,
+                heavy=dict(R=3, c1=3.0, alpha=(1.0, 1.0)))
+    args.update(kw)
+    return synth.make_case("small", **args)
+
+
+def run_oracle(case, **over):
+    p = dict(case.params)
+    p.update(over)
+    return O.vattn_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink,
+                          case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype, **p)
+
+
+# ----------------------------------------------------------------------------- P1
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_p1_full_residual_budget_equals_dense_sdpa(dtype):
+    case = small_case(dtype)
+    scale = float(np.float32(1.0 / math.sqrt(case.head_dim)))
+    out, det = run_oracle(case, force_budget=10**9)
+    for (b, h), r in det.items():
+        assert r["b"] == r["n_s"] and len(r["I_dyn"]) == r["n_s"]
+        ref = torch_sdpa(case, b, h, scale)
+        np.testing.assert_allclose(r["out"], ref, rtol=1e-12, atol=1e-13)
+    dense = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=dtype)
+    for (b, h) in det:
+        np.testing.assert_allclose(dense[b, h], torch_sdpa(case, b, h, scale), rtol=1e-12, atol=1e-13)
+
+
+def test_p1_sink_plus_window_cover_context():
+    case = small_case("fp32", sink=40, window=40)
+    scale = float(np.float32(1.0 / math.sqrt(case.head_dim)))
+    _, det = run_oracle(case)
+    for (b, h), r in det.items():
+        assert r["n_s"] == 0 and r["b"] == 0 and r["budgets"] == (0, 0, 0, 0)
+        assert len(r["I_f"]) == r["n"] and len(r["I_t"]) == 0
+        np.testing.assert_allclose(r["out"], torch_sdpa(case, b, h, scale), rtol=1e-12, atol=1e-13)
+
+
+def test_p1_explicit_scale_and_gqa_mapping():
+    # a different scale must change the result exactly as torch's scale= does; heads of one
+    # group share K/V but not q
+    case = small_case("fp32", seq_lens=(41,), Hq=6, Hkv=2, d=16)
+    _, det = run_oracle(case, force_budget=10**9, scale=0.37)
+    sc = float(np.float32(0.37))
+    for (b, h), r in det.items():
+        np.testing.assert_allclose(r["out"], torch_sdpa(case, b, h, sc), rtol=1e-12, atol=1e-13)
+
+
+def test_bf16_output_rounding_is_single_rne():
+    x = np.array([1.0, 1.00390625, 1.01171875, -3.0000001, 0.1, 1.0 + 2**-8 - 2**-30, 65280.0, 1e-3], np.float64)
+    got = O.f64_to_bf16_bits(x)
+    want = torch.tensor(x, dtype=torch.float64).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert (got == want).all()
+    # tie case: exactly halfway between two bf16 values goes to the even one
+    assert O.f64_to_bf16_bits(np.array([1.00390625]))[0] == 0x3F80       # 1 + 2^-8 -> 1.0
+    assert O.f64_to_bf16_bits(np.array([1.01171875]))[0] == 0x3F82       # 1 + 3*2^-8 -> 1 + 2^-6
+    # just above the halfway point must round up (a conversion through fp32 would lose the 2^-30
+    # and then break the tie downwards: the oracle rounds once)
+    assert O.f64_to_bf16_bits(np.array([1.0 + 2**-8 + 2**-30]))[0] == 0x3F81
+
+
+# ----------------------------------------------------------------------------- P2
+def test_p2_topk_and_residual_bruteforce():
+    rng = np.random.default_rng(5)
+    for trial in range(50):
+        n = int(rng.integers(1, 15))
+        s = rng.standard_normal(n).round(1)            # rounding creates ties
+        sink, window, k = int(rng.integers(0, 4)), int(rng.integers(0, 4)), int(rng.integers(0, 6))
+        I_f, I_t, R = O.deterministic_sets(s, sink, window, k)
+        ns_ = min(sink, n)
+        ls = max(n - window, ns_)
+        M = list(range(ns_, ls))
+        ranked = sorted(M, key=lambda i: (-s[i], i))   # full sort, ties -> lowest index
+        want_t = sorted(ranked[:min(k, len(M))])
+        assert list(I_t) == want_t
+        want_f = sorted(set(range(ns_)) | set(range(ls, n)) | set(want_t))
+        assert list(I_f) == want_f
+        assert list(R) == sorted(set(range(n)) - set(want_f))
+
+
+def test_p2_estimator_unbiased_over_all_subsets_and_variance():
+    rng = np.random.default_rng(9)
+    n, d = 12, 3
+    s = rng.standard_normal(n)
+    V = rng.standard_normal((n, d))
+    w = np.exp(s - s.max())
+    I_f, I_t, R = O.deterministic_sets(s, 1, 2, 2)
+    n_s = len(R)
+    assert n_s == 7
+    D_exact = w.sum()
+    N_exact = (w[:, None] * V).sum(axis=0)
+    for b in (1, 3, 7):
+        Ds, Ns = [], []
+        for sub in itertools.combinations(R.tolist(), b):
+            N, D = O.combine(w, V, I_f, np.array(sub), n_s)
+            Ds.append(D)
+            Ns.append(N)
+        Ds, Ns = np.array(Ds), np.array(Ns)
+        assert abs(Ds.mean() - D_exact) < 1e-12
+        np.testing.assert_allclose(Ns.mean(axis=0), N_exact, atol=1e-12)
+        # sampling without replacement: Var = n_s^2 (1 - b/n_s) S^2 / b, S^2 with n_s - 1
+        S2 = w[R].var(ddof=1)
+        assert abs(Ds.var() - n_s**2 * (1 - b / n_s) * S2 / b) < 1e-12
+    # b = n_s has a single subset and is exact
+    N, D = O.combine(w, V, I_f, R, n_s)
+    assert abs(D - D_exact) < 1e-14
+
+
+def test_p2_sample_is_smallest_key_index_pairs():
+    keys = np.array([5, 1, 9, 1, 7, 1, 3, 3], np.uint32)
+    R = np.array([1, 2, 3, 5, 6, 7])
+    pairs = sorted((int(keys[i]), int(i)) for i in R)
+    for c in range(0, 7):
+        want = sorted(i for _, i in pairs[:c])
+        assert O.sample(R, c, keys).tolist() == want
+    assert O.sample(R, 99, keys).tolist() == R.tolist()
+
+
+def test_sample_keys_layout_matches_philox_counter_definition():
+    n, seed, b, h, layer, step = 23, (0xDEADBEEF << 32) | 0x12345678, 3, 7, 5, 1000
+    for stream in (0, 1):
+        keys = O.sample_keys(n, seed, b, h, layer, step, stream)
+        for i in (0, 1, 2, 3, 4, 13, 22):
+            out = O.philox4x32_10(np.uint64(i >> 2), np.uint64((b << 16) | h), np.uint64(layer),
+                                  np.uint64((step << 1) | stream), seed & 0xFFFFFFFF, seed >> 32)
+            assert int(keys[i]) == int(out[i & 3])
+    assert not np.array_equal(O.sample_keys(n, seed, b, h, layer, step, 0), O.sample_keys(n, seed, b, h, layer, step, 1))
+
+
+# ----------------------------------------------------------------------------- P3
+def test_p3_eps_delta_definition_over_1000_seeds():
+    eps = delta = 0.1
+    case = synth.make_case("p3", dtype="fp32", B=1, Hq=1, Hkv=1, d=64, seq_lens=[8192], sink=128, window=128,
+                           k=int(0.025 * 8192), eps=eps, delta=delta, seed=0, gen_seed=31337, key_std=0.1,
+                           rho_v=2.0, heavy=None, params=dict(base_rate=0.025))
+    scale = float(np.float32(1.0 / 8.0))
+    ref = torch_sdpa(case, 0, 0, scale)
+    T, fails, used = 1000, 0, []
+    for seed in range(T):
+        case.seed = seed
+        _, det = run_oracle(case)
+        r = det[(0, 0)]
+        used.append(r["b"] / r["n_s"])
+        err = np.linalg.norm(r["out"] - ref) / np.linalg.norm(ref)
+        fails += err > eps
+    # the case must not be vacuous (budget well below the residual)
+    assert np.mean(used) < 0.5
+    slack = 3.0 * math.sqrt(delta * (1 - delta) / T)
+    assert fails / T <= delta + slack
+
+
+# ----------------------------------------------------------------------------- P4
+def test_p4_normal_quantiles_table():
+    for line in open(os.path.join(GOLD, "normal_quantiles.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        x, z = map(float, line.split())
+        assert abs(O.z_of(x) - z) < 6e-7
+
+
+def _stats(sigma2, trace, D_hat, N_norm):
+    return dict(sigma2=sigma2, trace=trace, D_hat=D_hat, N_hat_norm=N_norm)
+
+
+def test_p4_budget_closed_forms_and_scaling():
+    n_s, eps, delta = 1000, 0.125, 0.05          # eps exactly representable in fp32
+    st = _stats(0.04, 0.09, 500.0, 50.0)         # sigma = .2, sqrt(trace) = .3
+    b_D, b_N, b_S = O.budgets(st, n_s, eps, delta)
+    z = ZQ(float(np.float32(delta)))               # stdlib quantile: independent of the oracle's scipy call
+    assert abs(b_D - (z * n_s * 0.2 / (eps * 500.0)) ** 2) < 1e-9 * b_D
+    assert abs(b_N - (z * n_s * 0.3 / (eps * 50.0)) ** 2) < 1e-9 * b_N
+    # b(eps/2) = 4 b(eps) for all three
+    h_D, h_N, h_S = O.budgets(st, n_s, eps / 2, delta)
+    for a, b in ((h_D, b_D), (h_N, b_N), (h_S, b_S)):
+        assert abs(a - 4 * b) < 1e-9 * a
+    # Theorem: splitting eps and delta costs more than 4x either single-quantity budget,
+    # and the grid minimum is no worse than the midpoint split
+    assert b_S > 4 * max(b_D, b_N)
+    A, Bn = n_s * 0.2 / 500.0, n_s * 0.3 / 50.0
+    mid = 4 / eps**2 * (O.z_of(delta / 2) * (A + Bn)) ** 2
+    assert b_S <= mid * (1 + 1e-12)
+    # brute force over a fine (eps', delta') grid of the Theorem's min-max never beats the closed form by
+    # more than the grid resolution, and never exceeds it
+    best = math.inf
+    for dj in np.linspace(delta / 16, delta * 15 / 16, 15):
+        z1, z2 = O.z_of(dj), O.z_of(delta - dj)
+        for e1 in np.linspace(eps * 0.001, eps * 0.999, 4000):
+            val = max((z1 * A / (e1 / 2)) ** 2, (z2 * Bn / ((eps - e1) / 2)) ** 2)
+            best = min(best, val)
+    assert b_S <= best <= b_S * 1.01
+
+
+def test_p4_equal_residual_weights_give_base_budget():
+    # all keys identical -> all residual weights equal -> sigma^2 = 0 -> b_D = 0 -> b = b0 (D mode)
+    case = small_case("fp32", seq_lens=(400,), Hq=1, Hkv=1, d=16, heavy=None, sink=4, window=4, k=8)
+    vals = case.k_cache.copy()
+    vals[...] = vals[case.block_table[0, 0], 0, 0][None, None, None, :]
+    case.k_cache = vals
+    _, det = run_oracle(case, mode=1, base_rate=0.05)
+    r = det[(0, 0)]
+    assert r["stats"][1] == 0.0 and r["budgets"][0] == 0
+    assert r["b"] == r["b0"] == int(math.floor(float(np.float32(0.05)) * r["n_s"]))
+    # ties in the top-k go to the lowest indices of the middle range
+    assert r["I_t"].tolist() == list(range(4, 12))
+
+
+def test_p4_scalar_values_make_numerator_budget_equal_denominator_budget():
+    # d = 1 and V == 1: the numerator is the denominator, so b_N == b_D
+    rng = np.random.default_rng(3)
+    n = 300
+    K = rng.standard_normal((n, 1))
+    V = np.ones((n, 1))
+    r = O.decode_head(np.array([1.3]), K, V, sink=2, window=2, k=5, eps=0.05, delta=0.05, seed=1, batch_idx=0,
+                      head_idx=0, rng_head=0, base_rate=0.1, scale=1.0, mode=0)
+    b_D, b_N, _ = r["budgets_real"]
+    assert abs(b_D - b_N) <= 1e-12 * b_D
+
+
+def test_p4_two_point_population_by_hand():
+    # base sample = whole residual (base_rate 1): m tokens with weight a and m with weight b
+    m_, a, b = 20, 1.0, 0.5
+    n_s = 2 * m_
+    w = np.array([2.0] + [a] * m_ + [b] * m_)           # token 0 is the deterministic set, weight 2
+    V = np.ones((n_s + 1, 1))
+    st = O.base_stats(w, V, np.array([0]), np.arange(1, n_s + 1), n_s)
+    var = (n_s / (n_s - 1)) * ((a - b) / 2) ** 2        # unbiased sample variance of a two-point set
+    assert abs(st["sigma2"] - var) < 1e-15
+    D = 2.0 + m_ * (a + b)
+    assert abs(st["D_hat"] - D) < 1e-12 and abs(st["D_f"] - 2.0) < 1e-15
+    b_D, _, _ = O.budgets(st, n_s, 0.25, 0.05)
+    assert abs(b_D - (ZQ(float(np.float32(0.05))) * n_s * math.sqrt(var) / (0.25 * D)) ** 2) < 1e-9 * b_D
+    assert O.final_budget(b_D, 5, n_s) == min(max(math.ceil(b_D), 5), n_s)
+    assert O.final_budget(0.0, 5, n_s) == 5 and O.final_budget(1e30, 5, n_s) == n_s
+    assert O.final_budget(float("nan"), 5, n_s) == n_s and O.final_budget(3.2, 5, n_s, force_budget=7) == 7
+
+
+def test_base_sample_estimates_are_close_to_population_values():
+    # the paper's Table 9 reports a few % error for base-sample estimates at f_b = 0.025-0.1
+    case = synth.make_case("t9", dtype="fp32", B=1, Hq=1, Hkv=1, d=64, seq_lens=[16384], sink=128, window=128,
+                           k=409, eps=0.05, delta=0.05, seed=0, gen_seed=99, key_std=1.0, rho_v=1.0, heavy=None)
+    K = O.gather_rows(case.k_cache, case.block_table[0], 0, 16384, "fp32")
+    V = O.gather_rows(case.v_cache, case.block_table[0], 0, 16384, "fp32")
+    q = O.to_f64(case.q[0, 0], "fp32")
+    s = O.scores(q, K, 0.125)
+    w = np.exp(s - s.max())
+    I_f, I_t, R = O.deterministic_sets(s, 128, 128, 409)
+    pop_sigma2 = w[R].var(ddof=1)
+    pop_trace = ((w[R, None] * V[R]).var(axis=0, ddof=1)).sum()
+    errs = []
+    for seed in range(40):
+        I_bs = O.sample(R, O.base_size(len(R), 0.1), O.sample_keys(16384, seed, 0, 0, 0, 0, 0))
+        st = O.base_stats(w, V, I_f, I_bs, len(R))
+        errs.append((abs(st["sigma2"] - pop_sigma2) / pop_sigma2, abs(st["trace"] - pop_trace) / pop_trace))
+    errs = np.array(errs).mean(axis=0)
+    assert errs[0] < 0.15 and errs[1] < 0.15
+
+
+# ----------------------------------------------------------------------------- P5
+def test_p5_philox_known_answer_vectors():
+    rows = 0
+    for line in open(os.path.join(GOLD, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        v = [int(x, 16) for x in line.split()]
+        out = O.philox4x32_10(*[np.array([c], np.uint64) for c in v[:4]], v[4], v[5])
+        assert [int(o[0]) for o in out] == v[6:]
+        rows += 1
+    assert rows == 3
+
+
+# ----------------------------------------------------------------------------- P6
+def test_p6_sampler_uniform_over_subsets():
+    n, c = 12, 3
+    R = np.array([2, 3, 5, 6, 7, 8, 9, 10])              # residual of size 8
+    subsets = {s: 0 for s in itertools.combinations(R.tolist(), c)}
+    T = 28000
+    incl = np.zeros(n)
+    for seed in range(T):
+        pick = O.sample(R, c, O.sample_keys(n, seed, 0, 1, 2, 3, 1))
+        subsets[tuple(pick.tolist())] += 1               # KeyError if anything outside R is drawn
+        incl[pick] += 1
+    exp = T / len(subsets)
+    chi2 = sum((v - exp) ** 2 / exp for v in subsets.values())
+    assert len(subsets) == 56 and chi2 < 105.0            # 55 dof: P(chi2 > 105) ~ 5e-5
+    assert np.abs(incl[R] / T - c / len(R)).max() < 0.012
