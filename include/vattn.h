@@ -1,0 +1,150 @@
+/*
+ * libvattn — verified sparse-attention decode step (vAttention, arXiv 2510.05688) for sm_100a.
+ *
+ * C ABI.  All tensor arguments are DEVICE pointers unless a comment says "host".  The caller owns
+ * every tensor and the workspace; the library never allocates or frees device memory and
+ * vattn_decode / vattn_dense_decode never synchronise (they only enqueue work on `stream`).
+ * A plan holds host-side descriptors only.  One plan must not be used from two streams at once
+ * (its workspace is shared state).
+ *
+ * Tensor layouts
+ *   q, out        [batch, num_q_heads, head_dim], contiguous, 16-byte aligned, element type `dtype`
+ *   k_cache,
+ *   v_cache       paged: element (block p, kv head g, token t, dim j) at
+ *                 p*kv_stride_block + g*kv_stride_head + t*kv_stride_token + j   (element units);
+ *                 default "HND" = [num_blocks, num_kv_heads, block_size, head_dim] contiguous.
+ *                 Rows must be 16-byte aligned (strides multiples of 8 bf16 / 4 fp32 elements).
+ *   block_table   int32 [batch, max_blocks_per_seq]: logical page -> physical page
+ *   seq_lens      int32 [batch]: tokens n_b currently in each sequence (0 <= n_b <= max_seq_len)
+ * Query head h reads KV head h / (num_q_heads / num_kv_heads); every query head has its own
+ * index sets, budget and sample (the paper states its guarantee per attention head: Fig. 3 caption).
+ *
+ * Return codes: 0 OK; negative = error, nothing was enqueued.
+ */
+#ifndef VATTN_H_
+#define VATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VATTN_OK               0
+#define VATTN_ERR_INVALID_ARG -1   /* null / misaligned pointer, eps or delta outside (0,1), negative sink/window/k, Hq % Hkv != 0 */
+#define VATTN_ERR_UNSUPPORTED -2   /* head_dim not in {64,128}, block_size != 16, unknown dtype, GQA ratio > 64 */
+#define VATTN_ERR_WORKSPACE   -3   /* workspace missing, misaligned or too small */
+#define VATTN_ERR_CUDA        -4   /* a CUDA runtime call or kernel launch failed */
+
+#define VATTN_DTYPE_FP32 0
+#define VATTN_DTYPE_BF16 1
+
+/* bits of the device status word (vattn_last_status) */
+#define VATTN_STATUS_BAD_BLOCK      1u   /* a block_table entry was outside [0, num_blocks): page treated as page 0 */
+#define VATTN_STATUS_BAD_SEQLEN     2u   /* a seq_len was outside [0, max_seq_len]: clamped */
+#define VATTN_STATUS_BAND_OVERFLOW  4u   /* more near-tie top-k candidates than the fast list holds: exact slow path ran */
+#define VATTN_STATUS_NONFINITE      8u   /* a budget statistic was not finite: that head used the whole residual */
+
+typedef struct vattn_plan vattn_plan;    /* opaque; host memory */
+
+typedef struct {
+  int32_t batch, num_q_heads, num_kv_heads, head_dim;     /* head_dim in {64,128}; num_q_heads % num_kv_heads == 0 */
+  int32_t block_size;                                     /* tokens per page: 16 */
+  int32_t max_blocks_per_seq, num_blocks, max_seq_len;    /* max_seq_len <= max_blocks_per_seq * block_size */
+  int32_t dtype;                                          /* VATTN_DTYPE_*: element type of q, k_cache, v_cache, out */
+  int64_t kv_stride_block, kv_stride_head, kv_stride_token; /* elements; all zero = contiguous HND */
+} vattn_shape;
+
+/* Everything Algorithm 1/2 need beyond the short argument list of vattn_decode.  Zero = default. */
+typedef struct {
+  float   base_rate;       /* f_b: fraction of the residual n_s drawn as the base sample (Sec. 4.2, last paragraph);
+                              default 0.025.  b0 = min(n_s, max(2, floor(f_b * n_s))) */
+  float   topk_frac;       /* f_t: if > 0, k_b = floor(topk_frac * n_b) replaces the scalar k (Algorithm 1 line 3) */
+  float   scale;           /* softmax scale applied to <K[i], q>; default 1/sqrt(head_dim) rounded to fp32 */
+  int32_t mode;            /* which computation is kept verified (Algorithm 2): 0 SDPA (Theorem 4.3),
+                              1 denominator only, 2 numerator only (Corollaries D.2) */
+  int32_t layer, step;     /* Philox counter words; step < 2^31.  A step is a pure function of
+                              (seed, layer, batch row, head, step): nothing is carried between calls */
+  int32_t rng_head_is_kv;  /* 0: sampling keys per query head; 1: per KV head (the heads of a group share keys) */
+  int32_t force_budget;    /* < 0 (or 0 with force_budget_on == 0): off; else b = min(force_budget, n_s) */
+  int32_t force_budget_on; /* set to 1 to apply force_budget (so that a forced budget of 0 is expressible) */
+} vattn_params;
+
+/* Optional per-call introspection.  All DEVICE pointers; NULL = not wanted.  cap = max_seq_len. */
+typedef struct {
+  int32_t *topk_idx, *topk_cnt;   /* [B,Hq,cap], [B,Hq]  I_t ascending (I_f = sink range + I_t + window range) */
+  int32_t *base_idx, *base_cnt;   /* I_bs ascending, b0 */
+  int32_t *dyn_idx,  *dyn_cnt;    /* I_dyn ascending, b */
+  int32_t *budgets;               /* [B,Hq,4] ceil(b_D), ceil(b_N), ceil(b_SDPA) (saturating at 2^31-1), b */
+  double  *stats;                 /* [B,Hq,8] D_f, sigma^2, Tr(Sigma), D_hat, |N_hat|_2, n_s, b0, m (weights are
+                                     exp(s - m) with m the head's largest fp32 score) */
+  float   *scores;                /* [B,Hq,cap] fp32 scores s_i = scale * <K[i], q> */
+} vattn_debug;
+
+/* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG, UNSUPPORTED. */
+int    vattn_plan_create(const vattn_shape* shape, vattn_plan** out);
+void   vattn_plan_destroy(vattn_plan* plan);
+
+/* Bytes of device scratch a plan needs (a pure function of the shape), and handing it over.
+ * The pointer must be 256-byte aligned and stay valid while the plan is used.  The library
+ * zeroes what it needs on every call; the contents need not be initialised. */
+size_t vattn_workspace_bytes(const vattn_plan* plan);
+int    vattn_set_workspace(vattn_plan* plan, void* dev_ptr, size_t bytes);
+
+/* Copy parameters / debug pointers into the plan (host structs; NULL resets to defaults). */
+int    vattn_set_params(vattn_plan* plan, const vattn_params* params);
+int    vattn_set_debug(vattn_plan* plan, const vattn_debug* debug);
+
+/*
+ * One verified sparse-attention decode step (Algorithm 1 with budget_X of Algorithm 2), for every
+ * (batch row, query head):
+ *   I_f  = first `sink` tokens + last `window` tokens + the k middle tokens with the largest
+ *          scale*<K[i],q> (ties to the lowest index);            n_s = n - |I_f|
+ *   I_bs = b0 residual tokens, uniform without replacement (Philox stream 0)
+ *   b    = clamp(ceil(b_X(eps, delta; base-sample statistics)), b0, n_s)
+ *   I_dyn= b residual tokens, uniform without replacement (Philox stream 1)
+ *   out  = (N_f + n_s/b * sum_{I_dyn} w_i V[i]) / (D_f + n_s/b * sum_{I_dyn} w_i),  w_i = exp(s_i - m)
+ * (Sec. 4.1 numerator/denominator equations; SDPA_{S,p} of Sec. 3).  A uniform sample is "the c
+ * residual tokens with the smallest (key_i, i)", key_i = Philox4x32-10(key = seed,
+ * counter = (i>>2, batch<<16 | head, layer, step<<1 | stream))[i & 3].
+ * Degenerate inputs: n = 0 -> out row = 0; sink+window >= n -> exact attention, budget 0;
+ * k larger than the middle range is clipped.
+ * eps, delta in (0,1).  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                 const int32_t* block_table, const int32_t* seq_lens,
+                 int sink, int window, int k, float eps, float delta, uint64_t seed,
+                 void* out, void* stream /* cudaStream_t */);
+
+/* Dense attention over the same paged cache (full SDPA of Sec. 3), split over the context with a
+ * fixed-order merge: the latency the sparse step is compared with.  Uses the plan's workspace. */
+int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
+
+/* Same step as vattn_decode with HOST buffers for q, block_table, seq_lens and out (the caches stay on
+ * the device): copies the inputs in, runs the step, copies `out` back and waits for it.  `staging` is a
+ * caller-owned device buffer of at least vattn_host_staging_bytes(plan) bytes. */
+size_t vattn_host_staging_bytes(const vattn_plan* plan);
+int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table_host, const int32_t* seq_lens_host,
+                      int sink, int window, int k, float eps, float delta, uint64_t seed,
+                      void* out_host, void* staging, void* stream);
+
+/* OR of the status bits raised since the last call of this function on this plan.  Synchronises
+ * `stream`; not for the hot path.  Errors: INVALID_ARG, WORKSPACE, CUDA. */
+int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */);
+
+/* Number of kernels the last vattn_decode / vattn_dense_decode call on this plan enqueued. */
+int vattn_last_launch_count(const vattn_plan* plan);
+
+const char* vattn_strerror(int code);
+
+/* z(x) = Phi^{-1}(1 - x/2), the two-sided standard-normal quantile of Lemma 4.1, as the library
+ * evaluates it on the host (fp64) for the budget formulas.  0 < x < 2; NaN otherwise. */
+double vattn_normal_quantile(double x);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VATTN_H_ */

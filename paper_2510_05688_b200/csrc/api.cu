@@ -1,0 +1,311 @@
+// C ABI of libvattn: plan objects, argument checks, workspace layout and the launch sequence of one
+// decode step.  Host code only; no device memory is allocated or freed here.
+#include <math.h>
+#include <new>
+#include <string.h>
+#include "vattn_internal.cuh"
+
+struct vattn_plan {
+  vattn_shape shape;
+  vattn_params params;
+  vattn_debug dbg;
+  void* ws;
+  size_t ws_bytes;
+  bool status_ready;
+  int last_launches;
+  // derived
+  int G, npad, nwords, stat_splits, gat_splits, dense_splits;
+  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
+      off_det, off_gat, off_dense, total;
+};
+
+namespace {
+
+constexpr int kNumSM = 148;          // B200; the library is built for sm_100a only
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Upper-tail standard-normal quantile: the z with P(Z > z) = t, 0 < t < 1.  The Lemma's
+// Phi^{-1}(1 - delta/2) is upper_quantile(delta/2).  Rational first guess (Abramowitz & Stegun 26.2.23),
+// then Newton steps on erfc, which converge to the last bit or two of a double.
+double upper_quantile(double t) {
+  if (!(t > 0.0) || !(t < 1.0)) return NAN;
+  const bool flip = t > 0.5;
+  const double pp = flip ? 1.0 - t : t;
+  const double u = sqrt(-2.0 * log(pp));
+  double z = u - (2.515517 + u * (0.802853 + u * 0.010328)) / (1.0 + u * (1.432788 + u * (0.189269 + u * 0.001308)));
+  for (int it = 0; it < 8; ++it) {
+    const double f = 0.5 * erfc(z * M_SQRT1_2) - pp;
+    const double pdf = exp(-0.5 * z * z) * 0.3989422804014326779;
+    const double step = f / pdf;
+    z += step;
+    if (fabs(step) <= 1e-16 * fabs(z)) break;
+  }
+  return flip ? -z : z;
+}
+
+void derive(vattn_plan* pl) {
+  const vattn_shape& s = pl->shape;
+  pl->G = s.num_q_heads / s.num_kv_heads;
+  pl->npad = (s.max_seq_len + 31) / 32 * 32;
+  if (pl->npad == 0) pl->npad = 32;
+  pl->nwords = pl->npad / 32;
+  const int heads = s.batch * s.num_q_heads;
+  int sp = (4 * kNumSM + heads - 1) / heads;
+  pl->stat_splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
+  pl->gat_splits = pl->stat_splits;
+  const int GC = (pl->G + 3) / 4;
+  const int groups = s.batch * s.num_kv_heads * GC;
+  sp = (4 * kNumSM + groups - 1) / groups;
+  pl->dense_splits = sp < 1 ? 1 : (sp > 128 ? 128 : sp);
+  const size_t BH = (size_t)heads, D = (size_t)s.head_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  pl->off_scores = take(BH * pl->npad * sizeof(float));
+  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH) * sizeof(unsigned);
+  pl->off_zero = take(pl->zero_bytes);
+  pl->off_status = take(sizeof(unsigned));
+  pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
+  pl->off_topk = take(BH * pl->npad * sizeof(int));
+  pl->off_base = take(BH * pl->npad * sizeof(int));
+  pl->off_dyn = take(BH * pl->npad * sizeof(int));
+  pl->off_meta = take(BH * sizeof(HeadMeta));
+  pl->off_stat = take(BH * pl->stat_splits * (2 * D + 4) * sizeof(double));
+  pl->off_det = take(BH * (D + 1) * sizeof(double));
+  pl->off_gat = take(BH * pl->gat_splits * (D + 1) * sizeof(float));
+  pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
+  pl->total = off;
+}
+
+int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, const void* vc, const int32_t* bt,
+              const int32_t* sl, void* out) {
+  const vattn_shape& s = pl->shape;
+  const vattn_params& pr = pl->params;
+  memset(&p, 0, sizeof(p));
+  p.B = s.batch; p.Hq = s.num_q_heads; p.Hkv = s.num_kv_heads; p.G = pl->G; p.D = s.head_dim; p.dtype = s.dtype;
+  p.max_blocks = s.max_blocks_per_seq; p.num_blocks = s.num_blocks; p.max_seq_len = s.max_seq_len;
+  p.npad = pl->npad; p.nwords = pl->nwords;
+  if (s.kv_stride_block == 0 && s.kv_stride_head == 0 && s.kv_stride_token == 0) {
+    p.st = s.head_dim; p.sh = (long long)s.block_size * s.head_dim; p.sb = (long long)s.num_kv_heads * p.sh;
+  } else {
+    p.sb = s.kv_stride_block; p.sh = s.kv_stride_head; p.st = s.kv_stride_token;
+  }
+  p.q = q; p.kc = kc; p.vc = vc; p.bt = bt; p.seq_lens = sl; p.out = out;
+  p.topk_frac = pr.topk_frac;
+  p.base_rate = pr.base_rate > 0.f ? pr.base_rate : 0.025f;
+  p.scale = pr.scale != 0.f ? pr.scale : (float)(1.0 / sqrt((double)s.head_dim));
+  p.mode = pr.mode; p.layer = pr.layer; p.step = pr.step; p.rng_head_is_kv = pr.rng_head_is_kv;
+  p.force_budget = (pr.force_budget_on || pr.force_budget > 0) ? (pr.force_budget < 0 ? -1 : pr.force_budget) : -1;
+  unsigned char* w = static_cast<unsigned char*>(pl->ws);
+  p.scores = reinterpret_cast<float*>(w + pl->off_scores);
+  unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
+  const size_t BH = (size_t)s.batch * s.num_q_heads;
+  p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
+  p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
+  p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);
+  p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
+  p.base_idx = reinterpret_cast<int*>(w + pl->off_base);
+  p.dyn_idx = reinterpret_cast<int*>(w + pl->off_dyn);
+  p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
+  p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);
+  p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
+  p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
+  p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
+  p.stat_splits = pl->stat_splits; p.gat_splits = pl->gat_splits; p.dense_splits = pl->dense_splits;
+  p.dbg = pl->dbg;
+  return VATTN_OK;
+}
+
+inline bool misaligned(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) & (a - 1)) != 0; }
+
+int check_common(const vattn_plan* pl, const void* q, const void* kc, const void* vc, const int32_t* bt,
+                 const int32_t* sl, const void* out) {
+  if (!pl || !q || !kc || !vc || !bt || !sl || !out) return VATTN_ERR_INVALID_ARG;
+  if (misaligned(q, 16) || misaligned(kc, 16) || misaligned(vc, 16) || misaligned(out, 16) || misaligned(bt, 4) ||
+      misaligned(sl, 4))
+    return VATTN_ERR_INVALID_ARG;
+  if (!pl->ws || pl->ws_bytes < pl->total) return VATTN_ERR_WORKSPACE;
+  return VATTN_OK;
+}
+
+#define CU(x) do { if ((x) != cudaSuccess) return VATTN_ERR_CUDA; } while (0)
+
+int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st) {
+  if (!pl->status_ready) {
+    CU(cudaMemsetAsync(p.status, 0, sizeof(unsigned), st));
+    pl->status_ready = true;
+  }
+  CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
+  return VATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+double vattn_normal_quantile(double x) { return upper_quantile(0.5 * x); }
+
+int vattn_plan_create(const vattn_shape* shape, vattn_plan** out) {
+  if (!shape || !out) return VATTN_ERR_INVALID_ARG;
+  const vattn_shape& s = *shape;
+  if (s.batch <= 0 || s.num_q_heads <= 0 || s.num_kv_heads <= 0 || s.max_blocks_per_seq <= 0 || s.num_blocks <= 0 ||
+      s.max_seq_len < 0)
+    return VATTN_ERR_INVALID_ARG;
+  if (s.num_q_heads % s.num_kv_heads != 0) return VATTN_ERR_INVALID_ARG;
+  if (s.batch > 65535 || s.num_q_heads > 65535) return VATTN_ERR_INVALID_ARG;
+  if (s.head_dim != 64 && s.head_dim != 128) return VATTN_ERR_UNSUPPORTED;
+  if (s.block_size != VATTN_BLOCK) return VATTN_ERR_UNSUPPORTED;
+  if (s.dtype != VATTN_DTYPE_FP32 && s.dtype != VATTN_DTYPE_BF16) return VATTN_ERR_UNSUPPORTED;
+  if (s.num_q_heads / s.num_kv_heads > 64) return VATTN_ERR_UNSUPPORTED;
+  if (s.max_seq_len > VATTN_MAX_SEQ) return VATTN_ERR_UNSUPPORTED;
+  if ((long long)s.max_seq_len > (long long)s.max_blocks_per_seq * s.block_size) return VATTN_ERR_INVALID_ARG;
+  const bool custom = s.kv_stride_block || s.kv_stride_head || s.kv_stride_token;
+  if (custom) {
+    const int epl = s.dtype == VATTN_DTYPE_BF16 ? 8 : 4;
+    if (s.kv_stride_block <= 0 || s.kv_stride_head <= 0 || s.kv_stride_token < s.head_dim) return VATTN_ERR_INVALID_ARG;
+    if (s.kv_stride_block % epl || s.kv_stride_head % epl || s.kv_stride_token % epl) return VATTN_ERR_INVALID_ARG;
+  }
+  vattn_plan* pl = new (std::nothrow) vattn_plan();
+  if (!pl) return VATTN_ERR_INVALID_ARG;
+  memset(pl, 0, sizeof(*pl));
+  pl->shape = s;
+  pl->params.force_budget = -1;
+  derive(pl);
+  *out = pl;
+  return VATTN_OK;
+}
+
+void vattn_plan_destroy(vattn_plan* plan) { delete plan; }
+
+size_t vattn_workspace_bytes(const vattn_plan* plan) { return plan ? plan->total : 0; }
+
+int vattn_set_workspace(vattn_plan* plan, void* dev_ptr, size_t bytes) {
+  if (!plan) return VATTN_ERR_INVALID_ARG;
+  if (!dev_ptr || misaligned(dev_ptr, 256) || bytes < plan->total) return VATTN_ERR_WORKSPACE;
+  plan->ws = dev_ptr;
+  plan->ws_bytes = bytes;
+  plan->status_ready = false;
+  return VATTN_OK;
+}
+
+int vattn_set_params(vattn_plan* plan, const vattn_params* params) {
+  if (!plan) return VATTN_ERR_INVALID_ARG;
+  if (!params) { memset(&plan->params, 0, sizeof(plan->params)); plan->params.force_budget = -1; return VATTN_OK; }
+  const vattn_params& p = *params;
+  if (p.base_rate < 0.f || p.base_rate > 1.f || p.topk_frac < 0.f || p.topk_frac > 1.f) return VATTN_ERR_INVALID_ARG;
+  if (p.mode < 0 || p.mode > 2 || p.step < 0 || !(p.scale == p.scale) || isinf(p.scale)) return VATTN_ERR_INVALID_ARG;
+  plan->params = p;
+  return VATTN_OK;
+}
+
+int vattn_set_debug(vattn_plan* plan, const vattn_debug* debug) {
+  if (!plan) return VATTN_ERR_INVALID_ARG;
+  if (debug) plan->dbg = *debug; else memset(&plan->dbg, 0, sizeof(plan->dbg));
+  return VATTN_OK;
+}
+
+int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                 const int32_t* block_table, const int32_t* seq_lens, int sink, int window, int k, float eps,
+                 float delta, uint64_t seed, void* out, void* stream) {
+  int rc = check_common(plan, q, k_cache, v_cache, block_table, seq_lens, out);
+  if (rc != VATTN_OK) return rc;
+  if (!(eps > 0.f && eps < 1.f) || !(delta > 0.f && delta < 1.f) || sink < 0 || window < 0 || k < 0)
+    return VATTN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Prob p;
+  fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
+  p.sink = sink; p.window = window; p.k = k;
+  p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
+  p.eps = (double)eps; p.delta = (double)delta;
+  p.z_delta = upper_quantile(0.5 * p.delta);
+  for (int j = 1; j <= 15; ++j) {
+    p.z1[j - 1] = upper_quantile(0.5 * (p.delta * j / 16.0));
+    p.z2[j - 1] = upper_quantile(0.5 * (p.delta * (16 - j) / 16.0));
+  }
+  plan->last_launches = 0;
+  rc = prepare_stream(plan, p, st);
+  if (rc != VATTN_OK) return rc;
+  CU(launch_score(p, st));            plan->last_launches++;
+  if (p.dbg.scores)
+    CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
+                         sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
+  CU(launch_select_topk_base(p, st)); plan->last_launches++;
+  CU(launch_stats(p, st));            plan->last_launches++;
+  CU(launch_select_final(p, st));     plan->last_launches++;
+  CU(launch_gather(p, st));           plan->last_launches++;
+  return VATTN_OK;
+}
+
+int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                       const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+  int rc = check_common(plan, q, k_cache, v_cache, block_table, seq_lens, out);
+  if (rc != VATTN_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Prob p;
+  fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
+  plan->last_launches = 0;
+  rc = prepare_stream(plan, p, st);
+  if (rc != VATTN_OK) return rc;
+  int launches = 0;
+  CU(launch_dense(p, st, &launches));
+  plan->last_launches = launches;
+  return VATTN_OK;
+}
+
+size_t vattn_host_staging_bytes(const vattn_plan* plan) {
+  if (!plan) return 0;
+  const vattn_shape& s = plan->shape;
+  const size_t es = s.dtype == VATTN_DTYPE_BF16 ? 2 : 4;
+  const size_t qb = align_up((size_t)s.batch * s.num_q_heads * s.head_dim * es, 256);
+  return 2 * qb + align_up((size_t)s.batch * s.max_blocks_per_seq * 4, 256) + align_up((size_t)s.batch * 4, 256);
+}
+
+int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table_host, const int32_t* seq_lens_host, int sink, int window, int k,
+                      float eps, float delta, uint64_t seed, void* out_host, void* staging, void* stream) {
+  if (!plan || !q_host || !block_table_host || !seq_lens_host || !out_host || !staging || misaligned(staging, 256))
+    return VATTN_ERR_INVALID_ARG;
+  const vattn_shape& s = plan->shape;
+  const size_t es = s.dtype == VATTN_DTYPE_BF16 ? 2 : 4;
+  const size_t qbytes = (size_t)s.batch * s.num_q_heads * s.head_dim * es, qb = align_up(qbytes, 256);
+  const size_t btbytes = (size_t)s.batch * s.max_blocks_per_seq * 4, slbytes = (size_t)s.batch * 4;
+  unsigned char* d = static_cast<unsigned char*>(staging);
+  void* dq = d; void* dout = d + qb; int32_t* dbt = reinterpret_cast<int32_t*>(d + 2 * qb);
+  int32_t* dsl = reinterpret_cast<int32_t*>(d + 2 * qb + align_up(btbytes, 256));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CU(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(dbt, block_table_host, btbytes, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(dsl, seq_lens_host, slbytes, cudaMemcpyHostToDevice, st));
+  int rc = vattn_decode(plan, dq, k_cache, v_cache, dbt, dsl, sink, window, k, eps, delta, seed, dout, stream);
+  if (rc != VATTN_OK) return rc;
+  CU(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return VATTN_OK;
+}
+
+int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits) {
+  if (!plan || !bits) return VATTN_ERR_INVALID_ARG;
+  if (!plan->ws) return VATTN_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned* dev = reinterpret_cast<unsigned*>(static_cast<unsigned char*>(plan->ws) + plan->off_status);
+  if (!plan->status_ready) { *bits = 0; return VATTN_OK; }
+  CU(cudaMemcpyAsync(bits, dev, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemsetAsync(dev, 0, sizeof(unsigned), st));
+  CU(cudaStreamSynchronize(st));
+  return VATTN_OK;
+}
+
+int vattn_last_launch_count(const vattn_plan* plan) { return plan ? plan->last_launches : 0; }
+
+const char* vattn_strerror(int code) {
+  switch (code) {
+    case VATTN_OK: return "ok";
+    case VATTN_ERR_INVALID_ARG: return "invalid argument";
+    case VATTN_ERR_UNSUPPORTED: return "unsupported shape or element type";
+    case VATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case VATTN_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

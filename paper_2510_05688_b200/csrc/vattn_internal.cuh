@@ -1,0 +1,147 @@
+// Internal declarations shared by the kernels of libvattn (sm_100a).  Not part of the ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "vattn.h"
+
+#define VATTN_BLOCK 16                 // tokens per KV page
+#define VATTN_MAX_SEQ (1 << 18)        // longest sequence the select kernels' shared-memory bitmaps hold
+#define VATTN_KEYCACHE_MAX 49152       // tokens whose 32-bit select keys are cached in shared memory
+#define VATTN_BANDCAP 1024             // near-tie top-k candidates rescored by the fast path
+#define SEL_THREADS 1024
+#define ROW_THREADS 256
+
+// Per (batch row, query head) bookkeeping, written by the select kernel and completed by the
+// statistics kernel.
+struct HeadMeta {
+  int n;         // tokens in the sequence (clamped to [0, max_seq_len])
+  int s0;        // |I_s| = min(sink, n)
+  int l_start;   // first token of the local window; middle range M = [s0, l_start)
+  int kk;        // |I_t| = min(k, |M|)
+  int n_s;       // residual size |M| - kk
+  int b0;        // base-sample size
+  int b;         // final budget |I_dyn|
+  int pad0;
+  float m;       // largest fp32 score of the head (softmax stabiliser)
+  float gamma;   // bound on |fp32 score - exact score| for this head
+  int pad1, pad2;
+};
+
+// Everything a kernel needs, passed by value.
+struct Prob {
+  int B, Hq, Hkv, G, D, dtype;
+  int max_blocks, num_blocks, max_seq_len, npad, nwords;   // npad: max_seq_len rounded up to 32; nwords = npad/32
+  long long sb, sh, st;                                      // KV strides in elements
+  const void* q; const void* kc; const void* vc; const int* bt; const int* seq_lens; void* out;
+  int sink, window, k;
+  float topk_frac, base_rate, scale;
+  int mode, layer, step, rng_head_is_kv, force_budget;       // force_budget < 0: off
+  unsigned seed_lo, seed_hi;
+  double eps, delta, z_delta;
+  double z1[15], z2[15];                                     // z(delta*j/16), z(delta*(16-j)/16), j = 1..15
+  // workspace
+  float* scores;          // [B,Hq,npad]
+  unsigned* m_ord;        // [B,Hq]  order-preserving encoding of the running max score
+  unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
+  unsigned* tickets;      // [2,B,Hq] "last CTA done" counters (stats, gather)
+  unsigned* status;       // [1]
+  unsigned* bitmap;       // [B,Hq,nwords] membership of I_t
+  int* topk_idx;          // [B,Hq,npad]
+  int* base_idx;          // [B,Hq,npad]
+  int* dyn_idx;           // [B,Hq,npad]
+  HeadMeta* meta;         // [B,Hq]
+  double* stat_part;      // [B,Hq,stat_splits,2D+4]
+  double* det_sums;       // [B,Hq,D+1]  N_f then D_f
+  float* gat_part;        // [B,Hq,gat_splits,D+1]
+  float* dense_part;      // [B,Hq,dense_splits,D+2]
+  int stat_splits, gat_splits, dense_splits;
+  vattn_debug dbg;
+};
+
+// ---------------------------------------------------------------------------------------------
+// small device helpers
+__device__ __forceinline__ unsigned ord_f32(float f) {          // order-preserving float -> uint
+  unsigned u = __float_as_uint(f);
+  return u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float unord_f32(unsigned o) {
+  unsigned u = (o & 0x80000000u) ? (o ^ 0x80000000u) : ~o;
+  return __uint_as_float(u);
+}
+__device__ __forceinline__ unsigned long long ord_f64(double f) {
+  unsigned long long u = (unsigned long long)__double_as_longlong(f);
+  return u ^ ((u >> 63) ? 0xFFFFFFFFFFFFFFFFull : 0x8000000000000000ull);
+}
+
+struct bf16x8 { uint4 v; };
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int EPL = 4;                                  // elements per 16-byte load
+  __device__ static __forceinline__ void load(const float* p, float (&x)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  }
+  __device__ static __forceinline__ float to_float(float v) { return v; }
+  __device__ static __forceinline__ float from_float(float v) { return v; }
+};
+struct bf16_t { unsigned short bits; };
+template <> struct Elem<bf16_t> {
+  static constexpr int EPL = 8;
+  __device__ static __forceinline__ void load(const bf16_t* p, float (&x)[8]) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
+    x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
+  }
+  __device__ static __forceinline__ float to_float(bf16_t v) { return __uint_as_float(((unsigned)v.bits) << 16); }
+  __device__ static __forceinline__ bf16_t from_float(float f) {    // round to nearest even
+    unsigned u = __float_as_uint(f);
+    bf16_t r;
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) { r.bits = (unsigned short)((u >> 16) | 0x40); return r; }   // NaN
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    r.bits = (unsigned short)(u >> 16);
+    return r;
+  }
+};
+
+// physical page of logical page `lp` of batch row b (bounds-checked; a bad entry raises a status bit)
+__device__ __forceinline__ int page_of(const Prob& p, int b, int lp) {
+  int pg = p.bt[(long long)b * p.max_blocks + lp];
+  if ((unsigned)pg >= (unsigned)p.num_blocks) { atomicOr(p.status, VATTN_STATUS_BAD_BLOCK); pg = 0; }
+  return pg;
+}
+template <typename T>
+__device__ __forceinline__ const T* row_ptr(const Prob& p, const void* cache, int b, int g, int tok) {
+  int pg = page_of(p, b, tok >> 4);
+  return reinterpret_cast<const T*>(cache) + (long long)pg * p.sb + (long long)g * p.sh + (long long)(tok & 15) * p.st;
+}
+__device__ __forceinline__ int clamped_len(const Prob& p, int b) {
+  int n = p.seq_lens[b];
+  if (n < 0 || n > p.max_seq_len) { atomicOr(p.status, VATTN_STATUS_BAD_SEQLEN); n = n < 0 ? 0 : p.max_seq_len; }
+  return n;
+}
+
+// Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0,k1)
+__device__ __forceinline__ uint4 philox4x32_10(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
+                                               unsigned k0, unsigned k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    unsigned hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    unsigned hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    unsigned n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// launchers (one per translation unit)
+cudaError_t launch_score(const Prob& p, cudaStream_t s);
+cudaError_t launch_select_topk_base(const Prob& p, cudaStream_t s);
+cudaError_t launch_select_final(const Prob& p, cudaStream_t s);
+cudaError_t launch_stats(const Prob& p, cudaStream_t s);
+cudaError_t launch_gather(const Prob& p, cudaStream_t s);
+cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches);
+size_t select_smem_bytes(const Prob& p);

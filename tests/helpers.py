@@ -1,0 +1,92 @@
+"""Shared test helpers: run the CUDA path through the C ABI and compare it with the oracle."""
+import numpy as np
+
+from oracle import vattn_oracle as O
+
+BF16_TOL = 2e-2      # absolute-or-relative, bf16 outputs
+FP32_REL = 1e-5      # relative to the head's largest |output|, fp32 outputs
+
+
+def run_oracle(case, heads=None, **over):
+    p = dict(case.params)
+    p.update(over)
+    return O.vattn_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink,
+                          case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype, heads=heads, **p)
+
+
+def run_gpu(case, debug=True, plan=None, dev=None, **over):
+    """One vattn_decode call through the C ABI.  Returns (out as numpy, debug dict of numpy arrays, plan)."""
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    p = dict(case.params)
+    p.update(over)
+    if dev is None:
+        dev = vb.case_to_device(case)
+    if plan is None:
+        plan = vb.plan_for_case(case)
+    plan.set_params(**p)
+    dbg = plan.enable_debug() if debug else None
+    out = torch.empty_like(dev["q"])
+    plan.decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], case.sink, case.window,
+                case.k, case.eps, case.delta, case.seed, out)
+    torch.cuda.synchronize()
+    if case.dtype == "bf16":
+        out_np = out.view(torch.int16).cpu().numpy().view(np.uint16)
+    else:
+        out_np = out.cpu().numpy()
+    dbg_np = {k: v.cpu().numpy() for k, v in dbg.items()} if dbg else None
+    return out_np, dbg_np, plan
+
+
+def out_values(case, out):
+    if case.dtype == "bf16":
+        return (np.asarray(out, np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return np.asarray(out, np.float64)
+
+
+def assert_out_close(case, got, want, where=""):
+    g, w = out_values(case, got), out_values(case, want)
+    if case.dtype == "bf16":
+        bad = np.abs(g - w) > BF16_TOL * np.maximum(1.0, np.abs(w))
+        assert not bad.any(), f"{where}: bf16 output off by {np.abs(g - w).max():.3e}"
+    else:
+        ref = np.abs(w).max(axis=-1, keepdims=True)
+        err = np.abs(g - w) / np.maximum(ref, 1e-30)
+        assert err.max() <= FP32_REL, f"{where}: fp32 output rel err {err.max():.3e}"
+
+
+def assert_parity(case, out, dbg, det, out_ref, check_scores=True):
+    """Bit-exact index sets, budgets and samples; outputs within tolerance, for every head in `det`."""
+    for (b, h), r in det.items():
+        tag = f"{case.name} b={b} h={h}"
+        n = r["n"]
+        if n == 0:
+            assert dbg["topk_cnt"][b, h] == 0 and dbg["dyn_cnt"][b, h] == 0, tag
+            continue
+        kk = int(dbg["topk_cnt"][b, h])
+        assert kk == len(r["I_t"]), f"{tag}: |I_t| {kk} vs {len(r['I_t'])}"
+        assert np.array_equal(dbg["topk_idx"][b, h, :kk], r["I_t"]), f"{tag}: I_t differs"
+        b0 = int(dbg["base_cnt"][b, h])
+        assert b0 == r["b0"], f"{tag}: b0 {b0} vs {r['b0']}"
+        assert np.array_equal(dbg["base_idx"][b, h, :b0], r["I_bs"]), f"{tag}: I_bs differs"
+        assert tuple(int(x) for x in dbg["budgets"][b, h]) == tuple(r["budgets"]), \
+            f"{tag}: budgets {dbg['budgets'][b, h]} vs {r['budgets']}"
+        bb = int(dbg["dyn_cnt"][b, h])
+        assert bb == r["b"], tag
+        assert np.array_equal(dbg["dyn_idx"][b, h, :bb], r["I_dyn"]), f"{tag}: I_dyn differs"
+        st, sr = dbg["stats"][b, h], r["stats"]
+        assert st[5] == sr[5] and st[6] == sr[6], tag
+        np.testing.assert_allclose(st[7], sr[7], rtol=0, atol=1e-4, err_msg=tag)
+        # weights are relative to each side's own m: compare the m-free ratios
+        sc = np.exp(sr[7] - st[7])
+        np.testing.assert_allclose(st[0] * 1.0, sr[0] * sc, rtol=1e-9, err_msg=tag + " D_f")
+        np.testing.assert_allclose(st[3], sr[3] * sc, rtol=1e-9, err_msg=tag + " D_hat")
+        np.testing.assert_allclose(st[4], sr[4] * sc, rtol=1e-9, atol=1e-300, err_msg=tag + " N_hat")
+        np.testing.assert_allclose(st[1], sr[1] * sc * sc, rtol=1e-7, atol=1e-30, err_msg=tag + " sigma2")
+        np.testing.assert_allclose(st[2], sr[2] * sc * sc, rtol=1e-7, atol=1e-30, err_msg=tag + " trace")
+        if check_scores:
+            s32 = dbg["scores"][b, h, :n].astype(np.float64)
+            assert np.abs(s32 - r["scores"]).max() <= 2e-5 * max(1.0, np.abs(r["scores"]).max()), tag + " scores"
+    idx = sorted(det.keys())
+    bs = np.array([i[0] for i in idx]); hs = np.array([i[1] for i in idx])
+    assert_out_close(case, np.asarray(out)[bs, hs], np.asarray(out_ref)[bs, hs], case.name)

@@ -1,0 +1,198 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Index sets (I_t, I_bs, I_dyn), budgets and counts must be bit-exact; outputs within 1e-5 relative
+(fp32) / 2e-2 absolute-or-relative (bf16).  Small cases span several tiles and ragged tails; the
+five workload configurations run at full size.
+"""
+import numpy as np
+import pytest
+
+from oracle import vattn_oracle as O
+from paper_2510_05688_b200 import synth
+from helpers import assert_out_close, assert_parity, out_values, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def small(dtype, seq_lens, Hq=8, Hkv=2, d=128, **kw):
+    args = dict(dtype=dtype, B=len(seq_lens), Hq=Hq, Hkv=Hkv, d=d, seq_lens=list(seq_lens), sink=4, window=8, k=16,
+                eps=0.05, delta=0.05, seed=1234, gen_seed=42, key_std=1.0, rho_v=1.0,
+                heavy=dict(R=12, c1=5.0, alpha=(0.75, 1.25)), params=dict(base_rate=0.05))
+    args.update(kw)
+    return synth.make_case("small", **args)
+
+
+def check(case, **over):
+    out_ref, det = run_oracle(case, **over)
+    out, dbg, plan = run_gpu(case, **over)
+    assert_parity(case, out, dbg, det, out_ref)
+    return out, dbg, det, plan
+
+
+# ----------------------------------------------------------------------------- small shapes, ragged tails
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("fp32", 64), ("fp32", 128)])
+def test_small_ragged_batches(dtype, d):
+    case = small(dtype, [1, 15, 16, 17, 255, 600, 1000, 2049, 33], d=d)
+    check(case)
+    check(case, mode=1)
+    check(case, mode=2)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 1), (6, 2), (10, 2)])
+def test_gqa_ratios(Hq, Hkv):
+    # G = 1, 8 (two head chunks), 3 and 5 (partial head chunks)
+    check(small("bf16", [700, 129], Hq=Hq, Hkv=Hkv))
+
+
+def test_empty_and_covered_sequences():
+    case = small("bf16", [0, 5, 12, 300, 0], sink=4, window=8, k=3)
+    out, dbg, det, _ = check(case)
+    assert (out_values(case, out)[0] == 0).all() and (out_values(case, out)[4] == 0).all()
+    # sink + window >= n: exact attention, budget 0
+    for h in range(case.num_q_heads):
+        assert det[(1, h)]["n_s"] == 0 and dbg["dyn_cnt"][1, h] == 0
+    dense = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=case.dtype)
+    assert np.abs(out_values(case, out)[1:3] - dense[1:3]).max() < 2e-2
+
+
+def test_k_zero_and_k_larger_than_middle():
+    check(small("fp32", [400, 77], d=64, k=0))
+    check(small("fp32", [400, 77], d=64, k=100000))
+    check(small("bf16", [400, 77], sink=0, window=0, k=7))
+
+
+def test_topk_fraction_and_kv_head_rng():
+    check(small("bf16", [900, 350], k=0, params=dict(base_rate=0.05, topk_frac=0.03)))
+    check(small("bf16", [900, 350], params=dict(base_rate=0.1, rng_head_is_kv=1, layer=3, step=77)))
+
+
+def test_full_residual_budget_equals_dense_attention():
+    case = small("fp32", [513, 64], d=64)
+    out, dbg, det, _ = check(case, force_budget=10**9)
+    dense = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=case.dtype)
+    ref = np.abs(dense).max(axis=-1, keepdims=True)
+    assert (np.abs(out_values(case, out) - dense) / ref).max() < 1e-5
+    check(case, force_budget=0)
+    check(case, force_budget=37)
+
+
+def test_explicit_scale():
+    check(small("bf16", [300], params=dict(base_rate=0.05, scale=0.2)))
+
+
+def test_identical_keys_take_the_exact_tie_path():
+    # every key row identical: all scores tie, the near-tie band is the whole middle range
+    case = small("bf16", [3000], Hq=4, Hkv=2, heavy=None, k=40)
+    kc = case.k_cache.copy()
+    kc[...] = kc[case.block_table[0, 0], :, 0][None, :, None, :]
+    case.k_cache = kc
+    out, dbg, det, plan = check(case)
+    for h in range(4):
+        assert dbg["topk_idx"][0, h, :40].tolist() == list(range(4, 44))      # lowest indices win ties
+        assert dbg["stats"][0, h, 1] == 0.0                                     # sigma^2 exactly 0
+    assert plan.last_status() & 4                                               # band overflow was reported
+
+
+def test_zero_query_and_duplicated_rows():
+    case = small("bf16", [500], Hq=4, Hkv=2, heavy=None)
+    q = case.q.copy()
+    q[0, 1] = 0                                                                 # bf16 bit pattern of 0
+    case.q = q
+    kc = case.k_cache.copy()
+    pg = case.block_table[0]
+    kc[pg[3], :, 5] = kc[pg[9], :, 2]                                           # two identical rows (tokens 53, 146)
+    case.k_cache = kc
+    check(case)
+
+
+def test_bad_block_table_entry_sets_status_without_faulting():
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [200])
+    dev = vb.case_to_device(case)
+    dev["block_table"][0, 2] = case.num_blocks + 5
+    plan = vb.plan_for_case(case)
+    out = torch.empty_like(dev["q"])
+    plan.decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], 4, 8, 16, 0.05, 0.05,
+                1, out)
+    torch.cuda.synchronize()
+    assert plan.last_status() & vb.STATUS_BAD_BLOCK
+    assert plan.last_status() == 0                                              # reading clears the word
+
+
+def test_two_calls_are_bitwise_reproducible():
+    case = small("bf16", [2049, 700])
+    out1, dbg1, plan = run_gpu(case)
+    out2, dbg2, _ = run_gpu(case, plan=plan)
+    assert np.array_equal(out1, out2)
+    assert np.array_equal(dbg1["dyn_idx"], dbg2["dyn_idx"])
+
+
+def test_dense_kernel_matches_dense_sdpa():
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    for dtype, d in (("bf16", 128), ("fp32", 64), ("bf16", 64), ("fp32", 128)):
+        case = small(dtype, [1, 17, 0, 1000, 2049], d=d)
+        dev = vb.case_to_device(case)
+        plan = vb.plan_for_case(case)
+        out = torch.empty_like(dev["q"])
+        plan.dense_decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], out)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy().astype(np.float64)
+        ref = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=dtype)
+        tol = 2e-2 if dtype == "bf16" else 2e-5
+        assert (np.abs(got - ref) <= tol * np.maximum(1.0, np.abs(ref))).all(), (dtype, d, np.abs(got - ref).max())
+        assert plan.last_launch_count() == 1
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [900, 350])
+    out_dev, _, plan = run_gpu(case, debug=False)
+    dev = vb.case_to_device(case)
+    qh = dev["q"].cpu().pin_memory()
+    bth = dev["block_table"].cpu().pin_memory()
+    slh = dev["seq_lens"].cpu().pin_memory()
+    outh = torch.empty_like(qh).pin_memory()
+    plan.decode_host(qh, dev["k_cache"], dev["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
+                     case.delta, case.seed, outh)
+    assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), out_dev)
+
+
+# ----------------------------------------------------------------------------- the five workloads
+def test_config1_tiny():
+    case = synth.config1_tiny()
+    out, dbg, det, _ = check(case)                 # SDPA mode: the budget saturates at the residual
+    check(case, mode=1)                            # denominator mode: a budget below the residual
+    assert det[(0, 0)]["b"] == det[(0, 0)]["n_s"]
+
+
+def test_config2_llama8b_full_size():
+    case = synth.config2_llama8b()
+    out, dbg, det, _ = check(case)
+    dens = np.mean([(len(r["I_f"]) + r["b"]) / r["n"] for r in det.values()])
+    assert 0.09 < dens < 0.11                      # the calibrated ~10x sparsity operating point
+
+
+def test_config3_uniform_full_size_and_sparsity_sweep():
+    case = synth.config3_uniform()
+    check(case)
+    n_f = 128 + 128 + case.k
+    for S in (5, 10, 20):
+        check(case, force_budget=round(32768 / S) - n_f)
+
+
+def test_config4_serving_sampled_heads():
+    case = synth.config4_serving()
+    rng = np.random.default_rng(0)
+    heads = sorted({(int(b), int(h)) for b, h in zip(rng.integers(0, 32, 24), rng.integers(0, 32, 24))})
+    out_ref, det = run_oracle(case, heads=heads)
+    out, dbg, _ = run_gpu(case)
+    assert_parity(case, out, dbg, det, out_ref)
+
+
+@pytest.mark.parametrize("n", [1024, 1025, 1039, 1040, 2048, 9000, 32768])
+def test_config5_reasoning_steps(n):
+    case = synth.config5_reasoning(n=n, B=8 if n <= 2048 else 2)
+    check(case)
