@@ -72,7 +72,7 @@ def gather_rows(cache, block_row, g, n, dtype):
     """Logical rows 0..n-1 of KV head g: row i lives at cache[block_row[i // 16], g, i % 16, :]."""
     nb = (n + BLOCK - 1) // BLOCK
     pages = np.asarray(block_row[:nb], np.int64)
-    rows = to_f64(cache[pages, g], dtype).reshape(nb * BLOCK, -1)
+    rows = to_f64(cache[pages, g], dtype).reshape(nb * BLOCK, cache.shape[-1])
     return rows[:n]
 
 
