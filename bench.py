@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the verified sparse-attention decode step (one step = one pass of the whole hot path:
+score, select, statistics + budget, final sample, gather + combine) on the Llama-3.1-8B-shaped layer
+at 32K context and ~10x sparsity.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per decode-attention step with inputs resident
+in HBM (CUDA-graph replays, rotating over distinct cache pools so no replay sees a warm L2); `e2e`
+is the same step through the host-buffer entry point (pinned host q / block table / seq_lens in, out
+back); `roofline` is the dominant kernel against the measured HBM copy bandwidth; `cpu_baseline` is the
+fp64 CPU oracle timed on this machine.  With --impl reference the oracle itself is the timed program.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "decode_attention_us_per_step"
+UNIT = "us"
+POOLS = 4
+WORKLOAD = ("cfg2_llama8b: B=1, Hq=32, Hkv=8 (GQA 4), d=128, n=32768, bf16 paged KV (block 16, HND, permuted "
+            "block table), sink=window=128, k=819 (2.5%), f_b=0.025, eps=delta=0.05, heavy-hitter strength c1=9.85")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag, self.mark = index, [], False, None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, int(reasons)))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def summary(self, t0, t1):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples[-3:]
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+                 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+                 0x100: "display_clock_setting"}
+        bits = 0
+        for s in sel:
+            bits |= s[2]
+        return {"sm_mhz": float(np.median([s[1] for s in sel])), "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in names.items() if bits & b], "samples": len(sel)}
+
+
+def oracle_step(case, heads=None):
+    from oracle import vattn_oracle as O
+    return O.vattn_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink, case.window,
+                          case.k, case.eps, case.delta, case.seed, dtype=case.dtype, heads=heads, **case.params)
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([1] + [int(p.get("num_threads", 1)) for p in threadpool_info()])
+    except Exception:
+        return 1
+
+
+def run_reference(args, rank, world):
+    """The CPU oracle as the timed program: each step is one query head of the workload (1/32 of a
+    full step), scaled to a full step; the step count is cut if the run would exceed ~3 minutes."""
+    if rank != 0:
+        return
+    from paper_2510_05688_b200 import synth
+    case = synth.config2_llama8b()
+    heads_all = [(0, h) for h in range(case.num_q_heads)]
+    t0 = time.perf_counter()
+    oracle_step(case, heads=[heads_all[0]])
+    t_one = time.perf_counter() - t0
+    budget_s = 150.0
+    steps = max(1, min(args.steps, int(budget_s / max(t_one, 1e-3))))
+    warm = min(args.warmup, 3)
+    for i in range(warm):
+        oracle_step(case, heads=[heads_all[i % len(heads_all)]])
+    t0 = time.perf_counter()
+    for i in range(steps):
+        oracle_step(case, heads=[heads_all[i % len(heads_all)]])
+    dt = time.perf_counter() - t0
+    us_full = dt / steps * len(heads_all) * 1e6
+    sample = (f"each step = 1 of {len(heads_all)} query heads of the workload (K/V de-paging of its KV head "
+              f"included), time scaled x{len(heads_all)}; {steps} of the requested {args.steps} steps timed")
+    line = {"impl": "reference", "metric": METRIC, "value": us_full, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": us_full / 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": us_full, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": us_full, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--profile-only", action="store_true",
+                    help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if not args.profile_only else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_05688_b200 import binding as vb
+    from paper_2510_05688_b200 import build as vbuild
+    from paper_2510_05688_b200 import synth
+    from paper_2510_05688_b200.shard import max_over_ranks
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        vbuild.build()
+    if world > 1:
+        dist.barrier()
+    vb.lib()
+
+    # ---- workload: every rank runs its own copy of the layer (weak scaling, no exchange on the path)
+    case = synth.config2_llama8b()
+    dev0 = vb.case_to_device(case)
+    pools = [dev0] + [{k: v.clone() for k, v in dev0.items()} for _ in range(POOLS - 1)]
+    plan = vb.plan_for_case(case)
+    plan.set_params(**case.params)
+    outs = [torch.empty_like(dev0["q"]) for _ in range(POOLS)]
+    stream = torch.cuda.Stream()
+
+    def step(i, dense=False):
+        d = pools[i % POOLS]
+        if dense:
+            plan.dense_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], outs[i % POOLS],
+                              stream=stream)
+        else:
+            plan.decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], case.sink, case.window,
+                        case.k, case.eps, case.delta, case.seed, outs[i % POOLS], stream=stream)
+
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            step(i)
+        stream.synchronize()
+        if args.profile_only:
+            for i in range(max(1, args.steps)):
+                step(i)
+            stream.synchronize()
+            if rank == 0:
+                print(json.dumps({"profile_only": True, "steps": args.steps, "launches_per_step": plan.last_launch_count()}))
+            return
+
+        # one debug call for budgets / density (not timed)
+        dbg = plan.enable_debug()
+        step(0)
+        stream.synchronize()
+        b_dyn = dbg["dyn_cnt"].cpu().numpy().astype(np.int64)
+        b0s = dbg["base_cnt"].cpu().numpy().astype(np.int64)
+        kks = dbg["topk_cnt"].cpu().numpy().astype(np.int64)
+        status = plan.last_status(stream)
+        plan.disable_debug()
+        launches_per_step = plan.last_launch_count()
+
+        # CUDA graphs: one per pool, for the sparse step and for the dense comparison
+        def capture(dense):
+            graphs = []
+            for i in range(POOLS):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    step(i, dense)
+                graphs.append(g)
+            return graphs
+
+        def timed(graphs, steps, warm):
+            for i in range(warm):
+                graphs[i % POOLS].replay()
+            stream.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            e0.record(stream)
+            for i in range(steps):
+                graphs[i % POOLS].replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t1 = time.perf_counter()
+            if world > 1:
+                dist.barrier()
+            return e0.elapsed_time(e1) / steps, t0, t1
+
+        sparse_graphs = capture(False)
+        dense_graphs = capture(True)
+        sampler = ClockSampler(local)
+        sampler.start()
+        ms_step, t0, t1 = timed(sparse_graphs, args.steps, args.warmup)
+        sampler.stop_flag = True
+        sampler.join(timeout=2.0)
+        clocks = sampler.summary(t0, t1)
+        ms_dense, _, _ = timed(dense_graphs, min(args.steps, 2000), args.warmup)
+
+        # per-kernel timing (plain launches with events between the kernels)
+        plan.set_profiling(True)
+        prof_steps = min(args.steps, 200)
+        for i in range(prof_steps):
+            step(i)
+        stream.synchronize()
+        prof, calls = plan.read_profile()
+        plan.set_profiling(False)
+
+        # end to end through the host-buffer entry point
+        qh = dev0["q"].cpu().pin_memory()
+        bth = dev0["block_table"].cpu().pin_memory()
+        slh = dev0["seq_lens"].cpu().pin_memory()
+        outh = torch.empty_like(qh).pin_memory()
+        e2e_steps = min(args.steps, 500)
+
+        def e2e_step(i):
+            d = pools[i % POOLS]
+            plan.decode_host(qh, d["k_cache"], d["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
+                             case.delta, case.seed, outh, stream=stream)
+        for i in range(3):
+            e2e_step(i)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    ms_step_max = max_over_ranks(ms_step, world)
+    ms_e2e_max = max_over_ranks(ms_e2e, world)
+    ms_dense_max = max_over_ranks(ms_dense, world)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- algorithmic bytes per launch (what each kernel must move)
+    es, d, Hq, Hkv = 2, case.head_dim, case.num_q_heads, case.num_kv_heads
+    n_tot = int(case.seq_lens.sum())
+    n_f = kks.sum() + Hq * (min(case.sink, n_tot) + min(case.window, n_tot))
+    alg = {
+        "k_score": n_tot * Hkv * d * es + n_tot * Hq * 4,
+        "k_select_topk_base": n_tot * Hq * 4,
+        "k_stats": int(n_f + b0s.sum()) * d * es * 2,
+        "k_select_final": n_tot * Hq // 8,
+        "k_gather": int(b_dyn.sum()) * (d * es + 4),
+    }
+    peak, peak_kind = measured_peaks()
+    kern = {}
+    for name in vb.KERNEL_NAMES:
+        us = prof[name] / max(calls, 1) * 1e3
+        kern[name] = {"us": round(us, 2), "alg_bytes": int(alg[name]),
+                      "gbs": round(alg[name] / (us * 1e-6) / 1e9, 1) if us > 0 else None}
+    top = max(vb.KERNEL_NAMES, key=lambda k_: prof[k_])
+    top_us = prof[top] / max(calls, 1) * 1e3
+    achieved = alg[top] / (top_us * 1e-6) / 1e9
+    density = float(np.mean((kks + 256 + b_dyn) / n_tot))
+    sparse_bytes = sum(alg[k_] for k_ in ("k_score", "k_stats", "k_gather"))
+    dense_bytes = 2 * n_tot * Hkv * d * es
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        reps, t_cpu0 = 0, time.perf_counter()
+        while reps < 2 or (time.perf_counter() - t_cpu0 < 10.0 and reps < 16):
+            oracle_step(case)
+            reps += 1
+        cpu_us = (time.perf_counter() - t_cpu0) / reps * 1e6
+        cpu = {"value": cpu_us, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+               "sample": f"{reps} full steps of the same workload (all 32 heads, fp64 numpy)"}
+
+    us_step = ms_step_max * 1e3
+    line = {
+        "metric": METRIC, "value": us_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step_max, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": f"rotating {POOLS} distinct cache pools (134 MB of K+V each, "
+                   "more than the 126 MB L2 together with the previous pool)", "launch": "CUDA graph replay per step",
+                   "mean_density": round(density, 4), "sparsity_x": round(1.0 / density, 2),
+                   "mean_budget": float(b_dyn.mean()), "status_bits": status,
+                   "value_is": "max-over-ranks step time / n_gpus (each rank runs its own layer)"},
+        "e2e": {"value": ms_e2e_max * 1e3 / world, "unit": UNIT,
+                "h2d_bytes_per_step": int(qh.numel() * 2 + bth.numel() * 4 + slh.numel() * 4),
+                "d2h_bytes_per_step": int(outh.numel() * 2)},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "kernel": top, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "frac_of": peak_kind, "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
+                     "traffic": None, "alg_bytes_per_launch": int(alg[top]), "us_per_launch": round(top_us, 2)},
+        "kernels": kern,
+        "dense": {"us_per_step": round(ms_dense_max * 1e3, 2), "alg_bytes": int(dense_bytes),
+                  "gbs": round(dense_bytes / (ms_dense_max * 1e-3) / 1e9, 1),
+                  "sparse_over_dense_time": round(ms_step_max / ms_dense_max, 3),
+                  "sparse_alg_bytes": int(sparse_bytes)},
+        "cpu_baseline": cpu,
+        "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

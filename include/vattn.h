@@ -138,6 +138,16 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */)
 /* Number of kernels the last vattn_decode / vattn_dense_decode call on this plan enqueued. */
 int vattn_last_launch_count(const vattn_plan* plan);
 
+/* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
+ * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, select top-k +
+ * base sample, statistics + budget, select final sample, gather + combine), for up to 256 calls
+ * between two reads.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
+ * milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to *calls
+ * (host), and starts a new window.  Events add a little latency: do not enable in production. */
+#define VATTN_NUM_KERNELS 5
+int vattn_set_profiling(vattn_plan* plan, int enable);
+int vattn_read_profile(vattn_plan* plan, float* ms_sum, int* calls);
+
 const char* vattn_strerror(int code);
 
 /* z(x) = Phi^{-1}(1 - x/2), the two-sided standard-normal quantile of Lemma 4.1, as the library

@@ -18,7 +18,8 @@ STATUS_BAD_BLOCK, STATUS_BAD_SEQLEN, STATUS_BAND_OVERFLOW, STATUS_NONFINITE = 1,
 EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "vattn_set_workspace",
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
            "vattn_host_staging_bytes", "vattn_decode_host", "vattn_last_status", "vattn_last_launch_count",
-           "vattn_strerror", "vattn_normal_quantile"]
+           "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile"]
+KERNEL_NAMES = ["k_score", "k_select_topk_base", "k_stats", "k_select_final", "k_gather"]
 
 
 class Shape(C.Structure):
@@ -79,6 +80,10 @@ def lib() -> C.CDLL:
     L.vattn_last_launch_count.restype = i32
     L.vattn_strerror.argtypes = [i32]
     L.vattn_strerror.restype = C.c_char_p
+    L.vattn_set_profiling.argtypes = [vp, i32]
+    L.vattn_set_profiling.restype = i32
+    L.vattn_read_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+    L.vattn_read_profile.restype = i32
     L.vattn_normal_quantile.argtypes = [C.c_double]
     L.vattn_normal_quantile.restype = C.c_double
     _lib = L
@@ -194,6 +199,16 @@ class Plan:
         bits = C.c_uint32(0)
         _check(lib().vattn_last_status(self._h, C.c_void_p(_stream(stream)), C.byref(bits)), "vattn_last_status")
         return int(bits.value)
+
+    def set_profiling(self, enable: bool):
+        _check(lib().vattn_set_profiling(self._h, 1 if enable else 0), "vattn_set_profiling")
+
+    def read_profile(self):
+        """(dict kernel name -> summed ms, calls) since profiling was enabled or last read."""
+        ms = (C.c_float * len(KERNEL_NAMES))()
+        calls = C.c_int(0)
+        _check(lib().vattn_read_profile(self._h, ms, C.byref(calls)), "vattn_read_profile")
+        return {n: float(ms[i]) for i, n in enumerate(KERNEL_NAMES)}, int(calls.value)
 
     def last_launch_count(self) -> int:
         return int(lib().vattn_last_launch_count(self._h))

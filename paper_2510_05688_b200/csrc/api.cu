@@ -13,6 +13,10 @@ struct vattn_plan {
   size_t ws_bytes;
   bool status_ready;
   int last_launches;
+  // optional per-kernel timing (events are created on first use; no device memory involved)
+  bool profiling;
+  cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
+  int prof_calls;           // calls recorded since the last read
   // derived
   int G, npad, nwords, stat_splits, gat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
@@ -22,6 +26,12 @@ struct vattn_plan {
 namespace {
 
 constexpr int kNumSM = 148;          // B200; the library is built for sm_100a only
+constexpr int kProfCalls = 256;      // calls whose events are kept between two reads of the profile
+constexpr int kProfEvents = VATTN_NUM_KERNELS + 1;
+
+inline void prof_mark(vattn_plan* pl, int slot, cudaStream_t st) {
+  if (pl->profiling && pl->ev && pl->prof_calls < kProfCalls) cudaEventRecord(pl->ev[pl->prof_calls * kProfEvents + slot], st);
+}
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -175,7 +185,43 @@ int vattn_plan_create(const vattn_shape* shape, vattn_plan** out) {
   return VATTN_OK;
 }
 
-void vattn_plan_destroy(vattn_plan* plan) { delete plan; }
+void vattn_plan_destroy(vattn_plan* plan) {
+  if (!plan) return;
+  if (plan->ev) {
+    for (int i = 0; i < kProfCalls * kProfEvents; ++i) cudaEventDestroy(plan->ev[i]);
+    delete[] plan->ev;
+  }
+  delete plan;
+}
+
+int vattn_set_profiling(vattn_plan* plan, int enable) {
+  if (!plan) return VATTN_ERR_INVALID_ARG;
+  if (enable && !plan->ev) {
+    plan->ev = new (std::nothrow) cudaEvent_t[kProfCalls * kProfEvents];
+    if (!plan->ev) return VATTN_ERR_INVALID_ARG;
+    for (int i = 0; i < kProfCalls * kProfEvents; ++i)
+      if (cudaEventCreate(&plan->ev[i]) != cudaSuccess) return VATTN_ERR_CUDA;
+  }
+  plan->profiling = enable != 0;
+  plan->prof_calls = 0;
+  return VATTN_OK;
+}
+
+int vattn_read_profile(vattn_plan* plan, float* ms_sum, int* calls) {
+  if (!plan || !ms_sum || !calls) return VATTN_ERR_INVALID_ARG;
+  for (int k = 0; k < VATTN_NUM_KERNELS; ++k) ms_sum[k] = 0.f;
+  *calls = plan->prof_calls;
+  if (!plan->ev || plan->prof_calls == 0) return VATTN_OK;
+  CU(cudaEventSynchronize(plan->ev[(plan->prof_calls - 1) * kProfEvents + VATTN_NUM_KERNELS]));
+  for (int c = 0; c < plan->prof_calls; ++c)
+    for (int k = 0; k < VATTN_NUM_KERNELS; ++k) {
+      float ms = 0.f;
+      CU(cudaEventElapsedTime(&ms, plan->ev[c * kProfEvents + k], plan->ev[c * kProfEvents + k + 1]));
+      ms_sum[k] += ms;
+    }
+  plan->prof_calls = 0;
+  return VATTN_OK;
+}
 
 size_t vattn_workspace_bytes(const vattn_plan* plan) { return plan ? plan->total : 0; }
 
@@ -225,14 +271,21 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   plan->last_launches = 0;
   rc = prepare_stream(plan, p, st);
   if (rc != VATTN_OK) return rc;
+  prof_mark(plan, 0, st);
   CU(launch_score(p, st));            plan->last_launches++;
+  prof_mark(plan, 1, st);
   if (p.dbg.scores)
     CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
                          sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
   CU(launch_select_topk_base(p, st)); plan->last_launches++;
+  prof_mark(plan, 2, st);
   CU(launch_stats(p, st));            plan->last_launches++;
+  prof_mark(plan, 3, st);
   CU(launch_select_final(p, st));     plan->last_launches++;
+  prof_mark(plan, 4, st);
   CU(launch_gather(p, st));           plan->last_launches++;
+  prof_mark(plan, 5, st);
+  if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
   return VATTN_OK;
 }
 

@@ -451,11 +451,21 @@ size_t select_smem_bytes(const Prob& p) {
          sizeof(unsigned) * 256 + sizeof(int) * VATTN_BANDCAP + sizeof(int) * 64;
 }
 
+// Opt-in to large dynamic shared memory once per kernel and size (a function attribute, not a
+// stream operation; done before the first launch so that later launches can be stream-captured).
 template <typename KernelT>
 static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s) {
   const size_t smem = select_smem_bytes(p);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  static const void* seen_fn[32];
+  static size_t seen_sz[32];
+  static int nseen = 0;
+  bool done = false;
+  for (int i = 0; i < nseen; ++i) done = done || (seen_fn[i] == (const void*)kern && seen_sz[i] >= smem);
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (nseen < 32) { seen_fn[nseen] = (const void*)kern; seen_sz[nseen] = smem; ++nseen; }
+  }
   dim3 grid(p.Hq, p.B), block(NT);
   kern<<<grid, block, smem, s>>>(p, keycap_of(p));
   return cudaGetLastError();
