@@ -122,6 +122,34 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
 int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
 
+/*
+ * vattn_dense_decode for callers that cannot give the library a workspace.  (The paper has no
+ * counterpart: this is a deployment convenience.)  Who needs it: a serving engine that handed the
+ * whole GPU to its KV-cache pool at start-up and has no device memory left to carve a workspace
+ * from, or code on a latency-critical path that must not call cudaMalloc (which synchronises the
+ * device).  No plan is needed and nothing is allocated, on the host or on the device: the split
+ * partials live in a fixed array of VATTN_NOALLOC_SCRATCH_BYTES that is part of the library image, so
+ * every GPU that loads the library holds that much memory until the process exits.
+ *   - `scale` 0 means 1/sqrt(head_dim).  Arguments and layouts are those of vattn_dense_decode.
+ *   - The problem must fit: 256 + 12*batch*num_q_heads (rounded up to 256) +
+ *     batch*num_q_heads*(head_dim+2)*4 bytes <= VATTN_NOALLOC_SCRATCH_BYTES (about 8,000 (batch row, query
+ *     head) pairs at head_dim 128); larger problems return VATTN_ERR_WORKSPACE.  Fewer context splits are
+ *     used when the usual number does not fit, so results can differ from vattn_dense_decode in the
+ *     last bits.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls, from every thread and stream, share the one array: two calls that overlap on the GPU
+ *     race.  Serialise them on one stream or with events.  The part that must start at zero is cleared
+ *     on `stream` at the start of every call.
+ *   - Block-table entries outside [0, num_blocks) are read as page 0, as in vattn_dense_decode, but there
+ *     is no status word to query.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE (too large), CUDA.
+ */
+#define VATTN_NOALLOC_SCRATCH_BYTES (4u << 20)
+int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale, const void* q, const void* k_cache,
+                               const void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
+                               void* out, void* stream);
+
 /* Same step as vattn_decode with HOST buffers for q, block_table, seq_lens and out (the caches stay on
  * the device): copies the inputs in, runs the step, copies `out` back and waits for it.  `staging` is a
  * caller-owned device buffer of at least vattn_host_staging_bytes(plan) bytes. */

@@ -18,7 +18,9 @@ STATUS_BAD_BLOCK, STATUS_BAD_SEQLEN, STATUS_BAND_OVERFLOW, STATUS_NONFINITE = 1,
 EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "vattn_set_workspace",
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
            "vattn_host_staging_bytes", "vattn_decode_host", "vattn_last_status", "vattn_last_launch_count",
-           "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile"]
+           "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
+           "vattn_dense_decode_noalloc"]
+NOALLOC_SCRATCH_BYTES = 4 << 20
 KERNEL_NAMES = ["k_score", "k_select_topk_base", "k_stats", "k_select_final", "k_gather"]
 
 
@@ -84,6 +86,8 @@ def lib() -> C.CDLL:
     L.vattn_set_profiling.restype = i32
     L.vattn_read_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     L.vattn_read_profile.restype = i32
+    L.vattn_dense_decode_noalloc.argtypes = [C.POINTER(Shape), f32, vp, vp, vp, vp, vp, vp, vp]
+    L.vattn_dense_decode_noalloc.restype = i32
     L.vattn_normal_quantile.argtypes = [C.c_double]
     L.vattn_normal_quantile.restype = C.c_double
     _lib = L
@@ -219,6 +223,15 @@ def _stream(stream):
         import torch
         return torch.cuda.current_stream().cuda_stream
     return int(getattr(stream, "cuda_stream", stream))
+
+
+def dense_decode_noalloc(shape: Shape, q, k_cache, v_cache, block_table, seq_lens, out, scale=0.0, stream=None):
+    """Dense decode through the entry point that needs no plan and no workspace: for callers that
+    cannot allocate device memory (everything handed to a cache pool, or cudaMalloc off limits on
+    their path).  Returns the ABI's return code instead of raising, so callers can test the limits."""
+    return int(lib().vattn_dense_decode_noalloc(C.byref(shape), float(scale), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                                _ptr(block_table), _ptr(seq_lens), _ptr(out),
+                                                C.c_void_p(_stream(stream))))
 
 
 def normal_quantile(x: float) -> float:

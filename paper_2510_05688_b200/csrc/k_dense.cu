@@ -2,6 +2,8 @@
 // context is split over CTAs, every CTA keeps an online softmax for the (up to 4) query heads of a
 // KV-head group, and the last CTA of a group merges the split partials in a fixed order.
 // This is the comparison kernel: the latency the sparse step has to beat on the same cache.
+#include <math.h>
+#include <string.h>
 #include "vattn_internal.cuh"
 
 namespace {
@@ -206,4 +208,97 @@ cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches) {
   }
   if (launches) *launches = 1;
   return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Dense decode without any caller-provided scratch.
+//
+// Some callers cannot hand this library a workspace: a serving engine that claimed the whole GPU
+// for its KV-cache pool at start-up has nothing left to carve one from, and code on a latency-
+// critical path may not call cudaMalloc at all (it synchronises the device).  For them the split
+// partials and the "last CTA" tickets of the dense kernel live in the fixed array below, which
+// every GPU that loads this library holds until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[VATTN_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices];       // device address of g_noalloc_scratch, per device ordinal
+bool g_scratch_ready[kMaxDevices];
+
+// The array's name is only a host-side handle in host code; the address a kernel can use has to be
+// asked for, once per device, with that device current.
+cudaError_t noalloc_scratch(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_scratch_ready[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_addr[dev] = ptr;
+    g_scratch_ready[dev] = true;
+  }
+  *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+}  // namespace
+
+extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale, const void* q, const void* k_cache,
+                                          const void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
+                                          void* out, void* stream) {
+  if (!shape || !q || !k_cache || !v_cache || !block_table || !seq_lens || !out) return VATTN_ERR_INVALID_ARG;
+  const vattn_shape& s = *shape;
+  if (s.batch <= 0 || s.num_q_heads <= 0 || s.num_kv_heads <= 0 || s.max_blocks_per_seq <= 0 || s.num_blocks <= 0 ||
+      s.max_seq_len < 0 || s.num_q_heads % s.num_kv_heads != 0 || s.batch > 65535 || s.num_q_heads > 65535)
+    return VATTN_ERR_INVALID_ARG;
+  if ((s.head_dim != 64 && s.head_dim != 128) || s.block_size != VATTN_BLOCK ||
+      (s.dtype != VATTN_DTYPE_FP32 && s.dtype != VATTN_DTYPE_BF16) || s.num_q_heads / s.num_kv_heads > 64)
+    return VATTN_ERR_UNSUPPORTED;
+  if ((long long)s.max_seq_len > (long long)s.max_blocks_per_seq * s.block_size) return VATTN_ERR_INVALID_ARG;
+  const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_cache) |
+                         reinterpret_cast<uintptr_t>(v_cache) | reinterpret_cast<uintptr_t>(out);
+  if (bits & 15) return VATTN_ERR_INVALID_ARG;
+  if (!(scale == scale) || isinf(scale)) return VATTN_ERR_INVALID_ARG;
+
+  // layout inside the fixed array: status word | tickets (must start at zero) | split partials
+  const size_t BH = (size_t)s.batch * s.num_q_heads, D = (size_t)s.head_dim;
+  const int G = s.num_q_heads / s.num_kv_heads, GC = (G + 3) / 4;
+  const size_t groups = (size_t)s.batch * s.num_kv_heads * GC;
+  const size_t head_bytes = 256 + up256(3 * BH * sizeof(unsigned));
+  int splits = (int)((4 * 148 + groups - 1) / groups);
+  splits = splits < 1 ? 1 : (splits > 128 ? 128 : splits);
+  while (splits > 1 && head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES) --splits;
+  if (head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES)
+    return VATTN_ERR_WORKSPACE;     // batch * heads too large for the built-in scratch
+
+  void* base = nullptr;
+  if (noalloc_scratch(&base) != cudaSuccess) return VATTN_ERR_CUDA;
+  unsigned char* w = static_cast<unsigned char*>(base);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  Prob p;
+  memset(&p, 0, sizeof(p));
+  p.B = s.batch; p.Hq = s.num_q_heads; p.Hkv = s.num_kv_heads; p.G = G; p.D = s.head_dim; p.dtype = s.dtype;
+  p.max_blocks = s.max_blocks_per_seq; p.num_blocks = s.num_blocks; p.max_seq_len = s.max_seq_len;
+  if (s.kv_stride_block == 0 && s.kv_stride_head == 0 && s.kv_stride_token == 0) {
+    p.st = s.head_dim; p.sh = (long long)s.block_size * s.head_dim; p.sb = (long long)s.num_kv_heads * p.sh;
+  } else {
+    const int epl = s.dtype == VATTN_DTYPE_BF16 ? 8 : 4;
+    if (s.kv_stride_block <= 0 || s.kv_stride_head <= 0 || s.kv_stride_token < s.head_dim ||
+        s.kv_stride_block % epl || s.kv_stride_head % epl || s.kv_stride_token % epl)
+      return VATTN_ERR_INVALID_ARG;
+    p.sb = s.kv_stride_block; p.sh = s.kv_stride_head; p.st = s.kv_stride_token;
+  }
+  p.q = q; p.kc = k_cache; p.vc = v_cache; p.bt = block_table; p.seq_lens = seq_lens; p.out = out;
+  p.scale = scale != 0.f ? scale : (float)(1.0 / sqrt((double)s.head_dim));
+  p.status = reinterpret_cast<unsigned*>(w);
+  p.tickets = reinterpret_cast<unsigned*>(w + 256);
+  p.dense_part = reinterpret_cast<float*>(w + head_bytes);
+  p.dense_splits = splits;
+  // the array keeps whatever the previous call left: the tickets and the status word must be zero again
+  if (cudaMemsetAsync(w, 0, head_bytes, st) != cudaSuccess) return VATTN_ERR_CUDA;
+  if (launch_dense(p, st, nullptr) != cudaSuccess) return VATTN_ERR_CUDA;
+  return VATTN_OK;
 }
