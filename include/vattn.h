@@ -45,6 +45,7 @@ extern "C" {
 #define VATTN_STATUS_BAD_SEQLEN     2u   /* a seq_len was outside [0, max_seq_len]: clamped */
 #define VATTN_STATUS_BAND_OVERFLOW  4u   /* more near-tie top-k candidates than the fast list holds: exact slow path ran */
 #define VATTN_STATUS_NONFINITE      8u   /* a budget statistic was not finite: that head used the whole residual */
+#define VATTN_STATUS_WAIT_TIMEOUT  16u   /* a bounded wait for an asynchronous copy ran out: the step's output is invalid */
 
 typedef struct vattn_plan vattn_plan;    /* opaque; host memory */
 
@@ -80,6 +81,9 @@ typedef struct {
   double  *stats;                 /* [B,Hq,8] D_f, sigma^2, Tr(Sigma), D_hat, |N_hat|_2, n_s, b0, m (weights are
                                      exp(s - m) with m the head's largest fp32 score) */
   float   *scores;                /* [B,Hq,cap] fp32 scores s_i = scale * <K[i], q> */
+  int32_t *paths;                 /* [B,Hq] which code path selected each set: bit 0 top-k from the sampled threshold
+                                     estimate, bit 1 base sample from the pre-filtered list, bit 2 final sample from
+                                     the pre-filtered list (a clear bit = the full-context select ran) */
 } vattn_debug;
 
 /* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG, UNSUPPORTED. */

@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(_PKG, "libvattn.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-STATUS_BAD_BLOCK, STATUS_BAD_SEQLEN, STATUS_BAND_OVERFLOW, STATUS_NONFINITE = 1, 2, 4, 8
+STATUS_BAD_BLOCK, STATUS_BAD_SEQLEN, STATUS_BAND_OVERFLOW, STATUS_NONFINITE, STATUS_WAIT_TIMEOUT = 1, 2, 4, 8, 16
 
 EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "vattn_set_workspace",
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
@@ -40,7 +40,7 @@ class Params(C.Structure):
 class Debug(C.Structure):
     _fields_ = [("topk_idx", C.c_void_p), ("topk_cnt", C.c_void_p), ("base_idx", C.c_void_p),
                 ("base_cnt", C.c_void_p), ("dyn_idx", C.c_void_p), ("dyn_cnt", C.c_void_p),
-                ("budgets", C.c_void_p), ("stats", C.c_void_p), ("scores", C.c_void_p)]
+                ("budgets", C.c_void_p), ("stats", C.c_void_p), ("scores", C.c_void_p), ("paths", C.c_void_p)]
 
 
 _lib = None
@@ -166,7 +166,8 @@ class Plan:
             dyn_idx=torch.zeros(*BH, cap, dtype=i32, device=dev), dyn_cnt=torch.zeros(*BH, dtype=i32, device=dev),
             budgets=torch.zeros(*BH, 4, dtype=i32, device=dev),
             stats=torch.zeros(*BH, 8, dtype=torch.float64, device=dev),
-            scores=torch.zeros(*BH, cap, dtype=torch.float32, device=dev))
+            scores=torch.zeros(*BH, cap, dtype=torch.float32, device=dev),
+            paths=torch.zeros(*BH, dtype=i32, device=dev))
         d = Debug(**{k_: v.data_ptr() for k_, v in self.debug.items()})
         _check(lib().vattn_set_debug(self._h, C.byref(d)), "vattn_set_debug")
         return self.debug

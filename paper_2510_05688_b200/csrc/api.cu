@@ -13,6 +13,7 @@ struct vattn_plan {
   size_t ws_bytes;
   bool status_ready;
   int last_launches;
+  unsigned long long* devt;
   // optional per-kernel timing (events are created on first use; no device memory involved)
   bool profiling;
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
@@ -20,12 +21,15 @@ struct vattn_plan {
   // derived
   int G, npad, nwords, stat_splits, gat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
-      off_det, off_gat, off_dense, total;
+      off_det, off_gat, off_dense, off_cand, total;
+  int cand_cap;
 };
 
 namespace {
 
 constexpr int kNumSM = 148;          // B200; the library is built for sm_100a only
+constexpr int kMaxStatSplits = 16;    // split CTAs per head and row kind of the statistics kernel
+constexpr int kMaxGatherSplits = 32;  // split CTAs per head of the gather kernel
 constexpr int kProfCalls = 256;      // calls whose events are kept between two reads of the profile
 constexpr int kProfEvents = VATTN_NUM_KERNELS + 1;
 
@@ -61,9 +65,12 @@ void derive(vattn_plan* pl) {
   if (pl->npad == 0) pl->npad = 32;
   pl->nwords = pl->npad / 32;
   const int heads = s.batch * s.num_q_heads;
-  int sp = (4 * kNumSM + heads - 1) / heads;
-  pl->stat_splits = sp < 1 ? 1 : (sp > 32 ? 32 : sp);
-  pl->gat_splits = pl->stat_splits;
+  // row kernels (128-thread CTAs): one wave of about 5 (statistics, two CTA kinds per split) or 8
+  // (gather) CTAs per SM
+  int sp = (5 * kNumSM) / (2 * heads);
+  pl->stat_splits = sp < 1 ? 1 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
+  sp = (8 * kNumSM) / heads;
+  pl->gat_splits = sp < 1 ? 1 : (sp > kMaxGatherSplits ? kMaxGatherSplits : sp);
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
   sp = (4 * kNumSM + groups - 1) / groups;
@@ -72,7 +79,7 @@ void derive(vattn_plan* pl) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   pl->off_scores = take(BH * pl->npad * sizeof(float));
-  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH) * sizeof(unsigned);
+  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 2 * BH) * sizeof(unsigned);
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
@@ -80,10 +87,15 @@ void derive(vattn_plan* pl) {
   pl->off_base = take(BH * pl->npad * sizeof(int));
   pl->off_dyn = take(BH * pl->npad * sizeof(int));
   pl->off_meta = take(BH * sizeof(HeadMeta));
-  pl->off_stat = take(BH * pl->stat_splits * (2 * D + 4) * sizeof(double));
+  pl->off_stat = take(BH * 2 * kMaxStatSplits * (D + 3) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
   pl->off_gat = take(BH * pl->gat_splits * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
+  {
+    const double q4 = 0.25 * (double)pl->npad;
+    pl->cand_cap = ((int)(q4 + 8.0 * sqrt(q4) + 64.0) + 31) / 32 * 32;
+  }
+  pl->off_cand = take(2 * BH * (size_t)pl->cand_cap * sizeof(uint2));
   pl->total = off;
 }
 
@@ -111,6 +123,9 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
   const size_t BH = (size_t)s.batch * s.num_q_heads;
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
+  p.cand_cnt = p.tickets + 3 * BH;
+  p.cand = reinterpret_cast<uint2*>(w + pl->off_cand);
+  p.cand_cap = pl->cand_cap;
   p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
   p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);
   p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
@@ -123,6 +138,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.stat_splits = pl->stat_splits; p.gat_splits = pl->gat_splits; p.dense_splits = pl->dense_splits;
   p.dbg = pl->dbg;
+  p.devt = pl->devt;
   return VATTN_OK;
 }
 
@@ -261,6 +277,18 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   Prob p;
   fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
   p.sink = sink; p.window = window; p.k = k;
+  {
+    // statistics kernel: about 64 rows (8 per row group) per CTA, never more CTAs than rows warrant
+    const double msl = (double)plan->shape.max_seq_len;
+    double kmax = plan->params.topk_frac > 0.f ? floor((double)plan->params.topk_frac * msl) : (double)k;
+    double rows = (double)sink + (double)window + kmax;
+    if (rows > msl) rows = msl;
+    const double brows = (double)p.base_rate * msl;
+    if (brows > rows) rows = brows;
+    int want = (int)((rows + 63.0) / 64.0);
+    if (want < 1) want = 1;
+    if (want < p.stat_splits) p.stat_splits = want;
+  }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;
   p.z_delta = upper_quantile(0.5 * p.delta);
@@ -347,6 +375,10 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits) {
   CU(cudaStreamSynchronize(st));
   return VATTN_OK;
 }
+
+#ifdef VATTN_DEV_TIMING
+int vattn_dev_set_timing_buffer(vattn_plan* plan, void* ptr) { plan->devt = static_cast<unsigned long long*>(ptr); return 0; }
+#endif
 
 int vattn_last_launch_count(const vattn_plan* plan) { return plan ? plan->last_launches : 0; }
 

@@ -1,29 +1,487 @@
-// Score pass: s[b,h,i] = scale * <q[b,h], K[b,g,i]> for every token of the paged cache, the (up to 4)
-// query heads of a KV-head group together (the inner products of the SDPA definition, Sec. 3 of the
-// paper; Algorithm 1 line 3 ranks tokens by them).  Also keeps, per query head, the running maximum
-// score (softmax stabiliser) and, per KV head, max |K element| (used for the rounding-error bound of
-// these fp32 scores).
+// Score pass: s[b,h,i] = scale * <q[b,h], K[b,g,i]> for every token of the paged cache, the query heads
+// of a KV-head group together (the inner products of the SDPA definition, Sec. 3 of the paper;
+// Algorithm 1 line 3 ranks tokens by them).  Also keeps, per query head, the running maximum score
+// (softmax stabiliser) and, per KV head, max |K element| (for the rounding-error bound of the scores).
 //
-// HBM-bound stream over K: a warp owns whole 16-token pages; LPR lanes cover one row with one 16-byte
-// load each, so a warp instruction fetches 512 contiguous bytes.  Summation structure (this fixes the
-// error bound the select kernel uses): EPL sequential fp32 FMAs per lane, then a log2(LPR)-level
-// butterfly that halves the number of live partial sums at every level ("reduce-scatter"), one
-// multiply by `scale`: at most 13 roundings.
+// HBM-bound stream over K (every K row is read exactly once).  Two arithmetic paths:
+//  * bf16: the [16 tokens x d] x [d x 8 heads] contraction of a page runs on the tensor cores
+//    (mma.sync m16n8k16, fp32 accumulate).  K fragments are loaded straight from global memory with
+//    16-byte loads: a dot product does not care in which order its terms are paired, so the k-slots of
+//    the fragment layout are mapped onto d such that each thread owns 8 consecutive elements of a row.
+//    This removes the CUDA-core FMAs and the cross-lane reduction that made the pass ALU-co-bound.
+//  * fp32: CUDA-core FMAs, EPL sequential FMAs per lane and a butterfly that halves the live partial
+//    sums at every level (tf32 tensor cores would not keep fp32 accuracy).
+//
+// The same CTAs also pre-filter the sampling keys: Philox4x32-10 keys of streams 0 and 1 are computed
+// for every (token, head) of the tile and tokens whose key is below the stream's bound are appended to
+// per-head candidate lists, so the select kernels never run Philox over the whole context
+// (uniform-sample of Algorithm 1 line 7 / Algorithm 2 line 1 = the c smallest keys of the residual).
 #include "vattn_internal.cuh"
 
 namespace {
 
 constexpr int PPW = 4;      // pages per warp
 constexpr int WARPS = 4;    // warps per CTA
-constexpr int TILE = PPW * WARPS * VATTN_BLOCK;
+constexpr int TILE = PPW * WARPS * VATTN_BLOCK;   // 256 tokens
 
+// ---------------------------------------------------------------------------------------------
+// sampling-candidate pre-filter for the tile [tile0, tile0 + TILE) and heads h0 .. h0 + nh - 1
+template <int MAXH>
+__device__ void emit_candidates(const Prob& p, int b, int g, int h0, int nh, int tile0, int n,
+                                uint2 (*s_list)[TILE], unsigned* s_cnt) {
+  const int tid = threadIdx.x;
+  const Geo geo = head_geometry(p, n);
+  if (geo.n_s <= 0) return;                                    // uniform for the CTA
+  const unsigned bound0 = cand0_bound(geo);
+  for (int i = tid; i < 2 * MAXH; i += WARPS * 32) s_cnt[i] = 0;
+  __syncthreads();
+  const unsigned c3base = (unsigned)p.step << 1;
+  for (int item = tid; item < nh * (TILE / 4); item += WARPS * 32) {
+    const int hh = item / (TILE / 4), quad = item % (TILE / 4);
+    const int t0 = tile0 + quad * 4;
+    if (t0 >= geo.l_start || t0 + 4 <= geo.s0) continue;
+    const int hrng = p.rng_head_is_kv ? g : (h0 + hh);
+    const unsigned c1 = ((unsigned)b << 16) | (unsigned)hrng;
+#pragma unroll
+    for (int stream = 0; stream < 2; ++stream) {
+      const unsigned bound = stream ? VATTN_CAND1_BOUND : bound0;
+      if (bound == 0u) continue;
+      const uint4 r = philox4x32_10((unsigned)(t0 >> 2), c1, (unsigned)p.layer, c3base | (unsigned)stream,
+                                    p.seed_lo, p.seed_hi);
+      const unsigned key[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int tok = t0 + e;
+        if (key[e] < bound && tok >= geo.s0 && tok < geo.l_start) {
+          const unsigned pos = atomicAdd(&s_cnt[stream * MAXH + hh], 1u);
+          s_list[stream * MAXH + hh][pos] = make_uint2(key[e], (unsigned)tok);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int l = warp; l < 2 * MAXH; l += WARPS) {
+    const int stream = l / MAXH, hh = l % MAXH;
+    const unsigned cnt = s_cnt[l];
+    if (hh >= nh || cnt == 0) continue;
+    const long long bh = (long long)b * p.Hq + h0 + hh;
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(&p.cand_cnt[(long long)stream * p.B * p.Hq + bh], cnt);
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    uint2* dst = p.cand + ((long long)stream * p.B * p.Hq + bh) * p.cand_cap;
+    for (unsigned j = lane; j < cnt; j += 32)
+      if (base + j < (unsigned)p.cand_cap) dst[base + j] = s_list[l][j];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// bf16: tensor-core path, up to 8 heads per CTA
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                               unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D>
+__global__ void __launch_bounds__(WARPS * 32) k_score_mma(const Prob p) {
+  constexpr int NC = D / 32;            // 32-element chunks of a row; one chunk feeds two MMAs
+  __shared__ uint2 s_list[16][TILE];
+  __shared__ unsigned s_cnt[16];
+  DEV_BEGIN(p, 1);
+  const int b = blockIdx.z;
+  const int n = clamped_len(p, b);
+  const int tile0 = blockIdx.x * TILE;
+  if (tile0 >= n) return;
+  const int GC = (p.G + 7) >> 3;
+  const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gr = lane >> 2, t = lane & 3;       // fragment row / column-pair index
+  const int h0 = g * p.G + hc * 8;
+  const int nh = min(8, p.G - hc * 8);
+  const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
+
+  // B fragments: head (hc*8 + gr) of the group, this thread's 8 elements of every chunk
+  uint4 bq[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    bq[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (gr < nh)
+      bq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
+                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
+  }
+  DEV_MARK(p, 1, 2, blockIdx.x == 0 && blockIdx.y == 0);
+  float runmax[2] = {-INFINITY, -INFINITY};
+  unsigned kabs = 0u;                            // packed max of |bf16| (two 15-bit magnitudes)
+
+#pragma unroll
+  for (int pp = 0; pp < PPW; pp += 2) {
+    int tok0[2];
+    uint4 alo[2][NC], ahi[2][NC];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      tok0[u] = tile0 + (warp * PPW + pp + u) * VATTN_BLOCK;
+      if (tok0[u] < n) {
+        const bf16_t* base = kc + (long long)page_of(p, b, tok0[u] >> 4) * p.sb + (long long)g * p.sh;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          alo[u][c] = *reinterpret_cast<const uint4*>(base + (long long)gr * p.st + c * 32 + t * 8);
+          ahi[u][c] = *reinterpret_cast<const uint4*>(base + (long long)(gr + 8) * p.st + c * 32 + t * 8);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (tok0[u] >= n) continue;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      unsigned klo = 0u, khi = 0u;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        mma_bf16_16816(acc, alo[u][c].x, ahi[u][c].x, alo[u][c].y, ahi[u][c].y, bq[c].x, bq[c].y);
+        mma_bf16_16816(acc, alo[u][c].z, ahi[u][c].z, alo[u][c].w, ahi[u][c].w, bq[c].z, bq[c].w);
+        klo = __vimax3_u16x2(klo, alo[u][c].x & 0x7FFF7FFFu, alo[u][c].y & 0x7FFF7FFFu);
+        klo = __vimax3_u16x2(klo, alo[u][c].z & 0x7FFF7FFFu, alo[u][c].w & 0x7FFF7FFFu);
+        khi = __vimax3_u16x2(khi, ahi[u][c].x & 0x7FFF7FFFu, ahi[u][c].y & 0x7FFF7FFFu);
+        khi = __vimax3_u16x2(khi, ahi[u][c].z & 0x7FFF7FFFu, ahi[u][c].w & 0x7FFF7FFFu);
+      }
+      const int tk_lo = tok0[u] + gr, tk_hi = tok0[u] + gr + 8;
+      if (tk_lo < n) kabs = __vimax3_u16x2(kabs, klo, 0u);
+      if (tk_hi < n) kabs = __vimax3_u16x2(kabs, khi, 0u);
+      // acc[0],acc[1]: token gr, heads 2t, 2t+1;  acc[2],acc[3]: token gr+8
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int hl = 2 * t + e;
+        if (hl < nh) {
+          float* dst = p.scores + ((long long)b * p.Hq + h0 + hl) * p.npad;
+          const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
+          if (tk_lo < n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
+          if (tk_hi < n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int mask = 4; mask < 32; mask <<= 1) {
+    runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
+    runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
+  }
+#pragma unroll
+  for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
+  if (lane < 4) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int hl = 2 * lane + e;
+      if (hl < nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[b * p.Hq + h0 + hl], ord_f32(runmax[e]));
+    }
+  }
+  if (lane == 0) {
+    const unsigned mx = max(kabs & 0xFFFFu, kabs >> 16);          // bf16 magnitude bits
+    atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);               // = fp32 bits of that magnitude
+  }
+  DEV_MARK(p, 1, 3, blockIdx.x == 0 && blockIdx.y == 0);
+  emit_candidates<8>(p, b, g, h0, nh, tile0, n, s_list, s_cnt);
+  DEV_END(p, 1);
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// bf16, streaming variant: every warp owns a ring of NST shared-memory stages and keeps NST pages
+// (16 tokens x d, one contiguous slab of the paged cache) in flight with bulk asynchronous copies
+// (cp.async.bulk + mbarrier transaction counts); fragments are read back with 16-byte shared loads.
+// The copies need no registers while in flight, so an SM holds ~130 KB of outstanding reads with two
+// resident CTAs.  A warp walks the pages p = w, w + W, w + 2W, ... of its (batch row, KV head).
+constexpr int NST = 4;          // stages per warp
+constexpr int CWARPS = 8;       // warps of a CTA that pre-filter sampling keys (two per streaming warp)
+constexpr unsigned WAIT_SPINS = 1u << 20;
+
+__device__ __forceinline__ unsigned smem_u32(const void* ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: gives up after WAIT_SPINS polls and reports it
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (unsigned it = 0; it < WAIT_SPINS; ++it) {
+    __nanosleep(64);                      // leave the issue slots to the warps that have work
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// Sampling-candidate pre-filter, run by the CWARPS candidate warps of a CTA: Philox keys of streams 0
+// and 1 for every (token, head) of the CTA's pages; tokens whose key is below the stream's bound are
+// staged in CTA-wide lists, one per (stream, head), and appended to the global lists every CHUNK pages
+// per warp.  Lanes are items (stream, head, token quad); the 4 lanes of a list are adjacent, so the
+// positions inside a page come from ballots; one shared-memory atomic per (page, list) reserves the
+// range.  Global counters are bumped once per list and flush, which keeps the contended atomics rare.
+constexpr int CL = 256;          // staged entries per (stream, head) list of a CTA
+constexpr int CHUNK = 4;         // pages per candidate warp between two flushes (CWARPS*CHUNK*16*1/4 = 128 expected)
+
+__device__ __forceinline__ void cand_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(CWARPS * 32) : "memory"); }
+
+__device__ void candidate_warps(const Prob& p, int b, int g, int h0, int nh, int n, int page0, int wtot, int npages,
+                                int cw, uint2* clist, unsigned* s_cnt) {
+  const int lane = threadIdx.x & 31;
+  const Geo geo = head_geometry(p, n);
+  if (geo.n_s <= 0) return;                                   // uniform over the CTA
+  const unsigned bound0 = cand0_bound(geo);
+  const int nitems = 8 * nh, nrounds = (nitems + 31) >> 5;
+  const unsigned lmask = 0xFu << (lane & ~3), lt = (1u << lane) - 1u;
+  // pages of this CTA: page0 + j * wtot for the streaming warp j % WARPS; candidate warp cw takes the
+  // CTA-local page slots cw, cw + CWARPS, ...   (slot s = page page0_cta + (s % WARPS) + (s / WARPS) * wtot)
+  const int slots = (npages > page0) ? ((npages - 1 - page0) / wtot + 1) * WARPS : 0;   // upper bound, CTA-uniform
+  const int nchunks = (slots + CWARPS * CHUNK - 1) / (CWARPS * CHUNK);
+  if (cw * 32 + lane < 16) s_cnt[cw * 32 + lane] = 0u;
+  cand_barrier();
+  for (int c = 0; c < nchunks; ++c) {
+    for (int kk = 0; kk < CHUNK; ++kk) {
+      const int slot = (c * CHUNK + kk) * CWARPS + cw;
+      const int page = page0 + (slot % WARPS) + (slot / WARPS) * wtot;
+      const int tok0 = page << 4;
+      if (page >= npages || tok0 >= geo.l_start || tok0 + 16 <= geo.s0) continue;
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        if (r >= nrounds) break;
+        const int item = 32 * r + lane;
+        const int L = item >> 2, quad = item & 3;
+        const int stream = L / nh, hh = L % nh;
+        const unsigned bound = (item < nitems) ? (stream ? VATTN_CAND1_BOUND : bound0) : 0u;
+        const int t0 = tok0 + quad * 4;
+        unsigned key[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+        if (bound) {
+          const int hrng = p.rng_head_is_kv ? g : (h0 + hh);
+          const uint4 rr = philox4x32_10((unsigned)(t0 >> 2), ((unsigned)b << 16) | (unsigned)hrng, (unsigned)p.layer,
+                                         ((unsigned)p.step << 1) | (unsigned)stream, p.seed_lo, p.seed_hi);
+          key[0] = rr.x; key[1] = rr.y; key[2] = rr.z; key[3] = rr.w;
+        }
+        unsigned bal[4], total = 0u;
+        bool hit[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int tok = t0 + e;
+          hit[e] = key[e] < bound && tok >= geo.s0 && tok < geo.l_start;
+          bal[e] = __ballot_sync(0xFFFFFFFFu, hit[e]) & lmask;
+          total += __popc(bal[e]);
+        }
+        unsigned base = 0u;
+        if ((lane & 3) == 0 && total) base = atomicAdd(&s_cnt[L], total);
+        base = __shfl_sync(0xFFFFFFFFu, base, lane & ~3);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned pos = base + __popc(bal[e] & lt);
+          if (hit[e] && pos < (unsigned)CL) clist[L * CL + pos] = make_uint2(key[e], (unsigned)(t0 + e));
+          base += __popc(bal[e]);
+        }
+      }
+    }
+    cand_barrier();
+    // flush: candidate warp cw owns lists cw and cw + CWARPS
+    for (int L = cw; L < 2 * nh; L += CWARPS) {
+      const unsigned raw = s_cnt[L];
+      const unsigned cnt = raw < (unsigned)CL ? raw : (unsigned)CL;
+      if (raw == 0u) continue;
+      const long long slot_g = (long long)(L / nh) * p.B * p.Hq + (long long)b * p.Hq + h0 + (L % nh);
+      unsigned gbase = 0u;
+      // a list that overflowed its staging area is incomplete: poison the global count so that the select
+      // kernels draw from the full context instead
+      if (lane == 0) {
+        if (raw > (unsigned)CL) { atomicOr(&p.cand_cnt[slot_g], 0x80000000u); gbase = (unsigned)p.cand_cap; }
+        else gbase = atomicAdd(&p.cand_cnt[slot_g], cnt);
+      }
+      gbase = __shfl_sync(0xFFFFFFFFu, gbase, 0);
+      uint2* dst = p.cand + slot_g * p.cand_cap;
+      for (unsigned j = lane; j < cnt; j += 32)
+        if (gbase + j < (unsigned)p.cand_cap) dst[gbase + j] = clist[L * CL + j];
+      __syncwarp();
+      if (lane == 0) s_cnt[L] = 0u;
+    }
+    cand_barrier();
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Prob p) {
+  constexpr int NC = D / 32;
+  constexpr int ROWB = D * 2;                 // bytes per row
+  constexpr int PAGEB = VATTN_BLOCK * ROWB;   // bytes per (page, KV head) slab
+  extern __shared__ __align__(128) unsigned char smem_dyn[];
+  const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int role = wid >= WARPS;              // warps 0..3 stream K, warps 4..11 pre-filter sampling keys
+  const int cw = wid - WARPS;                 // candidate warp index (role 1)
+  const int warp = role ? (cw & (WARPS - 1)) : wid;      // the streaming warp whose pages this warp works on
+  unsigned char* ring = smem_dyn + (size_t)warp * NST * PAGEB;
+  uint2* clist = reinterpret_cast<uint2*>(smem_dyn + (size_t)WARPS * NST * PAGEB);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)WARPS * NST * PAGEB +
+                                                                   (size_t)16 * CL * sizeof(uint2)) + warp * NST;
+  unsigned* s_cnt = reinterpret_cast<unsigned*>(smem_dyn + (size_t)WARPS * NST * PAGEB + (size_t)16 * CL * sizeof(uint2) +
+                                                (size_t)WARPS * NST * 8);
+  DEV_BEGIN(p, 1);
+  const int b = blockIdx.z;
+  const int n = clamped_len(p, b);
+  const int npages = (n + 15) >> 4;
+  const int GC = (p.G + 7) >> 3;
+  const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
+  const int gr = lane >> 2, t = lane & 3;
+  const int h0 = g * p.G + hc * 8;
+  const int nh = min(8, p.G - hc * 8);
+  const int wglob = blockIdx.x * WARPS + warp, wtot = gridDim.x * WARPS;
+  const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;    // pages this warp owns
+  if (role == 1) {
+#ifndef VATTN_EXP_NOCAND
+#ifdef VATTN_DEV_TIMING
+    if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 4] = dev_gtime();
+#endif
+    candidate_warps(p, b, g, h0, nh, n, blockIdx.x * WARPS, wtot, npages, cw, clist, s_cnt);
+#ifdef VATTN_DEV_TIMING
+    if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 5] = dev_gtime();
+    if (p.devt && lane == 0) atomicMax(&p.devt[32 + 6], dev_gtime());
+#endif
+#endif
+    return;
+  }
+  if (mine == 0) return;                      // streaming warps use no CTA-wide barrier
+#ifdef VATTN_EXP_NOSTREAM
+  return;
+#endif
+  const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
+
+  if (lane < NST) mbar_init(&bars[lane], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+
+  // page ids of this warp's first 32 pages (lane l holds the l-th); refreshed every 32 pages
+  int pg_ids = 0;
+  auto load_ids = [&](int k_base) {
+    const int k = k_base + lane;
+    pg_ids = (k < mine) ? page_of(p, b, wglob + k * wtot) : 0;
+  };
+  auto issue = [&](int k, int pg) {       // lane 0 only
+    unsigned long long* bar = &bars[k % NST];
+    unsigned char* dst = ring + (size_t)(k % NST) * PAGEB;
+    const bf16_t* src = kc + (long long)pg * p.sb + (long long)g * p.sh;
+    mbar_expect_tx(bar, PAGEB);
+    if (p.st == D) bulk_g2s(dst, src, PAGEB, bar);
+    else
+      for (int r = 0; r < VATTN_BLOCK; ++r) bulk_g2s(dst + r * ROWB, src + (long long)r * p.st, ROWB, bar);
+  };
+  load_ids(0);
+  for (int k = 0; k < min(NST, mine); ++k) {
+    const int pg = __shfl_sync(0xFFFFFFFFu, pg_ids, k);
+    if (lane == 0) issue(k, pg);
+  }
+
+  uint4 bq[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    bq[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (gr < nh)
+      bq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
+                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
+  }
+  float runmax[2] = {-INFINITY, -INFINITY};
+  unsigned kabs = 0u;
+  bool failed = false;
+
+  for (int k = 0; k < mine; ++k) {
+    const int s = k % NST;
+    if (!mbar_wait(&bars[s], (unsigned)(k / NST) & 1u)) { failed = true; break; }
+    const unsigned char* stg = ring + (size_t)s * PAGEB;
+    const int tok0 = (wglob + k * wtot) << 4;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    unsigned klo = 0u, khi = 0u;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const uint4 alo = *reinterpret_cast<const uint4*>(stg + gr * ROWB + c * 64 + t * 16);
+      const uint4 ahi = *reinterpret_cast<const uint4*>(stg + (gr + 8) * ROWB + c * 64 + t * 16);
+      mma_bf16_16816(acc, alo.x, ahi.x, alo.y, ahi.y, bq[c].x, bq[c].y);
+      mma_bf16_16816(acc, alo.z, ahi.z, alo.w, ahi.w, bq[c].z, bq[c].w);
+      klo = __vimax3_u16x2(klo, alo.x & 0x7FFF7FFFu, alo.y & 0x7FFF7FFFu);
+      klo = __vimax3_u16x2(klo, alo.z & 0x7FFF7FFFu, alo.w & 0x7FFF7FFFu);
+      khi = __vimax3_u16x2(khi, ahi.x & 0x7FFF7FFFu, ahi.y & 0x7FFF7FFFu);
+      khi = __vimax3_u16x2(khi, ahi.z & 0x7FFF7FFFu, ahi.w & 0x7FFF7FFFu);
+    }
+    // the stage has been read (the MMAs consumed every fragment): refill it with page k + NST
+    __syncwarp();
+    if (k + NST < mine) {
+      if (((k + NST) & 31) == 0) load_ids(k + NST);
+      const int pg = __shfl_sync(0xFFFFFFFFu, pg_ids, (k + NST) & 31);
+      if (lane == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        issue(k + NST, pg);
+      }
+    }
+    const int tk_lo = tok0 + gr, tk_hi = tok0 + gr + 8;
+    if (tk_lo < n) kabs = __vimax3_u16x2(kabs, klo, 0u);
+    if (tk_hi < n) kabs = __vimax3_u16x2(kabs, khi, 0u);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int hl = 2 * t + e;
+      if (hl < nh) {
+        float* dst = p.scores + ((long long)b * p.Hq + h0 + hl) * p.npad;
+        const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
+#ifdef VATTN_EXP_NOSTORE
+        if (tk_lo < n) { runmax[e] = fmaxf(runmax[e], s_lo); }
+        if (tk_hi < n) { runmax[e] = fmaxf(runmax[e], s_hi); }
+#else
+        if (tk_lo < n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
+        if (tk_hi < n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
+#endif
+      }
+    }
+  }
+  if (failed) {
+    // give the copies still in flight a bounded chance to land before the shared memory is released
+    if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+    for (int s = 0; s < NST; ++s) mbar_wait(&bars[s], 0u) || mbar_wait(&bars[s], 1u);
+    return;
+  }
+#pragma unroll
+  for (int mask = 4; mask < 32; mask <<= 1) {
+    runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
+    runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
+  }
+#pragma unroll
+  for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
+  if (lane < 4) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int hl = 2 * lane + e;
+      if (hl < nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[b * p.Hq + h0 + hl], ord_f32(runmax[e]));
+    }
+  }
+  if (lane == 0) {
+    const unsigned mx = max(kabs & 0xFFFFu, kabs >> 16);
+    atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);
+  }
+  DEV_END(p, 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// fp32 (and generic) CUDA-core path, up to 4 heads per CTA
 template <typename T, int D>
-__global__ void __launch_bounds__(WARPS * 32) k_score(const Prob p) {
+__global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
   constexpr int EPL = Elem<T>::EPL;
   constexpr int LPR = D / EPL;       // lanes per row
   constexpr int RPI = 32 / LPR;      // rows per warp instruction
   constexpr int ITERS = 16 / RPI;    // instructions per page
   constexpr int NV = ITERS * 4;      // partial sums per lane per page (4 heads)
+  __shared__ uint2 s_list[8][TILE];
+  __shared__ unsigned s_cnt[8];
 
   const int b = blockIdx.z;
   const int n = clamped_len(p, b);
@@ -114,19 +572,44 @@ __global__ void __launch_bounds__(WARPS * 32) k_score(const Prob p) {
     }
   }
   if (lane == 0) atomicMax(&p.kabsmax[b * p.Hkv + g], __float_as_uint(kmax));
+  emit_candidates<4>(p, b, g, g * p.G + hc * 4, min(4, p.G - hc * 4), tile0, n, s_list, s_cnt);
 }
 
 }  // namespace
 
+template <int D>
+static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
+  const size_t smem = (size_t)WARPS * NST * VATTN_BLOCK * D * 2 + (size_t)16 * CL * sizeof(uint2) +
+                      (size_t)WARPS * NST * 8 + 16 * sizeof(unsigned);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  // one wave of two CTAs per SM; a warp walks pages with stride (CTAs along x) * WARPS
+  const int groups = p.Hkv * ((p.G + 7) / 8) * p.B;
+  const int pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
+  int cx = (2 * 148 + groups - 1) / groups;
+  const int cx_max = (pages + WARPS - 1) / WARPS;
+  if (cx > cx_max) cx = cx_max;
+  if (cx < 1) cx = 1;
+  dim3 grid(cx, p.Hkv * ((p.G + 7) / 8), p.B), block((WARPS + CWARPS) * 32);
+  k_score_stream<D><<<grid, block, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_score(const Prob& p, cudaStream_t s) {
-  const int GC = (p.G + 3) / 4;
-  dim3 grid((p.max_seq_len + TILE - 1) / TILE, p.Hkv * GC, p.B), block(WARPS * 32);
+  dim3 block(WARPS * 32);
+  const int tiles = (p.max_seq_len + TILE - 1) / TILE;
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) k_score<bf16_t, 128><<<grid, block, 0, s>>>(p);
-    else k_score<bf16_t, 64><<<grid, block, 0, s>>>(p);
+    // rows must be 16-byte aligned for the bulk copies (any stride that is a multiple of 8 elements is)
+    if (p.D == 128) return launch_stream<128>(p, s);
+    return launch_stream<64>(p, s);
   } else {
-    if (p.D == 128) k_score<float, 128><<<grid, block, 0, s>>>(p);
-    else k_score<float, 64><<<grid, block, 0, s>>>(p);
+    dim3 grid(tiles, p.Hkv * ((p.G + 3) / 4), p.B);
+    if (p.D == 128) k_score_fma<float, 128><<<grid, block, 0, s>>>(p);
+    else k_score_fma<float, 64><<<grid, block, 0, s>>>(p);
   }
   return cudaGetLastError();
 }

@@ -9,39 +9,65 @@
 // keys held in shared memory, followed by an ordered compaction through bitmaps, so every list comes
 // out ascending.  Keys are the order-reversed score for top-k and Philox4x32-10 words for sampling.
 //
+// Fast paths (one pass over the context instead of four): the top-k threshold is first estimated from a
+// strided sample of the scores (1024 linear bins between the sample minimum and the head maximum), one
+// pass collects the few thousand tokens above the estimate, and the exact radix select runs on those
+// candidates only.  Sampling draws from the candidate lists the score kernel pre-filtered (tokens whose
+// Philox key is below a bound): if the list holds at least c residual tokens, the c smallest keys of
+// the residual are all in it.  Whenever an estimate fails (too few / too many candidates, list
+// overflow, near-tie band reaching below the estimate) the generic full-context select runs instead.
+//
 // Exact top-k from fp32 scores: the stored scores differ from the exact inner products by at most
 // gamma (a bound from the summation structure of the score kernel).  After the fp32 threshold T is
 // known, tokens above T + 2*gamma are certainly selected and tokens below T - 2*gamma certainly not;
 // the few in between are rescored in fp64 from their K rows and ranked exactly.
 #include "vattn_internal.cuh"
 
+#ifdef VATTN_DEV_TIMING
+__device__ long long g_phase_clk[64][16];
+#define PHASE(i) do { __syncthreads(); if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.x < 64) g_phase_clk[blockIdx.x][i] = clock64(); } while (0)
+extern "C" int vattn_dev_read_phases(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_phase_clk, sizeof(long long) * 64 * 16); }
+#else
+#define PHASE(i) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int NT = SEL_THREADS;
 constexpr int NWARP = NT / 32;
 
+constexpr int CANDCAP = 4096;      // top-k candidates kept by the fast path
+constexpr int NBIN = 1024;          // linear bins of the threshold estimate (one per thread)
+constexpr int PAIRCAP0 = 4096;      // base-sample candidate pairs staged in shared memory
+
 struct Sm {
   double* band_s;     // [BANDCAP]
-  unsigned* keys;     // [keycap]
+  unsigned* keys;     // [bigbytes/4] select keys of the context, or staged (key, token) pairs
   unsigned* w0;       // [nwords] selected / "less than threshold" bitmap
   unsigned* w1;       // [nwords] "equal to threshold" / band bitmap
   unsigned* w2;       // [nwords] I_t bitmap (residual mask) / scratch
   int* scan;          // [nwords]
   unsigned* hist;     // [256]
   int* band_idx;      // [BANDCAP]
+  int* lin;           // [NBIN]
+  int* cand_idx;      // [CANDCAP]
+  unsigned* ckey;     // [CANDCAP] select keys of the candidates
   int* misc;          // [64]
 };
 
-__device__ __forceinline__ Sm carve(unsigned char* base, int keycap, int nwords) {
+__device__ __forceinline__ Sm carve(unsigned char* base, int bigbytes, int nwords) {
   Sm s;
   s.band_s = reinterpret_cast<double*>(base);            base += sizeof(double) * VATTN_BANDCAP;
-  s.keys = reinterpret_cast<unsigned*>(base);            base += sizeof(unsigned) * (size_t)keycap;
+  s.keys = reinterpret_cast<unsigned*>(base);            base += (size_t)bigbytes;
   s.w0 = reinterpret_cast<unsigned*>(base);              base += sizeof(unsigned) * (size_t)nwords;
   s.w1 = reinterpret_cast<unsigned*>(base);              base += sizeof(unsigned) * (size_t)nwords;
   s.w2 = reinterpret_cast<unsigned*>(base);              base += sizeof(unsigned) * (size_t)nwords;
   s.scan = reinterpret_cast<int*>(base);                 base += sizeof(int) * (size_t)nwords;
   s.hist = reinterpret_cast<unsigned*>(base);            base += sizeof(unsigned) * 256;
   s.band_idx = reinterpret_cast<int*>(base);             base += sizeof(int) * VATTN_BANDCAP;
+  s.lin = reinterpret_cast<int*>(base);                  base += sizeof(int) * NBIN;
+  s.cand_idx = reinterpret_cast<int*>(base);             base += sizeof(int) * CANDCAP;
+  s.ckey = reinterpret_cast<unsigned*>(base);            base += sizeof(unsigned) * CANDCAP;
   s.misc = reinterpret_cast<int*>(base);
   return s;
 }
@@ -247,6 +273,7 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
   }
   if (CACHED) fill_philox_keys(p, sm.keys, lo, hi, b, hrng, stream);
   __syncthreads();
+  PHASE(5);
   auto keyfn = [&](int i, unsigned& key) -> bool {
     if ((it[i >> 5] >> (i & 31)) & 1u) return false;
     key = CACHED ? sm.keys[i] : philox_key_of(p, i, b, hrng, stream);
@@ -254,6 +281,7 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
   };
   unsigned T; int need_eq;
   block_select<unsigned, false>(keyfn, lo, hi, c, sm.hist, sm.misc, T, need_eq);
+  PHASE(6);
   for (int w = warp; w < nw; w += NWARP) {
     const int i = w * 32 + lane;
     unsigned key = 0;
@@ -264,41 +292,380 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
     if (lane == 0) { sm.w0[w] = lt; sm.w1[w] = eq; }
   }
   __syncthreads();
+  PHASE(7);
   return finalize_emit(sm.w0, sm.w1, need_eq, nw, sm.scan, sm.misc, out_a, out_b);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Sampling from a pre-filtered candidate list: `cnt` (key, token) pairs in global memory whose keys
+// are below `bound`.  Succeeds (returns the number emitted, = c) when the list is complete and holds
+// at least c residual tokens; returns -1 when the caller has to draw from the full context.
+// The c-th smallest (key, token) pair is located with one linear-bin histogram over [0, bound) (the
+// keys are uniform, so a bin holds a handful of pairs) and an exact ranking inside that bin.
+__device__ int sample_from_candidates(const Prob& p, const Sm& sm, const uint2* glist, unsigned cnt, int paircap,
+                                      unsigned bound, int c, int nw, const unsigned* it, int* out_a, int* out_b) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (bound == 0u || cnt > (unsigned)p.cand_cap || cnt > (unsigned)paircap || (int)cnt < c) return -1;
+  uint2* pr = reinterpret_cast<uint2*>(sm.keys);
+  int* misc = sm.misc;
+  const float bscale = (float)NBIN / (float)bound;
+  auto bin_of = [&](unsigned key) -> int { const int x = (int)((float)key * bscale); return x > NBIN - 1 ? NBIN - 1 : x; };
+  sm.lin[tid] = 0;
+  if (tid == 0) { misc[2] = 0; misc[3] = 0; misc[4] = -1; }
+  __syncthreads();
+  int nvalid_local = 0;
+  for (int j = tid; j < (int)cnt; j += NT) {
+    uint2 e = glist[j];
+    const bool resid = !((it[e.y >> 5] >> (e.y & 31)) & 1u);
+    if (!resid) e.y |= 0x80000000u;                         // tokens of I_t stay in the list, marked
+    else atomicAdd(&sm.lin[bin_of(e.x)], 1);
+    pr[j] = e;
+    nvalid_local += resid;
+  }
+#pragma unroll
+  for (int mk = 16; mk >= 1; mk >>= 1) nvalid_local += __shfl_xor_sync(0xFFFFFFFFu, nvalid_local, mk);
+  if (lane == 0 && nvalid_local) atomicAdd(&misc[2], nvalid_local);
+  __syncthreads();
+  DEV_MARK(p, 6, 2, blockIdx.x == 0 && blockIdx.y == 0);
+  if (misc[2] < c) return -1;
+  const int mycnt = sm.lin[tid];
+  __syncthreads();
+  block_excl_scan(sm.lin, NBIN, misc);
+  const int excl = sm.lin[tid];
+  if (excl < c && c <= excl + mycnt) { misc[4] = tid; misc[5] = c - excl; }
+  __syncthreads();
+  const int jb = misc[4], r_in = misc[5];                   // the c-th smallest pair is the r_in-th of bin jb
+  DEV_MARK(p, 6, 3, blockIdx.x == 0 && blockIdx.y == 0);
+  for (int w = tid; w < nw; w += NT) sm.w0[w] = 0u;
+  for (int j = tid; j < (int)cnt; j += NT) {
+    const uint2 e = pr[j];
+    if ((e.y & 0x80000000u) || bin_of(e.x) != jb) continue;
+    const int pos = atomicAdd(&misc[3], 1);
+    if (pos < VATTN_BANDCAP) { sm.band_idx[pos] = j; }
+  }
+  __syncthreads();
+  const int nmem = misc[3];
+  if (nmem > VATTN_BANDCAP) return -1;
+  for (int a = tid; a < nmem; a += NT) {
+    const uint2 mine = pr[sm.band_idx[a]];
+    int rank = 0;
+    for (int u = 0; u < nmem; ++u) {
+      const uint2 o = pr[sm.band_idx[u]];
+      rank += (o.x < mine.x) || (o.x == mine.x && o.y < mine.y);
+    }
+    if (rank == r_in - 1) { misc[6] = (int)mine.x; misc[7] = (int)mine.y; }
+  }
+  __syncthreads();
+  const unsigned Tkey = (unsigned)misc[6], Tidx = (unsigned)misc[7];
+  DEV_MARK(p, 6, 4, blockIdx.x == 0 && blockIdx.y == 0);
+  for (int j = tid; j < (int)cnt; j += NT) {
+    const uint2 e = pr[j];
+    if (e.y & 0x80000000u) continue;
+    if (e.x < Tkey || (e.x == Tkey && e.y <= Tidx)) atomicOr(&sm.w0[e.y >> 5], 1u << (e.y & 31));
+  }
+  __syncthreads();
+  DEV_MARK(p, 6, 5, blockIdx.x == 0 && blockIdx.y == 0);
+  const int got = finalize_emit(sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
+  DEV_MARK(p, 6, 6, blockIdx.x == 0 && blockIdx.y == 0);
+  return got;
+}
+
+// ---------------------------------------------------------------------------------------------
+// top-k, fast path: requires the inverted ordered score keys of [s0, l_start) in sm.keys.
+//  1. a strided sample of the scores is binned linearly between its minimum and the head maximum; the
+//     bin edge below which about kk + margin tokens are expected becomes the candidate threshold U;
+//  2. one pass collects the tokens with score >= U (each thread keeps a 32-bit take mask, positions
+//     come from one block scan: no atomics in the loop);
+//  3. the kk-th largest candidate is located by a second linear-bin histogram over [U, m] and an exact
+//     ranking inside its bin;
+//  4. candidates above T + 2 gamma are members, those within 2 gamma are rescored in fp64.
+// On success the bitmap of I_t is in sm.w0.  Returns false (sm.w0 / sm.w1 undefined) when the generic
+// path has to run.
+template <typename T, int D>
+__device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qrow, int s0, int l_start, int kk,
+                          int nw, float m, float gamma) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int mlen = l_start - s0;
+  int* misc = sm.misc;
+  float* fmisc = reinterpret_cast<float*>(misc);
+  float U = -INFINITY;              // candidates are the tokens with score >= U
+  int ncand = 0;
+  if (tid == 0) { misc[2] = NBIN; misc[4] = 0; misc[5] = 0; misc[6] = -1; }
+  if (mlen <= CANDCAP) {
+    for (int j = tid; j < mlen; j += NT) { sm.cand_idx[j] = s0 + j; sm.ckey[j] = sm.keys[s0 + j]; }
+    ncand = mlen;
+    __syncthreads();
+  } else {
+    constexpr int SAMPLE = 2048;
+    const int stride = (mlen + SAMPLE - 1) / SAMPLE;
+    const int ms = (mlen + stride - 1) / stride;
+    float smin = (tid < ms) ? unord_f32(~sm.keys[s0 + tid * stride]) : INFINITY;
+#pragma unroll
+    for (int mk = 16; mk >= 1; mk >>= 1) smin = fminf(smin, __shfl_xor_sync(0xFFFFFFFFu, smin, mk));
+    sm.lin[tid] = 0;
+    if (lane == 0) fmisc[8 + warp] = smin;
+    __syncthreads();
+    smin = fmisc[8 + lane];
+#pragma unroll
+    for (int mk = 16; mk >= 1; mk >>= 1) smin = fminf(smin, __shfl_xor_sync(0xFFFFFFFFu, smin, mk));
+    const float range = m - smin;
+    const float inv_w = (range > 0.f) ? (float)NBIN / range : 0.f;
+    for (int j = tid; j < ms; j += NT) {
+      const float x = (m - unord_f32(~sm.keys[s0 + j * stride])) * inv_w;
+      atomicAdd(&sm.lin[x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0)], 1);
+    }
+    __syncthreads();
+    const int cnt = sm.lin[tid];
+    __syncthreads();
+    block_excl_scan(sm.lin, NBIN, misc);
+    const double fms = (double)kk * (double)ms / (double)mlen;
+    const int r = (int)(fms + 4.0 * sqrt(fms) + 8.0);
+    const int excl = sm.lin[tid];
+    if (excl < r && r <= excl + cnt) misc[2] = tid;
+    __syncthreads();
+    const int jstar = misc[2];
+    if (jstar >= NBIN - 1) return false;                      // the sample cannot place the threshold
+    DEV_MARK(p, 2, 10, blockIdx.x == 0 && blockIdx.y == 0);
+    U = m - (float)(jstar + 1) * (range / (float)NBIN);
+    if (U == 0.f) U = -0.f;                                   // both zeros must pass the key comparison
+    const unsigned Ukey = ~ord_f32(U);                        // score >= U  <=>  key <= Ukey
+    // one pass over the context: 32 tokens per thread, take mask in a register
+    unsigned take = 0u;
+    const int base_i = s0 + tid;
+#pragma unroll 8
+    for (int it = 0; it < 32; ++it) {
+      const int i = base_i + it * NT;
+      if (i < l_start && sm.keys[i] <= Ukey) take |= 1u << it;
+    }
+    for (int it = 32; base_i + it * NT < l_start; ++it) {     // contexts longer than 32 * NT tokens
+      if (sm.keys[base_i + it * NT] <= Ukey) { misc[6] = -2; }
+    }
+    __syncthreads();
+    sm.lin[tid] = __popc(take);
+    __syncthreads();
+    ncand = block_excl_scan(sm.lin, NBIN, misc);
+    if (misc[6] == -2 || ncand < kk || ncand > CANDCAP) return false;
+    int pos = sm.lin[tid];
+    while (take) {
+      const int it = __ffs(take) - 1;
+      take &= take - 1;
+      const int i = base_i + it * NT;
+      sm.cand_idx[pos] = i;
+      sm.ckey[pos] = sm.keys[i];
+      ++pos;
+    }
+    __syncthreads();
+  }
+  DEV_MARK(p, 2, 11, blockIdx.x == 0 && blockIdx.y == 0);
+  // ---- the kk-th largest candidate: linear bins over [cmin, m], exact ranking inside the bin
+  float cmin = INFINITY;
+  for (int j = tid; j < ncand; j += NT) cmin = fminf(cmin, unord_f32(~sm.ckey[j]));
+#pragma unroll
+  for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
+  sm.lin[tid] = 0;
+  if (lane == 0) fmisc[8 + warp] = cmin;
+  __syncthreads();
+  cmin = fmisc[8 + lane];
+#pragma unroll
+  for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
+  const float range2 = m - cmin;
+  const float inv_w2 = (range2 > 0.f) ? (float)NBIN / range2 : 0.f;
+  auto bin2 = [&](unsigned key) -> int {
+    const float x = (m - unord_f32(~key)) * inv_w2;
+    return x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0);
+  };
+  for (int j = tid; j < ncand; j += NT) atomicAdd(&sm.lin[bin2(sm.ckey[j])], 1);
+  __syncthreads();
+  const int cnt2 = sm.lin[tid];
+  __syncthreads();
+  block_excl_scan(sm.lin, NBIN, misc);
+  {
+    const int excl = sm.lin[tid];
+    if (excl < kk && kk <= excl + cnt2) { misc[6] = tid; misc[7] = kk - excl; }
+  }
+  __syncthreads();
+  const int jb = misc[6], r_in = misc[7];
+  if (jb < 0) return false;
+  for (int j = tid; j < ncand; j += NT) {
+    if (bin2(sm.ckey[j]) == jb) {
+      const int pos = atomicAdd(&misc[4], 1);
+      if (pos < VATTN_BANDCAP) sm.band_idx[pos] = j;
+    }
+  }
+  __syncthreads();
+  const int nmem = misc[4];
+  if (nmem > VATTN_BANDCAP) return false;
+  for (int a = tid; a < nmem; a += NT) {                      // r_in-th largest score of the bin (value only)
+    const unsigned mine = sm.ckey[sm.band_idx[a]];
+    int less = 0, leq = 0;                                    // inverted keys: smaller key = larger score
+    for (int u = 0; u < nmem; ++u) {
+      const unsigned o = sm.ckey[sm.band_idx[u]];
+      less += o < mine;
+      leq += o <= mine;
+    }
+    if (less < r_in && r_in <= leq) misc[3] = (int)mine;      // all writers hold the same key
+  }
+  __syncthreads();
+  const unsigned Tk = (unsigned)misc[3];
+  DEV_MARK(p, 2, 12, blockIdx.x == 0 && blockIdx.y == 0);
+  const float Tf = unord_f32(~Tk);
+  const float hi = __fadd_ru(Tf, 2.f * gamma), lo = __fadd_rd(Tf, -2.f * gamma);
+  // every token that could still enter the top-k (score >= lo) must be a candidate
+  if (!(lo >= U)) return false;
+  for (int w = tid; w < nw; w += NT) sm.w0[w] = 0u;
+  if (tid == 0) { misc[4] = 0; misc[5] = 0; }
+  __syncthreads();
+  int in_local = 0;
+  for (int j = tid; j < ncand; j += NT) {
+    const int idx = sm.cand_idx[j];
+    const float s = unord_f32(~sm.ckey[j]);
+    if (s > hi) { atomicOr(&sm.w0[idx >> 5], 1u << (idx & 31)); ++in_local; }
+    else if (s >= lo) {
+      const int pos = atomicAdd(&misc[5], 1);
+      if (pos < VATTN_BANDCAP) sm.band_idx[pos] = idx;
+    }
+  }
+#pragma unroll
+  for (int mk = 16; mk >= 1; mk >>= 1) in_local += __shfl_xor_sync(0xFFFFFFFFu, in_local, mk);
+  if (lane == 0 && in_local) atomicAdd(&misc[4], in_local);
+  __syncthreads();
+  const int n_in = misc[4], n_band = misc[5];
+  const int need = kk - n_in;
+  if (n_band > VATTN_BANDCAP) return false;
+  if (need >= n_band) {
+    for (int c = tid; c < n_band; c += NT) { const int idx = sm.band_idx[c]; atomicOr(&sm.w0[idx >> 5], 1u << (idx & 31)); }
+  } else {
+    for (int c = warp; c < n_band; c += NWARP) {
+      const double s64 = score64_warp<T, D>(p, b, g, qrow, sm.band_idx[c]);
+      if (lane == 0) sm.band_s[c] = s64;
+    }
+    __syncthreads();
+    for (int c = tid; c < n_band; c += NT) {
+      const double mine = sm.band_s[c];
+      const int mi = sm.band_idx[c];
+      int rank = 0;
+      for (int u = 0; u < n_band; ++u) {
+        const double o = sm.band_s[u];
+        rank += (o > mine) || (o == mine && sm.band_idx[u] < mi);
+      }
+      if (rank < need) atomicOr(&sm.w0[mi >> 5], 1u << (mi & 31));
+    }
+  }
+  __syncthreads();
+  return true;
+}
+
+// top-k, generic path: radix select over the whole middle range (any size, any score distribution)
 template <typename T, int D, bool CACHED>
-__global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int keycap) {
+__device__ void topk_generic(const Prob& p, const Sm& sm, int b, int g, const T* qrow, const float* sc, int s0,
+                             int l_start, int kk, int nw, float gamma) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  auto keyfn = [&](int i, unsigned& key) -> bool { key = CACHED ? sm.keys[i] : ~ord_f32(sc[i]); return true; };
+  unsigned Tk; int need_eq;
+  block_select<unsigned, true>(keyfn, s0, l_start, kk, sm.hist, sm.misc, Tk, need_eq);
+  const float Tf = unord_f32(~Tk);
+  const float hi = __fadd_ru(Tf, 2.f * gamma), lo = __fadd_rd(Tf, -2.f * gamma);
+  // certain members -> w0, near-tie band -> w1
+  for (int w = warp; w < nw; w += NWARP) {
+    const int i = w * 32 + lane;
+    const bool ok = (i >= s0) && (i < l_start);
+    const float s = ok ? (CACHED ? unord_f32(~sm.keys[i]) : sc[i]) : 0.f;
+    const unsigned in = __ballot_sync(0xFFFFFFFFu, ok && s > hi);
+    const unsigned band = __ballot_sync(0xFFFFFFFFu, ok && !(s > hi) && s >= lo);
+    if (lane == 0) { sm.w0[w] = in; sm.w1[w] = band; }
+  }
+  __syncthreads();
+  for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w0[w]);
+  __syncthreads();
+  const int n_in = block_excl_scan(sm.scan, nw, sm.misc);
+  for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w1[w]);
+  __syncthreads();
+  const int n_band = block_excl_scan(sm.scan, nw, sm.misc);      // scan[w] = rank of word w's first band bit
+  const int need = kk - n_in;                                     // 1 <= need <= n_band
+  if (need >= n_band) {
+    for (int w = tid; w < nw; w += NT) sm.w0[w] |= sm.w1[w];
+    __syncthreads();
+  } else if (n_band <= VATTN_BANDCAP) {
+    // band list ascending by index, exact scores, O(band^2) ranking by (-score, index)
+    for (int w = tid; w < nw; w += NT) {
+      unsigned bits = sm.w1[w];
+      int pos = sm.scan[w];
+      while (bits) { const int bit = __ffs(bits) - 1; bits &= bits - 1; sm.band_idx[pos++] = w * 32 + bit; }
+    }
+    __syncthreads();
+    for (int c = warp; c < n_band; c += NWARP) {
+      const double s64 = score64_warp<T, D>(p, b, g, qrow, sm.band_idx[c]);
+      if (lane == 0) sm.band_s[c] = s64;
+    }
+    __syncthreads();
+    for (int c = tid; c < n_band; c += NT) {
+      const double mine = sm.band_s[c];
+      int rank = 0;
+      for (int u = 0; u < n_band; ++u) {
+        const double o = sm.band_s[u];
+        rank += (o > mine) || (o == mine && u < c);
+      }
+      if (rank < need) { const int idx = sm.band_idx[c]; atomicOr(&sm.w0[idx >> 5], 1u << (idx & 31)); }
+    }
+    __syncthreads();
+  } else {
+    // too many near-ties for the list: exact 64-bit radix select over the band, scores recomputed on the fly
+    if (tid == 0) atomicOr(p.status, VATTN_STATUS_BAND_OVERFLOW);
+    auto key64 = [&](int i, unsigned long long& key) -> bool {
+      if (!((sm.w1[i >> 5] >> (i & 31)) & 1u)) return false;
+      key = ~ord_f64(score64_thread<T, D>(p, b, g, qrow, i));
+      return true;
+    };
+    unsigned long long T64; int need_eq64;
+    block_select<unsigned long long, true>(key64, s0, l_start, need, sm.hist, sm.misc, T64, need_eq64);
+    for (int w = warp; w < nw; w += NWARP) {
+      const int i = w * 32 + lane;
+      unsigned long long key = 0;
+      bool ok = (i >= s0) && (i < l_start);
+      if (ok) ok = key64(i, key);
+      const unsigned lt = __ballot_sync(0xFFFFFFFFu, ok && key < T64);
+      const unsigned eq = __ballot_sync(0xFFFFFFFFu, ok && key == T64);
+      if (lane == 0) { sm.w0[w] |= lt; sm.w2[w] = eq; }
+    }
+    __syncthreads();
+    for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w2[w]);
+    __syncthreads();
+    block_excl_scan(sm.scan, nw, sm.misc);
+    for (int w = tid; w < nw; w += NT) sm.w0[w] |= lowest_bits(sm.w2[w], need_eq64 - sm.scan[w]);
+    __syncthreads();
+  }
+}
+
+template <typename T, int D, bool CACHED>
+__global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bigbytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
-  const Sm sm = carve(smem_raw, keycap, p.nwords);
+  DEV_BEGIN(p, 2);
+  const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
 
   const int n = clamped_len(p, b);
-  const int s0 = min(p.sink, n);
-  const int l_start = max(n - p.window, s0);
+  const Geo geo = head_geometry(p, n);
+  const int s0 = geo.s0, l_start = geo.l_start, kk = geo.kk, n_s = geo.n_s, b0 = geo.b0;
   const int mlen = l_start - s0;
-  int kb = p.k;
-  if (p.topk_frac > 0.f) kb = (int)floor((double)p.topk_frac * (double)n);
-  const int kk = min(kb, mlen);
-  const int n_s = mlen - kk;
-  int b0 = 0;
-  if (n_s > 0) b0 = min(n_s, max(2, (int)floor((double)p.base_rate * (double)n_s)));
   const int nw = (n + 31) >> 5;
   const T* qrow = reinterpret_cast<const T*>(p.q) + (long long)bh * D;
   const float* sc = p.scores + (long long)bh * p.npad;
   const float m = (n > 0) ? unord_f32(p.m_ord[bh]) : 0.f;
 
-  // gamma: bound on |fp32 score - exact score| (13 roundings, see the score kernel)
+  // gamma: bound on |fp32 score - exact score|.  fp32 path: at most 13 roundings (x16 = margin).
+  // bf16 tensor-core path: 8 accumulation steps of 16 exact products each, every step assumed to lose
+  // up to 17 units of 2^-23 of the running magnitude (truncating adder) -> 8*17*2 = 272, taken as 512.
   if (warp == 0) {
     double sa = 0.0;
     for (int e = lane; e < D; e += 32) sa += fabs((double)Elem<T>::to_float(qrow[e]));
 #pragma unroll
     for (int mk = 16; mk >= 1; mk >>= 1) sa += __shfl_xor_sync(0xFFFFFFFFu, sa, mk);
     const double kmax = (double)__uint_as_float(p.kabsmax[b * p.Hkv + g]);
-    const double gm = 16.0 * 5.9604644775390625e-8 * fabs((double)p.scale) * sa * kmax * 1.000001;
+    const double roundings = (p.dtype == VATTN_DTYPE_BF16) ? 512.0 : 16.0;
+    const double gm = roundings * 5.9604644775390625e-8 * fabs((double)p.scale) * sa * kmax * 1.000001;
     if (lane == 0) reinterpret_cast<float*>(sm.misc)[48] = __double2float_ru(gm);
   }
   __syncthreads();
@@ -310,8 +677,11 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int ke
     if (p.dbg.base_cnt) p.dbg.base_cnt[bh] = b0;
   }
   unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
-  if (n == 0) return;
+  if (n == 0) { if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = 0; return; }
+  PHASE(0);
+  DEV_MARK(p, 2, 2, bh == 0);
 
+  int path = 0;
   // ------------------------------------------------------------------ top-k over the middle range
   for (int w = tid; w < nw; w += NT) { sm.w0[w] = 0u; sm.w1[w] = 0u; }
   __syncthreads();
@@ -325,85 +695,25 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int ke
     }
     __syncthreads();
   } else if (kk > 0) {
+    bool done = false;
     if (CACHED) {
       for (int i = s0 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(sc[i]);
       __syncthreads();
+      PHASE(1);
+      DEV_MARK(p, 2, 3, bh == 0);
+      done = topk_fast<T, D>(p, sm, b, g, qrow, s0, l_start, kk, nw, m, gamma);
+      PHASE(2);
+      DEV_MARK(p, 2, 4, bh == 0);
+      if (done) path |= 1;
     }
-    auto keyfn = [&](int i, unsigned& key) -> bool { key = CACHED ? sm.keys[i] : ~ord_f32(sc[i]); return true; };
-    unsigned Tk; int need_eq;
-    block_select<unsigned, true>(keyfn, s0, l_start, kk, sm.hist, sm.misc, Tk, need_eq);
-    const float Tf = unord_f32(~Tk);
-    const float hi = __fadd_ru(Tf, 2.f * gamma), lo = __fadd_rd(Tf, -2.f * gamma);
-    // certain members -> w0, near-tie band -> w1
-    for (int w = warp; w < nw; w += NWARP) {
-      const int i = w * 32 + lane;
-      const bool ok = (i >= s0) && (i < l_start);
-      const float s = ok ? (CACHED ? unord_f32(~sm.keys[i]) : sc[i]) : 0.f;
-      const unsigned in = __ballot_sync(0xFFFFFFFFu, ok && s > hi);
-      const unsigned band = __ballot_sync(0xFFFFFFFFu, ok && !(s > hi) && s >= lo);
-      if (lane == 0) { sm.w0[w] = in; sm.w1[w] = band; }
-    }
-    __syncthreads();
-    for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w0[w]);
-    __syncthreads();
-    const int n_in = block_excl_scan(sm.scan, nw, sm.misc);
-    for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w1[w]);
-    __syncthreads();
-    const int n_band = block_excl_scan(sm.scan, nw, sm.misc);      // scan[w] = rank of word w's first band bit
-    const int need = kk - n_in;                                     // 1 <= need <= n_band
-    if (need >= n_band) {
-      for (int w = tid; w < nw; w += NT) sm.w0[w] |= sm.w1[w];
+    if (!done) {
       __syncthreads();
-    } else if (n_band <= VATTN_BANDCAP) {
-      // band list ascending by index, exact scores, O(band^2) ranking by (-score, index)
-      for (int w = tid; w < nw; w += NT) {
-        unsigned bits = sm.w1[w];
-        int pos = sm.scan[w];
-        while (bits) { const int bit = __ffs(bits) - 1; bits &= bits - 1; sm.band_idx[pos++] = w * 32 + bit; }
-      }
+      for (int w = tid; w < nw; w += NT) { sm.w0[w] = 0u; sm.w1[w] = 0u; }
       __syncthreads();
-      for (int c = warp; c < n_band; c += NWARP) {
-        const double s64 = score64_warp<T, D>(p, b, g, qrow, sm.band_idx[c]);
-        if (lane == 0) sm.band_s[c] = s64;
-      }
-      __syncthreads();
-      for (int c = tid; c < n_band; c += NT) {
-        const double mine = sm.band_s[c];
-        int rank = 0;
-        for (int u = 0; u < n_band; ++u) {
-          const double o = sm.band_s[u];
-          rank += (o > mine) || (o == mine && u < c);
-        }
-        if (rank < need) { const int idx = sm.band_idx[c]; atomicOr(&sm.w0[idx >> 5], 1u << (idx & 31)); }
-      }
-      __syncthreads();
-    } else {
-      // too many near-ties for the list: exact 64-bit radix select over the band, scores recomputed on the fly
-      if (tid == 0) atomicOr(p.status, VATTN_STATUS_BAND_OVERFLOW);
-      auto key64 = [&](int i, unsigned long long& key) -> bool {
-        if (!((sm.w1[i >> 5] >> (i & 31)) & 1u)) return false;
-        key = ~ord_f64(score64_thread<T, D>(p, b, g, qrow, i));
-        return true;
-      };
-      unsigned long long T64; int need_eq64;
-      block_select<unsigned long long, true>(key64, s0, l_start, need, sm.hist, sm.misc, T64, need_eq64);
-      for (int w = warp; w < nw; w += NWARP) {
-        const int i = w * 32 + lane;
-        unsigned long long key = 0;
-        bool ok = (i >= s0) && (i < l_start);
-        if (ok) ok = key64(i, key);
-        const unsigned lt = __ballot_sync(0xFFFFFFFFu, ok && key < T64);
-        const unsigned eq = __ballot_sync(0xFFFFFFFFu, ok && key == T64);
-        if (lane == 0) { sm.w0[w] |= lt; sm.w2[w] = eq; }
-      }
-      __syncthreads();
-      for (int w = tid; w < nw; w += NT) sm.scan[w] = __popc(sm.w2[w]);
-      __syncthreads();
-      block_excl_scan(sm.scan, nw, sm.misc);
-      for (int w = tid; w < nw; w += NT) sm.w0[w] |= lowest_bits(sm.w2[w], need_eq64 - sm.scan[w]);
-      __syncthreads();
+      topk_generic<T, D, CACHED>(p, sm, b, g, qrow, sc, s0, l_start, kk, nw, gamma);
     }
   }
+  PHASE(3);
   // emit I_t ascending, keep its bitmap (shared w2 + global)
   int* tk_out = p.topk_idx + (long long)bh * p.npad;
   int* tk_dbg = p.dbg.topk_idx ? p.dbg.topk_idx + (long long)bh * p.max_seq_len : nullptr;
@@ -414,21 +724,34 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int ke
     gbitmap[w] = v;
   }
   __syncthreads();
+  PHASE(4);
+  DEV_MARK(p, 2, 5, bh == 0);
 
   // ------------------------------------------------------------------ base sample (Philox stream 0)
   const int hrng = p.rng_head_is_kv ? g : h;
   int* bs_out = p.base_idx + (long long)bh * p.npad;
   int* bs_dbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
-  sample_select<CACHED>(p, sm, s0, l_start, nw, b0, n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
+  int got = -1;
+  if (b0 > 0 && b0 < n_s)
+    got = sample_from_candidates(p, sm, p.cand + (long long)bh * p.cand_cap, p.cand_cnt[bh], bigbytes / 8,
+                                 cand0_bound(geo), b0, nw, sm.w2, bs_out, bs_dbg);
+  if (got < 0) {
+    __syncthreads();
+    sample_select<CACHED>(p, sm, s0, l_start, nw, b0, n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
+  } else path |= 2;
+  if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = path;
+  PHASE(8);
+  DEV_END(p, 2);
 }
 
 template <bool CACHED>
-__global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int keycap) {
+__global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
-  const Sm sm = carve(smem_raw, keycap, p.nwords);
+  DEV_BEGIN(p, 4);
+  const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   const HeadMeta meta = p.meta[bh];
   if (p.dbg.dyn_cnt && tid == 0) p.dbg.dyn_cnt[bh] = meta.b;
   if (meta.n == 0 || meta.b <= 0) return;
@@ -436,26 +759,50 @@ __global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int keycap
   const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
   for (int w = tid; w < nw; w += NT) sm.w2[w] = gbitmap[w];
   __syncthreads();
+  DEV_MARK(p, 4, 2, bh == 0);
   const int hrng = p.rng_head_is_kv ? g : h;
   int* out = p.dyn_idx + (long long)bh * p.npad;
   int* dbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)bh * p.max_seq_len : nullptr;
-  sample_select<CACHED>(p, sm, meta.s0, meta.l_start, nw, meta.b, meta.n_s, b, hrng, 1, sm.w2, out, dbg);
+  int got = -1;
+  if (meta.b < meta.n_s) {
+    const long long l1 = (long long)p.B * p.Hq + bh;
+    got = sample_from_candidates(p, sm, p.cand + l1 * p.cand_cap, p.cand_cnt[l1], bigbytes / 8, VATTN_CAND1_BOUND,
+                                 meta.b, nw, sm.w2, out, dbg);
+  }
+  if (got < 0) {
+    __syncthreads();
+    sample_select<CACHED>(p, sm, meta.s0, meta.l_start, nw, meta.b, meta.n_s, b, hrng, 1, sm.w2, out, dbg);
+  } else if (p.dbg.paths && tid == 0) p.dbg.paths[bh] |= 4;
+  DEV_END(p, 4);
 }
 
 }  // namespace
 
 static int keycap_of(const Prob& p) { return p.npad <= VATTN_KEYCACHE_MAX ? p.npad : 0; }
+// bytes of the shared "big" region: the context's select keys, or staged candidate pairs
+static int big_bytes(const Prob& p, bool final_kernel) {
+  const size_t keys = sizeof(unsigned) * (size_t)keycap_of(p);
+  const size_t pairs = sizeof(uint2) * (size_t)(final_kernel ? p.cand_cap : PAIRCAP0);
+  size_t b = keys > pairs ? keys : pairs;
+  const size_t fixed = sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
+                       sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64);
+  const size_t limit = 227 * 1024;
+  if (fixed + b > limit) b = (limit - fixed) / 16 * 16;       // fewer staged pairs: the list path then declines
+  return (int)b;
+}
 
 size_t select_smem_bytes(const Prob& p) {
-  return sizeof(double) * VATTN_BANDCAP + sizeof(unsigned) * (size_t)keycap_of(p) + 4 * sizeof(unsigned) * (size_t)p.nwords +
-         sizeof(unsigned) * 256 + sizeof(int) * VATTN_BANDCAP + sizeof(int) * 64;
+  return sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
+         sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64) + (size_t)big_bytes(p, true);
 }
 
 // Opt-in to large dynamic shared memory once per kernel and size (a function attribute, not a
 // stream operation; done before the first launch so that later launches can be stream-captured).
 template <typename KernelT>
-static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s) {
-  const size_t smem = select_smem_bytes(p);
+static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s, bool final_kernel) {
+  const int big = big_bytes(p, final_kernel);
+  const size_t smem = sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
+                      sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64) + (size_t)big;
   static const void* seen_fn[32];
   static size_t seen_sz[32];
   static int nseen = 0;
@@ -467,20 +814,20 @@ static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s) {
     if (nseen < 32) { seen_fn[nseen] = (const void*)kern; seen_sz[nseen] = smem; ++nseen; }
   }
   dim3 grid(p.Hq, p.B), block(NT);
-  kern<<<grid, block, smem, s>>>(p, keycap_of(p));
+  kern<<<grid, block, smem, s>>>(p, big);
   return cudaGetLastError();
 }
 
 cudaError_t launch_select_topk_base(const Prob& p, cudaStream_t s) {
   const bool cached = keycap_of(p) > 0;
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) return cached ? launch_sel(k_select_topk_base<bf16_t, 128, true>, p, s) : launch_sel(k_select_topk_base<bf16_t, 128, false>, p, s);
-    return cached ? launch_sel(k_select_topk_base<bf16_t, 64, true>, p, s) : launch_sel(k_select_topk_base<bf16_t, 64, false>, p, s);
+    if (p.D == 128) return cached ? launch_sel(k_select_topk_base<bf16_t, 128, true>, p, s, false) : launch_sel(k_select_topk_base<bf16_t, 128, false>, p, s, false);
+    return cached ? launch_sel(k_select_topk_base<bf16_t, 64, true>, p, s, false) : launch_sel(k_select_topk_base<bf16_t, 64, false>, p, s, false);
   }
-  if (p.D == 128) return cached ? launch_sel(k_select_topk_base<float, 128, true>, p, s) : launch_sel(k_select_topk_base<float, 128, false>, p, s);
-  return cached ? launch_sel(k_select_topk_base<float, 64, true>, p, s) : launch_sel(k_select_topk_base<float, 64, false>, p, s);
+  if (p.D == 128) return cached ? launch_sel(k_select_topk_base<float, 128, true>, p, s, false) : launch_sel(k_select_topk_base<float, 128, false>, p, s, false);
+  return cached ? launch_sel(k_select_topk_base<float, 64, true>, p, s, false) : launch_sel(k_select_topk_base<float, 64, false>, p, s, false);
 }
 
 cudaError_t launch_select_final(const Prob& p, cudaStream_t s) {
-  return keycap_of(p) > 0 ? launch_sel(k_select_final<true>, p, s) : launch_sel(k_select_final<false>, p, s);
+  return keycap_of(p) > 0 ? launch_sel(k_select_final<true>, p, s, true) : launch_sel(k_select_final<false>, p, s, true);
 }

@@ -10,34 +10,54 @@
 // Everything that decides the integer budget is fp64: the same inputs must give the same ceil() as a
 // plain fp64 evaluation.  Variances are accumulated around a pivot (the first base-sample row), which
 // removes the cancellation of the one-pass formula and makes a constant population give exactly 0.
+//
+// Grid: per head, `stat_splits` CTAs take the deterministic rows and `stat_splits` CTAs the base-sample
+// rows (two code paths with disjoint accumulators, which halves the register footprint of either).
+// A row group (LPR lanes) keeps 4 rows in flight: indices, page ids and the 16-byte row slices of a
+// batch are all requested before the first is used.
 #include "vattn_internal.cuh"
 #include <math_constants.h>
 
 namespace {
 
-constexpr int NT = ROW_THREADS;
+constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
+constexpr int UN = 4;            // rows in flight per row group
+constexpr int MAXS = 16;         // most split CTAs per head and kind
 
-template <typename T, int D>
-struct RowLayout {
-  static constexpr int EPL = Elem<T>::EPL;
-  static constexpr int LPR = D / EPL;
-  static constexpr int RPI = 32 / LPR;
+template <typename T> struct Raw;
+template <> struct Raw<float> {
+  float4 v;
+  __device__ __forceinline__ void ld(const float* p) { v = *reinterpret_cast<const float4*>(p); }
+  __device__ __forceinline__ float get(int e) const { return e == 0 ? v.x : e == 1 ? v.y : e == 2 ? v.z : v.w; }
+};
+template <> struct Raw<bf16_t> {
+  uint4 v;
+  __device__ __forceinline__ void ld(const bf16_t* p) { v = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ float get(int e) const {
+    const unsigned w = (e >> 1) == 0 ? v.x : (e >> 1) == 1 ? v.y : (e >> 1) == 2 ? v.z : v.w;
+    return __uint_as_float((e & 1) ? (w & 0xFFFF0000u) : (w << 16));
+  }
 };
 
-// fp64 weight of one token and its value slice, computed by the LPR lanes of a row group
+template <typename T>
+struct RowRegs { Raw<T> k, v; };
+
 template <typename T, int D>
-__device__ __forceinline__ double row_weight(const Prob& p, int b, int g, const float (&qf)[Elem<T>::EPL], int tok,
-                                             int j, double m, float (&v)[Elem<T>::EPL]) {
+__device__ __forceinline__ void load_row(const Prob& p, int b, int g, int tok, int j, RowRegs<T>& r) {
+  constexpr int EPL = Elem<T>::EPL;
+  const int pg = page_of(p, b, tok >> 4);
+  const long long off = (long long)pg * p.sb + (long long)g * p.sh + (long long)(tok & 15) * p.st + j * EPL;
+  r.k.ld(reinterpret_cast<const T*>(p.kc) + off);
+  r.v.ld(reinterpret_cast<const T*>(p.vc) + off);
+}
+// fp64 weight of one token, computed by the LPR lanes of a row group from its K slice
+template <typename T, int D>
+__device__ __forceinline__ double weight64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r, double m) {
   constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
-  const T* krow = row_ptr<T>(p, p.kc, b, g, tok);
-  const T* vrow = row_ptr<T>(p, p.vc, b, g, tok);
-  float kx[EPL];
-  Elem<T>::load(krow + j * EPL, kx);
-  Elem<T>::load(vrow + j * EPL, v);
   double acc = 0.0;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) acc = fma((double)qf[e], (double)kx[e], acc);
+  for (int e = 0; e < EPL; ++e) acc = fma((double)qf[e], (double)r.k.get(e), acc);
 #pragma unroll
   for (int mask = LPR / 2; mask >= 1; mask >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, mask);
   return exp(acc * (double)p.scale - m);
@@ -49,23 +69,26 @@ __device__ __forceinline__ int ceil_sat(double x) {
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(NT) k_stats(const Prob p) {
-  using L = RowLayout<T, D>;
-  constexpr int EPL = L::EPL, LPR = L::LPR, RPI = L::RPI;
-  constexpr int NE = 2 * D + 4;           // N_f[D], D_f, Sw, Sww, Sr[D], Srr
+__global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
+  constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR;
+  constexpr int NE = D + 3;               // det CTA: N_f[D], D_f;  base CTA: Sr[D], Sw, Sww, Srr
+  constexpr int RG = NWARP * RPI;         // row groups per CTA
   __shared__ double part[NWARP][NE];
-  __shared__ double tot[NE];
+  __shared__ double tot[2][NE];
   __shared__ double piv[D + 1];
   __shared__ int is_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z, g = h / p.G;
+  const int h = blockIdx.y, b = blockIdx.z, g = h / p.G;
   const int bh = b * p.Hq + h;
   const int S = p.stat_splits;
+  const bool base_cta = (int)blockIdx.x >= S;
+  const int split = base_cta ? blockIdx.x - S : blockIdx.x;
+  DEV_BEGIN(p, 3);
   HeadMeta& meta = p.meta[bh];
   const int n = meta.n, s0 = meta.s0, l_start = meta.l_start, kk = meta.kk, n_s = meta.n_s, b0 = meta.b0;
   if (n == 0) {
-    if (split == 0 && tid == 0) {
+    if (blockIdx.x == 0 && tid == 0) {
       meta.b = 0;
       if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
       if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
@@ -73,122 +96,166 @@ __global__ void __launch_bounds__(NT) k_stats(const Prob p) {
     return;
   }
   const int n_f = s0 + kk + (n - l_start);
-  const int total = n_f + b0;
+  const int total = base_cta ? b0 : n_f;
   const int chunk = (total + S - 1) / S;
   const int r_begin = min(total, split * chunk), r_end = min(total, r_begin + chunk);
   const int* tk = p.topk_idx + (long long)bh * p.npad;
   const int* bs = p.base_idx + (long long)bh * p.npad;
   const double m = (double)meta.m;
   const int rsub = lane / LPR, j = lane % LPR;
+  const int rg = warp * RPI + rsub;
+  const int iters = (r_end - r_begin + RG - 1) / RG;      // uniform over the CTA
 
   float qf[EPL];
   Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+  DEV_MARK(p, 3, 2, bh == 0 && blockIdx.x == 0);
 
-  // pivot = first base-sample row (every row group computes the same numbers)
-  double cw = 0.0, cr[EPL];
+  double acc[EPL], s1 = 0.0, s2 = 0.0, s3 = 0.0;           // det: N_f slice, D_f;  base: Sr slice, Sw, Sww, Srr
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) cr[e] = 0.0;
-  if (b0 > 0) {
-    float v[EPL];
-    cw = row_weight<T, D>(p, b, g, qf, bs[0], j, m, v);
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.0;
+
+  if (!base_cta) {
+    // ---------------------------------------------------------------- deterministic rows: sink, I_t, window
+    for (int k0 = 0; k0 < iters; k0 += UN) {
+      int tok[UN];
+      bool act[UN];
+      RowRegs<T> row[UN];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) cr[e] = cw * (double)v[e];
-    if (warp == 0 && rsub == 0) {
+      for (int u = 0; u < UN; ++u) {
+        const int r = r_begin + rg + (k0 + u) * RG;
+        act[u] = (k0 + u < iters) && (r < r_end);
+        tok[u] = 0;
+        if (act[u]) tok[u] = r < s0 ? r : (r < s0 + kk ? __ldg(tk + r - s0) : l_start + (r - s0 - kk));
+      }
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cr[e];
-      if (j == 0) piv[D] = cw;
+      for (int u = 0; u < UN; ++u) load_row<T, D>(p, b, g, tok[u], j, row[u]);   // idle slots re-read token 0
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const double w = weight64<T, D>(p, qf, row[u], m);     // every lane takes part in the shuffles
+        if (act[u]) {
+          s1 += w;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[e] = fma(w, (double)row[u].v.get(e), acc[e]);
+        }
+      }
     }
-  } else {
-    for (int e = tid; e <= D; e += NT) piv[e] = 0.0;
-  }
-
-  double Nf[EPL], Sr[EPL], Df = 0.0, Sw = 0.0, Sww = 0.0, Srr = 0.0;
+  } else if (b0 > 0) {
+    // ---------------------------------------------------------------- base-sample rows, shifted by the pivot
+    RowRegs<T> prow;
+    load_row<T, D>(p, b, g, __ldg(bs), j, prow);             // pivot = first base-sample row
+    double cw = 0.0, cr[EPL];
+    for (int k0 = 0; k0 < max(iters, 1); k0 += UN) {
+      int tok[UN];
+      bool act[UN];
+      RowRegs<T> row[UN];
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) { Nf[e] = 0.0; Sr[e] = 0.0; }
-
-  for (int r0 = r_begin + warp * RPI; r0 < r_end; r0 += NWARP * RPI) {
-    const int r = r0 + rsub;
-    const bool active = r < r_end;
-    int tok = 0;
-    bool is_base = false;
-    if (active) {
-      if (r < s0) tok = r;
-      else if (r < s0 + kk) tok = tk[r - s0];
-      else if (r < n_f) tok = l_start + (r - s0 - kk);
-      else { tok = bs[r - n_f]; is_base = true; }
-    }
-    float v[EPL];
-    // inactive row groups still take part in the shuffles (they recompute token 0 and drop it)
-    const double w = row_weight<T, D>(p, b, g, qf, tok, j, m, v);
-    if (active) {
-      if (!is_base) {
-        Df += w;
+      for (int u = 0; u < UN; ++u) {
+        const int r = r_begin + rg + (k0 + u) * RG;
+        act[u] = (k0 + u < iters) && (r < r_end);
+        tok[u] = act[u] ? __ldg(bs + r) : 0;
+      }
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) Nf[e] = fma(w, (double)v[e], Nf[e]);
-      } else {
-        const double dw = w - cw;
-        Sw += dw;
-        Sww = fma(dw, dw, Sww);
+      for (int u = 0; u < UN; ++u) load_row<T, D>(p, b, g, tok[u], j, row[u]);
+      if (k0 == 0) {
+        cw = weight64<T, D>(p, qf, prow, m);
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-          const double dr = w * (double)v[e] - cr[e];
-          Sr[e] += dr;
-          Srr = fma(dr, dr, Srr);
+        for (int e = 0; e < EPL; ++e) cr[e] = cw * (double)prow.v.get(e);
+        if (warp == 0 && rsub == 0) {
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cr[e];
+          if (j == 0) piv[D] = cw;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const double w = weight64<T, D>(p, qf, row[u], m);
+        if (act[u]) {
+          const double dw = w - cw;
+          s1 += dw;
+          s2 = fma(dw, dw, s2);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) {
+            const double dr = w * (double)row[u].v.get(e) - cr[e];
+            acc[e] += dr;
+            s3 = fma(dr, dr, s3);
+          }
         }
       }
     }
   }
+  DEV_MARK(p, 3, 3, bh == 0 && blockIdx.x == 0);
   // across the row groups of the warp
 #pragma unroll
   for (int mask = LPR; mask < 32; mask <<= 1) {
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      Nf[e] += __shfl_xor_sync(0xFFFFFFFFu, Nf[e], mask);
-      Sr[e] += __shfl_xor_sync(0xFFFFFFFFu, Sr[e], mask);
-    }
-    Df += __shfl_xor_sync(0xFFFFFFFFu, Df, mask);
-    Sw += __shfl_xor_sync(0xFFFFFFFFu, Sw, mask);
-    Sww += __shfl_xor_sync(0xFFFFFFFFu, Sww, mask);
+    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], mask);
+    s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, mask);
+    s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, mask);
   }
 #pragma unroll
-  for (int mask = 1; mask < 32; mask <<= 1) Srr += __shfl_xor_sync(0xFFFFFFFFu, Srr, mask);
+  for (int mask = 1; mask < 32; mask <<= 1) s3 += __shfl_xor_sync(0xFFFFFFFFu, s3, mask);
   if (rsub == 0) {
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) { part[warp][j * EPL + e] = Nf[e]; part[warp][D + 3 + j * EPL + e] = Sr[e]; }
-    if (j == 0) { part[warp][D] = Df; part[warp][D + 1] = Sw; part[warp][D + 2] = Sww; part[warp][2 * D + 3] = Srr; }
+    for (int e = 0; e < EPL; ++e) part[warp][j * EPL + e] = acc[e];
+    if (j == 0) { part[warp][D] = s1; part[warp][D + 1] = s2; part[warp][D + 2] = s3; }
   }
   __syncthreads();
-  double* gpart = p.stat_part + ((long long)bh * S + split) * NE;
+  double* gpart = p.stat_part + ((long long)bh * 2 * MAXS + blockIdx.x) * NE;
   for (int e = tid; e < NE; e += NT) {
     double s = 0.0;
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) s += part[w][e];
     gpart[e] = s;
   }
+  DEV_MARK(p, 3, 4, bh == 0 && blockIdx.x == 0);
   __threadfence();
   __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.tickets[bh], 1u) == (unsigned)(S - 1));
+  if (tid == 0) is_last = (atomicAdd(&p.tickets[bh], 1u) == (unsigned)(2 * S - 1));
   __syncthreads();
-  if (!is_last) return;
+  DEV_MARK(p, 3, 5, bh == 0 && blockIdx.x == 0);
+  if (!is_last) { DEV_END(p, 3); return; }
   __threadfence();
+  DEV_MARK(p, 3, 6, bh == 0);
 
   // ------------------------------------------------------------------ last CTA of this head
-  for (int e = tid; e < NE; e += NT) {
+  // every thread requests all partials of its element at once (one memory round trip), then adds them
+  // in split order; kind 0 = deterministic partials, kind 1 = base partials
+  for (int item = tid; item < 2 * NE; item += NT) {
+    const int kind = item / NE, e = item % NE;
+    const double* src = p.stat_part + ((long long)bh * 2 * MAXS + kind * S) * NE + e;
+    double v[MAXS];
+#pragma unroll
+    for (int sp = 0; sp < MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;
     double s = 0.0;
-    for (int sp = 0; sp < S; ++sp) s += __ldcg(p.stat_part + ((long long)bh * S + sp) * NE + e);
-    tot[e] = s;
+#pragma unroll
+    for (int sp = 0; sp < MAXS; ++sp) s += v[sp];
+    tot[kind][e] = s;
+  }
+  // the pivot again (deterministic: every CTA computes the same numbers), whatever kind this CTA is
+  if (b0 > 0) {
+    RowRegs<T> prow;
+    load_row<T, D>(p, b, g, __ldg(bs), j, prow);
+    const double cw = weight64<T, D>(p, qf, prow, m);
+    if (warp == 0 && rsub == 0) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cw * (double)prow.v.get(e);
+      if (j == 0) piv[D] = cw;
+    }
+  } else {
+    for (int e = tid; e <= D; e += NT) piv[e] = 0.0;
   }
   __syncthreads();
+  DEV_MARK(p, 3, 7, bh == 0);
   double* det = p.det_sums + (long long)bh * (D + 1);
-  for (int e = tid; e <= D; e += NT) det[e] = tot[e];
+  for (int e = tid; e <= D; e += NT) det[e] = tot[0][e];
   if (warp != 0) return;
 
-  const double Dfv = tot[D];
+  const double Dfv = tot[0][D];
   const double ratio = (b0 > 0) ? (double)n_s / (double)b0 : 0.0;
   double nn = 0.0, sr2 = 0.0;                 // |N_hat|^2 and sum_j (sum_i r'_ij)^2
   for (int e = lane; e < D; e += 32) {
-    const double srj = tot[D + 3 + e];
-    const double nh = tot[e] + ratio * (srj + (double)b0 * piv[e]);
+    const double srj = tot[1][e];
+    const double nh = tot[0][e] + ratio * (srj + (double)b0 * piv[e]);
     nn = fma(nh, nh, nn);
     sr2 = fma(srj, srj, sr2);
   }
@@ -203,7 +270,7 @@ __global__ void __launch_bounds__(NT) k_stats(const Prob p) {
   double sigma2 = 0.0, trace = 0.0, Dhat = Dfv;
   int bD = 0, bN = 0, bS = 0, bfin = 0;
   if (n_s > 0) {
-    const double Swv = tot[D + 1], Swwv = tot[D + 2], Srrv = tot[2 * D + 3];
+    const double Swv = tot[1][D], Swwv = tot[1][D + 1], Srrv = tot[1][D + 2];
     if (b0 >= 2) {
       sigma2 = fmax(0.0, (Swwv - Swv * Swv / (double)b0) / (double)(b0 - 1));
       trace = fmax(0.0, (Srrv - sr2 / (double)b0) / (double)(b0 - 1));
@@ -234,6 +301,7 @@ __global__ void __launch_bounds__(NT) k_stats(const Prob p) {
     }
   }
   meta.b = bfin;
+  DEV_END(p, 3);
   if (p.dbg.budgets) {
     int* o = p.dbg.budgets + bh * 4;
     o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bfin;
@@ -247,7 +315,8 @@ __global__ void __launch_bounds__(NT) k_stats(const Prob p) {
 }  // namespace
 
 cudaError_t launch_stats(const Prob& p, cudaStream_t s) {
-  dim3 grid(p.stat_splits, p.Hq, p.B), block(NT);
+  dim3 grid(2 * p.stat_splits, p.Hq, p.B), block(NT);
+  if (p.stat_splits < 1 || p.stat_splits > MAXS) return cudaErrorInvalidValue;
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (p.D == 128) k_stats<bf16_t, 128><<<grid, block, 0, s>>>(p);
     else k_stats<bf16_t, 64><<<grid, block, 0, s>>>(p);

@@ -6,7 +6,7 @@
 
 #define VATTN_BLOCK 16                 // tokens per KV page
 #define VATTN_MAX_SEQ (1 << 18)        // longest sequence the select kernels' shared-memory bitmaps hold
-#define VATTN_KEYCACHE_MAX 49152       // tokens whose 32-bit select keys are cached in shared memory
+#define VATTN_KEYCACHE_MAX 40960       // tokens whose 32-bit select keys are cached in shared memory
 #define VATTN_BANDCAP 1024             // near-tie top-k candidates rescored by the fast path
 #define SEL_THREADS 1024
 #define ROW_THREADS 256
@@ -43,7 +43,10 @@ struct Prob {
   float* scores;          // [B,Hq,npad]
   unsigned* m_ord;        // [B,Hq]  order-preserving encoding of the running max score
   unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
-  unsigned* tickets;      // [2,B,Hq] "last CTA done" counters (stats, gather)
+  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters (stats, gather, dense)
+  unsigned* cand_cnt;     // [2,B,Hq] entries appended to the sampling-candidate lists (may exceed cand_cap)
+  uint2* cand;            // [2,B,Hq,cand_cap] (Philox key, token) with key below the stream's pre-filter
+  int cand_cap;
   unsigned* status;       // [1]
   unsigned* bitmap;       // [B,Hq,nwords] membership of I_t
   int* topk_idx;          // [B,Hq,npad]
@@ -56,7 +59,21 @@ struct Prob {
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, gat_splits, dense_splits;
   vattn_debug dbg;
+  unsigned long long* devt;   // development timing buffer [8][32] (null unless a dev build sets it)
 };
+
+// Development-only phase timing (compiled in with -DVATTN_DEV_TIMING): slot 0/1 of a kernel's row hold
+// the earliest CTA start / latest CTA end, further slots are set by one chosen CTA.
+#ifdef VATTN_DEV_TIMING
+__device__ __forceinline__ unsigned long long dev_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define DEV_BEGIN(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMin(&(p).devt[(k) * 32 + 0], dev_gtime()); } while (0)
+#define DEV_END(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMax(&(p).devt[(k) * 32 + 1], dev_gtime()); } while (0)
+#define DEV_MARK(p, k, slot, cond) do { if ((p).devt && threadIdx.x == 0 && (cond)) (p).devt[(k) * 32 + (slot)] = dev_gtime(); } while (0)
+#else
+#define DEV_BEGIN(p, k) do { } while (0)
+#define DEV_END(p, k) do { } while (0)
+#define DEV_MARK(p, k, slot, cond) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // small device helpers
@@ -121,6 +138,33 @@ __device__ __forceinline__ int clamped_len(const Prob& p, int b) {
   int n = p.seq_lens[b];
   if (n < 0 || n > p.max_seq_len) { atomicOr(p.status, VATTN_STATUS_BAD_SEQLEN); n = n < 0 ? 0 : p.max_seq_len; }
   return n;
+}
+
+// Index-set geometry of one sequence (Algorithm 1 lines 1-5 with absolute sink/window counts):
+// sink range [0,s0), window [l_start,n), middle M = [s0,l_start), kk = |I_t|, n_s = |M| - kk, b0.
+struct Geo { int s0, l_start, kk, n_s, b0; };
+__device__ __forceinline__ Geo head_geometry(const Prob& p, int n) {
+  Geo g;
+  g.s0 = min(p.sink, n);
+  g.l_start = max(n - p.window, g.s0);
+  const int mlen = g.l_start - g.s0;
+  int kb = p.k;
+  if (p.topk_frac > 0.f) kb = (int)floor((double)p.topk_frac * (double)n);
+  g.kk = min(kb, mlen);
+  g.n_s = mlen - g.kk;
+  g.b0 = 0;
+  if (g.n_s > 0) g.b0 = min(g.n_s, max(2, (int)floor((double)p.base_rate * (double)g.n_s)));
+  return g;
+}
+// Pre-filters of the sampling-candidate lists: a token is a candidate of stream s when its Philox key
+// is below this bound.  Stream 1 keeps a quarter of the tokens; stream 0 keeps b0 + 6 sqrt(b0) + 16
+// expected tokens (none if that is more than a quarter: the select kernel then draws without the list).
+#define VATTN_CAND1_BOUND 0x40000000u
+__device__ __forceinline__ unsigned cand0_bound(const Geo& g) {
+  if (g.n_s <= 0 || g.b0 <= 0) return 0u;
+  const double want = (double)g.b0 + 6.0 * sqrt((double)g.b0) + 16.0;
+  const double frac = want / (double)g.n_s;
+  return frac > 0.25 ? 0u : (unsigned)(frac * 4294967296.0);
 }
 
 // Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0,k1)

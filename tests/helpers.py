@@ -76,7 +76,7 @@ def assert_parity(case, out, dbg, det, out_ref, check_scores=True):
         assert np.array_equal(dbg["dyn_idx"][b, h, :bb], r["I_dyn"]), f"{tag}: I_dyn differs"
         st, sr = dbg["stats"][b, h], r["stats"]
         assert st[5] == sr[5] and st[6] == sr[6], tag
-        np.testing.assert_allclose(st[7], sr[7], rtol=0, atol=1e-4, err_msg=tag)
+        np.testing.assert_allclose(st[7], sr[7], rtol=2e-6, atol=1e-4, err_msg=tag)     # m is an fp32 score
         # weights are relative to each side's own m: compare the m-free ratios
         sc = np.exp(sr[7] - st[7])
         np.testing.assert_allclose(st[0] * 1.0, sr[0] * sc, rtol=1e-9, err_msg=tag + " D_f")

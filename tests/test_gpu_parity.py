@@ -160,6 +160,44 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), out_dev)
 
 
+# ----------------------------------------------------------------------------- fast paths and their fallbacks at size
+def mid(**kw):
+    args = dict(dtype="bf16", B=1, Hq=8, Hkv=2, d=128, seq_lens=[20000], sink=64, window=64, k=500, eps=0.05,
+                delta=0.05, seed=99, gen_seed=4242, key_std=1.0, rho_v=1.0,
+                heavy=dict(R=64, c1=8.0, alpha=(0.75, 1.25)), params=dict(base_rate=0.025))
+    args.update(kw)
+    return synth.make_case("mid", **args)
+
+
+def test_large_base_rate_and_large_budget_draw_from_the_full_context():
+    # base sample of half the residual, and forced budgets above a quarter of it: no candidate list applies
+    _, dbg, _, _ = check(mid(params=dict(base_rate=0.5)))
+    assert (dbg["paths"] & 2 == 0).all()      # base sample drawn from the full context
+    _, dbg, _, _ = check(mid(), force_budget=9000)
+    assert (dbg["paths"] & 4 == 0).all() and (dbg["paths"] & 3 == 3).all()
+    _, dbg, _, _ = check(mid(), force_budget=4000)   # below a quarter: drawn from the pre-filtered list
+    assert (dbg["paths"] == 7).all()
+
+
+def test_single_huge_outlier_score_defeats_the_threshold_estimate():
+    case = mid(heavy=None)
+    kc = synth.bf16_bits_to_f32(case.k_cache)
+    q = synth.bf16_bits_to_f32(case.q)
+    tok = 7777
+    pg = case.block_table[0, tok // 16]
+    for g in range(2):                        # one key aligned with the group's first query, logit ~ +3000
+        kc[pg, g, tok % 16] = 3000.0 * np.sqrt(128.0) * q[0, g * 4] / float(q[0, g * 4] @ q[0, g * 4])
+    case.k_cache = synth.f32_to_bf16_bits(kc)
+    _, dbg, _, _ = check(case)
+    assert (dbg["paths"][0, 0] & 1) == 0 and (dbg["paths"][0, 4] & 1) == 0   # heads 0 and 4 see the outlier
+
+
+def test_many_topk_and_fp32_at_size():
+    _, dbg, _, _ = check(mid(k=6000))         # more top-k tokens than the candidate buffer holds
+    assert (dbg["paths"] & 1 == 0).all()
+    check(mid(dtype="fp32", d=64, seq_lens=[20000, 9000], B=2))
+
+
 # ----------------------------------------------------------------------------- the five workloads
 def test_config1_tiny():
     case = synth.config1_tiny()
@@ -173,6 +211,7 @@ def test_config2_llama8b_full_size():
     out, dbg, det, _ = check(case)
     dens = np.mean([(len(r["I_f"]) + r["b"]) / r["n"] for r in det.values()])
     assert 0.09 < dens < 0.11                      # the calibrated ~10x sparsity operating point
+    assert (dbg["paths"] == 7).all()               # the benchmark workload runs the fast paths on every head
 
 
 def test_config3_uniform_full_size_and_sparsity_sweep():
