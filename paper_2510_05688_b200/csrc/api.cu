@@ -21,7 +21,7 @@ struct vattn_plan {
   // derived
   int G, npad, nwords, stat_splits, gat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
-      off_det, off_gat, off_dense, off_cand, total;
+      off_det, off_piv, off_gat, off_dense, off_cand, total;
   int cand_cap;
 };
 
@@ -83,13 +83,14 @@ void derive(vattn_plan* pl) {
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
-  pl->off_topk = take(BH * pl->npad * sizeof(int));
-  pl->off_base = take(BH * pl->npad * sizeof(int));
-  pl->off_dyn = take(BH * pl->npad * sizeof(int));
+  pl->off_topk = take(2 * BH * pl->npad * sizeof(int));     // token indices, then physical slots
+  pl->off_base = take(2 * BH * pl->npad * sizeof(int));
+  pl->off_dyn = take(2 * BH * pl->npad * sizeof(int));
   pl->off_meta = take(BH * sizeof(HeadMeta));
   pl->off_stat = take(BH * 2 * kMaxStatSplits * (D + 3) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
-  pl->off_gat = take(BH * pl->gat_splits * (D + 1) * sizeof(float));
+  pl->off_piv = take(BH * (D + 1) * sizeof(double));
+  pl->off_gat = take(BH * kMaxGatherSplits * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
   {
     const double q4 = 0.25 * (double)pl->npad;
@@ -131,9 +132,11 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
   p.base_idx = reinterpret_cast<int*>(w + pl->off_base);
   p.dyn_idx = reinterpret_cast<int*>(w + pl->off_dyn);
+  p.phys_delta = (long long)BH * pl->npad;
   p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
   p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);
   p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
+  p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.stat_splits = pl->stat_splits; p.gat_splits = pl->gat_splits; p.dense_splits = pl->dense_splits;

@@ -2,148 +2,243 @@
 //     N = N_f + (n_s/b) * sum_{I_dyn} w_i V[i],   D = D_f + (n_s/b) * sum_{I_dyn} w_i,   out = N / D
 // which is SDPA_{S,p} of Sec. 3 with p = 1 on I_f and p = b/n_s on I_dyn.
 //
-// HBM-bound row gather: the b sampled V rows of a head (ascending token order, so rows of one page sit
-// next to each other) are split over `gat_splits` CTAs; LPR lanes fetch one row with one 16-byte load
-// each, several rows in flight per warp.  Weights come from the stored fp32 scores (no K re-read).
-// Partials are added in a fixed order by the last CTA of the head, so results are reproducible.
+// HBM-bound row gather.  Work unit = a chunk of consecutive entries of one head's I_dyn list.  LPR lanes
+// fetch one V row with one 16-byte load each; a row group keeps 4 rows in flight and requests the next
+// batch's indices (token + physical slot, written by the select kernel) while the current rows arrive.
+// Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
+// last CTA of the head ("ticket"), so results are reproducible.
+//
+// Two decompositions:
+//  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
+//    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
+//    grid stride: every SM gets the same number of rows whatever the budgets are;
+//  * per head (larger problems): grid (splits, heads, batch), every head cut into `gat_splits` chunks.
 #include "vattn_internal.cuh"
 
 namespace {
 
 constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
-constexpr int UNROLL = 4;
-constexpr int MAXS = 32;         // most split CTAs per head
+constexpr int UNROLL = 8;         // rows in flight per row group (16-byte slices kept raw until used)
+constexpr int MAXS = 32;           // most chunks (partials) per head
+constexpr int FLAT_MAX_HEADS = 128;
+constexpr int MIN_CHUNK = 64;      // rows of a chunk in the flat decomposition, unless the head has > 32 of them
 
 template <typename T, int D>
-__global__ void __launch_bounds__(NT) k_gather(const Prob p) {
-  constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR;
-  constexpr int NE = D + 1;
-  __shared__ float part[NWARP][NE];
-  __shared__ int is_last;
+struct Gather {
+  static constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR, NE = D + 1, RG = NWARP * RPI;
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z, g = h / p.G;
-  const int bh = b * p.Hq + h;
-  const int S = p.gat_splits;
-  DEV_BEGIN(p, 5);
-  const HeadMeta meta = p.meta[bh];
-  T* out = reinterpret_cast<T*>(p.out) + (long long)bh * D;
-  if (meta.n == 0) {
-    if (split == 0) for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
-    return;
-  }
-  const int nb = meta.b;
-  const int chunk = (nb + S - 1) / S;
-  const int r_begin = min(nb, split * chunk), r_end = min(nb, r_begin + chunk);
-  const int* dyn = p.dyn_idx + (long long)bh * p.npad;
-  const float* sc = p.scores + (long long)bh * p.npad;
-  const float m = meta.m;
-  const int rsub = lane / LPR, j = lane % LPR;
-
-  float acc[EPL], dd = 0.f;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-
-  DEV_MARK(p, 5, 2, bh == 0 && split == 0);
-  constexpr int RG = NWARP * RPI;                         // row groups per CTA
-  const int rg = warp * RPI + rsub;
-  const int iters = (r_end - r_begin + RG - 1) / RG;
-  for (int k0 = 0; k0 < iters; k0 += UNROLL) {
-    int tok[UNROLL];
-    float w[UNROLL];
-    float v[UNROLL][EPL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int r = r_begin + rg + (k0 + u) * RG;
-      tok[u] = (k0 + u < iters && r < r_end) ? __ldg(dyn + r) : -1;
+  static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[EPL]) {
+    if (EPL == 8) {
+      v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xFFFF0000u);
+      v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xFFFF0000u);
+      v[4 % EPL] = __uint_as_float(r.z << 16); v[5 % EPL] = __uint_as_float(r.z & 0xFFFF0000u);
+      v[6 % EPL] = __uint_as_float(r.w << 16); v[7 % EPL] = __uint_as_float(r.w & 0xFFFF0000u);
+    } else {
+      v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
     }
+  }
+  // rows [r_begin, r_end) of head bh -> partial `slot`; the last of `nslots` finishers combines
+  static __device__ void run(const Prob& p, int bh, const HeadMeta& meta, int r_begin, int r_end, int slot, int nslots,
+                             float (*part)[NE], int* is_last, float* s_den) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int h = bh % p.Hq, g = h / p.G;
+    T* out = reinterpret_cast<T*>(p.out) + (long long)bh * D;
+    if (meta.n == 0) {
+      if (slot == 0) for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
+      return;
+    }
+    const int* dyn = p.dyn_idx + (long long)bh * p.npad;
+    const int* dph = dyn + p.phys_delta;
+    const float* sc = p.scores + (long long)bh * p.npad;
+    const T* vc = reinterpret_cast<const T*>(p.vc) + (long long)g * p.sh;
+    const float m = meta.m;
+    const int rsub = lane / LPR, j = lane % LPR;
+    const int rg = warp * RPI + rsub;
+    const int iters = (r_end - r_begin + RG - 1) / RG;
+
+    float acc[EPL], dd = 0.f;
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      if (tok[u] >= 0) {
-        Elem<T>::load(row_ptr<T>(p, p.vc, b, g, tok[u]) + j * EPL, v[u]);
-        w[u] = __ldg(sc + tok[u]);
-      } else {
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+
+    int tok_n[UNROLL], ph_n[UNROLL];
+    auto fetch_idx = [&](int k0) {
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const int r = r_begin + rg + (k0 + u) * RG;
+        const bool ok = (k0 + u < iters) && (r < r_end);
+        tok_n[u] = ok ? __ldg(dyn + r) : -1;
+        ph_n[u] = ok ? __ldg(dph + r) : 0;
+      }
+    };
+    fetch_idx(0);
+    for (int k0 = 0; k0 < iters; k0 += UNROLL) {
+      int tok[UNROLL];
+      float w[UNROLL];
+      uint4 raw[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        tok[u] = tok_n[u];
+        raw[u] = make_uint4(0u, 0u, 0u, 0u);
         w[u] = 0.f;
+        if (tok[u] >= 0) {
+          const int ph = ph_n[u];
+          raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
+          w[u] = __ldg(sc + tok[u]);
+        }
+      }
+      if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);   // next batch's indices travel with this batch's rows
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) v[u][e] = 0.f;
+      for (int u = 0; u < UNROLL; ++u) {
+        const float ww = (tok[u] >= 0) ? expf(w[u] - m) : 0.f;
+        dd += ww;
+        float v[EPL];
+        unpack(raw[u], v);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(ww, v[e], acc[e]);
       }
     }
+    DEV_MARK(p, 5, 3, blockIdx.x == 0);
+#ifdef VATTN_DEV_TIMING
+    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 8], dev_gtime());
+#endif
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const float ww = (tok[u] >= 0) ? expf(w[u] - m) : 0.f;
-      dd += ww;
+    for (int mask = LPR; mask < 32; mask <<= 1) {
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[e] = fmaf(ww, v[u][e], acc[e]);
+      for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], mask);
+      dd += __shfl_xor_sync(0xFFFFFFFFu, dd, mask);
+    }
+    __syncthreads();                                  // `part` may still be read by the previous chunk
+    if (rsub == 0) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) part[warp][j * EPL + e] = acc[e];
+      if (j == 0) part[warp][D] = dd;
+    }
+    __syncthreads();
+    float* gpart = p.gat_part + ((long long)bh * MAXS + slot) * NE;
+    for (int e = tid; e < NE; e += NT) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) s += part[w][e];
+      gpart[e] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) *is_last = (atomicAdd(&p.tickets[p.B * p.Hq + bh], 1u) == (unsigned)(nslots - 1));
+    __syncthreads();
+    DEV_MARK(p, 5, 4, blockIdx.x == 0);
+#ifdef VATTN_DEV_TIMING
+    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 9], dev_gtime());
+#endif
+    if (!*is_last) return;
+    __threadfence();
+
+    // last finisher of the head: every thread requests all partials of its element at once (one memory
+    // round trip), adds them in slot order, scales by n_s/b and divides
+    const int nb = meta.b;
+    const double* det = p.det_sums + (long long)bh * (D + 1);
+    const double f = (nb > 0) ? (double)meta.n_s / (double)nb : 0.0;
+    const float* src0 = p.gat_part + (long long)bh * MAXS * NE;
+    float num_s[(D + NT - 1) / NT];
+    double det_e[(D + NT - 1) / NT];
+    const double det_d = __ldcg(det + D);             // N_f, D_f of the statistics kernel, requested with the partials
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) det_e[it] = (tid + it * NT < D) ? __ldcg(det + tid + it * NT) : 0.0;
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) {
+      const int e = tid + it * NT;
+      float vv[MAXS];
+#pragma unroll
+      for (int sp = 0; sp < MAXS; ++sp) vv[sp] = (sp < nslots && e < D) ? __ldcg(src0 + (long long)sp * NE + e) : 0.f;
+      float s = 0.f;
+#pragma unroll
+      for (int sp = 0; sp < MAXS; ++sp) s += vv[sp];
+      num_s[it] = s;
+    }
+    if (warp == 0) {                                  // the denominator: lane sp holds slot sp
+      const float vd = (lane < nslots) ? __ldcg(src0 + (long long)lane * NE + D) : 0.f;
+      float s = 0.f;
+#pragma unroll
+      for (int sp = 0; sp < MAXS; ++sp) s += __shfl_sync(0xFFFFFFFFu, vd, sp);
+      if (lane == 0) *s_den = s;
+    }
+    __syncthreads();
+#ifdef VATTN_DEV_TIMING
+    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 10], dev_gtime());
+#endif
+    const double den = det_d + f * (double)(*s_den);
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) {
+      const int e = tid + it * NT;
+      if (e < D) out[e] = Elem<T>::from_float((float)((det_e[it] + f * (double)num_s[it]) / den));
     }
   }
-  DEV_MARK(p, 5, 3, bh == 0 && split == 0);
-#pragma unroll
-  for (int mask = LPR; mask < 32; mask <<= 1) {
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], mask);
-    dd += __shfl_xor_sync(0xFFFFFFFFu, dd, mask);
-  }
-  if (rsub == 0) {
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) part[warp][j * EPL + e] = acc[e];
-    if (j == 0) part[warp][D] = dd;
-  }
-  __syncthreads();
-  float* gpart = p.gat_part + ((long long)bh * S + split) * NE;
-  for (int e = tid; e < NE; e += NT) {
-    float s = 0.f;
-#pragma unroll
-    for (int w = 0; w < NWARP; ++w) s += part[w][e];
-    gpart[e] = s;
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.tickets[p.B * p.Hq + bh], 1u) == (unsigned)(S - 1));
-  __syncthreads();
-  DEV_MARK(p, 5, 5, bh == 0 && split == 0);
-  if (!is_last) { DEV_END(p, 5); return; }
-  __threadfence();
-  DEV_MARK(p, 5, 6, bh == 0);
-#ifdef VATTN_DEV_TIMING
-  if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 9], dev_gtime());
-#endif
+};
 
-  // last CTA of the head: every thread requests all partials of its element at once (one memory
-  // round trip), adds them in split order, scales by n_s/b and divides
+template <typename T, int D>
+__global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
+  using G = Gather<T, D>;
+  __shared__ float part[NWARP][G::NE];
+  __shared__ int is_last;
   __shared__ float s_den;
-  const double* det = p.det_sums + (long long)bh * (D + 1);
-  const double f = (nb > 0) ? (double)meta.n_s / (double)nb : 0.0;
-  const float* src0 = p.gat_part + (long long)bh * S * NE;
-  float num_s[(D + NT - 1) / NT];
-#pragma unroll
-  for (int it = 0; it < (D + NT - 1) / NT; ++it) {
-    const int e = tid + it * NT;
-    float v[MAXS];
-#pragma unroll
-    for (int sp = 0; sp < MAXS; ++sp) v[sp] = (sp < S && e < D) ? __ldcg(src0 + (long long)sp * NE + e) : 0.f;
-    float s = 0.f;
-#pragma unroll
-    for (int sp = 0; sp < MAXS; ++sp) s += v[sp];
-    num_s[it] = s;
+  DEV_BEGIN(p, 5);
+  const int bh = blockIdx.z * p.Hq + blockIdx.y;
+  const int S = p.gat_splits;
+  const HeadMeta meta = p.meta[bh];
+  const int nb = meta.n > 0 ? meta.b : 0;
+  const int chunk = (nb + S - 1) / S;
+  const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
+  G::run(p, bh, meta, r_begin, r_end, blockIdx.x, S, part, &is_last, &s_den);
+  DEV_END(p, 5);
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
+  using G = Gather<T, D>;
+  __shared__ float part[NWARP][G::NE];
+  __shared__ int is_last;
+  __shared__ float s_den;
+  __shared__ int s_pref[FLAT_MAX_HEADS + 1], s_rows[FLAT_MAX_HEADS], s_b[FLAT_MAX_HEADS], s_w[NWARP];
+  __shared__ HeadMeta s_meta[FLAT_MAX_HEADS];
+  DEV_BEGIN(p, 5);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int BH = p.B * p.Hq;
+  // chunk counts of all heads and their prefix sum (every CTA computes the same numbers)
+  int nb = 0, rows = MIN_CHUNK, cnt = 0;
+  if (tid < BH) {
+    const HeadMeta mt = p.meta[tid];
+    s_meta[tid] = mt;
+    nb = mt.n > 0 ? mt.b : 0;
+    rows = max(MIN_CHUNK, (nb + MAXS - 1) / MAXS);
+    cnt = max(1, (nb + rows - 1) / rows);             // a head without samples still writes its output
+    s_rows[tid] = rows;
+    s_b[tid] = nb;
   }
-  if (warp == 0) {                                            // the denominator: lane sp holds split sp
-    float v = (lane < S) ? __ldcg(src0 + (long long)lane * NE + D) : 0.f;
-    float s = 0.f;
+  int incl = cnt;
 #pragma unroll
-    for (int sp = 0; sp < MAXS; ++sp) s += __shfl_sync(0xFFFFFFFFu, v, sp);
-    if (lane == 0) s_den = s;
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += v;
   }
+  if (lane == 31) s_w[warp] = incl;
   __syncthreads();
-  DEV_MARK(p, 5, 7, bh == 0);
-#ifdef VATTN_DEV_TIMING
-  if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 8], dev_gtime());
-#endif
-  const double den = det[D] + f * (double)s_den;
-#pragma unroll
-  for (int it = 0; it < (D + NT - 1) / NT; ++it) {
-    const int e = tid + it * NT;
-    if (e < D) out[e] = Elem<T>::from_float((float)((det[e] + f * (double)num_s[it]) / den));
+  int before = 0;
+  for (int w = 0; w < warp; ++w) before += s_w[w];
+  if (tid < BH) s_pref[tid] = before + incl - cnt;
+  if (tid == NT - 1) s_pref[BH] = before + incl;      // BH <= NT: the last thread's inclusive sum is the total
+  __syncthreads();
+  const int total = s_pref[BH];
+  DEV_MARK(p, 5, 2, blockIdx.x == 0);
+  for (int c = blockIdx.x; c < total; c += gridDim.x) {
+    int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (s_pref[mid] <= c) lo = mid; else hi = mid - 1;
+    }
+    const int bh = lo, ci = c - s_pref[bh];
+    const int r_begin = min(s_b[bh], ci * s_rows[bh]), r_end = min(s_b[bh], r_begin + s_rows[bh]);
+    G::run(p, bh, s_meta[bh], r_begin, r_end, ci, s_pref[bh + 1] - s_pref[bh], part, &is_last, &s_den);
+    __syncthreads();
   }
   DEV_END(p, 5);
 }
@@ -151,8 +246,22 @@ __global__ void __launch_bounds__(NT) k_gather(const Prob p) {
 }  // namespace
 
 cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
-  dim3 grid(p.gat_splits, p.Hq, p.B), block(NT);
   if (p.gat_splits < 1 || p.gat_splits > MAXS) return cudaErrorInvalidValue;
+  const int BH = p.B * p.Hq;
+  if (BH <= FLAT_MAX_HEADS) {
+    // at most 32 chunks of >= 64 rows per head; 8 CTAs per SM walk them with a grid stride
+    const long long most = (long long)BH * MAXS;
+    const int grid = (int)(most < 8 * 148 ? most : 8 * 148);
+    if (p.dtype == VATTN_DTYPE_BF16) {
+      if (p.D == 128) k_gather_flat<bf16_t, 128><<<grid, NT, 0, s>>>(p);
+      else k_gather_flat<bf16_t, 64><<<grid, NT, 0, s>>>(p);
+    } else {
+      if (p.D == 128) k_gather_flat<float, 128><<<grid, NT, 0, s>>>(p);
+      else k_gather_flat<float, 64><<<grid, NT, 0, s>>>(p);
+    }
+    return cudaGetLastError();
+  }
+  dim3 grid(p.gat_splits, p.Hq, p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (p.D == 128) k_gather<bf16_t, 128><<<grid, block, 0, s>>>(p);
     else k_gather<bf16_t, 64><<<grid, block, 0, s>>>(p);

@@ -4,11 +4,12 @@
 // (softmax stabiliser) and, per KV head, max |K element| (for the rounding-error bound of the scores).
 //
 // HBM-bound stream over K (every K row is read exactly once).  Two arithmetic paths:
-//  * bf16: the [16 tokens x d] x [d x 8 heads] contraction of a page runs on the tensor cores
-//    (mma.sync m16n8k16, fp32 accumulate).  K fragments are loaded straight from global memory with
-//    16-byte loads: a dot product does not care in which order its terms are paired, so the k-slots of
-//    the fragment layout are mapped onto d such that each thread owns 8 consecutive elements of a row.
-//    This removes the CUDA-core FMAs and the cross-lane reduction that made the pass ALU-co-bound.
+//  * bf16: pages travel into shared memory with bulk asynchronous copies (a 4-stage mbarrier ring per
+//    warp) and the [16 tokens x d] x [d x 8 heads] contraction of a page runs on the tensor cores
+//    (mma.sync m16n8k16, fp32 accumulate).  A dot product does not care in which order its terms are
+//    paired, so the k-slots of the fragment layout are mapped onto d such that each thread owns 8
+//    consecutive elements of a row and reads them with one 16-byte shared load.  This removes the
+//    CUDA-core FMAs and the cross-lane reduction that made a first version ALU-co-bound.
 //  * fp32: CUDA-core FMAs, EPL sequential FMAs per lane and a butterfly that halves the live partial
 //    sums at every level (tf32 tensor cores would not keep fp32 accuracy).
 //
@@ -83,107 +84,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsig
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-template <int D>
-__global__ void __launch_bounds__(WARPS * 32) k_score_mma(const Prob p) {
-  constexpr int NC = D / 32;            // 32-element chunks of a row; one chunk feeds two MMAs
-  __shared__ uint2 s_list[16][TILE];
-  __shared__ unsigned s_cnt[16];
-  DEV_BEGIN(p, 1);
-  const int b = blockIdx.z;
-  const int n = clamped_len(p, b);
-  const int tile0 = blockIdx.x * TILE;
-  if (tile0 >= n) return;
-  const int GC = (p.G + 7) >> 3;
-  const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int gr = lane >> 2, t = lane & 3;       // fragment row / column-pair index
-  const int h0 = g * p.G + hc * 8;
-  const int nh = min(8, p.G - hc * 8);
-  const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
-
-  // B fragments: head (hc*8 + gr) of the group, this thread's 8 elements of every chunk
-  uint4 bq[NC];
-#pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    bq[c] = make_uint4(0u, 0u, 0u, 0u);
-    if (gr < nh)
-      bq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
-                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
-  }
-  DEV_MARK(p, 1, 2, blockIdx.x == 0 && blockIdx.y == 0);
-  float runmax[2] = {-INFINITY, -INFINITY};
-  unsigned kabs = 0u;                            // packed max of |bf16| (two 15-bit magnitudes)
-
-#pragma unroll
-  for (int pp = 0; pp < PPW; pp += 2) {
-    int tok0[2];
-    uint4 alo[2][NC], ahi[2][NC];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      tok0[u] = tile0 + (warp * PPW + pp + u) * VATTN_BLOCK;
-      if (tok0[u] < n) {
-        const bf16_t* base = kc + (long long)page_of(p, b, tok0[u] >> 4) * p.sb + (long long)g * p.sh;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-          alo[u][c] = *reinterpret_cast<const uint4*>(base + (long long)gr * p.st + c * 32 + t * 8);
-          ahi[u][c] = *reinterpret_cast<const uint4*>(base + (long long)(gr + 8) * p.st + c * 32 + t * 8);
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (tok0[u] >= n) continue;
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      unsigned klo = 0u, khi = 0u;
-#pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        mma_bf16_16816(acc, alo[u][c].x, ahi[u][c].x, alo[u][c].y, ahi[u][c].y, bq[c].x, bq[c].y);
-        mma_bf16_16816(acc, alo[u][c].z, ahi[u][c].z, alo[u][c].w, ahi[u][c].w, bq[c].z, bq[c].w);
-        klo = __vimax3_u16x2(klo, alo[u][c].x & 0x7FFF7FFFu, alo[u][c].y & 0x7FFF7FFFu);
-        klo = __vimax3_u16x2(klo, alo[u][c].z & 0x7FFF7FFFu, alo[u][c].w & 0x7FFF7FFFu);
-        khi = __vimax3_u16x2(khi, ahi[u][c].x & 0x7FFF7FFFu, ahi[u][c].y & 0x7FFF7FFFu);
-        khi = __vimax3_u16x2(khi, ahi[u][c].z & 0x7FFF7FFFu, ahi[u][c].w & 0x7FFF7FFFu);
-      }
-      const int tk_lo = tok0[u] + gr, tk_hi = tok0[u] + gr + 8;
-      if (tk_lo < n) kabs = __vimax3_u16x2(kabs, klo, 0u);
-      if (tk_hi < n) kabs = __vimax3_u16x2(kabs, khi, 0u);
-      // acc[0],acc[1]: token gr, heads 2t, 2t+1;  acc[2],acc[3]: token gr+8
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int hl = 2 * t + e;
-        if (hl < nh) {
-          float* dst = p.scores + ((long long)b * p.Hq + h0 + hl) * p.npad;
-          const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
-          if (tk_lo < n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
-          if (tk_hi < n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int mask = 4; mask < 32; mask <<= 1) {
-    runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
-    runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
-  }
-#pragma unroll
-  for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
-  if (lane < 4) {
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int hl = 2 * lane + e;
-      if (hl < nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[b * p.Hq + h0 + hl], ord_f32(runmax[e]));
-    }
-  }
-  if (lane == 0) {
-    const unsigned mx = max(kabs & 0xFFFFu, kabs >> 16);          // bf16 magnitude bits
-    atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);               // = fp32 bits of that magnitude
-  }
-  DEV_MARK(p, 1, 3, blockIdx.x == 0 && blockIdx.y == 0);
-  emit_candidates<8>(p, b, g, h0, nh, tile0, n, s_list, s_cnt);
-  DEV_END(p, 1);
-}
-
 
 // ---------------------------------------------------------------------------------------------
 // bf16, streaming variant: every warp owns a ring of NST shared-memory stages and keeps NST pages
@@ -341,7 +241,6 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
   const int wglob = blockIdx.x * WARPS + warp, wtot = gridDim.x * WARPS;
   const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;    // pages this warp owns
   if (role == 1) {
-#ifndef VATTN_EXP_NOCAND
 #ifdef VATTN_DEV_TIMING
     if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 4] = dev_gtime();
 #endif
@@ -350,13 +249,9 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
     if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 5] = dev_gtime();
     if (p.devt && lane == 0) atomicMax(&p.devt[32 + 6], dev_gtime());
 #endif
-#endif
     return;
   }
   if (mine == 0) return;                      // streaming warps use no CTA-wide barrier
-#ifdef VATTN_EXP_NOSTREAM
-  return;
-#endif
   const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
 
   if (lane < NST) mbar_init(&bars[lane], 1);
@@ -434,13 +329,8 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
       if (hl < nh) {
         float* dst = p.scores + ((long long)b * p.Hq + h0 + hl) * p.npad;
         const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
-#ifdef VATTN_EXP_NOSTORE
-        if (tk_lo < n) { runmax[e] = fmaxf(runmax[e], s_lo); }
-        if (tk_hi < n) { runmax[e] = fmaxf(runmax[e], s_hi); }
-#else
         if (tk_lo < n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
         if (tk_hi < n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
-#endif
       }
     }
   }

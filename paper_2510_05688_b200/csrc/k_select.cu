@@ -23,14 +23,6 @@
 // the few in between are rescored in fp64 from their K rows and ranked exactly.
 #include "vattn_internal.cuh"
 
-#ifdef VATTN_DEV_TIMING
-__device__ long long g_phase_clk[64][16];
-#define PHASE(i) do { __syncthreads(); if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.x < 64) g_phase_clk[blockIdx.x][i] = clock64(); } while (0)
-extern "C" int vattn_dev_read_phases(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_phase_clk, sizeof(long long) * 64 * 16); }
-#else
-#define PHASE(i) do { } while (0)
-#endif
-
 namespace {
 
 constexpr int NT = SEL_THREADS;
@@ -174,8 +166,8 @@ __device__ __forceinline__ unsigned lowest_bits(unsigned word, int take) {
 
 // sel |= the `need_eq` lowest-index bits of eq; then write the selected token indices ascending to
 // out_a (and out_b if non-null).  Returns the number selected.
-__device__ int finalize_emit(unsigned* sel, const unsigned* eq, int need_eq, int nw, int* scan, int* misc,
-                             int* out_a, int* out_b) {
+__device__ int finalize_emit(const Prob& p, int b, unsigned* sel, const unsigned* eq, int need_eq, int nw, int* scan,
+                             int* misc, int* out_a, int* out_b) {
   const int tid = threadIdx.x;
   if (need_eq > 0) {
     for (int w = tid; w < nw; w += NT) scan[w] = __popc(eq[w]);
@@ -195,6 +187,7 @@ __device__ int finalize_emit(unsigned* sel, const unsigned* eq, int need_eq, int
       bits &= bits - 1;
       const int idx = w * 32 + bit;
       out_a[pos] = idx;
+      out_a[p.phys_delta + pos] = page_of(p, b, idx >> 4) * VATTN_BLOCK + (idx & 15);   // physical slot for the row kernels
       if (out_b) out_b[pos] = idx;
       ++pos;
     }
@@ -269,11 +262,10 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
       sm.w0[w] = m & ~it[w];
     }
     __syncthreads();
-    return finalize_emit(sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
+    return finalize_emit(p, b, sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
   }
   if (CACHED) fill_philox_keys(p, sm.keys, lo, hi, b, hrng, stream);
   __syncthreads();
-  PHASE(5);
   auto keyfn = [&](int i, unsigned& key) -> bool {
     if ((it[i >> 5] >> (i & 31)) & 1u) return false;
     key = CACHED ? sm.keys[i] : philox_key_of(p, i, b, hrng, stream);
@@ -281,7 +273,6 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
   };
   unsigned T; int need_eq;
   block_select<unsigned, false>(keyfn, lo, hi, c, sm.hist, sm.misc, T, need_eq);
-  PHASE(6);
   for (int w = warp; w < nw; w += NWARP) {
     const int i = w * 32 + lane;
     unsigned key = 0;
@@ -292,8 +283,7 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
     if (lane == 0) { sm.w0[w] = lt; sm.w1[w] = eq; }
   }
   __syncthreads();
-  PHASE(7);
-  return finalize_emit(sm.w0, sm.w1, need_eq, nw, sm.scan, sm.misc, out_a, out_b);
+  return finalize_emit(p, b, sm.w0, sm.w1, need_eq, nw, sm.scan, sm.misc, out_a, out_b);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -302,7 +292,7 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
 // at least c residual tokens; returns -1 when the caller has to draw from the full context.
 // The c-th smallest (key, token) pair is located with one linear-bin histogram over [0, bound) (the
 // keys are uniform, so a bin holds a handful of pairs) and an exact ranking inside that bin.
-__device__ int sample_from_candidates(const Prob& p, const Sm& sm, const uint2* glist, unsigned cnt, int paircap,
+__device__ int sample_from_candidates(const Prob& p, int b, const Sm& sm, const uint2* glist, unsigned cnt, int paircap,
                                       unsigned bound, int c, int nw, const unsigned* it, int* out_a, int* out_b) {
   const int tid = threadIdx.x, lane = tid & 31;
   if (bound == 0u || cnt > (unsigned)p.cand_cap || cnt > (unsigned)paircap || (int)cnt < c) return -1;
@@ -365,7 +355,7 @@ __device__ int sample_from_candidates(const Prob& p, const Sm& sm, const uint2* 
   }
   __syncthreads();
   DEV_MARK(p, 6, 5, blockIdx.x == 0 && blockIdx.y == 0);
-  const int got = finalize_emit(sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
+  const int got = finalize_emit(p, b, sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
   DEV_MARK(p, 6, 6, blockIdx.x == 0 && blockIdx.y == 0);
   return got;
 }
@@ -678,7 +668,6 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
   }
   unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
   if (n == 0) { if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = 0; return; }
-  PHASE(0);
   DEV_MARK(p, 2, 2, bh == 0);
 
   int path = 0;
@@ -699,10 +688,8 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
     if (CACHED) {
       for (int i = s0 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(sc[i]);
       __syncthreads();
-      PHASE(1);
       DEV_MARK(p, 2, 3, bh == 0);
       done = topk_fast<T, D>(p, sm, b, g, qrow, s0, l_start, kk, nw, m, gamma);
-      PHASE(2);
       DEV_MARK(p, 2, 4, bh == 0);
       if (done) path |= 1;
     }
@@ -713,18 +700,16 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
       topk_generic<T, D, CACHED>(p, sm, b, g, qrow, sc, s0, l_start, kk, nw, gamma);
     }
   }
-  PHASE(3);
   // emit I_t ascending, keep its bitmap (shared w2 + global)
   int* tk_out = p.topk_idx + (long long)bh * p.npad;
   int* tk_dbg = p.dbg.topk_idx ? p.dbg.topk_idx + (long long)bh * p.max_seq_len : nullptr;
-  finalize_emit(sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, tk_out, tk_dbg);
+  finalize_emit(p, b, sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, tk_out, tk_dbg);
   for (int w = tid; w < p.nwords; w += NT) {
     const unsigned v = (w < nw) ? sm.w0[w] : 0u;
     sm.w2[w] = v;
     gbitmap[w] = v;
   }
   __syncthreads();
-  PHASE(4);
   DEV_MARK(p, 2, 5, bh == 0);
 
   // ------------------------------------------------------------------ base sample (Philox stream 0)
@@ -733,14 +718,13 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
   int* bs_dbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
   int got = -1;
   if (b0 > 0 && b0 < n_s)
-    got = sample_from_candidates(p, sm, p.cand + (long long)bh * p.cand_cap, p.cand_cnt[bh], bigbytes / 8,
+    got = sample_from_candidates(p, b, sm, p.cand + (long long)bh * p.cand_cap, p.cand_cnt[bh], bigbytes / 8,
                                  cand0_bound(geo), b0, nw, sm.w2, bs_out, bs_dbg);
   if (got < 0) {
     __syncthreads();
     sample_select<CACHED>(p, sm, s0, l_start, nw, b0, n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
   } else path |= 2;
   if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = path;
-  PHASE(8);
   DEV_END(p, 2);
 }
 
@@ -766,7 +750,7 @@ __global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbyt
   int got = -1;
   if (meta.b < meta.n_s) {
     const long long l1 = (long long)p.B * p.Hq + bh;
-    got = sample_from_candidates(p, sm, p.cand + l1 * p.cand_cap, p.cand_cnt[l1], bigbytes / 8, VATTN_CAND1_BOUND,
+    got = sample_from_candidates(p, b, sm, p.cand + l1 * p.cand_cap, p.cand_cnt[l1], bigbytes / 8, VATTN_CAND1_BOUND,
                                  meta.b, nw, sm.w2, out, dbg);
   }
   if (got < 0) {

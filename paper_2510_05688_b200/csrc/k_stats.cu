@@ -43,14 +43,15 @@ template <> struct Raw<bf16_t> {
 template <typename T>
 struct RowRegs { Raw<T> k, v; };
 
+// K and V slices of the row in physical slot `ph` (= page * 16 + token % 16)
 template <typename T, int D>
-__device__ __forceinline__ void load_row(const Prob& p, int b, int g, int tok, int j, RowRegs<T>& r) {
+__device__ __forceinline__ void load_row(const Prob& p, int g, int ph, int j, RowRegs<T>& r) {
   constexpr int EPL = Elem<T>::EPL;
-  const int pg = page_of(p, b, tok >> 4);
-  const long long off = (long long)pg * p.sb + (long long)g * p.sh + (long long)(tok & 15) * p.st + j * EPL;
+  const long long off = (long long)(ph >> 4) * p.sb + (long long)g * p.sh + (long long)(ph & 15) * p.st + j * EPL;
   r.k.ld(reinterpret_cast<const T*>(p.kc) + off);
   r.v.ld(reinterpret_cast<const T*>(p.vc) + off);
 }
+__device__ __forceinline__ int phys_of(const Prob& p, int b, int tok) { return page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15); }
 // fp64 weight of one token, computed by the LPR lanes of a row group from its K slice
 template <typename T, int D>
 __device__ __forceinline__ double weight64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r, double m) {
@@ -99,8 +100,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const int total = base_cta ? b0 : n_f;
   const int chunk = (total + S - 1) / S;
   const int r_begin = min(total, split * chunk), r_end = min(total, r_begin + chunk);
-  const int* tk = p.topk_idx + (long long)bh * p.npad;
-  const int* bs = p.base_idx + (long long)bh * p.npad;
+  const int* tkph = p.topk_idx + (long long)bh * p.npad + p.phys_delta;     // physical slots of I_t
+  const int* bsph = p.base_idx + (long long)bh * p.npad + p.phys_delta;     // physical slots of I_bs
+  const int ph0 = phys_of(p, b, 0);
   const double m = (double)meta.m;
   const int rsub = lane / LPR, j = lane % LPR;
   const int rg = warp * RPI + rsub;
@@ -116,19 +118,26 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 
   if (!base_cta) {
     // ---------------------------------------------------------------- deterministic rows: sink, I_t, window
-    for (int k0 = 0; k0 < iters; k0 += UN) {
-      int tok[UN];
-      bool act[UN];
-      RowRegs<T> row[UN];
+    // physical slots of the next batch are requested while the current rows are in flight
+    int ph_n[UN];
+    bool act_n[UN];
+    auto fetch = [&](int k0) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        act[u] = (k0 + u < iters) && (r < r_end);
-        tok[u] = 0;
-        if (act[u]) tok[u] = r < s0 ? r : (r < s0 + kk ? __ldg(tk + r - s0) : l_start + (r - s0 - kk));
+        act_n[u] = (k0 + u < iters) && (r < r_end);
+        ph_n[u] = ph0;                                       // idle slots re-read the first row
+        if (act_n[u])
+          ph_n[u] = r < s0 ? phys_of(p, b, r) : (r < s0 + kk ? __ldg(tkph + r - s0) : phys_of(p, b, l_start + (r - s0 - kk)));
       }
+    };
+    fetch(0);
+    for (int k0 = 0; k0 < iters; k0 += UN) {
+      bool act[UN];
+      RowRegs<T> row[UN];
 #pragma unroll
-      for (int u = 0; u < UN; ++u) load_row<T, D>(p, b, g, tok[u], j, row[u]);   // idle slots re-read token 0
+      for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
+      fetch(k0 + UN);
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const double w = weight64<T, D>(p, qf, row[u], m);     // every lane takes part in the shuffles
@@ -142,20 +151,26 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   } else if (b0 > 0) {
     // ---------------------------------------------------------------- base-sample rows, shifted by the pivot
     RowRegs<T> prow;
-    load_row<T, D>(p, b, g, __ldg(bs), j, prow);             // pivot = first base-sample row
-    double cw = 0.0, cr[EPL];
-    for (int k0 = 0; k0 < max(iters, 1); k0 += UN) {
-      int tok[UN];
-      bool act[UN];
-      RowRegs<T> row[UN];
+    const int piv_ph = __ldg(bsph);                          // pivot = first base-sample row
+    int ph_n[UN];
+    bool act_n[UN];
+    auto fetch = [&](int k0) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        act[u] = (k0 + u < iters) && (r < r_end);
-        tok[u] = act[u] ? __ldg(bs + r) : 0;
+        act_n[u] = (k0 + u < iters) && (r < r_end);
+        ph_n[u] = act_n[u] ? __ldg(bsph + r) : piv_ph;
       }
+    };
+    fetch(0);
+    load_row<T, D>(p, g, piv_ph, j, prow);
+    double cw = 0.0, cr[EPL];
+    for (int k0 = 0; k0 < max(iters, 1); k0 += UN) {
+      bool act[UN];
+      RowRegs<T> row[UN];
 #pragma unroll
-      for (int u = 0; u < UN; ++u) load_row<T, D>(p, b, g, tok[u], j, row[u]);
+      for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
+      fetch(k0 + UN);
       if (k0 == 0) {
         cw = weight64<T, D>(p, qf, prow, m);
 #pragma unroll
@@ -207,6 +222,8 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     for (int w = 0; w < NWARP; ++w) s += part[w][e];
     gpart[e] = s;
   }
+  if (base_cta && split == 0 && b0 > 0)              // the pivot travels with this CTA's partial
+    for (int e = tid; e <= D; e += NT) p.stat_piv[(long long)bh * (D + 1) + e] = piv[e];
   DEV_MARK(p, 3, 4, bh == 0 && blockIdx.x == 0);
   __threadfence();
   __syncthreads();
@@ -231,19 +248,8 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     for (int sp = 0; sp < MAXS; ++sp) s += v[sp];
     tot[kind][e] = s;
   }
-  // the pivot again (deterministic: every CTA computes the same numbers), whatever kind this CTA is
-  if (b0 > 0) {
-    RowRegs<T> prow;
-    load_row<T, D>(p, b, g, __ldg(bs), j, prow);
-    const double cw = weight64<T, D>(p, qf, prow, m);
-    if (warp == 0 && rsub == 0) {
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cw * (double)prow.v.get(e);
-      if (j == 0) piv[D] = cw;
-    }
-  } else {
-    for (int e = tid; e <= D; e += NT) piv[e] = 0.0;
-  }
+  // the pivot the base CTAs used (all of them computed the same numbers; split 0 published them)
+  for (int e = tid; e <= D; e += NT) piv[e] = (b0 > 0) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
   __syncthreads();
   DEV_MARK(p, 3, 7, bh == 0);
   double* det = p.det_sums + (long long)bh * (D + 1);

@@ -49,12 +49,14 @@ struct Prob {
   int cand_cap;
   unsigned* status;       // [1]
   unsigned* bitmap;       // [B,Hq,nwords] membership of I_t
-  int* topk_idx;          // [B,Hq,npad]
-  int* base_idx;          // [B,Hq,npad]
-  int* dyn_idx;           // [B,Hq,npad]
+  int* topk_idx;          // [B,Hq,npad] token indices, ascending; the list of physical slots
+  int* base_idx;          // [B,Hq,npad]   (page * 16 + token % 16 of every entry) lies phys_delta
+  int* dyn_idx;           // [B,Hq,npad]   elements behind each index list
+  long long phys_delta;
   HeadMeta* meta;         // [B,Hq]
   double* stat_part;      // [B,Hq,stat_splits,2D+4]
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
+  double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
   float* gat_part;        // [B,Hq,gat_splits,D+1]
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, gat_splits, dense_splits;

@@ -160,6 +160,58 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), out_dev)
 
 
+def test_seeded_random_shapes():
+    # odd sizes, sink + window around n, k from 0 to more than the middle range, ragged batches
+    rng = np.random.default_rng(2024)
+    for trial in range(12):
+        B = int(rng.integers(1, 5))
+        lens = [int(x) for x in rng.integers(1, 601, size=B)]
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 3, 4, 8]))
+        d = int(rng.choice([64, 128]))
+        dtype = str(rng.choice(["bf16", "fp32"]))
+        case = small(dtype, lens, Hq=Hkv * G, Hkv=Hkv, d=d, sink=int(rng.integers(0, 40)), window=int(rng.integers(0, 40)),
+                     k=int(rng.integers(0, 80)), seed=int(rng.integers(0, 2**40)), gen_seed=1000 + trial,
+                     eps=float(rng.choice([0.05, 0.1, 0.3])), delta=float(rng.choice([0.05, 0.2])),
+                     params=dict(base_rate=float(rng.choice([0.025, 0.1, 0.5])), mode=int(rng.integers(0, 3)),
+                                 layer=int(rng.integers(0, 32)), step=int(rng.integers(0, 1000))))
+        check(case)
+
+
+def test_appending_rows_between_steps_reuses_the_plan():
+    # reasoning-length decode: one K/V row per sequence is appended between steps, the step word advances,
+    # nothing but seq_lens and the new rows changes
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    B, n0, steps = 2, 1036, 5
+    full = synth.make_case("grow", dtype="bf16", B=B, Hq=8, Hkv=2, d=128, seq_lens=[n0 + steps] * B, sink=16, window=16,
+                           k=26, eps=0.05, delta=0.05, seed=5, gen_seed=77, rho_v=1.0,
+                           heavy=dict(R=16, c1=6.0, alpha=(0.75, 1.25)), params=dict(base_rate=0.05), poison_unused=False)
+    dev_full = vb.case_to_device(full)
+    # start from caches in which the rows beyond n0 are not written yet
+    kc, vc = dev_full["k_cache"].clone(), dev_full["v_cache"].clone()
+    bt = full.block_table
+    for b in range(B):
+        for i in range(n0, n0 + steps):
+            kc[bt[b, i // 16], :, i % 16] = 0
+            vc[bt[b, i // 16], :, i % 16] = 0
+    plan = vb.plan_for_case(full)
+    out = torch.empty_like(dev_full["q"])
+    for s in range(steps):
+        n = n0 + s
+        for b in range(B):                       # the harness appends row n-1 of every sequence
+            i = n - 1
+            kc[bt[b, i // 16], :, i % 16] = dev_full["k_cache"][bt[b, i // 16], :, i % 16]
+            vc[bt[b, i // 16], :, i % 16] = dev_full["v_cache"][bt[b, i // 16], :, i % 16]
+        case = synth.Case(name="grow", dtype="bf16", q=full.q, k_cache=full.k_cache, v_cache=full.v_cache,
+                          block_table=full.block_table, seq_lens=np.array([n] * B, np.int32), sink=16, window=16,
+                          k=int(0.025 * n), eps=0.05, delta=0.05, seed=5, params=dict(base_rate=0.05, step=s))
+        dev = dict(dev_full, k_cache=kc, v_cache=vc, seq_lens=torch.from_numpy(case.seq_lens).cuda())
+        out_ref, det = run_oracle(case)
+        got, dbg, _ = run_gpu(case, plan=plan, dev=dev)
+        assert_parity(case, got, dbg, det, out_ref)
+
+
 # ----------------------------------------------------------------------------- fast paths and their fallbacks at size
 def mid(**kw):
     args = dict(dtype="bf16", B=1, Hq=8, Hkv=2, d=128, seq_lens=[20000], sink=64, window=64, k=500, eps=0.05,
