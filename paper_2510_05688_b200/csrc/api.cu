@@ -68,7 +68,8 @@ void derive(vattn_plan* pl) {
   // row kernels (128-thread CTAs): one wave of about 5 (statistics, two CTA kinds per split) or 8
   // (gather) CTAs per SM
   int sp = (5 * kNumSM) / (2 * heads);
-  pl->stat_splits = sp < 1 ? 1 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
+  // (when even one CTA per kind and head overfills the wave the kernel is throughput-bound: split freely)
+  pl->stat_splits = sp < 1 ? 4 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
   sp = (8 * kNumSM) / heads;
   pl->gat_splits = sp < 1 ? 1 : (sp > kMaxGatherSplits ? kMaxGatherSplits : sp);
   const int GC = (pl->G + 3) / 4;
@@ -288,7 +289,7 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
     if (rows > msl) rows = msl;
     const double brows = (double)p.base_rate * msl;
     if (brows > rows) rows = brows;
-    int want = (int)((rows + 63.0) / 64.0);
+    int want = (int)((rows + 127.0) / 128.0) * 2;          // about 64 rows per CTA
     if (want < 1) want = 1;
     if (want < p.stat_splits) p.stat_splits = want;
   }

@@ -12,7 +12,8 @@
 //  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
 //    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
 //    grid stride: every SM gets the same number of rows whatever the budgets are;
-//  * per head (larger problems): grid (splits, heads, batch), every head cut into `gat_splits` chunks.
+//  * per head (larger problems): grid (32, heads, batch); a head with budget b uses ceil(b / chunk) of its
+//    32 CTAs, chunk = max(64, ceil(b / 32)) rows, the others exit at once.
 #include "vattn_internal.cuh"
 
 namespace {
@@ -182,13 +183,16 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   __shared__ int is_last;
   __shared__ float s_den;
   DEV_BEGIN(p, 5);
+  pdl_wait();
   const int bh = blockIdx.z * p.Hq + blockIdx.y;
-  const int S = p.gat_splits;
   const HeadMeta meta = p.meta[bh];
   const int nb = meta.n > 0 ? meta.b : 0;
-  const int chunk = (nb + S - 1) / S;
+  // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
+  const int chunk = max(MIN_CHUNK, (nb + MAXS - 1) / MAXS);
+  const int nslots = max(1, (nb + chunk - 1) / chunk);
+  if ((int)blockIdx.x >= nslots) return;
   const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
-  G::run(p, bh, meta, r_begin, r_end, blockIdx.x, S, part, &is_last, &s_den);
+  G::run(p, bh, meta, r_begin, r_end, blockIdx.x, nslots, part, &is_last, &s_den);
   DEV_END(p, 5);
 }
 
@@ -201,6 +205,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __shared__ int s_pref[FLAT_MAX_HEADS + 1], s_rows[FLAT_MAX_HEADS], s_b[FLAT_MAX_HEADS], s_w[NWARP];
   __shared__ HeadMeta s_meta[FLAT_MAX_HEADS];
   DEV_BEGIN(p, 5);
+  pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int BH = p.B * p.Hq;
   // chunk counts of all heads and their prefix sum (every CTA computes the same numbers)
@@ -253,21 +258,21 @@ cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
     const long long most = (long long)BH * MAXS;
     const int grid = (int)(most < 8 * 148 ? most : 8 * 148);
     if (p.dtype == VATTN_DTYPE_BF16) {
-      if (p.D == 128) k_gather_flat<bf16_t, 128><<<grid, NT, 0, s>>>(p);
-      else k_gather_flat<bf16_t, 64><<<grid, NT, 0, s>>>(p);
+      if (p.D == 128) return launch_pdl(k_gather_flat<bf16_t, 128>, dim3(grid), dim3(NT), 0, s, p);
+      else return launch_pdl(k_gather_flat<bf16_t, 64>, dim3(grid), dim3(NT), 0, s, p);
     } else {
-      if (p.D == 128) k_gather_flat<float, 128><<<grid, NT, 0, s>>>(p);
-      else k_gather_flat<float, 64><<<grid, NT, 0, s>>>(p);
+      if (p.D == 128) return launch_pdl(k_gather_flat<float, 128>, dim3(grid), dim3(NT), 0, s, p);
+      else return launch_pdl(k_gather_flat<float, 64>, dim3(grid), dim3(NT), 0, s, p);
     }
     return cudaGetLastError();
   }
-  dim3 grid(p.gat_splits, p.Hq, p.B), block(NT);
+  dim3 grid(MAXS, p.Hq, p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) k_gather<bf16_t, 128><<<grid, block, 0, s>>>(p);
-    else k_gather<bf16_t, 64><<<grid, block, 0, s>>>(p);
+    if (p.D == 128) return launch_pdl(k_gather<bf16_t, 128>, grid, block, 0, s, p);
+    else return launch_pdl(k_gather<bf16_t, 64>, grid, block, 0, s, p);
   } else {
-    if (p.D == 128) k_gather<float, 128><<<grid, block, 0, s>>>(p);
-    else k_gather<float, 64><<<grid, block, 0, s>>>(p);
+    if (p.D == 128) return launch_pdl(k_gather<float, 128>, grid, block, 0, s, p);
+    else return launch_pdl(k_gather<float, 64>, grid, block, 0, s, p);
   }
   return cudaGetLastError();
 }

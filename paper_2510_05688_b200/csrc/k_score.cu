@@ -230,6 +230,7 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
   unsigned* s_cnt = reinterpret_cast<unsigned*>(smem_dyn + (size_t)WARPS * NST * PAGEB + (size_t)16 * CL * sizeof(uint2) +
                                                 (size_t)WARPS * NST * 8);
   DEV_BEGIN(p, 1);
+  pdl_trigger();
   const int b = blockIdx.z;
   const int n = clamped_len(p, b);
   const int npages = (n + 15) >> 4;

@@ -633,6 +633,8 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 2);
+  pdl_trigger();
+  pdl_wait();
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
 
@@ -735,6 +737,8 @@ __global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbyt
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 4);
+  pdl_trigger();
+  pdl_wait();
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   const HeadMeta meta = p.meta[bh];
   if (p.dbg.dyn_cnt && tid == 0) p.dbg.dyn_cnt[bh] = meta.b;
@@ -798,8 +802,7 @@ static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s, bool 
     if (nseen < 32) { seen_fn[nseen] = (const void*)kern; seen_sz[nseen] = smem; ++nseen; }
   }
   dim3 grid(p.Hq, p.B), block(NT);
-  kern<<<grid, block, smem, s>>>(p, big);
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, block, smem, s, p, big);
 }
 
 cudaError_t launch_select_topk_base(const Prob& p, cudaStream_t s) {

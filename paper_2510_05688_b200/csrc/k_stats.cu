@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const bool base_cta = (int)blockIdx.x >= S;
   const int split = base_cta ? blockIdx.x - S : blockIdx.x;
   DEV_BEGIN(p, 3);
+  pdl_trigger();
+  pdl_wait();
   HeadMeta& meta = p.meta[bh];
   const int n = meta.n, s0 = meta.s0, l_start = meta.l_start, kk = meta.kk, n_s = meta.n_s, b0 = meta.b0;
   if (n == 0) {
@@ -324,11 +326,11 @@ cudaError_t launch_stats(const Prob& p, cudaStream_t s) {
   dim3 grid(2 * p.stat_splits, p.Hq, p.B), block(NT);
   if (p.stat_splits < 1 || p.stat_splits > MAXS) return cudaErrorInvalidValue;
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) k_stats<bf16_t, 128><<<grid, block, 0, s>>>(p);
-    else k_stats<bf16_t, 64><<<grid, block, 0, s>>>(p);
+    if (p.D == 128) return launch_pdl(k_stats<bf16_t, 128>, grid, block, 0, s, p);
+    else return launch_pdl(k_stats<bf16_t, 64>, grid, block, 0, s, p);
   } else {
-    if (p.D == 128) k_stats<float, 128><<<grid, block, 0, s>>>(p);
-    else k_stats<float, 64><<<grid, block, 0, s>>>(p);
+    if (p.D == 128) return launch_pdl(k_stats<float, 128>, grid, block, 0, s, p);
+    else return launch_pdl(k_stats<float, 64>, grid, block, 0, s, p);
   }
   return cudaGetLastError();
 }

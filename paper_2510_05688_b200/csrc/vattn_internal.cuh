@@ -77,6 +77,24 @@ __device__ __forceinline__ unsigned long long dev_gtime() { unsigned long long t
 #define DEV_MARK(p, k, slot, cond) do { } while (0)
 #endif
 
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
+// stream is still running; it must call pdl_wait() before touching anything the predecessor writes (the
+// wait returns once the predecessor has completed and its writes are visible).  pdl_trigger() in the
+// predecessor lets the dependent grid start launching early; the dependent still waits for completion.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // small device helpers
 __device__ __forceinline__ unsigned ord_f32(float f) {          // order-preserving float -> uint
