@@ -93,12 +93,14 @@ def oracle_step(case, heads=None):
                           case.k, case.eps, case.delta, case.seed, dtype=case.dtype, heads=heads, **case.params)
 
 
-def oracle_threads():
-    try:
-        from threadpoolctl import threadpool_info
-        return max([1] + [int(p.get("num_threads", 1)) for p in threadpool_info()])
-    except Exception:
-        return 1
+def cpu_seconds():
+    t = os.times()
+    return t.user + t.system
+
+
+def cores_used(cpu_s, wall_s):
+    """Average number of host threads the timed oracle section kept busy (CPU time / wall time)."""
+    return round(max(1.0, cpu_s / max(wall_s, 1e-9)), 1)
 
 
 def run_reference(args, rank, world):
@@ -117,18 +119,18 @@ def run_reference(args, rank, world):
     warm = min(args.warmup, 3)
     for i in range(warm):
         oracle_step(case, heads=[heads_all[i % len(heads_all)]])
-    t0 = time.perf_counter()
+    t0, c0 = time.perf_counter(), cpu_seconds()
     for i in range(steps):
         oracle_step(case, heads=[heads_all[i % len(heads_all)]])
     dt = time.perf_counter() - t0
+    ncores = cores_used(cpu_seconds() - c0, dt)
     us_full = dt / steps * len(heads_all) * 1e6
     sample = (f"each step = 1 of {len(heads_all)} query heads of the workload (K/V de-paging of its KV head "
               f"included), time scaled x{len(heads_all)}; {steps} of the requested {args.steps} steps timed")
     line = {"impl": "reference", "metric": METRIC, "value": us_full, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": us_full / 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
-            "cpu_baseline": {"value": us_full, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                             "sample": sample},
+            "cpu_baseline": {"value": us_full, "unit": UNIT, "cores": ncores, "kind": "oracle", "sample": sample},
             "e2e": {"value": us_full, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -334,8 +336,8 @@ def main():
         "k_select_final": n_tot * Hq // 8,
         "k_gather": int(b_dyn.sum()) * (d * es + 4),
     }
-    # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2.md
-    traffic = {"k_score": 68.41e6, "k_select_topk_base": 4.61e6, "k_stats": 25.60e6, "k_select_final": 2.28e6,
+    # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2_llama8b.md
+    traffic = {"k_score": 68.39e6, "k_select_topk_base": 4.61e6, "k_stats": 25.60e6, "k_select_final": 2.28e6,
                "k_gather": 20.13e6}
     peak, peak_kind = measured_peaks()
     kern = {}
@@ -352,12 +354,13 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        reps, t_cpu0 = 0, time.perf_counter()
+        reps, t_cpu0, c_cpu0 = 0, time.perf_counter(), cpu_seconds()
         while reps < 2 or (time.perf_counter() - t_cpu0 < 10.0 and reps < 16):
             oracle_step(case)
             reps += 1
-        cpu_us = (time.perf_counter() - t_cpu0) / reps * 1e6
-        cpu = {"value": cpu_us, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+        wall = time.perf_counter() - t_cpu0
+        cpu_us = wall / reps * 1e6
+        cpu = {"value": cpu_us, "unit": UNIT, "cores": cores_used(cpu_seconds() - c_cpu0, wall), "kind": "oracle",
                "sample": f"{reps} full steps of the same workload (all 32 heads, fp64 numpy)"}
 
     us_step = ms_step_max * 1e3
