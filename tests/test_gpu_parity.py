@@ -44,6 +44,48 @@ def test_gqa_ratios(Hq, Hkv):
     check(small("bf16", [700, 129], Hq=Hq, Hkv=Hkv))
 
 
+def test_sixteen_heads_per_kv_head():
+    check(small("bf16", [530, 90], Hq=16, Hkv=1))            # G = 16: two chunks of 8 heads in the score pass
+
+
+def test_context_beyond_the_shared_memory_key_cache():
+    # 45,000 tokens: the select kernels take their keys from global memory (generic path)
+    case = synth.make_case("long", dtype="bf16", B=1, Hq=2, Hkv=1, d=128, seq_lens=[45000], sink=64, window=64, k=700,
+                           eps=0.1, delta=0.1, seed=3, gen_seed=808, rho_v=1.0,
+                           heavy=dict(R=64, c1=8.0, alpha=(0.75, 1.25)), params=dict(base_rate=0.02))
+    _, dbg, _, _ = check(case)
+    assert (dbg["paths"] & 1 == 0).all()
+
+
+def test_padded_cache_strides():
+    # rows 16-byte aligned but not contiguous: token stride d + 8, head stride padded, as a caller's cache may be
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [700, 129])
+    d, Hkv, nblk = case.head_dim, case.num_kv_heads, case.num_blocks
+    st, sh = d + 8, 16 * (d + 8) + 24
+    sb = Hkv * sh + 40
+    dev = vb.case_to_device(case)
+
+    def pad(cache):
+        buf = torch.full((nblk * sb,), 7.0, dtype=cache.dtype, device="cuda")
+        view = torch.as_strided(buf, (nblk, Hkv, 16, d), (sb, sh, st, 1))
+        view.copy_(cache)
+        return buf
+    kbuf, vbuf = pad(dev["k_cache"]), pad(dev["v_cache"])
+    plan = vb.Plan(batch=case.batch, num_q_heads=case.num_q_heads, num_kv_heads=Hkv, head_dim=d,
+                   max_blocks_per_seq=case.max_blocks_per_seq, num_blocks=nblk, max_seq_len=case.max_blocks_per_seq * 16,
+                   dtype=vb.DTYPE_BF16, kv_strides=(sb, sh, st))
+    out_ref, det = run_oracle(case)
+    got, dbg, _ = run_gpu(case, plan=plan, dev=dict(dev, k_cache=kbuf, v_cache=vbuf))
+    assert_parity(case, got, dbg, det, out_ref)
+    out = torch.empty_like(dev["q"])
+    plan.dense_decode(dev["q"], kbuf, vbuf, dev["block_table"], dev["seq_lens"], out)
+    torch.cuda.synchronize()
+    ref = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype="bf16")
+    assert (np.abs(out.float().cpu().numpy() - ref) <= 2e-2 * np.maximum(1.0, np.abs(ref))).all()
+
+
 def test_empty_and_covered_sequences():
     case = small("bf16", [0, 5, 12, 300, 0], sink=4, window=8, k=3)
     out, dbg, det, _ = check(case)
