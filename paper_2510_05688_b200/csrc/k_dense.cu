@@ -194,14 +194,275 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// bf16 tensor-core variant.  Same split-KV structure, but every warp streams pages through a ring of
+// shared-memory stages (bulk asynchronous copies, mbarrier transaction counts) and both contractions of
+// a page run on the tensor cores (mma.sync m16n8k16, fp32 accumulate):
+//     S^T[head, token] = q K^T     A = q fragments (heads as M, zero rows above the group size),
+//                                  B = K rows read with 16-byte shared loads (k-slots mapped onto d so
+//                                      that a thread owns 8 consecutive elements of a row)
+//     out[head, dim]  += P V       A = exp(S - m) packed to bf16 straight from the S^T accumulators,
+//                                  B = V through ldmatrix.trans; V rows are copied one by one into rows
+//                                      padded to 272 bytes so the transposing loads are conflict-free
+constexpr int DN_WARPS = 6;
+constexpr int DN_NST = 2;
+
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], const void* smem_row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem_row)));
+}
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // round to nearest even, lo in bits 0..15
+  unsigned r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
+  constexpr int NC = D / 32;                   // 32-element chunks of a K row
+  constexpr int ROWB = D * 2, KPAGE = 16 * ROWB;
+  constexpr int VROWB = ROWB + 16, VPAGE = 16 * VROWB;       // padded V rows
+  constexpr int STAGE = KPAGE + VPAGE;
+  constexpr int NB = D / 8;                    // 8-dim column blocks of the output
+  constexpr int NE = D + 2;
+  extern __shared__ __align__(128) unsigned char smem_dyn[];
+  __shared__ float s_m[DN_WARPS][8], s_l[DN_WARPS][8];
+  __shared__ int is_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int gr = lane >> 2, t = lane & 3;
+  unsigned char* ring = smem_dyn + (size_t)warp * DN_NST * STAGE;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)DN_WARPS * DN_NST * STAGE) + warp * DN_NST;
+  float* s_acc = reinterpret_cast<float*>(smem_dyn);          // [DN_WARPS][8][D], reuses the rings after the main loop
+
+  const int split = blockIdx.x, b = blockIdx.z, S = gridDim.x;
+  const int GC = (p.G + 7) >> 3;
+  const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
+  const int h0 = g * p.G + hc * 8, nh = min(8, p.G - hc * 8);
+  const int n = clamped_len(p, b);
+  const int npages = (n + 15) >> 4;
+  const int wglob = split * DN_WARPS + warp, wtot = S * DN_WARPS;
+  const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;
+  const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
+  const bf16_t* vc = reinterpret_cast<const bf16_t*>(p.vc);
+
+  if (lane < DN_NST) mbar_init(&bars[lane], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+
+  int pg_ids = 0;
+  auto load_ids = [&](int k_base) {
+    const int k = k_base + lane;
+    pg_ids = (k < mine) ? page_of(p, b, wglob + k * wtot) : 0;
+  };
+  // whole warp: lane 0 arms the barrier, then lanes 0..15 copy one V row each (into padded rows) and
+  // lanes 16..31 the K page (one copy, or one row each when rows are not contiguous)
+  auto issue = [&](int k, int pg) {
+    unsigned long long* bar = &bars[k % DN_NST];
+    unsigned char* dst = ring + (size_t)(k % DN_NST) * STAGE;
+    const long long off = (long long)pg * p.sb + (long long)g * p.sh;
+    if (lane == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_expect_tx(bar, 2 * KPAGE);
+    }
+    __syncwarp();
+    if (lane < 16) bulk_g2s(dst + KPAGE + lane * VROWB, vc + off + (long long)lane * p.st, ROWB, bar);
+    else if (p.st == D) { if (lane == 16) bulk_g2s(dst, kc + off, KPAGE, bar); }
+    else bulk_g2s(dst + (lane - 16) * ROWB, kc + off + (long long)(lane - 16) * p.st, ROWB, bar);
+  };
+  load_ids(0);
+  for (int k = 0; k < min(DN_NST, mine); ++k) issue(k, __shfl_sync(0xFFFFFFFFu, pg_ids, k));
+  // q as the A operand: head (h0 + gr) in rows 0..7, rows 8..15 zero
+  uint4 aq[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    aq[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (gr < nh)
+      aq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
+                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
+  }
+  float m_run = -INFINITY, l_run = 0.f;        // head gr of this thread's row; l is this lane's share
+  float acc[NB][2];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) { acc[nb][0] = 0.f; acc[nb][1] = 0.f; }
+  bool failed = false;
+
+  for (int k = 0; k < mine; ++k) {
+    const int s = k % DN_NST;
+    if (!mbar_wait(&bars[s], (unsigned)(k / DN_NST) & 1u)) { failed = true; break; }
+    unsigned char* stg = ring + (size_t)s * STAGE;
+    const int tok0 = (wglob + k * wtot) << 4;
+    if (tok0 + 16 > n) {                       // last page: rows beyond n may hold anything; clear their V
+      for (int r = n - tok0; r < 16; ++r)
+        for (int c = lane; c < ROWB / 4; c += 32) reinterpret_cast<unsigned*>(stg + KPAGE + r * VROWB)[c] = 0u;
+      __syncwarp();
+    }
+    // S^T for tokens 0..7 (sa) and 8..15 (sb): only c[0], c[1] (head gr) are meaningful
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const uint4 klo = *reinterpret_cast<const uint4*>(stg + gr * ROWB + c * 64 + t * 16);
+      const uint4 khi = *reinterpret_cast<const uint4*>(stg + (gr + 8) * ROWB + c * 64 + t * 16);
+      mma_bf16_16816(sa, aq[c].x, 0u, aq[c].y, 0u, klo.x, klo.y);
+      mma_bf16_16816(sa, aq[c].z, 0u, aq[c].w, 0u, klo.z, klo.w);
+      mma_bf16_16816(sb, aq[c].x, 0u, aq[c].y, 0u, khi.x, khi.y);
+      mma_bf16_16816(sb, aq[c].z, 0u, aq[c].w, 0u, khi.z, khi.w);
+    }
+    // this thread: head gr, tokens tok0 + {2t, 2t+1, 8+2t, 9+2t}
+    float sc[4] = {sa[0], sa[1], sb[0], sb[1]};
+    const int tk[4] = {tok0 + 2 * t, tok0 + 2 * t + 1, tok0 + 8 + 2 * t, tok0 + 9 + 2 * t};
+    float mx = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      sc[e] = (tk[e] < n) ? p.scale * sc[e] : -INFINITY;
+      mx = fmaxf(mx, sc[e]);
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);      // a page has at least one valid token, so m_new is finite
+    const float alpha = (m_run == -INFINITY) ? 0.f : __expf(m_run - m_new);
+    float pr[4], psum = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { pr[e] = __expf(sc[e] - m_new); psum += pr[e]; }
+    l_run = l_run * alpha + psum;
+    m_run = m_new;
+    const unsigned pa0 = pack_bf16x2(pr[0], pr[1]), pa2 = pack_bf16x2(pr[2], pr[3]);
+    // out += P V, 16 dims per ldmatrix.x4.trans (two 8-dim column blocks)
+    const int mj = lane >> 3, mr = lane & 7;   // matrix and row this lane addresses
+    const unsigned char* vrow = stg + KPAGE + ((mj & 1) * 8 + mr) * VROWB + (mj >> 1) * 16;
+#pragma unroll
+    for (int nb = 0; nb < NB; nb += 2) {
+      unsigned vb[4];
+      ldmatrix_x4_trans(vb, vrow + nb * 16);
+      float c0[4] = {acc[nb][0] * alpha, acc[nb][1] * alpha, 0.f, 0.f};
+      float c1[4] = {acc[nb + 1][0] * alpha, acc[nb + 1][1] * alpha, 0.f, 0.f};
+      mma_bf16_16816(c0, pa0, 0u, pa2, 0u, vb[0], vb[1]);
+      mma_bf16_16816(c1, pa0, 0u, pa2, 0u, vb[2], vb[3]);
+      acc[nb][0] = c0[0]; acc[nb][1] = c0[1];
+      acc[nb + 1][0] = c1[0]; acc[nb + 1][1] = c1[1];
+    }
+    __syncwarp();
+    if (k + DN_NST < mine) {
+      if (((k + DN_NST) & 31) == 0) load_ids(k + DN_NST);
+      issue(k + DN_NST, __shfl_sync(0xFFFFFFFFu, pg_ids, (k + DN_NST) & 31));
+    }
+  }
+  if (failed) {
+    if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+    for (int s = 0; s < DN_NST; ++s) mbar_wait(&bars[s], 0u) || mbar_wait(&bars[s], 1u);
+  }
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
+  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+  __syncthreads();                             // every warp is done with its ring: reuse it for the partials
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) {
+    s_acc[(warp * 8 + gr) * D + nb * 8 + 2 * t] = acc[nb][0];
+    s_acc[(warp * 8 + gr) * D + nb * 8 + 2 * t + 1] = acc[nb][1];
+  }
+  if (t == 0) { s_m[warp][gr] = m_run; s_l[warp][gr] = l_run; }
+  __syncthreads();
+  // CTA partial -> global: [D] unnormalised sum, m, l per head
+  for (int idx = tid; idx < 8 * NE; idx += DN_WARPS * 32) {
+    const int hh = idx / NE, e = idx % NE;
+    if (hh >= nh) continue;
+    float mc = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < DN_WARPS; ++w) mc = fmaxf(mc, s_m[w][hh]);
+    float val;
+    if (e == D) val = mc;
+    else {
+      val = 0.f;
+#pragma unroll
+      for (int w = 0; w < DN_WARPS; ++w) {
+        const float sc = (s_m[w][hh] == -INFINITY) ? 0.f : __expf(s_m[w][hh] - mc);
+        val += sc * (e < D ? s_acc[(w * 8 + hh) * D + e] : s_l[w][hh]);
+      }
+    }
+    p.dense_part[(((long long)b * p.Hq + h0 + hh) * S + split) * NE + e] = val;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = (atomicAdd(&p.tickets[2 * p.B * p.Hq + b * p.Hq + blockIdx.y], 1u) == (unsigned)(S - 1));
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // last CTA of the group: split maxima and sums first (shared memory), then every output element adds
+  // its S partials with the loads of 8 splits in flight at a time, in split order
+  __shared__ float g_m[8][128], g_sc[8][128], g_den[8];
+  for (int idx = tid; idx < 8 * S; idx += DN_WARPS * 32) {
+    const int hh = idx / S, sp = idx % S;
+    if (hh < nh) g_m[hh][sp] = __ldcg(p.dense_part + (((long long)b * p.Hq + h0 + hh) * S + sp) * NE + D);
+  }
+  __syncthreads();
+  for (int hh = warp; hh < nh; hh += DN_WARPS) {
+    float mg = -INFINITY;
+    for (int sp = lane; sp < S; sp += 32) mg = fmaxf(mg, g_m[hh][sp]);
+#pragma unroll
+    for (int mk = 16; mk >= 1; mk >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xFFFFFFFFu, mg, mk));
+    float den = 0.f;
+    for (int sp0 = 0; sp0 < S; sp0 += 32) {          // fixed order: chunks of 32 splits, lanes in a shuffle tree
+      const int sp = sp0 + lane;
+      float scv = 0.f, lv = 0.f;
+      if (sp < S) {
+        const float ms = g_m[hh][sp];
+        scv = (ms == -INFINITY) ? 0.f : __expf(ms - mg);
+        g_sc[hh][sp] = scv;
+        lv = scv * __ldcg(p.dense_part + (((long long)b * p.Hq + h0 + hh) * S + sp) * NE + D + 1);
+      }
+#pragma unroll
+      for (int mk = 16; mk >= 1; mk >>= 1) lv += __shfl_xor_sync(0xFFFFFFFFu, lv, mk);
+      den += lv;
+    }
+    if (lane == 0) g_den[hh] = den;
+  }
+  __syncthreads();
+  for (int idx = tid; idx < 8 * D; idx += DN_WARPS * 32) {
+    const int hh = idx / D, e = idx % D;
+    if (hh >= nh) continue;
+    const long long bh = (long long)b * p.Hq + h0 + hh;
+    const float* base = p.dense_part + bh * S * NE + e;
+    float num = 0.f;
+    for (int sp0 = 0; sp0 < S; sp0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (sp0 + u < S) ? __ldcg(base + (long long)(sp0 + u) * NE) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) num += (sp0 + u < S) ? g_sc[hh][sp0 + u] * v[u] : 0.f;
+    }
+    reinterpret_cast<bf16_t*>(p.out)[bh * D + e] = Elem<bf16_t>::from_float(n > 0 ? num / g_den[hh] : 0.f);
+  }
+}
+
+template <int D>
+static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
+  constexpr int STAGE = 16 * D * 2 + 16 * (D * 2 + 16);
+  const size_t ring = (size_t)DN_WARPS * DN_NST * STAGE;
+  const size_t accb = (size_t)DN_WARPS * 8 * D * sizeof(float);
+  const size_t smem = (ring > accb ? ring : accb) + DN_WARPS * DN_NST * 8;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(k_dense_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int GC = (p.G + 7) / 8;
+  const int groups = p.B * p.Hkv * GC;
+  int S = (2 * 148 + groups - 1) / groups;               // one wave of two CTAs per SM (registers and shared memory)
+  if (S > p.dense_splits) S = p.dense_splits;
+  if (S < 1) S = 1;
+  dim3 grid(S, p.Hkv * GC, p.B), block(DN_WARPS * 32);
+  k_dense_mma<D><<<grid, block, smem, s>>>(p);
+  return cudaGetLastError();
+}
 }  // namespace
 
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches) {
   const int GC = (p.G + 3) / 4;
   dim3 grid(p.dense_splits, p.Hkv * GC, p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) k_dense<bf16_t, 128><<<grid, block, 0, s>>>(p);
-    else k_dense<bf16_t, 64><<<grid, block, 0, s>>>(p);
+    if (launches) *launches = 1;
+    return p.D == 128 ? launch_dense_mma<128>(p, s) : launch_dense_mma<64>(p, s);
   } else {
     if (p.D == 128) k_dense<float, 128><<<grid, block, 0, s>>>(p);
     else k_dense<float, 64><<<grid, block, 0, s>>>(p);

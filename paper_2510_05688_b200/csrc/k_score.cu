@@ -78,13 +78,6 @@ __device__ void emit_candidates(const Prob& p, int b, int g, int h0, int nh, int
 
 // ---------------------------------------------------------------------------------------------
 // bf16: tensor-core path, up to 8 heads per CTA
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
-                                               unsigned b0, unsigned b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 // ---------------------------------------------------------------------------------------------
 // bf16, streaming variant: every warp owns a ring of NST shared-memory stages and keeps NST pages
 // (16 tokens x d, one contiguous slab of the paged cache) in flight with bulk asynchronous copies
@@ -93,34 +86,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsig
 // resident CTAs.  A warp walks the pages p = w, w + W, w + 2W, ... of its (batch row, KV head).
 constexpr int NST = 4;          // stages per warp
 constexpr int CWARPS = 8;       // warps of a CTA that pre-filter sampling keys (two per streaming warp)
-constexpr unsigned WAIT_SPINS = 1u << 20;
-
-__device__ __forceinline__ unsigned smem_u32(const void* ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
-  unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// bounded wait: gives up after WAIT_SPINS polls and reports it
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  for (unsigned it = 0; it < WAIT_SPINS; ++it) {
-    __nanosleep(64);                      // leave the issue slots to the warps that have work
-    if (mbar_try_wait(bar, parity)) return true;
-  }
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes, unsigned long long* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
 
 // Sampling-candidate pre-filter, run by the CWARPS candidate warps of a CTA: Philox keys of streams 0
 // and 1 for every (token, head) of the CTA's pages; tokens whose key is below the stream's bound are
