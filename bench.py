@@ -136,6 +136,69 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def time_other_configs(vb, synth, torch, steps=40, pools=3):
+    """Sparse step and own dense kernel on the other workload configurations (plain launches back to
+    back on the current stream, rotating over `pools` copies of the cache so the L2 is not warm)."""
+    out = {}
+
+    def run(name, case, **over):
+        dev0 = vb.case_to_device(case)
+        devs = [dev0] + [dict(dev0, k_cache=dev0["k_cache"].clone(), v_cache=dev0["v_cache"].clone())
+                         for _ in range(pools - 1)]
+        plan = vb.plan_for_case(case)
+        params = dict(case.params)
+        params.update(over)
+        plan.set_params(**params)
+        o = torch.empty_like(dev0["q"])
+        dbg = plan.enable_debug()
+
+        def sparse(i):
+            d = devs[i % pools]
+            plan.decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], case.sink, case.window,
+                        case.k, case.eps, case.delta, case.seed, o)
+
+        def dense(i):
+            d = devs[i % pools]
+            plan.dense_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], o)
+        sparse(0)
+        torch.cuda.synchronize()
+        n = case.seq_lens.astype(np.float64)[:, None]
+        dens = float(np.mean((dbg["topk_cnt"].cpu().numpy() + min(case.sink, int(n.max())) + min(case.window, int(n.max()))
+                              + dbg["dyn_cnt"].cpu().numpy())[case.seq_lens > 0] / n[case.seq_lens > 0]))
+        plan.disable_debug()
+        res = {"mean_density": round(dens, 4)}
+        for label, fn in (("sparse_us", sparse), ("dense_us", dense)):
+            for i in range(3):
+                fn(i)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            res[label] = round(e0.elapsed_time(e1) / steps * 1e3, 1)
+        plan.set_profiling(True)
+        for i in range(10):
+            sparse(i)
+        torch.cuda.synchronize()
+        prof, calls = plan.read_profile()
+        plan.set_profiling(False)
+        res["kernels_us"] = {k_: round(v / max(calls, 1) * 1e3, 1) for k_, v in prof.items()}
+        out[name] = res
+        del devs, plan
+
+    run("cfg1_tiny", synth.config1_tiny())
+    c3 = synth.config3_uniform()
+    n_f = 128 + 128 + c3.k
+    run("cfg3_uniform_natural", c3)
+    for S in (5, 10, 20):
+        run(f"cfg3_uniform_{S}x", c3, force_budget=round(32768 / S) - n_f)
+    run("cfg5_reasoning_B8_n32768", synth.config5_reasoning(n=32768, B=8))
+    run("cfg4_serving_B32", synth.config4_serving(), )
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -145,6 +208,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--flashinfer", action="store_true",
                     help="also time FlashInfer's paged batch decode (third-party dense kernel) as external context")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="also time the other workload configurations (tiny, near-uniform sweep, batched serving, "
+                         "reasoning-length) and add them to the JSON line as `other_configs`")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
     args = ap.parse_args()
@@ -317,6 +383,10 @@ def main():
         torch.cuda.synchronize()
         ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
+    other = None
+    if args.all_configs and rank == 0:
+        other = time_other_configs(vb, synth, torch)
+
     ms_step_max = max_over_ranks(ms_step, world)
     ms_e2e_max = max_over_ranks(ms_e2e, world)
     ms_dense_max = max_over_ranks(ms_dense, world)
@@ -390,6 +460,8 @@ def main():
         "cpu_baseline": cpu,
         "clocks": clocks,
     }
+    if other is not None:
+        line["other_configs"] = other
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

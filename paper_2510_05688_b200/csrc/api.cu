@@ -69,7 +69,7 @@ void derive(vattn_plan* pl) {
   // (gather) CTAs per SM
   int sp = (5 * kNumSM) / (2 * heads);
   // (when even one CTA per kind and head overfills the wave the kernel is throughput-bound: split freely)
-  pl->stat_splits = sp < 1 ? 4 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
+  pl->stat_splits = sp < 4 ? 4 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
   sp = (8 * kNumSM) / heads;
   pl->gat_splits = sp < 1 ? 1 : (sp > kMaxGatherSplits ? kMaxGatherSplits : sp);
   const int GC = (pl->G + 3) / 4;

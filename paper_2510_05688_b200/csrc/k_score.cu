@@ -446,7 +446,10 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   // one wave of two CTAs per SM; a warp walks pages with stride (CTAs along x) * WARPS
   const int groups = p.Hkv * ((p.G + 7) / 8) * p.B;
   const int pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
-  int cx = (2 * 148 + groups - 1) / groups;
+  // one wave when the (batch row, KV head) groups leave room for it; with more groups than SMs the
+  // sequences are ragged anyway: cut them finer (about two waves) so that long ones do not set the time
+  int cx = groups <= 148 ? (2 * 148) / groups : (4 * 148 + groups - 1) / groups;
+  if (groups > 148 && cx < 2) cx = 2;
   const int cx_max = (pages + WARPS - 1) / WARPS;
   if (cx > cx_max) cx = cx_max;
   if (cx < 1) cx = 1;
