@@ -19,7 +19,7 @@ struct vattn_plan {
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
   int prof_calls;           // calls recorded since the last read
   // derived
-  int G, npad, nwords, stat_splits, gat_splits, dense_splits;
+  int G, npad, nwords, stat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
       off_det, off_piv, off_gat, off_dense, off_cand, total;
   int cand_cap;
@@ -65,13 +65,10 @@ void derive(vattn_plan* pl) {
   if (pl->npad == 0) pl->npad = 32;
   pl->nwords = pl->npad / 32;
   const int heads = s.batch * s.num_q_heads;
-  // row kernels (128-thread CTAs): one wave of about 5 (statistics, two CTA kinds per split) or 8
-  // (gather) CTAs per SM
+  // statistics kernel (128-thread CTAs, two CTA kinds per split): one wave of about 5 CTAs per SM
   int sp = (5 * kNumSM) / (2 * heads);
   // (when even one CTA per kind and head overfills the wave the kernel is throughput-bound: split freely)
   pl->stat_splits = sp < 4 ? 4 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
-  sp = (8 * kNumSM) / heads;
-  pl->gat_splits = sp < 1 ? 1 : (sp > kMaxGatherSplits ? kMaxGatherSplits : sp);
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
   sp = (4 * kNumSM + groups - 1) / groups;
@@ -140,7 +137,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
-  p.stat_splits = pl->stat_splits; p.gat_splits = pl->gat_splits; p.dense_splits = pl->dense_splits;
+  p.stat_splits = pl->stat_splits; p.dense_splits = pl->dense_splits;
   p.dbg = pl->dbg;
   p.devt = pl->devt;
   return VATTN_OK;

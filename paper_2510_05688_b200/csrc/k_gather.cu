@@ -251,7 +251,6 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
 }  // namespace
 
 cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
-  if (p.gat_splits < 1 || p.gat_splits > MAXS) return cudaErrorInvalidValue;
   const int BH = p.B * p.Hq;
   if (BH <= FLAT_MAX_HEADS) {
     // at most 32 chunks of >= 64 rows per head; 8 CTAs per SM walk them with a grid stride

@@ -779,11 +779,6 @@ static int big_bytes(const Prob& p, bool final_kernel) {
   return (int)b;
 }
 
-size_t select_smem_bytes(const Prob& p) {
-  return sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
-         sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64) + (size_t)big_bytes(p, true);
-}
-
 // Opt-in to large dynamic shared memory once per kernel and size (a function attribute, not a
 // stream operation; done before the first launch so that later launches can be stream-captured).
 template <typename KernelT>

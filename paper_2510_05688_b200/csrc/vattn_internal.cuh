@@ -54,12 +54,12 @@ struct Prob {
   int* dyn_idx;           // [B,Hq,npad]   elements behind each index list
   long long phys_delta;
   HeadMeta* meta;         // [B,Hq]
-  double* stat_part;      // [B,Hq,stat_splits,2D+4]
+  double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (det CTAs, then base CTAs)
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
   double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
-  float* gat_part;        // [B,Hq,gat_splits,D+1]
+  float* gat_part;        // [B,Hq,32,D+1]    partials of the gather kernel, one per chunk
   float* dense_part;      // [B,Hq,dense_splits,D+2]
-  int stat_splits, gat_splits, dense_splits;
+  int stat_splits, dense_splits;
   vattn_debug dbg;
   unsigned long long* devt;   // development timing buffer [8][32] (null unless a dev build sets it)
 };
@@ -246,4 +246,3 @@ cudaError_t launch_select_final(const Prob& p, cudaStream_t s);
 cudaError_t launch_stats(const Prob& p, cudaStream_t s);
 cudaError_t launch_gather(const Prob& p, cudaStream_t s);
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches);
-size_t select_smem_bytes(const Prob& p);
