@@ -188,7 +188,8 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   const HeadMeta meta = p.meta[bh];
   const int nb = meta.n > 0 ? meta.b : 0;
   // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
-  const int chunk = max(MIN_CHUNK, (nb + MAXS - 1) / MAXS);
+  // (with this many heads the kernel is throughput-bound: 4 batches per row group amortise the fixed hops)
+  const int chunk = max(4 * MIN_CHUNK, (nb + MAXS - 1) / MAXS);
   const int nslots = max(1, (nb + chunk - 1) / chunk);
   if ((int)blockIdx.x >= nslots) return;
   const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);

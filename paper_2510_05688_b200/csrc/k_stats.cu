@@ -52,16 +52,37 @@ __device__ __forceinline__ void load_row(const Prob& p, int g, int ph, int j, Ro
   r.v.ld(reinterpret_cast<const T*>(p.vc) + off);
 }
 __device__ __forceinline__ int phys_of(const Prob& p, int b, int tok) { return page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15); }
-// fp64 weight of one token, computed by the LPR lanes of a row group from its K slice
+// fp64 inner product <q, K[row]> computed by the LPR lanes of a row group from their K slices
 template <typename T, int D>
-__device__ __forceinline__ double weight64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r, double m) {
+__device__ __forceinline__ double dot64(const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r) {
   constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
   double acc = 0.0;
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc = fma((double)qf[e], (double)r.k.get(e), acc);
 #pragma unroll
   for (int mask = LPR / 2; mask >= 1; mask >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, mask);
-  return exp(acc * (double)p.scale - m);
+  return acc;
+}
+// fp64 weight of one token
+template <typename T, int D>
+__device__ __forceinline__ double weight64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r, double m) {
+  return exp(dot64<T, D>(qf, r) * (double)p.scale - m);
+}
+// weights of the UN rows of a batch with ONE exp per lane: lane j of the row group evaluates the row
+// j % UN, the results are handed round with shuffles (every lane of a group holds all UN inner products)
+template <typename T, int D>
+__device__ __forceinline__ void weights64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T> (&row)[UN],
+                                          double m, int j, double (&w)[UN]) {
+  constexpr int LPR = D / Elem<T>::EPL;
+  static_assert(UN == 4 && LPR >= UN, "one lane per row of the batch");
+  double d[UN];
+#pragma unroll
+  for (int u = 0; u < UN; ++u) d[u] = dot64<T, D>(qf, row[u]);
+  const int mu = j & (UN - 1);
+  const double mine = mu == 0 ? d[0] : (mu == 1 ? d[1] : (mu == 2 ? d[2] : d[3]));
+  const double wm = exp(mine * (double)p.scale - m);
+#pragma unroll
+  for (int u = 0; u < UN; ++u) w[u] = __shfl_sync(0xFFFFFFFFu, wm, u, LPR);
 }
 
 __device__ __forceinline__ int ceil_sat(double x) {
@@ -140,9 +161,11 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
       fetch(k0 + UN);
+      double wv[UN];
+      weights64<T, D>(p, qf, row, m, j, wv);                   // every lane takes part in the shuffles
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
-        const double w = weight64<T, D>(p, qf, row[u], m);     // every lane takes part in the shuffles
+        const double w = wv[u];
         if (act[u]) {
           s1 += w;
 #pragma unroll
@@ -183,9 +206,11 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
           if (j == 0) piv[D] = cw;
         }
       }
+      double wv[UN];
+      weights64<T, D>(p, qf, row, m, j, wv);
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
-        const double w = weight64<T, D>(p, qf, row[u], m);
+        const double w = wv[u];
         if (act[u]) {
           const double dw = w - cw;
           s1 += dw;
