@@ -75,15 +75,16 @@ typedef struct {
 /* Optional per-call introspection.  All DEVICE pointers; NULL = not wanted.  cap = max_seq_len. */
 typedef struct {
   int32_t *topk_idx, *topk_cnt;   /* [B,Hq,cap], [B,Hq]  I_t ascending (I_f = sink range + I_t + window range) */
-  int32_t *base_idx, *base_cnt;   /* I_bs ascending, b0 */
-  int32_t *dyn_idx,  *dyn_cnt;    /* I_dyn ascending, b */
+  int32_t *base_idx, *base_cnt;   /* I_bs, b0: in ascending (Philox key, token) order when drawn from the sorted
+                                     candidate list (paths bit 1), in ascending token order otherwise: a set */
+  int32_t *dyn_idx,  *dyn_cnt;    /* I_dyn, b: likewise (paths bit 2) */
   int32_t *budgets;               /* [B,Hq,4] ceil(b_D), ceil(b_N), ceil(b_SDPA) (saturating at 2^31-1), b */
   double  *stats;                 /* [B,Hq,8] D_f, sigma^2, Tr(Sigma), D_hat, |N_hat|_2, n_s, b0, m (weights are
                                      exp(s - m) with m the head's largest fp32 score) */
   float   *scores;                /* [B,Hq,cap] fp32 scores s_i = scale * <K[i], q> */
   int32_t *paths;                 /* [B,Hq] which code path selected each set: bit 0 top-k from the sampled threshold
-                                     estimate, bit 1 base sample from the pre-filtered list, bit 2 final sample from
-                                     the pre-filtered list (a clear bit = the full-context select ran) */
+                                     estimate, bit 1 base sample from the pre-filtered list, bit 2 final sample =
+                                     prefix of the pre-sorted list (a clear bit = the full-context select ran) */
 } vattn_debug;
 
 /* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG, UNSUPPORTED. */
@@ -171,12 +172,14 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */)
 int vattn_last_launch_count(const vattn_plan* plan);
 
 /* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
- * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, select top-k +
- * base sample, statistics + budget, select final sample, gather + combine), for up to 256 calls
- * between two reads.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
+ * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, top-k select,
+ * sampling sort, statistics + budget, slow-path final select, gather + combine), for up to 256 calls
+ * between two reads.  The events serialise kernels that otherwise overlap (the sampling sort runs beside
+ * the top-k select, the first half of the statistics beside the sampling), so the per-kernel times add up
+ * to more than an unprofiled step takes.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
  * milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to *calls
  * (host), and starts a new window.  Events add a little latency: do not enable in production. */
-#define VATTN_NUM_KERNELS 5
+#define VATTN_NUM_KERNELS 6
 int vattn_set_profiling(vattn_plan* plan, int enable);
 int vattn_read_profile(vattn_plan* plan, float* ms_sum, int* calls);
 

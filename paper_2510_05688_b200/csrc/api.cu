@@ -21,7 +21,7 @@ struct vattn_plan {
   // derived
   int G, npad, nwords, stat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
-      off_det, off_piv, off_gat, off_dense, off_cand, total;
+      off_det, off_piv, off_gat, off_dense, off_cand, off_sort, total;
   int cand_cap;
 };
 
@@ -95,6 +95,7 @@ void derive(vattn_plan* pl) {
     pl->cand_cap = ((int)(q4 + 8.0 * sqrt(q4) + 64.0) + 31) / 32 * 32;
   }
   pl->off_cand = take(2 * BH * (size_t)pl->cand_cap * sizeof(uint2));
+  pl->off_sort = take(2 * BH * (size_t)pl->cand_cap * sizeof(int));       // sorted tokens, then physical slots
   pl->total = off;
 }
 
@@ -125,6 +126,8 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.cand_cnt = p.tickets + 3 * BH;
   p.cand = reinterpret_cast<uint2*>(w + pl->off_cand);
   p.cand_cap = pl->cand_cap;
+  p.sort_idx = reinterpret_cast<int*>(w + pl->off_sort);
+  p.sort_phys_delta = (long long)BH * pl->cand_cap;
   p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
   p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);
   p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
@@ -306,14 +309,18 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   if (p.dbg.scores)
     CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
                          sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
-  CU(launch_select_topk_base(p, st)); plan->last_launches++;
+  // score -> top-k -> sampling (its sort runs concurrently with top-k, before its dependency wait) ->
+  // statistics + budget -> slow-path select (usually nothing to do) -> gather.
+  CU(launch_select_topk(p, st));      plan->last_launches++;
   prof_mark(plan, 2, st);
-  CU(launch_stats(p, st));            plan->last_launches++;
+  CU(launch_presort(p, st));          plan->last_launches++;
   prof_mark(plan, 3, st);
-  CU(launch_select_final(p, st));     plan->last_launches++;
+  CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 4, st);
-  CU(launch_gather(p, st));           plan->last_launches++;
+  CU(launch_select_final(p, st));     plan->last_launches++;
   prof_mark(plan, 5, st);
+  CU(launch_gather(p, st));           plan->last_launches++;
+  prof_mark(plan, 6, st);
   if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
   return VATTN_OK;
 }

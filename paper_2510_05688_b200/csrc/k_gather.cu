@@ -49,8 +49,11 @@ struct Gather {
       if (slot == 0) for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
       return;
     }
-    const int* dyn = p.dyn_idx + (long long)bh * p.npad;
-    const int* dph = dyn + p.phys_delta;
+    // I_dyn: the first b entries of the pre-sorted residual list when the budget fits it, else the list the
+    // slow-path select wrote (same predicate as in k_select_final)
+    const bool presorted = meta.b < meta.n_s && meta.sorted_cnt >= meta.b;
+    const int* dyn = presorted ? p.sort_idx + (long long)bh * p.cand_cap : p.dyn_idx + (long long)bh * p.npad;
+    const int* dph = dyn + (presorted ? p.sort_phys_delta : p.phys_delta);
     const float* sc = p.scores + (long long)bh * p.npad;
     const T* vc = reinterpret_cast<const T*>(p.vc) + (long long)g * p.sh;
     const float m = meta.m;
@@ -100,6 +103,7 @@ struct Gather {
       }
     }
     DEV_MARK(p, 5, 3, blockIdx.x == 0);
+    DEV_AT(p, 256 + blockIdx.x * 4 + 1);
 #ifdef VATTN_DEV_TIMING
     if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 8], dev_gtime());
 #endif
@@ -235,6 +239,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __syncthreads();
   const int total = s_pref[BH];
   DEV_MARK(p, 5, 2, blockIdx.x == 0);
+  DEV_AT(p, 256 + blockIdx.x * 4);
   for (int c = blockIdx.x; c < total; c += gridDim.x) {
     int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
     while (lo < hi) {

@@ -1,21 +1,23 @@
 // Index selection: one CTA per (batch row, query head).
 //
-//  k_select_topk_base : I_t = the k middle tokens with the largest score, ties to the lowest index
-//                       (Algorithm 1 line 3, "oracle top-k" of Sec. 3), then the base sample
-//                       I_bs = uniform-sample of b0 residual tokens (Algorithm 2 line 1).
-//  k_select_final     : I_dyn = uniform-sample of b residual tokens (Algorithm 1 line 7).
+//  k_select_topk  : I_t = the k middle tokens with the largest score, ties to the lowest index
+//                   (Algorithm 1 line 3, "oracle top-k" of Sec. 3).
+//  k_presort      : the base sample I_bs = uniform-sample of b0 residual tokens (Algorithm 2 line 1) and the
+//                   residual in the order in which the final sample draws it (Algorithm 1 line 7).
+//  k_select_final : I_dyn = uniform-sample of b residual tokens, for the heads k_presort could not serve.
 //
-// Both selections are "the c smallest (key, index) pairs": an 8-bit-digit radix select over 32-bit
-// keys held in shared memory, followed by an ordered compaction through bitmaps, so every list comes
-// out ascending.  Keys are the order-reversed score for top-k and Philox4x32-10 words for sampling.
+// All selections are "the c smallest (key, index) pairs".  The generic form is an 8-bit-digit radix select
+// over 32-bit keys held in shared memory, followed by an ordered compaction through bitmaps, so its lists
+// come out ascending.  Keys are the order-reversed score for top-k and Philox4x32-10 words for sampling.
 //
 // Fast paths (one pass over the context instead of four): the top-k threshold is first estimated from a
 // strided sample of the scores (1024 linear bins between the sample minimum and the head maximum), one
 // pass collects the few thousand tokens above the estimate, and the exact radix select runs on those
-// candidates only.  Sampling draws from the candidate lists the score kernel pre-filtered (tokens whose
+// candidates only.  Sampling sorts the candidate lists the score kernel pre-filtered (tokens whose
 // Philox key is below a bound): if the list holds at least c residual tokens, the c smallest keys of
-// the residual are all in it.  Whenever an estimate fails (too few / too many candidates, list
-// overflow, near-tie band reaching below the estimate) the generic full-context select runs instead.
+// the residual are its first c residual entries.  Whenever an estimate fails (too few / too many
+// candidates, list overflow, near-tie band reaching below the estimate) the generic full-context select
+// runs instead.
 //
 // Exact top-k from fp32 scores: the stored scores differ from the exact inner products by at most
 // gamma (a bound from the summation structure of the score kernel).  After the fp32 threshold T is
@@ -287,80 +289,6 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sampling from a pre-filtered candidate list: `cnt` (key, token) pairs in global memory whose keys
-// are below `bound`.  Succeeds (returns the number emitted, = c) when the list is complete and holds
-// at least c residual tokens; returns -1 when the caller has to draw from the full context.
-// The c-th smallest (key, token) pair is located with one linear-bin histogram over [0, bound) (the
-// keys are uniform, so a bin holds a handful of pairs) and an exact ranking inside that bin.
-__device__ int sample_from_candidates(const Prob& p, int b, const Sm& sm, const uint2* glist, unsigned cnt, int paircap,
-                                      unsigned bound, int c, int nw, const unsigned* it, int* out_a, int* out_b) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  if (bound == 0u || cnt > (unsigned)p.cand_cap || cnt > (unsigned)paircap || (int)cnt < c) return -1;
-  uint2* pr = reinterpret_cast<uint2*>(sm.keys);
-  int* misc = sm.misc;
-  const float bscale = (float)NBIN / (float)bound;
-  auto bin_of = [&](unsigned key) -> int { const int x = (int)((float)key * bscale); return x > NBIN - 1 ? NBIN - 1 : x; };
-  sm.lin[tid] = 0;
-  if (tid == 0) { misc[2] = 0; misc[3] = 0; misc[4] = -1; }
-  __syncthreads();
-  int nvalid_local = 0;
-  for (int j = tid; j < (int)cnt; j += NT) {
-    uint2 e = glist[j];
-    const bool resid = !((it[e.y >> 5] >> (e.y & 31)) & 1u);
-    if (!resid) e.y |= 0x80000000u;                         // tokens of I_t stay in the list, marked
-    else atomicAdd(&sm.lin[bin_of(e.x)], 1);
-    pr[j] = e;
-    nvalid_local += resid;
-  }
-#pragma unroll
-  for (int mk = 16; mk >= 1; mk >>= 1) nvalid_local += __shfl_xor_sync(0xFFFFFFFFu, nvalid_local, mk);
-  if (lane == 0 && nvalid_local) atomicAdd(&misc[2], nvalid_local);
-  __syncthreads();
-  DEV_MARK(p, 6, 2, blockIdx.x == 0 && blockIdx.y == 0);
-  if (misc[2] < c) return -1;
-  const int mycnt = sm.lin[tid];
-  __syncthreads();
-  block_excl_scan(sm.lin, NBIN, misc);
-  const int excl = sm.lin[tid];
-  if (excl < c && c <= excl + mycnt) { misc[4] = tid; misc[5] = c - excl; }
-  __syncthreads();
-  const int jb = misc[4], r_in = misc[5];                   // the c-th smallest pair is the r_in-th of bin jb
-  DEV_MARK(p, 6, 3, blockIdx.x == 0 && blockIdx.y == 0);
-  for (int w = tid; w < nw; w += NT) sm.w0[w] = 0u;
-  for (int j = tid; j < (int)cnt; j += NT) {
-    const uint2 e = pr[j];
-    if ((e.y & 0x80000000u) || bin_of(e.x) != jb) continue;
-    const int pos = atomicAdd(&misc[3], 1);
-    if (pos < VATTN_BANDCAP) { sm.band_idx[pos] = j; }
-  }
-  __syncthreads();
-  const int nmem = misc[3];
-  if (nmem > VATTN_BANDCAP) return -1;
-  for (int a = tid; a < nmem; a += NT) {
-    const uint2 mine = pr[sm.band_idx[a]];
-    int rank = 0;
-    for (int u = 0; u < nmem; ++u) {
-      const uint2 o = pr[sm.band_idx[u]];
-      rank += (o.x < mine.x) || (o.x == mine.x && o.y < mine.y);
-    }
-    if (rank == r_in - 1) { misc[6] = (int)mine.x; misc[7] = (int)mine.y; }
-  }
-  __syncthreads();
-  const unsigned Tkey = (unsigned)misc[6], Tidx = (unsigned)misc[7];
-  DEV_MARK(p, 6, 4, blockIdx.x == 0 && blockIdx.y == 0);
-  for (int j = tid; j < (int)cnt; j += NT) {
-    const uint2 e = pr[j];
-    if (e.y & 0x80000000u) continue;
-    if (e.x < Tkey || (e.x == Tkey && e.y <= Tidx)) atomicOr(&sm.w0[e.y >> 5], 1u << (e.y & 31));
-  }
-  __syncthreads();
-  DEV_MARK(p, 6, 5, blockIdx.x == 0 && blockIdx.y == 0);
-  const int got = finalize_emit(p, b, sm.w0, sm.w1, 0, nw, sm.scan, sm.misc, out_a, out_b);
-  DEV_MARK(p, 6, 6, blockIdx.x == 0 && blockIdx.y == 0);
-  return got;
-}
-
-// ---------------------------------------------------------------------------------------------
 // top-k, fast path: requires the inverted ordered score keys of [s0, l_start) in sm.keys.
 //  1. a strided sample of the scores is binned linearly between its minimum and the head maximum; the
 //     bin edge below which about kk + margin tokens are expected becomes the candidate threshold U;
@@ -627,14 +555,14 @@ __device__ void topk_generic(const Prob& p, const Sm& sm, int b, int g, const T*
 }
 
 template <typename T, int D, bool CACHED>
-__global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bigbytes) {
+__global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 2);
-  pdl_trigger();
   pdl_wait();
+  pdl_trigger();                      // dependents may read the score kernel's outputs before their own wait
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
 
@@ -714,22 +642,192 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk_base(const Prob p, int bi
   __syncthreads();
   DEV_MARK(p, 2, 5, bh == 0);
 
-  // ------------------------------------------------------------------ base sample (Philox stream 0)
-  const int hrng = p.rng_head_is_kv ? g : h;
-  int* bs_out = p.base_idx + (long long)bh * p.npad;
-  int* bs_dbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
-  int got = -1;
-  if (b0 > 0 && b0 < n_s)
-    got = sample_from_candidates(p, b, sm, p.cand + (long long)bh * p.cand_cap, p.cand_cnt[bh], bigbytes / 8,
-                                 cand0_bound(geo), b0, nw, sm.w2, bs_out, bs_dbg);
-  if (got < 0) {
-    __syncthreads();
-    sample_select<CACHED>(p, sm, s0, l_start, nw, b0, n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
-  } else path |= 2;
   if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = path;
   DEV_END(p, 2);
 }
 
+// Sampling without a selection on the critical path (Algorithm 2 line 1 and Algorithm 1 line 7).
+// grid.z = Philox stream: 0 draws the base sample I_bs, 1 prepares the final sample I_dyn.
+//
+// "The c smallest (key, token) pairs of the residual" is a prefix of the residual's pairs in sorted order,
+// whatever c is.  The pre-filtered candidate list of the score kernel holds every middle token whose key
+// is below a bound, so sorting it needs nothing from the top-k selection: it happens BEFORE this grid's
+// dependency wait, while k_select_topk still runs on other SMs (counting sort into 4096 buckets by a
+// monotone function of the key, then every pair ranks itself inside its bucket).  After the wait only the
+// members of I_t are dropped, by an order-preserving compaction: stream 0 keeps the first b0 survivors,
+// stream 1 all of them (the gather kernel later reads the first b, once b is known).  Lists that cannot
+// serve (overflow, too long for shared memory, fewer than b0 survivors, b0 = whole residual) fall back to
+// the full-context select: here for stream 0, in k_select_final for stream 1 (sorted_cnt = -1).
+constexpr int SORT_BUCKETS = 4096;
+constexpr int SORT_BUCKET_MAX = 64;
+constexpr size_t SORT_FIXED_BYTES = sizeof(int) * (2 * SORT_BUCKETS + 1 + 64);      // + nwords words
+template <bool CACHED>
+__global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, int bigbytes) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.x, b = blockIdx.y, stream = blockIdx.z, g = h / p.G;
+  const int bh = b * p.Hq + h;
+  const int devk = stream ? 7 : 0;
+  (void)devk;
+  DEV_BEGIN(p, devk);
+  uint2* pairs = reinterpret_cast<uint2*>(smem_raw);          // [paircap] bucketed (key, token), later sorted (token, slot)
+  int* srt = reinterpret_cast<int*>(pairs + paircap);         // [paircap] tokens in sorted order
+  int* off = srt + paircap;                                   // [SORT_BUCKETS + 1] bucket starts
+  int* cur = off + SORT_BUCKETS + 1;                          // [SORT_BUCKETS] fill cursors
+  int* misc = cur + SORT_BUCKETS;                             // [64]
+  unsigned* bits = reinterpret_cast<unsigned*>(misc + 64);    // [nwords] bitmap of I_t
+
+  // ------------------------------------------------ before the wait: step inputs and score-kernel lists only
+  const int n = clamped_len(p, b);
+  const Geo geo = head_geometry(p, n);
+  const long long l = (long long)stream * p.B * p.Hq + bh;
+  const unsigned bound = stream ? VATTN_CAND1_BOUND : cand0_bound(geo);
+  bool usable = n > 0 && geo.n_s > 0 && bound != 0u && (stream == 1 || geo.b0 < geo.n_s);
+  unsigned cnt = 0;
+  if (usable) {
+    cnt = __ldcg(p.cand_cnt + l);
+    usable = cnt <= (unsigned)p.cand_cap && cnt <= (unsigned)paircap;
+  }
+  int nall = 0;
+  if (usable) {
+    const uint2* glist = p.cand + l * p.cand_cap;
+    const float bscale = (float)SORT_BUCKETS / (float)bound;
+    auto bucket_of = [&](unsigned key) -> int {               // monotone in key
+      const int x = (int)((float)key * bscale);
+      return x > SORT_BUCKETS - 1 ? SORT_BUCKETS - 1 : x;
+    };
+    for (int j = tid; j <= SORT_BUCKETS; j += NT) off[j] = 0;
+    if (tid == 0) misc[0] = 0;
+    __syncthreads();
+    for (int j0 = tid; j0 < (int)cnt; j0 += 4 * NT) {
+      uint2 e[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) e[u] = (j0 + u * NT < (int)cnt) ? __ldcg(glist + j0 + u * NT) : make_uint2(0u, 0xFFFFFFFFu);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (e[u].y < (unsigned)n) atomicAdd(&off[bucket_of(e[u].x)], 1);
+    }
+    __syncthreads();
+    for (int j = tid; j < SORT_BUCKETS; j += NT)
+      if (off[j] > SORT_BUCKET_MAX) misc[0] = 1;
+    __syncthreads();
+    nall = block_excl_scan(off, SORT_BUCKETS, misc);           // scratch misc[8..40]
+    if (misc[0]) usable = false;
+    else {
+      for (int j = tid; j < SORT_BUCKETS; j += NT) cur[j] = off[j];
+      if (tid == 0) off[SORT_BUCKETS] = nall;
+      __syncthreads();
+      for (int j0 = tid; j0 < (int)cnt; j0 += 4 * NT) {
+        uint2 e[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e[u] = (j0 + u * NT < (int)cnt) ? __ldcg(glist + j0 + u * NT) : make_uint2(0u, 0xFFFFFFFFu);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (e[u].y < (unsigned)n) pairs[atomicAdd(&cur[bucket_of(e[u].x)], 1)] = e[u];
+      }
+      __syncthreads();
+      // neighbouring threads hold pairs of the same bucket: the reads below are mostly broadcasts
+      for (int i = tid; i < nall; i += NT) {
+        const uint2 e = pairs[i];
+        const int bk = bucket_of(e.x);
+        const int lo = off[bk], hi = off[bk + 1];
+        int rank = 0;
+        for (int v = lo; v < hi; ++v) {
+          const uint2 o = pairs[v];
+          rank += (o.x < e.x) || (o.x == e.x && o.y < e.y);
+        }
+        srt[lo + rank] = (int)e.y;
+      }
+      __syncthreads();
+      for (int i = tid; i < nall; i += NT) {                   // the keys are spent: (token, physical slot) in their place
+        const int tok = srt[i];
+        pairs[i] = make_uint2((unsigned)tok, (unsigned)(page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15)));
+      }
+    }
+  }
+  DEV_MARK(p, devk, 2, bh == 0);
+  pdl_wait();                         // the bitmap of I_t and meta come from k_select_topk
+  pdl_trigger();
+  DEV_MARK(p, devk, 3, bh == 0);
+  HeadMeta& meta = p.meta[bh];
+  if (n == 0 || geo.n_s <= 0) { if (stream == 1 && tid == 0) meta.sorted_cnt = 0; return; }
+  if (stream == 0 && geo.b0 <= 0) return;
+  const int nw = (n + 31) >> 5;
+  const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
+
+  if (usable) {
+    for (int w = tid; w < nw; w += NT) bits[w] = __ldcg(gbitmap + w);
+    __syncthreads();                                           // also orders the last writes to pairs[]
+    // order-preserving compaction: warp w owns the sorted entries [w_lo, w_hi)
+    const int seg = ((nall + NWARP - 1) / NWARP + 31) & ~31;
+    const int w_lo = min(nall, warp * seg), w_hi = min(nall, w_lo + seg);
+    int kept = 0;
+    for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
+      const int i = i0 + lane;
+      bool keep = false;
+      if (i < w_hi) { const unsigned tok = pairs[i].x; keep = !((bits[tok >> 5] >> (tok & 31)) & 1u); }
+      kept += __popc(__ballot_sync(0xFFFFFFFFu, keep));
+    }
+    if (lane == 0) misc[8 + warp] = kept;
+    __syncthreads();
+    if (warp == 0) {
+      const int v = misc[8 + lane];
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += u;
+      }
+      misc[8 + lane] = incl - v;
+      if (lane == 31) misc[40] = incl;
+    }
+    __syncthreads();
+    const int total = misc[40];
+    if (stream == 1 || total >= geo.b0) {
+      const int limit = stream ? total : geo.b0;
+      int* out = stream ? p.sort_idx + (long long)bh * p.cand_cap : p.base_idx + (long long)bh * p.npad;
+      const long long delta = stream ? p.sort_phys_delta : p.phys_delta;
+      int* dbg = (stream == 0 && p.dbg.base_idx) ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
+      int run = misc[8 + warp];
+      for (int i0 = w_lo; i0 < w_hi && run < limit; i0 += 32) {
+        const int i = i0 + lane;
+        bool keep = false;
+        uint2 e = make_uint2(0u, 0u);
+        if (i < w_hi) { e = pairs[i]; keep = !((bits[e.x >> 5] >> (e.x & 31)) & 1u); }
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, keep);
+        const int pos = run + __popc(bal & ((1u << lane) - 1u));
+        if (keep && pos < limit) {
+          out[pos] = (int)e.x;
+          out[delta + pos] = (int)e.y;
+          if (dbg) dbg[pos] = (int)e.x;
+        }
+        run += __popc(bal);
+      }
+      if (tid == 0) {
+        if (stream == 1) meta.sorted_cnt = total;
+        else if (p.dbg.paths) atomicOr(&p.dbg.paths[bh], 2);
+      }
+      DEV_END(p, devk);
+      return;
+    }
+  }
+  if (stream == 1) { if (tid == 0) meta.sorted_cnt = -1; return; }
+  // base sample from the full context
+  __syncthreads();
+  const Sm sm = carve(smem_raw, bigbytes, p.nwords);
+  for (int w = tid; w < nw; w += NT) sm.w2[w] = __ldcg(gbitmap + w);
+  __syncthreads();
+  const int hrng = p.rng_head_is_kv ? g : h;
+  int* bs_out = p.base_idx + (long long)bh * p.npad;
+  int* bs_dbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
+  sample_select<CACHED>(p, sm, geo.s0, geo.l_start, nw, geo.b0, geo.n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
+  DEV_END(p, devk);
+}
+
+// Final sample, slow path and introspection.  When the budget fits the pre-sorted list (b <= sorted_cnt
+// and b < n_s) the gather kernel reads I_dyn = sorted[0..b) directly and this kernel only copies it to
+// the debug buffer if one is registered.  Otherwise (whole residual, budget beyond the list, unusable
+// list) it draws the sample from the full context and writes it ascending to dyn_idx.
 template <bool CACHED>
 __global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -739,28 +837,27 @@ __global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbyt
   DEV_BEGIN(p, 4);
   pdl_trigger();
   pdl_wait();
-  const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   const HeadMeta meta = p.meta[bh];
   if (p.dbg.dyn_cnt && tid == 0) p.dbg.dyn_cnt[bh] = meta.b;
   if (meta.n == 0 || meta.b <= 0) return;
+  if (meta.b < meta.n_s && meta.sorted_cnt >= meta.b) {
+    if (p.dbg.dyn_idx) {
+      const int* src = p.sort_idx + (long long)bh * p.cand_cap;
+      int* dbg = p.dbg.dyn_idx + (long long)bh * p.max_seq_len;
+      for (int i = tid; i < meta.b; i += NT) dbg[i] = src[i];
+    }
+    if (p.dbg.paths && tid == 0) atomicOr(&p.dbg.paths[bh], 4);
+    return;
+  }
+  const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   const int nw = (meta.n + 31) >> 5;
   const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
   for (int w = tid; w < nw; w += NT) sm.w2[w] = gbitmap[w];
   __syncthreads();
-  DEV_MARK(p, 4, 2, bh == 0);
   const int hrng = p.rng_head_is_kv ? g : h;
   int* out = p.dyn_idx + (long long)bh * p.npad;
   int* dbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)bh * p.max_seq_len : nullptr;
-  int got = -1;
-  if (meta.b < meta.n_s) {
-    const long long l1 = (long long)p.B * p.Hq + bh;
-    got = sample_from_candidates(p, b, sm, p.cand + l1 * p.cand_cap, p.cand_cnt[l1], bigbytes / 8, VATTN_CAND1_BOUND,
-                                 meta.b, nw, sm.w2, out, dbg);
-  }
-  if (got < 0) {
-    __syncthreads();
-    sample_select<CACHED>(p, sm, meta.s0, meta.l_start, nw, meta.b, meta.n_s, b, hrng, 1, sm.w2, out, dbg);
-  } else if (p.dbg.paths && tid == 0) p.dbg.paths[bh] |= 4;
+  sample_select<CACHED>(p, sm, meta.s0, meta.l_start, nw, meta.b, meta.n_s, b, hrng, 1, sm.w2, out, dbg);
   DEV_END(p, 4);
 }
 
@@ -800,14 +897,43 @@ static cudaError_t launch_sel(KernelT kern, const Prob& p, cudaStream_t s, bool 
   return launch_pdl(kern, grid, block, smem, s, p, big);
 }
 
-cudaError_t launch_select_topk_base(const Prob& p, cudaStream_t s) {
+cudaError_t launch_select_topk(const Prob& p, cudaStream_t s) {
   const bool cached = keycap_of(p) > 0;
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) return cached ? launch_sel(k_select_topk_base<bf16_t, 128, true>, p, s, false) : launch_sel(k_select_topk_base<bf16_t, 128, false>, p, s, false);
-    return cached ? launch_sel(k_select_topk_base<bf16_t, 64, true>, p, s, false) : launch_sel(k_select_topk_base<bf16_t, 64, false>, p, s, false);
+    if (p.D == 128) return cached ? launch_sel(k_select_topk<bf16_t, 128, true>, p, s, false) : launch_sel(k_select_topk<bf16_t, 128, false>, p, s, false);
+    return cached ? launch_sel(k_select_topk<bf16_t, 64, true>, p, s, false) : launch_sel(k_select_topk<bf16_t, 64, false>, p, s, false);
   }
-  if (p.D == 128) return cached ? launch_sel(k_select_topk_base<float, 128, true>, p, s, false) : launch_sel(k_select_topk_base<float, 128, false>, p, s, false);
-  return cached ? launch_sel(k_select_topk_base<float, 64, true>, p, s, false) : launch_sel(k_select_topk_base<float, 64, false>, p, s, false);
+  if (p.D == 128) return cached ? launch_sel(k_select_topk<float, 128, true>, p, s, false) : launch_sel(k_select_topk<float, 128, false>, p, s, false);
+  return cached ? launch_sel(k_select_topk<float, 64, true>, p, s, false) : launch_sel(k_select_topk<float, 64, false>, p, s, false);
+}
+
+static size_t select_smem_bytes(const Prob& p, bool final_kernel) {
+  return sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
+         sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64) + (size_t)big_bytes(p, final_kernel);
+}
+
+template <typename KernelT>
+static cudaError_t launch_presort_t(KernelT kern, const Prob& p, cudaStream_t s) {
+  const size_t fixed = SORT_FIXED_BYTES + sizeof(unsigned) * (size_t)p.nwords;
+  const size_t limit = 227 * 1024;
+  const size_t per_pair = sizeof(uint2) + sizeof(int);
+  size_t paircap = (size_t)p.cand_cap;
+  if (fixed + paircap * per_pair > limit) paircap = (limit - fixed) / per_pair;   // longer lists take the slow path
+  size_t smem = fixed + paircap * per_pair;
+  const size_t sel = select_smem_bytes(p, false);              // the stream-0 fallback reuses the buffer
+  if (sel > smem) smem = sel;
+  static size_t attr_sz[2] = {0, 0};
+  const int which = keycap_of(p) > 0 ? 1 : 0;
+  if (attr_sz[which] < smem) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_sz[which] = smem;
+  }
+  return launch_pdl(kern, dim3(p.Hq, p.B, 2), dim3(NT), smem, s, p, (int)paircap, big_bytes(p, false));
+}
+
+cudaError_t launch_presort(const Prob& p, cudaStream_t s) {
+  return keycap_of(p) > 0 ? launch_presort_t(k_presort<true>, p, s) : launch_presort_t(k_presort<false>, p, s);
 }
 
 cudaError_t launch_select_final(const Prob& p, cudaStream_t s) {

@@ -101,18 +101,25 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   __shared__ int is_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int h = blockIdx.y, b = blockIdx.z, g = h / p.G;
+  // grid (S, Hq, 2 B): the deterministic-row CTAs of every head come first in dispatch order, so they take
+  // the SMs that are free while the select kernels still run; the base-row CTAs follow
+  const bool base_cta = (int)blockIdx.z >= p.B;
+  const int h = blockIdx.y, b = base_cta ? blockIdx.z - p.B : blockIdx.z, g = h / p.G;
   const int bh = b * p.Hq + h;
   const int S = p.stat_splits;
-  const bool base_cta = (int)blockIdx.x >= S;
-  const int split = base_cta ? blockIdx.x - S : blockIdx.x;
+  const int split = blockIdx.x;
+  const int vx = (base_cta ? S : 0) + split;       // position among the head's 2 S partials
   DEV_BEGIN(p, 3);
   pdl_trigger();
-  pdl_wait();
+  // Deterministic-row CTAs read only what k_select_topk wrote, which completed before this grid could
+  // start (the grid before this one lets its dependents go only after its own wait on k_select_topk);
+  // base-row CTAs need I_bs from the grid before this one and wait for it.
+  if (base_cta) pdl_wait();
   HeadMeta& meta = p.meta[bh];
-  const int n = meta.n, s0 = meta.s0, l_start = meta.l_start, kk = meta.kk, n_s = meta.n_s, b0 = meta.b0;
+  const HeadMeta mt = ld_meta(p.meta + bh);
+  const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, n_s = mt.n_s, b0 = mt.b0;
   if (n == 0) {
-    if (blockIdx.x == 0 && tid == 0) {
+    if (vx == 0 && tid == 0) {
       meta.b = 0;
       if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
       if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
@@ -126,14 +133,14 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const int* tkph = p.topk_idx + (long long)bh * p.npad + p.phys_delta;     // physical slots of I_t
   const int* bsph = p.base_idx + (long long)bh * p.npad + p.phys_delta;     // physical slots of I_bs
   const int ph0 = phys_of(p, b, 0);
-  const double m = (double)meta.m;
+  const double m = (double)mt.m;
   const int rsub = lane / LPR, j = lane % LPR;
   const int rg = warp * RPI + rsub;
   const int iters = (r_end - r_begin + RG - 1) / RG;      // uniform over the CTA
 
   float qf[EPL];
   Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
-  DEV_MARK(p, 3, 2, bh == 0 && blockIdx.x == 0);
+  DEV_MARK(p, 3, 2, bh == 0 && vx == 0);
 
   double acc[EPL], s1 = 0.0, s2 = 0.0, s3 = 0.0;           // det: N_f slice, D_f;  base: Sr slice, Sw, Sww, Srr
 #pragma unroll
@@ -225,7 +232,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
       }
     }
   }
-  DEV_MARK(p, 3, 3, bh == 0 && blockIdx.x == 0);
+  DEV_MARK(p, 3, 3, bh == 0 && vx == 0);
   // across the row groups of the warp
 #pragma unroll
   for (int mask = LPR; mask < 32; mask <<= 1) {
@@ -242,7 +249,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     if (j == 0) { part[warp][D] = s1; part[warp][D + 1] = s2; part[warp][D + 2] = s3; }
   }
   __syncthreads();
-  double* gpart = p.stat_part + ((long long)bh * 2 * MAXS + blockIdx.x) * NE;
+  double* gpart = p.stat_part + ((long long)bh * 2 * MAXS + vx) * NE;
   for (int e = tid; e < NE; e += NT) {
     double s = 0.0;
 #pragma unroll
@@ -251,12 +258,12 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   }
   if (base_cta && split == 0 && b0 > 0)              // the pivot travels with this CTA's partial
     for (int e = tid; e <= D; e += NT) p.stat_piv[(long long)bh * (D + 1) + e] = piv[e];
-  DEV_MARK(p, 3, 4, bh == 0 && blockIdx.x == 0);
+  DEV_MARK(p, 3, 4, bh == 0 && vx == 0);
   __threadfence();
   __syncthreads();
   if (tid == 0) is_last = (atomicAdd(&p.tickets[bh], 1u) == (unsigned)(2 * S - 1));
   __syncthreads();
-  DEV_MARK(p, 3, 5, bh == 0 && blockIdx.x == 0);
+  DEV_MARK(p, 3, 5, bh == 0 && vx == 0);
   if (!is_last) { DEV_END(p, 3); return; }
   __threadfence();
   DEV_MARK(p, 3, 6, bh == 0);
@@ -348,7 +355,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 }  // namespace
 
 cudaError_t launch_stats(const Prob& p, cudaStream_t s) {
-  dim3 grid(2 * p.stat_splits, p.Hq, p.B), block(NT);
+  dim3 grid(p.stat_splits, p.Hq, 2 * p.B), block(NT);
   if (p.stat_splits < 1 || p.stat_splits > MAXS) return cudaErrorInvalidValue;
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (p.D == 128) return launch_pdl(k_stats<bf16_t, 128>, grid, block, 0, s, p);

@@ -21,7 +21,7 @@ struct HeadMeta {
   int n_s;       // residual size |M| - kk
   int b0;        // base-sample size
   int b;         // final budget |I_dyn|
-  int pad0;
+  int sorted_cnt; // entries of the pre-sorted stream-1 residual list (-1: list unusable)
   float m;       // largest fp32 score of the head (softmax stabiliser)
   float gamma;   // bound on |fp32 score - exact score| for this head
   int pad1, pad2;
@@ -53,6 +53,8 @@ struct Prob {
   int* base_idx;          // [B,Hq,npad]   (page * 16 + token % 16 of every entry) lies phys_delta
   int* dyn_idx;           // [B,Hq,npad]   elements behind each index list
   long long phys_delta;
+  int* sort_idx;          // [B,Hq,cand_cap] residual stream-1 candidates sorted by (key, token); physical slots
+  long long sort_phys_delta;  //   lie sort_phys_delta elements behind
   HeadMeta* meta;         // [B,Hq]
   double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (det CTAs, then base CTAs)
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
@@ -71,10 +73,12 @@ __device__ __forceinline__ unsigned long long dev_gtime() { unsigned long long t
 #define DEV_BEGIN(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMin(&(p).devt[(k) * 32 + 0], dev_gtime()); } while (0)
 #define DEV_END(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMax(&(p).devt[(k) * 32 + 1], dev_gtime()); } while (0)
 #define DEV_MARK(p, k, slot, cond) do { if ((p).devt && threadIdx.x == 0 && (cond)) (p).devt[(k) * 32 + (slot)] = dev_gtime(); } while (0)
+#define DEV_AT(p, index) do { if ((p).devt && threadIdx.x == 0) (p).devt[(index)] = dev_gtime(); } while (0)
 #else
 #define DEV_BEGIN(p, k) do { } while (0)
 #define DEV_END(p, k) do { } while (0)
 #define DEV_MARK(p, k, slot, cond) do { } while (0)
+#define DEV_AT(p, index) do { } while (0)
 #endif
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
@@ -239,9 +243,20 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsig
 }
 
 
+// HeadMeta through L2 (ld.cg): for kernels that are let loose before their stream predecessor has
+// finished and therefore cannot count on the launch-boundary L1 invalidation.
+static_assert(sizeof(HeadMeta) == 48, "HeadMeta is read as three 16-byte words");
+__device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
+  union { HeadMeta m; int4 v[3]; } u;
+  const int4* src = reinterpret_cast<const int4*>(g);
+  u.v[0] = __ldcg(src); u.v[1] = __ldcg(src + 1); u.v[2] = __ldcg(src + 2);
+  return u.m;
+}
+
 // launchers (one per translation unit)
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
-cudaError_t launch_select_topk_base(const Prob& p, cudaStream_t s);
+cudaError_t launch_select_topk(const Prob& p, cudaStream_t s);
+cudaError_t launch_presort(const Prob& p, cudaStream_t s);
 cudaError_t launch_select_final(const Prob& p, cudaStream_t s);
 cudaError_t launch_stats(const Prob& p, cudaStream_t s);
 cudaError_t launch_gather(const Prob& p, cudaStream_t s);
