@@ -22,7 +22,7 @@ struct vattn_plan {
   int G, npad, nwords, stat_splits, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
       off_det, off_piv, off_gat, off_dense, off_cand, off_sort, total;
-  int cand_cap;
+  int cand_cap, gat_slots;
 };
 
 namespace {
@@ -88,7 +88,8 @@ void derive(vattn_plan* pl) {
   pl->off_stat = take(BH * 2 * kMaxStatSplits * (D + 3) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
-  pl->off_gat = take(BH * kMaxGatherSplits * (D + 1) * sizeof(float));
+  pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? VATTN_GATHER_FLAT_SLOTS : kMaxGatherSplits;
+  pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
   {
     const double q4 = 0.25 * (double)pl->npad;
@@ -139,6 +140,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
   p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
+  p.gat_slots = pl->gat_slots;
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.stat_splits = pl->stat_splits; p.dense_splits = pl->dense_splits;
   p.dbg = pl->dbg;
@@ -292,6 +294,9 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
     int want = (int)((rows + 127.0) / 128.0) * 2;          // about 64 rows per CTA
     if (want < 1) want = 1;
     if (want < p.stat_splits) p.stat_splits = want;
+#ifdef VATTN_DEV_STAT_SPLITS
+    p.stat_splits = VATTN_DEV_STAT_SPLITS;
+#endif
   }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;

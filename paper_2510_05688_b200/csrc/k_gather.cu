@@ -3,17 +3,19 @@
 // which is SDPA_{S,p} of Sec. 3 with p = 1 on I_f and p = b/n_s on I_dyn.
 //
 // HBM-bound row gather.  Work unit = a chunk of consecutive entries of one head's I_dyn list.  LPR lanes
-// fetch one V row with one 16-byte load each; a row group keeps 4 rows in flight and requests the next
-// batch's indices (token + physical slot, written by the select kernel) while the current rows arrive.
+// fetch one V row with one 16-byte load each; a row group keeps 8 rows in flight and requests the next
+// batch's indices (token + physical slot, written by the select kernels) while the current rows arrive.
 // Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
 // last CTA of the head ("ticket"), so results are reproducible.
 //
 // Two decompositions:
 //  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
 //    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
-//    grid stride: every SM gets the same number of rows whatever the budgets are;
+//    grid stride.  A chunk is exactly what one CTA keeps in flight at once (one batch: 64 rows of 128 bf16),
+//    so a step with up to 1184 chunks costs one memory round trip per CTA; a head uses up to 128 chunks
+//    (longer lists get chunks of two, three, ... batches);
 //  * per head (larger problems): grid (32, heads, batch); a head with budget b uses ceil(b / chunk) of its
-//    32 CTAs, chunk = max(64, ceil(b / 32)) rows, the others exit at once.
+//    32 CTAs, chunk = max(256, ceil(b / 32)) rows, the others exit at once.
 #include "vattn_internal.cuh"
 
 namespace {
@@ -21,9 +23,10 @@ namespace {
 constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
 constexpr int UNROLL = 8;         // rows in flight per row group (16-byte slices kept raw until used)
-constexpr int MAXS = 32;           // most chunks (partials) per head
-constexpr int FLAT_MAX_HEADS = 128;
-constexpr int MIN_CHUNK = 64;      // rows of a chunk in the flat decomposition, unless the head has > 32 of them
+constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
+constexpr int FLAT_MAXS = VATTN_GATHER_FLAT_SLOTS;   // ... flat decomposition
+constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
+constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
 
 template <typename T, int D>
 struct Gather {
@@ -120,7 +123,7 @@ struct Gather {
       if (j == 0) part[warp][D] = dd;
     }
     __syncthreads();
-    float* gpart = p.gat_part + ((long long)bh * MAXS + slot) * NE;
+    float* gpart = p.gat_part + ((long long)bh * p.gat_slots + slot) * NE;
     for (int e = tid; e < NE; e += NT) {
       float s = 0.f;
 #pragma unroll
@@ -143,7 +146,7 @@ struct Gather {
     const int nb = meta.b;
     const double* det = p.det_sums + (long long)bh * (D + 1);
     const double f = (nb > 0) ? (double)meta.n_s / (double)nb : 0.0;
-    const float* src0 = p.gat_part + (long long)bh * MAXS * NE;
+    const float* src0 = p.gat_part + (long long)bh * p.gat_slots * NE;
     float num_s[(D + NT - 1) / NT];
     double det_e[(D + NT - 1) / NT];
     const double det_d = __ldcg(det + D);             // N_f, D_f of the statistics kernel, requested with the partials
@@ -152,19 +155,23 @@ struct Gather {
 #pragma unroll
     for (int it = 0; it < (D + NT - 1) / NT; ++it) {
       const int e = tid + it * NT;
-      float vv[MAXS];
-#pragma unroll
-      for (int sp = 0; sp < MAXS; ++sp) vv[sp] = (sp < nslots && e < D) ? __ldcg(src0 + (long long)sp * NE + e) : 0.f;
       float s = 0.f;
+      for (int s0 = 0; s0 < nslots; s0 += 32) {       // 32 partials per round trip, added in slot order
+        float vv[32];
 #pragma unroll
-      for (int sp = 0; sp < MAXS; ++sp) s += vv[sp];
+        for (int sp = 0; sp < 32; ++sp) vv[sp] = (s0 + sp < nslots && e < D) ? __ldcg(src0 + (long long)(s0 + sp) * NE + e) : 0.f;
+#pragma unroll
+        for (int sp = 0; sp < 32; ++sp) s += vv[sp];
+      }
       num_s[it] = s;
     }
-    if (warp == 0) {                                  // the denominator: lane sp holds slot sp
-      const float vd = (lane < nslots) ? __ldcg(src0 + (long long)lane * NE + D) : 0.f;
+    if (warp == 0) {                                  // the denominator: lane sp holds slot s0 + sp
       float s = 0.f;
+      for (int s0 = 0; s0 < nslots; s0 += 32) {
+        const float vd = (s0 + lane < nslots) ? __ldcg(src0 + (long long)(s0 + lane) * NE + D) : 0.f;
 #pragma unroll
-      for (int sp = 0; sp < MAXS; ++sp) s += __shfl_sync(0xFFFFFFFFu, vd, sp);
+        for (int sp = 0; sp < 32; ++sp) s += __shfl_sync(0xFFFFFFFFu, vd, sp);
+      }
       if (lane == 0) *s_den = s;
     }
     __syncthreads();
@@ -214,12 +221,14 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int BH = p.B * p.Hq;
   // chunk counts of all heads and their prefix sum (every CTA computes the same numbers)
-  int nb = 0, rows = MIN_CHUNK, cnt = 0;
+  constexpr int BATCH = G::RG * UNROLL;               // rows a CTA keeps in flight at once
+  int nb = 0, rows = BATCH, cnt = 0;
   if (tid < BH) {
     const HeadMeta mt = p.meta[tid];
     s_meta[tid] = mt;
     nb = mt.n > 0 ? mt.b : 0;
-    rows = max(MIN_CHUNK, (nb + MAXS - 1) / MAXS);
+    const int batches = (nb + BATCH - 1) / BATCH;
+    rows = BATCH * max(1, (batches + FLAT_MAXS - 1) / FLAT_MAXS);
     cnt = max(1, (nb + rows - 1) / rows);             // a head without samples still writes its output
     s_rows[tid] = rows;
     s_b[tid] = nb;
@@ -259,8 +268,9 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
 cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
   const int BH = p.B * p.Hq;
   if (BH <= FLAT_MAX_HEADS) {
-    // at most 32 chunks of >= 64 rows per head; 8 CTAs per SM walk them with a grid stride
-    const long long most = (long long)BH * MAXS;
+    // at most FLAT_MAXS chunks per head; 8 CTAs per SM walk them with a grid stride
+    if (p.gat_slots < FLAT_MAXS) return cudaErrorInvalidValue;
+    const long long most = (long long)BH * FLAT_MAXS;
     const int grid = (int)(most < 8 * 148 ? most : 8 * 148);
     if (p.dtype == VATTN_DTYPE_BF16) {
       if (p.D == 128) return launch_pdl(k_gather_flat<bf16_t, 128>, dim3(grid), dim3(NT), 0, s, p);
@@ -271,6 +281,7 @@ cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
     }
     return cudaGetLastError();
   }
+  if (p.gat_slots < MAXS) return cudaErrorInvalidValue;
   dim3 grid(MAXS, p.Hq, p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (p.D == 128) return launch_pdl(k_gather<bf16_t, 128>, grid, block, 0, s, p);

@@ -115,6 +115,10 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   // start (the grid before this one lets its dependents go only after its own wait on k_select_topk);
   // base-row CTAs need I_bs from the grid before this one and wait for it.
   if (base_cta) pdl_wait();
+#ifdef VATTN_DEV_TIMING
+  const int dv = 256 + 8192 + (b * p.Hq + blockIdx.y) * 8;
+  if (base_cta && split == 0) DEV_AT(p, dv + 0);
+#endif
   HeadMeta& meta = p.meta[bh];
   const HeadMeta mt = ld_meta(p.meta + bh);
   const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, n_s = mt.n_s, b0 = mt.b0;
@@ -233,6 +237,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     }
   }
   DEV_MARK(p, 3, 3, bh == 0 && vx == 0);
+#ifdef VATTN_DEV_TIMING
+  if (split == 0) DEV_AT(p, dv + (base_cta ? 1 : 5));
+#endif
   // across the row groups of the warp
 #pragma unroll
   for (int mask = LPR; mask < 32; mask <<= 1) {
@@ -267,6 +274,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   if (!is_last) { DEV_END(p, 3); return; }
   __threadfence();
   DEV_MARK(p, 3, 6, bh == 0);
+#ifdef VATTN_DEV_TIMING
+  DEV_AT(p, dv + 2);
+#endif
 
   // ------------------------------------------------------------------ last CTA of this head
   // every thread requests all partials of its element at once (one memory round trip), then adds them
@@ -286,6 +296,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   for (int e = tid; e <= D; e += NT) piv[e] = (b0 > 0) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
   __syncthreads();
   DEV_MARK(p, 3, 7, bh == 0);
+#ifdef VATTN_DEV_TIMING
+  DEV_AT(p, dv + 3);
+#endif
   double* det = p.det_sums + (long long)bh * (D + 1);
   for (int e = tid; e <= D; e += NT) det[e] = tot[0][e];
   if (warp != 0) return;
@@ -342,6 +355,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   }
   meta.b = bfin;
   DEV_END(p, 3);
+#ifdef VATTN_DEV_TIMING
+  if (p.devt) p.devt[dv + 4] = dev_gtime();
+#endif
   if (p.dbg.budgets) {
     int* o = p.dbg.budgets + bh * 4;
     o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bfin;

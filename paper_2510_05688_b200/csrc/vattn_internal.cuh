@@ -59,7 +59,8 @@ struct Prob {
   double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (det CTAs, then base CTAs)
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
   double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
-  float* gat_part;        // [B,Hq,32,D+1]    partials of the gather kernel, one per chunk
+  float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
+  int gat_slots;          // 128 when batch * heads <= 128 (flat decomposition), else 32
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, dense_splits;
   vattn_debug dbg;
@@ -184,6 +185,8 @@ __device__ __forceinline__ Geo head_geometry(const Prob& p, int n) {
 // is below this bound.  Stream 1 keeps a quarter of the tokens; stream 0 keeps b0 + 6 sqrt(b0) + 16
 // expected tokens (none if that is more than a quarter: the select kernel then draws without the list).
 #define VATTN_CAND1_BOUND 0x40000000u
+#define VATTN_GATHER_FLAT_HEADS 128   // the gather kernel's flat decomposition serves up to this many heads ...
+#define VATTN_GATHER_FLAT_SLOTS 128   // ... with up to this many chunks (partials) each
 __device__ __forceinline__ unsigned cand0_bound(const Geo& g) {
   if (g.n_s <= 0 || g.b0 <= 0) return 0u;
   const double want = (double)g.b0 + 6.0 * sqrt((double)g.b0) + 16.0;
