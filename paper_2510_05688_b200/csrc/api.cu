@@ -294,9 +294,6 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
     int want = (int)((rows + 127.0) / 128.0) * 2;          // about 64 rows per CTA
     if (want < 1) want = 1;
     if (want < p.stat_splits) p.stat_splits = want;
-#ifdef VATTN_DEV_STAT_SPLITS
-    p.stat_splits = VATTN_DEV_STAT_SPLITS;
-#endif
   }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;

@@ -263,19 +263,21 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
     if (!mbar_wait(&bars[s], (unsigned)(k / NST) & 1u)) { failed = true; break; }
     const unsigned char* stg = ring + (size_t)s * PAGEB;
     const int tok0 = (wglob + k * wtot) << 4;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};   // two independent MMA chains
     unsigned klo = 0u, khi = 0u;
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
       const uint4 alo = *reinterpret_cast<const uint4*>(stg + gr * ROWB + c * 64 + t * 16);
       const uint4 ahi = *reinterpret_cast<const uint4*>(stg + (gr + 8) * ROWB + c * 64 + t * 16);
       mma_bf16_16816(acc, alo.x, ahi.x, alo.y, ahi.y, bq[c].x, bq[c].y);
-      mma_bf16_16816(acc, alo.z, ahi.z, alo.w, ahi.w, bq[c].z, bq[c].w);
+      mma_bf16_16816(acc1, alo.z, ahi.z, alo.w, ahi.w, bq[c].z, bq[c].w);
       klo = __vimax3_u16x2(klo, alo.x & 0x7FFF7FFFu, alo.y & 0x7FFF7FFFu);
       klo = __vimax3_u16x2(klo, alo.z & 0x7FFF7FFFu, alo.w & 0x7FFF7FFFu);
       khi = __vimax3_u16x2(khi, ahi.x & 0x7FFF7FFFu, ahi.y & 0x7FFF7FFFu);
       khi = __vimax3_u16x2(khi, ahi.z & 0x7FFF7FFFu, ahi.w & 0x7FFF7FFFu);
     }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e] += acc1[e];
     // the stage has been read (the MMAs consumed every fragment): refill it with page k + NST
     __syncwarp();
     if (k + NST < mine) {
@@ -446,10 +448,18 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   // one wave of two CTAs per SM; a warp walks pages with stride (CTAs along x) * WARPS
   const int groups = p.Hkv * ((p.G + 7) / 8) * p.B;
   const int pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
-  // one wave when the (batch row, KV head) groups leave room for it; with more groups than SMs the
-  // sequences are ragged anyway: cut them finer (about two waves) so that long ones do not set the time
-  int cx = groups <= 148 ? (2 * 148) / groups : (4 * 148 + groups - 1) / groups;
-  if (groups > 148 && cx < 2) cx = 2;
+  // A single sequence whose groups divide the 2 x 148 resident CTAs (almost) evenly runs as one wave.  Anything
+  // else (several sequences, possibly of different lengths; a group count that leaves SMs idle) is cut into
+  // about eight waves of CTAs with at least 32 pages each, which the hardware scheduler balances.
+  const int slots = 2 * 148;
+  int cx = slots / groups;
+  if (cx < 1) cx = 1;
+  const bool one_wave = p.B == 1 && groups * cx <= slots && (slots - groups * cx) * 20 < slots;
+  if (!one_wave) {
+    cx = (8 * slots + groups - 1) / groups;
+    const int cx_fine = (pages + 31) / 32;
+    if (cx > cx_fine) cx = cx_fine;
+  }
   const int cx_max = (pages + WARPS - 1) / WARPS;
   if (cx > cx_max) cx = cx_max;
   if (cx < 1) cx = 1;

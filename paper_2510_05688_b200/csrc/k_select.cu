@@ -561,11 +561,10 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 2);
-  pdl_wait();
-  pdl_trigger();                      // dependents may read the score kernel's outputs before their own wait
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
 
+  // before the wait: everything that depends on the step's inputs only
   const int n = clamped_len(p, b);
   const Geo geo = head_geometry(p, n);
   const int s0 = geo.s0, l_start = geo.l_start, kk = geo.kk, n_s = geo.n_s, b0 = geo.b0;
@@ -573,20 +572,36 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   const int nw = (n + 31) >> 5;
   const T* qrow = reinterpret_cast<const T*>(p.q) + (long long)bh * D;
   const float* sc = p.scores + (long long)bh * p.npad;
-  const float m = (n > 0) ? unord_f32(p.m_ord[bh]) : 0.f;
-
-  // gamma: bound on |fp32 score - exact score|.  fp32 path: at most 13 roundings (x16 = margin).
-  // bf16 tensor-core path: 8 accumulation steps of 16 exact products each, every step assumed to lose
-  // up to 17 units of 2^-23 of the running magnitude (truncating adder) -> 8*17*2 = 272, taken as 512.
+  double sa = 0.0;                      // sum |q_e| (warp 0)
   if (warp == 0) {
-    double sa = 0.0;
     for (int e = lane; e < D; e += 32) sa += fabs((double)Elem<T>::to_float(qrow[e]));
 #pragma unroll
     for (int mk = 16; mk >= 1; mk >>= 1) sa += __shfl_xor_sync(0xFFFFFFFFu, sa, mk);
-    const double kmax = (double)__uint_as_float(p.kabsmax[b * p.Hkv + g]);
+  }
+  for (int w = tid; w < nw; w += NT) { sm.w0[w] = 0u; sm.w1[w] = 0u; }
+  pdl_wait();
+  pdl_trigger();                      // dependents may read the score kernel's outputs before their own wait
+  const float m = (n > 0) ? unord_f32(__ldcg(p.m_ord + bh)) : 0.f;
+
+  // gamma: bound on |fp32 score - exact score|.  fp32 path: at most 13 roundings (x16 = margin).
+  // bf16 tensor-core path: at most 8 accumulation steps of 16 exact products each (two chains of 4 and one
+  // addition for d = 128), every step assumed to lose up to 17 units of 2^-23 of the running magnitude
+  // (truncating adder) -> 8*17*2 = 272, taken as 512.
+  if (warp == 0) {
+    const double kmax = (double)__uint_as_float(__ldcg(p.kabsmax + b * p.Hkv + g));
     const double roundings = (p.dtype == VATTN_DTYPE_BF16) ? 512.0 : 16.0;
     const double gm = roundings * 5.9604644775390625e-8 * fabs((double)p.scale) * sa * kmax * 1.000001;
     if (lane == 0) reinterpret_cast<float*>(sm.misc)[48] = __double2float_ru(gm);
+  }
+  if (CACHED && kk > 0 && kk < mlen) {
+    // order-reversed score keys of the middle range: 16-byte loads over the aligned body
+    const int a0 = min(l_start, (s0 + 3) & ~3), a1 = max(a0, l_start & ~3);
+    for (int i = s0 + tid; i < a0; i += NT) sm.keys[i] = ~ord_f32(__ldcg(sc + i));
+    for (int i = a1 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(__ldcg(sc + i));
+    for (int i = a0 + 4 * tid; i < a1; i += 4 * NT) {
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(sc + i));
+      *reinterpret_cast<uint4*>(sm.keys + i) = make_uint4(~ord_f32(v.x), ~ord_f32(v.y), ~ord_f32(v.z), ~ord_f32(v.w));
+    }
   }
   __syncthreads();
   const float gamma = reinterpret_cast<float*>(sm.misc)[48];
@@ -602,8 +617,6 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
 
   int path = 0;
   // ------------------------------------------------------------------ top-k over the middle range
-  for (int w = tid; w < nw; w += NT) { sm.w0[w] = 0u; sm.w1[w] = 0u; }
-  __syncthreads();
   if (kk > 0 && kk == mlen) {
     for (int w = tid; w < nw; w += NT) {
       const int i0 = w * 32;
@@ -616,8 +629,6 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   } else if (kk > 0) {
     bool done = false;
     if (CACHED) {
-      for (int i = s0 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(sc[i]);
-      __syncthreads();
       DEV_MARK(p, 2, 3, bh == 0);
       done = topk_fast<T, D>(p, sm, b, g, qrow, s0, l_start, kk, nw, m, gamma);
       DEV_MARK(p, 2, 4, bh == 0);

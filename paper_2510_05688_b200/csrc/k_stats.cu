@@ -111,18 +111,17 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const int vx = (base_cta ? S : 0) + split;       // position among the head's 2 S partials
   DEV_BEGIN(p, 3);
   pdl_trigger();
-  // Deterministic-row CTAs read only what k_select_topk wrote, which completed before this grid could
-  // start (the grid before this one lets its dependents go only after its own wait on k_select_topk);
-  // base-row CTAs need I_bs from the grid before this one and wait for it.
-  if (base_cta) pdl_wait();
+  // What k_select_topk wrote (meta, I_t) is complete before this grid can start: the grid before this one
+  // lets its dependents go only after its own wait on k_select_topk.  Only the base-row CTAs need the
+  // grid before this one itself (I_bs), and they wait for it as late as possible.
 #ifdef VATTN_DEV_TIMING
   const int dv = 256 + 8192 + (b * p.Hq + blockIdx.y) * 8;
-  if (base_cta && split == 0) DEV_AT(p, dv + 0);
 #endif
   HeadMeta& meta = p.meta[bh];
   const HeadMeta mt = ld_meta(p.meta + bh);
   const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, n_s = mt.n_s, b0 = mt.b0;
   if (n == 0) {
+    if (base_cta) pdl_wait();                      // every base-row CTA waits: "this grid done" implies "the one before done"
     if (vx == 0 && tid == 0) {
       meta.b = 0;
       if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
@@ -184,7 +183,13 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
         }
       }
     }
-  } else if (b0 > 0) {
+  } else {
+    pdl_wait();
+#ifdef VATTN_DEV_TIMING
+    if (split == 0) DEV_AT(p, dv + 0);
+#endif
+  }
+  if (base_cta && b0 > 0) {
     // ---------------------------------------------------------------- base-sample rows, shifted by the pivot
     RowRegs<T> prow;
     const int piv_ph = __ldg(bsph);                          // pivot = first base-sample row
