@@ -401,6 +401,7 @@ def main():
     n_f = kks.sum() + Hq * (min(case.sink, n_tot) + min(case.window, n_tot))
     alg = {
         "k_score": n_tot * Hkv * d * es + n_tot * Hq * 4,
+        "k_cand": int(0.27 * n_tot * Hq) * 8,
         "k_select_topk": n_tot * Hq * 4,
         "k_presort": int(0.25 * n_tot * Hq) * 8 + int(b0s.sum()) * 8 + 2 * n_tot * Hq // 8,
         "k_stats": int(n_f + b0s.sum()) * d * es * 2,
@@ -408,7 +409,7 @@ def main():
         "k_gather": int(b_dyn.sum()) * (d * es + 4),
     }
     # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2_llama8b.md
-    traffic = {"k_score": 68.39e6, "k_select_topk": 4.61e6, "k_presort": None,
+    traffic = {"k_score": 68.39e6, "k_cand": None, "k_select_topk": 4.61e6, "k_presort": None,
                "k_stats": 25.60e6, "k_select_final": None, "k_gather": 20.13e6}
     peak, peak_kind = measured_peaks()
     kern = {}

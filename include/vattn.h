@@ -172,14 +172,15 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */)
 int vattn_last_launch_count(const vattn_plan* plan);
 
 /* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
- * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, top-k select,
- * sampling sort, statistics + budget, slow-path final select, gather + combine), for up to 256 calls
- * between two reads.  The events serialise kernels that otherwise overlap (the sampling sort runs beside
- * the top-k select, the first half of the statistics beside the sampling), so the per-kernel times add up
- * to more than an unprofiled step takes.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
+ * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, sampling-key
+ * pre-filter, top-k select, sampling sort, statistics + budget, slow-path final select, gather +
+ * combine), for up to 256 calls between two reads.  The events serialise kernels that otherwise overlap
+ * (the key pre-filter runs beside the score kernel, the sampling sort beside the top-k select, the first
+ * half of the statistics beside the sampling), so the per-kernel times add up to more than an unprofiled
+ * step takes.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
  * milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to *calls
  * (host), and starts a new window.  Events add a little latency: do not enable in production. */
-#define VATTN_NUM_KERNELS 6
+#define VATTN_NUM_KERNELS 7
 int vattn_set_profiling(vattn_plan* plan, int enable);
 int vattn_read_profile(vattn_plan* plan, float* ms_sum, int* calls);
 

@@ -77,7 +77,7 @@ void derive(vattn_plan* pl) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   pl->off_scores = take(BH * pl->npad * sizeof(float));
-  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 2 * BH) * sizeof(unsigned);
+  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 2 * BH + 4) * sizeof(unsigned);
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
@@ -125,6 +125,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   const size_t BH = (size_t)s.batch * s.num_q_heads;
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
   p.cand_cnt = p.tickets + 3 * BH;
+  p.unit_ctr = p.cand_cnt + 2 * BH;
   p.cand = reinterpret_cast<uint2*>(w + pl->off_cand);
   p.cand_cap = pl->cand_cap;
   p.sort_idx = reinterpret_cast<int*>(w + pl->off_sort);
@@ -306,23 +307,27 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   rc = prepare_stream(plan, p, st);
   if (rc != VATTN_OK) return rc;
   prof_mark(plan, 0, st);
+  // score || key pre-filter -> top-k || sampling sort -> sampling compaction -> statistics + budget ->
+  // slow-path select (usually nothing to do) -> gather.  The overlaps come from programmatic dependent
+  // launches (see the kernels): the pre-filter runs beside the persistent score kernel, the sort of its
+  // lists beside the top-k select.
   CU(launch_score(p, st));            plan->last_launches++;
   prof_mark(plan, 1, st);
+  CU(launch_cand(p, st));             plan->last_launches++;
+  prof_mark(plan, 2, st);
   if (p.dbg.scores)
     CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
                          sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
-  // score -> top-k -> sampling (its sort runs concurrently with top-k, before its dependency wait) ->
-  // statistics + budget -> slow-path select (usually nothing to do) -> gather.
   CU(launch_select_topk(p, st));      plan->last_launches++;
-  prof_mark(plan, 2, st);
-  CU(launch_presort(p, st));          plan->last_launches++;
   prof_mark(plan, 3, st);
-  CU(launch_stats(p, st));            plan->last_launches++;
+  CU(launch_presort(p, st));          plan->last_launches++;
   prof_mark(plan, 4, st);
-  CU(launch_select_final(p, st));     plan->last_launches++;
+  CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 5, st);
-  CU(launch_gather(p, st));           plan->last_launches++;
+  CU(launch_select_final(p, st));     plan->last_launches++;
   prof_mark(plan, 6, st);
+  CU(launch_gather(p, st));           plan->last_launches++;
+  prof_mark(plan, 7, st);
   if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
   return VATTN_OK;
 }

@@ -4,265 +4,239 @@
 // (softmax stabiliser) and, per KV head, max |K element| (for the rounding-error bound of the scores).
 //
 // HBM-bound stream over K (every K row is read exactly once).  Two arithmetic paths:
-//  * bf16: pages travel into shared memory with bulk asynchronous copies (a 4-stage mbarrier ring per
-//    warp) and the [16 tokens x d] x [d x 8 heads] contraction of a page runs on the tensor cores
-//    (mma.sync m16n8k16, fp32 accumulate).  A dot product does not care in which order its terms are
-//    paired, so the k-slots of the fragment layout are mapped onto d such that each thread owns 8
-//    consecutive elements of a row and reads them with one 16-byte shared load.  This removes the
-//    CUDA-core FMAs and the cross-lane reduction that made a first version ALU-co-bound.
+//  * bf16: a persistent grid of two CTAs per SM.  The work is cut into units (batch row, KV-head group,
+//    run of consecutive pages) on the device, from the actual sequence lengths; CTAs take their first unit
+//    by index and the following ones from an atomic counter, so ragged batches balance themselves.  In a
+//    CTA one producer warp walks the CTA's units and keeps a ring of S page-sized stages full with bulk
+//    asynchronous copies (cp.async.bulk + mbarrier transaction counts; one 4 KB slab per page, the group's
+//    query rows ride along with the first pages of a unit); four consumer warps take the stages in turn
+//    (full / empty mbarriers, bounded waits) and run the [16 tokens x d] x [d x 8 heads] contraction of a
+//    page on the tensor cores (mma.sync m16n8k16, fp32 accumulate, two independent chains).  A dot product
+//    does not care in which order its terms are paired, so the k-slots of the fragment layout are mapped
+//    onto d such that each thread owns 8 consecutive elements of a row and reads them with one 16-byte
+//    shared load.  The ring never drains between units.
 //  * fp32: CUDA-core FMAs, EPL sequential FMAs per lane and a butterfly that halves the live partial
 //    sums at every level (tf32 tensor cores would not keep fp32 accuracy).
-//
-// The same CTAs also pre-filter the sampling keys: Philox4x32-10 keys of streams 0 and 1 are computed
-// for every (token, head) of the tile and tokens whose key is below the stream's bound are appended to
-// per-head candidate lists, so the select kernels never run Philox over the whole context
-// (uniform-sample of Algorithm 1 line 7 / Algorithm 2 line 1 = the c smallest keys of the residual).
 #include "vattn_internal.cuh"
 
 namespace {
 
-constexpr int PPW = 4;      // pages per warp
-constexpr int WARPS = 4;    // warps per CTA
-constexpr int TILE = PPW * WARPS * VATTN_BLOCK;   // 256 tokens
+constexpr int PPW = 4;      // pages per warp                         (fp32 path)
+constexpr int WARPS = 4;    // warps per CTA                          (fp32 path)
+constexpr int TILE = PPW * WARPS * VATTN_BLOCK;   // 256 tokens       (fp32 path)
 
 // ---------------------------------------------------------------------------------------------
-// sampling-candidate pre-filter for the tile [tile0, tile0 + TILE) and heads h0 .. h0 + nh - 1
-template <int MAXH>
-__device__ void emit_candidates(const Prob& p, int b, int g, int h0, int nh, int tile0, int n,
-                                uint2 (*s_list)[TILE], unsigned* s_cnt) {
-  const int tid = threadIdx.x;
-  const Geo geo = head_geometry(p, n);
-  if (geo.n_s <= 0) return;                                    // uniform for the CTA
-  const unsigned bound0 = cand0_bound(geo);
-  for (int i = tid; i < 2 * MAXH; i += WARPS * 32) s_cnt[i] = 0;
-  __syncthreads();
-  const unsigned c3base = (unsigned)p.step << 1;
-  for (int item = tid; item < nh * (TILE / 4); item += WARPS * 32) {
-    const int hh = item / (TILE / 4), quad = item % (TILE / 4);
-    const int t0 = tile0 + quad * 4;
-    if (t0 >= geo.l_start || t0 + 4 <= geo.s0) continue;
-    const int hrng = p.rng_head_is_kv ? g : (h0 + hh);
-    const unsigned c1 = ((unsigned)b << 16) | (unsigned)hrng;
-#pragma unroll
-    for (int stream = 0; stream < 2; ++stream) {
-      const unsigned bound = stream ? VATTN_CAND1_BOUND : bound0;
-      if (bound == 0u) continue;
-      const uint4 r = philox4x32_10((unsigned)(t0 >> 2), c1, (unsigned)p.layer, c3base | (unsigned)stream,
-                                    p.seed_lo, p.seed_hi);
-      const unsigned key[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int tok = t0 + e;
-        if (key[e] < bound && tok >= geo.s0 && tok < geo.l_start) {
-          const unsigned pos = atomicAdd(&s_cnt[stream * MAXH + hh], 1u);
-          s_list[stream * MAXH + hh][pos] = make_uint2(key[e], (unsigned)tok);
-        }
-      }
-    }
-  }
-  __syncthreads();
-  const int warp = tid >> 5, lane = tid & 31;
-  for (int l = warp; l < 2 * MAXH; l += WARPS) {
-    const int stream = l / MAXH, hh = l % MAXH;
-    const unsigned cnt = s_cnt[l];
-    if (hh >= nh || cnt == 0) continue;
-    const long long bh = (long long)b * p.Hq + h0 + hh;
-    unsigned base = 0;
-    if (lane == 0) base = atomicAdd(&p.cand_cnt[(long long)stream * p.B * p.Hq + bh], cnt);
-    base = __shfl_sync(0xFFFFFFFFu, base, 0);
-    uint2* dst = p.cand + ((long long)stream * p.B * p.Hq + bh) * p.cand_cap;
-    for (unsigned j = lane; j < cnt; j += 32)
-      if (base + j < (unsigned)p.cand_cap) dst[base + j] = s_list[l][j];
-  }
-}
+// bf16: persistent producer / consumer kernel
+constexpr int CWN = 4;                              // consumer warps per CTA
+constexpr int SCORE_THREADS = (CWN + 1) * 32;       // + one producer warp
+constexpr int MIN_UNIT_PAGES = 16;
+constexpr int UNITS_PER_CTA = 8;                    // target for batches (a single sequence gets one unit per CTA)
 
-// ---------------------------------------------------------------------------------------------
-// bf16: tensor-core path, up to 8 heads per CTA
-// ---------------------------------------------------------------------------------------------
-// bf16, streaming variant: every warp owns a ring of NST shared-memory stages and keeps NST pages
-// (16 tokens x d, one contiguous slab of the paged cache) in flight with bulk asynchronous copies
-// (cp.async.bulk + mbarrier transaction counts); fragments are read back with 16-byte shared loads.
-// The copies need no registers while in flight, so an SM holds ~130 KB of outstanding reads with two
-// resident CTAs.  A warp walks the pages p = w, w + W, w + 2W, ... of its (batch row, KV head).
-constexpr int NST = 4;          // stages per warp
-constexpr int CWARPS = 8;       // warps of a CTA that pre-filter sampling keys (two per streaming warp)
+struct __align__(16) StageMeta {   // written by the producer before it arms the stage's full barrier
+  int tok0;             // first token of the page; < 0: no more work for the consumer that owns this stage
+  int n;                // tokens of the sequence
+  int bh0;              // batch row * Hq + first query head of the group slice
+  int nh_unit;          // query heads in the slice (<= 8) | running unit number of the CTA << 4: a change of
+};                      // the unit tells the consumer to flush its maxima and reload q
 
-// Sampling-candidate pre-filter, run by the CWARPS candidate warps of a CTA: Philox keys of streams 0
-// and 1 for every (token, head) of the CTA's pages; tokens whose key is below the stream's bound are
-// staged in CTA-wide lists, one per (stream, head), and appended to the global lists every CHUNK pages
-// per warp.  Lanes are items (stream, head, token quad); the 4 lanes of a list are adjacent, so the
-// positions inside a page come from ballots; one shared-memory atomic per (page, list) reserves the
-// range.  Global counters are bumped once per list and flush, which keeps the contended atomics rare.
-constexpr int CL = 256;          // staged entries per (stream, head) list of a CTA
-constexpr int CHUNK = 4;         // pages per candidate warp between two flushes (CWARPS*CHUNK*16*1/4 = 128 expected)
-
-__device__ __forceinline__ void cand_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(CWARPS * 32) : "memory"); }
-
-__device__ void candidate_warps(const Prob& p, int b, int g, int h0, int nh, int n, int page0, int wtot, int npages,
-                                int cw, uint2* clist, unsigned* s_cnt) {
-  const int lane = threadIdx.x & 31;
-  const Geo geo = head_geometry(p, n);
-  if (geo.n_s <= 0) return;                                   // uniform over the CTA
-  const unsigned bound0 = cand0_bound(geo);
-  const int nitems = 8 * nh, nrounds = (nitems + 31) >> 5;
-  const unsigned lmask = 0xFu << (lane & ~3), lt = (1u << lane) - 1u;
-  // pages of this CTA: page0 + j * wtot for the streaming warp j % WARPS; candidate warp cw takes the
-  // CTA-local page slots cw, cw + CWARPS, ...   (slot s = page page0_cta + (s % WARPS) + (s / WARPS) * wtot)
-  const int slots = (npages > page0) ? ((npages - 1 - page0) / wtot + 1) * WARPS : 0;   // upper bound, CTA-uniform
-  const int nchunks = (slots + CWARPS * CHUNK - 1) / (CWARPS * CHUNK);
-  if (cw * 32 + lane < 16) s_cnt[cw * 32 + lane] = 0u;
-  cand_barrier();
-  for (int c = 0; c < nchunks; ++c) {
-    for (int kk = 0; kk < CHUNK; ++kk) {
-      const int slot = (c * CHUNK + kk) * CWARPS + cw;
-      const int page = page0 + (slot % WARPS) + (slot / WARPS) * wtot;
-      const int tok0 = page << 4;
-      if (page >= npages || tok0 >= geo.l_start || tok0 + 16 <= geo.s0) continue;
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        if (r >= nrounds) break;
-        const int item = 32 * r + lane;
-        const int L = item >> 2, quad = item & 3;
-        const int stream = L / nh, hh = L % nh;
-        const unsigned bound = (item < nitems) ? (stream ? VATTN_CAND1_BOUND : bound0) : 0u;
-        const int t0 = tok0 + quad * 4;
-        unsigned key[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-        if (bound) {
-          const int hrng = p.rng_head_is_kv ? g : (h0 + hh);
-          const uint4 rr = philox4x32_10((unsigned)(t0 >> 2), ((unsigned)b << 16) | (unsigned)hrng, (unsigned)p.layer,
-                                         ((unsigned)p.step << 1) | (unsigned)stream, p.seed_lo, p.seed_hi);
-          key[0] = rr.x; key[1] = rr.y; key[2] = rr.z; key[3] = rr.w;
-        }
-        unsigned bal[4], total = 0u;
-        bool hit[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int tok = t0 + e;
-          hit[e] = key[e] < bound && tok >= geo.s0 && tok < geo.l_start;
-          bal[e] = __ballot_sync(0xFFFFFFFFu, hit[e]) & lmask;
-          total += __popc(bal[e]);
-        }
-        unsigned base = 0u;
-        if ((lane & 3) == 0 && total) base = atomicAdd(&s_cnt[L], total);
-        base = __shfl_sync(0xFFFFFFFFu, base, lane & ~3);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const unsigned pos = base + __popc(bal[e] & lt);
-          if (hit[e] && pos < (unsigned)CL) clist[L * CL + pos] = make_uint2(key[e], (unsigned)(t0 + e));
-          base += __popc(bal[e]);
-        }
-      }
-    }
-    cand_barrier();
-    // flush: candidate warp cw owns lists cw and cw + CWARPS
-    for (int L = cw; L < 2 * nh; L += CWARPS) {
-      const unsigned raw = s_cnt[L];
-      const unsigned cnt = raw < (unsigned)CL ? raw : (unsigned)CL;
-      if (raw == 0u) continue;
-      const long long slot_g = (long long)(L / nh) * p.B * p.Hq + (long long)b * p.Hq + h0 + (L % nh);
-      unsigned gbase = 0u;
-      // a list that overflowed its staging area is incomplete: poison the global count so that the select
-      // kernels draw from the full context instead
-      if (lane == 0) {
-        if (raw > (unsigned)CL) { atomicOr(&p.cand_cnt[slot_g], 0x80000000u); gbase = (unsigned)p.cand_cap; }
-        else gbase = atomicAdd(&p.cand_cnt[slot_g], cnt);
-      }
-      gbase = __shfl_sync(0xFFFFFFFFu, gbase, 0);
-      uint2* dst = p.cand + slot_g * p.cand_cap;
-      for (unsigned j = lane; j < cnt; j += 32)
-        if (gbase + j < (unsigned)p.cand_cap) dst[gbase + j] = clist[L * CL + j];
-      __syncwarp();
-      if (lane == 0) s_cnt[L] = 0u;
-    }
-    cand_barrier();
-  }
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 template <int D>
-__global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Prob p) {
+__global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p, int qslot_bytes) {
   constexpr int NC = D / 32;
   constexpr int ROWB = D * 2;                 // bytes per row
   constexpr int PAGEB = VATTN_BLOCK * ROWB;   // bytes per (page, KV head) slab
+  constexpr int S = 2048 / D;                 // stages: 64 KB of pages in flight per CTA
   extern __shared__ __align__(128) unsigned char smem_dyn[];
-  const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int role = wid >= WARPS;              // warps 0..3 stream K, warps 4..11 pre-filter sampling keys
-  const int cw = wid - WARPS;                 // candidate warp index (role 1)
-  const int warp = role ? (cw & (WARPS - 1)) : wid;      // the streaming warp whose pages this warp works on
-  unsigned char* ring = smem_dyn + (size_t)warp * NST * PAGEB;
-  uint2* clist = reinterpret_cast<uint2*>(smem_dyn + (size_t)WARPS * NST * PAGEB);
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)WARPS * NST * PAGEB +
-                                                                   (size_t)16 * CL * sizeof(uint2)) + warp * NST;
-  unsigned* s_cnt = reinterpret_cast<unsigned*>(smem_dyn + (size_t)WARPS * NST * PAGEB + (size_t)16 * CL * sizeof(uint2) +
-                                                (size_t)WARPS * NST * 8);
+  unsigned char* ring = smem_dyn;
+  unsigned char* qring = ring + (size_t)S * PAGEB;
+  StageMeta* meta = reinterpret_cast<StageMeta*>(qring + (size_t)S * qslot_bytes);
+  unsigned long long* full = reinterpret_cast<unsigned long long*>(meta + S);
+  unsigned long long* empty = full + S;
+  int* s_len = reinterpret_cast<int*>(empty + S);    // [B]   clamped sequence lengths
+  int* s_pref = s_len + p.B;                         // [B+1] units before batch row b
+  int* s_misc = s_pref + p.B + 1;                    // [16]
+  const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
   DEV_BEGIN(p, 1);
   pdl_trigger();
-  const int b = blockIdx.z;
-  const int n = clamped_len(p, b);
-  const int npages = (n + 15) >> 4;
+
+  // ---- units: every CTA derives the same decomposition from the sequence lengths
   const int GC = (p.G + 7) >> 3;
-  const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
-  const int gr = lane >> 2, t = lane & 3;
-  const int h0 = g * p.G + hc * 8;
-  const int nh = min(8, p.G - hc * 8);
-  const int wglob = blockIdx.x * WARPS + warp, wtot = gridDim.x * WARPS;
-  const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;    // pages this warp owns
-  if (role == 1) {
-#ifdef VATTN_DEV_TIMING
-    if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 4] = dev_gtime();
-#endif
-    candidate_warps(p, b, g, h0, nh, n, blockIdx.x * WARPS, wtot, npages, cw, clist, s_cnt);
-#ifdef VATTN_DEV_TIMING
-    if (p.devt && lane == 0 && wglob == 0 && blockIdx.y == 0) p.devt[32 + 5] = dev_gtime();
-    if (p.devt && lane == 0) atomicMax(&p.devt[32 + 6], dev_gtime());
-#endif
-    return;
+  const int GPB = p.Hkv * GC;                         // (KV head, head slice) groups per batch row
+  int my_pages = 0;
+  for (int b = tid; b < p.B; b += SCORE_THREADS) {
+    const int n = clamped_len(p, b);
+    s_len[b] = n;
+    my_pages += (n + 15) >> 4;
   }
-  if (mine == 0) return;                      // streaming warps use no CTA-wide barrier
+#pragma unroll
+  for (int mk = 16; mk >= 1; mk >>= 1) my_pages += __shfl_xor_sync(0xFFFFFFFFu, my_pages, mk);
+  if (lane == 0) s_misc[wid] = my_pages;
+  if (tid < S) { mbar_init(&full[tid], 1); mbar_init(&empty[tid], 1); }
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  __syncthreads();
+  long long pages_total = 0;
+  for (int w = 0; w <= CWN; ++w) pages_total += s_misc[w];
+  const long long want_units = (long long)gridDim.x * (p.B == 1 ? 1 : UNITS_PER_CTA);
+  long long ch64 = (pages_total * GPB + want_units - 1) / want_units;
+  const int CH = (int)(ch64 < MIN_UNIT_PAGES ? MIN_UNIT_PAGES : ch64);      // pages per unit
+  if (wid == 0) {                                     // exclusive prefix of the units per batch row
+    int carry = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      const int units = (b < p.B) ? GPB * ((((s_len[b] + 15) >> 4) + CH - 1) / CH) : 0;
+      int incl = units;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (b < p.B) s_pref[b] = carry + incl - units;
+      carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (lane == 0) s_pref[p.B] = carry;
+  }
+  __syncthreads();
+  const int U = s_pref[p.B];
   const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
 
-  if (lane < NST) mbar_init(&bars[lane], 1);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncwarp();
-
-  // page ids of this warp's first 32 pages (lane l holds the l-th); refreshed every 32 pages
-  int pg_ids = 0;
-  auto load_ids = [&](int k_base) {
-    const int k = k_base + lane;
-    pg_ids = (k < mine) ? page_of(p, b, wglob + k * wtot) : 0;
-  };
-  auto issue = [&](int k, int pg) {       // lane 0 only
-    unsigned long long* bar = &bars[k % NST];
-    unsigned char* dst = ring + (size_t)(k % NST) * PAGEB;
-    const bf16_t* src = kc + (long long)pg * p.sb + (long long)g * p.sh;
-    mbar_expect_tx(bar, PAGEB);
-    if (p.st == D) bulk_g2s(dst, src, PAGEB, bar);
-    else
-      for (int r = 0; r < VATTN_BLOCK; ++r) bulk_g2s(dst + r * ROWB, src + (long long)r * p.st, ROWB, bar);
-  };
-  load_ids(0);
-  for (int k = 0; k < min(NST, mine); ++k) {
-    const int pg = __shfl_sync(0xFFFFFFFFu, pg_ids, k);
-    if (lane == 0) issue(k, pg);
+  if (wid == CWN) {
+    // =============================================================== producer warp
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    long long i = 0;                                  // stages armed so far
+    int ucount = 0;
+    bool failed = false;
+    int u = blockIdx.x;
+    while (u < U && !failed) {
+      unsigned nxt = 0u;
+      if (lane == 0) nxt = atomicAdd(p.unit_ctr, 1u);  // the unit after this one; the round trip hides behind this unit
+      int lo = 0, hi = p.B - 1;                        // last batch row whose first unit is <= u
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_pref[mid] <= u) lo = mid; else hi = mid - 1;
+      }
+      const int b = lo, n = s_len[b], np = (n + 15) >> 4;
+      const int chunks = (np + CH - 1) / CH;
+      const int r = u - s_pref[b];
+      const int gc = r / chunks, chunk = r % chunks;
+      const int g = gc / GC, hc = gc % GC;
+      const int h0 = g * p.G + hc * 8, nh = min(8, p.G - hc * 8);
+      const int pA = chunk * CH, cnt = min(CH, np - pA);
+      const bf16_t* qsrc = reinterpret_cast<const bf16_t*>(p.q) + ((long long)b * p.Hq + h0) * D;
+      // S lanes arm S stages at a time, each lane its own: wait for the stage to be handed back, describe the
+      // page, post the copy.  The page ids of the next round are requested before this round's waits.
+      int pid_next = (lane < S && lane < cnt) ? page_of(p, b, pA + lane) : 0;
+      for (int k0 = 0; k0 < cnt; k0 += S) {
+        const int pid = pid_next;
+        pid_next = (lane < S && k0 + S + lane < cnt) ? page_of(p, b, pA + k0 + S + lane) : 0;
+        bool ok = true;
+        if (lane < S && k0 + lane < cnt) {
+          const long long ii = i + lane;
+          const int stage = (int)(ii % S);
+          if (ii >= S) ok = mbar_wait(&empty[stage], (unsigned)((ii / S) - 1) & 1u);
+          if (ok) {
+            const int k = k0 + lane;
+            StageMeta m;
+            m.tok0 = (pA + k) << 4; m.n = n; m.bh0 = b * p.Hq + h0; m.nh_unit = nh | (ucount << 4);
+            meta[stage] = m;
+            const bool with_q = k < CWN;              // every consumer meets q on its first page of the unit
+            const unsigned qbytes = (unsigned)(nh * ROWB);
+            unsigned char* dst = ring + (size_t)stage * PAGEB;
+            const bf16_t* src = kc + (long long)pid * p.sb + (long long)g * p.sh;
+            mbar_expect_tx(&full[stage], PAGEB + (with_q ? qbytes : 0u));
+            if (with_q) bulk_g2s(qring + (size_t)stage * qslot_bytes, qsrc, qbytes, &full[stage]);
+            if (p.st == D) bulk_g2s(dst, src, PAGEB, &full[stage]);
+            else
+              for (int rr = 0; rr < VATTN_BLOCK; ++rr) bulk_g2s(dst + rr * ROWB, src + (long long)rr * p.st, ROWB, &full[stage]);
+          }
+        }
+        i += min(S, cnt - k0);
+        if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
+      }
+      ++ucount;
+      u = (int)gridDim.x + (int)__shfl_sync(0xFFFFFFFFu, nxt, 0);
+    }
+    // one end mark per consumer (consumer w owns the stages i = w mod CWN)
+    if (!failed) {
+      bool ok = true;
+      if (lane < CWN) {
+        const long long ii = i + lane;
+        const int stage = (int)(ii % S);
+        if (ii >= S) ok = mbar_wait(&empty[stage], (unsigned)((ii / S) - 1) & 1u);
+        if (ok) {
+          StageMeta m;
+          m.tok0 = -1; m.n = 0; m.bh0 = 0; m.nh_unit = 0;
+          meta[stage] = m;
+          mbar_arrive(&full[stage]);
+        }
+      }
+      i += CWN;
+      if (!__all_sync(0xFFFFFFFFu, ok)) failed = true;
+    }
+    if (failed) {
+      // a consumer gave up: report, and give the copies still in flight a bounded chance to land before the
+      // shared memory is released
+      if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+      // (a stage that was never armed simply runs into the wait limit)
+      for (long long j = (i > S ? i - S : 0) + lane; j < i; j += 32) mbar_wait(&full[j % S], (unsigned)(j / S) & 1u);
+    }
+    DEV_END(p, 1);
+    return;
   }
 
+  // ================================================================= consumer warps
+  const int gr = lane >> 2, t = lane & 3;
   uint4 bq[NC];
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    bq[c] = make_uint4(0u, 0u, 0u, 0u);
-    if (gr < nh)
-      bq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
-                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
-  }
+  for (int c = 0; c < NC; ++c) bq[c] = make_uint4(0u, 0u, 0u, 0u);
   float runmax[2] = {-INFINITY, -INFINITY};
   unsigned kabs = 0u;
-  bool failed = false;
+  int cur_unit = -1, cur_bh0 = 0, cur_nh = 0;       // cur_unit holds nh_unit of the unit in progress
+  auto flush = [&]() {                                // running maxima of the unit just finished
+    if (cur_unit < 0) return;
+#pragma unroll
+    for (int mask = 4; mask < 32; mask <<= 1) {
+      runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
+      runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
+    }
+#pragma unroll
+    for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
+    if (lane < 4) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int hl = 2 * lane + e;
+        if (hl < cur_nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[cur_bh0 + hl], ord_f32(runmax[e]));
+      }
+    }
+    if (lane == 0) {
+      const unsigned mx = max(kabs & 0xFFFFu, kabs >> 16);
+      const int b = cur_bh0 / p.Hq, g = (cur_bh0 % p.Hq) / p.G;
+      atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);
+    }
+    runmax[0] = runmax[1] = -INFINITY;
+    kabs = 0u;
+  };
 
-  for (int k = 0; k < mine; ++k) {
-    const int s = k % NST;
-    if (!mbar_wait(&bars[s], (unsigned)(k / NST) & 1u)) { failed = true; break; }
-    const unsigned char* stg = ring + (size_t)s * PAGEB;
-    const int tok0 = (wglob + k * wtot) << 4;
+  for (long long i = wid;; i += CWN) {
+    const int stage = (int)(i % S);
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full[stage], (unsigned)(i / S) & 1u))) {   // warp-uniform decision
+      if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+      break;
+    }
+    const StageMeta m = meta[stage];
+    if (m.tok0 < 0) break;
+    const int m_nh = m.nh_unit & 15;
+    if (m.nh_unit != cur_unit) {
+      flush();
+      cur_unit = m.nh_unit; cur_bh0 = m.bh0; cur_nh = m_nh;
+      const unsigned char* qs = qring + (size_t)stage * qslot_bytes;
+#pragma unroll
+      for (int c = 0; c < NC; ++c)
+        bq[c] = (gr < m_nh) ? *reinterpret_cast<const uint4*>(qs + gr * ROWB + c * 64 + t * 16) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    const unsigned char* stg = ring + (size_t)stage * PAGEB;
     float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};   // two independent MMA chains
     unsigned klo = 0u, khi = 0u;
 #pragma unroll
@@ -276,57 +250,26 @@ __global__ void __launch_bounds__((WARPS + CWARPS) * 32) k_score_stream(const Pr
       khi = __vimax3_u16x2(khi, ahi.x & 0x7FFF7FFFu, ahi.y & 0x7FFF7FFFu);
       khi = __vimax3_u16x2(khi, ahi.z & 0x7FFF7FFFu, ahi.w & 0x7FFF7FFFu);
     }
+    // the stage (page and query rows) has been read: hand it back to the producer
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty[stage]);
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] += acc1[e];
-    // the stage has been read (the MMAs consumed every fragment): refill it with page k + NST
-    __syncwarp();
-    if (k + NST < mine) {
-      if (((k + NST) & 31) == 0) load_ids(k + NST);
-      const int pg = __shfl_sync(0xFFFFFFFFu, pg_ids, (k + NST) & 31);
-      if (lane == 0) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        issue(k + NST, pg);
-      }
-    }
-    const int tk_lo = tok0 + gr, tk_hi = tok0 + gr + 8;
-    if (tk_lo < n) kabs = __vimax3_u16x2(kabs, klo, 0u);
-    if (tk_hi < n) kabs = __vimax3_u16x2(kabs, khi, 0u);
+    const int tk_lo = m.tok0 + gr, tk_hi = m.tok0 + gr + 8;
+    if (tk_lo < m.n) kabs = __vimax3_u16x2(kabs, klo, 0u);
+    if (tk_hi < m.n) kabs = __vimax3_u16x2(kabs, khi, 0u);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int hl = 2 * t + e;
-      if (hl < nh) {
-        float* dst = p.scores + ((long long)b * p.Hq + h0 + hl) * p.npad;
+      if (hl < m_nh) {
+        float* dst = p.scores + (long long)(m.bh0 + hl) * p.npad;
         const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
-        if (tk_lo < n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
-        if (tk_hi < n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
+        if (tk_lo < m.n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
+        if (tk_hi < m.n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
       }
     }
   }
-  if (failed) {
-    // give the copies still in flight a bounded chance to land before the shared memory is released
-    if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
-    for (int s = 0; s < NST; ++s) mbar_wait(&bars[s], 0u) || mbar_wait(&bars[s], 1u);
-    return;
-  }
-#pragma unroll
-  for (int mask = 4; mask < 32; mask <<= 1) {
-    runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
-    runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
-  }
-#pragma unroll
-  for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
-  if (lane < 4) {
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int hl = 2 * lane + e;
-      if (hl < nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[b * p.Hq + h0 + hl], ord_f32(runmax[e]));
-    }
-  }
-  if (lane == 0) {
-    const unsigned mx = max(kabs & 0xFFFFu, kabs >> 16);
-    atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);
-  }
-  DEV_END(p, 1);
+  flush();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -338,9 +281,6 @@ __global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
   constexpr int RPI = 32 / LPR;      // rows per warp instruction
   constexpr int ITERS = 16 / RPI;    // instructions per page
   constexpr int NV = ITERS * 4;      // partial sums per lane per page (4 heads)
-  __shared__ uint2 s_list[8][TILE];
-  __shared__ unsigned s_cnt[8];
-
   const int b = blockIdx.z;
   const int n = clamped_len(p, b);
   const int tile0 = blockIdx.x * TILE;
@@ -430,41 +370,31 @@ __global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
     }
   }
   if (lane == 0) atomicMax(&p.kabsmax[b * p.Hkv + g], __float_as_uint(kmax));
-  emit_candidates<4>(p, b, g, g * p.G + hc * 4, min(4, p.G - hc * 4), tile0, n, s_list, s_cnt);
 }
 
 }  // namespace
 
 template <int D>
 static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
-  const size_t smem = (size_t)WARPS * NST * VATTN_BLOCK * D * 2 + (size_t)16 * CL * sizeof(uint2) +
-                      (size_t)WARPS * NST * 8 + 16 * sizeof(unsigned);
-  static bool attr_done = false;
-  if (!attr_done) {
+  constexpr int S = 2048 / D, PAGEB = VATTN_BLOCK * D * 2;
+  const int nh_max = p.G < 8 ? p.G : 8;
+  const int qslot_bytes = nh_max * D * 2;
+  const size_t smem = (size_t)S * PAGEB + (size_t)S * qslot_bytes + (size_t)S * sizeof(StageMeta) + (size_t)2 * S * 8 +
+                      sizeof(int) * ((size_t)2 * p.B + 1 + 16);
+  if (smem > 110 * 1024) return cudaErrorInvalidValue;        // batch too large for the in-kernel unit table
+  static size_t attr_sz = 0;
+  if (attr_sz < smem) {
     cudaError_t e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    attr_sz = smem;
   }
-  // one wave of two CTAs per SM; a warp walks pages with stride (CTAs along x) * WARPS
-  const int groups = p.Hkv * ((p.G + 7) / 8) * p.B;
-  const int pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
-  // A single sequence whose groups divide the 2 x 148 resident CTAs (almost) evenly runs as one wave.  Anything
-  // else (several sequences, possibly of different lengths; a group count that leaves SMs idle) is cut into
-  // about eight waves of CTAs with at least 32 pages each, which the hardware scheduler balances.
-  const int slots = 2 * 148;
-  int cx = slots / groups;
-  if (cx < 1) cx = 1;
-  const bool one_wave = p.B == 1 && groups * cx <= slots && (slots - groups * cx) * 20 < slots;
-  if (!one_wave) {
-    cx = (8 * slots + groups - 1) / groups;
-    const int cx_fine = (pages + 31) / 32;
-    if (cx > cx_fine) cx = cx_fine;
-  }
-  const int cx_max = (pages + WARPS - 1) / WARPS;
-  if (cx > cx_max) cx = cx_max;
-  if (cx < 1) cx = 1;
-  dim3 grid(cx, p.Hkv * ((p.G + 7) / 8), p.B), block((WARPS + CWARPS) * 32);
-  k_score_stream<D><<<grid, block, smem, s>>>(p);
+  // persistent: two CTAs per SM, fewer when the problem cannot have that many units
+  const long long pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
+  const long long units_max = (long long)p.B * p.Hkv * ((p.G + 7) / 8) * ((pages + MIN_UNIT_PAGES - 1) / MIN_UNIT_PAGES);
+  const int grid = (int)(units_max < 2 * 148 ? (units_max < 1 ? 1 : units_max) : 2 * 148);
+  k_score_stream<D><<<grid, SCORE_THREADS, smem, s>>>(p, qslot_bytes);
   return cudaGetLastError();
 }
 

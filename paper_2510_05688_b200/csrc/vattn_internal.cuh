@@ -45,6 +45,7 @@ struct Prob {
   unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
   unsigned* tickets;      // [3,B,Hq] "last CTA done" counters (stats, gather, dense)
   unsigned* cand_cnt;     // [2,B,Hq] entries appended to the sampling-candidate lists (may exceed cand_cap)
+  unsigned* unit_ctr;     // [1] work-unit counter of the persistent score kernel
   uint2* cand;            // [2,B,Hq,cand_cap] (Philox key, token) with key below the stream's pre-filter
   int cand_cap;
   unsigned* status;       // [1]
@@ -199,8 +200,9 @@ __device__ __forceinline__ uint4 philox4x32_10(unsigned c0, unsigned c1, unsigne
                                                unsigned k0, unsigned k1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    unsigned hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    unsigned hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const unsigned long long p0 = (unsigned long long)c0 * 0xD2511F53ull;      // one widening multiply each
+    const unsigned long long p1 = (unsigned long long)c2 * 0xCD9E8D57ull;
+    const unsigned hi0 = (unsigned)(p0 >> 32), lo0 = (unsigned)p0, hi1 = (unsigned)(p1 >> 32), lo1 = (unsigned)p1;
     unsigned n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
     k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
@@ -258,6 +260,7 @@ __device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
 
 // launchers (one per translation unit)
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
+cudaError_t launch_cand(const Prob& p, cudaStream_t s);
 cudaError_t launch_select_topk(const Prob& p, cudaStream_t s);
 cudaError_t launch_presort(const Prob& p, cudaStream_t s);
 cudaError_t launch_select_final(const Prob& p, cudaStream_t s);
