@@ -171,6 +171,12 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */)
 /* Number of kernels the last vattn_decode / vattn_dense_decode call on this plan enqueued. */
 int vattn_last_launch_count(const vattn_plan* plan);
 
+/* Measurement aid: while kernels > 0, vattn_decode enqueues only its first `kernels` kernels (in the order
+ * listed for vattn_set_profiling below) and leaves `out` untouched; 0 restores the whole step.  Lets a
+ * harness time one kernel launched back to back, without the launch gaps that events inside a step see.
+ * Errors: INVALID_ARG (kernels outside [0, VATTN_NUM_KERNELS]). */
+int vattn_set_stop_after(vattn_plan* plan, int kernels);
+
 /* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
  * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, sampling-key
  * pre-filter, top-k select, sampling sort, statistics + budget, slow-path final select, gather +

@@ -19,7 +19,7 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
            "vattn_host_staging_bytes", "vattn_decode_host", "vattn_last_status", "vattn_last_launch_count",
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
-           "vattn_dense_decode_noalloc"]
+           "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
 KERNEL_NAMES = ["k_score", "k_cand", "k_select_topk", "k_presort", "k_stats", "k_select_final", "k_gather"]
 
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
     L.vattn_last_launch_count.restype = i32
     L.vattn_strerror.argtypes = [i32]
     L.vattn_strerror.restype = C.c_char_p
+    L.vattn_set_stop_after.argtypes = [vp, i32]
+    L.vattn_set_stop_after.restype = i32
     L.vattn_set_profiling.argtypes = [vp, i32]
     L.vattn_set_profiling.restype = i32
     L.vattn_read_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
@@ -204,6 +206,10 @@ class Plan:
         bits = C.c_uint32(0)
         _check(lib().vattn_last_status(self._h, C.c_void_p(_stream(stream)), C.byref(bits)), "vattn_last_status")
         return int(bits.value)
+
+    def set_stop_after(self, kernels: int):
+        """Measurement aid: decode() enqueues only its first `kernels` kernels (0 = the whole step)."""
+        _check(lib().vattn_set_stop_after(self._h, int(kernels)), "vattn_set_stop_after")
 
     def set_profiling(self, enable: bool):
         _check(lib().vattn_set_profiling(self._h, 1 if enable else 0), "vattn_set_profiling")

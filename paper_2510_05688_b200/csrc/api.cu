@@ -16,6 +16,7 @@ struct vattn_plan {
   unsigned long long* devt;
   // optional per-kernel timing (events are created on first use; no device memory involved)
   bool profiling;
+  int stop_after;           // measurement aid: enqueue only the first stop_after kernels of a step (0 = all)
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
   int prof_calls;           // calls recorded since the last read
   // derived
@@ -163,12 +164,15 @@ int check_common(const vattn_plan* pl, const void* q, const void* kc, const void
 
 #define CU(x) do { if ((x) != cudaSuccess) return VATTN_ERR_CUDA; } while (0)
 
-int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st) {
+// clears the per-step counters: with a kernel for the sparse step (the score kernel overlaps it), with a
+// memset node otherwise
+int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st, bool with_kernel) {
   if (!pl->status_ready) {
     CU(cudaMemsetAsync(p.status, 0, sizeof(unsigned), st));
     pl->status_ready = true;
   }
-  CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
+  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, st));
+  else CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
   return VATTN_OK;
 }
 
@@ -215,6 +219,12 @@ void vattn_plan_destroy(vattn_plan* plan) {
     delete[] plan->ev;
   }
   delete plan;
+}
+
+int vattn_set_stop_after(vattn_plan* plan, int kernels) {
+  if (!plan || kernels < 0 || kernels > VATTN_NUM_KERNELS) return VATTN_ERR_INVALID_ARG;
+  plan->stop_after = kernels;
+  return VATTN_OK;
 }
 
 int vattn_set_profiling(vattn_plan* plan, int enable) {
@@ -304,8 +314,9 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
     p.z2[j - 1] = upper_quantile(0.5 * (p.delta * (16 - j) / 16.0));
   }
   plan->last_launches = 0;
-  rc = prepare_stream(plan, p, st);
+  rc = prepare_stream(plan, p, st, true);
   if (rc != VATTN_OK) return rc;
+  plan->last_launches++;                      // the counter-clearing kernel
   prof_mark(plan, 0, st);
   // score || key pre-filter -> top-k || sampling sort -> sampling compaction -> statistics + budget ->
   // slow-path select (usually nothing to do) -> gather.  The overlaps come from programmatic dependent
@@ -313,19 +324,25 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   // lists beside the top-k select.
   CU(launch_score(p, st));            plan->last_launches++;
   prof_mark(plan, 1, st);
+  if (plan->stop_after == 1) return VATTN_OK;
   CU(launch_cand(p, st));             plan->last_launches++;
   prof_mark(plan, 2, st);
+  if (plan->stop_after == 2) return VATTN_OK;
   if (p.dbg.scores)
     CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
                          sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
   CU(launch_select_topk(p, st));      plan->last_launches++;
   prof_mark(plan, 3, st);
+  if (plan->stop_after == 3) return VATTN_OK;
   CU(launch_presort(p, st));          plan->last_launches++;
   prof_mark(plan, 4, st);
+  if (plan->stop_after == 4) return VATTN_OK;
   CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 5, st);
+  if (plan->stop_after == 5) return VATTN_OK;
   CU(launch_select_final(p, st));     plan->last_launches++;
   prof_mark(plan, 6, st);
+  if (plan->stop_after == 6) return VATTN_OK;
   CU(launch_gather(p, st));           plan->last_launches++;
   prof_mark(plan, 7, st);
   if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
@@ -340,7 +357,7 @@ int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, con
   Prob p;
   fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
   plan->last_launches = 0;
-  rc = prepare_stream(plan, p, st);
+  rc = prepare_stream(plan, p, st, false);
   if (rc != VATTN_OK) return rc;
   int launches = 0;
   CU(launch_dense(p, st, &launches));

@@ -39,6 +39,15 @@ struct __align__(16) StageMeta {   // written by the producer before it arms the
   int nh_unit;          // query heads in the slice (<= 8) | running unit number of the CTA << 4: a change of
 };                      // the unit tells the consumer to flush its maxima and reload q
 
+// Clears the per-step counters (running maxima, tickets, list lengths, unit counter).  A kernel rather than a
+// memset node so that the score kernel behind it can start its prologue and its first copies meanwhile: it
+// lets its dependents go at once and waits for the previous step before it writes.
+__global__ void __launch_bounds__(256) k_zero(unsigned* z, int words) {
+  pdl_trigger();
+  pdl_wait();
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += gridDim.x * blockDim.x) z[i] = 0u;
+}
+
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -60,7 +69,6 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
   int* s_misc = s_pref + p.B + 1;                    // [16]
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
   DEV_BEGIN(p, 1);
-  pdl_trigger();
 
   // ---- units: every CTA derives the same decomposition from the sequence lengths
   const int GC = (p.G + 7) >> 3;
@@ -109,9 +117,9 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     int ucount = 0;
     bool failed = false;
     int u = blockIdx.x;
+    bool first = true;
     while (u < U && !failed) {
       unsigned nxt = 0u;
-      if (lane == 0) nxt = atomicAdd(p.unit_ctr, 1u);  // the unit after this one; the round trip hides behind this unit
       int lo = 0, hi = p.B - 1;                        // last batch row whose first unit is <= u
       while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
@@ -154,10 +162,17 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
         }
         i += min(S, cnt - k0);
         if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
+        if (k0 == 0) {
+          // The first copies of the CTA are under way; from here on the kernel touches what the grid before
+          // it clears (k_zero), so wait for it, and only then let the key pre-filter behind this grid start.
+          if (first) { pdl_wait(); pdl_trigger(); first = false; }
+          if (lane == 0) nxt = atomicAdd(p.unit_ctr, 1u);  // the unit after this one; the round trip hides behind this unit
+        }
       }
       ++ucount;
       u = (int)gridDim.x + (int)__shfl_sync(0xFFFFFFFFu, nxt, 0);
     }
+    if (first) { pdl_wait(); pdl_trigger(); }
     // one end mark per consumer (consumer w owns the stages i = w mod CWN)
     if (!failed) {
       bool ok = true;
@@ -219,6 +234,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     kabs = 0u;
   };
 
+  pdl_wait();                                         // scores and counters of the previous step are free now
+  pdl_trigger();
   for (long long i = wid;; i += CWN) {
     const int stage = (int)(i % S);
     if (!__all_sync(0xFFFFFFFFu, mbar_wait(&full[stage], (unsigned)(i / S) & 1u))) {   // warp-uniform decision
@@ -394,8 +411,15 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   const long long pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
   const long long units_max = (long long)p.B * p.Hkv * ((p.G + 7) / 8) * ((pages + MIN_UNIT_PAGES - 1) / MIN_UNIT_PAGES);
   const int grid = (int)(units_max < 2 * 148 ? (units_max < 1 ? 1 : units_max) : 2 * 148);
-  k_score_stream<D><<<grid, SCORE_THREADS, smem, s>>>(p, qslot_bytes);
-  return cudaGetLastError();
+  return launch_pdl(k_score_stream<D>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
+}
+
+cudaError_t launch_zero(unsigned* z, size_t bytes, cudaStream_t s) {
+  const int words = (int)(bytes / sizeof(unsigned));
+  int grid = (words + 1023) / 1024;
+  if (grid > 148) grid = 148;
+  if (grid < 1) grid = 1;
+  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words);
 }
 
 cudaError_t launch_score(const Prob& p, cudaStream_t s) {
