@@ -445,12 +445,12 @@ def main():
         "k_select_topk": n_tot * Hq * 4,
         "k_presort": int(0.25 * n_tot * Hq) * 8 + int(b0s.sum()) * 8 + 2 * n_tot * Hq // 8,
         "k_stats": int(n_f + b0s.sum()) * d * es * 2,
-        "k_select_final": n_tot * Hq // 8,
+        "k_budget": n_tot * Hq // 8,
         "k_gather": int(b_dyn.sum()) * (d * es + 4),
     }
     # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2_llama8b.md
     traffic = {"k_score": 68.02e6, "k_cand": 0.02e6, "k_select_topk": 4.33e6, "k_presort": 2.55e6,
-               "k_stats": 25.59e6, "k_select_final": 0.04e6, "k_gather": 20.14e6}
+               "k_stats": 25.59e6, "k_budget": 0.04e6, "k_gather": 20.14e6}
     peak, peak_kind = measured_peaks()
     kern = {}
     for name in vb.KERNEL_NAMES:

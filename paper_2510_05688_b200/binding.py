@@ -21,7 +21,7 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
            "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
-KERNEL_NAMES = ["k_score", "k_cand", "k_select_topk", "k_presort", "k_stats", "k_select_final", "k_gather"]
+KERNEL_NAMES = ["k_score", "k_cand", "k_select_topk", "k_presort", "k_stats", "k_budget", "k_gather"]
 
 
 class Shape(C.Structure):

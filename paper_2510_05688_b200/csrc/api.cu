@@ -340,7 +340,7 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 5, st);
   if (plan->stop_after == 5) return VATTN_OK;
-  CU(launch_select_final(p, st));     plan->last_launches++;
+  CU(launch_budget(p, st));     plan->last_launches++;
   prof_mark(plan, 6, st);
   if (plan->stop_after == 6) return VATTN_OK;
   CU(launch_gather(p, st));           plan->last_launches++;

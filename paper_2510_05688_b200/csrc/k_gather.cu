@@ -53,7 +53,7 @@ struct Gather {
       return;
     }
     // I_dyn: the first b entries of the pre-sorted residual list when the budget fits it, else the list the
-    // slow-path select wrote (same predicate as in k_select_final)
+    // slow-path select wrote (same predicate as in k_budget)
     const bool presorted = meta.b < meta.n_s && meta.sorted_cnt >= meta.b;
     const int* dyn = presorted ? p.sort_idx + (long long)bh * p.cand_cap : p.dyn_idx + (long long)bh * p.npad;
     const int* dph = dyn + (presorted ? p.sort_phys_delta : p.phys_delta);

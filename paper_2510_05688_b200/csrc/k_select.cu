@@ -4,7 +4,8 @@
 //                   (Algorithm 1 line 3, "oracle top-k" of Sec. 3).
 //  k_presort      : the base sample I_bs = uniform-sample of b0 residual tokens (Algorithm 2 line 1) and the
 //                   residual in the order in which the final sample draws it (Algorithm 1 line 7).
-//  k_select_final : I_dyn = uniform-sample of b residual tokens, for the heads k_presort could not serve.
+//  k_budget       : the budget b from the statistics partials, then I_dyn = uniform-sample of b residual
+//                   tokens for the heads k_presort could not serve.
 //
 // All selections are "the c smallest (key, index) pairs".  The generic form is an 8-bit-digit radix select
 // over 32-bit keys held in shared memory, followed by an ordered compaction through bitmaps, so its lists
@@ -24,6 +25,7 @@
 // known, tokens above T + 2*gamma are certainly selected and tokens below T - 2*gamma certainly not;
 // the few in between are rescored in fp64 from their K rows and ranked exactly.
 #include "vattn_internal.cuh"
+#include <math_constants.h>
 
 namespace {
 
@@ -668,7 +670,7 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
 // members of I_t are dropped, by an order-preserving compaction: stream 0 keeps the first b0 survivors,
 // stream 1 all of them (the gather kernel later reads the first b, once b is known).  Lists that cannot
 // serve (overflow, too long for shared memory, fewer than b0 survivors, b0 = whole residual) fall back to
-// the full-context select: here for stream 0, in k_select_final for stream 1 (sorted_cnt = -1).
+// the full-context select: here for stream 0, in k_budget for stream 1 (sorted_cnt = -1).
 constexpr int SORT_BUCKETS = 4096;
 constexpr int SORT_BUCKET_MAX = 64;
 constexpr size_t SORT_FIXED_BYTES = sizeof(int) * (2 * SORT_BUCKETS + 1 + 64);      // + nwords words
@@ -835,22 +837,138 @@ __global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, in
   DEV_END(p, devk);
 }
 
-// Final sample, slow path and introspection.  When the budget fits the pre-sorted list (b <= sorted_cnt
-// and b < n_s) the gather kernel reads I_dyn = sorted[0..b) directly and this kernel only copies it to
-// the debug buffer if one is registered.  Otherwise (whole residual, budget beyond the list, unusable
-// list) it draws the sample from the full context and writes it ascending to dyn_idx.
+// Budget (Algorithm 2, Theorem 4.3 / Corollaries D.2) and the slow path of the final sample.
+//
+// One CTA per head.  The partials of the statistics kernel are added in split order (every thread requests
+// all partials of its element at once: one memory round trip), then warp 0 evaluates
+//     sigma^2, Tr(Sigma), D_hat, |N_hat|,  b_D, b_N, b_SDPA,  b = clamp(ceil(b_X), b0, n_s)
+// in fp64 (the two square-root / division chains on two lanes, the 15 split points of b_SDPA on 15 lanes).
+// Heads whose I_dyn is a prefix of the pre-sorted list (b < n_s and b <= sorted_cnt) are done: the gather
+// kernel reads the prefix (it is copied to the debug buffer when one is registered).  For the others the
+// sample is drawn from the full context and written ascending to dyn_idx.
+__device__ __forceinline__ int ceil_sat(double x) {
+  if (!isfinite(x) || x >= 2147483647.0) return 2147483647;
+  return (int)ceil(x);
+}
+
 template <bool CACHED>
-__global__ void __launch_bounds__(NT, 1) k_select_final(const Prob p, int bigbytes) {
+__global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int tid = threadIdx.x;
+  __shared__ double tot[2][128 + 3];
+  __shared__ double piv[128 + 1];
+  __shared__ int s_b;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 4);
   pdl_trigger();
   pdl_wait();
-  const HeadMeta meta = p.meta[bh];
-  if (p.dbg.dyn_cnt && tid == 0) p.dbg.dyn_cnt[bh] = meta.b;
-  if (meta.n == 0 || meta.b <= 0) return;
+  HeadMeta meta = p.meta[bh];
+  const int D = p.D, NE = D + 3, S = p.stat_splits;
+  const int n_s = meta.n_s, b0 = meta.b0;
+  if (meta.n == 0) {
+    if (tid == 0) {
+      p.meta[bh].b = 0;
+      if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = 0;
+      if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
+      if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
+    }
+    return;
+  }
+  // ---- partial sums in split order; kind 0 = deterministic rows, kind 1 = base-sample rows
+  for (int item = tid; item < 2 * NE; item += NT) {
+    const int kind = item / NE, e = item % NE;
+    const double* src = p.stat_part + ((long long)bh * 2 * VATTN_STAT_MAXS + kind * S) * NE + e;
+    double v[VATTN_STAT_MAXS];
+#pragma unroll
+    for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;
+    double sum = 0.0;
+#pragma unroll
+    for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) sum += v[sp];
+    tot[kind][e] = sum;
+  }
+  // the pivot the base-row CTAs used (all of them computed the same numbers; split 0 published them)
+  for (int e = tid; e <= D; e += NT) piv[e] = (b0 > 0) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
+  __syncthreads();
+  double* det = p.det_sums + (long long)bh * (D + 1);
+  for (int e = tid; e <= D; e += NT) det[e] = tot[0][e];
+  if (warp == 0) {
+    const double Dfv = tot[0][D];
+    const double ratio = (b0 > 0) ? (double)n_s / (double)b0 : 0.0;
+    double nn = 0.0, sr2 = 0.0;                 // |N_hat|^2 and sum_j (sum_i r'_ij)^2
+    for (int e = lane; e < D; e += 32) {
+      const double srj = tot[1][e];
+      const double nh = tot[0][e] + ratio * (srj + (double)b0 * piv[e]);
+      nn = fma(nh, nh, nn);
+      sr2 = fma(srj, srj, sr2);
+    }
+#pragma unroll
+    for (int mask = 16; mask >= 1; mask >>= 1) {
+      nn += __shfl_xor_sync(0xFFFFFFFFu, nn, mask);
+      sr2 += __shfl_xor_sync(0xFFFFFFFFu, sr2, mask);
+    }
+    const double Nnorm = sqrt(nn);
+    double sigma2 = 0.0, trace = 0.0, Dhat = Dfv, A = 0.0, Bn = 0.0;
+    int bD = 0, bN = 0, bS = 0, bfin = 0;
+    if (n_s > 0) {                              // uniform over the warp
+      const double Swv = tot[1][D], Swwv = tot[1][D + 1], Srrv = tot[1][D + 2];
+      // lane 0: the denominator chain, lane 1: the numerator chain (each: division, square root, division)
+      if (lane == 0) {
+        if (b0 >= 2) sigma2 = fmax(0.0, (Swwv - Swv * Swv / (double)b0) / (double)(b0 - 1));
+        Dhat = Dfv + ratio * (Swv + (double)b0 * piv[D]);
+        A = (double)n_s * sqrt(sigma2) / Dhat;
+      } else if (lane == 1) {
+        if (b0 >= 2) trace = fmax(0.0, (Srrv - sr2 / (double)b0) / (double)(b0 - 1));
+        Bn = (double)n_s * sqrt(trace) / Nnorm;
+      }
+      A = __shfl_sync(0xFFFFFFFFu, A, 0);
+      Bn = __shfl_sync(0xFFFFFFFFu, Bn, 1);
+      trace = __shfl_sync(0xFFFFFFFFu, trace, 1);
+      // b_SDPA: lane jj takes split point jj of the failure probability
+      double c2 = CUDART_INF;
+      if (lane < 15) {
+        const double c = p.z1[lane] * A + p.z2[lane] * Bn;
+        c2 = c * c;
+      }
+      const bool nan = __any_sync(0xFFFFFFFFu, c2 != c2);
+      double mn = c2;
+#pragma unroll
+      for (int mask = 16; mask >= 1; mask >>= 1) mn = fmin(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, mask));
+      if (lane == 0) {
+        double t = p.z_delta * A / p.eps;
+        const double b_D = t * t;
+        t = p.z_delta * Bn / p.eps;
+        const double b_N = t * t;
+        const double b_S = nan ? CUDART_NAN : 4.0 / (p.eps * p.eps) * mn;
+        bD = ceil_sat(b_D); bN = ceil_sat(b_N); bS = ceil_sat(b_S);
+        const double bx = p.mode == 1 ? b_D : (p.mode == 2 ? b_N : b_S);
+        if (p.force_budget >= 0) bfin = min(p.force_budget, n_s);
+        else {
+          if (!isfinite(bx)) atomicOr(p.status, VATTN_STATUS_NONFINITE);
+          bfin = min(max(ceil_sat(bx), b0), n_s);
+        }
+      }
+    }
+    if (lane == 0) {
+      s_b = bfin;
+      p.meta[bh].b = bfin;
+      if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = bfin;
+      if (p.dbg.budgets) {
+        int* o = p.dbg.budgets + bh * 4;
+        o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bfin;
+      }
+      if (p.dbg.stats) {
+        double* o = p.dbg.stats + bh * 8;
+        o[0] = Dfv; o[1] = sigma2; o[2] = trace; o[3] = Dhat; o[4] = Nnorm; o[5] = (double)n_s; o[6] = (double)b0;
+        o[7] = (double)meta.m;
+      }
+    }
+  }
+  __syncthreads();
+  meta.b = s_b;
+  DEV_MARK(p, 4, 2, bh == 0);
+  if (meta.b <= 0) return;
+  // ---- final sample
   if (meta.b < meta.n_s && meta.sorted_cnt >= meta.b) {
     if (p.dbg.dyn_idx) {
       const int* src = p.sort_idx + (long long)bh * p.cand_cap;
@@ -882,7 +1000,7 @@ static int big_bytes(const Prob& p, bool final_kernel) {
   size_t b = keys > pairs ? keys : pairs;
   const size_t fixed = sizeof(double) * VATTN_BANDCAP + 4 * sizeof(unsigned) * (size_t)p.nwords + sizeof(unsigned) * 256 +
                        sizeof(int) * (VATTN_BANDCAP + NBIN + 2 * CANDCAP + 64);
-  const size_t limit = 227 * 1024;
+  const size_t limit = 222 * 1024;                            // 227 KB per CTA minus the kernels' static arrays
   if (fixed + b > limit) b = (limit - fixed) / 16 * 16;       // fewer staged pairs: the list path then declines
   return (int)b;
 }
@@ -947,6 +1065,6 @@ cudaError_t launch_presort(const Prob& p, cudaStream_t s) {
   return keycap_of(p) > 0 ? launch_presort_t(k_presort<true>, p, s) : launch_presort_t(k_presort<false>, p, s);
 }
 
-cudaError_t launch_select_final(const Prob& p, cudaStream_t s) {
-  return keycap_of(p) > 0 ? launch_sel(k_select_final<true>, p, s, true) : launch_sel(k_select_final<false>, p, s, true);
+cudaError_t launch_budget(const Prob& p, cudaStream_t s) {
+  return keycap_of(p) > 0 ? launch_sel(k_budget<true>, p, s, true) : launch_sel(k_budget<false>, p, s, true);
 }

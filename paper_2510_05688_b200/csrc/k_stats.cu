@@ -4,8 +4,8 @@
 // are gathered (K and V), rescored in fp64 and reduced:
 //     D_f = sum_{I_f} w_i,  N_f = sum_{I_f} w_i V[i]                       (Sec. 4.1, N_f and D_f)
 //     sum w, sum w^2, sum r, sum r.r over I_bs with r_i = w_i V[i]           (Algorithm 2, get-stats)
-// with w_i = exp(s_i - m).  The last CTA of a head ("ticket") adds the partials in a fixed order and
-// evaluates the budgets of Corollaries D.2 and Theorem 4.3, b = clamp(ceil(b_X), b0, n_s).
+// with w_i = exp(s_i - m).  Every CTA leaves one partial; the budget kernel behind this one adds them in a
+// fixed order and evaluates the budgets of Corollaries D.2 and Theorem 4.3.
 //
 // Everything that decides the integer budget is fp64: the same inputs must give the same ceil() as a
 // plain fp64 evaluation.  Variances are accumulated around a pivot (the first base-sample row), which
@@ -13,8 +13,9 @@
 //
 // Grid: per head, `stat_splits` CTAs take the deterministic rows and `stat_splits` CTAs the base-sample
 // rows (two code paths with disjoint accumulators, which halves the register footprint of either).
-// A row group (LPR lanes) keeps 4 rows in flight: indices, page ids and the 16-byte row slices of a
-// batch are all requested before the first is used.
+// A row group (LPR lanes) works in batches of UN rows and keeps two batches in flight: the 16-byte row
+// slices of batch k + 1 and the indices of batch k + 2 are requested before batch k is reduced, so the
+// fp64 arithmetic of one batch hides the memory round trip of the next.
 #include "vattn_internal.cuh"
 #include <math_constants.h>
 
@@ -22,8 +23,8 @@ namespace {
 
 constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
-constexpr int UN = 4;            // rows in flight per row group
-constexpr int MAXS = 16;         // most split CTAs per head and kind
+constexpr int UN = 2;            // rows per batch of a row group; two batches are in flight (double buffer)
+constexpr int MAXS = VATTN_STAT_MAXS;   // most split CTAs per head and kind
 
 template <typename T> struct Raw;
 template <> struct Raw<float> {
@@ -74,20 +75,17 @@ template <typename T, int D>
 __device__ __forceinline__ void weights64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T> (&row)[UN],
                                           double m, int j, double (&w)[UN]) {
   constexpr int LPR = D / Elem<T>::EPL;
-  static_assert(UN == 4 && LPR >= UN, "one lane per row of the batch");
+  static_assert((UN == 2 || UN == 4) && LPR >= UN, "one lane per row of the batch");
   double d[UN];
 #pragma unroll
   for (int u = 0; u < UN; ++u) d[u] = dot64<T, D>(qf, row[u]);
   const int mu = j & (UN - 1);
-  const double mine = mu == 0 ? d[0] : (mu == 1 ? d[1] : (mu == 2 ? d[2] : d[3]));
+  double mine = d[0];
+#pragma unroll
+  for (int u = 1; u < UN; ++u) mine = (mu == u) ? d[u] : mine;
   const double wm = exp(mine * (double)p.scale - m);
 #pragma unroll
   for (int u = 0; u < UN; ++u) w[u] = __shfl_sync(0xFFFFFFFFu, wm, u, LPR);
-}
-
-__device__ __forceinline__ int ceil_sat(double x) {
-  if (!isfinite(x) || x >= 2147483647.0) return 2147483647;
-  return (int)ceil(x);
 }
 
 template <typename T, int D>
@@ -96,9 +94,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   constexpr int NE = D + 3;               // det CTA: N_f[D], D_f;  base CTA: Sr[D], Sw, Sww, Srr
   constexpr int RG = NWARP * RPI;         // row groups per CTA
   __shared__ double part[NWARP][NE];
-  __shared__ double tot[2][NE];
   __shared__ double piv[D + 1];
-  __shared__ int is_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // grid (S, Hq, 2 B): the deterministic-row CTAs of every head come first in dispatch order, so they take
@@ -117,16 +113,10 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 #ifdef VATTN_DEV_TIMING
   const int dv = 256 + 8192 + (b * p.Hq + blockIdx.y) * 8;
 #endif
-  HeadMeta& meta = p.meta[bh];
   const HeadMeta mt = ld_meta(p.meta + bh);
-  const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, n_s = mt.n_s, b0 = mt.b0;
+  const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, b0 = mt.b0;
   if (n == 0) {
     if (base_cta) pdl_wait();                      // every base-row CTA waits: "this grid done" implies "the one before done"
-    if (vx == 0 && tid == 0) {
-      meta.b = 0;
-      if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
-      if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
-    }
     return;
   }
   const int n_f = s0 + kk + (n - l_start);
@@ -164,13 +154,11 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
           ph_n[u] = r < s0 ? phys_of(p, b, r) : (r < s0 + kk ? __ldg(tkph + r - s0) : phys_of(p, b, l_start + (r - s0 - kk)));
       }
     };
-    fetch(0);
-    for (int k0 = 0; k0 < iters; k0 += UN) {
-      bool act[UN];
-      RowRegs<T> row[UN];
+    auto issue = [&](RowRegs<T> (&row)[UN], bool (&act)[UN]) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
-      fetch(k0 + UN);
+    };
+    auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
       double wv[UN];
       weights64<T, D>(p, qf, row, m, j, wv);                   // every lane takes part in the shuffles
 #pragma unroll
@@ -182,6 +170,20 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
           for (int e = 0; e < EPL; ++e) acc[e] = fma(w, (double)row[u].v.get(e), acc[e]);
         }
       }
+    };
+    RowRegs<T> rowA[UN], rowB[UN];
+    bool actA[UN], actB[UN];
+    fetch(0);
+    issue(rowA, actA);
+    fetch(UN);
+    for (int k0 = 0; k0 < iters; k0 += 2 * UN) {
+      issue(rowB, actB);
+      fetch(k0 + 2 * UN);
+      reduce(rowA, actA);
+      if (k0 + UN >= iters) break;                             // uniform over the CTA
+      issue(rowA, actA);
+      fetch(k0 + 3 * UN);
+      reduce(rowB, actB);
     }
   } else {
     pdl_wait();
@@ -203,25 +205,12 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
         ph_n[u] = act_n[u] ? __ldg(bsph + r) : piv_ph;
       }
     };
-    fetch(0);
-    load_row<T, D>(p, g, piv_ph, j, prow);
-    double cw = 0.0, cr[EPL];
-    for (int k0 = 0; k0 < max(iters, 1); k0 += UN) {
-      bool act[UN];
-      RowRegs<T> row[UN];
+    auto issue = [&](RowRegs<T> (&row)[UN], bool (&act)[UN]) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
-      fetch(k0 + UN);
-      if (k0 == 0) {
-        cw = weight64<T, D>(p, qf, prow, m);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) cr[e] = cw * (double)prow.v.get(e);
-        if (warp == 0 && rsub == 0) {
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cr[e];
-          if (j == 0) piv[D] = cw;
-        }
-      }
+    };
+    double cw = 0.0, cr[EPL];
+    auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
       double wv[UN];
       weights64<T, D>(p, qf, row, m, j, wv);
 #pragma unroll
@@ -239,6 +228,30 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
           }
         }
       }
+    };
+    RowRegs<T> rowA[UN], rowB[UN];
+    bool actA[UN], actB[UN];
+    fetch(0);
+    load_row<T, D>(p, g, piv_ph, j, prow);
+    issue(rowA, actA);
+    fetch(UN);
+    issue(rowB, actB);
+    fetch(2 * UN);
+    cw = weight64<T, D>(p, qf, prow, m);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) cr[e] = cw * (double)prow.v.get(e);
+    if (warp == 0 && rsub == 0) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cr[e];
+      if (j == 0) piv[D] = cw;
+    }
+    for (int k0 = 0; k0 < max(iters, 1); k0 += 2 * UN) {
+      if (k0 > 0) { issue(rowB, actB); fetch(k0 + 2 * UN); }
+      reduce(rowA, actA);
+      if (k0 + UN >= iters) break;                             // uniform over the CTA
+      issue(rowA, actA);
+      fetch(k0 + 3 * UN);
+      reduce(rowB, actB);
     }
   }
   DEV_MARK(p, 3, 3, bh == 0 && vx == 0);
@@ -270,107 +283,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   }
   if (base_cta && split == 0 && b0 > 0)              // the pivot travels with this CTA's partial
     for (int e = tid; e <= D; e += NT) p.stat_piv[(long long)bh * (D + 1) + e] = piv[e];
-  DEV_MARK(p, 3, 4, bh == 0 && vx == 0);
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.tickets[bh], 1u) == (unsigned)(2 * S - 1));
-  __syncthreads();
-  DEV_MARK(p, 3, 5, bh == 0 && vx == 0);
-  if (!is_last) { DEV_END(p, 3); return; }
-  __threadfence();
-  DEV_MARK(p, 3, 6, bh == 0);
-#ifdef VATTN_DEV_TIMING
-  DEV_AT(p, dv + 2);
-#endif
-
-  // ------------------------------------------------------------------ last CTA of this head
-  // every thread requests all partials of its element at once (one memory round trip), then adds them
-  // in split order; kind 0 = deterministic partials, kind 1 = base partials
-  for (int item = tid; item < 2 * NE; item += NT) {
-    const int kind = item / NE, e = item % NE;
-    const double* src = p.stat_part + ((long long)bh * 2 * MAXS + kind * S) * NE + e;
-    double v[MAXS];
-#pragma unroll
-    for (int sp = 0; sp < MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;
-    double s = 0.0;
-#pragma unroll
-    for (int sp = 0; sp < MAXS; ++sp) s += v[sp];
-    tot[kind][e] = s;
-  }
-  // the pivot the base CTAs used (all of them computed the same numbers; split 0 published them)
-  for (int e = tid; e <= D; e += NT) piv[e] = (b0 > 0) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
-  __syncthreads();
-  DEV_MARK(p, 3, 7, bh == 0);
-#ifdef VATTN_DEV_TIMING
-  DEV_AT(p, dv + 3);
-#endif
-  double* det = p.det_sums + (long long)bh * (D + 1);
-  for (int e = tid; e <= D; e += NT) det[e] = tot[0][e];
-  if (warp != 0) return;
-
-  const double Dfv = tot[0][D];
-  const double ratio = (b0 > 0) ? (double)n_s / (double)b0 : 0.0;
-  double nn = 0.0, sr2 = 0.0;                 // |N_hat|^2 and sum_j (sum_i r'_ij)^2
-  for (int e = lane; e < D; e += 32) {
-    const double srj = tot[1][e];
-    const double nh = tot[0][e] + ratio * (srj + (double)b0 * piv[e]);
-    nn = fma(nh, nh, nn);
-    sr2 = fma(srj, srj, sr2);
-  }
-#pragma unroll
-  for (int mask = 16; mask >= 1; mask >>= 1) {
-    nn += __shfl_xor_sync(0xFFFFFFFFu, nn, mask);
-    sr2 += __shfl_xor_sync(0xFFFFFFFFu, sr2, mask);
-  }
-  if (lane != 0) return;
-
-  const double Nnorm = sqrt(nn);
-  double sigma2 = 0.0, trace = 0.0, Dhat = Dfv;
-  int bD = 0, bN = 0, bS = 0, bfin = 0;
-  if (n_s > 0) {
-    const double Swv = tot[1][D], Swwv = tot[1][D + 1], Srrv = tot[1][D + 2];
-    if (b0 >= 2) {
-      sigma2 = fmax(0.0, (Swwv - Swv * Swv / (double)b0) / (double)(b0 - 1));
-      trace = fmax(0.0, (Srrv - sr2 / (double)b0) / (double)(b0 - 1));
-    }
-    Dhat = Dfv + ratio * (Swv + (double)b0 * piv[D]);
-    const double A = (double)n_s * sqrt(sigma2) / Dhat;
-    const double Bn = (double)n_s * sqrt(trace) / Nnorm;
-    double t = p.z_delta * A / p.eps;
-    const double b_D = t * t;
-    t = p.z_delta * Bn / p.eps;
-    const double b_N = t * t;
-    double mn = CUDART_INF;
-    bool nan = false;
-#pragma unroll
-    for (int jj = 0; jj < 15; ++jj) {
-      const double c = p.z1[jj] * A + p.z2[jj] * Bn;
-      const double c2 = c * c;
-      if (c2 != c2) nan = true;
-      mn = fmin(mn, c2);
-    }
-    const double b_S = nan ? CUDART_NAN : 4.0 / (p.eps * p.eps) * mn;
-    bD = ceil_sat(b_D); bN = ceil_sat(b_N); bS = ceil_sat(b_S);
-    const double bx = p.mode == 1 ? b_D : (p.mode == 2 ? b_N : b_S);
-    if (p.force_budget >= 0) bfin = min(p.force_budget, n_s);
-    else {
-      if (!isfinite(bx)) atomicOr(p.status, VATTN_STATUS_NONFINITE);
-      bfin = min(max(ceil_sat(bx), b0), n_s);
-    }
-  }
-  meta.b = bfin;
   DEV_END(p, 3);
-#ifdef VATTN_DEV_TIMING
-  if (p.devt) p.devt[dv + 4] = dev_gtime();
-#endif
-  if (p.dbg.budgets) {
-    int* o = p.dbg.budgets + bh * 4;
-    o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bfin;
-  }
-  if (p.dbg.stats) {
-    double* o = p.dbg.stats + bh * 8;
-    o[0] = Dfv; o[1] = sigma2; o[2] = trace; o[3] = Dhat; o[4] = Nnorm; o[5] = (double)n_s; o[6] = (double)b0; o[7] = m;
-  }
 }
 
 }  // namespace
