@@ -186,12 +186,15 @@ __device__ int finalize_emit(const Prob& p, int b, unsigned* sel, const unsigned
   for (int w = tid; w < nw; w += NT) {
     unsigned bits = sel[w];
     int pos = scan[w];
+    // the 32 tokens of a word lie in two pages: both ids are requested before the first is needed
+    const int pg_lo = (bits & 0xFFFFu) ? page_of(p, b, 2 * w) : 0;
+    const int pg_hi = (bits >> 16) ? page_of(p, b, 2 * w + 1) : 0;
     while (bits) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
       const int idx = w * 32 + bit;
       out_a[pos] = idx;
-      out_a[p.phys_delta + pos] = page_of(p, b, idx >> 4) * VATTN_BLOCK + (idx & 15);   // physical slot for the row kernels
+      out_a[p.phys_delta + pos] = (bit < 16 ? pg_lo : pg_hi) * VATTN_BLOCK + (idx & 15);   // physical slot for the row kernels
       if (out_b) out_b[pos] = idx;
       ++pos;
     }
