@@ -91,6 +91,9 @@ def test_workspace_and_argument_errors_without_gpu():
     assert L.vattn_set_params(h, C.byref(p)) == vb.OK
     assert L.vattn_set_params(h, None) == vb.OK
     assert L.vattn_strerror(vb.ERR_WORKSPACE).decode().startswith("workspace")
+    assert L.vattn_set_stop_after(h, -1) == vb.ERR_INVALID_ARG
+    assert L.vattn_set_stop_after(h, len(vb.KERNEL_NAMES) + 1) == vb.ERR_INVALID_ARG
+    assert L.vattn_set_stop_after(h, 1) == vb.OK and L.vattn_set_stop_after(h, 0) == vb.OK
     L.vattn_plan_destroy(h)
     L.vattn_plan_destroy(h2)
 

@@ -291,6 +291,49 @@ def test_many_topk_and_fp32_at_size():
     check(mid(dtype="fp32", d=64, seq_lens=[20000, 9000], B=2))
 
 
+def test_many_short_sequences_in_one_batch():
+    # 48 ragged rows, some of them empty: the score pass cuts them into many small work units that its CTAs
+    # take from a counter, and every list kernel meets heads without any work
+    rng = np.random.default_rng(77)
+    lens = [int(x) for x in rng.integers(0, 700, size=48)]
+    lens[3] = 0
+    lens[17] = 0
+    lens[47] = 1
+    check(small("bf16", lens, Hq=8, Hkv=2))
+
+
+def test_eps_delta_guarantee_holds_on_the_cuda_path():
+    # Definition 4.1 of the paper on the product path: over many seeds, the relative error of the sparse
+    # output against exact attention exceeds eps with frequency at most delta (plus binomial slack)
+    import math
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    eps = delta = 0.1
+    case = synth.make_case("guarantee", dtype="fp32", B=1, Hq=8, Hkv=2, d=64, seq_lens=[8192], sink=128, window=128,
+                           k=int(0.025 * 8192), eps=eps, delta=delta, seed=0, gen_seed=31337, key_std=0.1,
+                           rho_v=2.0, heavy=None, params=dict(base_rate=0.025))
+    ref = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=case.dtype)
+    dev = vb.case_to_device(case)
+    plan = vb.plan_for_case(case)
+    plan.set_params(**case.params)
+    dbg = plan.enable_debug()
+    out = torch.empty_like(dev["q"])
+    seeds, fails, trials, used = 128, 0, 0, []
+    for seed in range(seeds):
+        plan.decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], case.sink, case.window,
+                    case.k, case.eps, case.delta, seed, out)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy().astype(np.float64)
+        err = np.linalg.norm(got[0] - ref[0], axis=-1) / np.linalg.norm(ref[0], axis=-1)
+        fails += int((err > eps).sum())
+        trials += err.size
+        used.append(float(dbg["dyn_cnt"].cpu().numpy().mean()))
+    n_s = 8192 - 256 - case.k
+    assert np.mean(used) < 0.5 * n_s                       # not vacuous: budgets well below the residual
+    assert fails / trials <= delta + 3.0 * math.sqrt(delta * (1 - delta) / trials)
+    assert plan.last_status() == 0
+
+
 # ----------------------------------------------------------------------------- the five workloads
 def test_config1_tiny():
     case = synth.config1_tiny()
