@@ -102,6 +102,31 @@ __device__ int block_excl_scan(int* a, int nw, int* misc) {
   return total;
 }
 
+// Exclusive prefix sum over the CTA of one value per thread, with a single barrier: warp scans, the 32 warp
+// totals go through `wtot` (32 ints of shared memory that no thread touches between this call's barrier and
+// the next barrier of the caller), and every warp scans the totals itself.  `total` = sum over the CTA.
+__device__ __forceinline__ int block_scan_reg(int val, int* wtot, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = val;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += v;
+  }
+  if (lane == 31) wtot[warp] = incl;
+  __syncthreads();
+  const int mine = (lane < NWARP) ? wtot[lane] : 0;
+  int winc = mine;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, winc, off);
+    if (lane >= off) winc += v;
+  }
+  total = __shfl_sync(0xFFFFFFFFu, winc, 31);
+  const int before = __shfl_sync(0xFFFFFFFFu, winc - mine, warp);
+  return before + incl - val;
+}
+
 // Radix select of the c-th smallest key among the valid tokens of [lo, hi).  1 <= c <= #valid.
 // On return every thread knows T (the c-th smallest key) and need_eq (how many keys equal to T are
 // selected; all keys < T are).  keyfn(i, key) returns validity.
@@ -180,9 +205,17 @@ __device__ int finalize_emit(const Prob& p, int b, unsigned* sel, const unsigned
     for (int w = tid; w < nw; w += NT) sel[w] |= lowest_bits(eq[w], need_eq - scan[w]);
     __syncthreads();
   }
-  for (int w = tid; w < nw; w += NT) scan[w] = __popc(sel[w]);
-  __syncthreads();
-  const int total = block_excl_scan(scan, nw, misc);
+  int total;
+  if (nw <= NT) {                                     // one word per thread: prefix in registers, one barrier
+    __syncthreads();                                  // sel[] complete; the scratch below is free
+    const int mine = (tid < nw) ? __popc(sel[tid]) : 0;
+    const int excl = block_scan_reg(mine, misc + 8, total);
+    if (tid < nw) scan[tid] = excl;
+  } else {
+    for (int w = tid; w < nw; w += NT) scan[w] = __popc(sel[w]);
+    __syncthreads();
+    total = block_excl_scan(scan, nw, misc);
+  }
   for (int w = tid; w < nw; w += NT) {
     unsigned bits = sel[w];
     int pos = scan[w];
@@ -313,6 +346,8 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
   float* fmisc = reinterpret_cast<float*>(misc);
   float U = -INFINITY;              // candidates are the tokens with score >= U
   int ncand = 0;
+  float range2 = 0.f, inv_w2 = 0.f;  // linear bins of the candidates: bin = (m - score) * inv_w2
+  bool have_hist = false;           // the candidate pass has filled the bins already
   if (tid == 0) { misc[2] = NBIN; misc[4] = 0; misc[5] = 0; misc[6] = -1; }
   if (mlen <= CANDCAP) {
     for (int j = tid; j < mlen; j += NT) { sm.cand_idx[j] = s0 + j; sm.ckey[j] = sm.keys[s0 + j]; }
@@ -339,12 +374,12 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     }
     __syncthreads();
     const int cnt = sm.lin[tid];
-    __syncthreads();
-    block_excl_scan(sm.lin, NBIN, misc);
+    int tot1;
+    const int excl1 = block_scan_reg(cnt, reinterpret_cast<int*>(sm.hist), tot1);
     const double fms = (double)kk * (double)ms / (double)mlen;
     const int r = (int)(fms + 4.0 * sqrt(fms) + 8.0);
-    const int excl = sm.lin[tid];
-    if (excl < r && r <= excl + cnt) misc[2] = tid;
+    if (excl1 < r && r <= excl1 + cnt) misc[2] = tid;
+    sm.lin[tid] = 0;                                            // every thread has read its bin: reuse for pass two
     __syncthreads();
     const int jstar = misc[2];
     if (jstar >= NBIN - 1) return false;                      // the sample cannot place the threshold
@@ -352,7 +387,11 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     U = m - (float)(jstar + 1) * (range / (float)NBIN);
     if (U == 0.f) U = -0.f;                                   // both zeros must pass the key comparison
     const unsigned Ukey = ~ord_f32(U);                        // score >= U  <=>  key <= Ukey
-    // one pass over the context: 32 tokens per thread, take mask in a register
+    // One pass over the context: 32 tokens per thread, take mask in a register (no atomics in the loop);
+    // positions come from one scan; the candidates are written and counted in linear bins over [U, m].
+    range2 = m - U;
+    inv_w2 = (range2 > 0.f) ? (float)NBIN / range2 : 0.f;
+    have_hist = true;
     unsigned take = 0u;
     const int base_i = s0 + tid;
 #pragma unroll 8
@@ -360,50 +399,53 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
       const int i = base_i + it * NT;
       if (i < l_start && sm.keys[i] <= Ukey) take |= 1u << it;
     }
-    for (int it = 32; base_i + it * NT < l_start; ++it) {     // contexts longer than 32 * NT tokens
-      if (sm.keys[base_i + it * NT] <= Ukey) { misc[6] = -2; }
-    }
-    __syncthreads();
-    sm.lin[tid] = __popc(take);
-    __syncthreads();
-    ncand = block_excl_scan(sm.lin, NBIN, misc);
-    if (misc[6] == -2 || ncand < kk || ncand > CANDCAP) return false;
-    int pos = sm.lin[tid];
+    bool beyond = false;
+    for (int it = 32; base_i + it * NT < l_start; ++it)       // contexts longer than 32 * NT tokens
+      beyond = beyond || (sm.keys[base_i + it * NT] <= Ukey);
+    if (beyond) misc[6] = -2;
+    int pos = block_scan_reg(__popc(take), reinterpret_cast<int*>(sm.hist) + 64, ncand);
+    if (misc[6] == -2 || ncand < kk || ncand > CANDCAP) return false;     // (misc[6] was written before the barrier)
     while (take) {
       const int it = __ffs(take) - 1;
       take &= take - 1;
       const int i = base_i + it * NT;
+      const unsigned key = sm.keys[i];
       sm.cand_idx[pos] = i;
-      sm.ckey[pos] = sm.keys[i];
+      sm.ckey[pos] = key;
+      const float x = (m - unord_f32(~key)) * inv_w2;
+      atomicAdd(&sm.lin[x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0)], 1);
       ++pos;
     }
     __syncthreads();
   }
   DEV_MARK(p, 2, 11, blockIdx.x == 0 && blockIdx.y == 0);
-  // ---- the kk-th largest candidate: linear bins over [cmin, m], exact ranking inside the bin
-  float cmin = INFINITY;
-  for (int j = tid; j < ncand; j += NT) cmin = fminf(cmin, unord_f32(~sm.ckey[j]));
+  // ---- the kk-th largest candidate: linear bins over [cmin, m] (or [U, m]), exact ranking inside the bin
+  if (!have_hist) {
+    float cmin = INFINITY;
+    for (int j = tid; j < ncand; j += NT) cmin = fminf(cmin, unord_f32(~sm.ckey[j]));
 #pragma unroll
-  for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
-  sm.lin[tid] = 0;
-  if (lane == 0) fmisc[8 + warp] = cmin;
-  __syncthreads();
-  cmin = fmisc[8 + lane];
+    for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
+    sm.lin[tid] = 0;
+    if (lane == 0) fmisc[8 + warp] = cmin;
+    __syncthreads();
+    cmin = fmisc[8 + lane];
 #pragma unroll
-  for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
-  const float range2 = m - cmin;
-  const float inv_w2 = (range2 > 0.f) ? (float)NBIN / range2 : 0.f;
+    for (int mk = 16; mk >= 1; mk >>= 1) cmin = fminf(cmin, __shfl_xor_sync(0xFFFFFFFFu, cmin, mk));
+    range2 = m - cmin;
+    inv_w2 = (range2 > 0.f) ? (float)NBIN / range2 : 0.f;
+  }
   auto bin2 = [&](unsigned key) -> int {
     const float x = (m - unord_f32(~key)) * inv_w2;
     return x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0);
   };
-  for (int j = tid; j < ncand; j += NT) atomicAdd(&sm.lin[bin2(sm.ckey[j])], 1);
-  __syncthreads();
+  if (!have_hist) {
+    for (int j = tid; j < ncand; j += NT) atomicAdd(&sm.lin[bin2(sm.ckey[j])], 1);
+    __syncthreads();
+  }
   const int cnt2 = sm.lin[tid];
-  __syncthreads();
-  block_excl_scan(sm.lin, NBIN, misc);
   {
-    const int excl = sm.lin[tid];
+    int tot2;
+    const int excl = block_scan_reg(cnt2, reinterpret_cast<int*>(sm.hist) + 32, tot2);
     if (excl < kk && kk <= excl + cnt2) { misc[6] = tid; misc[7] = kk - excl; }
   }
   __syncthreads();
