@@ -185,25 +185,22 @@ def time_other_configs(vb, synth, torch, steps=40, pools=3):
         prof, calls = plan.read_profile()
         plan.set_profiling(False)
 
-        # the bandwidth kernel alone, launched back to back (16 launches per graph, pools rotating): its
-        # duration without the launch gap that the events inside a step include
+        # the score pass alone, launched back to back (no events in between)
         plan.set_stop_after(1)
-        B2B = 4 * POOLS
-        g_score = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_score, stream=stream):
-            for i in range(B2B):
-                step(i)
-        for _ in range(3):
-            g_score.replay()
-        stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(20):
-            g_score.replay()
-        e1.record(stream)
+        for i in range(3):
+            sparse(i)
         torch.cuda.synchronize()
-        us_score_b2b = e0.elapsed_time(e1) / (20 * B2B) * 1e3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            sparse(i)
+        e1.record()
+        torch.cuda.synchronize()
         plan.set_stop_after(0)
+        res["k_score_alone_us"] = round(e0.elapsed_time(e1) / steps * 1e3, 1)
+        res["k_score_alone_gbs"] = round((float(case.seq_lens.sum()) * case.num_kv_heads * case.head_dim *
+                                          (2 if case.dtype == "bf16" else 4) + float(case.seq_lens.sum()) *
+                                          case.num_q_heads * 4) / (res["k_score_alone_us"] * 1e-6) / 1e9, 1)
         res["kernels_us"] = {k_: round(v / max(calls, 1) * 1e3, 1) for k_, v in prof.items()}
         out[name] = res
         del devs, plan
