@@ -157,7 +157,15 @@ int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale, const void
 
 /* Same step as vattn_decode with HOST buffers for q, block_table, seq_lens and out (the caches stay on
  * the device): copies the inputs in, runs the step, copies `out` back and waits for it.  `staging` is a
- * caller-owned device buffer of at least vattn_host_staging_bytes(plan) bytes. */
+ * caller-owned device buffer of at least vattn_host_staging_bytes(plan) bytes.  Host buffers that are
+ * page-locked and mapped into the device's address space are read by one small kernel and `out` is
+ * written to the host buffer by the step itself (no copy-engine transfers, which cost several
+ * microseconds each at these sizes); any other host memory goes through cudaMemcpyAsync.
+ * A decode loop repeats this call with the same buffers: from the second call with one argument set on
+ * (all pointers, scalars and the stream equal; page-locked host buffers; `stream` not being captured by
+ * the caller; no debug buffers, profiling or stop-after in effect) the copies and kernels are recorded as
+ * one CUDA graph that later calls replay, which reads the host buffers' current contents.  The plan keeps
+ * the graphs of the 8 most recent argument sets (host objects; no device memory); every setter drops them. */
 size_t vattn_host_staging_bytes(const vattn_plan* plan);
 int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
                       const int32_t* block_table_host, const int32_t* seq_lens_host,

@@ -24,6 +24,21 @@ struct vattn_plan {
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
       off_det, off_piv, off_gat, off_dense, off_cand, off_sort, total;
   int cand_cap, gat_slots;
+  // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
+  struct HostStep {
+    bool used, pinned, mapped;
+    void *q_dev, *bt_dev, *sl_dev, *out_dev;   // device addresses of the host buffers when they are mapped
+    int hits, launches;
+    cudaGraphExec_t exec;
+    const void *q, *kc, *vc, *bt, *sl, *out, *staging, *stream;
+    int sink, window, k;
+    float eps, delta;
+    uint64_t seed;
+    unsigned long long gen;
+  } host_steps[8];
+  int host_next;
+  bool inputs_just_staged;     // set around the step of a host call whose inputs a kernel has just copied in
+  unsigned long long gen;      // bumped by every setter: steps captured under older settings are dropped
 };
 
 namespace {
@@ -171,7 +186,7 @@ int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st, bool with_ker
     CU(cudaMemsetAsync(p.status, 0, sizeof(unsigned), st));
     pl->status_ready = true;
   }
-  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, st));
+  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, st));
   else CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
   return VATTN_OK;
 }
@@ -214,6 +229,8 @@ int vattn_plan_create(const vattn_shape* shape, vattn_plan** out) {
 
 void vattn_plan_destroy(vattn_plan* plan) {
   if (!plan) return;
+  for (auto& e : plan->host_steps)
+    if (e.used && e.exec) cudaGraphExecDestroy(e.exec);
   if (plan->ev) {
     for (int i = 0; i < kProfCalls * kProfEvents; ++i) cudaEventDestroy(plan->ev[i]);
     delete[] plan->ev;
@@ -224,6 +241,7 @@ void vattn_plan_destroy(vattn_plan* plan) {
 int vattn_set_stop_after(vattn_plan* plan, int kernels) {
   if (!plan || kernels < 0 || kernels > VATTN_NUM_KERNELS) return VATTN_ERR_INVALID_ARG;
   plan->stop_after = kernels;
+  plan->gen++;
   return VATTN_OK;
 }
 
@@ -236,6 +254,7 @@ int vattn_set_profiling(vattn_plan* plan, int enable) {
       if (cudaEventCreate(&plan->ev[i]) != cudaSuccess) return VATTN_ERR_CUDA;
   }
   plan->profiling = enable != 0;
+  plan->gen++;
   plan->prof_calls = 0;
   return VATTN_OK;
 }
@@ -264,11 +283,13 @@ int vattn_set_workspace(vattn_plan* plan, void* dev_ptr, size_t bytes) {
   plan->ws = dev_ptr;
   plan->ws_bytes = bytes;
   plan->status_ready = false;
+  plan->gen++;
   return VATTN_OK;
 }
 
 int vattn_set_params(vattn_plan* plan, const vattn_params* params) {
   if (!plan) return VATTN_ERR_INVALID_ARG;
+  plan->gen++;
   if (!params) { memset(&plan->params, 0, sizeof(plan->params)); plan->params.force_budget = -1; return VATTN_OK; }
   const vattn_params& p = *params;
   if (p.base_rate < 0.f || p.base_rate > 1.f || p.topk_frac < 0.f || p.topk_frac > 1.f) return VATTN_ERR_INVALID_ARG;
@@ -280,6 +301,7 @@ int vattn_set_params(vattn_plan* plan, const vattn_params* params) {
 int vattn_set_debug(vattn_plan* plan, const vattn_debug* debug) {
   if (!plan) return VATTN_ERR_INVALID_ARG;
   if (debug) plan->dbg = *debug; else memset(&plan->dbg, 0, sizeof(plan->dbg));
+  plan->gen++;
   return VATTN_OK;
 }
 
@@ -373,11 +395,22 @@ size_t vattn_host_staging_bytes(const vattn_plan* plan) {
   return 2 * qb + align_up((size_t)s.batch * s.max_blocks_per_seq * 4, 256) + align_up((size_t)s.batch * 4, 256);
 }
 
-int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
-                      const int32_t* block_table_host, const int32_t* seq_lens_host, int sink, int window, int k,
-                      float eps, float delta, uint64_t seed, void* out_host, void* staging, void* stream) {
-  if (!plan || !q_host || !block_table_host || !seq_lens_host || !out_host || !staging || misaligned(staging, 256))
-    return VATTN_ERR_INVALID_ARG;
+// Host buffers that are page-locked and mapped are read and written by kernels directly: one small kernel
+// copies q, block_table and seq_lens into the staging buffer (three DMA copies of a few KB cost about 6 us
+// each; this costs one PCIe round trip), and the step writes `out` straight into the host buffer.
+__global__ void __launch_bounds__(256) k_stage_in(unsigned* dst0, const unsigned* src0, int n0, unsigned* dst1,
+                                                  const unsigned* src1, int n1, unsigned* dst2, const unsigned* src2, int n2) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x, nt = gridDim.x * blockDim.x;
+  for (int i = t; i < n0; i += nt) dst0[i] = src0[i];
+  for (int i = t; i < n1; i += nt) dst1[i] = src1[i];
+  for (int i = t; i < n2; i += nt) dst2[i] = src2[i];
+}
+
+// copies in, step, copy out: the stream work of one host step (no synchronisation)
+static int enqueue_host_step(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
+                             const int32_t* block_table_host, const int32_t* seq_lens_host, int sink, int window, int k,
+                             float eps, float delta, uint64_t seed, void* out_host, void* staging, cudaStream_t st,
+                             const vattn_plan::HostStep* mapped) {
   const vattn_shape& s = plan->shape;
   const size_t es = s.dtype == VATTN_DTYPE_BF16 ? 2 : 4;
   const size_t qbytes = (size_t)s.batch * s.num_q_heads * s.head_dim * es, qb = align_up(qbytes, 256);
@@ -385,14 +418,125 @@ int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache,
   unsigned char* d = static_cast<unsigned char*>(staging);
   void* dq = d; void* dout = d + qb; int32_t* dbt = reinterpret_cast<int32_t*>(d + 2 * qb);
   int32_t* dsl = reinterpret_cast<int32_t*>(d + 2 * qb + align_up(btbytes, 256));
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (mapped) {
+    const int words = (int)((qbytes + btbytes + slbytes) / 4);
+    int grid = (words + 255) / 256;                 // one word per thread: a single PCIe round trip
+    if (grid > 296) grid = 296;
+    if (grid < 1) grid = 1;
+    k_stage_in<<<grid, 256, 0, st>>>(static_cast<unsigned*>(dq), static_cast<const unsigned*>(mapped->q_dev), (int)(qbytes / 4),
+                                     reinterpret_cast<unsigned*>(dbt), static_cast<const unsigned*>(mapped->bt_dev),
+                                     (int)(btbytes / 4), reinterpret_cast<unsigned*>(dsl),
+                                     static_cast<const unsigned*>(mapped->sl_dev), (int)(slbytes / 4));
+    CU(cudaGetLastError());
+    plan->inputs_just_staged = true;
+    const int rc = vattn_decode(plan, dq, k_cache, v_cache, dbt, dsl, sink, window, k, eps, delta, seed, mapped->out_dev, st);
+    plan->inputs_just_staged = false;
+    if (rc == VATTN_OK) plan->last_launches++;
+    return rc;
+  }
   CU(cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, st));
   CU(cudaMemcpyAsync(dbt, block_table_host, btbytes, cudaMemcpyHostToDevice, st));
   CU(cudaMemcpyAsync(dsl, seq_lens_host, slbytes, cudaMemcpyHostToDevice, st));
-  int rc = vattn_decode(plan, dq, k_cache, v_cache, dbt, dsl, sink, window, k, eps, delta, seed, dout, stream);
+  int rc = vattn_decode(plan, dq, k_cache, v_cache, dbt, dsl, sink, window, k, eps, delta, seed, dout, st);
   if (rc != VATTN_OK) return rc;
   CU(cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, st));
-  CU(cudaStreamSynchronize(st));
+  return VATTN_OK;
+}
+
+static bool is_pinned_host(const void* ptr) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess) { cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost;
+}
+
+static void* mapped_device_pointer(const void* host) {
+  void* dev = nullptr;
+  if (cudaHostGetDevicePointer(&dev, const_cast<void*>(host), 0) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return dev;
+}
+
+int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table_host, const int32_t* seq_lens_host, int sink, int window, int k,
+                      float eps, float delta, uint64_t seed, void* out_host, void* staging, void* stream) {
+  if (!plan || !q_host || !block_table_host || !seq_lens_host || !out_host || !staging || misaligned(staging, 256))
+    return VATTN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // A caller that repeats a step with the same buffers (a decode loop) gets it as one CUDA graph from the
+  // third call on: the second call with an argument set records it, later ones replay it.  Only with
+  // page-locked host buffers, outside any capture of the caller, and with no introspection switched on.
+  vattn_plan::HostStep* e = nullptr;
+  const vattn_debug& dg = plan->dbg;
+  const bool plain_only = plan->profiling || plan->stop_after != 0 || plan->devt != nullptr || dg.topk_idx || dg.topk_cnt ||
+                          dg.base_idx || dg.base_cnt || dg.dyn_idx || dg.dyn_cnt || dg.budgets || dg.stats || dg.scores ||
+                          dg.paths;
+  if (!plain_only) {
+    for (auto& c : plan->host_steps)
+      if (c.used && c.gen == plan->gen && c.q == q_host && c.kc == k_cache && c.vc == v_cache && c.bt == block_table_host &&
+          c.sl == seq_lens_host && c.out == out_host && c.staging == staging && c.stream == stream && c.sink == sink &&
+          c.window == window && c.k == k && c.eps == eps && c.delta == delta && c.seed == seed) { e = &c; break; }
+    if (!e) {
+      e = &plan->host_steps[plan->host_next];
+      plan->host_next = (plan->host_next + 1) % 8;
+      if (e->used && e->exec) cudaGraphExecDestroy(e->exec);
+      *e = vattn_plan::HostStep{};
+      e->used = true; e->gen = plan->gen;
+      e->q = q_host; e->kc = k_cache; e->vc = v_cache; e->bt = block_table_host; e->sl = seq_lens_host; e->out = out_host;
+      e->staging = staging; e->stream = stream; e->sink = sink; e->window = window; e->k = k; e->eps = eps; e->delta = delta;
+      e->seed = seed;
+      e->pinned = is_pinned_host(q_host) && is_pinned_host(block_table_host) && is_pinned_host(seq_lens_host) &&
+                  is_pinned_host(out_host);
+      if (e->pinned) {
+        e->q_dev = mapped_device_pointer(q_host);
+        e->bt_dev = mapped_device_pointer(block_table_host);
+        e->sl_dev = mapped_device_pointer(seq_lens_host);
+        e->out_dev = mapped_device_pointer(out_host);
+        e->mapped = e->q_dev && e->bt_dev && e->sl_dev && e->out_dev && !misaligned(e->out_dev, 16) && !misaligned(e->q_dev, 4);
+      }
+    }
+    if (e->exec) {
+      CU(cudaGraphLaunch(e->exec, st));
+      CU(cudaStreamSynchronize(st));
+      plan->last_launches = e->launches;
+      return VATTN_OK;
+    }
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    const bool capturable_stream = st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread;   // not the default streams
+    if (e->pinned && e->hits >= 1 && capturable_stream && cudaStreamIsCapturing(st, &cs) == cudaSuccess &&
+        cs == cudaStreamCaptureStatusNone) {
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); e->pinned = false; goto plain; }
+      const int rc = enqueue_host_step(plan, q_host, k_cache, v_cache, block_table_host, seq_lens_host, sink, window, k, eps,
+                                       delta, seed, out_host, staging, st, e->mapped ? e : nullptr);
+      const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      if (rc != VATTN_OK || ce != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        e->pinned = false;                              // do not try again with this argument set
+        if (rc != VATTN_OK) return rc;
+      } else {
+        cudaGraphExec_t exec = nullptr;
+        const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ie == cudaSuccess) {
+          e->exec = exec;
+          e->launches = plan->last_launches;
+          CU(cudaGraphLaunch(e->exec, st));
+          CU(cudaStreamSynchronize(st));
+          return VATTN_OK;
+        }
+        cudaGetLastError();
+        e->pinned = false;
+      }
+    }
+  plain:
+    e->hits++;
+  }
+  {
+    const int rc = enqueue_host_step(plan, q_host, k_cache, v_cache, block_table_host, seq_lens_host, sink, window, k, eps,
+                                     delta, seed, out_host, staging, st, (e && e->mapped) ? e : nullptr);
+    if (rc != VATTN_OK) return rc;
+    CU(cudaStreamSynchronize(st));
+  }
   return VATTN_OK;
 }
 

@@ -42,9 +42,12 @@ struct __align__(16) StageMeta {   // written by the producer before it arms the
 // Clears the per-step counters (running maxima, tickets, list lengths, unit counter).  A kernel rather than a
 // memset node so that the score kernel behind it can start its prologue and its first copies meanwhile: it
 // lets its dependents go at once and waits for the previous step before it writes.
-__global__ void __launch_bounds__(256) k_zero(unsigned* z, int words) {
-  pdl_trigger();
+// (`late`: the grid before this one wrote the step's inputs, which the score kernel reads in its prologue, so
+// the dependents may only go once that grid has completed.)
+__global__ void __launch_bounds__(256) k_zero(unsigned* z, int words, int late) {
+  if (!late) pdl_trigger();
   pdl_wait();
+  if (late) pdl_trigger();
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += gridDim.x * blockDim.x) z[i] = 0u;
 }
 
@@ -414,12 +417,12 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   return launch_pdl(k_score_stream<D>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
 }
 
-cudaError_t launch_zero(unsigned* z, size_t bytes, cudaStream_t s) {
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, cudaStream_t s) {
   const int words = (int)(bytes / sizeof(unsigned));
   int grid = (words + 1023) / 1024;
   if (grid > 148) grid = 148;
   if (grid < 1) grid = 1;
-  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words);
+  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words, late ? 1 : 0);
 }
 
 cudaError_t launch_score(const Prob& p, cudaStream_t s) {

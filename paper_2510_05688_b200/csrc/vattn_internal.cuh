@@ -260,7 +260,7 @@ __device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
 }
 
 // launchers (one per translation unit)
-cudaError_t launch_zero(unsigned* z, size_t bytes, cudaStream_t s);
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, cudaStream_t s);
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
 cudaError_t launch_cand(const Prob& p, cudaStream_t s);
 cudaError_t launch_select_topk(const Prob& p, cudaStream_t s);

@@ -200,6 +200,21 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     plan.decode_host(qh, dev["k_cache"], dev["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
                      case.delta, case.seed, outh)
     assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), out_dev)
+    # a decode loop: the same buffers again and again (from the third call on the step replays as one CUDA
+    # graph), with new contents in the host buffers every time
+    rng = np.random.default_rng(5)
+    for it in range(5):
+        case.q = synth.f32_to_bf16_bits(rng.standard_normal(case.q.shape).astype(np.float32))
+        lens = np.array([900 - 7 * it, 350 - it], dtype=np.int32)
+        case.seq_lens = lens
+        qh.view(torch.int16).copy_(torch.from_numpy(case.q.view(np.int16)))
+        slh.copy_(torch.from_numpy(lens))
+        outh.zero_()
+        plan.decode_host(qh, dev["k_cache"], dev["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
+                         case.delta, case.seed, outh)
+        want, _, _ = run_gpu(case, debug=False)               # a plan of its own: setters would drop the graph
+        assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), want), f"host step {it}"
+    assert plan.last_status() == 0
 
 
 def test_seeded_random_shapes():
