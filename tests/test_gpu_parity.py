@@ -306,6 +306,18 @@ def test_many_topk_and_fp32_at_size():
     check(mid(dtype="fp32", d=64, seq_lens=[20000, 9000], B=2))
 
 
+def test_maximum_context_length():
+    # 262,144 tokens (the largest context a plan accepts), one head: top-k and the final sample run their
+    # full-context paths (keys from global memory, a stream-1 candidate list too long for shared memory), the
+    # score pass walks 16,384 pages
+    case = synth.make_case("max", dtype="bf16", B=1, Hq=1, Hkv=1, d=128, seq_lens=[262144], sink=128, window=128, k=3000,
+                           eps=0.1, delta=0.1, seed=11, gen_seed=909, rho_v=1.0,
+                           heavy=dict(R=128, c1=9.0, alpha=(0.75, 1.25)), params=dict(base_rate=0.01))
+    _, dbg, det, _ = check(case)
+    assert det[(0, 0)]["b"] < det[(0, 0)]["n_s"]
+    assert (dbg["paths"] & 5 == 0).all()
+
+
 def test_many_short_sequences_in_one_batch():
     # 48 ragged rows, some of them empty: the score pass cuts them into many small work units that its CTAs
     # take from a counter, and every list kernel meets heads without any work
