@@ -106,10 +106,6 @@ struct Gather {
       }
     }
     DEV_MARK(p, 5, 3, blockIdx.x == 0);
-    DEV_AT(p, 256 + blockIdx.x * 4 + 1);
-#ifdef VATTN_DEV_TIMING
-    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 8], dev_gtime());
-#endif
 #pragma unroll
     for (int mask = LPR; mask < 32; mask <<= 1) {
 #pragma unroll
@@ -135,9 +131,6 @@ struct Gather {
     if (tid == 0) *is_last = (atomicAdd(&p.tickets[p.B * p.Hq + bh], 1u) == (unsigned)(nslots - 1));
     __syncthreads();
     DEV_MARK(p, 5, 4, blockIdx.x == 0);
-#ifdef VATTN_DEV_TIMING
-    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 9], dev_gtime());
-#endif
     if (!*is_last) return;
     __threadfence();
 
@@ -175,9 +168,6 @@ struct Gather {
       if (lane == 0) *s_den = s;
     }
     __syncthreads();
-#ifdef VATTN_DEV_TIMING
-    if (p.devt && tid == 0) atomicMax(&p.devt[5 * 32 + 10], dev_gtime());
-#endif
     const double den = det_d + f * (double)(*s_den);
 #pragma unroll
     for (int it = 0; it < (D + NT - 1) / NT; ++it) {
@@ -248,7 +238,6 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __syncthreads();
   const int total = s_pref[BH];
   DEV_MARK(p, 5, 2, blockIdx.x == 0);
-  DEV_AT(p, 256 + blockIdx.x * 4);
   for (int c = blockIdx.x; c < total; c += gridDim.x) {
     int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
     while (lo < hi) {

@@ -110,9 +110,6 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   // What k_select_topk wrote (meta, I_t) is complete before this grid can start: the grid before this one
   // lets its dependents go only after its own wait on k_select_topk.  Only the base-row CTAs need the
   // grid before this one itself (I_bs), and they wait for it as late as possible.
-#ifdef VATTN_DEV_TIMING
-  const int dv = 256 + 8192 + (b * p.Hq + blockIdx.y) * 8;
-#endif
   const HeadMeta mt = ld_meta(p.meta + bh);
   const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, b0 = mt.b0;
   if (n == 0) {
@@ -187,9 +184,6 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     }
   } else {
     pdl_wait();
-#ifdef VATTN_DEV_TIMING
-    if (split == 0) DEV_AT(p, dv + 0);
-#endif
   }
   if (base_cta && b0 > 0) {
     // ---------------------------------------------------------------- base-sample rows, shifted by the pivot
@@ -255,9 +249,6 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     }
   }
   DEV_MARK(p, 3, 3, bh == 0 && vx == 0);
-#ifdef VATTN_DEV_TIMING
-  if (split == 0) DEV_AT(p, dv + (base_cta ? 1 : 5));
-#endif
   // across the row groups of the warp
 #pragma unroll
   for (int mask = LPR; mask < 32; mask <<= 1) {

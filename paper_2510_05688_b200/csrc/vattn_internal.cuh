@@ -75,12 +75,10 @@ __device__ __forceinline__ unsigned long long dev_gtime() { unsigned long long t
 #define DEV_BEGIN(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMin(&(p).devt[(k) * 32 + 0], dev_gtime()); } while (0)
 #define DEV_END(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMax(&(p).devt[(k) * 32 + 1], dev_gtime()); } while (0)
 #define DEV_MARK(p, k, slot, cond) do { if ((p).devt && threadIdx.x == 0 && (cond)) (p).devt[(k) * 32 + (slot)] = dev_gtime(); } while (0)
-#define DEV_AT(p, index) do { if ((p).devt && threadIdx.x == 0) (p).devt[(index)] = dev_gtime(); } while (0)
 #else
 #define DEV_BEGIN(p, k) do { } while (0)
 #define DEV_END(p, k) do { } while (0)
 #define DEV_MARK(p, k, slot, cond) do { } while (0)
-#define DEV_AT(p, index) do { } while (0)
 #endif
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
