@@ -339,6 +339,24 @@ def main():
         clocks = sampler.summary(t0, t1)
         ms_dense, _, _ = timed(dense_graphs, min(args.steps, 2000), args.warmup)
 
+        # spread of the step time: 200 replays timed one by one (each pair of events adds a little)
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(200)]
+        for i, (a, b_) in enumerate(pairs):
+            a.record(stream)
+            sparse_graphs[i % POOLS].replay()
+            b_.record(stream)
+        torch.cuda.synchronize()
+        each = np.array([a.elapsed_time(b_) * 1e3 for a, b_ in pairs])
+        step_pct = {"p10": round(float(np.percentile(each, 10)), 2), "p50": round(float(np.percentile(each, 50)), 2),
+                    "p90": round(float(np.percentile(each, 90)), 2), "n": len(pairs)}
+
+        # the K+V gather variant (weights recomputed from the K rows of the sampled tokens)
+        plan.set_params(**dict(case.params, gather_mode=1))
+        kv_graphs = capture(False)
+        ms_kv, _, _ = timed(kv_graphs, min(args.steps, 500), args.warmup)
+        plan.set_params(**case.params)
+        del kv_graphs
+
         # optional external context: a third-party dense paged-decode kernel on the same cache
         fi_us = None
         if args.flashinfer:
@@ -484,7 +502,8 @@ def main():
         "config": {"workload": WORKLOAD, "l2": f"rotating {POOLS} distinct cache pools (134 MB of K+V each, "
                    "more than the 126 MB L2 together with the previous pool)", "launch": "CUDA graph replay per step",
                    "mean_density": round(density, 4), "sparsity_x": round(1.0 / density, 2),
-                   "mean_budget": float(b_dyn.mean()), "status_bits": status,
+                   "mean_budget": float(b_dyn.mean()), "status_bits": status, "step_us_percentiles": step_pct,
+                   "kv_gather_variant_us_per_step": round(ms_kv * 1e3, 2),
                    "value_is": "max-over-ranks step time / n_gpus (each rank runs its own layer)"},
         "e2e": {"value": ms_e2e_max * 1e3 / world, "unit": UNIT,
                 "h2d_bytes_per_step": int(qh.numel() * 2 + bth.numel() * 4 + slh.numel() * 4),

@@ -70,6 +70,10 @@ typedef struct {
   int32_t rng_head_is_kv;  /* 0: sampling keys per query head; 1: per KV head (the heads of a group share keys) */
   int32_t force_budget;    /* < 0 (or 0 with force_budget_on == 0): off; else b = min(force_budget, n_s) */
   int32_t force_budget_on; /* set to 1 to apply force_budget (so that a forced budget of 0 is expressible) */
+  int32_t gather_mode;     /* 0: the sampled tokens' weights exp(s_i - m) come from the scores of the score pass and
+                              only their V rows are read (default); 1: K and V rows are read and the scores are
+                              recomputed from the K rows in fp32: the traffic of a pipeline whose selector leaves
+                              no scores behind (the paper's composition with an approximate top-k, Sec. 4) */
 } vattn_params;
 
 /* Optional per-call introspection.  All DEVICE pointers; NULL = not wanted.  cap = max_seq_len. */

@@ -34,7 +34,7 @@ class Shape(C.Structure):
 class Params(C.Structure):
     _fields_ = [("base_rate", C.c_float), ("topk_frac", C.c_float), ("scale", C.c_float), ("mode", C.c_int32),
                 ("layer", C.c_int32), ("step", C.c_int32), ("rng_head_is_kv", C.c_int32),
-                ("force_budget", C.c_int32), ("force_budget_on", C.c_int32)]
+                ("force_budget", C.c_int32), ("force_budget_on", C.c_int32), ("gather_mode", C.c_int32)]
 
 
 class Debug(C.Structure):

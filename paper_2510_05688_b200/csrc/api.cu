@@ -134,6 +134,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.base_rate = pr.base_rate > 0.f ? pr.base_rate : 0.025f;
   p.scale = pr.scale != 0.f ? pr.scale : (float)(1.0 / sqrt((double)s.head_dim));
   p.mode = pr.mode; p.layer = pr.layer; p.step = pr.step; p.rng_head_is_kv = pr.rng_head_is_kv;
+  p.gather_kv = pr.gather_mode == 1;
   p.force_budget = (pr.force_budget_on || pr.force_budget > 0) ? (pr.force_budget < 0 ? -1 : pr.force_budget) : -1;
   unsigned char* w = static_cast<unsigned char*>(pl->ws);
   p.scores = reinterpret_cast<float*>(w + pl->off_scores);
@@ -294,6 +295,7 @@ int vattn_set_params(vattn_plan* plan, const vattn_params* params) {
   const vattn_params& p = *params;
   if (p.base_rate < 0.f || p.base_rate > 1.f || p.topk_frac < 0.f || p.topk_frac > 1.f) return VATTN_ERR_INVALID_ARG;
   if (p.mode < 0 || p.mode > 2 || p.step < 0 || !(p.scale == p.scale) || isinf(p.scale)) return VATTN_ERR_INVALID_ARG;
+  if (p.gather_mode < 0 || p.gather_mode > 1) return VATTN_ERR_INVALID_ARG;
   plan->params = p;
   return VATTN_OK;
 }

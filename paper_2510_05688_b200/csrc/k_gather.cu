@@ -28,7 +28,7 @@ constexpr int FLAT_MAXS = VATTN_GATHER_FLAT_SLOTS;   // ... flat decomposition
 constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
 constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
 
-template <typename T, int D>
+template <typename T, int D, bool KV>
 struct Gather {
   static constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR, NE = D + 1, RG = NWARP * RPI;
 
@@ -78,23 +78,53 @@ struct Gather {
         ph_n[u] = ok ? __ldg(dph + r) : 0;
       }
     };
+    // K+V variant: the score of a sampled token is recomputed from its K row (what a selector that leaves no
+    // scores for the whole context behind would need); the K slices of a batch come first, then its V slices
+    float qf[EPL];
+    const T* kcg = reinterpret_cast<const T*>(p.kc) + (long long)g * p.sh;
+    if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
     fetch_idx(0);
     for (int k0 = 0; k0 < iters; k0 += UNROLL) {
       int tok[UNROLL];
       float w[UNROLL];
       uint4 raw[UNROLL];
+      if (KV) {
+        long long off[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        tok[u] = tok_n[u];
-        raw[u] = make_uint4(0u, 0u, 0u, 0u);
-        w[u] = 0.f;
-        if (tok[u] >= 0) {
+        for (int u = 0; u < UNROLL; ++u) {
+          tok[u] = tok_n[u];
           const int ph = ph_n[u];
-          raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
-          w[u] = __ldg(sc + tok[u]);
+          off[u] = (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL;
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(kcg + off[u]);
         }
+        if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          float kv[EPL], dot = 0.f;
+          unpack(raw[u], kv);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kv[e], dot);
+#pragma unroll
+          for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
+          w[u] = p.scale * dot;
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(vc + off[u]);
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          tok[u] = tok_n[u];
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          w[u] = 0.f;
+          if (tok[u] >= 0) {
+            const int ph = ph_n[u];
+            raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
+            w[u] = __ldg(sc + tok[u]);
+          }
+        }
+        if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);   // next batch's indices travel with this batch's rows
       }
-      if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);   // next batch's indices travel with this batch's rows
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
         const float ww = (tok[u] >= 0) ? expf(w[u] - m) : 0.f;
@@ -177,9 +207,9 @@ struct Gather {
   }
 };
 
-template <typename T, int D>
+template <typename T, int D, bool KV>
 __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
-  using G = Gather<T, D>;
+  using G = Gather<T, D, KV>;
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
@@ -198,9 +228,9 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   DEV_END(p, 5);
 }
 
-template <typename T, int D>
+template <typename T, int D, bool KV>
 __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
-  using G = Gather<T, D>;
+  using G = Gather<T, D, KV>;
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
@@ -254,30 +284,25 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
 
 }  // namespace
 
-cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
+template <typename T, int D, bool KV>
+static cudaError_t launch_gather_t(const Prob& p, cudaStream_t s) {
   const int BH = p.B * p.Hq;
   if (BH <= FLAT_MAX_HEADS) {
     // at most FLAT_MAXS chunks per head; 8 CTAs per SM walk them with a grid stride
     if (p.gat_slots < FLAT_MAXS) return cudaErrorInvalidValue;
     const long long most = (long long)BH * FLAT_MAXS;
     const int grid = (int)(most < 8 * 148 ? most : 8 * 148);
-    if (p.dtype == VATTN_DTYPE_BF16) {
-      if (p.D == 128) return launch_pdl(k_gather_flat<bf16_t, 128>, dim3(grid), dim3(NT), 0, s, p);
-      else return launch_pdl(k_gather_flat<bf16_t, 64>, dim3(grid), dim3(NT), 0, s, p);
-    } else {
-      if (p.D == 128) return launch_pdl(k_gather_flat<float, 128>, dim3(grid), dim3(NT), 0, s, p);
-      else return launch_pdl(k_gather_flat<float, 64>, dim3(grid), dim3(NT), 0, s, p);
-    }
-    return cudaGetLastError();
+    return launch_pdl(k_gather_flat<T, D, KV>, dim3(grid), dim3(NT), 0, s, p);
   }
   if (p.gat_slots < MAXS) return cudaErrorInvalidValue;
-  dim3 grid(MAXS, p.Hq, p.B), block(NT);
+  return launch_pdl(k_gather<T, D, KV>, dim3(MAXS, p.Hq, p.B), dim3(NT), 0, s, p);
+}
+
+cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
   if (p.dtype == VATTN_DTYPE_BF16) {
-    if (p.D == 128) return launch_pdl(k_gather<bf16_t, 128>, grid, block, 0, s, p);
-    else return launch_pdl(k_gather<bf16_t, 64>, grid, block, 0, s, p);
-  } else {
-    if (p.D == 128) return launch_pdl(k_gather<float, 128>, grid, block, 0, s, p);
-    else return launch_pdl(k_gather<float, 64>, grid, block, 0, s, p);
+    if (p.D == 128) return p.gather_kv ? launch_gather_t<bf16_t, 128, true>(p, s) : launch_gather_t<bf16_t, 128, false>(p, s);
+    return p.gather_kv ? launch_gather_t<bf16_t, 64, true>(p, s) : launch_gather_t<bf16_t, 64, false>(p, s);
   }
-  return cudaGetLastError();
+  if (p.D == 128) return p.gather_kv ? launch_gather_t<float, 128, true>(p, s) : launch_gather_t<float, 128, false>(p, s);
+  return p.gather_kv ? launch_gather_t<float, 64, true>(p, s) : launch_gather_t<float, 64, false>(p, s);
 }

@@ -36,6 +36,7 @@ struct Prob {
   int sink, window, k;
   float topk_frac, base_rate, scale;
   int mode, layer, step, rng_head_is_kv, force_budget;       // force_budget < 0: off
+  int gather_kv;          // 1: the gather kernel recomputes the weights of the sampled tokens from their K rows
   unsigned seed_lo, seed_hi;
   double eps, delta, z_delta;
   double z1[15], z2[15];                                     // z(delta*j/16), z(delta*(16-j)/16), j = 1..15

@@ -10,6 +10,7 @@ FP32_REL = 1e-5      # relative to the head's largest |output|, fp32 outputs
 def run_oracle(case, heads=None, **over):
     p = dict(case.params)
     p.update(over)
+    p.pop("gather_mode", None)          # where the weights are read from is not part of what is computed
     return O.vattn_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink,
                           case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype, heads=heads, **p)
 

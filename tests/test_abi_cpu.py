@@ -87,7 +87,9 @@ def test_workspace_and_argument_errors_without_gpu():
     assert L.vattn_set_params(h, C.byref(p)) == vb.ERR_INVALID_ARG
     p.base_rate, p.mode = 0.05, 3
     assert L.vattn_set_params(h, C.byref(p)) == vb.ERR_INVALID_ARG
-    p.mode = 1
+    p.mode, p.gather_mode = 1, 2
+    assert L.vattn_set_params(h, C.byref(p)) == vb.ERR_INVALID_ARG
+    p.gather_mode = 1
     assert L.vattn_set_params(h, C.byref(p)) == vb.OK
     assert L.vattn_set_params(h, None) == vb.OK
     assert L.vattn_strerror(vb.ERR_WORKSPACE).decode().startswith("workspace")

@@ -318,6 +318,15 @@ def test_maximum_context_length():
     assert (dbg["paths"] & 5 == 0).all()
 
 
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("fp32", 64), ("fp32", 128)])
+def test_gather_that_recomputes_the_weights_from_k_rows(dtype, d):
+    check(small(dtype, [1, 17, 600, 2049], d=d), gather_mode=1)
+
+
+def test_gather_from_k_rows_at_size():
+    check(mid(), gather_mode=1)
+
+
 def test_many_short_sequences_in_one_batch():
     # 48 ragged rows, some of them empty: the score pass cuts them into many small work units that its CTAs
     # take from a counter, and every list kernel meets heads without any work
