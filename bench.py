@@ -450,7 +450,8 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- algorithmic bytes per launch (what each kernel must move)
+    # ---- algorithmic bytes per launch: what each kernel must move (K rows and score words for the score pass,
+    # 8-byte candidate pairs for the sampling kernels, K and V rows for the statistics, V rows for the gather)
     es, d, Hq, Hkv = 2, case.head_dim, case.num_q_heads, case.num_kv_heads
     n_tot = int(case.seq_lens.sum())
     n_f = kks.sum() + Hq * (min(case.sink, n_tot) + min(case.window, n_tot))

@@ -23,7 +23,7 @@ known-answer vectors, the (eps, delta) definition over 1,000 seeds).  The *exact
 for a given seed* have no counterpart in the paper (it prints no worked example and fixes no
 random generator): for those values parity is unpinned beyond the pins above.
 
-Readings taken where the paper is silent (listed with reasons in the design doc):
+Readings taken where the paper is silent:
   * softmax scale is a parameter (default 1/sqrt(d)); exp is stabilised by the global max m,
     which cancels in N/D and in both budget ratios;
   * sink/window are absolute token counts, top-k is taken over the middle range only, ties go
