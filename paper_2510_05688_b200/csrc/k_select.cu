@@ -338,8 +338,8 @@ __device__ int sample_select(const Prob& p, const Sm& sm, int lo, int hi, int nw
 // On success the bitmap of I_t is in sm.w0.  Returns false (sm.w0 / sm.w1 undefined) when the generic
 // path has to run.
 template <typename T, int D>
-__device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qrow, int s0, int l_start, int kk,
-                          int nw, float m, float gamma) {
+__device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qrow, const float* sc,
+                          unsigned long long* kbar, int& landed, int s0, int l_start, int kk, int nw, float m, float gamma) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int mlen = l_start - s0;
   int* misc = sm.misc;
@@ -349,15 +349,21 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
   float range2 = 0.f, inv_w2 = 0.f;  // linear bins of the candidates: bin = (m - score) * inv_w2
   bool have_hist = false;           // the candidate pass has filled the bins already
   if (tid == 0) { misc[2] = NBIN; misc[4] = 0; misc[5] = 0; misc[6] = -1; }
+  const float* sf = reinterpret_cast<const float*>(sm.keys);   // raw scores, valid once the bulk copy has landed
   if (mlen <= CANDCAP) {
-    for (int j = tid; j < mlen; j += NT) { sm.cand_idx[j] = s0 + j; sm.ckey[j] = sm.keys[s0 + j]; }
+    landed = __syncthreads_and(mbar_wait(kbar, 0u)) ? 1 : -1;
+    if (landed < 0) return false;
+    for (int j = tid; j < mlen; j += NT) { sm.cand_idx[j] = s0 + j; sm.ckey[j] = ~ord_f32(sf[s0 + j]); }
     ncand = mlen;
     __syncthreads();
   } else {
     constexpr int SAMPLE = 2048;
     const int stride = (mlen + SAMPLE - 1) / SAMPLE;
     const int ms = (mlen + stride - 1) / stride;
-    float smin = (tid < ms) ? unord_f32(~sm.keys[s0 + tid * stride]) : INFINITY;
+    float smp[2];                                               // this thread's sample scores (ms <= 2048 = 2 NT)
+    smp[0] = (tid < ms) ? __ldcg(sc + s0 + tid * stride) : INFINITY;
+    smp[1] = (tid + NT < ms) ? __ldcg(sc + s0 + (tid + NT) * stride) : INFINITY;
+    float smin = fminf(smp[0], smp[1]);
 #pragma unroll
     for (int mk = 16; mk >= 1; mk >>= 1) smin = fminf(smin, __shfl_xor_sync(0xFFFFFFFFu, smin, mk));
     sm.lin[tid] = 0;
@@ -368,9 +374,12 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     for (int mk = 16; mk >= 1; mk >>= 1) smin = fminf(smin, __shfl_xor_sync(0xFFFFFFFFu, smin, mk));
     const float range = m - smin;
     const float inv_w = (range > 0.f) ? (float)NBIN / range : 0.f;
-    for (int j = tid; j < ms; j += NT) {
-      const float x = (m - unord_f32(~sm.keys[s0 + j * stride])) * inv_w;
-      atomicAdd(&sm.lin[x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0)], 1);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (tid + u * NT < ms) {
+        const float x = (m - smp[u]) * inv_w;
+        atomicAdd(&sm.lin[x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0)], 1);
+      }
     }
     __syncthreads();
     const int cnt = sm.lin[tid];
@@ -380,13 +389,12 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     const int r = (int)(fms + 4.0 * sqrt(fms) + 8.0);
     if (excl1 < r && r <= excl1 + cnt) misc[2] = tid;
     sm.lin[tid] = 0;                                            // every thread has read its bin: reuse for pass two
-    __syncthreads();
+    landed = __syncthreads_and(mbar_wait(kbar, 0u)) ? 1 : -1;  // the scores have had the estimate's time to arrive
+    if (landed < 0) return false;
     const int jstar = misc[2];
     if (jstar >= NBIN - 1) return false;                      // the sample cannot place the threshold
     DEV_MARK(p, 2, 10, blockIdx.x == 0 && blockIdx.y == 0);
     U = m - (float)(jstar + 1) * (range / (float)NBIN);
-    if (U == 0.f) U = -0.f;                                   // both zeros must pass the key comparison
-    const unsigned Ukey = ~ord_f32(U);                        // score >= U  <=>  key <= Ukey
     // One pass over the context: 32 tokens per thread, take mask in a register (no atomics in the loop);
     // positions come from one scan; the candidates are written and counted in linear bins over [U, m].
     range2 = m - U;
@@ -397,11 +405,11 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
 #pragma unroll 8
     for (int it = 0; it < 32; ++it) {
       const int i = base_i + it * NT;
-      if (i < l_start && sm.keys[i] <= Ukey) take |= 1u << it;
+      if (i < l_start && sf[i] >= U) take |= 1u << it;
     }
     bool beyond = false;
     for (int it = 32; base_i + it * NT < l_start; ++it)       // contexts longer than 32 * NT tokens
-      beyond = beyond || (sm.keys[base_i + it * NT] <= Ukey);
+      beyond = beyond || (sf[base_i + it * NT] >= U);
     if (beyond) misc[6] = -2;
     int pos = block_scan_reg(__popc(take), reinterpret_cast<int*>(sm.hist) + 64, ncand);
     if (misc[6] == -2 || ncand < kk || ncand > CANDCAP) return false;     // (misc[6] was written before the barrier)
@@ -409,10 +417,10 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
       const int it = __ffs(take) - 1;
       take &= take - 1;
       const int i = base_i + it * NT;
-      const unsigned key = sm.keys[i];
+      const float sv = sf[i];
       sm.cand_idx[pos] = i;
-      sm.ckey[pos] = key;
-      const float x = (m - unord_f32(~key)) * inv_w2;
+      sm.ckey[pos] = ~ord_f32(sv);
+      const float x = (m - sv) * inv_w2;
       atomicAdd(&sm.lin[x >= (float)(NBIN - 1) ? NBIN - 1 : (x > 0.f ? (int)x : 0)], 1);
       ++pos;
     }
@@ -608,6 +616,7 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
   DEV_BEGIN(p, 2);
+  __shared__ unsigned long long kbar;         // completion of the bulk copy of the scores
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
 
@@ -640,15 +649,17 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
     const double gm = roundings * 5.9604644775390625e-8 * fabs((double)p.scale) * sa * kmax * 1.000001;
     if (lane == 0) reinterpret_cast<float*>(sm.misc)[48] = __double2float_ru(gm);
   }
-  if (CACHED && kk > 0 && kk < mlen) {
-    // order-reversed score keys of the middle range: 16-byte loads over the aligned body
-    const int a0 = min(l_start, (s0 + 3) & ~3), a1 = max(a0, l_start & ~3);
-    for (int i = s0 + tid; i < a0; i += NT) sm.keys[i] = ~ord_f32(__ldcg(sc + i));
-    for (int i = a1 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(__ldcg(sc + i));
-    for (int i = a0 + 4 * tid; i < a1; i += 4 * NT) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(sc + i));
-      *reinterpret_cast<uint4*>(sm.keys + i) = make_uint4(~ord_f32(v.x), ~ord_f32(v.y), ~ord_f32(v.z), ~ord_f32(v.w));
-    }
+  const bool staged = CACHED && kk > 0 && kk < mlen;
+  if (staged && tid == 0) {
+    // the scores of the middle range travel to shared memory as one asynchronous bulk copy (raw fp32, the
+    // 16-byte aligned span around [s0, l_start)); the threshold estimate below runs meanwhile on a sample
+    // it reads from global memory
+    const int a0 = s0 & ~3, a1 = (l_start + 3) & ~3;             // within the padded row: npad is a multiple of 32
+    mbar_init(&kbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_expect_tx(&kbar, (unsigned)(a1 - a0) * 4u);
+    bulk_g2s(sm.keys + a0, sc + a0, (unsigned)(a1 - a0) * 4u, &kbar);
   }
   __syncthreads();
   const float gamma = reinterpret_cast<float*>(sm.misc)[48];
@@ -677,9 +688,20 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
     bool done = false;
     if (CACHED) {
       DEV_MARK(p, 2, 3, bh == 0);
-      done = topk_fast<T, D>(p, sm, b, g, qrow, s0, l_start, kk, nw, m, gamma);
+      int landed = 0;                                  // 1: the scores are in shared memory, -1: the copy never arrived
+      done = topk_fast<T, D>(p, sm, b, g, qrow, sc, &kbar, landed, s0, l_start, kk, nw, m, gamma);
       DEV_MARK(p, 2, 4, bh == 0);
       if (done) path |= 1;
+      if (!done) {
+        // the generic select wants order-reversed integer keys: wait for the copy if nobody has yet, convert
+        if (landed == 0) landed = __syncthreads_and(mbar_wait(&kbar, 0u)) ? 1 : -1;
+        if (landed < 0) {                              // give up on this head: report, leave I_t empty
+          if (tid == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+          mbar_wait(&kbar, 0u);                        // a second bounded chance before the buffer is released
+        } else {
+          for (int i = s0 + tid; i < l_start; i += NT) sm.keys[i] = ~ord_f32(__uint_as_float(sm.keys[i]));
+        }
+      }
     }
     if (!done) {
       __syncthreads();
