@@ -89,6 +89,11 @@ typedef struct {
   int32_t *paths;                 /* [B,Hq] which code path selected each set: bit 0 top-k from the sampled threshold
                                      estimate, bit 1 base sample from the pre-filtered list, bit 2 final sample =
                                      prefix of the pre-sorted list (a clear bit = the full-context select ran) */
+  unsigned long long *kernel_ticks; /* [VATTN_NUM_KERNELS + 1][2] device-side time stamps in ns (%globaltimer) of the
+                                     counter-clearing kernel (row 0) and the kernels of a step in the order listed
+                                     for vattn_set_profiling: [k][0] = earliest CTA start, [k][1] = latest end.
+                                     Folded with atomic min / max: set [k][0] = UINT64_MAX and [k][1] = 0 before the
+                                     step to be observed.  Unlike event profiling this leaves the step as it is */
 } vattn_debug;
 
 /* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG, UNSUPPORTED. */

@@ -40,7 +40,8 @@ class Params(C.Structure):
 class Debug(C.Structure):
     _fields_ = [("topk_idx", C.c_void_p), ("topk_cnt", C.c_void_p), ("base_idx", C.c_void_p),
                 ("base_cnt", C.c_void_p), ("dyn_idx", C.c_void_p), ("dyn_cnt", C.c_void_p),
-                ("budgets", C.c_void_p), ("stats", C.c_void_p), ("scores", C.c_void_p), ("paths", C.c_void_p)]
+                ("budgets", C.c_void_p), ("stats", C.c_void_p), ("scores", C.c_void_p), ("paths", C.c_void_p),
+                ("kernel_ticks", C.c_void_p)]
 
 
 _lib = None
@@ -177,6 +178,20 @@ class Plan:
     def disable_debug(self):
         _check(lib().vattn_set_debug(self._h, None), "vattn_set_debug")
         self.debug = None
+
+    def enable_kernel_ticks(self):
+        """Register only the device-side time-stamp buffer ([kernels + 1, 2] int64; row 0 = the clearing kernel).
+        Call reset_kernel_ticks() before the step to observe, read the tensor after it."""
+        import torch
+        self.ticks = torch.zeros(len(KERNEL_NAMES) + 1, 2, dtype=torch.int64, device=self.device)
+        d = Debug(kernel_ticks=self.ticks.data_ptr())
+        _check(lib().vattn_set_debug(self._h, C.byref(d)), "vattn_set_debug")
+        self.reset_kernel_ticks()
+        return self.ticks
+
+    def reset_kernel_ticks(self):
+        self.ticks[:, 0] = -1          # all ones: the largest unsigned value, for the atomic minimum
+        self.ticks[:, 1] = 0
 
     def decode(self, q, k_cache, v_cache, block_table, seq_lens, sink, window, k, eps, delta, seed, out, stream=None):
         _check(lib().vattn_decode(self._h, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),

@@ -13,7 +13,6 @@ struct vattn_plan {
   size_t ws_bytes;
   bool status_ready;
   int last_launches;
-  unsigned long long* devt;
   // optional per-kernel timing (events are created on first use; no device memory involved)
   bool profiling;
   int stop_after;           // measurement aid: enqueue only the first stop_after kernels of a step (0 = all)
@@ -162,7 +161,6 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.stat_splits = pl->stat_splits; p.dense_splits = pl->dense_splits;
   p.dbg = pl->dbg;
-  p.devt = pl->devt;
   return VATTN_OK;
 }
 
@@ -187,7 +185,7 @@ int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st, bool with_ker
     CU(cudaMemsetAsync(p.status, 0, sizeof(unsigned), st));
     pl->status_ready = true;
   }
-  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, st));
+  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, p.dbg.kernel_ticks, st));
   else CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
   return VATTN_OK;
 }
@@ -468,7 +466,7 @@ int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache,
   // page-locked host buffers, outside any capture of the caller, and with no introspection switched on.
   vattn_plan::HostStep* e = nullptr;
   const vattn_debug& dg = plan->dbg;
-  const bool plain_only = plan->profiling || plan->stop_after != 0 || plan->devt != nullptr || dg.topk_idx || dg.topk_cnt ||
+  const bool plain_only = plan->profiling || plan->stop_after != 0 || dg.kernel_ticks || dg.topk_idx || dg.topk_cnt ||
                           dg.base_idx || dg.base_cnt || dg.dyn_idx || dg.dyn_cnt || dg.budgets || dg.stats || dg.scores ||
                           dg.paths;
   if (!plain_only) {
@@ -553,10 +551,6 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits) {
   CU(cudaStreamSynchronize(st));
   return VATTN_OK;
 }
-
-#ifdef VATTN_DEV_TIMING
-int vattn_dev_set_timing_buffer(vattn_plan* plan, void* ptr) { plan->devt = static_cast<unsigned long long*>(ptr); return 0; }
-#endif
 
 int vattn_last_launch_count(const vattn_plan* plan) { return plan ? plan->last_launches : 0; }
 

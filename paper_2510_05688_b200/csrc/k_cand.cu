@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(CT, 4) k_cand(const Prob p) {
   __shared__ uint2 lst[2][CCAP];
   __shared__ unsigned cnt[2], gbase[2];
   pdl_trigger();
-  DEV_BEGIN(p, 6);
+  TICK_BEGIN(p, VATTN_K_CAND);
   const int tid = threadIdx.x, lane = tid & 31;
   const int b = blockIdx.z, h = blockIdx.y, tile0 = blockIdx.x * CTILE;
   const int bh = b * p.Hq + h;
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(CT, 4) k_cand(const Prob p) {
   }
   // This grid does not wait for the score kernel before it, so one of its CTAs does at the end: "this grid
   // has completed" then implies "the score kernel has completed" for the kernels behind it.
-  DEV_END(p, 6);
+  TICK_END(p, VATTN_K_CAND);
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) pdl_wait();
 }
 

@@ -135,7 +135,6 @@ struct Gather {
         for (int e = 0; e < EPL; ++e) acc[e] = fmaf(ww, v[e], acc[e]);
       }
     }
-    DEV_MARK(p, 5, 3, blockIdx.x == 0);
 #pragma unroll
     for (int mask = LPR; mask < 32; mask <<= 1) {
 #pragma unroll
@@ -160,7 +159,6 @@ struct Gather {
     __syncthreads();
     if (tid == 0) *is_last = (atomicAdd(&p.tickets[p.B * p.Hq + bh], 1u) == (unsigned)(nslots - 1));
     __syncthreads();
-    DEV_MARK(p, 5, 4, blockIdx.x == 0);
     if (!*is_last) return;
     __threadfence();
 
@@ -213,7 +211,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
-  DEV_BEGIN(p, 5);
+  TICK_BEGIN(p, VATTN_K_GATHER);
   pdl_wait();
   const int bh = blockIdx.z * p.Hq + blockIdx.y;
   const HeadMeta meta = p.meta[bh];
@@ -225,7 +223,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   if ((int)blockIdx.x >= nslots) return;
   const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
   G::run(p, bh, meta, r_begin, r_end, blockIdx.x, nslots, part, &is_last, &s_den);
-  DEV_END(p, 5);
+  TICK_END(p, VATTN_K_GATHER);
 }
 
 template <typename T, int D, bool KV>
@@ -236,7 +234,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __shared__ float s_den;
   __shared__ int s_pref[FLAT_MAX_HEADS + 1], s_rows[FLAT_MAX_HEADS], s_b[FLAT_MAX_HEADS], s_w[NWARP];
   __shared__ HeadMeta s_meta[FLAT_MAX_HEADS];
-  DEV_BEGIN(p, 5);
+  TICK_BEGIN(p, VATTN_K_GATHER);
   pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int BH = p.B * p.Hq;
@@ -267,7 +265,6 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   if (tid == NT - 1) s_pref[BH] = before + incl;      // BH <= NT: the last thread's inclusive sum is the total
   __syncthreads();
   const int total = s_pref[BH];
-  DEV_MARK(p, 5, 2, blockIdx.x == 0);
   for (int c = blockIdx.x; c < total; c += gridDim.x) {
     int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
     while (lo < hi) {
@@ -279,7 +276,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
     G::run(p, bh, s_meta[bh], r_begin, r_end, ci, s_pref[bh + 1] - s_pref[bh], part, &is_last, &s_den);
     __syncthreads();
   }
-  DEV_END(p, 5);
+  TICK_END(p, VATTN_K_GATHER);
 }
 
 }  // namespace

@@ -44,11 +44,13 @@ struct __align__(16) StageMeta {   // written by the producer before it arms the
 // lets its dependents go at once and waits for the previous step before it writes.
 // (`late`: the grid before this one wrote the step's inputs, which the score kernel reads in its prologue, so
 // the dependents may only go once that grid has completed.)
-__global__ void __launch_bounds__(256) k_zero(unsigned* z, int words, int late) {
+__global__ void __launch_bounds__(256) k_zero(unsigned* z, int words, int late, unsigned long long* ticks) {
+  if (ticks && threadIdx.x == 0) atomicMin(ticks + 2 * VATTN_K_ZERO, gtime_ns());
   if (!late) pdl_trigger();
   pdl_wait();
   if (late) pdl_trigger();
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += gridDim.x * blockDim.x) z[i] = 0u;
+  if (ticks && threadIdx.x == 0) atomicMax(ticks + 2 * VATTN_K_ZERO + 1, gtime_ns());
 }
 
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
@@ -71,7 +73,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
   int* s_pref = s_len + p.B;                         // [B+1] units before batch row b
   int* s_misc = s_pref + p.B + 1;                    // [16]
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
-  DEV_BEGIN(p, 1);
+  TICK_BEGIN(p, VATTN_K_SCORE);
 
   // ---- units: every CTA derives the same decomposition from the sequence lengths
   const int GC = (p.G + 7) >> 3;
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
       // (a stage that was never armed simply runs into the wait limit)
       for (long long j = (i > S ? i - S : 0) + lane; j < i; j += 32) mbar_wait(&full[j % S], (unsigned)(j / S) & 1u);
     }
-    DEV_END(p, 1);
+    TICK_END_IF(p, VATTN_K_SCORE, lane == 0);
     return;
   }
 
@@ -290,6 +292,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     }
   }
   flush();
+  TICK_END(p, VATTN_K_SCORE);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -417,12 +420,12 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   return launch_pdl(k_score_stream<D>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
 }
 
-cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, cudaStream_t s) {
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, unsigned long long* ticks, cudaStream_t s) {
   const int words = (int)(bytes / sizeof(unsigned));
   int grid = (words + 1023) / 1024;
   if (grid > 148) grid = 148;
   if (grid < 1) grid = 1;
-  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words, late ? 1 : 0);
+  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words, late ? 1 : 0, ticks);
 }
 
 cudaError_t launch_score(const Prob& p, cudaStream_t s) {

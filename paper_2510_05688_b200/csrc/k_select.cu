@@ -393,7 +393,6 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     if (landed < 0) return false;
     const int jstar = misc[2];
     if (jstar >= NBIN - 1) return false;                      // the sample cannot place the threshold
-    DEV_MARK(p, 2, 10, blockIdx.x == 0 && blockIdx.y == 0);
     U = m - (float)(jstar + 1) * (range / (float)NBIN);
     // One pass over the context: 32 tokens per thread, take mask in a register (no atomics in the loop);
     // positions come from one scan; the candidates are written and counted in linear bins over [U, m].
@@ -426,7 +425,6 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
     }
     __syncthreads();
   }
-  DEV_MARK(p, 2, 11, blockIdx.x == 0 && blockIdx.y == 0);
   // ---- the kk-th largest candidate: linear bins over [cmin, m] (or [U, m]), exact ranking inside the bin
   if (!have_hist) {
     float cmin = INFINITY;
@@ -480,7 +478,6 @@ __device__ bool topk_fast(const Prob& p, const Sm& sm, int b, int g, const T* qr
   }
   __syncthreads();
   const unsigned Tk = (unsigned)misc[3];
-  DEV_MARK(p, 2, 12, blockIdx.x == 0 && blockIdx.y == 0);
   const float Tf = unord_f32(~Tk);
   const float hi = __fadd_ru(Tf, 2.f * gamma), lo = __fadd_rd(Tf, -2.f * gamma);
   // every token that could still enter the top-k (score >= lo) must be a candidate
@@ -615,7 +612,7 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
-  DEV_BEGIN(p, 2);
+  TICK_BEGIN(p, VATTN_K_TOPK);
   __shared__ unsigned long long kbar;         // completion of the bulk copy of the scores
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
   HeadMeta& meta = p.meta[bh];
@@ -671,7 +668,6 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   }
   unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
   if (n == 0) { if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = 0; return; }
-  DEV_MARK(p, 2, 2, bh == 0);
 
   int path = 0;
   // ------------------------------------------------------------------ top-k over the middle range
@@ -687,10 +683,8 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
   } else if (kk > 0) {
     bool done = false;
     if (CACHED) {
-      DEV_MARK(p, 2, 3, bh == 0);
       int landed = 0;                                  // 1: the scores are in shared memory, -1: the copy never arrived
       done = topk_fast<T, D>(p, sm, b, g, qrow, sc, &kbar, landed, s0, l_start, kk, nw, m, gamma);
-      DEV_MARK(p, 2, 4, bh == 0);
       if (done) path |= 1;
       if (!done) {
         // the generic select wants order-reversed integer keys: wait for the copy if nobody has yet, convert
@@ -720,10 +714,9 @@ __global__ void __launch_bounds__(NT, 1) k_select_topk(const Prob p, int bigbyte
     gbitmap[w] = v;
   }
   __syncthreads();
-  DEV_MARK(p, 2, 5, bh == 0);
 
   if (p.dbg.paths && tid == 0) p.dbg.paths[bh] = path;
-  DEV_END(p, 2);
+  TICK_END(p, VATTN_K_TOPK);
 }
 
 // Sampling without a selection on the critical path (Algorithm 2 line 1 and Algorithm 1 line 7).
@@ -747,9 +740,7 @@ __global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, in
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, stream = blockIdx.z, g = h / p.G;
   const int bh = b * p.Hq + h;
-  const int devk = stream ? 7 : 0;
-  (void)devk;
-  DEV_BEGIN(p, devk);
+  TICK_BEGIN(p, VATTN_K_PRESORT);
   uint2* pairs = reinterpret_cast<uint2*>(smem_raw);          // [paircap] bucketed (key, token), later sorted (token, slot)
   int* srt = reinterpret_cast<int*>(pairs + paircap);         // [paircap] tokens in sorted order
   int* off = srt + paircap;                                   // [SORT_BUCKETS + 1] bucket starts
@@ -825,10 +816,8 @@ __global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, in
       }
     }
   }
-  DEV_MARK(p, devk, 2, bh == 0);
   pdl_wait();                         // the bitmap of I_t and meta come from k_select_topk
   pdl_trigger();
-  DEV_MARK(p, devk, 3, bh == 0);
   HeadMeta& meta = p.meta[bh];
   if (n == 0 || geo.n_s <= 0) { if (stream == 1 && tid == 0) meta.sorted_cnt = 0; return; }
   if (stream == 0 && geo.b0 <= 0) return;
@@ -887,7 +876,7 @@ __global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, in
         if (stream == 1) meta.sorted_cnt = total;
         else if (p.dbg.paths) atomicOr(&p.dbg.paths[bh], 2);
       }
-      DEV_END(p, devk);
+      TICK_END(p, VATTN_K_PRESORT);
       return;
     }
   }
@@ -901,7 +890,7 @@ __global__ void __launch_bounds__(NT, 1) k_presort(const Prob p, int paircap, in
   int* bs_out = p.base_idx + (long long)bh * p.npad;
   int* bs_dbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
   sample_select<CACHED>(p, sm, geo.s0, geo.l_start, nw, geo.b0, geo.n_s, b, hrng, 0, sm.w2, bs_out, bs_dbg);
-  DEV_END(p, devk);
+  TICK_END(p, VATTN_K_PRESORT);
 }
 
 // Budget (Algorithm 2, Theorem 4.3 / Corollaries D.2) and the slow path of the final sample.
@@ -927,7 +916,7 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x, b = blockIdx.y, g = h / p.G;
   const int bh = b * p.Hq + h;
-  DEV_BEGIN(p, 4);
+  TICK_BEGIN(p, VATTN_K_BUDGET);
   pdl_trigger();
   pdl_wait();
   HeadMeta meta = p.meta[bh];
@@ -1033,7 +1022,6 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   }
   __syncthreads();
   meta.b = s_b;
-  DEV_MARK(p, 4, 2, bh == 0);
   if (meta.b <= 0) return;
   // ---- final sample
   if (meta.b < meta.n_s && meta.sorted_cnt >= meta.b) {
@@ -1054,7 +1042,7 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   int* out = p.dyn_idx + (long long)bh * p.npad;
   int* dbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)bh * p.max_seq_len : nullptr;
   sample_select<CACHED>(p, sm, meta.s0, meta.l_start, nw, meta.b, meta.n_s, b, hrng, 1, sm.w2, out, dbg);
-  DEV_END(p, 4);
+  TICK_END(p, VATTN_K_BUDGET);
 }
 
 }  // namespace

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const int S = p.stat_splits;
   const int split = blockIdx.x;
   const int vx = (base_cta ? S : 0) + split;       // position among the head's 2 S partials
-  DEV_BEGIN(p, 3);
+  TICK_BEGIN(p, VATTN_K_STATS);
   pdl_trigger();
   // What k_select_topk wrote (meta, I_t) is complete before this grid can start: the grid before this one
   // lets its dependents go only after its own wait on k_select_topk.  Only the base-row CTAs need the
@@ -130,7 +130,6 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 
   float qf[EPL];
   Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
-  DEV_MARK(p, 3, 2, bh == 0 && vx == 0);
 
   double acc[EPL], s1 = 0.0, s2 = 0.0, s3 = 0.0;           // det: N_f slice, D_f;  base: Sr slice, Sw, Sww, Srr
 #pragma unroll
@@ -248,7 +247,6 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
       reduce(rowB, actB);
     }
   }
-  DEV_MARK(p, 3, 3, bh == 0 && vx == 0);
   // across the row groups of the warp
 #pragma unroll
   for (int mask = LPR; mask < 32; mask <<= 1) {
@@ -274,7 +272,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   }
   if (base_cta && split == 0 && b0 > 0)              // the pivot travels with this CTA's partial
     for (int e = tid; e <= D; e += NT) p.stat_piv[(long long)bh * (D + 1) + e] = piv[e];
-  DEV_END(p, 3);
+  TICK_END(p, VATTN_K_STATS);
 }
 
 }  // namespace

@@ -66,21 +66,24 @@ struct Prob {
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, dense_splits;
   vattn_debug dbg;
-  unsigned long long* devt;   // development timing buffer [8][32] (null unless a dev build sets it)
 };
 
-// Development-only phase timing (compiled in with -DVATTN_DEV_TIMING): slot 0/1 of a kernel's row hold
-// the earliest CTA start / latest CTA end, further slots are set by one chosen CTA.
-#ifdef VATTN_DEV_TIMING
-__device__ __forceinline__ unsigned long long dev_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define DEV_BEGIN(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMin(&(p).devt[(k) * 32 + 0], dev_gtime()); } while (0)
-#define DEV_END(p, k) do { if ((p).devt && threadIdx.x == 0) atomicMax(&(p).devt[(k) * 32 + 1], dev_gtime()); } while (0)
-#define DEV_MARK(p, k, slot, cond) do { if ((p).devt && threadIdx.x == 0 && (cond)) (p).devt[(k) * 32 + (slot)] = dev_gtime(); } while (0)
-#else
-#define DEV_BEGIN(p, k) do { } while (0)
-#define DEV_END(p, k) do { } while (0)
-#define DEV_MARK(p, k, slot, cond) do { } while (0)
-#endif
+// Optional device-side kernel time stamps (vattn_debug.kernel_ticks): thread 0 of every CTA folds
+// %globaltimer into [k][0] = earliest start and [k][1] = latest end of kernel k.  Unlike events between the
+// kernels this does not serialise the step: it shows the overlapped timeline of a real (graph-replayed) step.
+__device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TICK_BEGIN(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMin((p).dbg.kernel_ticks + 2 * (k), gtime_ns()); } while (0)
+#define TICK_END(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
+#define TICK_END_IF(p, k, cond) do { if ((p).dbg.kernel_ticks && (cond)) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
+// kernel numbers
+#define VATTN_K_ZERO 0
+#define VATTN_K_SCORE 1
+#define VATTN_K_CAND 2
+#define VATTN_K_TOPK 3
+#define VATTN_K_PRESORT 4
+#define VATTN_K_STATS 5
+#define VATTN_K_BUDGET 6
+#define VATTN_K_GATHER 7
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
 // stream is still running; it must call pdl_wait() before touching anything the predecessor writes (the
@@ -259,7 +262,7 @@ __device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
 }
 
 // launchers (one per translation unit)
-cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, cudaStream_t s);
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, unsigned long long* ticks, cudaStream_t s);
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
 cudaError_t launch_cand(const Prob& p, cudaStream_t s);
 cudaError_t launch_select_topk(const Prob& p, cudaStream_t s);
