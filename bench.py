@@ -365,7 +365,7 @@ def main():
         tl = np.median(np.stack(tl), axis=0)
         plan.disable_debug()
         del tl_graphs
-        timeline = {name: [round(float(tl[k_, 0]), 2), round(float(tl[k_, 1]), 2)]
+        timeline = {name: [round(float(tl[k_, 0]), 2), round(float(tl[k_, 1]), 2) if tl[k_, 1] > 0 else None]
                     for k_, name in enumerate(["k_zero"] + vb.KERNEL_NAMES)}
 
         # the K+V gather variant (weights recomputed from the K rows of the sampled tokens)

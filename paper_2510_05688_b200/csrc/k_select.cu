@@ -1022,7 +1022,7 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   }
   __syncthreads();
   meta.b = s_b;
-  if (meta.b <= 0) return;
+  if (meta.b <= 0) { TICK_END(p, VATTN_K_BUDGET); return; }
   // ---- final sample
   if (meta.b < meta.n_s && meta.sorted_cnt >= meta.b) {
     if (p.dbg.dyn_idx) {
@@ -1031,6 +1031,7 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
       for (int i = tid; i < meta.b; i += NT) dbg[i] = src[i];
     }
     if (p.dbg.paths && tid == 0) atomicOr(&p.dbg.paths[bh], 4);
+    TICK_END(p, VATTN_K_BUDGET);
     return;
   }
   const Sm sm = carve(smem_raw, bigbytes, p.nwords);
