@@ -96,7 +96,9 @@ typedef struct {
                                      step to be observed.  Unlike event profiling this leaves the step as it is */
 } vattn_debug;
 
-/* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG, UNSUPPORTED. */
+/* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG,
+ * UNSUPPORTED (head_dim other than 64 / 128, block_size other than 16, more than 64 query heads per KV head,
+ * max_seq_len above 262,144, a bf16 batch above 1,536 rows). */
 int    vattn_plan_create(const vattn_shape* shape, vattn_plan** out);
 void   vattn_plan_destroy(vattn_plan* plan);
 

@@ -404,7 +404,7 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   const int qslot_bytes = nh_max * D * 2;
   const size_t smem = (size_t)S * PAGEB + (size_t)S * qslot_bytes + (size_t)S * sizeof(StageMeta) + (size_t)2 * S * 8 +
                       sizeof(int) * ((size_t)2 * p.B + 1 + 16);
-  if (smem > 110 * 1024) return cudaErrorInvalidValue;        // batch too large for the in-kernel unit table
+  if (smem > 113 * 1024) return cudaErrorInvalidValue;        // two CTAs per SM (plan creation bounds the batch)
   static size_t attr_sz = 0;
   if (attr_sz < smem) {
     cudaError_t e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -188,6 +188,7 @@ __device__ __forceinline__ Geo head_geometry(const Prob& p, int n) {
 // is below this bound.  Stream 1 keeps a quarter of the tokens; stream 0 keeps b0 + 6 sqrt(b0) + 16
 // expected tokens (none if that is more than a quarter: the select kernel then draws without the list).
 #define VATTN_CAND1_BOUND 0x40000000u
+#define VATTN_MAX_BATCH_BF16 1536     // batch rows a bf16 plan accepts (12 bytes of shared memory per row in k_score)
 #define VATTN_STAT_MAXS 16            // most split CTAs per head and row kind of the statistics kernel
 #define VATTN_GATHER_FLAT_HEADS 128   // the gather kernel's flat decomposition serves up to this many heads ...
 #define VATTN_GATHER_FLAT_SLOTS 128   // ... with up to this many chunks (partials) each

@@ -54,6 +54,13 @@ def test_plan_create_validates_shape():
     assert create(dtype=5)[0] == vb.ERR_UNSUPPORTED
     assert create(max_seq_len=129)[0] == vb.ERR_INVALID_ARG        # exceeds max_blocks_per_seq * 16
     assert create(max_seq_len=1 << 20, max_blocks_per_seq=1 << 16)[0] == vb.ERR_UNSUPPORTED
+    assert create(batch=1537)[0] == vb.ERR_UNSUPPORTED             # bf16: per-row tables of the score kernel
+    rc, h = create(batch=1536)
+    assert rc == vb.OK
+    vb.lib().vattn_plan_destroy(h)
+    rc, h = create(batch=4000, dtype=vb.DTYPE_FP32)
+    assert rc == vb.OK
+    vb.lib().vattn_plan_destroy(h)
     assert vb.lib().vattn_plan_create(None, None) == vb.ERR_INVALID_ARG
 
 
