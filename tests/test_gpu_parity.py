@@ -327,6 +327,13 @@ def test_gather_from_k_rows_at_size():
     check(mid(), gather_mode=1)
 
 
+def test_largest_bf16_batch():
+    # 1,536 rows (the most a bf16 plan accepts): the score kernel's per-row tables fill its shared memory
+    rng = np.random.default_rng(78)
+    lens = [int(x) for x in rng.integers(0, 72, size=1536)]
+    check(small("bf16", lens, Hq=2, Hkv=1))
+
+
 def test_many_short_sequences_in_one_batch():
     # 48 ragged rows, some of them empty: the score pass cuts them into many small work units that its CTAs
     # take from a counter, and every list kernel meets heads without any work
