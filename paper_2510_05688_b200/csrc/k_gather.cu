@@ -31,6 +31,7 @@ constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposit
 template <typename T, int D, bool KV>
 struct Gather {
   static constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR, NE = D + 1, RG = NWARP * RPI;
+  static_assert(LPR >= UNROLL, "each row of a batch needs a lane of its row group to own its weight");
 
   static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[EPL]) {
     if (EPL == 8) {
@@ -85,8 +86,9 @@ struct Gather {
     if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
     fetch_idx(0);
     for (int k0 = 0; k0 < iters; k0 += UNROLL) {
-      int tok[UNROLL];
-      float w[UNROLL];
+      // lane u of a row group owns row u's weight: one score load and one exp per row instead of LPR
+      int tok[UNROLL], tok_mine = -1;
+      float w_mine = 0.f;
       uint4 raw[UNROLL];
       if (KV) {
         long long off[UNROLL];
@@ -107,7 +109,7 @@ struct Gather {
           for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kv[e], dot);
 #pragma unroll
           for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
-          w[u] = p.scale * dot;
+          if (j == u) { w_mine = p.scale * dot; tok_mine = tok[u]; }
           raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(vc + off[u]);
         }
@@ -116,18 +118,19 @@ struct Gather {
         for (int u = 0; u < UNROLL; ++u) {
           tok[u] = tok_n[u];
           raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          w[u] = 0.f;
+          if (j == u) tok_mine = tok[u];
           if (tok[u] >= 0) {
             const int ph = ph_n[u];
             raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
-            w[u] = __ldg(sc + tok[u]);
           }
         }
+        if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);
         if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);   // next batch's indices travel with this batch's rows
       }
+      const float e_mine = (tok_mine >= 0) ? expf(w_mine - m) : 0.f;
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
-        const float ww = (tok[u] >= 0) ? expf(w[u] - m) : 0.f;
+        const float ww = __shfl_sync(0xFFFFFFFFu, e_mine, u, LPR);
         dd += ww;
         float v[EPL];
         unpack(raw[u], v);
