@@ -134,8 +134,8 @@ class Plan:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h is not None and h.value:
-            lib().vattn_plan_destroy(h)
+        if h is not None and h.value and _lib is not None:      # module globals are gone at interpreter exit
+            _lib.vattn_plan_destroy(h)
             self._h = None
 
     # -- direct ABI calls
