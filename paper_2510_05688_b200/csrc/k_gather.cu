@@ -17,6 +17,7 @@
 //  * per head (larger problems): grid (32, heads, batch); a head with budget b uses ceil(b / chunk) of its
 //    32 CTAs, chunk = max(256, ceil(b / 32)) rows, the others exit at once.
 #include "vattn_internal.cuh"
+#include <type_traits>
 
 namespace {
 
@@ -69,23 +70,32 @@ struct Gather {
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
 
+    // A batch = UNROLL rows per row group.  Batches whose rows all exist (every one but a chunk's last) run a
+    // body without per-row validity tests; FULL is a compile-time tag.
+    const int full_iters = ((r_end - r_begin) / (RG * UNROLL)) * UNROLL;
     int tok_n[UNROLL], ph_n[UNROLL];
-    auto fetch_idx = [&](int k0) {
+    auto fetch_idx = [&](int k0, auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        const bool ok = (k0 + u < iters) && (r < r_end);
+        const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
         tok_n[u] = ok ? __ldg(dyn + r) : -1;
         ph_n[u] = ok ? __ldg(dph + r) : 0;
       }
+    };
+    auto fetch_next = [&](int k0) {                   // indices of the batch that starts at iteration k0, if any
+      if (k0 >= iters) return;
+      if (k0 + UNROLL <= full_iters) fetch_idx(k0, std::true_type{});
+      else fetch_idx(k0, std::false_type{});
     };
     // K+V variant: the score of a sampled token is recomputed from its K row (what a selector that leaves no
     // scores for the whole context behind would need); the K slices of a batch come first, then its V slices
     float qf[EPL];
     const T* kcg = reinterpret_cast<const T*>(p.kc) + (long long)g * p.sh;
     if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
-    fetch_idx(0);
-    for (int k0 = 0; k0 < iters; k0 += UNROLL) {
+    auto batch = [&](int k0, auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
       // lane u of a row group owns row u's weight: one score load and one exp per row instead of LPR
       int tok[UNROLL], tok_mine = -1;
       float w_mine = 0.f;
@@ -97,10 +107,10 @@ struct Gather {
           tok[u] = tok_n[u];
           const int ph = ph_n[u];
           off[u] = (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL;
-          raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(kcg + off[u]);
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (FULL || tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(kcg + off[u]);
         }
-        if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);
+        fetch_next(k0 + UNROLL);
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           float kv[EPL], dot = 0.f;
@@ -110,22 +120,22 @@ struct Gather {
 #pragma unroll
           for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
           if (j == u) { w_mine = p.scale * dot; tok_mine = tok[u]; }
-          raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(vc + off[u]);
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (FULL || tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(vc + off[u]);
         }
       } else {
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           tok[u] = tok_n[u];
-          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (j == u) tok_mine = tok[u];
-          if (tok[u] >= 0) {
+          if (FULL || tok[u] >= 0) {
             const int ph = ph_n[u];
             raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
           }
         }
         if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);
-        if (k0 + UNROLL < iters) fetch_idx(k0 + UNROLL);   // next batch's indices travel with this batch's rows
+        fetch_next(k0 + UNROLL);                        // next batch's indices travel with this batch's rows
       }
       const float e_mine = (tok_mine >= 0) ? expf(w_mine - m) : 0.f;
 #pragma unroll
@@ -137,6 +147,11 @@ struct Gather {
 #pragma unroll
         for (int e = 0; e < EPL; ++e) acc[e] = fmaf(ww, v[e], acc[e]);
       }
+    };
+    fetch_next(0);
+    for (int k0 = 0; k0 < iters; k0 += UNROLL) {
+      if (k0 + UNROLL <= full_iters) batch(k0, std::true_type{});   // uniform over the CTA
+      else batch(k0, std::false_type{});
     }
 #pragma unroll
     for (int mask = LPR; mask < 32; mask <<= 1) {
