@@ -372,8 +372,14 @@ def main():
         plan.set_params(**dict(case.params, gather_mode=1))
         kv_graphs = capture(False)
         ms_kv, _, _ = timed(kv_graphs, min(args.steps, 500), args.warmup)
-        plan.set_params(**case.params)
         del kv_graphs
+        # sampling keys per KV head: the heads of a group draw nested samples, so their sampled rows coincide
+        # (another sample than the default's, hence other budgets: a variant, not the headline)
+        plan.set_params(**dict(case.params, rng_head_is_kv=1))
+        grp_graphs = capture(False)
+        ms_grp, _, _ = timed(grp_graphs, min(args.steps, 500), args.warmup)
+        plan.set_params(**case.params)
+        del grp_graphs
 
         # optional external context: a third-party dense paged-decode kernel on the same cache
         fi_us = None
@@ -523,6 +529,7 @@ def main():
                    "mean_density": round(density, 4), "sparsity_x": round(1.0 / density, 2),
                    "mean_budget": float(b_dyn.mean()), "status_bits": status, "step_us_percentiles": step_pct,
                    "kv_gather_variant_us_per_step": round(ms_kv * 1e3, 2),
+                   "kv_head_sampling_keys_variant_us_per_step": round(ms_grp * 1e3, 2),
                    "value_is": "max-over-ranks step time / n_gpus (each rank runs its own layer)"},
         "e2e": {"value": ms_e2e_max * 1e3 / world, "unit": UNIT,
                 "h2d_bytes_per_step": int(qh.numel() * 2 + bth.numel() * 4 + slh.numel() * 4),
