@@ -230,6 +230,9 @@ def main():
                          "reasoning-length) and add them to the JSON line as `other_configs`")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
+    ap.add_argument("--profile-config", default="cfg2", choices=["cfg2", "cfg5", "cfg4"],
+                    help="with --profile-only: the workload to run (cfg5: batch 8 at n=32768; cfg4: batch 32, mixed "
+                         "lengths; one cache pool each, 1.1 GB and 2.6 GB)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if not args.profile_only else args.warmup
 
@@ -261,15 +264,19 @@ def main():
 
     # ---- workload: every rank runs its own copy of the layer (weak scaling, no exchange on the path)
     case = synth.config2_llama8b()
+    npools = POOLS
+    if args.profile_only and args.profile_config != "cfg2":
+        case = {"cfg5": synth.config5_reasoning, "cfg4": synth.config4_serving}[args.profile_config]()
+        npools = 1                                         # the cache alone is several times the L2
     dev0 = vb.case_to_device(case)
-    pools = [dev0] + [{k: v.clone() for k, v in dev0.items()} for _ in range(POOLS - 1)]
+    pools = [dev0] + [{k: v.clone() for k, v in dev0.items()} for _ in range(npools - 1)]
     plan = vb.plan_for_case(case)
     plan.set_params(**case.params)
     outs = [torch.empty_like(dev0["q"]) for _ in range(POOLS)]
     stream = torch.cuda.Stream()
 
     def step(i, dense=False):
-        d = pools[i % POOLS]
+        d = pools[i % npools]
         if dense:
             plan.dense_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], outs[i % POOLS],
                               stream=stream)
