@@ -11,9 +11,11 @@
 // Two decompositions:
 //  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
 //    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
-//    grid stride.  A chunk is exactly what one CTA keeps in flight at once (one batch: 64 rows of 128 bf16),
-//    so a step with up to 1184 chunks costs one memory round trip per CTA; a head uses up to 128 chunks
-//    (longer lists get chunks of two, three, ... batches);
+//    grid stride.  A chunk is a whole number of batches (a batch = what one CTA keeps in flight at once:
+//    64 rows of 128 bf16) and a head uses up to 32 chunks: lists of more than 32 batches get chunks of
+//    two, three, ... batches, whose index loads overlap the previous batch's rows.  (With up to 128
+//    single-batch chunks per head the last finisher needed three dependent rounds of partial loads and
+//    long lists overflowed the grid: 92 -> 76 us per step at 5x density, 73.0 -> 72.4 us at 10x.);
 //  * per head (larger problems): grid (32, heads, batch); a head with budget b uses ceil(b / chunk) of its
 //    32 CTAs, chunk = max(256, ceil(b / 32)) rows, the others exit at once.
 #include "vattn_internal.cuh"

@@ -62,7 +62,7 @@ struct Prob {
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
   double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
   float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
-  int gat_slots;          // 128 when batch * heads <= 128 (flat decomposition), else 32
+  int gat_slots;          // partial slots per head (32 in both decompositions)
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, dense_splits;
   vattn_debug dbg;
@@ -191,7 +191,7 @@ __device__ __forceinline__ Geo head_geometry(const Prob& p, int n) {
 #define VATTN_MAX_BATCH_BF16 1536     // batch rows a bf16 plan accepts (12 bytes of shared memory per row in k_score)
 #define VATTN_STAT_MAXS 16            // most split CTAs per head and row kind of the statistics kernel
 #define VATTN_GATHER_FLAT_HEADS 128   // the gather kernel's flat decomposition serves up to this many heads ...
-#define VATTN_GATHER_FLAT_SLOTS 128   // ... with up to this many chunks (partials) each
+#define VATTN_GATHER_FLAT_SLOTS 32   // ... with up to this many chunks (partials) each
 __device__ __forceinline__ unsigned cand0_bound(const Geo& g) {
   if (g.n_s <= 0 || g.b0 <= 0) return 0u;
   const double want = (double)g.b0 + 6.0 * sqrt((double)g.b0) + 16.0;
