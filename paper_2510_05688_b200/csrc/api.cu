@@ -19,7 +19,7 @@ struct vattn_plan {
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
   int prof_calls;           // calls recorded since the last read
   // derived
-  int G, npad, nwords, stat_splits, dense_splits;
+  int G, npad, nwords, stat_splits, stat_splits_base, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
       off_det, off_piv, off_gat, off_dense, off_cand, off_sort, total;
   int cand_cap, gat_slots;
@@ -80,13 +80,23 @@ void derive(vattn_plan* pl) {
   if (pl->npad == 0) pl->npad = 32;
   pl->nwords = pl->npad / 32;
   const int heads = s.batch * s.num_q_heads;
-  // statistics kernel (128-thread CTAs, two CTA kinds per split): one wave of about 5 CTAs per SM
-  int sp = (5 * kNumSM) / (2 * heads);
-  // (when even one CTA per kind and head overfills the wave the kernel is throughput-bound: split freely)
-  pl->stat_splits = sp < 4 ? 4 : (sp > kMaxStatSplits ? kMaxStatSplits : sp);
+  // statistics kernel (128-thread CTAs, 5 per SM): one wave for both kinds of CTA.  The base-sample rows are
+  // on the step's critical path (they wait for the sample), the deterministic rows start earlier: three
+  // fifths of the wave go to the former (14 + 9 CTAs per head at 32 heads; 11 + 11 made the step 2 us longer,
+  // 16 + 7 left the deterministic CTAs as the last to finish).  (When even four CTAs per kind and head
+  // overfill the wave the kernel is throughput-bound: split freely.)
+  const int wave = (5 * kNumSM) / heads;
+  if (wave < 8) {
+    pl->stat_splits = pl->stat_splits_base = 4;
+  } else {
+    const int sb = (3 * wave + 2) / 5;
+    pl->stat_splits_base = sb > kMaxStatSplits ? kMaxStatSplits : sb;
+    const int sd = wave - pl->stat_splits_base;
+    pl->stat_splits = sd < 4 ? 4 : (sd > kMaxStatSplits ? kMaxStatSplits : sd);
+  }
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
-  sp = (4 * kNumSM + groups - 1) / groups;
+  const int sp = (4 * kNumSM + groups - 1) / groups;
   pl->dense_splits = sp < 1 ? 1 : (sp > 128 ? 128 : sp);
   const size_t BH = (size_t)heads, D = (size_t)s.head_dim;
   size_t off = 0;
@@ -159,7 +169,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
   p.gat_slots = pl->gat_slots;
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
-  p.stat_splits = pl->stat_splits; p.dense_splits = pl->dense_splits;
+  p.stat_splits = pl->stat_splits; p.stat_splits_base = pl->stat_splits_base; p.dense_splits = pl->dense_splits;
   p.dbg = pl->dbg;
   return VATTN_OK;
 }
@@ -319,16 +329,18 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
   p.sink = sink; p.window = window; p.k = k;
   {
-    // statistics kernel: about 64 rows (8 per row group) per CTA, never more CTAs than rows warrant
+    // statistics kernel: never more CTAs than rows warrant (about 64 deterministic, 48 base-sample rows each)
     const double msl = (double)plan->shape.max_seq_len;
     double kmax = plan->params.topk_frac > 0.f ? floor((double)plan->params.topk_frac * msl) : (double)k;
     double rows = (double)sink + (double)window + kmax;
     if (rows > msl) rows = msl;
-    const double brows = (double)p.base_rate * msl;
-    if (brows > rows) rows = brows;
-    int want = (int)((rows + 127.0) / 128.0) * 2;          // about 64 rows per CTA
+    int want = (int)((rows + 127.0) / 128.0) * 2;
     if (want < 1) want = 1;
     if (want < p.stat_splits) p.stat_splits = want;
+    const double brows = (double)p.base_rate * msl;
+    want = (int)((brows + 95.0) / 96.0) * 2;
+    if (want < 1) want = 1;
+    if (want < p.stat_splits_base) p.stat_splits_base = want;
   }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;

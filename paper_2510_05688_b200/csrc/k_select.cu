@@ -920,7 +920,7 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   pdl_trigger();
   pdl_wait();
   HeadMeta meta = p.meta[bh];
-  const int D = p.D, NE = D + 3, S = p.stat_splits;
+  const int D = p.D, NE = D + 3;
   const int n_s = meta.n_s, b0 = meta.b0;
   if (meta.n == 0) {
     if (tid == 0) {
@@ -934,7 +934,8 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   // ---- partial sums in split order; kind 0 = deterministic rows, kind 1 = base-sample rows
   for (int item = tid; item < 2 * NE; item += NT) {
     const int kind = item / NE, e = item % NE;
-    const double* src = p.stat_part + ((long long)bh * 2 * VATTN_STAT_MAXS + kind * S) * NE + e;
+    const int S = kind ? p.stat_splits_base : p.stat_splits;
+    const double* src = p.stat_part + ((long long)bh * 2 * VATTN_STAT_MAXS + kind * VATTN_STAT_MAXS) * NE + e;
     double v[VATTN_STAT_MAXS];
 #pragma unroll
     for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;

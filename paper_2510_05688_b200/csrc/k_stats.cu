@@ -102,9 +102,13 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const bool base_cta = (int)blockIdx.z >= p.B;
   const int h = blockIdx.y, b = base_cta ? blockIdx.z - p.B : blockIdx.z, g = h / p.G;
   const int bh = b * p.Hq + h;
-  const int S = p.stat_splits;
+  const int S = base_cta ? p.stat_splits_base : p.stat_splits;   // CTAs of this kind per head
   const int split = blockIdx.x;
-  const int vx = (base_cta ? S : 0) + split;       // position among the head's 2 S partials
+  const int vx = (base_cta ? MAXS : 0) + split;    // position among the head's 2 MAXS partial slots
+  if (split >= S) {                                // the grid is as wide as the larger of the two split counts
+    if (base_cta) pdl_wait();                      // (every base-row CTA waits, see below)
+    return;
+  }
   TICK_BEGIN(p, VATTN_K_STATS);
   pdl_trigger();
   // What k_select_topk wrote (meta, I_t) is complete before this grid can start: the grid before this one
@@ -278,8 +282,8 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 }  // namespace
 
 cudaError_t launch_stats(const Prob& p, cudaStream_t s) {
-  dim3 grid(p.stat_splits, p.Hq, 2 * p.B), block(NT);
-  if (p.stat_splits < 1 || p.stat_splits > MAXS) return cudaErrorInvalidValue;
+  if (p.stat_splits < 1 || p.stat_splits > MAXS || p.stat_splits_base < 1 || p.stat_splits_base > MAXS) return cudaErrorInvalidValue;
+  dim3 grid(p.stat_splits > p.stat_splits_base ? p.stat_splits : p.stat_splits_base, p.Hq, 2 * p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (p.D == 128) return launch_pdl(k_stats<bf16_t, 128>, grid, block, 0, s, p);
     else return launch_pdl(k_stats<bf16_t, 64>, grid, block, 0, s, p);

@@ -64,7 +64,7 @@ struct Prob {
   float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
   int gat_slots;          // partial slots per head (32 in both decompositions)
   float* dense_part;      // [B,Hq,dense_splits,D+2]
-  int stat_splits, dense_splits;
+  int stat_splits, stat_splits_base, dense_splits;   // statistics CTAs per head: deterministic rows, base-sample rows
   vattn_debug dbg;
 };
 
