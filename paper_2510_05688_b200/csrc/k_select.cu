@@ -919,8 +919,34 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
   TICK_BEGIN(p, VATTN_K_BUDGET);
   pdl_trigger();
   pdl_wait();
-  HeadMeta meta = p.meta[bh];
   const int D = p.D, NE = D + 3;
+  // ---- partial sums in split order; kind 0 = deterministic rows, kind 1 = base-sample rows.  The requests
+  // depend on nothing but the head's number: they go out together with the read of the head's meta record.
+  double item_sum[(2 * (128 + 3) + NT - 1) / NT];
+#pragma unroll
+  for (int it = 0; it < (2 * (128 + 3) + NT - 1) / NT; ++it) {
+    const int item = tid + it * NT;
+    double sum = 0.0;
+    if (item < 2 * NE) {
+      const int kind = item / NE, e = item % NE;
+      const int S = kind ? p.stat_splits_base : p.stat_splits;
+      const double* src = p.stat_part + ((long long)bh * 2 * VATTN_STAT_MAXS + kind * VATTN_STAT_MAXS) * NE + e;
+      double v[VATTN_STAT_MAXS];
+#pragma unroll
+      for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;
+#pragma unroll
+      for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) sum += v[sp];
+    }
+    item_sum[it] = sum;
+  }
+  // the pivot the base-row CTAs used (all of them computed the same numbers; split 0 published them)
+  double piv_v[(128 + 1 + NT - 1) / NT];
+#pragma unroll
+  for (int it = 0; it < (128 + 1 + NT - 1) / NT; ++it) {
+    const int e = tid + it * NT;
+    piv_v[it] = (e <= D) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
+  }
+  HeadMeta meta = p.meta[bh];
   const int n_s = meta.n_s, b0 = meta.b0;
   if (meta.n == 0) {
     if (tid == 0) {
@@ -931,21 +957,16 @@ __global__ void __launch_bounds__(NT, 1) k_budget(const Prob p, int bigbytes) {
     }
     return;
   }
-  // ---- partial sums in split order; kind 0 = deterministic rows, kind 1 = base-sample rows
-  for (int item = tid; item < 2 * NE; item += NT) {
-    const int kind = item / NE, e = item % NE;
-    const int S = kind ? p.stat_splits_base : p.stat_splits;
-    const double* src = p.stat_part + ((long long)bh * 2 * VATTN_STAT_MAXS + kind * VATTN_STAT_MAXS) * NE + e;
-    double v[VATTN_STAT_MAXS];
 #pragma unroll
-    for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) v[sp] = (sp < S) ? __ldcg(src + (long long)sp * NE) : 0.0;
-    double sum = 0.0;
-#pragma unroll
-    for (int sp = 0; sp < VATTN_STAT_MAXS; ++sp) sum += v[sp];
-    tot[kind][e] = sum;
+  for (int it = 0; it < (2 * (128 + 3) + NT - 1) / NT; ++it) {
+    const int item = tid + it * NT;
+    if (item < 2 * NE) tot[item / NE][item % NE] = item_sum[it];
   }
-  // the pivot the base-row CTAs used (all of them computed the same numbers; split 0 published them)
-  for (int e = tid; e <= D; e += NT) piv[e] = (b0 > 0) ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
+#pragma unroll
+  for (int it = 0; it < (128 + 1 + NT - 1) / NT; ++it) {
+    const int e = tid + it * NT;
+    if (e <= D) piv[e] = (b0 > 0) ? piv_v[it] : 0.0;     // no base sample: the record holds an earlier step's numbers
+  }
   __syncthreads();
   double* det = p.det_sums + (long long)bh * (D + 1);
   for (int e = tid; e <= D; e += NT) det[e] = tot[0][e];
