@@ -113,7 +113,13 @@ void derive(vattn_plan* pl) {
   pl->off_stat = take(BH * 2 * kMaxStatSplits * (D + 3) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
-  pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? VATTN_GATHER_FLAT_SLOTS : kMaxGatherSplits;
+  // partial slots (chunks) per head of the gather kernel: 32, except that a handful of heads may use more of
+  // the 8 x 148 CTAs (64 to 128 chunks each when that many fit the grid at once)
+  {
+    const size_t fit = (size_t)(8 * kNumSM) / BH;
+    const size_t flat = fit >= 2 * VATTN_GATHER_FLAT_SLOTS ? (fit > 128 ? 128 : fit) : VATTN_GATHER_FLAT_SLOTS;
+    pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? (int)flat : kMaxGatherSplits;
+  }
   pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
   {

@@ -12,7 +12,8 @@
 //  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
 //    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
 //    grid stride.  A chunk is a whole number of batches (a batch = what one CTA keeps in flight at once:
-//    64 rows of 128 bf16) and a head uses up to 32 chunks: lists of more than 32 batches get chunks of
+//    64 rows of 128 bf16) and a head uses up to 32 chunks (64 to 128 when no more than 18 heads share the
+//    grid): lists of more batches than that get chunks of
 //    two, three, ... batches, whose index loads overlap the previous batch's rows.  (With up to 128
 //    single-batch chunks per head the last finisher needed three dependent rounds of partial loads and
 //    long lists overflowed the grid: 92 -> 76 us per step at 5x density, 73.0 -> 72.4 us at 10x.);
@@ -27,7 +28,6 @@ constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
 constexpr int UNROLL = 8;         // rows in flight per row group (16-byte slices kept raw until used)
 constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
-constexpr int FLAT_MAXS = VATTN_GATHER_FLAT_SLOTS;   // ... flat decomposition
 constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
 constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
 
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
     s_meta[tid] = mt;
     nb = mt.n > 0 ? mt.b : 0;
     const int batches = (nb + BATCH - 1) / BATCH;
-    rows = BATCH * max(1, (batches + FLAT_MAXS - 1) / FLAT_MAXS);
+    rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
     cnt = max(1, (nb + rows - 1) / rows);             // a head without samples still writes its output
     s_rows[tid] = rows;
     s_b[tid] = nb;
@@ -305,9 +305,9 @@ template <typename T, int D, bool KV>
 static cudaError_t launch_gather_t(const Prob& p, cudaStream_t s) {
   const int BH = p.B * p.Hq;
   if (BH <= FLAT_MAX_HEADS) {
-    // at most FLAT_MAXS chunks per head; 8 CTAs per SM walk them with a grid stride
-    if (p.gat_slots < FLAT_MAXS) return cudaErrorInvalidValue;
-    const long long most = (long long)BH * FLAT_MAXS;
+    // at most gat_slots chunks per head; 8 CTAs per SM walk them with a grid stride
+    if (p.gat_slots < VATTN_GATHER_FLAT_SLOTS) return cudaErrorInvalidValue;
+    const long long most = (long long)BH * p.gat_slots;
     const int grid = (int)(most < 8 * 148 ? most : 8 * 148);
     return launch_pdl(k_gather_flat<T, D, KV>, dim3(grid), dim3(NT), 0, s, p);
   }

@@ -62,7 +62,7 @@ struct Prob {
   double* det_sums;       // [B,Hq,D+1]  N_f then D_f
   double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
   float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
-  int gat_slots;          // partial slots per head (32 in both decompositions)
+  int gat_slots;          // partial slots (chunks) per head: 32; 64 to 128 when at most 18 heads share the grid
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int stat_splits, stat_splits_base, dense_splits;   // statistics CTAs per head: deterministic rows, base-sample rows
   vattn_debug dbg;
