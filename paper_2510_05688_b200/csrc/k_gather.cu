@@ -3,7 +3,7 @@
 // which is SDPA_{S,p} of Sec. 3 with p = 1 on I_f and p = b/n_s on I_dyn.
 //
 // HBM-bound row gather.  Work unit = a chunk of consecutive entries of one head's I_dyn list.  LPR lanes
-// fetch one V row with one 16-byte load each; a row group keeps 8 rows in flight and requests the next
+// fetch one V row with one 16-byte load each; a row group keeps 4 rows in flight and requests the next
 // batch's indices (token + physical slot, written by the select kernels) while the current rows arrive.
 // Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
 // last CTA of the head ("ticket"), so results are reproducible.
@@ -12,7 +12,7 @@
 //  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
 //    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
 //    grid stride.  A chunk is a whole number of batches (a batch = what one CTA keeps in flight at once:
-//    64 rows of 128 bf16) and a head uses up to 32 chunks (64 to 128 when no more than 18 heads share the
+//    32 rows of 128 bf16) and a head uses up to 32 chunks (64 to 128 when no more than 18 heads share the
 //    grid): lists of more batches than that get chunks of
 //    two, three, ... batches, whose index loads overlap the previous batch's rows.  (With up to 128
 //    single-batch chunks per head the last finisher needed three dependent rounds of partial loads and
@@ -26,7 +26,7 @@ namespace {
 
 constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
-constexpr int UNROLL = 8;         // rows in flight per row group (16-byte slices kept raw until used)
+constexpr int UNROLL = 4;         // rows in flight per row group (16-byte slices kept raw until used); 8 and 2 are slower
 constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
 constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
 constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
@@ -226,7 +226,7 @@ struct Gather {
 };
 
 template <typename T, int D, bool KV>
-__global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
+__global__ void __launch_bounds__(NT, 10) k_gather(const Prob p) {
   using G = Gather<T, D, KV>;
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
