@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   constexpr int RG = NWARP * RPI;         // row groups per CTA
   __shared__ double part[NWARP][NE];
   __shared__ double piv[D + 1];
+  __shared__ double pivT[D];             // the pivot's w*V, element-major per lane: pivT[e * LPR + j]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // grid (S, Hq, 2 B): the deterministic-row CTAs of every head come first in dispatch order, so they take
@@ -206,7 +207,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
     };
-    double cw = 0.0, cr[EPL];
+    double cw = 0.0;
     auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
       double wv[UN];
       weights64<T, D>(p, qf, row, m, j, wv);
@@ -219,7 +220,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
           s2 = fma(dw, dw, s2);
 #pragma unroll
           for (int e = 0; e < EPL; ++e) {
-            const double dr = w * (double)row[u].v.get(e) - cr[e];
+            const double dr = w * (double)row[u].v.get(e) - pivT[e * LPR + j];
             acc[e] += dr;
             s3 = fma(dr, dr, s3);
           }
@@ -235,13 +236,16 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     issue(rowB, actB);
     fetch(2 * UN);
     cw = weight64<T, D>(p, qf, prow, m);
+    if (warp == 0 && rsub == 0) {                     // every row group holds the same pivot: one of them shares it
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) cr[e] = cw * (double)prow.v.get(e);
-    if (warp == 0 && rsub == 0) {
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) piv[j * EPL + e] = cr[e];
+      for (int e = 0; e < EPL; ++e) {
+        const double c = cw * (double)prow.v.get(e);
+        piv[j * EPL + e] = c;
+        pivT[e * LPR + j] = c;
+      }
       if (j == 0) piv[D] = cw;
     }
+    __syncthreads();
     for (int k0 = 0; k0 < max(iters, 1); k0 += 2 * UN) {
       if (k0 > 0) { issue(rowB, actB); fetch(k0 + 2 * UN); }
       reduce(rowA, actA);
