@@ -55,30 +55,30 @@ __device__ __forceinline__ void load_row(const Prob& p, int g, int ph, int j, Ro
 __device__ __forceinline__ int phys_of(const Prob& p, int b, int tok) { return page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15); }
 // fp64 inner product <q, K[row]> computed by the LPR lanes of a row group from their K slices
 template <typename T, int D>
-__device__ __forceinline__ double dot64(const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r) {
+__device__ __forceinline__ double dot64(const double* qs, const RowRegs<T>& r) {
   constexpr int EPL = Elem<T>::EPL, LPR = D / EPL;
   double acc = 0.0;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) acc = fma((double)qf[e], (double)r.k.get(e), acc);
+  for (int e = 0; e < EPL; ++e) acc = fma(qs[e * LPR], (double)r.k.get(e), acc);
 #pragma unroll
   for (int mask = LPR / 2; mask >= 1; mask >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, mask);
   return acc;
 }
 // fp64 weight of one token
 template <typename T, int D>
-__device__ __forceinline__ double weight64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T>& r, double m) {
-  return exp(dot64<T, D>(qf, r) * (double)p.scale - m);
+__device__ __forceinline__ double weight64(const Prob& p, const double* qs, const RowRegs<T>& r, double m) {
+  return exp(dot64<T, D>(qs, r) * (double)p.scale - m);
 }
 // weights of the UN rows of a batch with ONE exp per lane: lane j of the row group evaluates the row
 // j % UN, the results are handed round with shuffles (every lane of a group holds all UN inner products)
 template <typename T, int D>
-__device__ __forceinline__ void weights64(const Prob& p, const float (&qf)[Elem<T>::EPL], const RowRegs<T> (&row)[UN],
+__device__ __forceinline__ void weights64(const Prob& p, const double* qs, const RowRegs<T> (&row)[UN],
                                           double m, int j, double (&w)[UN]) {
   constexpr int LPR = D / Elem<T>::EPL;
   static_assert((UN == 2 || UN == 4) && LPR >= UN, "one lane per row of the batch");
   double d[UN];
 #pragma unroll
-  for (int u = 0; u < UN; ++u) d[u] = dot64<T, D>(qf, row[u]);
+  for (int u = 0; u < UN; ++u) d[u] = dot64<T, D>(qs, row[u]);
   const int mu = j & (UN - 1);
   double mine = d[0];
 #pragma unroll
@@ -133,8 +133,17 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
   const int rg = warp * RPI + rsub;
   const int iters = (r_end - r_begin + RG - 1) / RG;      // uniform over the CTA
 
-  float qf[EPL];
-  Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+  // q in fp64, element-major per lane (qT[e * LPR + j]): read from shared memory where it is used instead of
+  // living in 16 registers
+  __shared__ double qT[D];
+  if (warp == 0 && rsub == 0) {
+    float qf[EPL];
+    Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) qT[e * LPR + j] = (double)qf[e];
+  }
+  __syncthreads();
+  const double* qs = qT + j;
 
   double acc[EPL], s1 = 0.0, s2 = 0.0, s3 = 0.0;           // det: N_f slice, D_f;  base: Sr slice, Sw, Sww, Srr
 #pragma unroll
@@ -161,7 +170,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     };
     auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
       double wv[UN];
-      weights64<T, D>(p, qf, row, m, j, wv);                   // every lane takes part in the shuffles
+      weights64<T, D>(p, qs, row, m, j, wv);                   // every lane takes part in the shuffles
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const double w = wv[u];
@@ -210,7 +219,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     double cw = 0.0;
     auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
       double wv[UN];
-      weights64<T, D>(p, qf, row, m, j, wv);
+      weights64<T, D>(p, qs, row, m, j, wv);
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const double w = wv[u];
@@ -235,7 +244,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const Prob p) {
     fetch(UN);
     issue(rowB, actB);
     fetch(2 * UN);
-    cw = weight64<T, D>(p, qf, prow, m);
+    cw = weight64<T, D>(p, qs, prow, m);
     if (warp == 0 && rsub == 0) {                     // every row group holds the same pivot: one of them shares it
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
