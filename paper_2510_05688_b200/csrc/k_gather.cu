@@ -226,7 +226,7 @@ struct Gather {
 };
 
 template <typename T, int D, bool KV>
-__global__ void __launch_bounds__(NT, 10) k_gather(const Prob p) {
+__global__ void __launch_bounds__(NT, KV ? 8 : 10) k_gather(const Prob p) {
   using G = Gather<T, D, KV>;
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
