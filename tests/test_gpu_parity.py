@@ -345,6 +345,17 @@ def test_many_short_sequences_in_one_batch():
     check(small("bf16", lens, Hq=8, Hkv=2))
 
 
+@pytest.mark.parametrize("B,Hq,Hkv", [(2, 32, 8), (4, 32, 8), (17, 8, 2)])
+def test_head_counts_around_the_decomposition_thresholds(B, Hq, Hkv):
+    # 64 heads: statistics CTAs split unevenly between the two row kinds, flat gather with 32 chunks per head;
+    # 128 heads: even split (the wave is overfull), the flat gather's largest head count; 136 heads: the
+    # per-head gather.  Forced budgets of 3,000 rows give chunks of several batches and a ragged last batch.
+    lens = [int(x) for x in np.random.default_rng(5 + B).integers(3500, 5200, size=B)]
+    case = small("bf16", lens, Hq=Hq, Hkv=Hkv, sink=16, window=32, k=64)
+    check(case)
+    check(case, force_budget=3001)
+
+
 def test_eps_delta_guarantee_holds_on_the_cuda_path():
     # Definition 4.1 of the paper on the product path: over many seeds, the relative error of the sparse
     # output against exact attention exceeds eps with frequency at most delta (plus binomial slack)
