@@ -118,6 +118,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
   if (wid == CWN) {
     // =============================================================== producer warp
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    const unsigned long long kpolicy = l2_evict_first_policy();
     long long i = 0;                                  // stages armed so far
     int ucount = 0;
     bool failed = false;
@@ -160,9 +161,9 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
             const bf16_t* src = kc + (long long)pid * p.sb + (long long)g * p.sh;
             mbar_expect_tx(&full[stage], PAGEB + (with_q ? qbytes : 0u));
             if (with_q) bulk_g2s(qring + (size_t)stage * qslot_bytes, qsrc, qbytes, &full[stage]);
-            if (p.st == D) bulk_g2s(dst, src, PAGEB, &full[stage]);
+            if (p.st == D) bulk_g2s_stream(dst, src, PAGEB, &full[stage], kpolicy);
             else
-              for (int rr = 0; rr < VATTN_BLOCK; ++rr) bulk_g2s(dst + rr * ROWB, src + (long long)rr * p.st, ROWB, &full[stage]);
+              for (int rr = 0; rr < VATTN_BLOCK; ++rr) bulk_g2s_stream(dst + rr * ROWB, src + (long long)rr * p.st, ROWB, &full[stage], kpolicy);
           }
         }
         i += min(S, cnt - k0);
