@@ -256,6 +256,7 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     const int k = k_base + lane;
     pg_ids = (k < mine) ? page_of(p, b, wglob + k * wtot) : 0;
   };
+  const unsigned long long stream_policy = l2_evict_first_policy();
   // whole warp: lane 0 arms the barrier, then lanes 0..15 copy one V row each (into padded rows) and
   // lanes 16..31 the K page (one copy, or one row each when rows are not contiguous)
   auto issue = [&](int k, int pg) {
@@ -267,9 +268,10 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
       mbar_expect_tx(bar, 2 * KPAGE);
     }
     __syncwarp();
-    if (lane < 16) bulk_g2s(dst + KPAGE + lane * VROWB, vc + off + (long long)lane * p.st, ROWB, bar);
-    else if (p.st == D) { if (lane == 16) bulk_g2s(dst, kc + off, KPAGE, bar); }
-    else bulk_g2s(dst + (lane - 16) * ROWB, kc + off + (long long)(lane - 16) * p.st, ROWB, bar);
+    // K and V are read once: evict-first in L2
+    if (lane < 16) bulk_g2s_stream(dst + KPAGE + lane * VROWB, vc + off + (long long)lane * p.st, ROWB, bar, stream_policy);
+    else if (p.st == D) { if (lane == 16) bulk_g2s_stream(dst, kc + off, KPAGE, bar, stream_policy); }
+    else bulk_g2s_stream(dst + (lane - 16) * ROWB, kc + off + (long long)(lane - 16) * p.st, ROWB, bar, stream_policy);
   };
   load_ids(0);
   for (int k = 0; k < min(DN_NST, mine); ++k) issue(k, __shfl_sync(0xFFFFFFFFu, pg_ids, k));
