@@ -5,7 +5,8 @@
 // HBM-bound row gather.  Work unit = a chunk of consecutive entries of one head's I_dyn list.  LPR lanes
 // fetch one V row with one 16-byte load each; a row group keeps 4 rows in flight and requests the next
 // batch's indices (token + physical slot, written by the select kernels) while the current rows arrive.
-// Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
+// Rows are fetched with streaming loads (read once: first to leave the caches, so that the scores and index
+// lists stay in L2).  Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
 // last CTA of the head ("ticket"), so results are reproducible.
 //
 // Two decompositions:
@@ -110,7 +111,7 @@ struct Gather {
           const int ph = ph_n[u];
           off[u] = (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL;
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (FULL || tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(kcg + off[u]);
+          if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(kcg + off[u]));
         }
         fetch_next(k0 + UNROLL);
 #pragma unroll
@@ -123,7 +124,7 @@ struct Gather {
           for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
           if (j == u) { w_mine = p.scale * dot; tok_mine = tok[u]; }
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (FULL || tok[u] >= 0) raw[u] = *reinterpret_cast<const uint4*>(vc + off[u]);
+          if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + off[u]));
         }
       } else {
 #pragma unroll
@@ -133,7 +134,7 @@ struct Gather {
           if (j == u) tok_mine = tok[u];
           if (FULL || tok[u] >= 0) {
             const int ph = ph_n[u];
-            raw[u] = *reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL);
+            raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL));
           }
         }
         if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);

@@ -26,15 +26,17 @@ constexpr int NWARP = NT / 32;
 constexpr int UN = 2;            // rows per batch of a row group; two batches are in flight (double buffer)
 constexpr int MAXS = VATTN_STAT_MAXS;   // most split CTAs per head and kind
 
+// 16-byte row slices, fetched with streaming loads: a row is read once, so it should be the first to leave the
+// caches (the scores, index lists and partials that the step re-reads stay in L2)
 template <typename T> struct Raw;
 template <> struct Raw<float> {
   float4 v;
-  __device__ __forceinline__ void ld(const float* p) { v = *reinterpret_cast<const float4*>(p); }
+  __device__ __forceinline__ void ld(const float* p) { v = __ldcs(reinterpret_cast<const float4*>(p)); }
   __device__ __forceinline__ float get(int e) const { return e == 0 ? v.x : e == 1 ? v.y : e == 2 ? v.z : v.w; }
 };
 template <> struct Raw<bf16_t> {
   uint4 v;
-  __device__ __forceinline__ void ld(const bf16_t* p) { v = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ void ld(const bf16_t* p) { v = __ldcs(reinterpret_cast<const uint4*>(p)); }
   __device__ __forceinline__ float get(int e) const {
     const unsigned w = (e >> 1) == 0 ? v.x : (e >> 1) == 1 ? v.y : (e >> 1) == 2 ? v.z : v.w;
     return __uint_as_float((e & 1) ? (w & 0xFFFF0000u) : (w << 16));
