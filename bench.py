@@ -496,7 +496,7 @@ def main():
         "k_gather": int(b_dyn.sum()) * (d * es + 4),
     }
     # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2_llama8b.md
-    traffic = {"k_score": 67.90e6, "k_cand": 0.02e6, "k_select_topk": 4.33e6, "k_presort": 2.55e6,
+    traffic = {"k_score": 68.86e6, "k_cand": 0.02e6, "k_select_topk": 4.33e6, "k_presort": 2.55e6,
                "k_stats": 25.57e6, "k_budget": 0.88e6, "k_gather": 20.13e6}
     peak, peak_kind = measured_peaks()
     kern = {}
