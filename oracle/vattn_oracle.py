@@ -9,7 +9,7 @@ Every function follows a passage of the paper, taken in the paper's order and no
 
   scores            <K[i], q>                                 (Sec. 3, full SDPA equation)
   deterministic_sets I_s, I_l, I_t, I_f, n_s                  (Algorithm 1, lines 1-5)
-  sample            uniform-sample(I_f, ., n)                 (Algorithm 1 line 7; Algorithm 2 line 1)
+  walk_order, sample uniform-sample(I_f, ., n)                (Algorithm 1 line 7; Algorithm 2 line 1)
   base_stats        get-stats / compute-stats                 (Algorithm 2; Corollaries D.2)
   budgets           b_D, b_N (Corollaries D.2), b_SDPA (Theorem 4.3), lower cap by the base budget
                     (captions of the epsilon/delta ablation figures in App. F)
@@ -29,8 +29,10 @@ Readings taken where the paper is silent:
   * sink/window are absolute token counts, top-k is taken over the middle range only, ties go
     to the lowest index;
   * uniform sampling is WITHOUT replacement (so a budget equal to the residual gives dense SDPA);
-    it is realised as "the c smallest (Philox key, index) pairs", with independent key streams
-    for the base sample (stream 0) and the final sample (stream 1);
+    it is realised as "the first c residual tokens met when the middle range is walked in the order
+    of a keyed pseudorandom permutation" (a Feistel network with cycle walking whose round keys are
+    Philox4x32-10 words), with independent keys for the base sample (stream 0) and the final
+    sample (stream 1);
   * sample variances use the unbiased (b0 - 1) denominator; tau uses the full estimates
     D_hat = D_f + ..., N_hat = N_f + ... as the corollaries define them;
   * the Theorem's min over (eps', delta') is taken in closed form over eps' and on the grid
@@ -108,32 +110,88 @@ def philox4x32_10(c0, c1, c2, c3, k0, k1):
     return (c0.astype(np.uint32), c1.astype(np.uint32), c2.astype(np.uint32), c3.astype(np.uint32))
 
 
-def sample_keys(n, seed, batch_idx, head_idx, layer, step, stream):
-    """32-bit sampling key of every token i < n for one (batch row, head, layer, step, stream).
+def walk_round_keys(seed, batch_idx, head_idx, layer, step, stream):
+    """Eight 32-bit round keys of one (batch row, head, layer, step, stream):
 
-    key_i = Philox4x32-10(key = (seed_lo, seed_hi),
-                          ctr = (i >> 2, (batch << 16) | head, layer, (step << 1) | stream))[i & 3]
-    """
-    nq = (n + 3) // 4
-    i4 = np.arange(nq, dtype=np.uint64)
+    the words of Philox4x32-10(key = (seed_lo, seed_hi), ctr = (c, (batch << 16) | head, layer,
+    (step << 1) | stream)) for c = 0 and c = 1."""
     w1 = ((int(batch_idx) & 0xFFFF) << 16) | (int(head_idx) & 0xFFFF)
     w3 = ((int(step) << 1) | int(stream)) & 0xFFFFFFFF
-    out = philox4x32_10(i4, np.uint64(w1), np.uint64(int(layer) & 0xFFFFFFFF), np.uint64(w3),
-                        int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
-    return np.stack(out, axis=1).reshape(-1)[:n]
+    out = philox4x32_10(np.arange(2, dtype=np.uint64), np.uint64(w1), np.uint64(int(layer) & 0xFFFFFFFF),
+                        np.uint64(w3), int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)
+    return [int(out[j][c]) for c in range(2) for j in range(4)]
 
 
-def sample(residual, c, keys):
-    """uniform-sample: the c residual indices with the smallest (key, index), returned ascending.
+_MIX_A = np.uint64(0x9E3779B1)
+_MIX_B = np.uint64(0x85EBCA77)
+_MIX_C = np.uint64(0xC2B2AE3D)
 
-    Ranking all residual tokens by an independent uniform key and keeping the first c is a
-    uniform draw of c indices without replacement (Algorithm 1 line 7, Algorithm 2 line 1)."""
-    residual = np.asarray(residual, np.int64)
+
+def _mix32(x, key):
+    """Round function of the permutation: xor with the round key, then three rounds of
+    (multiply by an odd constant mod 2^32, xor-shift right), so that the low output bits depend on
+    every input bit."""
+    v = (np.asarray(x, np.uint64) ^ np.uint64(key)) & _MASK32
+    v = (v * _MIX_A) & _MASK32
+    v ^= v >> np.uint64(15)
+    v = (v * _MIX_B) & _MASK32
+    v ^= v >> np.uint64(13)
+    v = (v * _MIX_C) & _MASK32
+    v ^= v >> np.uint64(16)
+    return v
+
+
+def walk_bits(mlen):
+    """Width of the permutation's domain: the smallest w >= 2 with 2^w >= mlen."""
+    return max(2, int(max(int(mlen) - 1, 0)).bit_length())
+
+
+def feistel(x, w, keys):
+    """Keyed bijection of [0, 2^w): an alternating Feistel network of 8 rounds on the halves
+    L (high floor(w/2) bits) and R (low ceil(w/2) bits).  Even rounds replace L by
+    L xor (mix32(R, key_i) mod 2^|L|), odd rounds R by R xor (mix32(L, key_i) mod 2^|R|); each round is
+    invertible whatever mix32 is, so the composition is a permutation."""
+    lw = w // 2
+    rw = w - lw
+    x = np.asarray(x, np.uint64)
+    L = x >> np.uint64(rw)
+    R = x & np.uint64((1 << rw) - 1)
+    for i in range(8):
+        if i % 2 == 0:
+            L = L ^ (_mix32(R, keys[i]) & np.uint64((1 << lw) - 1))
+        else:
+            R = R ^ (_mix32(L, keys[i]) & np.uint64((1 << rw) - 1))
+    return (L << np.uint64(rw)) | R
+
+
+def walk_order(mlen, keys):
+    """sigma(0), ..., sigma(mlen-1): the keyed permutation of [0, mlen) obtained from `feistel` on
+    [0, 2^w) by cycle walking (apply the bijection again while the image is >= mlen)."""
+    mlen = int(mlen)
+    w = walk_bits(mlen)
+    x = feistel(np.arange(mlen, dtype=np.uint64), w, keys)
+    while True:
+        out = x >= np.uint64(mlen)
+        if not out.any():
+            return x.astype(np.int64)
+        x[out] = feistel(x[out], w, keys)
+
+
+def sample(in_residual, c, first, order):
+    """uniform-sample: walk the middle range [first, first + len(order)) in the order
+    first + sigma(0), first + sigma(1), ... and keep the first c tokens that are residual tokens;
+    returned ascending.
+
+    sigma is a keyed pseudorandom permutation of the middle range, so the residual tokens appear in
+    a uniformly random order and the first c of them are a uniform draw of c residual tokens without
+    replacement (Algorithm 1 line 7, Algorithm 2 line 1).  Any prefix of the walk is itself such a
+    draw, which is what lets the base sample and the final sample be read off walks of their own."""
     c = int(c)
-    if c <= 0 or residual.size == 0:
+    if c <= 0 or len(order) == 0:
         return np.zeros(0, np.int64)
-    order = np.lexsort((residual, keys[residual]))      # primary: key, secondary: index
-    return np.sort(residual[order[:c]])
+    toks = int(first) + np.asarray(order, np.int64)
+    toks = toks[np.asarray(in_residual, bool)[toks]]
+    return np.sort(toks[:c])
 
 
 # ----------------------------------------------------------------------------- Algorithm 1, lines 1-5
@@ -254,8 +312,13 @@ def dense_sdpa(q, K, V, scale):
 
 # ----------------------------------------------------------------------------- one head, one step
 def decode_head(q, K, V, *, sink, window, k, eps, delta, seed, batch_idx, head_idx, rng_head,
-                base_rate=0.025, scale=None, mode=0, layer=0, step=0, force_budget=-1):
-    """Algorithm 1 for one (batch row, query head).  q [d], K,V [n,d] fp64.  Returns a dict."""
+                base_rate=0.025, scale=None, mode=0, layer=0, step=0, force_budget=-1, nested_base=0):
+    """Algorithm 1 for one (batch row, query head).  q [d], K,V [n,d] fp64.  Returns a dict.
+
+    nested_base = 1 reads the base sample off the final sample's walk (I_bs = its first b0 residual
+    tokens, I_dyn = its first b: I_bs is a subset of I_dyn), the reuse of budget-calculation rows that the
+    implementation paragraph of Sec. 4.2 describes; 0 (default) draws the two independently, as the
+    separate uniform-sample calls of Algorithm 2 line 1 and Algorithm 1 line 7 read."""
     n, d = K.shape
     if scale is None:
         scale = float(np.float32(1.0 / np.sqrt(d)))
@@ -278,12 +341,17 @@ def decode_head(q, K, V, *, sink, window, k, eps, delta, seed, batch_idx, head_i
                    stats=np.array([D, 0.0, 0.0, D, np.sqrt((N ** 2).sum()), 0.0, 0.0, m]))
         return res
     b0 = base_size(n_s, base_rate)
-    I_bs = sample(R, b0, sample_keys(n, seed, batch_idx, rng_head, layer, step, 0))
+    first = min(int(sink), n)                       # the middle range starts behind the sink tokens
+    mlen = max(n - int(window), first) - first
+    in_R = np.zeros(n, bool)
+    in_R[R] = True
+    I_bs = sample(in_R, b0, first,
+                  walk_order(mlen, walk_round_keys(seed, batch_idx, rng_head, layer, step, 1 if nested_base else 0)))
     st = base_stats(w, V, I_f, I_bs, n_s)
     b_D, b_N, b_S = budgets(st, n_s, eps, delta)
     bx = (b_S, b_D, b_N)[int(mode)]
     b = final_budget(bx, b0, n_s, force_budget)
-    I_dyn = sample(R, b, sample_keys(n, seed, batch_idx, rng_head, layer, step, 1))
+    I_dyn = sample(in_R, b, first, walk_order(mlen, walk_round_keys(seed, batch_idx, rng_head, layer, step, 1)))
     N, D = combine(w, V, I_f, I_dyn, n_s)
     res.update(out=N / D, I_bs=I_bs, I_dyn=I_dyn, b0=b0, b=b,
                budgets=(ceil_sat(b_D), ceil_sat(b_N), ceil_sat(b_S), b),
@@ -301,7 +369,7 @@ def resolve_k(k, topk_frac, n):
 
 def vattn_decode(q, k_cache, v_cache, block_table, seq_lens, sink, window, k, eps, delta, seed, *,
                  dtype, base_rate=0.025, topk_frac=0.0, scale=None, mode=0, layer=0, step=0,
-                 rng_head_is_kv=0, force_budget=-1, heads=None):
+                 rng_head_is_kv=0, force_budget=-1, nested_base=0, heads=None):
     """One decode step over the paged cache.  Returns (out [B,Hq,d] in the storage type, details).
 
     q [B,Hq,d]; caches [num_blocks,Hkv,16,d]; every query head h uses KV head h // (Hq/Hkv) and
@@ -329,7 +397,8 @@ def vattn_decode(q, k_cache, v_cache, block_table, seq_lens, sink, window, k, ep
         r = decode_head(to_f64(q[b, h], dtype), K, V, sink=sink, window=window,
                         k=resolve_k(k, topk_frac, n), eps=eps, delta=delta, seed=seed, batch_idx=b,
                         head_idx=h, rng_head=(g if rng_head_is_kv else h), base_rate=base_rate,
-                        scale=scale, mode=mode, layer=layer, step=step, force_budget=force_budget)
+                        scale=scale, mode=mode, layer=layer, step=step, force_budget=force_budget,
+                        nested_base=nested_base)
         out64[b, h] = r["out"]
         details[(b, h)] = r
     out = f64_to_bf16_bits(out64) if dtype == "bf16" else out64.astype(np.float32)

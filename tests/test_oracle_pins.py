@@ -7,8 +7,10 @@ P2  tiny inputs: top-k against a full sort, the residual against a set differenc
     must equal the finite-population formula for sampling without replacement.
 P3  the (eps, delta) definition (Definition 4.1 of the paper) over 1,000 seeds.
 P4  closed-form budgets (Lemma 4.1, Corollaries D.2, Theorem 4.3) on hand-computable populations.
-P5  Philox4x32-10 against the published known-answer vectors.
-P6  the sampler is uniform over subsets (chi-square) and never selects outside the residual.
+P5  Philox4x32-10 against the published known-answer vectors; the walk permutation against brute force
+    (a bijection, undone by the network run backwards; cycle walking stays inside the middle range).
+P6  the sampler is uniform over subsets and over walk positions (chi-square) and never selects outside the
+    residual.
 """
 import itertools
 import math
@@ -161,25 +163,128 @@ def test_p2_estimator_unbiased_over_all_subsets_and_variance():
     assert abs(D - D_exact) < 1e-14
 
 
-def test_p2_sample_is_smallest_key_index_pairs():
-    keys = np.array([5, 1, 9, 1, 7, 1, 3, 3], np.uint32)
-    R = np.array([1, 2, 3, 5, 6, 7])
-    pairs = sorted((int(keys[i]), int(i)) for i in R)
+def test_p2_sample_is_first_residual_tokens_of_the_walk():
+    # a hand-written walk order over the middle range [2, 10): the sample is its first c residual tokens
+    order = np.array([4, 0, 7, 2, 6, 1, 3, 5])                  # sigma(0..7); tokens 6, 2, 9, 4, 8, 3, 5, 7
+    in_R = np.zeros(12, bool)
+    in_R[[2, 3, 5, 6, 8, 9]] = True                             # tokens 4 and 7 are top-k members
+    walk = [6, 2, 9, 8, 3, 5]                                   # the walk with the members struck out
     for c in range(0, 7):
-        want = sorted(i for _, i in pairs[:c])
-        assert O.sample(R, c, keys).tolist() == want
-    assert O.sample(R, 99, keys).tolist() == R.tolist()
+        assert O.sample(in_R, c, 2, order).tolist() == sorted(walk[:c])
+    assert O.sample(in_R, 99, 2, order).tolist() == [2, 3, 5, 6, 8, 9]
+    assert O.sample(in_R, 3, 2, np.zeros(0, np.int64)).tolist() == []
 
 
-def test_sample_keys_layout_matches_philox_counter_definition():
-    n, seed, b, h, layer, step = 23, (0xDEADBEEF << 32) | 0x12345678, 3, 7, 5, 1000
+def test_walk_round_keys_are_the_philox_words_of_counters_0_and_1():
+    seed, b, h, layer, step = (0xDEADBEEF << 32) | 0x12345678, 3, 7, 5, 1000
     for stream in (0, 1):
-        keys = O.sample_keys(n, seed, b, h, layer, step, stream)
-        for i in (0, 1, 2, 3, 4, 13, 22):
-            out = O.philox4x32_10(np.uint64(i >> 2), np.uint64((b << 16) | h), np.uint64(layer),
+        keys = O.walk_round_keys(seed, b, h, layer, step, stream)
+        want = []
+        for c in (0, 1):
+            out = O.philox4x32_10(np.uint64(c), np.uint64((b << 16) | h), np.uint64(layer),
                                   np.uint64((step << 1) | stream), seed & 0xFFFFFFFF, seed >> 32)
-            assert int(keys[i]) == int(out[i & 3])
-    assert not np.array_equal(O.sample_keys(n, seed, b, h, layer, step, 0), O.sample_keys(n, seed, b, h, layer, step, 1))
+            want += [int(o) for o in out]
+        assert keys == want and len(set(keys)) == 8
+    assert O.walk_round_keys(seed, b, h, layer, step, 0) != O.walk_round_keys(seed, b, h, layer, step, 1)
+    assert O.walk_round_keys(seed, b, h, layer, step, 0) != O.walk_round_keys(seed, b, h + 1, layer, step, 0)
+
+
+def _unfeistel(y, w, keys):
+    """The network run backwards, written out here on Python ints (not the oracle's code): undoing
+    round i needs only the half that round i left untouched."""
+    lw = w // 2
+    rw = w - lw
+    L, R = y >> rw, y & ((1 << rw) - 1)
+
+    def mix(x, k):
+        v = (x ^ k) & 0xFFFFFFFF
+        v = (v * 0x9E3779B1) & 0xFFFFFFFF
+        v ^= v >> 15
+        v = (v * 0x85EBCA77) & 0xFFFFFFFF
+        v ^= v >> 13
+        v = (v * 0xC2B2AE3D) & 0xFFFFFFFF
+        v ^= v >> 16
+        return v
+    for i in reversed(range(8)):
+        if i % 2 == 0:
+            L ^= mix(R, keys[i]) & ((1 << lw) - 1)
+        else:
+            R ^= mix(L, keys[i]) & ((1 << rw) - 1)
+    return (L << rw) | R
+
+
+def test_feistel_is_a_bijection_and_the_reversed_network_undoes_it():
+    rng = np.random.default_rng(12)
+    for w in range(2, 14):
+        keys = [int(x) for x in rng.integers(0, 2**32, size=8)]
+        img = O.feistel(np.arange(1 << w, dtype=np.uint64), w, keys)
+        assert sorted(img.tolist()) == list(range(1 << w))
+        for x in (0, 1, (1 << w) - 1, (1 << w) // 3):
+            assert _unfeistel(int(img[x]), w, keys) == x
+    assert [O.walk_bits(m) for m in (0, 1, 2, 4, 5, 8, 9, 1024, 1025, 32512)] == [2, 2, 2, 2, 3, 3, 4, 10, 11, 15]
+
+
+def test_walk_order_is_a_permutation_of_the_middle_range():
+    rng = np.random.default_rng(13)
+    for mlen in list(range(0, 70)) + [127, 128, 129, 1000, 4097, 32512]:
+        keys = [int(x) for x in rng.integers(0, 2**32, size=8)]
+        order = O.walk_order(mlen, keys)
+        assert sorted(order.tolist()) == list(range(mlen))
+    # cycle walking: the image of j is the first point of the orbit j -> feistel(j) -> ... below mlen
+    keys = [int(x) for x in rng.integers(0, 2**32, size=8)]
+    mlen, w = 37, 6
+    order = O.walk_order(mlen, keys)
+    for j in range(mlen):
+        y = int(O.feistel(np.array([j], np.uint64), w, keys)[0])
+        while y >= mlen:
+            y = int(O.feistel(np.array([y], np.uint64), w, keys)[0])
+        assert y == int(order[j])
+
+
+def test_walk_positions_are_uniform_and_streams_are_unrelated():
+    # over seeds, sigma(j) is uniform on [0, mlen) for fixed j, and neighbouring images are not tied together
+    mlen, T = 13, 26000
+    hits = np.zeros((3, mlen))
+    gap = np.zeros(mlen)
+    same = 0
+    for seed in range(T):
+        o0 = O.walk_order(mlen, O.walk_round_keys(seed, 2, 5, 1, 9, 0))
+        o1 = O.walk_order(mlen, O.walk_round_keys(seed, 2, 5, 1, 9, 1))
+        for r, j in enumerate((0, 6, 12)):
+            hits[r, o0[j]] += 1
+        gap[(o0[1] - o0[0]) % mlen] += 1
+        same += int(o0[0] == o1[0])
+    exp = T / mlen
+    for r in range(3):
+        assert ((hits[r] - exp) ** 2 / exp).sum() < 40.0          # 12 dof: P(chi2 > 40) ~ 7e-5
+    assert gap[0] == 0
+    expg = T / (mlen - 1)
+    assert ((gap[1:] - expg) ** 2 / expg).sum() < 38.0            # 11 dof
+    assert abs(same / T - 1.0 / mlen) < 4.0 * math.sqrt((1 / mlen) * (1 - 1 / mlen) / T)
+
+
+def test_resolve_k_and_base_size_by_hand():
+    # k = floor(f32(f_t) * n) with the product in fp64: f32(0.02) = 0.0199999995529651..., so 0.02 * 4150 falls
+    # just below 83
+    assert [O.resolve_k(7, 0.02, n) for n in (4097, 4150, 4151)] == [81, 82, 83]
+    assert O.resolve_k(7, 0.0, 4150) == 7 and O.resolve_k(7, None, 10) == 7
+    assert O.resolve_k(0, 0.5, 9) == 4 and O.resolve_k(3, 1.0, 9) == 9
+    # b0 = min(n_s, max(2, floor(f32(f_b) * n_s))): f32(0.025) = 0.02500000037..., so 0.025 * 80 = 2.00000003 -> 2
+    assert [O.base_size(ns, 0.025) for ns in (1, 2, 3, 79, 80, 120)] == [1, 2, 2, 2, 2, 3]
+    assert O.base_size(0, 0.025) == 0 and O.base_size(40, 1.0) == 40 and O.base_size(1000, 0.1) == 100
+
+
+def test_nested_base_sample_is_a_prefix_of_the_final_sample():
+    case = small_case("fp32", seq_lens=(300,), Hq=2, Hkv=1, d=16, sink=4, window=4, k=8)
+    _, det = run_oracle(case, base_rate=0.1, nested_base=1, force_budget=60)
+    _, ind = run_oracle(case, base_rate=0.1, force_budget=60)
+    for key, r in det.items():
+        assert r["b"] == 60 and r["b0"] == 28 and set(r["I_bs"].tolist()) <= set(r["I_dyn"].tolist())
+        # the final sample's walk is the same in both variants; only the base sample moves
+        assert not set(ind[key]["I_bs"].tolist()) <= set(ind[key]["I_dyn"].tolist())
+        keys1 = O.walk_round_keys(case.seed, key[0], key[1], 0, 0, 1)
+        walk = [4 + int(x) for x in O.walk_order(300 - 8, keys1) if (4 + int(x)) not in set(r["I_t"].tolist())]
+        assert sorted(walk[:r["b0"]]) == r["I_bs"].tolist() and sorted(walk[:r["b"]]) == r["I_dyn"].tolist()
 
 
 # ----------------------------------------------------------------------------- P3
@@ -303,7 +408,10 @@ def test_base_sample_estimates_are_close_to_population_values():
     pop_trace = ((w[R, None] * V[R]).var(axis=0, ddof=1)).sum()
     errs = []
     for seed in range(40):
-        I_bs = O.sample(R, O.base_size(len(R), 0.1), O.sample_keys(16384, seed, 0, 0, 0, 0, 0))
+        in_R = np.zeros(16384, bool)
+        in_R[R] = True
+        I_bs = O.sample(in_R, O.base_size(len(R), 0.1), 128,
+                        O.walk_order(16384 - 256, O.walk_round_keys(seed, 0, 0, 0, 0, 0)))
         st = O.base_stats(w, V, I_f, I_bs, len(R))
         errs.append((abs(st["sigma2"] - pop_sigma2) / pop_sigma2, abs(st["trace"] - pop_trace) / pop_trace))
     errs = np.array(errs).mean(axis=0)
@@ -326,12 +434,14 @@ def test_p5_philox_known_answer_vectors():
 # ----------------------------------------------------------------------------- P6
 def test_p6_sampler_uniform_over_subsets():
     n, c = 12, 3
-    R = np.array([2, 3, 5, 6, 7, 8, 9, 10])              # residual of size 8
+    R = np.array([2, 3, 5, 6, 7, 8, 9, 10])              # residual of size 8: middle range [1, 11) minus {1, 4}
+    in_R = np.zeros(n, bool)
+    in_R[R] = True
     subsets = {s: 0 for s in itertools.combinations(R.tolist(), c)}
     T = 28000
     incl = np.zeros(n)
     for seed in range(T):
-        pick = O.sample(R, c, O.sample_keys(n, seed, 0, 1, 2, 3, 1))
+        pick = O.sample(in_R, c, 1, O.walk_order(10, O.walk_round_keys(seed, 0, 1, 2, 3, 1)))
         subsets[tuple(pick.tolist())] += 1               # KeyError if anything outside R is drawn
         incl[pick] += 1
     exp = T / len(subsets)
