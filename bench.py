@@ -1,6 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the verified sparse-attention decode step (one step = one pass of the whole hot path:
-score, select, statistics + budget, final sample, gather + combine) on the Llama-3.1-8B-shaped layer
+score pass; top-k selection and sample lists; statistics rows; budget, final sample and combination) on
+the Llama-3.1-8B-shaped layer
 at 32K context and ~10x sparsity.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -30,6 +31,23 @@ UNIT = "us"
 POOLS = 4
 WORKLOAD = ("cfg2_llama8b: B=1, Hq=32, Hkv=8 (GQA 4), d=128, n=32768, bf16 paged KV (block 16, HND, permuted "
             "block table), sink=window=128, k=819 (2.5%), f_b=0.025, eps=delta=0.05, heavy-hitter strength c1=9.85")
+
+
+def read_traffic():
+    """DRAM bytes per launch (read + write) of each kernel on this workload, from the tracked ncu summary
+    profiles/dram_traffic_cfg2.txt (lines `kernel bytes`; the header names the commit it was captured at)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic_cfg2.txt")
+    vals, note = {}, "none: no ncu capture of the current kernels has been summarised"
+    if os.path.exists(path):
+        for ln in open(path):
+            if ln.startswith("#"):
+                if "captured at" in ln:
+                    note = ln.lstrip("# ").strip()
+                continue
+            parts = ln.split()
+            if len(parts) >= 2:
+                vals[parts[0]] = float(parts[1])
+    return vals, note
 
 
 def measured_peaks():
@@ -115,8 +133,8 @@ def run_reference(args, rank, world):
     oracle_step(case, heads=[heads_all[0]])
     t_one = time.perf_counter() - t0
     budget_s = 150.0
-    steps = max(1, min(args.steps, int(budget_s / max(t_one, 1e-3))))
-    warm = min(args.warmup, 3)
+    steps = max(1, min(args.steps, int(budget_s / max(t_one, 1e-3)) - args.warmup))
+    warm = args.warmup
     for i in range(warm):
         oracle_step(case, heads=[heads_all[i % len(heads_all)]])
     t0, c0 = time.perf_counter(), cpu_seconds()
@@ -130,7 +148,8 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": us_full, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": us_full / 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
-            "cpu_baseline": {"value": us_full, "unit": UNIT, "cores": ncores, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": us_full, "unit": UNIT, "cores": ncores, "host_cores": os.cpu_count(),
+                             "kind": "oracle", "sample": sample},
             "e2e": {"value": us_full, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -373,7 +392,7 @@ def main():
         plan.disable_debug()
         del tl_graphs
         timeline = {name: [round(float(tl[k_, 0]), 2), round(float(tl[k_, 1]), 2) if tl[k_, 1] > 0 else None]
-                    for k_, name in enumerate(["k_zero"] + vb.KERNEL_NAMES)}
+                    for k_, name in enumerate(vb.TICK_NAMES)}
 
         # the K+V gather variant (weights recomputed from the K rows of the sampled tokens)
         plan.set_params(**dict(case.params, gather_mode=1))
@@ -456,7 +475,9 @@ def main():
             d = pools[i % POOLS]
             plan.decode_host(qh, d["k_cache"], d["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
                              case.delta, case.seed, outh, stream=stream)
-        for i in range(3):
+        # the entry point records a call's CUDA graph on the second call with one argument set: warm up until every
+        # pool's graph exists, so that only replays are timed
+        for i in range(max(args.warmup, 2 * POOLS + 1)):
             e2e_step(i)
         if world > 1:
             dist.barrier()
@@ -481,39 +502,49 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- algorithmic bytes per launch: what each kernel must move (K rows and score words for the score pass,
-    # 8-byte candidate pairs for the sampling kernels, K and V rows for the statistics, V rows for the gather)
+    # ---- algorithmic bytes per launch: what each kernel must move.  Score pass: every K row once, 4 bytes written
+    # per (token, query head).  Per-head kernel: the scores once (selection), K and V rows of I_f and I_bs (rescored
+    # in fp64), V row + 4-byte score of every token of I_dyn.
     es, d, Hq, Hkv = 2, case.head_dim, case.num_q_heads, case.num_kv_heads
     n_tot = int(case.seq_lens.sum())
     n_f = kks.sum() + Hq * (min(case.sink, n_tot) + min(case.window, n_tot))
     alg = {
         "k_score": n_tot * Hkv * d * es + n_tot * Hq * 4,
-        "k_cand": int(0.27 * n_tot * Hq) * 8,
-        "k_select_topk": n_tot * Hq * 4,
-        "k_presort": int(0.25 * n_tot * Hq) * 8 + int(b0s.sum()) * 8 + 2 * n_tot * Hq // 8,
+        "k_walk": int(5 * b0s.sum()) * 4,
+        "k_select": n_tot * Hq * 4 + int(kks.sum()) * 8 + int(b0s.sum()) * 8 + int(min(8 * b0s.max(), n_tot)) * Hq * 12,
         "k_stats": int(n_f + b0s.sum()) * d * es * 2,
-        "k_budget": n_tot * Hq // 8,
-        "k_gather": int(b_dyn.sum()) * (d * es + 4),
+        "k_final": int(b_dyn.sum()) * (d * es + 8),
     }
-    # DRAM bytes per launch (read + write) from the ncu capture summarised in profiles/ncu_step_cfg2_llama8b.md
-    traffic = {"k_score": 68.86e6, "k_cand": 0.02e6, "k_select_topk": 4.33e6, "k_presort": 2.55e6,
-               "k_stats": 25.57e6, "k_budget": 0.88e6, "k_gather": 20.13e6}
+    rows_bytes = alg["k_stats"] + alg["k_final"]
+    traffic, traffic_note = read_traffic()
     peak, peak_kind = measured_peaks()
     kern = {}
     for name in vb.KERNEL_NAMES:
         us = prof[name] / max(calls, 1) * 1e3
         kern[name] = {"us": round(us, 2), "alg_bytes": int(alg[name]),
                       "gbs": round(alg[name] / (us * 1e-6) / 1e9, 1) if us > 0 else None}
-    # dominant kernel = the one that moves most of the step's bytes (59 % of them) and the only one bound by
-    # bandwidth at this size; the kernel with the largest event time is reported beside it
+    # dominant kernel = the one that moves most of the step's bytes
     top = "k_score"
     top_us = prof[top] / max(calls, 1) * 1e3
     achieved = alg[top] / (top_us * 1e-6) / 1e9
-    slow = max(vb.KERNEL_NAMES, key=lambda k_: prof[k_])
     b2b_gbs = alg[top] / (us_score_b2b * 1e-6) / 1e9
     density = float(np.mean((kks + 256 + b_dyn) / n_tot))
-    sparse_bytes = sum(alg[k_] for k_ in ("k_score", "k_stats", "k_gather"))
+    sparse_bytes = alg["k_score"] + rows_bytes
     dense_bytes = 2 * n_tot * Hkv * d * es
+
+    def span(name):
+        a, b_ = timeline[name]
+        return (b_ - a) if (a is not None and b_ is not None and b_ > a) else None
+
+    def frac_of(bytes_, us):
+        if not us:
+            return None
+        g = bytes_ / (us * 1e-6) / 1e9
+        return {"us": round(us, 2), "achieved": round(g, 1), "frac": round(g / peak, 4), "frac_of_8TBs_nominal": round(g / 8000.0, 4)}
+    # the row kernels (statistics, final sample): device-side spans inside graph-replayed steps
+    rows_span = None
+    if timeline["k_stats"][0] is not None and timeline["k_final"][1] is not None:
+        rows_span = timeline["k_final"][1] - timeline["k_stats"][0]
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -523,8 +554,9 @@ def main():
             reps += 1
         wall = time.perf_counter() - t_cpu0
         cpu_us = wall / reps * 1e6
-        cpu = {"value": cpu_us, "unit": UNIT, "cores": cores_used(cpu_seconds() - c_cpu0, wall), "kind": "oracle",
-               "sample": f"{reps} full steps of the same workload (all 32 heads, fp64 numpy)"}
+        cpu = {"value": cpu_us, "unit": UNIT, "cores": cores_used(cpu_seconds() - c_cpu0, wall),
+               "host_cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"{reps} full steps of the same workload (all 32 heads, fp64 numpy, one thread)"}
 
     us_step = ms_step_max * 1e3
     line = {
@@ -544,18 +576,21 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": top, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "frac_of": peak_kind, "frac_of_8TBs_nominal": round(achieved / 8000.0, 4),
-                     "traffic": traffic.get(top), "alg_bytes_per_launch": int(alg[top]), "us_per_launch": round(top_us, 2),
+                     "traffic": traffic.get(top), "traffic_source": traffic_note,
+                     "alg_bytes_per_launch": int(alg[top]), "us_per_launch": round(top_us, 2),
                      "timing": "CUDA events around the kernel inside plain-launched steps (includes the launch gap)",
                      "back_to_back": {"us_per_launch": round(us_score_b2b, 2), "achieved": round(b2b_gbs, 1),
                                       "frac": round(b2b_gbs / peak, 4),
                                       "timing": "the kernel alone, 16 launches per CUDA graph, pools rotating"},
-                     "device_timer": {"us_per_launch": round(timeline["k_score"][1] - timeline["k_score"][0], 2),
-                                      "achieved": round(alg[top] / ((timeline["k_score"][1] - timeline["k_score"][0]) * 1e-6) / 1e9, 1),
-                                      "frac": round(alg[top] / ((timeline["k_score"][1] - timeline["k_score"][0]) * 1e-6) / 1e9 / peak, 4),
-                                      "timing": "first CTA start to last CTA end (%globaltimer) inside graph-replayed steps, "
-                                                "the key pre-filter running beside it"},
-                     "largest_event_time": {"kernel": slow, "us_per_launch": kern[slow]["us"], "achieved": kern[slow]["gbs"],
-                                            "frac": round((kern[slow]["gbs"] or 0.0) / peak, 4)}},
+                     "device_timer": dict(frac_of(alg[top], span("k_score")) or {},
+                                          timing="first CTA start to last CTA end (%globaltimer) inside graph-replayed steps")},
+        # the gather / reduce part of the step (rows of I_f, I_bs and I_dyn) and the whole step, against the same peak
+        "roofline_rows": dict(frac_of(rows_bytes, rows_span) or {}, kernel="k_stats + k_final", alg_bytes=int(rows_bytes),
+                              traffic=(traffic.get("k_stats", 0) + traffic.get("k_final", 0)) or None,
+                              timing="first CTA of k_stats to last CTA of k_final (%globaltimer), graph-replayed steps"),
+        "roofline_k_stats": dict(frac_of(alg["k_stats"], span("k_stats")) or {}, alg_bytes=int(alg["k_stats"])),
+        "roofline_k_final": dict(frac_of(alg["k_final"], span("k_final")) or {}, alg_bytes=int(alg["k_final"])),
+        "roofline_step": dict(frac_of(sparse_bytes, us_step) or {}, alg_bytes=int(sparse_bytes)),
         "kernels": kern,
         "timeline_us": timeline,
         "dense": {"us_per_step": round(ms_dense_max * 1e3, 2), "alg_bytes": int(dense_bytes),

@@ -74,24 +74,33 @@ typedef struct {
                               only their V rows are read (default); 1: K and V rows are read and the scores are
                               recomputed from the K rows in fp32: the traffic of a pipeline whose selector leaves
                               no scores behind (the paper's composition with an approximate top-k, Sec. 4) */
+  int32_t nested_base;     /* 0: base sample and final sample are independent draws (Algorithm 2 line 1 and
+                              Algorithm 1 line 7 are separate calls); 1: the base sample is the first b0 tokens of
+                              the final sample's walk, so I_bs is a subset of I_dyn (the reuse of the rows read for
+                              the budget that the implementation paragraph of Sec. 4.2 describes) */
 } vattn_params;
 
 /* Optional per-call introspection.  All DEVICE pointers; NULL = not wanted.  cap = max_seq_len. */
 typedef struct {
   int32_t *topk_idx, *topk_cnt;   /* [B,Hq,cap], [B,Hq]  I_t ascending (I_f = sink range + I_t + window range) */
-  int32_t *base_idx, *base_cnt;   /* I_bs, b0: in ascending (Philox key, token) order when drawn from the sorted
-                                     candidate list (paths bit 1), in ascending token order otherwise: a set */
-  int32_t *dyn_idx,  *dyn_cnt;    /* I_dyn, b: likewise (paths bit 2) */
+  int32_t *base_idx, *base_cnt;   /* I_bs, b0: in the order of the walk that drew it (compare as a set) */
+  int32_t *dyn_idx,  *dyn_cnt;    /* I_dyn, b: likewise */
   int32_t *budgets;               /* [B,Hq,4] ceil(b_D), ceil(b_N), ceil(b_SDPA) (saturating at 2^31-1), b */
   double  *stats;                 /* [B,Hq,8] D_f, sigma^2, Tr(Sigma), D_hat, |N_hat|_2, n_s, b0, m (weights are
                                      exp(s - m) with m the head's largest fp32 score) */
   float   *scores;                /* [B,Hq,cap] fp32 scores s_i = scale * <K[i], q> */
-  int32_t *paths;                 /* [B,Hq] which code path selected each set: bit 0 top-k from the sampled threshold
-                                     estimate, bit 1 base sample from the pre-filtered list, bit 2 final sample =
-                                     prefix of the pre-sorted list (a clear bit = the full-context select ran) */
-  unsigned long long *kernel_ticks; /* [VATTN_NUM_KERNELS + 1][2] device-side time stamps in ns (%globaltimer) of the
-                                     counter-clearing kernel (row 0) and the kernels of a step in the order listed
-                                     for vattn_set_profiling: [k][0] = earliest CTA start, [k][1] = latest end.
+  int32_t *paths;                 /* [B,Hq] which code path the top-k selection took: bit 0 the usual one (one histogram
+                                     of the keys' top bits, then an exact selection among the few candidates around
+                                     the threshold; clear: the radix select over the whole middle range), bit 1
+                                     near-tie tokens were rescored in fp64 and ranked from a list, bit 2 they were
+                                     too many for the list and the exact 64-bit radix select ran
+                                     (VATTN_STATUS_BAND_OVERFLOW) */
+  unsigned long long *kernel_ticks; /* [VATTN_NUM_TICKS][2] device-side time stamps in ns (%globaltimer): rows 0-5 the
+                                     counter-clearing kernel, the score kernel, the walk kernel, the selection kernel,
+                                     the statistics kernel and the final-sample kernel ([k][0] = earliest CTA start,
+                                     [k][1] = latest end); row 6 the top-k selection proper (first CTA past its
+                                     dependency wait .. last CTA with I_t complete); row 7 the budget (first final-sample CTA past its
+                                     dependency wait .. last CTA that knows its budget).
                                      Folded with atomic min / max: set [k][0] = UINT64_MAX and [k][1] = 0 before the
                                      step to be observed.  Unlike event profiling this leaves the step as it is */
 } vattn_debug;
@@ -121,9 +130,12 @@ int    vattn_set_debug(vattn_plan* plan, const vattn_debug* debug);
  *   b    = clamp(ceil(b_X(eps, delta; base-sample statistics)), b0, n_s)
  *   I_dyn= b residual tokens, uniform without replacement (Philox stream 1)
  *   out  = (N_f + n_s/b * sum_{I_dyn} w_i V[i]) / (D_f + n_s/b * sum_{I_dyn} w_i),  w_i = exp(s_i - m)
- * (Sec. 4.1 numerator/denominator equations; SDPA_{S,p} of Sec. 3).  A uniform sample is "the c
- * residual tokens with the smallest (key_i, i)", key_i = Philox4x32-10(key = seed,
- * counter = (i>>2, batch<<16 | head, layer, step<<1 | stream))[i & 3].
+ * (Sec. 4.1 numerator/denominator equations; SDPA_{S,p} of Sec. 3).  A uniform sample of c tokens is
+ * "the first c residual tokens met when the middle range [sink, n - window) is walked in the order
+ * sink + sigma(0), sink + sigma(1), ...": sigma is a keyed permutation of the middle range, an 8-round
+ * alternating Feistel network on ceil(log2(range)) bits (at least 2) with cycle walking, whose round keys are
+ * the eight words of Philox4x32-10(key = seed, counter = (c, batch<<16 | head, layer, step<<1 | stream)),
+ * c = 0, 1, and whose round function is xor with the round key followed by three multiply / xor-shift steps.
  * Degenerate inputs: n = 0 -> out row = 0; sink+window >= n -> exact attention, budget 0;
  * k larger than the middle range is clipped.
  * eps, delta in (0,1).  Errors: INVALID_ARG, WORKSPACE, CUDA.
@@ -197,15 +209,14 @@ int vattn_last_launch_count(const vattn_plan* plan);
 int vattn_set_stop_after(vattn_plan* plan, int kernels);
 
 /* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
- * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score, sampling-key
- * pre-filter, top-k select, sampling sort, statistics + budget, slow-path final select, gather +
- * combine), for up to 256 calls between two reads.  The events serialise kernels that otherwise overlap
- * (the key pre-filter runs beside the score kernel, the sampling sort beside the top-k select, the first
- * half of the statistics beside the sampling), so the per-kernel times add up to more than an unprofiled
- * step takes.  vattn_read_profile waits for the last recorded call, writes the summed elapsed
- * milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to *calls
- * (host), and starts a new window.  Events add a little latency: do not enable in production. */
-#define VATTN_NUM_KERNELS 7
+ * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score pass; walk tokens;
+ * selection and sample lists; deterministic and base-sample rows; budget, final sample and combination), for up to 256 calls between
+ * two reads.  The events keep a kernel's prologue from running beside its predecessor, so the times add up to
+ * more than an unprofiled step takes.  vattn_read_profile waits for the last recorded call, writes the
+ * summed elapsed milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to
+ * *calls (host), and starts a new window.  Events add a little latency: do not enable in production. */
+#define VATTN_NUM_KERNELS 5
+#define VATTN_NUM_TICKS 8
 int vattn_set_profiling(vattn_plan* plan, int enable);
 int vattn_read_profile(vattn_plan* plan, float* ms_sum, int* calls);
 

@@ -21,7 +21,9 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
            "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
-KERNEL_NAMES = ["k_score", "k_cand", "k_select_topk", "k_presort", "k_stats", "k_budget", "k_gather"]
+KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_final"]
+NUM_TICKS = 32
+TICK_NAMES = ["k_zero", "k_score", "k_walk", "k_select", "k_stats", "k_final", "topk", "budget"]
 
 
 class Shape(C.Structure):
@@ -34,7 +36,8 @@ class Shape(C.Structure):
 class Params(C.Structure):
     _fields_ = [("base_rate", C.c_float), ("topk_frac", C.c_float), ("scale", C.c_float), ("mode", C.c_int32),
                 ("layer", C.c_int32), ("step", C.c_int32), ("rng_head_is_kv", C.c_int32),
-                ("force_budget", C.c_int32), ("force_budget_on", C.c_int32), ("gather_mode", C.c_int32)]
+                ("force_budget", C.c_int32), ("force_budget_on", C.c_int32), ("gather_mode", C.c_int32),
+                ("nested_base", C.c_int32)]
 
 
 class Debug(C.Structure):
@@ -180,10 +183,10 @@ class Plan:
         self.debug = None
 
     def enable_kernel_ticks(self):
-        """Register only the device-side time-stamp buffer ([kernels + 1, 2] int64; row 0 = the clearing kernel).
+        """Register only the device-side time-stamp buffer ([NUM_TICKS, 2] int64, rows named by TICK_NAMES).
         Call reset_kernel_ticks() before the step to observe, read the tensor after it."""
         import torch
-        self.ticks = torch.zeros(len(KERNEL_NAMES) + 1, 2, dtype=torch.int64, device=self.device)
+        self.ticks = torch.zeros(NUM_TICKS, 2, dtype=torch.int64, device=self.device)
         d = Debug(kernel_ticks=self.ticks.data_ptr())
         _check(lib().vattn_set_debug(self._h, C.byref(d)), "vattn_set_debug")
         self.reset_kernel_ticks()

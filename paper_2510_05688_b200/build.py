@@ -21,8 +21,9 @@ LIB = os.path.join(PKG, "libvattn.so")
 STAMP = os.path.join(PKG, "libvattn.stamp")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-              "-Xcompiler", "-fPIC", "-shared", "--use_fast_math=false"]
-NVCC_FLAGS = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC", "-shared"]
+# extra -D definitions for measurement builds, e.g. VATTN_DEFINES="VATTN_PHASE_TICKS" (more device-side time stamps)
+NVCC_FLAGS += ["-D" + d for d in os.environ.get("VATTN_DEFINES", "").split() if d]
 
 
 def _nvcc() -> str:
@@ -43,6 +44,7 @@ def _digest() -> str:
     for f in files:
         h.update(f.encode())
         h.update(open(f, "rb").read())
+    h.update(os.environ.get("VATTN_DEFINES", "").encode())
     return h.hexdigest()
 
 

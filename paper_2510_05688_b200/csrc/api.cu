@@ -19,10 +19,10 @@ struct vattn_plan {
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
   int prof_calls;           // calls recorded since the last read
   // derived
-  int G, npad, nwords, stat_splits, stat_splits_base, dense_splits;
-  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_topk, off_base, off_dyn, off_meta, off_stat,
-      off_det, off_piv, off_gat, off_dense, off_cand, off_sort, total;
-  int cand_cap, gat_slots;
+  int G, npad, nwords, dense_splits;
+  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_dyn, off_meta, off_stat,
+      off_piv, off_gat, off_dense, total;
+  int splits;                  // CTAs per head of the row kernels
   // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
   struct HostStep {
     bool used, pinned, mapped;
@@ -42,9 +42,6 @@ struct vattn_plan {
 
 namespace {
 
-constexpr int kNumSM = 148;          // B200; the library is built for sm_100a only
-constexpr int kMaxStatSplits = 16;    // split CTAs per head and row kind of the statistics kernel
-constexpr int kMaxGatherSplits = 32;  // split CTAs per head of the gather kernel
 constexpr int kProfCalls = 256;      // calls whose events are kept between two reads of the profile
 constexpr int kProfEvents = VATTN_NUM_KERNELS + 1;
 
@@ -80,54 +77,34 @@ void derive(vattn_plan* pl) {
   if (pl->npad == 0) pl->npad = 32;
   pl->nwords = pl->npad / 32;
   const int heads = s.batch * s.num_q_heads;
-  // statistics kernel (128-thread CTAs, 5 per SM): one wave for both kinds of CTA.  The base-sample rows are
-  // on the step's critical path (they wait for the sample), the deterministic rows start earlier: three
-  // fifths of the wave go to the former (14 + 9 CTAs per head at 32 heads; 11 + 11 made the step 2 us longer,
-  // 16 + 7 left the deterministic CTAs as the last to finish).  (When even four CTAs per kind and head
-  // overfill the wave the kernel is throughput-bound: split freely.)
-  const int wave = (5 * kNumSM) / heads;
-  if (wave < 8) {
-    pl->stat_splits = pl->stat_splits_base = 4;
-  } else {
-    const int sb = (3 * wave + 2) / 5;
-    pl->stat_splits_base = sb > kMaxStatSplits ? kMaxStatSplits : sb;
-    const int sd = wave - pl->stat_splits_base;
-    pl->stat_splits = sd < 4 ? 4 : (sd > kMaxStatSplits ? kMaxStatSplits : sd);
-  }
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
-  const int sp = (4 * kNumSM + groups - 1) / groups;
+  const int sp = (4 * device_sm_count() + groups - 1) / groups;
   pl->dense_splits = sp < 1 ? 1 : (sp > 128 ? 128 : sp);
+  // row kernels: two CTAs of 8 warps per SM, shared evenly by the heads
+  {
+    const int sp2 = (2 * device_sm_count()) / heads;
+    pl->splits = sp2 < 1 ? 1 : (sp2 > VATTN_MAX_SPLITS ? VATTN_MAX_SPLITS : sp2);
+  }
   const size_t BH = (size_t)heads, D = (size_t)s.head_dim;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   pl->off_scores = take(BH * pl->npad * sizeof(float));
-  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 2 * BH + 4) * sizeof(unsigned);
+  // cleared every step: running maxima [BH], max |K| [B*Hkv], tickets [3*BH], the score kernel's unit counter
+  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 4) * sizeof(unsigned);
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
+  pl->off_vtab = take(BH * VATTN_BANDCAP * sizeof(int));
   pl->off_topk = take(2 * BH * pl->npad * sizeof(int));     // token indices, then physical slots
   pl->off_base = take(2 * BH * pl->npad * sizeof(int));
-  pl->off_dyn = take(2 * BH * pl->npad * sizeof(int));
+  pl->off_walk = take(2 * BH * pl->npad * sizeof(int));     // tokens of the first walk positions, both walks
+  pl->off_dyn = take(3 * BH * pl->npad * sizeof(int));      // tokens, physical slots, score bits
   pl->off_meta = take(BH * sizeof(HeadMeta));
-  pl->off_stat = take(BH * 2 * kMaxStatSplits * (D + 3) * sizeof(double));
-  pl->off_det = take(BH * (D + 1) * sizeof(double));
+  pl->off_stat = take(BH * (size_t)pl->splits * 2 * (D + 3) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
-  // partial slots (chunks) per head of the gather kernel: 32, except that a handful of heads may use more of
-  // the 8 x 148 CTAs (64 to 128 chunks each when that many fit the grid at once)
-  {
-    const size_t fit = (size_t)(8 * kNumSM) / BH;
-    const size_t flat = fit >= 2 * VATTN_GATHER_FLAT_SLOTS ? (fit > 128 ? 128 : fit) : VATTN_GATHER_FLAT_SLOTS;
-    pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? (int)flat : kMaxGatherSplits;
-  }
-  pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
+  pl->off_gat = take(BH * (size_t)pl->splits * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
-  {
-    const double q4 = 0.25 * (double)pl->npad;
-    pl->cand_cap = ((int)(q4 + 8.0 * sqrt(q4) + 64.0) + 31) / 32 * 32;
-  }
-  pl->off_cand = take(2 * BH * (size_t)pl->cand_cap * sizeof(uint2));
-  pl->off_sort = take(2 * BH * (size_t)pl->cand_cap * sizeof(int));       // sorted tokens, then physical slots
   pl->total = off;
 }
 
@@ -151,31 +128,27 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.mode = pr.mode; p.layer = pr.layer; p.step = pr.step; p.rng_head_is_kv = pr.rng_head_is_kv;
   p.gather_kv = pr.gather_mode == 1;
   p.force_budget = (pr.force_budget_on || pr.force_budget > 0) ? (pr.force_budget < 0 ? -1 : pr.force_budget) : -1;
+  p.nested_base = pr.nested_base ? 1 : 0;
   unsigned char* w = static_cast<unsigned char*>(pl->ws);
   p.scores = reinterpret_cast<float*>(w + pl->off_scores);
   unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
   const size_t BH = (size_t)s.batch * s.num_q_heads;
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
-  p.cand_cnt = p.tickets + 3 * BH;
-  p.unit_ctr = p.cand_cnt + 2 * BH;
-  p.cand = reinterpret_cast<uint2*>(w + pl->off_cand);
-  p.cand_cap = pl->cand_cap;
-  p.sort_idx = reinterpret_cast<int*>(w + pl->off_sort);
-  p.sort_phys_delta = (long long)BH * pl->cand_cap;
+  p.unit_ctr = p.tickets + 3 * BH;
   p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
   p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);
+  p.vtab = reinterpret_cast<int*>(w + pl->off_vtab);
   p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
   p.base_idx = reinterpret_cast<int*>(w + pl->off_base);
+  p.walk_tok = reinterpret_cast<int*>(w + pl->off_walk);
   p.dyn_idx = reinterpret_cast<int*>(w + pl->off_dyn);
-  p.phys_delta = (long long)BH * pl->npad;
   p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
   p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);
-  p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
   p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
-  p.gat_slots = pl->gat_slots;
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
-  p.stat_splits = pl->stat_splits; p.stat_splits_base = pl->stat_splits_base; p.dense_splits = pl->dense_splits;
+  p.dense_splits = pl->dense_splits;
+  p.splits = pl->splits;
   p.dbg = pl->dbg;
   return VATTN_OK;
 }
@@ -201,12 +174,25 @@ int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st, bool with_ker
     CU(cudaMemsetAsync(p.status, 0, sizeof(unsigned), st));
     pl->status_ready = true;
   }
-  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, p.dbg.kernel_ticks, st));
+  // The clearing kernel may run ahead of its stream predecessor only when that is this library's own input
+  // staging kernel; a caller's kernel (a GEMM, RoPE, a KV append that writes what this step reads) is waited for.
+  if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, pl->inputs_just_staged, p.dbg.kernel_ticks, st));
   else CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
   return VATTN_OK;
 }
 
 }  // namespace
+
+int device_sm_count() {
+  static int cached[VATTN_MAXDEV];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= VATTN_MAXDEV) { cudaGetLastError(); return 148; }
+  int n = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { cudaGetLastError(); return 148; }
+  __atomic_store_n(&cached[dev], n, __ATOMIC_RELEASE);
+  return n;
+}
 
 extern "C" {
 
@@ -311,7 +297,7 @@ int vattn_set_params(vattn_plan* plan, const vattn_params* params) {
   const vattn_params& p = *params;
   if (p.base_rate < 0.f || p.base_rate > 1.f || p.topk_frac < 0.f || p.topk_frac > 1.f) return VATTN_ERR_INVALID_ARG;
   if (p.mode < 0 || p.mode > 2 || p.step < 0 || !(p.scale == p.scale) || isinf(p.scale)) return VATTN_ERR_INVALID_ARG;
-  if (p.gather_mode < 0 || p.gather_mode > 1) return VATTN_ERR_INVALID_ARG;
+  if (p.gather_mode < 0 || p.gather_mode > 1 || p.nested_base < 0 || p.nested_base > 1) return VATTN_ERR_INVALID_ARG;
   plan->params = p;
   return VATTN_OK;
 }
@@ -334,20 +320,6 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   Prob p;
   fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
   p.sink = sink; p.window = window; p.k = k;
-  {
-    // statistics kernel: never more CTAs than rows warrant (about 64 deterministic, 48 base-sample rows each)
-    const double msl = (double)plan->shape.max_seq_len;
-    double kmax = plan->params.topk_frac > 0.f ? floor((double)plan->params.topk_frac * msl) : (double)k;
-    double rows = (double)sink + (double)window + kmax;
-    if (rows > msl) rows = msl;
-    int want = (int)((rows + 127.0) / 128.0) * 2;
-    if (want < 1) want = 1;
-    if (want < p.stat_splits) p.stat_splits = want;
-    const double brows = (double)p.base_rate * msl;
-    want = (int)((brows + 95.0) / 96.0) * 2;
-    if (want < 1) want = 1;
-    if (want < p.stat_splits_base) p.stat_splits_base = want;
-  }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;
   p.z_delta = upper_quantile(0.5 * p.delta);
@@ -360,33 +332,26 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   if (rc != VATTN_OK) return rc;
   plan->last_launches++;                      // the counter-clearing kernel
   prof_mark(plan, 0, st);
-  // score || key pre-filter -> top-k || sampling sort -> sampling compaction -> statistics + budget ->
-  // slow-path select (usually nothing to do) -> gather.  The overlaps come from programmatic dependent
-  // launches (see the kernels): the pre-filter runs beside the persistent score kernel, the sort of its
-  // lists beside the top-k select.
+  // score pass (walk tokens beside it) -> selection and sample lists (one CTA per head) -> deterministic and base-sample rows ->
+  // budget, final sample, combination.  Every kernel is launched with programmatic dependent launch: its prologue
+  // runs while its predecessor drains.
   CU(launch_score(p, st));            plan->last_launches++;
   prof_mark(plan, 1, st);
   if (plan->stop_after == 1) return VATTN_OK;
-  CU(launch_cand(p, st));             plan->last_launches++;
-  prof_mark(plan, 2, st);
-  if (plan->stop_after == 2) return VATTN_OK;
   if (p.dbg.scores)
     CU(cudaMemcpy2DAsync(p.dbg.scores, sizeof(float) * (size_t)p.max_seq_len, p.scores, sizeof(float) * (size_t)p.npad,
                          sizeof(float) * (size_t)p.max_seq_len, (size_t)p.B * p.Hq, cudaMemcpyDeviceToDevice, st));
-  CU(launch_select_topk(p, st));      plan->last_launches++;
+  CU(launch_walk(p, st));             plan->last_launches++;
+  prof_mark(plan, 2, st);
+  if (plan->stop_after == 2) return VATTN_OK;
+  CU(launch_select(p, st));           plan->last_launches++;
   prof_mark(plan, 3, st);
   if (plan->stop_after == 3) return VATTN_OK;
-  CU(launch_presort(p, st));          plan->last_launches++;
+  CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 4, st);
   if (plan->stop_after == 4) return VATTN_OK;
-  CU(launch_stats(p, st));            plan->last_launches++;
+  CU(launch_final(p, st));            plan->last_launches++;
   prof_mark(plan, 5, st);
-  if (plan->stop_after == 5) return VATTN_OK;
-  CU(launch_budget(p, st));     plan->last_launches++;
-  prof_mark(plan, 6, st);
-  if (plan->stop_after == 6) return VATTN_OK;
-  CU(launch_gather(p, st));           plan->last_launches++;
-  prof_mark(plan, 7, st);
   if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
   return VATTN_OK;
 }

@@ -442,15 +442,12 @@ static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
   const size_t ring = (size_t)DN_WARPS * DN_NST * STAGE;
   const size_t accb = (size_t)DN_WARPS * 8 * D * sizeof(float);
   const size_t smem = (ring > accb ? ring : accb) + DN_WARPS * DN_NST * 8;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_dense_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static size_t have[VATTN_MAXDEV];
+  cudaError_t e = optin_smem(k_dense_mma<D>, smem, have);
+  if (e != cudaSuccess) return e;
   const int GC = (p.G + 7) / 8;
   const int groups = p.B * p.Hkv * GC;
-  int S = (2 * 148 + groups - 1) / groups;               // one wave of two CTAs per SM (registers and shared memory)
+  int S = (2 * device_sm_count() + groups - 1) / groups;               // one wave of two CTAs per SM (registers and shared memory)
   if (S > p.dense_splits) S = p.dense_splits;
   if (S < 1) S = 1;
   dim3 grid(S, p.Hkv * GC, p.B), block(DN_WARPS * 32);
@@ -530,7 +527,7 @@ extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale,
   const int G = s.num_q_heads / s.num_kv_heads, GC = (G + 3) / 4;
   const size_t groups = (size_t)s.batch * s.num_kv_heads * GC;
   const size_t head_bytes = 256 + up256(3 * BH * sizeof(unsigned));
-  int splits = (int)((4 * 148 + groups - 1) / groups);
+  int splits = (int)((4 * (size_t)device_sm_count() + groups - 1) / groups);
   splits = splits < 1 ? 1 : (splits > 128 ? 128 : splits);
   while (splits > 1 && head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES) --splits;
   if (head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES)

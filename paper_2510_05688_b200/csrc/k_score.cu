@@ -406,27 +406,29 @@ static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
   const size_t smem = (size_t)S * PAGEB + (size_t)S * qslot_bytes + (size_t)S * sizeof(StageMeta) + (size_t)2 * S * 8 +
                       sizeof(int) * ((size_t)2 * p.B + 1 + 16);
   if (smem > 113 * 1024) return cudaErrorInvalidValue;        // two CTAs per SM (plan creation bounds the batch)
-  static size_t attr_sz = 0;
-  if (attr_sz < smem) {
-    cudaError_t e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_score_stream<D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    attr_sz = smem;
-  }
+  static size_t have[VATTN_MAXDEV];
+  cudaError_t e = optin_smem(k_score_stream<D>, smem, have, true);
+  if (e != cudaSuccess) return e;
   // persistent: two CTAs per SM, fewer when the problem cannot have that many units
   const long long pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
   const long long units_max = (long long)p.B * p.Hkv * ((p.G + 7) / 8) * ((pages + MIN_UNIT_PAGES - 1) / MIN_UNIT_PAGES);
-  const int grid = (int)(units_max < 2 * 148 ? (units_max < 1 ? 1 : units_max) : 2 * 148);
+  const int slots = 2 * device_sm_count();
+  const int grid = (int)(units_max < slots ? (units_max < 1 ? 1 : units_max) : slots);
   return launch_pdl(k_score_stream<D>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
 }
 
-cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, unsigned long long* ticks, cudaStream_t s) {
+// `pdl`: launch with the programmatic-serialization attribute, i.e. let this grid start while the kernel before it
+// in the stream still runs.  Only sound when that kernel is one of this library's own (it then has no stores
+// left that the step reads once its CTAs have let their dependents go); against a caller's kernel the launch
+// is an ordinary one.
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool pdl, bool late, unsigned long long* ticks, cudaStream_t s) {
   const int words = (int)(bytes / sizeof(unsigned));
   int grid = (words + 1023) / 1024;
   if (grid > 148) grid = 148;
   if (grid < 1) grid = 1;
-  return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words, late ? 1 : 0, ticks);
+  if (pdl) return launch_pdl(k_zero, dim3(grid), dim3(256), 0, s, z, words, late ? 1 : 0, ticks);
+  k_zero<<<grid, 256, 0, s>>>(z, words, 1, ticks);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_score(const Prob& p, cudaStream_t s) {

@@ -5,26 +5,29 @@
 #include "vattn.h"
 
 #define VATTN_BLOCK 16                 // tokens per KV page
-#define VATTN_MAX_SEQ (1 << 18)        // longest sequence the select kernels' shared-memory bitmaps hold
-#define VATTN_KEYCACHE_MAX 40960       // tokens whose 32-bit select keys are cached in shared memory
-#define VATTN_BANDCAP 1024             // near-tie top-k candidates rescored by the fast path
-#define SEL_THREADS 1024
-#define ROW_THREADS 256
+#define VATTN_MAX_SEQ (1 << 18)        // longest sequence a plan accepts
+#define VATTN_BANDCAP 1024             // near-tie top-k candidates ranked from a list (more: exact radix select)
+#define SEL_THREADS 1024               // threads of the selection kernel (one CTA per head)
+#define ROW_THREADS 256                // threads of the row kernels
+#define VATTN_MAX_SPLITS 16            // most CTAs per head of the row kernels
 
-// Per (batch row, query head) bookkeeping, written by the select kernel and completed by the
-// statistics kernel.
+// Per (batch row, query head) record, written by the selection kernel for the row kernels.
 struct HeadMeta {
-  int n;         // tokens in the sequence (clamped to [0, max_seq_len])
-  int s0;        // |I_s| = min(sink, n)
-  int l_start;   // first token of the local window; middle range M = [s0, l_start)
-  int kk;        // |I_t| = min(k, |M|)
-  int n_s;       // residual size |M| - kk
-  int b0;        // base-sample size
-  int b;         // final budget |I_dyn|
-  int sorted_cnt; // entries of the pre-sorted stream-1 residual list (-1: list unusable)
-  float m;       // largest fp32 score of the head (softmax stabiliser)
-  float gamma;   // bound on |fp32 score - exact score| for this head
-  int pad1, pad2;
+  int n;            // tokens in the sequence (clamped to [0, max_seq_len])
+  int s0;           // |I_s| = min(sink, n)
+  int l_start;      // first token of the local window; middle range M = [s0, l_start)
+  int kk;           // |I_t| = min(k, |M|)
+  int n_s;          // residual size |M| - kk
+  int b0;           // base-sample size
+  int nbt;          // near-tie tokens of the top-k threshold (listed in vtab unless band_mode is set)
+  int band_mode;    // 1: the near-ties were too many for the list; their verdicts are bits of the bitmap
+  float m;          // largest fp32 score of the head (softmax stabiliser)
+  float hi, lo;     // a middle token is in I_t if its score is above hi; scores in [lo, hi] are near-ties
+  int run1;         // the list of I_t is two ascending runs: [0, run1) and [run1, kk)
+  int dyn_listed;   // residual tokens of the final sample's walk that the selection kernel listed ...
+  int dyn_J;        // ... and the walk positions they cover
+  int path;         // code path of the selection (vattn_debug.paths)
+  int pad;
 };
 
 // Everything a kernel needs, passed by value.
@@ -36,7 +39,8 @@ struct Prob {
   int sink, window, k;
   float topk_frac, base_rate, scale;
   int mode, layer, step, rng_head_is_kv, force_budget;       // force_budget < 0: off
-  int gather_kv;          // 1: the gather kernel recomputes the weights of the sampled tokens from their K rows
+  int nested_base;        // 1: the base sample is the head of the final sample's walk
+  int gather_kv;          // 1: the weights of the sampled tokens are recomputed from their K rows
   unsigned seed_lo, seed_hi;
   double eps, delta, z_delta;
   double z1[15], z2[15];                                     // z(delta*j/16), z(delta*(16-j)/16), j = 1..15
@@ -44,27 +48,24 @@ struct Prob {
   float* scores;          // [B,Hq,npad]
   unsigned* m_ord;        // [B,Hq]  order-preserving encoding of the running max score
   unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
-  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters (stats, gather, dense)
-  unsigned* cand_cnt;     // [2,B,Hq] entries appended to the sampling-candidate lists (may exceed cand_cap)
   unsigned* unit_ctr;     // [1] work-unit counter of the persistent score kernel
-  uint2* cand;            // [2,B,Hq,cand_cap] (Philox key, token) with key below the stream's pre-filter
-  int cand_cap;
+  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters: [1] final sample, [2] dense kernel
   unsigned* status;       // [1]
-  unsigned* bitmap;       // [B,Hq,nwords] membership of I_t
-  int* topk_idx;          // [B,Hq,npad] token indices, ascending; the list of physical slots
-  int* base_idx;          // [B,Hq,npad]   (page * 16 + token % 16 of every entry) lies phys_delta
-  int* dyn_idx;           // [B,Hq,npad]   elements behind each index list
-  long long phys_delta;
-  int* sort_idx;          // [B,Hq,cand_cap] residual stream-1 candidates sorted by (key, token); physical slots
-  long long sort_phys_delta;  //   lie sort_phys_delta elements behind
+  unsigned* bitmap;       // [B,Hq,nwords] near-tie tokens that made it into I_t (used when they are too many for a list)
+  int* vtab;              // [B,Hq,BANDCAP] near-tie tokens ascending, bit 31 = member of I_t
+  int* topk_idx;          // [B,Hq,2,npad] I_t as two ascending runs, then the physical slot (page * 16 + token % 16) of
+                          //               every entry
+  int* base_idx;          // [B,Hq,2,npad] I_bs in walk order: tokens, physical slots
+  int* walk_tok;          // [B,Hq,2,npad] tokens of the first walk positions of both walks (computed beside the score pass)
+  int* dyn_idx;           // [B,Hq,3,npad] head of the final sample's walk: tokens, physical slots, fp32 score bits
+                          //               (scratch of the near-tie overflow path while the selection runs)
   HeadMeta* meta;         // [B,Hq]
-  double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (det CTAs, then base CTAs)
-  double* det_sums;       // [B,Hq,D+1]  N_f then D_f
-  double* stat_piv;       // [B,Hq,D+1]  pivot row of the base-sample statistics: w*V then w
-  float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
-  int gat_slots;          // partial slots (chunks) per head: 32; 64 to 128 when at most 18 heads share the grid
+  double* stat_part;      // [B,Hq,splits,2,D+3] sums of the statistics kernel: deterministic rows, base-sample rows
+  double* stat_piv;       // [B,Hq,D+1] pivot row of the base-sample sums: w*V then w
+  float* gat_part;        // [B,Hq,splits,D+1] sums of the final sample
   float* dense_part;      // [B,Hq,dense_splits,D+2]
-  int stat_splits, stat_splits_base, dense_splits;   // statistics CTAs per head: deterministic rows, base-sample rows
+  int dense_splits;
+  int splits;             // CTAs per head of the row kernels
   vattn_debug dbg;
 };
 
@@ -75,15 +76,15 @@ __device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t;
 #define TICK_BEGIN(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMin((p).dbg.kernel_ticks + 2 * (k), gtime_ns()); } while (0)
 #define TICK_END(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
 #define TICK_END_IF(p, k, cond) do { if ((p).dbg.kernel_ticks && (cond)) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
-// kernel numbers
+// rows of kernel_ticks
 #define VATTN_K_ZERO 0
 #define VATTN_K_SCORE 1
-#define VATTN_K_CAND 2
-#define VATTN_K_TOPK 3
-#define VATTN_K_PRESORT 4
-#define VATTN_K_STATS 5
-#define VATTN_K_BUDGET 6
-#define VATTN_K_GATHER 7
+#define VATTN_K_WALK 2
+#define VATTN_K_SELECT 3
+#define VATTN_K_STATS 4
+#define VATTN_K_FINAL 5
+#define VATTN_T_TOPK 6       // [0]: first selection CTA past its dependency wait, [1]: last CTA with I_t complete
+#define VATTN_T_BUDGET 7     // [0]: first final-sample CTA past its dependency wait, [1]: last CTA that knows its budget
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
 // stream is still running; it must call pdl_wait() before touching anything the predecessor writes (the
@@ -184,20 +185,7 @@ __device__ __forceinline__ Geo head_geometry(const Prob& p, int n) {
   if (g.n_s > 0) g.b0 = min(g.n_s, max(2, (int)floor((double)p.base_rate * (double)g.n_s)));
   return g;
 }
-// Pre-filters of the sampling-candidate lists: a token is a candidate of stream s when its Philox key
-// is below this bound.  Stream 1 keeps a quarter of the tokens; stream 0 keeps b0 + 6 sqrt(b0) + 16
-// expected tokens (none if that is more than a quarter: the select kernel then draws without the list).
-#define VATTN_CAND1_BOUND 0x40000000u
 #define VATTN_MAX_BATCH_BF16 1536     // batch rows a bf16 plan accepts (12 bytes of shared memory per row in k_score)
-#define VATTN_STAT_MAXS 16            // most split CTAs per head and row kind of the statistics kernel
-#define VATTN_GATHER_FLAT_HEADS 128   // the gather kernel's flat decomposition serves up to this many heads ...
-#define VATTN_GATHER_FLAT_SLOTS 32   // ... with up to this many chunks (partials) each
-__device__ __forceinline__ unsigned cand0_bound(const Geo& g) {
-  if (g.n_s <= 0 || g.b0 <= 0) return 0u;
-  const double want = (double)g.b0 + 6.0 * sqrt((double)g.b0) + 16.0;
-  const double frac = want / (double)g.n_s;
-  return frac > 0.25 ? 0u : (unsigned)(frac * 4294967296.0);
-}
 
 // Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0,k1)
 __device__ __forceinline__ uint4 philox4x32_10(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
@@ -212,6 +200,74 @@ __device__ __forceinline__ uint4 philox4x32_10(unsigned c0, unsigned c1, unsigne
     k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
   }
   return make_uint4(c0, c1, c2, c3);
+}
+
+// ---------------------------------------------------------------------------------------------
+// uniform-sample (Algorithm 1 line 7, Algorithm 2 line 1) = the first c residual tokens met when the middle range
+// is walked in the order s0 + sigma(0), s0 + sigma(1), ...; sigma is a keyed permutation of [0, mlen): an 8-round
+// alternating Feistel network on the smallest domain 2^w >= mlen (w >= 2) with cycle walking.  Round keys: the
+// eight words of Philox4x32-10(key = seed, counter = (c, batch << 16 | head, layer, step << 1 | stream)), c = 0, 1.
+__device__ __forceinline__ unsigned mix32(unsigned x, unsigned key) {
+  unsigned v = (x ^ key) * 0x9E3779B1u;
+  v ^= v >> 15; v *= 0x85EBCA77u;
+  v ^= v >> 13; v *= 0xC2B2AE3Du;
+  v ^= v >> 16;
+  return v;
+}
+struct Walk { unsigned k[8]; int lw, rw; unsigned mlen; };
+__device__ __forceinline__ Walk make_walk(const unsigned* keys, int mlen) {
+  Walk w;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w.k[i] = keys[i];
+  const int wbits = max(2, 32 - __clz(max(mlen - 1, 0)));
+  w.lw = wbits >> 1; w.rw = wbits - w.lw; w.mlen = (unsigned)max(mlen, 1);
+  return w;
+}
+__device__ __forceinline__ int walk_at(const Walk& w, int j) {
+  const unsigned ml = (1u << w.lw) - 1u, mr = (1u << w.rw) - 1u;
+  unsigned x = (unsigned)j;
+  do {
+    unsigned L = x >> w.rw, R = x & mr;
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      L ^= mix32(R, w.k[i]) & ml;
+      R ^= mix32(L, w.k[i + 1]) & mr;
+    }
+    x = (L << w.rw) | R;
+  } while (x >= w.mlen);
+  return (int)x;
+}
+// Walk positions expected to hold the first `want` residual tokens, with a margin of four standard deviations
+// (the selection kernel walks on if the margin was not enough).
+__device__ __forceinline__ int walk_region(int want, int n_s, int mlen, int kk) {
+  if (want <= 0 || n_s <= 0) return 0;
+  if (want >= n_s) return mlen;
+  const double miss = (double)want * (double)mlen / (double)n_s;
+  const long long span = (long long)(miss + 4.0 * sqrt(miss * (double)kk / (double)mlen + 1.0) + 8.0);
+  return (int)(span < (long long)mlen ? span : (long long)mlen);
+}
+// residual tokens of the final sample's walk that are listed ahead of the budget: eight base budgets (budgets beyond
+// that make the final-sample kernel walk on), or the forced budget
+__device__ __forceinline__ int dyn_listed_want(const Prob& p, int n_s, int b0) {
+  if (n_s <= 0) return 0;
+  return min(n_s, p.force_budget >= 0 ? p.force_budget : 8 * b0);
+}
+// round keys of one (batch row, head, stream) into keys[0..8): two threads, one Philox call each
+__device__ __forceinline__ void walk_keys(const Prob& p, int b, int hrng, int stream, int half, unsigned* keys) {
+  const uint4 w4 = philox4x32_10((unsigned)half, ((unsigned)b << 16) | (unsigned)hrng, (unsigned)p.layer,
+                                 ((unsigned)p.step << 1) | (unsigned)stream, p.seed_lo, p.seed_hi);
+  keys[half * 4 + 0] = w4.x; keys[half * 4 + 1] = w4.y; keys[half * 4 + 2] = w4.z; keys[half * 4 + 3] = w4.w;
+}
+// is middle token `tok` (fp32 score s) a member of I_t?  vt: the head's near-tie list (shared or global memory)
+__device__ __forceinline__ bool in_topk(const HeadMeta& mt, const int* vt, const unsigned* bitmap, int tok, float s) {
+  if (s > mt.hi) return true;
+  if (!(s >= mt.lo)) return false;
+  if (mt.band_mode) return (__ldcg(bitmap + (tok >> 5)) >> (tok & 31)) & 1u;
+  for (int c = 0; c < mt.nbt; ++c) {
+    const int e = vt[c];
+    if ((e & 0x7FFFFFFF) == tok) return e < 0;
+  }
+  return false;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -264,23 +320,34 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], unsigned a0, unsig
 }
 
 
-// HeadMeta through L2 (ld.cg): for kernels that are let loose before their stream predecessor has
-// finished and therefore cannot count on the launch-boundary L1 invalidation.
-static_assert(sizeof(HeadMeta) == 48, "HeadMeta is read as three 16-byte words");
-__device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
-  union { HeadMeta m; int4 v[3]; } u;
-  const int4* src = reinterpret_cast<const int4*>(g);
-  u.v[0] = __ldcg(src); u.v[1] = __ldcg(src + 1); u.v[2] = __ldcg(src + 2);
-  return u.m;
+// The opt-in to more than 48 KB of dynamic shared memory (and the carve-out preference) is a property of a
+// kernel in ONE device's context: it is made once per device ordinal (`have` = bytes already granted there).
+constexpr int VATTN_MAXDEV = 64;
+template <typename KernelT>
+inline cudaError_t optin_smem(KernelT kern, size_t smem, size_t* have, bool prefer_max_carveout = false) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= VATTN_MAXDEV) return cudaErrorInvalidDevice;
+  if (__atomic_load_n(&have[dev], __ATOMIC_ACQUIRE) >= smem + 1) return cudaSuccess;
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  if (prefer_max_carveout) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+  }
+  __atomic_store_n(&have[dev], smem + 1, __ATOMIC_RELEASE);
+  return cudaSuccess;
 }
 
 // launchers (one per translation unit)
-cudaError_t launch_zero(unsigned* z, size_t bytes, bool late, unsigned long long* ticks, cudaStream_t s);
+cudaError_t launch_zero(unsigned* z, size_t bytes, bool pdl, bool late, unsigned long long* ticks, cudaStream_t s);
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
-cudaError_t launch_cand(const Prob& p, cudaStream_t s);
-cudaError_t launch_select_topk(const Prob& p, cudaStream_t s);
-cudaError_t launch_presort(const Prob& p, cudaStream_t s);
-cudaError_t launch_budget(const Prob& p, cudaStream_t s);
+cudaError_t launch_walk(const Prob& p, cudaStream_t s);
+cudaError_t launch_select(const Prob& p, cudaStream_t s);
 cudaError_t launch_stats(const Prob& p, cudaStream_t s);
-cudaError_t launch_gather(const Prob& p, cudaStream_t s);
+cudaError_t launch_final(const Prob& p, cudaStream_t s);
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches);
+int device_sm_count();                                   // SMs of the current device (cached per device)

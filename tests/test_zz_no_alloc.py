@@ -4,12 +4,14 @@ A serving engine that gave the whole GPU to its KV-cache pool, or code that must
 its path, cannot create a plan workspace.  vattn_dense_decode_noalloc keeps its scratch in a fixed array
 inside the library instead.  This test calls it through the C ABI twice in a row (the array keeps the
 previous call's contents, so the second call proves the clearing) and compares each result with the
-ordinary entry point, within the tolerance the dense parity test uses.  It lives in a file pytest
-collects last, so a failure here cannot hide any other test under -x.
+ordinary entry point and with the CPU reference of dense attention, within the tolerance the dense
+parity test uses.  It lives in a file pytest collects last, so a failure here cannot hide any other
+test under -x.
 """
 import numpy as np
 import pytest
 
+from oracle import vattn_oracle as O
 from paper_2510_05688_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +32,7 @@ def test_noalloc_dense_matches_planned_dense_on_two_calls_in_a_row():
         plan = vb.plan_for_case(case)
         ref = torch.empty_like(dev["q"])
         plan.dense_decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], ref)
+        cpu = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=case.dtype)
         for call in range(2):
             out = torch.full_like(dev["q"], 7.0)
             rc = vb.dense_decode_noalloc(plan.shape, dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"],
@@ -39,6 +42,7 @@ def test_noalloc_dense_matches_planned_dense_on_two_calls_in_a_row():
             a, b = out.float().cpu().numpy().astype(np.float64), ref.float().cpu().numpy().astype(np.float64)
             tol = 2e-2 if case.dtype == "bf16" else 2e-5
             assert (np.abs(a - b) <= tol * np.maximum(1.0, np.abs(b))).all(), (case.dtype, call, np.abs(a - b).max())
+            assert (np.abs(a - cpu) <= tol * np.maximum(1.0, np.abs(cpu))).all(), (case.dtype, call, np.abs(a - cpu).max())
 
 
 def test_noalloc_rejects_problems_beyond_the_fixed_scratch():
