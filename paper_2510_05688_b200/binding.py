@@ -22,7 +22,7 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
 KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_final"]
-NUM_TICKS = 32
+NUM_TICKS = 8
 TICK_NAMES = ["k_zero", "k_score", "k_walk", "k_select", "k_stats", "k_final", "topk", "budget"]
 
 

@@ -21,8 +21,8 @@ struct vattn_plan {
   // derived
   int G, npad, nwords, dense_splits;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_dyn, off_meta, off_stat,
-      off_piv, off_gat, off_dense, total;
-  int splits;                  // CTAs per head of the row kernels
+      off_piv, off_det, off_budget, off_gat, off_dense, total;
+  int splits, gat_slots;                  // CTAs per head of the row kernels
   // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
   struct HostStep {
     bool used, pinned, mapped;
@@ -103,7 +103,11 @@ void derive(vattn_plan* pl) {
   pl->off_meta = take(BH * sizeof(HeadMeta));
   pl->off_stat = take(BH * (size_t)pl->splits * 2 * (D + 3) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
-  pl->off_gat = take(BH * (size_t)pl->splits * (D + 1) * sizeof(float));
+  pl->off_det = take(BH * (D + 1) * sizeof(double));
+  pl->off_budget = take(BH * sizeof(int));
+  // partial slots of the final sample per head: up to 32 units of listed rows, plus one per CTA of the head
+  pl->gat_slots = 32 + pl->splits;
+  pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
   pl->total = off;
 }
@@ -145,7 +149,10 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
   p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);
   p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
+  p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
+  p.budget = reinterpret_cast<int*>(w + pl->off_budget);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
+  p.gat_slots = pl->gat_slots;
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.dense_splits = pl->dense_splits;
   p.splits = pl->splits;

@@ -6,8 +6,9 @@
 //           budget is fp64, so that the same inputs give the same ceil() as a plain fp64 evaluation.  Variances
 //           are accumulated around a pivot (the first base-sample row), which removes the cancellation of the
 //           one-pass formula and makes a constant population give exactly 0.
-//  k_final  the budget b_D, b_N (Corollaries D.2), b_SDPA (Theorem 4.3), b = clamp(ceil(b_X), b0, n_s), evaluated
-//           by every CTA of the head from the statistics' partial sums; then the sampled part of the estimator
+//           The last CTA of a head to finish adds the head's partial sums in a fixed order and evaluates the budget
+//           b_D, b_N (Corollaries D.2), b_SDPA (Theorem 4.3), b = clamp(ceil(b_X), b0, n_s).
+//  k_final  the sampled part of the estimator
 //               N = N_f + (n_s/b) sum_{I_dyn} w_i V[i],   D = D_f + (n_s/b) sum_{I_dyn} w_i,   out = N / D
 //           (Sec. 4.1; SDPA_{S,p} of Sec. 3 with p = 1 on I_f and p = b/n_s on I_dyn).  I_dyn = the first b residual
 //           tokens of the final sample's walk: the part the selection kernel listed, and, for larger budgets,
@@ -21,7 +22,7 @@
 #include <math_constants.h>
 
 #ifdef VATTN_PHASE_TICKS
-#define DBGT(k) do { TICK_BEGIN(p, 28 + (k)); TICK_END(p, 28 + (k)); } while (0)
+#define DBGT(k) do { TICK_BEGIN(p, 24 + (k)); TICK_END(p, 24 + (k)); } while (0)
 #else
 #define DBGT(k) do { } while (0)
 #endif
@@ -168,10 +169,19 @@ __global__ void __launch_bounds__(NT, 2) k_stats(const Prob p) {
   __syncthreads();
   pdl_wait();                                          // the selection kernel is complete: lists, meta
   pdl_trigger();
+  DBGT(0);
   const HeadMeta mt = p.meta[bh];
   const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, b0 = mt.b0;
   double* gpart = p.stat_part + ((long long)bh * S + s) * 2 * NE;
-  if (n == 0) return;
+  if (n == 0) {
+    if (s == 0 && tid == 0) {
+      p.budget[bh] = 0;
+      if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = 0;
+      if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
+      if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
+    }
+    return;
+  }
   const int n_f = s0 + kk + (n - l_start);
   const int* tkph = p.topk_idx + (long long)bh * 2 * p.npad + p.npad;      // physical slots of I_t
   const int* bsph = p.base_idx + (long long)bh * 2 * p.npad + p.npad;      // physical slots of I_bs
@@ -192,25 +202,36 @@ __global__ void __launch_bounds__(NT, 2) k_stats(const Prob p) {
   const int rsub = lane / LPR, j = lane % LPR;
   const double* qs = qT + j;
   const double md = (double)mt.m;
+  // The warps of a CTA are split between the two kinds of rows in proportion to their numbers, so that both kinds
+  // stream at the same time (a warp's batches follow each other through its two-stage ring; fewer, longer chains
+  // beat two rounds that each pay the first fetch).  Warps [0, wd) take the deterministic rows (sink, I_t, window),
+  // warps [wd, 8) the base sample.
+  int wd = NWARP;
+  if (b0 > 0) {
+    wd = (NWARP * n_f + (n_f + b0) / 2) / (n_f + b0);
+    wd = wd < 1 ? 1 : (wd > NWARP - 1 ? NWARP - 1 : wd);
+  }
+  const bool base_w = warp >= wd;
+  const int total = base_w ? b0 : n_f;
+  const int GWk = S * (base_w ? NWARP - wd : wd), gwk = s * (base_w ? NWARP - wd : wd) + (base_w ? warp - wd : warp);
 
   double acc[EPL], s1 = 0.0, s2 = 0.0, s3 = 0.0;
-  double cw = 0.0, pv[EPL];                            // pivot; zero while the deterministic rows are added
+  double cw = 0.0, pv[EPL];                            // pivot of the base-sample sums; zero for the deterministic rows
 #pragma unroll
   for (int e = 0; e < EPL; ++e) { acc[e] = 0.0; pv[e] = 0.0; }
+  bool have_piv = !base_w;
 
-#pragma unroll 1
-  for (int round = 0; round < 2; ++round) {            // 0: deterministic rows (sink, I_t, window), 1: base sample
-    const int total = round == 0 ? n_f : b0;
+  {
     const int nbat_all = (total + RB - 1) / RB;
-    int beta = gw;                                     // this warp's batches: beta, beta + GW, ...
+    int beta = gwk;                                    // this warp's batches: beta, beta + GWk, ...
 #pragma unroll 1
     while (beta < nbat_all) {
       int cnt = 0;
-      for (int q_ = 0; q_ < WL / RB && beta < nbat_all; ++q_, beta += GW) {
+      for (int q_ = 0; q_ < WL / RB && beta < nbat_all; ++q_, beta += GWk) {
         const int rho = beta * RB + lane;
         if (lane < RB && rho < total) {
           int ph;
-          if (round == 1) ph = bsph[rho];
+          if (base_w) ph = bsph[rho];
           else if (rho < s0) ph = page_of(p, b, rho >> 4) * VATTN_BLOCK + (rho & 15);
           else if (rho < s0 + kk) ph = tkph[rho - s0];
           else { const int t2 = l_start + (rho - s0 - kk); ph = page_of(p, b, t2 >> 4) * VATTN_BLOCK + (t2 & 15); }
@@ -221,9 +242,32 @@ __global__ void __launch_bounds__(NT, 2) k_stats(const Prob p) {
       __syncwarp();
       const int nbat = (cnt + RB - 1) / RB;
       R_::template issue<true>(p, rg, g, lph, min(RB, cnt));
+      if (nbat > 1) R_::template issue<true>(p, rg, g, lph + RB, min(RB, cnt - RB));
+      if (!have_piv) {
+        // the pivot: every row group of the base warps evaluates it from the rows requested above (identical numbers)
+        const bool ok = __all_sync(FULL, mbar_wait(&bars[NWARP * 2], 0u));
+        if (!ok && lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+        Raw<T> kr, vr;
+        kr.ld(pivrow + j * 16);
+        vr.ld(pivrow + RWB + j * 16);
+        double dd = 0.0;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) dd = fma(qs[e * LPR], (double)kr.get(e), dd);
+#pragma unroll
+        for (int mask = LPR / 2; mask >= 1; mask >>= 1) dd += __shfl_xor_sync(FULL, dd, mask);
+        cw = exp(dd * (double)p.scale - md);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) pv[e] = cw * (double)vr.get(e);
+        if (s == 0 && warp == wd && rsub == 0) {
+          double* gp = p.stat_piv + (long long)bh * (D + 1);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) gp[j * EPL + e] = pv[e];
+          if (j == 0) gp[D] = cw;
+        }
+        have_piv = true;
+      }
 #pragma unroll 1
       for (int k = 0; k < nbat; ++k) {
-        if (k + 1 < nbat) R_::template issue<true>(p, rg, g, lph + (k + 1) * RB, min(RB, cnt - (k + 1) * RB));
         const unsigned char* stg = R_::arrive(p, rg);
         const int nr = min(RB, cnt - k * RB);
         if (stg) {
@@ -265,126 +309,85 @@ __global__ void __launch_bounds__(NT, 2) k_stats(const Prob p) {
           }
         }
         __syncwarp();
+        // the stage just read is free: request the batch after the next one
+        if (k + 2 < nbat) R_::template issue<true>(p, rg, g, lph + (k + 2) * RB, min(RB, cnt - (k + 2) * RB));
       }
     }
-    // ---- the round's sums: warp, CTA (fixed order), out
+  }
+  // a base warp without rows still has to publish the pivot when it is the one in charge
+  if (!have_piv && s == 0 && warp == wd) {
+    const bool ok = __all_sync(FULL, mbar_wait(&bars[NWARP * 2], 0u));
+    if (!ok && lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
+    Raw<T> kr, vr;
+    kr.ld(pivrow + j * 16);
+    vr.ld(pivrow + RWB + j * 16);
+    double dd = 0.0;
 #pragma unroll
-    for (int mask = LPR; mask < 32; mask <<= 1) {
+    for (int e = 0; e < EPL; ++e) dd = fma(qs[e * LPR], (double)kr.get(e), dd);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(FULL, acc[e], mask);
-      s1 += __shfl_xor_sync(FULL, s1, mask);
-      s2 += __shfl_xor_sync(FULL, s2, mask);
-    }
-#pragma unroll
-    for (int mask = 1; mask < 32; mask <<= 1) s3 += __shfl_xor_sync(FULL, s3, mask);
+    for (int mask = LPR / 2; mask >= 1; mask >>= 1) dd += __shfl_xor_sync(FULL, dd, mask);
+    cw = exp(dd * (double)p.scale - md);
     if (rsub == 0) {
-      double* wp = wpart + warp * NE;
+      double* gp = p.stat_piv + (long long)bh * (D + 1);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) wp[j * EPL + e] = acc[e];
-      if (j == 0) { wp[D] = s1; wp[D + 1] = s2; wp[D + 2] = s3; }
+      for (int e = 0; e < EPL; ++e) gp[j * EPL + e] = cw * (double)vr.get(e);
+      if (j == 0) gp[D] = cw;
     }
-    __syncthreads();
-    for (int e = tid; e < NE; e += NT) {
-      double sum = 0.0;
-#pragma unroll
-      for (int w = 0; w < NWARP; ++w) sum += wpart[w * NE + e];
-      gpart[round * NE + e] = sum;
-    }
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = 0.0;
-    s1 = s2 = s3 = 0.0;
-    if (round == 0 && b0 > 0) {
-      // the pivot: every row group evaluates it from the rows requested above (identical numbers everywhere)
-      const bool ok = __all_sync(FULL, mbar_wait(&bars[NWARP * 2], 0u));
-      if (!ok && lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
-      Raw<T> kr, vr;
-      kr.ld(pivrow + j * 16);
-      vr.ld(pivrow + RWB + j * 16);
-      double dd = 0.0;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) dd = fma(qs[e * LPR], (double)kr.get(e), dd);
-#pragma unroll
-      for (int mask = LPR / 2; mask >= 1; mask >>= 1) dd += __shfl_xor_sync(FULL, dd, mask);
-      cw = exp(dd * (double)p.scale - md);
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) pv[e] = cw * (double)vr.get(e);
-      if (s == 0 && warp == 0 && rsub == 0) {
-        double* gp = p.stat_piv + (long long)bh * (D + 1);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) gp[j * EPL + e] = pv[e];
-        if (j == 0) gp[D] = cw;
-      }
-    }
-    __syncthreads();                                   // `wpart` is free again
   }
-  (void)piv;
-  TICK_END(p, VATTN_K_STATS);
-}
-
-// ---------------------------------------------------------------------------------------------
-// k_final
-template <int D>
-constexpr size_t final_smem() {
-  return up16((size_t)NWARP * 2 * STAGE_BYTES) + up16(2 * (D + 3) * 8) + up16((D + 1) * 8) + up16((size_t)NWARP * (D + 1) * 4) +
-         up16(LCAP * 4) * 2 + up16(VATTN_BANDCAP * 4) + up16((NWARP * 2 + 2) * 8) + up16(128 * 4) + up16(16 * 4) + 128;
-}
-
-template <typename T, int D>
-__global__ void __launch_bounds__(NT, 2) k_final(const Prob p) {
-  using R_ = Rows<T, D>;
-  constexpr int EPL = R_::EPL, LPR = R_::LPR, RPI = R_::RPI, RWB = R_::RWB;
-  constexpr int NE = D + 3;
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* sp_ = smem_raw;
-  unsigned char* stage = sp_;                                           sp_ += up16((size_t)NWARP * 2 * STAGE_BYTES);
-  double* tot = reinterpret_cast<double*>(sp_);                         sp_ += up16(2 * NE * 8);     // [2][NE]
-  double* piv = reinterpret_cast<double*>(sp_);                         sp_ += up16((D + 1) * 8);
-  float* fw = reinterpret_cast<float*>(sp_);                            sp_ += up16((size_t)NWARP * (D + 1) * 4);
-  int* cl_ph = reinterpret_cast<int*>(sp_);                             sp_ += up16(LCAP * 4);       // the CTA's listed rows
-  int* cl_sc = reinterpret_cast<int*>(sp_);                             sp_ += up16(LCAP * 4);
-  int* vt = reinterpret_cast<int*>(sp_);                                sp_ += up16(VATTN_BANDCAP * 4);
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(sp_); sp_ += up16((NWARP * 2 + 2) * 8);
-  int* misc = reinterpret_cast<int*>(sp_);                              sp_ += up16(128 * 4);
-  unsigned* rkeys = reinterpret_cast<unsigned*>(sp_);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int S = (int)gridDim.x, s = (int)blockIdx.x, bh = (int)blockIdx.y;
-  const int b = bh / p.Hq, h = bh % p.Hq, g = h / p.G;
-  TICK_BEGIN(p, VATTN_K_FINAL);
-  if (tid < NWARP * 2) mbar_init(&bars[tid], 1);
-  if (tid < 2) walk_keys(p, b, p.rng_head_is_kv ? g : h, 1, tid, rkeys);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  DBGT(1);
+  // ---- sums: warp, CTA (fixed order: the deterministic warps, the base-sample warps), out
+#pragma unroll
+  for (int mask = LPR; mask < 32; mask <<= 1) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(FULL, acc[e], mask);
+    s1 += __shfl_xor_sync(FULL, s1, mask);
+    s2 += __shfl_xor_sync(FULL, s2, mask);
+  }
+#pragma unroll
+  for (int mask = 1; mask < 32; mask <<= 1) s3 += __shfl_xor_sync(FULL, s3, mask);
+  if (rsub == 0) {
+    double* wp = wpart + warp * NE;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) wp[j * EPL + e] = acc[e];
+    if (j == 0) { wp[D] = s1; wp[D + 1] = s2; wp[D + 2] = s3; }
+  }
   __syncthreads();
-  pdl_wait();                                          // the statistics kernel (and with it the selection) is complete
-  pdl_trigger();
-  TICK_BEGIN(p, VATTN_T_BUDGET);
-  const HeadMeta mt = p.meta[bh];
-  const int n = mt.n, s0 = mt.s0, l_start = mt.l_start, kk = mt.kk, n_s = mt.n_s, b0 = mt.b0;
-  T* out = reinterpret_cast<T*>(p.out) + (long long)bh * D;
-  if (n == 0) {
-    if (s == 0) {
-      for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
-      if (tid == 0) {
-        if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = 0;
-        if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
-        if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
-      }
-    }
-    return;
+  for (int item = tid; item < 2 * NE; item += NT) {
+    const int kind = item / NE, e = item % NE;
+    double sum = 0.0;
+    for (int w = kind ? wd : 0; w < (kind ? NWARP : wd); ++w) sum += wpart[w * NE + e];
+    gpart[item] = sum;
   }
-  // ------------------------------------------------------------------ budget (every CTA for itself)
+  DBGT(2);
+  // ------------------------------------------------------------------ budget, by the last CTA of the head
+  __threadfence();
+  __syncthreads();                                     // (also: `wpart` has been read)
+  int* flag = reinterpret_cast<int*>(pivrow);
+  if (tid == 0) flag[0] = (atomicAdd(&p.tickets[bh], 1u) == (unsigned)(S - 1));
+  __syncthreads();
+  if (!flag[0]) { TICK_END(p, VATTN_K_STATS); return; }
+  __threadfence();
+  double* tot = wpart;                                 // [2][NE] sums over the head's CTAs, in CTA order
   {
     const double* gp = p.stat_part + (long long)bh * S * 2 * NE;
     for (int item = tid; item < 2 * NE; item += NT) {
+      double v[VATTN_MAX_SPLITS];                      // all partials of the element at once (one memory round trip)
+#pragma unroll
+      for (int sp = 0; sp < VATTN_MAX_SPLITS; ++sp) v[sp] = sp < S ? __ldcg(gp + (long long)sp * 2 * NE + item) : 0.0;
       double sum = 0.0;
-      for (int sp = 0; sp < S; ++sp) sum += __ldcg(gp + (long long)sp * 2 * NE + item);     // fixed order
+#pragma unroll
+      for (int sp = 0; sp < VATTN_MAX_SPLITS; ++sp) sum += v[sp];                             // fixed order
       tot[item] = sum;
     }
     for (int e = tid; e <= D; e += NT) piv[e] = b0 > 0 ? __ldcg(p.stat_piv + (long long)bh * (D + 1) + e) : 0.0;
-    for (int c = tid; c < mt.nbt; c += NT) vt[c] = __ldcg(p.vtab + (long long)bh * VATTN_BANDCAP + c);
   }
   __syncthreads();
+  {
+    double* det = p.det_sums + (long long)bh * (D + 1);       // N_f, D_f for the final combination
+    for (int e = tid; e <= D; e += NT) det[e] = tot[e];
+  }
   if (warp == 0) {
+    const int n_s = mt.n_s;
     const double* t0 = tot;
     const double* t1 = tot + NE;
     const double Dfv = t0[D];
@@ -434,144 +437,200 @@ __global__ void __launch_bounds__(NT, 2) k_final(const Prob p) {
       const double bx = p.mode == 1 ? b_D : (p.mode == 2 ? b_N : b_S);
       if (p.force_budget >= 0) bf = min(p.force_budget, n_s);
       else {
-        if (!isfinite(bx) && s == 0 && lane == 0) atomicOr(p.status, VATTN_STATUS_NONFINITE);
+        if (!isfinite(bx) && lane == 0) atomicOr(p.status, VATTN_STATUS_NONFINITE);
         bf = min(max(ceil_sat(bx), b0), n_s);
       }
     }
     if (lane == 0) {
-      misc[2] = bf;
-      if (s == 0) {
-        if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = bf;
-        if (p.dbg.budgets) {
-          int* o = p.dbg.budgets + bh * 4;
-          o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bf;
-        }
-        if (p.dbg.stats) {
-          double* o = p.dbg.stats + bh * 8;
-          o[0] = Dfv; o[1] = sigma2; o[2] = trace; o[3] = Dhat; o[4] = Nnorm; o[5] = (double)n_s; o[6] = (double)b0;
-          o[7] = (double)mt.m;
-        }
+      p.budget[bh] = bf;
+      if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = bf;
+      if (p.dbg.budgets) {
+        int* o = p.dbg.budgets + bh * 4;
+        o[0] = bD; o[1] = bN; o[2] = bS; o[3] = bf;
+      }
+      if (p.dbg.stats) {
+        double* o = p.dbg.stats + bh * 8;
+        o[0] = Dfv; o[1] = sigma2; o[2] = trace; o[3] = Dhat; o[4] = Nnorm; o[5] = (double)n_s; o[6] = (double)b0;
+        o[7] = (double)mt.m;
       }
     }
   }
-  __syncthreads();
-  const int bfin = misc[2];
-  TICK_END(p, VATTN_T_BUDGET);
-  DBGT(0);
+  DBGT(5);
+  TICK_END(p, VATTN_K_STATS);
+}
 
-  // ------------------------------------------------------------------ rows of the final sample
-  // Ranks of the walk are dealt out in units of U rows (one batch per warp): CTA s takes the units s, s + S, ...
-  // A round lists up to LCAP of the CTA's rows in shared memory (physical slot, score), from
-  //   (1) the list the selection kernel wrote (ranks below min(b, listed)),
-  //   (2) further walk positions, evaluated here by all threads (listed <= rank < b < n_s), or
-  //   (3) every residual token in token order (b = n_s: no walk needed; every CTA passes over all tokens, so the
-  //       rank of a token among the residual tokens is known everywhere),
-  // then the warps stream the listed rows through their rings and reduce them.
+// ---------------------------------------------------------------------------------------------
+// k_final
+constexpr int FLAT_MAX_HEADS = 4096;   // heads whose work units are dealt out over the whole grid
+template <int D>
+constexpr size_t final_smem() {
+  return up16((size_t)NWARP * 2 * STAGE_BYTES) + up16((size_t)NWARP * (D + 1) * 4) + up16(LCAP * 4) * 2 + up16(VATTN_BANDCAP * 4) +
+         up16((NWARP * 2 + 2) * 8) + up16(128 * 4) + up16(16 * 4) + up16((FLAT_MAX_HEADS + 1) * 4) + 128;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(NT, 2) k_final(const Prob p) {
+  using R_ = Rows<T, D>;
+  constexpr int EPL = R_::EPL, LPR = R_::LPR, RPI = R_::RPI, RWB = R_::RWB;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* sp_ = smem_raw;
+  unsigned char* stage = sp_;                                           sp_ += up16((size_t)NWARP * 2 * STAGE_BYTES);
+  float* fw = reinterpret_cast<float*>(sp_);                            sp_ += up16((size_t)NWARP * (D + 1) * 4);
+  int* cl_ph = reinterpret_cast<int*>(sp_);                             sp_ += up16(LCAP * 4);       // the CTA's listed rows
+  int* cl_sc = reinterpret_cast<int*>(sp_);                             sp_ += up16(LCAP * 4);
+  int* vt = reinterpret_cast<int*>(sp_);                                sp_ += up16(VATTN_BANDCAP * 4);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(sp_); sp_ += up16((NWARP * 2 + 2) * 8);
+  int* misc = reinterpret_cast<int*>(sp_);                              sp_ += up16(128 * 4);
+  unsigned* rkeys = reinterpret_cast<unsigned*>(sp_);                   sp_ += up16(16 * 4);
+  int* upref = reinterpret_cast<int*>(sp_);                             // [BH + 1] units before head hh (flat mode)
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int S = (int)gridDim.x, s = (int)blockIdx.x, bh = (int)blockIdx.y;
+  const int BH = p.B * p.Hq;
+  const int b = bh / p.Hq, h = bh % p.Hq, g = h / p.G;
+  TICK_BEGIN(p, VATTN_K_FINAL);
+  if (tid < NWARP * 2) mbar_init(&bars[tid], 1);
+  if (tid < 2) walk_keys(p, b, p.rng_head_is_kv ? g : h, 1, tid, rkeys);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  pdl_wait();                                          // the statistics kernel (and with it the selection) is complete
+  pdl_trigger();
+  TICK_BEGIN(p, VATTN_T_BUDGET);
+
+  // ------------------------------------------------------------------ work units
+  // The rows the selection kernel listed for head hh, ranks [0, lim_hh), lim = min(b, listed) (nothing when b is the
+  // whole residual), are cut into units of U rows, one batch per warp.  Budgets differ a lot between heads, so the
+  // units of all heads form one list that the CTAs of the grid walk with a stride (up to 4,096 heads; beyond that a
+  // head's units stay with its own CTAs).  Rows beyond the listed ones (rare) are done by the head's own CTAs.
+  const bool kv = p.gather_kv != 0;
+  const int RB = kv ? R_::RB_KV : R_::RB_V;
+  const int U = RB * NWARP;
+  const bool flat = BH <= FLAT_MAX_HEADS;
+  // (without the flat list a head's units stay with its S CTAs: units of about a 1/S share)
+  constexpr int MAXU = 32;                             // most units (partial slots) of listed rows per head
+  int ugoal = U;                                       // rows per unit the grid aims at: about one unit per CTA
+  auto unit_rows = [&](int lim) -> int {               // rows per unit of a head: a whole number of U, at most MAXU units
+    const int nb = (lim + U - 1) / U;
+    const int fit = ((nb + MAXU - 1) / MAXU) * U;
+    return fit > ugoal ? fit : ugoal;
+  };
+  auto units_of = [&](int lim) -> int { const int ur = unit_rows(lim); return (lim + ur - 1) / ur; };
+  auto lim_of = [&](int hh) -> int {
+    const HeadMeta* mh = p.meta + hh;
+    const int nn = __ldcg(&mh->n), ns_ = __ldcg(&mh->n_s), li = __ldcg(&mh->dyn_listed);
+    const int bb = __ldcg(p.budget + hh);
+    if (nn == 0 || bb <= 0 || bb >= ns_) return 0;
+    return min(bb, li);
+  };
+  if (flat) {
+    // exclusive prefix of the unit counts (BH <= 4096: 16 heads per thread at most)
+    const int per = (BH + NT - 1) / NT;
+    int loc = 0, tot1;
+    for (int q_ = 0; q_ < per; ++q_) { const int hh = tid * per + q_; if (hh < BH) loc += lim_of(hh); }
+    block_scan_reg_rows(loc, misc + 32, tot1);         // listed rows of the whole step
+    ugoal = ((tot1 / (S * BH) + U) / U) * U;
+    __syncthreads();
+    loc = 0;
+    for (int q_ = 0; q_ < per; ++q_) { const int hh = tid * per + q_; if (hh < BH) loc += units_of(lim_of(hh)); }
+    int run = block_scan_reg_rows(loc, misc + 32, tot1);
+    for (int q_ = 0; q_ < per; ++q_) {
+      const int hh = tid * per + q_;
+      if (hh < BH) { upref[hh] = run; run += units_of(lim_of(hh)); }
+    }
+    if (tid == 0) upref[BH] = tot1;
+    __syncthreads();
+  }
+  const HeadMeta mt = p.meta[bh];
+  const int bfin = __ldcg(p.budget + bh);
+  if (!flat) ugoal = (((bfin < mt.dyn_listed ? bfin : mt.dyn_listed) / S + U) / U) * U;
+  TICK_END(p, VATTN_T_BUDGET);
+  DBGT(8);
+  const int my_lim = (mt.n == 0 || bfin <= 0 || bfin >= mt.n_s) ? 0 : min(bfin, mt.dyn_listed);
+  const bool whole = mt.n > 0 && bfin > 0 && bfin >= mt.n_s;          // this head's sample is its whole residual
+  const bool extend = mt.n > 0 && bfin > my_lim && !whole;            // this head's walk goes on beyond the list
+  // partial slots of head hh: one per unit, then one per CTA of the head when it has rows beyond the list
+  auto parts_of = [&](int hh_units, bool extra) { return hh_units + (extra ? S : 0); };
+
   Ring rg;
   rg.bar = bars + warp * 2;
   rg.stg = stage + (size_t)warp * 2 * STAGE_BYTES;
   rg.issued = rg.consumed = 0;
   const int rsub = lane / LPR, j = lane % LPR;
-  const float m = mt.m;
-  const bool kv = p.gather_kv != 0;
-  const int RB = kv ? R_::RB_KV : R_::RB_V;
-  const int U = RB * NWARP;
-  const float* sc = p.scores + (long long)bh * p.npad;
-  const int* dl = p.dyn_idx + (long long)bh * 3 * p.npad;
-  const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
-  int* ddbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)bh * p.max_seq_len : nullptr;
   float facc[EPL], fd = 0.f, qf[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) { facc[e] = 0.f; qf[e] = 0.f; }
-  if (kv) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
-  const bool whole = bfin >= n_s;                      // the sample is the whole residual
-  const int lim = whole ? 0 : min(bfin, mt.dyn_listed);       // ranks served from the list
-  const Walk wk = make_walk(rkeys, l_start - s0);
-  int phase = lim > 0 ? 1 : (whole ? 3 : 2);
-  int ucur = s;                                        // phase 1: next unit of the list
-  int J = mt.dyn_J, have = whole ? 0 : mt.dyn_listed;  // phase 2: next walk position; residual tokens before the round
-  int tcur = s0;                                       // phase 3: next token
-  if (bfin <= 0) phase = 0;
-#pragma unroll 1
-  while (phase != 0) {
-    int cnt = 0;                                       // rows listed this round (uniform over the CTA)
-    if (phase == 1) {
-      // units of the selection kernel's list
-      int nun = 0, first = ucur;
-      while (nun < LCAP / U && ucur * U < lim) { ++nun; ucur += S; }
-      for (int x = tid; x < nun * U; x += NT) {
-        const int rank = (first + (x / U) * S) * U + x % U;
-        if (rank < lim) {
-          cl_ph[x] = dl[p.npad + rank];
-          cl_sc[x] = dl[2 * p.npad + rank];
-          if (ddbg) ddbg[rank] = dl[rank];
-        }
-      }
-      // rows of the round: all units but the last are full
-      cnt = nun > 0 ? (nun - 1) * U + min(U, lim - (first + (nun - 1) * S) * U) : 0;
-      if (ucur * U >= lim) phase = (bfin > lim) ? 2 : 0;
-      if (cnt == 0 && phase == 1) phase = 0;
-    } else {
-      // (2) WPT consecutive walk positions per thread, or (3) WPT consecutive tokens per thread
-      int tokc[WPT]; float svc[WPT];
-      int nres = 0;
-      const int base = phase == 2 ? J : tcur;
-      const int end = phase == 2 ? (l_start - s0) : l_start;
+
+  // one partial slot is complete: CTA sums in warp order, the slot, the head's ticket; the last finisher of the head
+  // adds the slots in order, scales by n_s/b, adds N_f and D_f and divides
+  auto finish_part = [&](int hh, int slot, int nparts) {
 #pragma unroll
-      for (int q_ = 0; q_ < WPT; ++q_) {
-        tokc[q_] = -1; svc[q_] = 0.f;
-        const int x = base + tid * WPT + q_;
-        if (x < end) {
-          const int tok = phase == 2 ? s0 + walk_at(wk, x) : x;
-          const float sv = __ldg(sc + tok);
-          if (!in_topk(mt, vt, gbitmap, tok, sv)) { tokc[q_] = tok; svc[q_] = sv; ++nres; }
-        }
-      }
-      // ranks (phase 2) from a prefix sum; ownership by rank unit (phase 2) or by block of 128 tokens (phase 3)
-      int tot1;
-      int rank = have + block_scan_reg_rows(nres, misc + 32, tot1);
-      int own = 0;
-      unsigned ownm = 0u;
+    for (int mask = LPR; mask < 32; mask <<= 1) {
 #pragma unroll
-      for (int q_ = 0; q_ < WPT; ++q_) {
-        if (tokc[q_] >= 0) {
-          const bool mine = phase == 2 ? (rank < bfin && (rank / U) % S == s) : ((tokc[q_] >> 7) % S == s);
-          if (mine) { ownm |= 1u << q_; ++own; if (ddbg) ddbg[rank] = tokc[q_]; }
-          ++rank;
+      for (int e = 0; e < EPL; ++e) facc[e] += __shfl_xor_sync(FULL, facc[e], mask);
+      fd += __shfl_xor_sync(FULL, fd, mask);
+    }
+    if (rsub == 0) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) fw[warp * (D + 1) + j * EPL + e] = facc[e];
+      if (j == 0) fw[warp * (D + 1) + D] = fd;
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) facc[e] = 0.f;
+    fd = 0.f;
+    __syncthreads();
+    float* gpart = p.gat_part + ((long long)hh * p.gat_slots + slot) * (D + 1);
+    for (int e = tid; e <= D; e += NT) {
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) sum += fw[w * (D + 1) + e];
+      gpart[e] = sum;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) misc[0] = (atomicAdd(&p.tickets[(long long)BH + hh], 1u) == (unsigned)(nparts - 1));
+    __syncthreads();
+    if (misc[0]) {
+      __threadfence();
+      const int ns_ = __ldcg(&p.meta[hh].n_s), bb = __ldcg(p.budget + hh);
+      const double f = (bb > 0) ? (double)ns_ / (double)bb : 0.0;
+      const float* src0 = p.gat_part + (long long)hh * p.gat_slots * (D + 1);
+      const double* det = p.det_sums + (long long)hh * (D + 1);
+      // every thread requests the partials of its element 16 at a time (one memory round trip each), adds in slot order
+      T* o = reinterpret_cast<T*>(p.out) + (long long)hh * D;
+      for (int e = tid; e <= D; e += NT) {
+        float sum = 0.f;
+        for (int sp0 = 0; sp0 < nparts; sp0 += 16) {
+          float v[16];
+#pragma unroll
+          for (int q_ = 0; q_ < 16; ++q_) v[q_] = sp0 + q_ < nparts ? __ldcg(src0 + (long long)(sp0 + q_) * (D + 1) + e) : 0.f;
+#pragma unroll
+          for (int q_ = 0; q_ < 16; ++q_) sum += v[q_];
         }
+        fw[e] = sum;
       }
       __syncthreads();
-      int tot2;
-      int pos = block_scan_reg_rows(own, misc + 32, tot2);
-#pragma unroll
-      for (int q_ = 0; q_ < WPT; ++q_) {
-        if ((ownm >> q_) & 1u) {
-          const int tok = tokc[q_];
-          cl_ph[pos] = page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15);
-          cl_sc[pos] = __float_as_int(svc[q_]);
-          ++pos;
-        }
-      }
-      cnt = tot2;
-      have += tot1;
-      if (phase == 2) { J += NT * WPT; if (have >= bfin || J >= l_start - s0) phase = 0; }
-      else { tcur += NT * WPT; if (tcur >= l_start) phase = 0; }
+      const double den = __ldcg(det + D) + f * (double)fw[D];        // D_f + n_s/b * sum w
+      for (int e = tid; e < D; e += NT) o[e] = Elem<T>::from_float((float)((__ldcg(det + e) + f * (double)fw[e]) / den));
     }
     __syncthreads();
-    DBGT(1);
-    // ---- the warps stream the round's rows: warp w takes the batches w, w + NWARP, ...
+  };
+  // the warps stream the CTA's `cnt` listed rows (cl_ph, cl_sc) of head hh: warp w takes the batches w, w + NWARP, ...
+  auto stream_rows = [&](int hh, int cnt) {
+    const int gh = (hh % p.Hq) / p.G;
+    const float m = __ldcg(&p.meta[hh].m);
+    if (kv) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)hh * D + j * EPL, qf);
     const int nbat_all = (cnt + RB - 1) / RB;
     int k = warp;
     if (k < nbat_all) {
-      if (kv) R_::template issue<true>(p, rg, g, cl_ph + k * RB, min(RB, cnt - k * RB));
-      else R_::template issue<false>(p, rg, g, cl_ph + k * RB, min(RB, cnt - k * RB));
+      if (kv) R_::template issue<true>(p, rg, gh, cl_ph + k * RB, min(RB, cnt - k * RB));
+      else R_::template issue<false>(p, rg, gh, cl_ph + k * RB, min(RB, cnt - k * RB));
     }
 #pragma unroll 1
     for (; k < nbat_all; k += NWARP) {
       const int kn = k + NWARP;
       if (kn < nbat_all) {
-        if (kv) R_::template issue<true>(p, rg, g, cl_ph + kn * RB, min(RB, cnt - kn * RB));
-        else R_::template issue<false>(p, rg, g, cl_ph + kn * RB, min(RB, cnt - kn * RB));
+        if (kv) R_::template issue<true>(p, rg, gh, cl_ph + kn * RB, min(RB, cnt - kn * RB));
+        else R_::template issue<false>(p, rg, gh, cl_ph + kn * RB, min(RB, cnt - kn * RB));
       }
       const unsigned char* stg = R_::arrive(p, rg);
       const int nr = min(RB, cnt - k * RB);
@@ -623,48 +682,122 @@ __global__ void __launch_bounds__(NT, 2) k_final(const Prob p) {
       }
       __syncwarp();
     }
-    __syncthreads();                                   // the CTA's list is free for the next round
-    DBGT(2);
-  }
-  // ------------------------------------------------------------------ sums: warp, CTA, head; the last CTA combines
-#pragma unroll
-  for (int mask = LPR; mask < 32; mask <<= 1) {
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) facc[e] += __shfl_xor_sync(FULL, facc[e], mask);
-    fd += __shfl_xor_sync(FULL, fd, mask);
-  }
-  if (rsub == 0) {
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) fw[warp * (D + 1) + j * EPL + e] = facc[e];
-    if (j == 0) fw[warp * (D + 1) + D] = fd;
-  }
-  __syncthreads();
-  float* gpart = p.gat_part + ((long long)bh * S + s) * (D + 1);
-  for (int e = tid; e <= D; e += NT) {
-    float sum = 0.f;
-#pragma unroll
-    for (int w = 0; w < NWARP; ++w) sum += fw[w * (D + 1) + e];
-    gpart[e] = sum;
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) misc[0] = (atomicAdd(&p.tickets[(long long)p.B * p.Hq + bh], 1u) == (unsigned)(S - 1));
-  __syncthreads();
-  DBGT(3);
-  if (!misc[0]) { TICK_END(p, VATTN_K_FINAL); return; }
-  __threadfence();
+  };
+
+  // ------------------------------------------------------------------ (1) the listed rows, unit by unit
   {
-    const double f = (bfin > 0) ? (double)n_s / (double)bfin : 0.0;
-    const float* src0 = p.gat_part + (long long)bh * S * (D + 1);
-    float dsum = 0.f;
-    for (int sp = 0; sp < S; ++sp) dsum += __ldcg(src0 + (long long)sp * (D + 1) + D);
-    const double den = tot[D] + f * (double)dsum;      // D_f + n_s/b * sum w
-    for (int e = tid; e < D; e += NT) {
-      float sum = 0.f;
-      for (int sp = 0; sp < S; ++sp) sum += __ldcg(src0 + (long long)sp * (D + 1) + e);     // fixed order
-      out[e] = Elem<T>::from_float((float)((tot[e] + f * (double)sum) / den));
+    const int ncta = S * BH, cid = bh * S + s;
+    const int total_units = flat ? upref[BH] : units_of(my_lim);
+#pragma unroll 1
+    for (int gu = flat ? cid : s; gu < total_units; gu += flat ? ncta : S) {
+      int hh = bh, u = gu;
+      if (flat) {
+        int lo = 0, hi2 = BH - 1;                      // last head whose first unit is <= gu
+        while (lo < hi2) { const int mid = (lo + hi2 + 1) >> 1; if (upref[mid] <= gu) lo = mid; else hi2 = mid - 1; }
+        hh = lo; u = gu - upref[hh];
+      }
+      const int lim = flat ? lim_of(hh) : my_lim;
+      const int units = units_of(lim), urows = unit_rows(lim);
+      const int bb = __ldcg(p.budget + hh);
+      const bool extra = bb > lim;                     // that head also has rows beyond its list (its own CTAs' slots)
+      const int* dl = p.dyn_idx + (long long)hh * 3 * p.npad;
+      int* ddbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)hh * p.max_seq_len : nullptr;
+      const int r_end = min(lim, (u + 1) * urows);
+#pragma unroll 1
+      for (int r0 = u * urows; r0 < r_end; r0 += LCAP) {         // rounds of up to LCAP rows
+        const int cnt = min(LCAP, r_end - r0);
+        for (int x = tid; x < cnt; x += NT) {
+          cl_ph[x] = dl[p.npad + r0 + x];
+          cl_sc[x] = dl[2 * p.npad + r0 + x];
+          if (ddbg) ddbg[r0 + x] = dl[r0 + x];
+        }
+        __syncthreads();
+        DBGT(9);
+        stream_rows(hh, cnt);
+        __syncthreads();
+        DBGT(10);
+      }
+      finish_part(hh, u, parts_of(units, extra));
+      DBGT(11);
     }
   }
+  DBGT(12);
+  if (mt.n == 0) {
+    if (s == 0) {
+      T* o = reinterpret_cast<T*>(p.out) + (long long)bh * D;
+      for (int e = tid; e < D; e += NT) o[e] = Elem<T>::from_float(0.f);
+    }
+    TICK_END(p, VATTN_K_FINAL);
+    return;
+  }
+  // ------------------------------------------------------------------ (2) rows beyond the list, by the head's own CTAs
+  //   further walk positions, evaluated by all threads (listed <= rank < b < n_s), or every residual token in token
+  //   order (b = n_s: no walk needed; every CTA passes over all tokens, so the rank of a token is known everywhere)
+  const int my_units = units_of(my_lim);
+  if (whole || extend) {
+    const int s0 = mt.s0, l_start = mt.l_start;
+    for (int c = tid; c < mt.nbt; c += NT) vt[c] = __ldcg(p.vtab + (long long)bh * VATTN_BANDCAP + c);
+    __syncthreads();
+    const float* sc = p.scores + (long long)bh * p.npad;
+    const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
+    int* ddbg = p.dbg.dyn_idx ? p.dbg.dyn_idx + (long long)bh * p.max_seq_len : nullptr;
+    const Walk wk = make_walk(rkeys, l_start - s0);
+    int J = mt.dyn_J, have = whole ? 0 : mt.dyn_listed;
+    int tcur = s0;
+    bool more = true;
+#pragma unroll 1
+    while (more) {
+      int tokc[WPT]; float svc[WPT];
+      int nres = 0;
+      const int base = whole ? tcur : J;
+      const int end = whole ? l_start : (l_start - s0);
+#pragma unroll
+      for (int q_ = 0; q_ < WPT; ++q_) {
+        tokc[q_] = -1; svc[q_] = 0.f;
+        const int x = base + tid * WPT + q_;
+        if (x < end) {
+          const int tok = whole ? x : s0 + walk_at(wk, x);
+          const float sv = __ldg(sc + tok);
+          if (!in_topk(mt, vt, gbitmap, tok, sv)) { tokc[q_] = tok; svc[q_] = sv; ++nres; }
+        }
+      }
+      int tot1;
+      int rank = have + block_scan_reg_rows(nres, misc + 32, tot1);
+      int own = 0;
+      unsigned ownm = 0u;
+#pragma unroll
+      for (int q_ = 0; q_ < WPT; ++q_) {
+        if (tokc[q_] >= 0) {
+          const bool mine = whole ? ((tokc[q_] >> 7) % S == s) : (rank < bfin && (rank / U) % S == s);   // U rows per CTA in turn
+          if (mine) { ownm |= 1u << q_; ++own; if (ddbg) ddbg[rank] = tokc[q_]; }
+          ++rank;
+        }
+      }
+      __syncthreads();
+      int tot2;
+      int pos = block_scan_reg_rows(own, misc + 32, tot2);
+#pragma unroll
+      for (int q_ = 0; q_ < WPT; ++q_) {
+        if ((ownm >> q_) & 1u) {
+          const int tok = tokc[q_];
+          cl_ph[pos] = page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15);
+          cl_sc[pos] = __float_as_int(svc[q_]);
+          ++pos;
+        }
+      }
+      have += tot1;
+      if (whole) { tcur += NT * WPT; more = tcur < l_start; }
+      else { J += NT * WPT; more = have < bfin && J < l_start - s0; }
+      __syncthreads();
+      stream_rows(bh, tot2);
+      __syncthreads();                                 // the CTA's list is free for the next round
+    }
+    finish_part(bh, my_units + s, parts_of(my_units, true));
+  } else if (my_units == 0 && s == 0) {
+    // nothing sampled (no residual): the output is the deterministic part alone; one empty slot triggers the division
+    finish_part(bh, 0, 1);
+  }
+  DBGT(13);
   TICK_END(p, VATTN_K_FINAL);
 }
 

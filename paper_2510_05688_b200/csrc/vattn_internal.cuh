@@ -49,7 +49,7 @@ struct Prob {
   unsigned* m_ord;        // [B,Hq]  order-preserving encoding of the running max score
   unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
   unsigned* unit_ctr;     // [1] work-unit counter of the persistent score kernel
-  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters: [1] final sample, [2] dense kernel
+  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters: [0] statistics, [1] final sample, [2] dense kernel
   unsigned* status;       // [1]
   unsigned* bitmap;       // [B,Hq,nwords] near-tie tokens that made it into I_t (used when they are too many for a list)
   int* vtab;              // [B,Hq,BANDCAP] near-tie tokens ascending, bit 31 = member of I_t
@@ -62,7 +62,11 @@ struct Prob {
   HeadMeta* meta;         // [B,Hq]
   double* stat_part;      // [B,Hq,splits,2,D+3] sums of the statistics kernel: deterministic rows, base-sample rows
   double* stat_piv;       // [B,Hq,D+1] pivot row of the base-sample sums: w*V then w
-  float* gat_part;        // [B,Hq,splits,D+1] sums of the final sample
+  double* det_sums;       // [B,Hq,D+1] N_f then D_f
+  int* budget;            // [B,Hq] the budget b (written by the statistics kernel)
+  float* gat_part;        // [B,Hq,gat_slots,D+1] sums of the final sample: one slot per unit of listed rows, then one
+                          //                      per CTA of the head for rows beyond the list
+  int gat_slots;
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int dense_splits;
   int splits;             // CTAs per head of the row kernels
