@@ -513,9 +513,9 @@ def main():
         "k_walk": int(5 * b0s.sum()) * 4,
         "k_select": n_tot * Hq * 4 + int(kks.sum()) * 8 + int(b0s.sum()) * 8 + int(min(8 * b0s.max(), n_tot)) * Hq * 12,
         "k_stats": int(n_f + b0s.sum()) * d * es * 2,
-        "k_final": int(b_dyn.sum()) * (d * es + 8),
+        "k_gather": int(b_dyn.sum()) * (d * es + 12),
     }
-    rows_bytes = alg["k_stats"] + alg["k_final"]
+    rows_bytes = alg["k_stats"] + alg["k_gather"]
     traffic, traffic_note = read_traffic()
     peak, peak_kind = measured_peaks()
     kern = {}
@@ -543,8 +543,8 @@ def main():
         return {"us": round(us, 2), "achieved": round(g, 1), "frac": round(g / peak, 4), "frac_of_8TBs_nominal": round(g / 8000.0, 4)}
     # the row kernels (statistics, final sample): device-side spans inside graph-replayed steps
     rows_span = None
-    if timeline["k_stats"][0] is not None and timeline["k_final"][1] is not None:
-        rows_span = timeline["k_final"][1] - timeline["k_stats"][0]
+    if timeline["k_stats"][0] is not None and timeline["k_gather"][1] is not None:
+        rows_span = timeline["k_gather"][1] - timeline["k_stats"][0]
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -585,11 +585,13 @@ def main():
                      "device_timer": dict(frac_of(alg[top], span("k_score")) or {},
                                           timing="first CTA start to last CTA end (%globaltimer) inside graph-replayed steps")},
         # the gather / reduce part of the step (rows of I_f, I_bs and I_dyn) and the whole step, against the same peak
-        "roofline_rows": dict(frac_of(rows_bytes, rows_span) or {}, kernel="k_stats + k_final", alg_bytes=int(rows_bytes),
-                              traffic=(traffic.get("k_stats", 0) + traffic.get("k_final", 0)) or None,
-                              timing="first CTA of k_stats to last CTA of k_final (%globaltimer), graph-replayed steps"),
+        "roofline_rows": dict(frac_of(rows_bytes, rows_span) or {}, kernel="k_stats + k_gather", alg_bytes=int(rows_bytes),
+                              traffic=(traffic.get("k_stats", 0) + traffic.get("k_gather", 0)) or None,
+                              timing="first CTA of k_stats to last CTA of k_gather (%globaltimer), graph-replayed steps"),
         "roofline_k_stats": dict(frac_of(alg["k_stats"], span("k_stats")) or {}, alg_bytes=int(alg["k_stats"])),
-        "roofline_k_final": dict(frac_of(alg["k_final"], span("k_final")) or {}, alg_bytes=int(alg["k_final"])),
+        "roofline_k_gather": dict(frac_of(alg["k_gather"], (timeline["k_gather"][1] - timeline["budget"][1])
+                                          if timeline["k_gather"][1] and timeline["budget"][1] else None) or {},
+                                  alg_bytes=int(alg["k_gather"]), timing="last budget known to last CTA of k_gather"),
         "roofline_step": dict(frac_of(sparse_bytes, us_step) or {}, alg_bytes=int(sparse_bytes)),
         "kernels": kern,
         "timeline_us": timeline,

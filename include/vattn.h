@@ -97,10 +97,10 @@ typedef struct {
                                      (VATTN_STATUS_BAND_OVERFLOW) */
   unsigned long long *kernel_ticks; /* [VATTN_NUM_TICKS][2] device-side time stamps in ns (%globaltimer): rows 0-5 the
                                      counter-clearing kernel, the score kernel, the walk kernel, the selection kernel,
-                                     the statistics kernel and the final-sample kernel ([k][0] = earliest CTA start,
+                                     the statistics kernel and the gather kernel ([k][0] = earliest CTA start,
                                      [k][1] = latest end); row 6 the top-k selection proper (first CTA past its
-                                     dependency wait .. last CTA with I_t complete); row 7 the budget (first final-sample CTA past its
-                                     dependency wait .. last CTA that knows its budget).
+                                     dependency wait .. last CTA with I_t complete); row 7 the budgets (first head
+                                     whose statistics are complete .. last head that knows its budget).
                                      Folded with atomic min / max: set [k][0] = UINT64_MAX and [k][1] = 0 before the
                                      step to be observed.  Unlike event profiling this leaves the step as it is */
 } vattn_debug;
@@ -210,8 +210,8 @@ int vattn_set_stop_after(vattn_plan* plan, int kernels);
 
 /* Optional per-kernel timing of vattn_decode, for measurement harnesses.  While enabled, every call
  * records CUDA events on `stream` around each of its VATTN_NUM_KERNELS kernels (score pass; walk tokens;
- * selection and sample lists; deterministic and base-sample rows; budget, final sample and combination), for up to 256 calls between
- * two reads.  The events keep a kernel's prologue from running beside its predecessor, so the times add up to
+ * selection and sample lists; deterministic and base-sample rows with the budget; final sample and combination),
+ * for up to 256 calls between two reads.  The events keep a kernel's prologue from running beside its predecessor, so the times add up to
  * more than an unprofiled step takes.  vattn_read_profile waits for the last recorded call, writes the
  * summed elapsed milliseconds per kernel to ms_sum[VATTN_NUM_KERNELS] (host) and the number of calls to
  * *calls (host), and starts a new window.  Events add a little latency: do not enable in production. */

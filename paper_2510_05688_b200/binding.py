@@ -21,9 +21,11 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
            "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
-KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_final"]
+KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_gather"]
 NUM_TICKS = 8
-TICK_NAMES = ["k_zero", "k_score", "k_walk", "k_select", "k_stats", "k_final", "topk", "budget"]
+# measurement builds (VATTN_DEFINES="VATTN_PHASE_TICKS") stamp phases inside the kernels into further rows
+TICK_ROWS = 2560 if "VATTN_PHASE_TICKS" in os.environ.get("VATTN_DEFINES", "") else NUM_TICKS
+TICK_NAMES = ["k_zero", "k_score", "k_walk", "k_select", "k_stats", "k_gather", "topk", "budget"]
 
 
 class Shape(C.Structure):
@@ -186,7 +188,7 @@ class Plan:
         """Register only the device-side time-stamp buffer ([NUM_TICKS, 2] int64, rows named by TICK_NAMES).
         Call reset_kernel_ticks() before the step to observe, read the tensor after it."""
         import torch
-        self.ticks = torch.zeros(NUM_TICKS, 2, dtype=torch.int64, device=self.device)
+        self.ticks = torch.zeros(TICK_ROWS, 2, dtype=torch.int64, device=self.device)
         d = Debug(kernel_ticks=self.ticks.data_ptr())
         _check(lib().vattn_set_debug(self._h, C.byref(d)), "vattn_set_debug")
         self.reset_kernel_ticks()

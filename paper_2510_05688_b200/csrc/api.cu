@@ -19,10 +19,10 @@ struct vattn_plan {
   cudaEvent_t* ev;          // [kProfCalls][kProfEvents]
   int prof_calls;           // calls recorded since the last read
   // derived
-  int G, npad, nwords, dense_splits;
-  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_dyn, off_meta, off_stat,
-      off_piv, off_det, off_budget, off_gat, off_dense, total;
-  int splits, gat_slots;                  // CTAs per head of the row kernels
+  int G, npad, nwords, dense_splits, stat_splits, stat_splits_base;
+  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_holes, off_dyn, off_meta, off_stat,
+      off_piv, off_det, off_gmeta, off_gat, off_dense, total;
+  int gat_slots;
   // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
   struct HostStep {
     bool used, pinned, mapped;
@@ -81,32 +81,48 @@ void derive(vattn_plan* pl) {
   const int groups = s.batch * s.num_kv_heads * GC;
   const int sp = (4 * device_sm_count() + groups - 1) / groups;
   pl->dense_splits = sp < 1 ? 1 : (sp > 128 ? 128 : sp);
-  // row kernels: two CTAs of 8 warps per SM, shared evenly by the heads
+  // statistics kernel (128-thread CTAs, 5 per SM): one wave for both kinds of CTA.  The base-sample rows are on
+  // the step's critical path (they wait for the sample's list), the deterministic rows start earlier: three fifths
+  // of the wave go to the former.  (When even four CTAs per kind and head overfill the wave the kernel is
+  // throughput-bound: split freely.)
   {
-    const int sp2 = (2 * device_sm_count()) / heads;
-    pl->splits = sp2 < 1 ? 1 : (sp2 > VATTN_MAX_SPLITS ? VATTN_MAX_SPLITS : sp2);
+    const int wave = (5 * device_sm_count()) / heads;
+    if (wave < 8) {
+      pl->stat_splits = pl->stat_splits_base = 4;
+    } else {
+      const int sb = (3 * wave + 2) / 5;
+      pl->stat_splits_base = sb > VATTN_STAT_MAXS ? VATTN_STAT_MAXS : sb;
+      const int sd = wave - pl->stat_splits_base;
+      pl->stat_splits = sd < 4 ? 4 : (sd > VATTN_STAT_MAXS ? VATTN_STAT_MAXS : sd);
+    }
   }
   const size_t BH = (size_t)heads, D = (size_t)s.head_dim;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   pl->off_scores = take(BH * pl->npad * sizeof(float));
-  // cleared every step: running maxima [BH], max |K| [B*Hkv], tickets [3*BH], the score kernel's unit counter
-  pl->zero_bytes = (BH + (size_t)s.batch * s.num_kv_heads + 3 * BH + 4) * sizeof(unsigned);
+  // cleared every step: running maxima [BH], max |K| [B*Hkv], tickets [4*BH], the score kernel's unit counter
+  pl->zero_bytes = align_up((BH + (size_t)s.batch * s.num_kv_heads + 4 * BH + 4) * sizeof(unsigned), 8) + BH * 8;   // ... and the 64-bit words [BH]
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
   pl->off_vtab = take(BH * VATTN_BANDCAP * sizeof(int));
   pl->off_topk = take(2 * BH * pl->npad * sizeof(int));     // token indices, then physical slots
   pl->off_base = take(2 * BH * pl->npad * sizeof(int));
-  pl->off_walk = take(2 * BH * pl->npad * sizeof(int));     // tokens of the first walk positions, both walks
+  pl->off_walk = take(4 * BH * pl->npad * sizeof(int));     // first walk positions of both walks: tokens, physical slots
+  pl->off_holes = take(BH * VATTN_BANDCAP * sizeof(int));
   pl->off_dyn = take(3 * BH * pl->npad * sizeof(int));      // tokens, physical slots, score bits
   pl->off_meta = take(BH * sizeof(HeadMeta));
-  pl->off_stat = take(BH * (size_t)pl->splits * 2 * (D + 3) * sizeof(double));
+  pl->off_stat = take(BH * 2 * VATTN_STAT_MAXS * (D + 3) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
-  pl->off_budget = take(BH * sizeof(int));
-  // partial slots of the final sample per head: up to 32 units of listed rows, plus one per CTA of the head
-  pl->gat_slots = 32 + pl->splits;
+  pl->off_gmeta = take(BH * sizeof(int4));
+  // partial slots (chunks) per head of the gather kernel: 32, except that a handful of heads may use more of
+  // the 8 CTAs per SM (64 to 128 chunks each when that many fit the grid at once)
+  {
+    const size_t fit = (size_t)(8 * device_sm_count()) / BH;
+    const size_t flat = fit >= 2 * VATTN_GATHER_FLAT_SLOTS ? (fit > 128 ? 128 : fit) : VATTN_GATHER_FLAT_SLOTS;
+    pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? (int)flat : 32;   // per-head decomposition: up to 32 chunks
+  }
   pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
   pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
   pl->total = off;
@@ -138,24 +154,26 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
   const size_t BH = (size_t)s.batch * s.num_q_heads;
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
-  p.unit_ctr = p.tickets + 3 * BH;
+  p.unit_ctr = p.tickets + 4 * BH;
+  p.flags64 = reinterpret_cast<unsigned long long*>(w + pl->off_zero + pl->zero_bytes - BH * 8);
   p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
   p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);
   p.vtab = reinterpret_cast<int*>(w + pl->off_vtab);
   p.topk_idx = reinterpret_cast<int*>(w + pl->off_topk);
   p.base_idx = reinterpret_cast<int*>(w + pl->off_base);
   p.walk_tok = reinterpret_cast<int*>(w + pl->off_walk);
+  p.hole_pos = reinterpret_cast<int*>(w + pl->off_holes);
   p.dyn_idx = reinterpret_cast<int*>(w + pl->off_dyn);
   p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
   p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);
   p.stat_piv = reinterpret_cast<double*>(w + pl->off_piv);
   p.det_sums = reinterpret_cast<double*>(w + pl->off_det);
-  p.budget = reinterpret_cast<int*>(w + pl->off_budget);
+  p.gat_meta = reinterpret_cast<int4*>(w + pl->off_gmeta);
   p.gat_part = reinterpret_cast<float*>(w + pl->off_gat);
   p.gat_slots = pl->gat_slots;
   p.dense_part = reinterpret_cast<float*>(w + pl->off_dense);
   p.dense_splits = pl->dense_splits;
-  p.splits = pl->splits;
+  p.stat_splits = pl->stat_splits; p.stat_splits_base = pl->stat_splits_base;
   p.dbg = pl->dbg;
   return VATTN_OK;
 }
@@ -327,6 +345,20 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   Prob p;
   fill_prob(plan, p, q, k_cache, v_cache, block_table, seq_lens, out);
   p.sink = sink; p.window = window; p.k = k;
+  {
+    // statistics kernel: never more CTAs than rows warrant (about 64 deterministic, 48 base-sample rows each)
+    const double msl = (double)plan->shape.max_seq_len;
+    double kmax = plan->params.topk_frac > 0.f ? floor((double)plan->params.topk_frac * msl) : (double)k;
+    double rows = (double)sink + (double)window + kmax;
+    if (rows > msl) rows = msl;
+    int want = (int)((rows + 127.0) / 128.0) * 2;
+    if (want < 1) want = 1;
+    if (want < p.stat_splits) p.stat_splits = want;
+    const double brows = (double)p.base_rate * msl;
+    want = (int)((brows + 95.0) / 96.0) * 2;
+    if (want < 1) want = 1;
+    if (want < p.stat_splits_base) p.stat_splits_base = want;
+  }
   p.seed_lo = (unsigned)(seed & 0xFFFFFFFFull); p.seed_hi = (unsigned)(seed >> 32);
   p.eps = (double)eps; p.delta = (double)delta;
   p.z_delta = upper_quantile(0.5 * p.delta);
@@ -339,8 +371,9 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   if (rc != VATTN_OK) return rc;
   plan->last_launches++;                      // the counter-clearing kernel
   prof_mark(plan, 0, st);
-  // score pass (walk tokens beside it) -> selection and sample lists (one CTA per head) -> deterministic and base-sample rows ->
-  // budget, final sample, combination.  Every kernel is launched with programmatic dependent launch: its prologue
+  // score pass (walk tokens beside it) -> selection and sample lists (one CTA per head) -> deterministic and
+  // base-sample rows (started per head by flags of the selection kernel), budget by the last CTA of a head -> final
+  // sample, combination.  Every kernel is launched with programmatic dependent launch: its prologue
   // runs while its predecessor drains.
   CU(launch_score(p, st));            plan->last_launches++;
   prof_mark(plan, 1, st);
@@ -357,7 +390,7 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
   CU(launch_stats(p, st));            plan->last_launches++;
   prof_mark(plan, 4, st);
   if (plan->stop_after == 4) return VATTN_OK;
-  CU(launch_final(p, st));            plan->last_launches++;
+  CU(launch_gather(p, st));           plan->last_launches++;
   prof_mark(plan, 5, st);
   if (plan->profiling && plan->prof_calls < kProfCalls) plan->prof_calls++;
   return VATTN_OK;

@@ -1,0 +1,361 @@
+// Sampled part of the estimator and the final combination (Sec. 4.1 of the paper):
+//     N = N_f + (n_s/b) * sum_{I_dyn} w_i V[i],   D = D_f + (n_s/b) * sum_{I_dyn} w_i,   out = N / D
+// which is SDPA_{S,p} of Sec. 3 with p = 1 on I_f and p = b/n_s on I_dyn.
+//
+// HBM-bound row gather.  Work unit = a chunk of consecutive entries of one head's I_dyn list.  LPR lanes
+// fetch one V row with one 16-byte load each; a row group keeps 4 rows in flight and requests the next
+// batch's indices (token + physical slot, written by the select kernels) while the current rows arrive.
+// Rows are fetched with streaming loads (read once: first to leave the caches, so that the scores and index
+// lists stay in L2).  Weights come from the stored fp32 scores (no K re-read).  Partials are added in chunk order by the
+// last CTA of the head ("ticket"), so results are reproducible.
+//
+// Two decompositions:
+//  * flat (batch * heads <= 128): budgets differ a lot between heads, so the chunks of all heads form one
+//    list (a prefix sum over the heads' chunk counts, recomputed by every CTA) that the CTAs walk with a
+//    grid stride.  A chunk is a whole number of batches (a batch = what one CTA keeps in flight at once:
+//    32 rows of 128 bf16) and a head uses up to 32 chunks (64 to 128 when no more than 18 heads share the
+//    grid): lists of more batches than that get chunks of
+//    two, three, ... batches, whose index loads overlap the previous batch's rows.  (With up to 128
+//    single-batch chunks per head the last finisher needed three dependent rounds of partial loads and
+//    long lists overflowed the grid: 92 -> 76 us per step at 5x density, 73.0 -> 72.4 us at 10x.);
+//  * per head (larger problems): grid (32, heads, batch); a head with budget b uses ceil(b / chunk) of its
+//    32 CTAs, chunk = max(256, ceil(b / 32)) rows, the others exit at once.
+#include "vattn_internal.cuh"
+#include <type_traits>
+
+namespace {
+
+// what this kernel needs of a head, as the statistics kernel left it (16 bytes: the table of all heads is four cache
+// lines at 32 heads, and every CTA reads all of it)
+// b: the budget; L: entries to visit (a prefix of the final sample's walk array, members of I_t marked, or the b
+// entries of the head's list when `list` is set); n = 0: an empty row
+struct GMeta { int b, n_s; float m; int n, L, list; };
+__device__ __forceinline__ GMeta ld_gmeta(const int4* g) {
+  const int4 v = __ldcg(g);
+  GMeta r; r.b = v.x; r.n_s = v.y; r.m = __int_as_float(v.z);
+  r.n = v.w < 0 ? 0 : 1; r.L = v.w < 0 ? 0 : (v.w >> 1); r.list = v.w < 0 ? 0 : (v.w & 1);
+  return r;
+}
+
+constexpr int NT = 128;
+constexpr int NWARP = NT / 32;
+constexpr int UNROLL = 4;         // rows in flight per row group (16-byte slices kept raw until used); 8 and 2 are slower
+constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
+constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
+constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
+
+template <typename T, int D, bool KV>
+struct Gather {
+  static constexpr int EPL = Elem<T>::EPL, LPR = D / EPL, RPI = 32 / LPR, NE = D + 1, RG = NWARP * RPI;
+  static_assert(LPR >= UNROLL, "each row of a batch needs a lane of its row group to own its weight");
+
+  static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[EPL]) {
+    if (EPL == 8) {
+      v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xFFFF0000u);
+      v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xFFFF0000u);
+      v[4 % EPL] = __uint_as_float(r.z << 16); v[5 % EPL] = __uint_as_float(r.z & 0xFFFF0000u);
+      v[6 % EPL] = __uint_as_float(r.w << 16); v[7 % EPL] = __uint_as_float(r.w & 0xFFFF0000u);
+    } else {
+      v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
+  }
+  // rows [r_begin, r_end) of head bh -> partial `slot`; the last of `nslots` finishers combines
+  static __device__ void run(const Prob& p, int bh, const GMeta& meta, int r_begin, int r_end, int slot, int nslots,
+                             float (*part)[NE], int* is_last, float* s_den) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int h = bh % p.Hq, g = h / p.G;
+    T* out = reinterpret_cast<T*>(p.out) + (long long)bh * D;
+    if (meta.n == 0) {
+      if (slot == 0) for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
+      return;
+    }
+    // I_dyn: the unmarked entries of a prefix of the final sample's walk array (a marked entry, token -1, is a
+    // member of I_t: its row is fetched like the others and weighs nothing), or the head's list
+    const int* dyn = meta.list ? p.dyn_idx + (long long)bh * 3 * p.npad : p.walk_tok + ((long long)bh * 4 + 2) * p.npad;
+    const int* dph = dyn + p.npad;
+    const float* sc = p.scores + (long long)bh * p.npad;
+    const T* vc = reinterpret_cast<const T*>(p.vc) + (long long)g * p.sh;
+    const float m = meta.m;
+    const int rsub = lane / LPR, j = lane % LPR;
+    const int rg = warp * RPI + rsub;
+    const int iters = (r_end - r_begin + RG - 1) / RG;
+
+    float acc[EPL], dd = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+
+    // A batch = UNROLL rows per row group.  Batches whose rows all exist (every one but a chunk's last) run a
+    // body without per-row validity tests; FULL is a compile-time tag.
+    const int full_iters = ((r_end - r_begin) / (RG * UNROLL)) * UNROLL;
+    int tok_n[UNROLL], ph_n[UNROLL];
+    auto fetch_idx = [&](int k0, auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const int r = r_begin + rg + (k0 + u) * RG;
+        const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
+        tok_n[u] = ok ? __ldg(dyn + r) : -1;
+        ph_n[u] = ok ? __ldg(dph + r) : 0;
+      }
+    };
+    auto fetch_next = [&](int k0) {                   // indices of the batch that starts at iteration k0, if any
+      if (k0 >= iters) return;
+      if (k0 + UNROLL <= full_iters) fetch_idx(k0, std::true_type{});
+      else fetch_idx(k0, std::false_type{});
+    };
+    // K+V variant: the score of a sampled token is recomputed from its K row (what a selector that leaves no
+    // scores for the whole context behind would need); the K slices of a batch come first, then its V slices
+    float qf[EPL];
+    const T* kcg = reinterpret_cast<const T*>(p.kc) + (long long)g * p.sh;
+    if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+    auto batch = [&](int k0, auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
+      // lane u of a row group owns row u's weight: one score load and one exp per row instead of LPR
+      int tok[UNROLL], tok_mine = -1;
+      float w_mine = 0.f;
+      uint4 raw[UNROLL];
+      if (KV) {
+        long long off[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          tok[u] = tok_n[u];
+          const int ph = ph_n[u];
+          off[u] = (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL;
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(kcg + off[u]));
+        }
+        fetch_next(k0 + UNROLL);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          float kv[EPL], dot = 0.f;
+          unpack(raw[u], kv);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kv[e], dot);
+#pragma unroll
+          for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
+          if (j == u) { w_mine = p.scale * dot; tok_mine = tok[u]; }
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + off[u]));
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          tok[u] = tok_n[u];
+          if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (j == u) tok_mine = tok[u];
+          if (FULL || tok[u] >= 0) {
+            const int ph = ph_n[u];
+            raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL));
+          }
+        }
+        if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);
+        fetch_next(k0 + UNROLL);                        // next batch's indices travel with this batch's rows
+      }
+      const float e_mine = (tok_mine >= 0) ? expf(w_mine - m) : 0.f;
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const float ww = __shfl_sync(0xFFFFFFFFu, e_mine, u, LPR);
+        dd += ww;
+        float v[EPL];
+        unpack(raw[u], v);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(ww, v[e], acc[e]);
+      }
+    };
+    fetch_next(0);
+    for (int k0 = 0; k0 < iters; k0 += UNROLL) {
+      if (k0 + UNROLL <= full_iters) batch(k0, std::true_type{});   // uniform over the CTA
+      else batch(k0, std::false_type{});
+    }
+#pragma unroll
+    for (int mask = LPR; mask < 32; mask <<= 1) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], mask);
+      dd += __shfl_xor_sync(0xFFFFFFFFu, dd, mask);
+    }
+    __syncthreads();                                  // `part` may still be read by the previous chunk
+    DBGT(22);
+    if (rsub == 0) {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) part[warp][j * EPL + e] = acc[e];
+      if (j == 0) part[warp][D] = dd;
+    }
+    __syncthreads();
+    float* gpart = p.gat_part + ((long long)bh * p.gat_slots + slot) * NE;
+    for (int e = tid; e < NE; e += NT) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) s += part[w][e];
+      gpart[e] = s;
+    }
+    // (the barrier orders every thread's writes before thread 0's fence, which is cumulative; likewise on the way in)
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      *is_last = (atomicAdd(&p.tickets[p.B * p.Hq + bh], 1u) == (unsigned)(nslots - 1));
+      __threadfence();
+    }
+    __syncthreads();
+    DBGT(23);
+    if (!*is_last) return;
+
+    // last finisher of the head: every thread requests all partials of its element at once (one memory
+    // round trip), adds them in slot order, scales by n_s/b and divides
+    const int nb = meta.b;
+    const double* det = p.det_sums + (long long)bh * (D + 1);
+    const double f = (nb > 0) ? (double)meta.n_s / (double)nb : 0.0;
+    const float* src0 = p.gat_part + (long long)bh * p.gat_slots * NE;
+    float num_s[(D + NT - 1) / NT];
+    double det_e[(D + NT - 1) / NT];
+    const double det_d = __ldcg(det + D);             // N_f, D_f of the statistics kernel, requested with the partials
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) det_e[it] = (tid + it * NT < D) ? __ldcg(det + tid + it * NT) : 0.0;
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) {
+      const int e = tid + it * NT;
+      float s = 0.f;
+      for (int s0 = 0; s0 < nslots; s0 += 32) {       // 32 partials per round trip, added in slot order
+        float vv[32];
+#pragma unroll
+        for (int sp = 0; sp < 32; ++sp) vv[sp] = (s0 + sp < nslots && e < D) ? __ldcg(src0 + (long long)(s0 + sp) * NE + e) : 0.f;
+#pragma unroll
+        for (int sp = 0; sp < 32; ++sp) s += vv[sp];
+      }
+      num_s[it] = s;
+    }
+    if (warp == 0) {                                  // the denominator: lane sp holds slot s0 + sp
+      float s = 0.f;
+      for (int s0 = 0; s0 < nslots; s0 += 32) {
+        const float vd = (s0 + lane < nslots) ? __ldcg(src0 + (long long)(s0 + lane) * NE + D) : 0.f;
+#pragma unroll
+        for (int sp = 0; sp < 32; ++sp) s += __shfl_sync(0xFFFFFFFFu, vd, sp);
+      }
+      if (lane == 0) *s_den = s;
+    }
+    __syncthreads();
+    const double den = det_d + f * (double)(*s_den);
+#pragma unroll
+    for (int it = 0; it < (D + NT - 1) / NT; ++it) {
+      const int e = tid + it * NT;
+      if (e < D) out[e] = Elem<T>::from_float((float)((det_e[it] + f * (double)num_s[it]) / den));
+    }
+  }
+};
+
+template <typename T, int D, bool KV>
+__global__ void __launch_bounds__(NT, KV ? 8 : 10) k_gather(const Prob p) {
+  using G = Gather<T, D, KV>;
+  __shared__ float part[NWARP][G::NE];
+  __shared__ int is_last;
+  __shared__ float s_den;
+  TICK_BEGIN(p, VATTN_K_GATHER);
+  pdl_wait();
+  const int bh = blockIdx.z * p.Hq + blockIdx.y;
+  const GMeta meta = ld_gmeta(p.gat_meta + bh);
+  const int nb = meta.n > 0 ? meta.L : 0;              // entries to visit
+  // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
+  // (with this many heads the kernel is throughput-bound: 4 batches per row group amortise the fixed hops)
+  const int chunk = max(4 * MIN_CHUNK, (nb + MAXS - 1) / MAXS);
+  const int nslots = max(1, (nb + chunk - 1) / chunk);
+  if ((int)blockIdx.x >= nslots) return;
+  const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
+  G::run(p, bh, meta, r_begin, r_end, blockIdx.x, nslots, part, &is_last, &s_den);
+  TICK_END(p, VATTN_K_GATHER);
+}
+
+template <typename T, int D, bool KV>
+__global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
+  using G = Gather<T, D, KV>;
+  __shared__ float part[NWARP][G::NE];
+  __shared__ int is_last;
+  __shared__ float s_den;
+  __shared__ int s_pref[FLAT_MAX_HEADS + 1], s_rows[FLAT_MAX_HEADS], s_b[FLAT_MAX_HEADS], s_w[NWARP];
+  __shared__ GMeta s_meta[FLAT_MAX_HEADS];
+  TICK_BEGIN(p, VATTN_K_GATHER);
+  pdl_wait();
+  DBGT(20);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int BH = p.B * p.Hq;
+  // chunk counts of all heads and their prefix sum (every CTA computes the same numbers)
+  constexpr int BATCH = G::RG * UNROLL;               // rows a CTA keeps in flight at once
+  int nb = 0, rows = BATCH, cnt = 0;
+  if (tid < BH) {
+    const GMeta mt = ld_gmeta(p.gat_meta + tid);
+    s_meta[tid] = mt;
+    nb = mt.n > 0 ? mt.L : 0;                          // entries to visit
+    const int batches = (nb + BATCH - 1) / BATCH;
+    rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
+    cnt = max(1, (nb + rows - 1) / rows);             // a head without samples still writes its output
+    s_rows[tid] = rows;
+    s_b[tid] = nb;
+  }
+  int incl = cnt;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += v;
+  }
+  if (lane == 31) s_w[warp] = incl;
+  __syncthreads();
+  int before = 0;
+  for (int w = 0; w < warp; ++w) before += s_w[w];
+  if (tid < BH) s_pref[tid] = before + incl - cnt;
+  if (tid == NT - 1) s_pref[BH] = before + incl;      // BH <= NT: the last thread's inclusive sum is the total
+  __syncthreads();
+  const int total = s_pref[BH];
+  DBGT(21);
+#ifdef VATTN_PHASE_TICKS
+  if (p.dbg.kernel_ticks && tid == 0) p.dbg.kernel_ticks[2 * (64 + blockIdx.x)] = gtime_ns();
+#endif
+  // CTAs with neighbouring indices tend to share an SM (an SM that the kernel before has just left takes the next
+  // eight), and chunks with neighbouring numbers belong to one head, so all of them are long or all short: deal the
+  // chunks out with a stride instead, c0 -> (c0 mod 8) * ceil(total / 8) + c0 / 8
+  const int q8 = (total + 7) >> 3;
+  for (int c0 = blockIdx.x; c0 < 8 * q8; c0 += gridDim.x) {
+    const int c = (c0 & 7) * q8 + (c0 >> 3);
+    if (c >= total) continue;
+    int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (s_pref[mid] <= c) lo = mid; else hi = mid - 1;
+    }
+    const int bh = lo, ci = c - s_pref[bh];
+    const int r_begin = min(s_b[bh], ci * s_rows[bh]), r_end = min(s_b[bh], r_begin + s_rows[bh]);
+    G::run(p, bh, s_meta[bh], r_begin, r_end, ci, s_pref[bh + 1] - s_pref[bh], part, &is_last, &s_den);
+    __syncthreads();
+#ifdef VATTN_PHASE_TICKS
+    if (p.dbg.kernel_ticks && tid == 0) {
+      p.dbg.kernel_ticks[2 * (64 + blockIdx.x) + 1] = gtime_ns();
+      p.dbg.kernel_ticks[2 * (64 + 1200 + blockIdx.x)] = (unsigned long long)(r_end - r_begin);
+      p.dbg.kernel_ticks[2 * (64 + 1200 + blockIdx.x) + 1] = (unsigned long long)bh;
+    }
+#endif
+  }
+  TICK_END(p, VATTN_K_GATHER);
+}
+
+}  // namespace
+
+template <typename T, int D, bool KV>
+static cudaError_t launch_gather_t(const Prob& p, cudaStream_t s) {
+  const int BH = p.B * p.Hq;
+  if (BH <= FLAT_MAX_HEADS) {
+    // at most gat_slots chunks per head; 8 CTAs per SM walk them with a grid stride
+    if (p.gat_slots < VATTN_GATHER_FLAT_SLOTS) return cudaErrorInvalidValue;
+    const long long most = (long long)BH * p.gat_slots;
+    const long long cap = 8ll * device_sm_count();
+    const int grid = (int)(most < cap ? most : cap);
+    return launch_pdl(k_gather_flat<T, D, KV>, dim3(grid), dim3(NT), 0, s, p);
+  }
+  if (p.gat_slots < MAXS) return cudaErrorInvalidValue;
+  return launch_pdl(k_gather<T, D, KV>, dim3(MAXS, p.Hq, p.B), dim3(NT), 0, s, p);
+}
+
+cudaError_t launch_gather(const Prob& p, cudaStream_t s) {
+  if (p.dtype == VATTN_DTYPE_BF16) {
+    if (p.D == 128) return p.gather_kv ? launch_gather_t<bf16_t, 128, true>(p, s) : launch_gather_t<bf16_t, 128, false>(p, s);
+    return p.gather_kv ? launch_gather_t<bf16_t, 64, true>(p, s) : launch_gather_t<bf16_t, 64, false>(p, s);
+  }
+  if (p.D == 128) return p.gather_kv ? launch_gather_t<float, 128, true>(p, s) : launch_gather_t<float, 128, false>(p, s);
+  return p.gather_kv ? launch_gather_t<float, 64, true>(p, s) : launch_gather_t<float, 64, false>(p, s);
+}

@@ -26,11 +26,7 @@
 #include "vattn_internal.cuh"
 #include <math_constants.h>
 
-#ifdef VATTN_PHASE_TICKS
-#define DBGT(k) do { TICK_BEGIN(p, 8 + (k)); TICK_END(p, 8 + (k)); } while (0)
-#else
-#define DBGT(k) do { } while (0)
-#endif
+
 
 namespace {
 
@@ -289,12 +285,15 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   HeadMeta mt;
   mt.n = n; mt.s0 = s0; mt.l_start = l_start; mt.kk = kk; mt.n_s = n_s; mt.b0 = b0;
   mt.nbt = 0; mt.band_mode = 0; mt.m = 0.f; mt.hi = CUDART_INF_F; mt.lo = CUDART_INF_F;
-  mt.run1 = 0; mt.dyn_listed = 0; mt.dyn_J = 0; mt.path = 0; mt.pad = 0;
+  mt.run1 = 0; mt.dyn_listed = 0; mt.dyn_J = 0; mt.path = 0; mt.b = 0;
   if (n == 0) {
     pdl_wait();
     pdl_trigger();
     if (tid == 0) {
+      mt.base_J = 0; mt.base_piv = 0; mt.base_list = 0; mt.holes1 = 0;
       p.meta[bh] = mt;
+      __threadfence();
+      asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(2ull) : "memory");
       if (p.dbg.topk_cnt) p.dbg.topk_cnt[bh] = 0;
       if (p.dbg.base_cnt) p.dbg.base_cnt[bh] = 0;
       if (p.dbg.paths) p.dbg.paths[bh] = 0;
@@ -311,6 +310,8 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     for (int mk = 16; mk >= 1; mk >>= 1) sa += __shfl_xor_sync(FULL, sa, mk);
   }
   for (int w = tid; w < ((n + 31) >> 5); w += NT) gbitmap[w] = 0u;     // only the overflow path sets and reads bits
+  // the first entries of the head's list of marked positions are read unconditionally by the budget: "none" until set
+  if (tid < 256) p.hole_pos[(long long)bh * VATTN_BANDCAP + tid] = 0x7FFFFFFF;
 
   pdl_wait();                                          // the score pass is complete: scores, maxima
   pdl_trigger();
@@ -654,9 +655,15 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   mt.hi = hi; mt.lo = lo; mt.nbt = band_mode ? 0 : nbt; mt.band_mode = band_mode; mt.run1 = run1; mt.path = path;
   TICK_END(p, VATTN_T_TOPK);
 
-  // the near-tie list for the row kernels
+  // the near-tie list for the budget's list path
   int* gvtab = p.vtab + (long long)bh * VATTN_BANDCAP;
   for (int c = tid; c < mt.nbt; c += NT) gvtab[c] = sm.vtab[c];
+  if (tid == 0) {
+    if (p.dbg.topk_cnt) p.dbg.topk_cnt[bh] = kk;
+    if (p.dbg.base_cnt) p.dbg.base_cnt[bh] = b0;
+    if (p.dbg.paths) p.dbg.paths[bh] = path;
+  }
+  __syncthreads();                                     // the list of I_t is read back below (through L2: ld.cg)
   if (p.dbg.topk_idx) {
     // I_t ascending for the debug buffer: two ascending runs merged by rank
     __threadfence();
@@ -671,24 +678,95 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     }
   }
 
-  // ------------------------------------------------------------------ walks: the base sample, the head of the final sample
-  // A thread evaluates WPT consecutive walk positions; the rank of a residual token is a prefix sum away.
-  // Round of walk `stream`: list the residual tokens of rank [have, want) found at positions [J, Jn).
-  // Rounds of 4096 walk positions, four consecutive ones per thread (one 16-byte read of the tokens computed
-  // ahead); the rank of a residual token is a prefix sum away.  Listed entries are staged in shared memory in rank
-  // order and written out with consecutive threads on consecutive words.
-  int* bl_tok = p.base_idx + (long long)bh * 2 * p.npad;
-  int* dl_tok = p.dyn_idx + (long long)bh * 3 * p.npad;
+  // ------------------------------------------------------------------ the samples
+  // uniform-sample(R, c) is the first c residual tokens of a walk of the middle range.  The walk kernel left the
+  // first positions of both walks (tokens, physical slots) in the walk arrays; what is missing is which of those
+  // tokens are members of I_t.  Each member's walk position is sigma^-1(token): the member is marked there (token =
+  // -1), and a sample of c residual tokens becomes "the unmarked entries among the first J", J = c + the number of
+  // marked positions below J (a fixed point reached in a few steps).  No list is compacted; the row kernels skip
+  // marked entries.  For the final sample (c = the budget, not known yet) the marked positions are left in hole_pos.
+  int* wa0 = p.walk_tok + (long long)bh * 4 * p.npad;            // base sample's walk: tokens (slots at + npad)
+  int* wa1 = wa0 + 2 * p.npad;                                   // final sample's walk
+  const int W0 = walk_region(n_s > 0 ? b0 : 0, n_s, mlen, kk);   // entries the walk kernel wrote
+  const int W1 = walk_region(dyn_listed_want(p, n_s, b0), n_s, mlen, kk);
+  int* hp0 = sm.hist;                                  // marked positions of the base walk (over the histograms)
+  int* cnts = sm.misc + 8;                             // [0] marked positions of the base walk, [1] of the final walk
+  int base_J = 0, base_list = 0, holes1 = 0, dyn_J = 0, dyn_listed = 0, piv_ph = 0;
+  if (n_s > 0 && kk <= NT * 4) {
+    int* hp1 = p.hole_pos + (long long)bh * VATTN_BANDCAP;
+    // physical slots of the first entries of the base walk: one of them is the pivot (the first unmarked entry)
+    int pvph = 0;
+    if (warp == 0 && lane < 4 && lane < W0) pvph = __ldcg(wa0 + p.npad + lane);
+    if (tid == 0) { cnts[0] = 0; cnts[1] = 0; }
+    const Walk wk0 = make_walk(sm.rkeys + (p.nested_base ? 8 : 0), mlen), wk1 = make_walk(sm.rkeys + 8, mlen);
+    __syncthreads();
+    DBGT(16);
+    for (int a = tid; a < kk; a += NT) {
+      const int t = __ldcg(tk + a) - s0;
+      const int x1 = walk_inv(wk1, t);
+      const int x0 = p.nested_base ? x1 : walk_inv(wk0, t);
+      if (x0 < W0) {
+        wa0[x0] = -1;
+        const int i0 = atomicAdd(&cnts[0], 1);
+        if (i0 < HBINS) hp0[i0] = x0;
+      }
+      if (x1 < W1) {
+        wa1[x1] = -1;
+        const int i1 = atomicAdd(&cnts[1], 1);
+        if (i1 < VATTN_BANDCAP) hp1[i1] = x1;
+      }
+    }
+    __syncthreads();
+    DBGT(17);
+    const int H0 = cnts[0];
+    holes1 = cnts[1];
+    if (H0 > HBINS) base_list = 1;
+    else if (warp == 0) {
+      // J = b0 + #{marked positions < J}; the pivot = the first unmarked position
+      int J = b0;
+      for (int it = 0; it < 64; ++it) {
+        int c = 0;
+        for (int i = lane; i < H0; i += 32) c += hp0[i] < J;
+#pragma unroll
+        for (int mk = 16; mk >= 1; mk >>= 1) c += __shfl_xor_sync(FULL, c, mk);
+        if (b0 + c == J) break;
+        J = b0 + c;
+      }
+      int pivx = 0;
+      for (int it = 0; it < 64; ++it) {
+        int hit = 0;
+        for (int i = lane; i < H0; i += 32) hit |= hp0[i] == pivx;
+        if (!__any_sync(FULL, hit)) break;
+        ++pivx;
+      }
+      int ph = __shfl_sync(FULL, pvph, pivx & 3);
+      if (pivx >= 4 && pivx < W0) ph = __ldcg(wa0 + p.npad + pivx);
+      if (lane == 0) { sm.misc[4] = J; sm.misc[5] = ph; sm.misc[6] = (J > W0 || pivx >= W0) ? 1 : 0; }
+    }
+    __syncthreads();
+    if (!base_list) { base_J = sm.misc[4]; piv_ph = sm.misc[5]; base_list = sm.misc[6]; }
+    if (holes1 <= VATTN_BANDCAP) { dyn_J = W1; dyn_listed = W1 - holes1; }
+  } else if (n_s > 0) {
+    base_list = 1;
+  }
+  if (base_J >= (1 << 22)) base_list = 1;              // the published word has 22 bits for it
+  mt.base_J = base_J; mt.base_piv = 0; mt.base_list = base_list; mt.holes1 = min(holes1, VATTN_BANDCAP);
+  mt.dyn_J = dyn_J; mt.dyn_listed = dyn_listed;
+  DBGT(6);
+
+  // The base sample as a list: for the debug buffer, and for the row kernels when the walk array fell short.
+  // Rounds of 4096 walk positions, four consecutive ones per thread; the rank of a residual token is a prefix sum
+  // away.  Listed entries are staged in shared memory in rank order and written out with consecutive threads on
+  // consecutive words.
   int* bdbg = p.dbg.base_idx ? p.dbg.base_idx + (long long)bh * p.max_seq_len : nullptr;
-  int* st_tok = sm.hist, * st_ph = sm.hist + LROUND, * st_sc = sm.hist + 2 * LROUND;    // over the histograms and candidates
-  __syncthreads();
-#pragma unroll 1
-  for (int which = 0; which < 2; ++which) {            // 0: base sample, 1: head of the final sample's walk
-    // how many residual tokens to list: the base sample exactly; of the final sample as many as budgets usually need
-    const int want = which == 0 ? (n_s > 0 ? b0 : 0) : dyn_listed_want(p, n_s, b0);
-    const Walk wk = make_walk(sm.rkeys + ((which == 1 || p.nested_base) ? 8 : 0), mlen);
-    const int* pre = p.walk_tok + ((long long)bh * 2 + which) * p.npad;       // tokens of the first Jpre positions
-    const int Jpre = walk_region(want, n_s, mlen, kk);
+  if (n_s > 0 && (base_list || bdbg)) {
+    int* bl_tok = p.base_idx + (long long)bh * 2 * p.npad;
+    int* st_tok = sm.hist, * st_ph = sm.hist + LROUND;
+    __syncthreads();                                   // marks in the walk array are read back below (ld.cg)
+    const int want = b0;
+    const Walk wk = make_walk(sm.rkeys + (p.nested_base ? 8 : 0), mlen);
+    const int* pre = wa0;
+    const int Jpre = W0;
     int have = 0, J = 0;
 #pragma unroll 1
     while (have < want && J < mlen) {
@@ -696,69 +774,54 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
       int Jn = J < Jpre ? Jpre : J + walk_region(want - have, n_s, mlen, kk);
       Jn = min(min(Jn, mlen), J + LROUND);
       const int j0 = J + tid * 4;
-      int tokc[4], phc[4]; float svc[4];
-      {
-        uint4 t4 = make_uint4(0u, 0u, 0u, 0u);
-        if (j0 < Jn && j0 < Jpre) t4 = __ldcg(reinterpret_cast<const uint4*>(pre + j0));
-        const unsigned tq[4] = {t4.x, t4.y, t4.z, t4.w};
-#pragma unroll
-        for (int q_ = 0; q_ < 4; ++q_) {
-          const int jj = j0 + q_;
-          tokc[q_] = -1;
-          if (jj < Jn) tokc[q_] = jj < Jpre ? (int)tq[q_] : s0 + walk_at(wk, jj);
-        }
-      }
+      int tokc[4], phc[4];
 #pragma unroll
       for (int q_ = 0; q_ < 4; ++q_) {
-        svc[q_] = 0.f; phc[q_] = 0;
-        if (tokc[q_] >= 0) {
-          svc[q_] = cached ? unord_f32(~keys[key_slot(tokc[q_])]) : __ldg(sc + tokc[q_]);
-          phc[q_] = __ldg(p.bt + (long long)b * p.max_blocks + (tokc[q_] >> 4));
+        const int jj = j0 + q_;
+        tokc[q_] = -1; phc[q_] = 0;
+        if (jj < Jn) {
+          // (a marked entry reads -1; with too many members for marking, none is marked: test them all)
+          const int tok = jj < Jpre ? __ldcg(pre + jj) : s0 + walk_at(wk, jj);
+          if (tok >= 0) {
+            const float sv = cached ? unord_f32(~keys[key_slot(tok)]) : __ldg(sc + tok);
+            if (!in_topk(mt, sm.vtab, gbitmap, tok, sv)) tokc[q_] = tok;
+          }
+          if (tokc[q_] >= 0) phc[q_] = page_of(p, b, tokc[q_] >> 4);
         }
       }
       int cnt = 0;
 #pragma unroll
-      for (int q_ = 0; q_ < 4; ++q_) {
-        if (tokc[q_] >= 0) {
-          if (in_topk(mt, sm.vtab, gbitmap, tokc[q_], svc[q_])) tokc[q_] = -1; else ++cnt;
-        }
-      }
-      DBGT(12 + which);
+      for (int q_ = 0; q_ < 4; ++q_) cnt += tokc[q_] >= 0;
       int tot1;
       int idx = block_scan_reg(cnt, sm.misc + 32, tot1);          // rank inside the round
-      DBGT(14 + which);
-      // the base sample ends at rank b0; of the final sample's walk every residual token of the positions
-      // evaluated is listed, so that "listed" and "positions covered" describe the same prefix of the walk
-      const int nlist = which == 1 ? tot1 : min(tot1, want - have);
+      const int nlist = min(tot1, want - have);
 #pragma unroll
       for (int q_ = 0; q_ < 4; ++q_) {
         if (tokc[q_] >= 0) {
-          if (idx < nlist) {
-            int pg = phc[q_];
-            if ((unsigned)pg >= (unsigned)p.num_blocks) { atomicOr(p.status, VATTN_STATUS_BAD_BLOCK); pg = 0; }
-            st_tok[idx] = tokc[q_]; st_ph[idx] = pg * VATTN_BLOCK + (tokc[q_] & 15); st_sc[idx] = __float_as_int(svc[q_]);
-          }
+          if (idx < nlist) { st_tok[idx] = tokc[q_]; st_ph[idx] = phc[q_] * VATTN_BLOCK + (tokc[q_] & 15); }
           ++idx;
         }
       }
       __syncthreads();
       for (int x = tid; x < nlist; x += NT) {
         const int r_ = have + x;
-        if (which == 0) { bl_tok[r_] = st_tok[x]; bl_tok[p.npad + r_] = st_ph[x]; if (bdbg) bdbg[r_] = st_tok[x]; }
-        else { dl_tok[r_] = st_tok[x]; dl_tok[p.npad + r_] = st_ph[x]; dl_tok[2 * p.npad + r_] = st_sc[x]; }
+        bl_tok[r_] = st_tok[x]; bl_tok[p.npad + r_] = st_ph[x];
+        if (bdbg) bdbg[r_] = st_tok[x];
       }
       have += tot1;
       J = Jn;
       __syncthreads();
     }
-    DBGT(6 + which);
-    if (which == 1) { mt.dyn_listed = have; mt.dyn_J = J; }
   }
+  // the head's record, then "I_t is written and marked" for the statistics kernel.  The barrier orders every
+  // thread's writes before thread 0's release, which is cumulative: one fence, not one per thread.
+  __syncthreads();
   if (tid == 0) {
     p.meta[bh] = mt;
-    if (p.dbg.topk_cnt) p.dbg.topk_cnt[bh] = kk;
-    if (p.dbg.base_cnt) p.dbg.base_cnt[bh] = b0;
-    if (p.dbg.paths) p.dbg.paths[bh] = path;
+    __threadfence();
+    const unsigned long long word = 2ull | ((unsigned long long)base_list << 2) | ((unsigned long long)(unsigned)base_J << 3) |
+                                    ((unsigned long long)(unsigned)piv_ph << 32);
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(word) : "memory");
   }
   TICK_END(p, VATTN_K_SELECT);
 }
@@ -782,10 +845,14 @@ __global__ void __launch_bounds__(256) k_walk(const Prob p) {
     const int J0 = walk_region(geo.b0, geo.n_s, mlen, geo.kk);
     const int J1 = walk_region(dyn_listed_want(p, geo.n_s, geo.b0), geo.n_s, mlen, geo.kk);
     const Walk w0 = make_walk(keys + (p.nested_base ? 8 : 0), mlen), w1 = make_walk(keys + 8, mlen);
-    int* out0 = p.walk_tok + (long long)bh * 2 * p.npad;
+    int* out0 = p.walk_tok + (long long)bh * 4 * p.npad;       // [walk][tokens, physical slots][npad]
     for (int x = blockIdx.x * 256 + tid; x < J0 + J1; x += gridDim.x * 256) {
-      if (x < J0) out0[x] = geo.s0 + walk_at(w0, x);
-      else out0[p.npad + (x - J0)] = geo.s0 + walk_at(w1, x - J0);
+      const bool first = x < J0;
+      const int xx = first ? x : x - J0;
+      const int tok = geo.s0 + walk_at(first ? w0 : w1, xx);
+      int* dst = out0 + (first ? 0 : 2 * p.npad) + xx;
+      dst[0] = tok;
+      dst[p.npad] = page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15);
     }
   }
   TICK_END(p, VATTN_K_WALK);

@@ -8,8 +8,9 @@
 #define VATTN_MAX_SEQ (1 << 18)        // longest sequence a plan accepts
 #define VATTN_BANDCAP 1024             // near-tie top-k candidates ranked from a list (more: exact radix select)
 #define SEL_THREADS 1024               // threads of the selection kernel (one CTA per head)
-#define ROW_THREADS 256                // threads of the row kernels
-#define VATTN_MAX_SPLITS 16            // most CTAs per head of the row kernels
+#define VATTN_STAT_MAXS 16             // most split CTAs per head and row kind of the statistics kernel
+#define VATTN_GATHER_FLAT_HEADS 128    // the gather kernel's flat decomposition serves up to this many heads ...
+#define VATTN_GATHER_FLAT_SLOTS 32     // ... with up to this many chunks (partials) each
 
 // Per (batch row, query head) record, written by the selection kernel for the row kernels.
 struct HeadMeta {
@@ -24,10 +25,14 @@ struct HeadMeta {
   float m;          // largest fp32 score of the head (softmax stabiliser)
   float hi, lo;     // a middle token is in I_t if its score is above hi; scores in [lo, hi] are near-ties
   int run1;         // the list of I_t is two ascending runs: [0, run1) and [run1, kk)
-  int dyn_listed;   // residual tokens of the final sample's walk that the selection kernel listed ...
-  int dyn_J;        // ... and the walk positions they cover
+  int dyn_listed;   // residual tokens among the first dyn_J positions of the final sample's walk: budgets up to
+  int dyn_J;        //   this many are served from the walk arrays (members of I_t marked), larger ones from a list
   int path;         // code path of the selection (vattn_debug.paths)
-  int pad;
+  int b;            // final budget |I_dyn| (written by the statistics kernel)
+  int base_J;       // the base sample = the unmarked entries among the first base_J of its walk array ...
+  int base_piv;     //   (unused);  base_list = 1: it is in base_idx instead
+  int base_list;    //   (b0 entries, none marked)
+  int holes1;       // marked entries among the first dyn_J of the final sample's walk (their positions in hole_pos)
 };
 
 // Everything a kernel needs, passed by value.
@@ -49,27 +54,33 @@ struct Prob {
   unsigned* m_ord;        // [B,Hq]  order-preserving encoding of the running max score
   unsigned* kabsmax;      // [B,Hkv] bits of max |K element| over the sequence
   unsigned* unit_ctr;     // [1] work-unit counter of the persistent score kernel
-  unsigned* tickets;      // [3,B,Hq] "last CTA done" counters: [0] statistics, [1] final sample, [2] dense kernel
+  unsigned long long* flags64;   // [B,Hq] word the selection kernel publishes per head when I_t is written and marked in
+                          //   the walk arrays: 2 | base_list << 2 | base_J << 3 | pivot's physical slot << 32 (zero: not yet)
+  unsigned* tickets;      // [4,B,Hq] "last CTA done" counters of [1] the gather kernel, [2] the dense kernel and
+                          //          [3] the statistics kernel ([0] unused)
   unsigned* status;       // [1]
   unsigned* bitmap;       // [B,Hq,nwords] near-tie tokens that made it into I_t (used when they are too many for a list)
   int* vtab;              // [B,Hq,BANDCAP] near-tie tokens ascending, bit 31 = member of I_t
   int* topk_idx;          // [B,Hq,2,npad] I_t as two ascending runs, then the physical slot (page * 16 + token % 16) of
                           //               every entry
   int* base_idx;          // [B,Hq,2,npad] I_bs in walk order: tokens, physical slots
-  int* walk_tok;          // [B,Hq,2,npad] tokens of the first walk positions of both walks (computed beside the score pass)
-  int* dyn_idx;           // [B,Hq,3,npad] head of the final sample's walk: tokens, physical slots, fp32 score bits
+  int* walk_tok;          // [B,Hq,2,2,npad] the first positions of both walks (computed beside the score pass): per
+                          //   walk the tokens, then their physical slots.  The selection kernel marks the members
+                          //   of I_t (token = -1; the slot stays valid): a sample is the unmarked entries of a prefix
+  int* hole_pos;          // [B,Hq,VATTN_BANDCAP] positions of the marked entries of the final sample's walk array, in
+                          //   no particular order; the first 256 words read INT_MAX where there is none
+  int* dyn_idx;           // [B,Hq,3,npad] I_dyn as a list (tokens, physical slots) for budgets beyond the walk arrays
                           //               (scratch of the near-tie overflow path while the selection runs)
   HeadMeta* meta;         // [B,Hq]
-  double* stat_part;      // [B,Hq,splits,2,D+3] sums of the statistics kernel: deterministic rows, base-sample rows
+  double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (deterministic-row CTAs, then base-row CTAs)
   double* stat_piv;       // [B,Hq,D+1] pivot row of the base-sample sums: w*V then w
   double* det_sums;       // [B,Hq,D+1] N_f then D_f
-  int* budget;            // [B,Hq] the budget b (written by the statistics kernel)
-  float* gat_part;        // [B,Hq,gat_slots,D+1] sums of the final sample: one slot per unit of listed rows, then one
-                          //                      per CTA of the head for rows beyond the list
-  int gat_slots;
+  int4* gat_meta;         // [B,Hq] what the gather kernel needs of a head: b, n_s, bits of m, n
+  float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
+  int gat_slots;          // partial slots (chunks) per head: 32; 64 to 128 when at most 18 heads share the grid
+  int stat_splits, stat_splits_base;   // statistics CTAs per head: deterministic rows, base-sample rows
   float* dense_part;      // [B,Hq,dense_splits,D+2]
   int dense_splits;
-  int splits;             // CTAs per head of the row kernels
   vattn_debug dbg;
 };
 
@@ -80,15 +91,21 @@ __device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t;
 #define TICK_BEGIN(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMin((p).dbg.kernel_ticks + 2 * (k), gtime_ns()); } while (0)
 #define TICK_END(p, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
 #define TICK_END_IF(p, k, cond) do { if ((p).dbg.kernel_ticks && (cond)) atomicMax((p).dbg.kernel_ticks + 2 * (k) + 1, gtime_ns()); } while (0)
+// measurement builds (-DVATTN_PHASE_TICKS): stamps of phases inside the kernels, rows 8 + k of a larger tick buffer
+#ifdef VATTN_PHASE_TICKS
+#define DBGT(k) do { TICK_BEGIN(p, 8 + (k)); TICK_END(p, 8 + (k)); } while (0)
+#else
+#define DBGT(k) do { } while (0)
+#endif
 // rows of kernel_ticks
 #define VATTN_K_ZERO 0
 #define VATTN_K_SCORE 1
 #define VATTN_K_WALK 2
 #define VATTN_K_SELECT 3
 #define VATTN_K_STATS 4
-#define VATTN_K_FINAL 5
+#define VATTN_K_GATHER 5
 #define VATTN_T_TOPK 6       // [0]: first selection CTA past its dependency wait, [1]: last CTA with I_t complete
-#define VATTN_T_BUDGET 7     // [0]: first final-sample CTA past its dependency wait, [1]: last CTA that knows its budget
+#define VATTN_T_BUDGET 7     // [0]: first head whose statistics are complete, [1]: last head that knows its budget
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
 // stream is still running; it must call pdl_wait() before touching anything the predecessor writes (the
@@ -241,6 +258,21 @@ __device__ __forceinline__ int walk_at(const Walk& w, int j) {
   } while (x >= w.mlen);
   return (int)x;
 }
+// sigma^-1: the walk position at which middle token t (relative to s0) is met
+__device__ __forceinline__ int walk_inv(const Walk& w, int t) {
+  const unsigned ml = (1u << w.lw) - 1u, mr = (1u << w.rw) - 1u;
+  unsigned x = (unsigned)t;
+  do {
+    unsigned L = x >> w.rw, R = x & mr;
+#pragma unroll
+    for (int i = 6; i >= 0; i -= 2) {
+      R ^= mix32(L, w.k[i + 1]) & mr;
+      L ^= mix32(R, w.k[i]) & ml;
+    }
+    x = (L << w.rw) | R;
+  } while (x >= w.mlen);
+  return (int)x;
+}
 // Walk positions expected to hold the first `want` residual tokens, with a margin of four standard deviations
 // (the selection kernel walks on if the margin was not enough).
 __device__ __forceinline__ int walk_region(int want, int n_s, int mlen, int kk) {
@@ -346,12 +378,23 @@ inline cudaError_t optin_smem(KernelT kern, size_t smem, size_t* have, bool pref
   return cudaSuccess;
 }
 
+// HeadMeta through L2 (ld.cg): for kernels that read it before their stream predecessor has completed (after a
+// flag) and therefore cannot count on the launch-boundary L1 invalidation.
+static_assert(sizeof(HeadMeta) == 80, "HeadMeta is read as five 16-byte words");
+__device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
+  union U { HeadMeta m; int4 v[5]; __device__ U() {} } u;
+  const int4* src = reinterpret_cast<const int4*>(g);
+  u.v[0] = __ldcg(src); u.v[1] = __ldcg(src + 1); u.v[2] = __ldcg(src + 2); u.v[3] = __ldcg(src + 3);
+  u.v[4] = __ldcg(src + 4);
+  return u.m;
+}
+
 // launchers (one per translation unit)
 cudaError_t launch_zero(unsigned* z, size_t bytes, bool pdl, bool late, unsigned long long* ticks, cudaStream_t s);
 cudaError_t launch_score(const Prob& p, cudaStream_t s);
 cudaError_t launch_walk(const Prob& p, cudaStream_t s);
 cudaError_t launch_select(const Prob& p, cudaStream_t s);
 cudaError_t launch_stats(const Prob& p, cudaStream_t s);
-cudaError_t launch_final(const Prob& p, cudaStream_t s);
+cudaError_t launch_gather(const Prob& p, cudaStream_t s);
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches);
 int device_sm_count();                                   // SMs of the current device (cached per device)
