@@ -100,8 +100,8 @@ void derive(vattn_plan* pl) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   pl->off_scores = take(BH * pl->npad * sizeof(float));
-  // cleared every step: running maxima [BH], max |K| [B*Hkv], tickets [4*BH], the score kernel's unit counter
-  pl->zero_bytes = align_up((BH + (size_t)s.batch * s.num_kv_heads + 4 * BH + 4) * sizeof(unsigned), 8) + BH * 8;   // ... and the 64-bit words [BH]
+  // cleared every step: running maxima [BH], max |K| [B*Hkv], tickets [5*BH], the score kernel's unit counter
+  pl->zero_bytes = align_up((BH + (size_t)s.batch * s.num_kv_heads + 5 * BH + 4) * sizeof(unsigned), 8) + BH * 8;   // ... and the 64-bit words [BH]
   pl->off_zero = take(pl->zero_bytes);
   pl->off_status = take(sizeof(unsigned));
   pl->off_bitmap = take(BH * pl->nwords * sizeof(unsigned));
@@ -154,7 +154,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
   const size_t BH = (size_t)s.batch * s.num_q_heads;
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
-  p.unit_ctr = p.tickets + 4 * BH;
+  p.unit_ctr = p.tickets + 5 * BH;
   p.flags64 = reinterpret_cast<unsigned long long*>(w + pl->off_zero + pl->zero_bytes - BH * 8);
   p.status = reinterpret_cast<unsigned*>(w + pl->off_status);
   p.bitmap = reinterpret_cast<unsigned*>(w + pl->off_bitmap);

@@ -41,6 +41,7 @@ constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
 constexpr int UNROLL = 4;         // rows in flight per row group (16-byte slices kept raw until used); 8 and 2 are slower
 constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
+constexpr unsigned READY_SPINS = 1u << 16;   // polls of a head's "budget published" word before the grid-level wait takes over
 constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
 constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
 
@@ -198,6 +199,7 @@ struct Gather {
     __syncthreads();
     DBGT(23);
     if (!*is_last) return;
+    DBGH(bh, 5);
 
     // last finisher of the head: every thread requests all partials of its element at once (one memory
     // round trip), adds them in slot order, scales by n_s/b and divides
@@ -269,69 +271,48 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
-  __shared__ int s_pref[FLAT_MAX_HEADS + 1], s_rows[FLAT_MAX_HEADS], s_b[FLAT_MAX_HEADS], s_w[NWARP];
-  __shared__ GMeta s_meta[FLAT_MAX_HEADS];
+  __shared__ unsigned s_ready;
   TICK_BEGIN(p, VATTN_K_GATHER);
-  pdl_wait();
-  DBGT(20);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int BH = p.B * p.Hq;
-  // chunk counts of all heads and their prefix sum (every CTA computes the same numbers)
   constexpr int BATCH = G::RG * UNROLL;               // rows a CTA keeps in flight at once
-  int nb = 0, rows = BATCH, cnt = 0;
-  if (tid < BH) {
-    const GMeta mt = ld_gmeta(p.gat_meta + tid);
-    s_meta[tid] = mt;
-    nb = mt.n > 0 ? mt.L : 0;                          // entries to visit
-    const int batches = (nb + BATCH - 1) / BATCH;
-    rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
-    cnt = max(1, (nb + rows - 1) / rows);             // a head without samples still writes its output
-    s_rows[tid] = rows;
-    s_b[tid] = nb;
-  }
-  int incl = cnt;
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-    if (lane >= off) incl += v;
-  }
-  if (lane == 31) s_w[warp] = incl;
-  __syncthreads();
-  int before = 0;
-  for (int w = 0; w < warp; ++w) before += s_w[w];
-  if (tid < BH) s_pref[tid] = before + incl - cnt;
-  if (tid == NT - 1) s_pref[BH] = before + incl;      // BH <= NT: the last thread's inclusive sum is the total
-  __syncthreads();
-  const int total = s_pref[BH];
-  DBGT(21);
-#ifdef VATTN_PHASE_TICKS
-  if (p.dbg.kernel_ticks && tid == 0) p.dbg.kernel_ticks[2 * (64 + blockIdx.x)] = gtime_ns();
-#endif
-  // CTAs with neighbouring indices tend to share an SM (an SM that the kernel before has just left takes the next
-  // eight), and chunks with neighbouring numbers belong to one head, so all of them are long or all short: deal the
-  // chunks out with a stride instead, c0 -> (c0 mod 8) * ceil(total / 8) + c0 / 8
-  const int q8 = (total + 7) >> 3;
-  for (int c0 = blockIdx.x; c0 < 8 * q8; c0 += gridDim.x) {
-    const int c = (c0 & 7) * q8 + (c0 >> 3);
-    if (c >= total) continue;
-    int lo = 0, hi = BH - 1;                          // last head whose first chunk is <= c
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (s_pref[mid] <= c) lo = mid; else hi = mid - 1;
+  // Work unit u = chunk u / BH of head u % BH: neighbouring CTAs (which tend to share an SM) serve different heads,
+  // whose chunks differ in length.  A head's units start as soon as its budget is published (a per-head word that
+  // the statistics kernel's last CTA of the head releases), not when all budgets are known.  Every CTA of the
+  // statistics kernel had started before this grid was launched (programmatic dependent launch), so the wait
+  // cannot starve; it is bounded all the same and falls back to the grid-level dependency wait.
+  bool waited = false;
+  for (int u = blockIdx.x; u < BH * p.gat_slots; u += gridDim.x) {
+    const int bh = u % BH, ci = u / BH;
+    if (tid == 0) {
+      unsigned v = 0u;
+      if (!waited) {
+        const unsigned* fl = p.tickets + bh;
+        for (unsigned it = 0; it < READY_SPINS; ++it) {     // relaxed polls, one acquire at the end
+          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(fl) : "memory");
+          if (v != 0u) break;
+          __nanosleep(128);
+        }
+        asm volatile("fence.acq_rel.gpu;" ::: "memory");
+      }
+      s_ready = v;
     }
-    const int bh = lo, ci = c - s_pref[bh];
-    const int r_begin = min(s_b[bh], ci * s_rows[bh]), r_end = min(s_b[bh], r_begin + s_rows[bh]);
-    G::run(p, bh, s_meta[bh], r_begin, r_end, ci, s_pref[bh + 1] - s_pref[bh], part, &is_last, &s_den);
     __syncthreads();
-#ifdef VATTN_PHASE_TICKS
-    if (p.dbg.kernel_ticks && tid == 0) {
-      p.dbg.kernel_ticks[2 * (64 + blockIdx.x) + 1] = gtime_ns();
-      p.dbg.kernel_ticks[2 * (64 + 1200 + blockIdx.x)] = (unsigned long long)(r_end - r_begin);
-      p.dbg.kernel_ticks[2 * (64 + 1200 + blockIdx.x) + 1] = (unsigned long long)bh;
+    if (!waited && s_ready == 0u) { pdl_wait(); waited = true; }      // uniform over the CTA
+    DBGT(21);
+    const GMeta meta = ld_gmeta(p.gat_meta + bh);
+    const int nb = meta.n > 0 ? meta.L : 0;            // entries to visit
+    const int batches = (nb + BATCH - 1) / BATCH;
+    const int rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
+    const int nslots = max(1, (nb + rows - 1) / rows); // a head without samples still writes its output
+    if (ci < nslots) {
+      const int r_begin = min(nb, ci * rows), r_end = min(nb, r_begin + rows);
+      G::run(p, bh, meta, r_begin, r_end, ci, nslots, part, &is_last, &s_den);
     }
-#endif
+    __syncthreads();
   }
   TICK_END(p, VATTN_K_GATHER);
+  if (!waited) pdl_wait();                             // "this grid has completed" implies "the one before has"
 }
 
 }  // namespace

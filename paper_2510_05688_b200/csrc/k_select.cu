@@ -294,6 +294,7 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
       p.meta[bh] = mt;
       __threadfence();
       asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(2ull) : "memory");
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + 4 * p.B * p.Hq + bh), "r"(1u) : "memory");
       if (p.dbg.topk_cnt) p.dbg.topk_cnt[bh] = 0;
       if (p.dbg.base_cnt) p.dbg.base_cnt[bh] = 0;
       if (p.dbg.paths) p.dbg.paths[bh] = 0;
@@ -654,6 +655,7 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   }
   mt.hi = hi; mt.lo = lo; mt.nbt = band_mode ? 0 : nbt; mt.band_mode = band_mode; mt.run1 = run1; mt.path = path;
   TICK_END(p, VATTN_T_TOPK);
+  DBGH(bh, 0);
 
   // the near-tie list for the budget's list path
   int* gvtab = p.vtab + (long long)bh * VATTN_BANDCAP;
@@ -664,6 +666,9 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     if (p.dbg.paths) p.dbg.paths[bh] = path;
   }
   __syncthreads();                                     // the list of I_t is read back below (through L2: ld.cg)
+  // "the list of I_t is written": the statistics kernel's deterministic-row CTAs start while the samples are
+  // prepared below (the barrier orders every thread's writes before thread 0's release, which is cumulative)
+  if (tid == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + 4 * p.B * p.Hq + bh), "r"(1u) : "memory");
   if (p.dbg.topk_idx) {
     // I_t ascending for the debug buffer: two ascending runs merged by rank
     __threadfence();
@@ -818,10 +823,10 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   __syncthreads();
   if (tid == 0) {
     p.meta[bh] = mt;
-    __threadfence();
     const unsigned long long word = 2ull | ((unsigned long long)base_list << 2) | ((unsigned long long)(unsigned)base_J << 3) |
                                     ((unsigned long long)(unsigned)piv_ph << 32);
     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(word) : "memory");
+    DBGH(bh, 1);
   }
   TICK_END(p, VATTN_K_SELECT);
 }

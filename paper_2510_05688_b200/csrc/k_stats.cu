@@ -134,6 +134,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   // ---- everything this function reads from memory is requested up front (one round trip): the head's record,
   //      the pivot, and the partials: thread e adds element e of both kinds in split order, threads 0..3 the scalar
   //      sums (kind 0 = deterministic rows: [D] = D_f; kind 1 = base-sample rows: [D] = Sw, [D+1] = Sww, [D+2] = Srr)
+  DBGX(bh, 0);
   HeadMeta mt = ld_meta(p.meta + bh);
   const double* src = p.stat_part + (long long)bh * 2 * MAXS * NE;
   const int S0 = p.stat_splits, S1 = p.stat_splits_base;
@@ -177,6 +178,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   if (tid == 0) piv[D] = b0 > 0 ? pvD : 0.0;
   __syncthreads();
   DBGT(30);
+  DBGX(bh, 1);
   double* det = p.det_sums + (long long)bh * (D + 1);
   for (int e = tid; e < D; e += NT) det[e] = tot[e];
   if (warp == 0) {
@@ -203,6 +205,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
     double sigma2 = 0.0, trace = 0.0, Dhat = Dfv;
     int bD = 0, bN = 0, bS = 0, bf = 0;
+    DBGX(bh, 2);
     if (n_s > 0) {
       const double Swv = __shfl_sync(FULLMASK, sv, 1), Swwv = __shfl_sync(FULLMASK, sv, 2), Srrv = __shfl_sync(FULLMASK, sv, 3);
       // lane 0: the denominator chain A = n_s sigma / D_hat, lane 1: the numerator chain B = n_s sqrt(Tr) / |N_hat|,
@@ -214,6 +217,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
       const double den2 = lane == 0 ? Dhat * Dhat : nn;
       const double ab = (double)n_s * sqrt(var / den2);
       const double A = __shfl_sync(FULLMASK, ab, 0), Bn = __shfl_sync(FULLMASK, ab, 1);
+      DBGX(bh, 3);
       sigma2 = __shfl_sync(FULLMASK, var, 0);
       trace = __shfl_sync(FULLMASK, var, 1);
       // lanes 0..14: the split points of b_SDPA; lane 15: b_D; lane 16: b_N (one body: (c1 A + c2 B)^2, the
@@ -236,7 +240,9 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
     // I_dyn = the unmarked entries among the first J of the final sample's walk array, J = b + the marked
     // positions below J (a fixed point, reached in a few steps); budgets beyond the array take a list (below)
+    DBGX(bh, 4);
     const bool listed = bf > mt.dyn_listed;
+    const int nholes = min(max(mt.holes1, 0), VATTN_BANDCAP);
     int J = bf;
     if (!listed) {
       const int* hd = p.hole_pos + (long long)bh * VATTN_BANDCAP;
@@ -244,18 +250,22 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
         int c = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) c += __popc(__ballot_sync(FULLMASK, hp[i] < J));
-        for (int i0 = 256; i0 < mt.holes1; i0 += 32) {         // (uniform over the warp)
-          const int v = i0 + lane < mt.holes1 ? __ldcg(hd + i0 + lane) : 0x7FFFFFFF;
+        for (int i0 = 256; i0 < nholes; i0 += 32) {         // (uniform over the warp)
+          const int v = i0 + lane < nholes ? __ldcg(hd + i0 + lane) : 0x7FFFFFFF;
           c += __popc(__ballot_sync(FULLMASK, v < J));
         }
         if (bf + c == J) break;
         J = bf + c;
       }
     }
+    DBGX(bh, 5);
     if (lane == 0) {
-      misc[4] = bf;
+      misc[4] = bf; misc[5] = listed ? 1 : 0;
       p.meta[bh].b = bf;
       p.gat_meta[bh] = make_int4(bf, n_s, __float_as_int(mt.m), (J << 1) | (listed ? 1 : 0));
+      if (!listed) {                                   // "the budget is known" for the gather kernel's CTAs of this head
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
+      }
       if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = bf;
       if (p.dbg.budgets) {
         int* o = p.dbg.budgets + bh * 4;
@@ -269,6 +279,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
   }
   DBGT(32);
+  DBGX(bh, 6);
   __syncthreads();
   const int bfin = misc[4];
   int* dl = p.dyn_idx + (long long)bh * 3 * p.npad;
@@ -312,8 +323,14 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
       cur += NT * WPT;
     }
   }
+  if (misc[5]) {                                       // a listed head: its list is complete now
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
+    }
+  }
   if (p.dbg.dyn_idx) {
-    __threadfence();
     __syncthreads();
     int* dbg = p.dbg.dyn_idx + (long long)bh * p.max_seq_len;
     for (int i = tid; i < bfin; i += NT) dbg[i] = __ldcg(dl + i);
@@ -330,10 +347,11 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   __shared__ double pivT[D];             // the pivot's w*V, element-major per lane: pivT[e * LPR + j]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // grid (S, Hq, 2 B): the deterministic-row CTAs of every head come first in dispatch order, so they take
-  // the SMs that are free while the select kernels still run; the base-row CTAs follow
-  const bool base_cta = (int)blockIdx.z >= p.B;
-  const int h = blockIdx.y, b = base_cta ? blockIdx.z - p.B : blockIdx.z, g = h / p.G;
+  // grid (S, Hq, 2 B): the base-row CTAs of every head come first in dispatch order (they have the longer way to
+  // go: pivot, then rows): while the selection kernel holds its SMs not all CTAs of this grid fit the others, and
+  // the ones that start late should be deterministic-row CTAs
+  const bool base_cta = (int)blockIdx.z < p.B;
+  const int h = blockIdx.y, b = base_cta ? blockIdx.z : blockIdx.z - p.B, g = h / p.G;
   const int bh = b * p.Hq + h;
   const int S = base_cta ? p.stat_splits_base : p.stat_splits;   // CTAs of this kind per head
   const int split = blockIdx.x;
@@ -350,14 +368,25 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   __shared__ unsigned long long s_word;
   __shared__ int s_flag;
   __shared__ int s_misc[8];
+  // deterministic-row CTAs wait for "the list of I_t is written" (a 32-bit word, published first), base-row CTAs
+  // for the 64-bit word
+  const unsigned* fl32 = p.tickets + 4 * p.B * p.Hq + bh;
   if (tid == 0) {
     const unsigned long long* fl = p.flags64 + bh;
     unsigned long long v = 0ull;
+    // (relaxed polls, one acquire when the word has arrived: an acquire per poll would cost the SM an L1
+    // invalidation each time, for every waiting CTA)
     for (unsigned it = 0; it < FLAG_SPINS; ++it) {
-      asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fl) : "memory");
+      if (base_cta) asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fl) : "memory");
+      else {
+        unsigned v32;
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v32) : "l"(fl32) : "memory");
+        v = v32;
+      }
       if (v != 0ull) break;
-      __nanosleep(64);
+      __nanosleep(128);
     }
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
     s_word = v;
   }
   const int n = clamped_len(p, b);
@@ -367,17 +396,20 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   __syncthreads();
   if (s_word == 0ull) {                            // the bounded wait ran out
     pdl_wait();
-    if (tid == 0) s_word = __ldcg(p.flags64 + bh);
+    if (tid == 0) s_word = base_cta ? __ldcg(p.flags64 + bh) : 1ull;
     __syncthreads();
   }
   const unsigned long long word = s_word;
   if (base_cta) DBGT(36);
+  if (base_cta && split == 0) DBGH(bh, 6);
   const int base_list = (int)((word >> 2) & 1ull), base_J = (int)((word >> 3) & 0x3FFFFFull), word_piv = (int)(word >> 32);
   if (n == 0) {                                    // an empty row: no sums, budget 0
     if (base_cta && split == 0) {
       pdl_wait();
       if (tid == 0) {
         p.gat_meta[bh] = make_int4(0, 0, 0, -1);
+        __threadfence();
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
         if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = 0;
         if (p.dbg.budgets) for (int e = 0; e < 4; ++e) p.dbg.budgets[bh * 4 + e] = 0;
         if (p.dbg.stats) for (int e = 0; e < 8; ++e) p.dbg.stats[bh * 8 + e] = 0.0;
@@ -565,14 +597,19 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
     __threadfence();
   }
   __syncthreads();
+  if (base_cta && split == 0) DBGH(bh, 2);              // (one base CTA's rows are done)
   if (s_flag) {
+    DBGH(bh, 3);
+    DBGX(bh, 8);
     // the rest of the list needs the selection kernel's last words (how far it listed the walk): wait for that
     // grid as a whole, which also makes "this grid has completed" imply "the selection kernel has" for the gather
     // kernel behind
     pdl_wait();
+    DBGX(bh, 9);
     DBGT(35);
     TICK_BEGIN(p, VATTN_T_BUDGET);
     head_budget(p, b, h, bh, &part[0][0], piv, pivT, s_misc);
+    DBGH(bh, 4);
     TICK_END(p, VATTN_T_BUDGET);
   }
   TICK_END(p, VATTN_K_STATS);

@@ -56,8 +56,9 @@ struct Prob {
   unsigned* unit_ctr;     // [1] work-unit counter of the persistent score kernel
   unsigned long long* flags64;   // [B,Hq] word the selection kernel publishes per head when I_t is written and marked in
                           //   the walk arrays: 2 | base_list << 2 | base_J << 3 | pivot's physical slot << 32 (zero: not yet)
-  unsigned* tickets;      // [4,B,Hq] "last CTA done" counters of [1] the gather kernel, [2] the dense kernel and
-                          //          [3] the statistics kernel ([0] unused)
+  unsigned* tickets;      // [5,B,Hq] [0] "the head's budget is published" (statistics kernel -> gather kernel);
+                          //          "last CTA done" counters of [1] the gather kernel, [2] the dense kernel and [3] the
+                          //          statistics kernel; [4] "the list of I_t is written" (selection -> statistics kernel)
   unsigned* status;       // [1]
   unsigned* bitmap;       // [B,Hq,nwords] near-tie tokens that made it into I_t (used when they are too many for a list)
   int* vtab;              // [B,Hq,BANDCAP] near-tie tokens ascending, bit 31 = member of I_t
@@ -94,8 +95,14 @@ __device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t;
 // measurement builds (-DVATTN_PHASE_TICKS): stamps of phases inside the kernels, rows 8 + k of a larger tick buffer
 #ifdef VATTN_PHASE_TICKS
 #define DBGT(k) do { TICK_BEGIN(p, 8 + (k)); TICK_END(p, 8 + (k)); } while (0)
+// per-head stamps: row 64 + 4 * bh + (k >> 1), column k & 1
+#define DBGH(bh, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) (p).dbg.kernel_ticks[2 * (64 + 4 * (bh) + ((k) >> 1)) + ((k) & 1)] = gtime_ns(); } while (0)
+// stamps of one head (the first), slot k < 32: row 200 + (k >> 1), column k & 1; by one thread
+#define DBGX(bh, k) do { if ((p).dbg.kernel_ticks && (bh) == 0 && (threadIdx.x & 31) == 0 && threadIdx.x < 32) (p).dbg.kernel_ticks[2 * (200 + ((k) >> 1)) + ((k) & 1)] = gtime_ns(); } while (0)
 #else
 #define DBGT(k) do { } while (0)
+#define DBGH(bh, k) do { } while (0)
+#define DBGX(bh, k) do { } while (0)
 #endif
 // rows of kernel_ticks
 #define VATTN_K_ZERO 0
