@@ -109,13 +109,13 @@ void derive(vattn_plan* pl) {
   pl->off_topk = take(2 * BH * pl->npad * sizeof(int));     // token indices, then physical slots
   pl->off_base = take(2 * BH * pl->npad * sizeof(int));
   pl->off_walk = take(4 * BH * pl->npad * sizeof(int));     // first walk positions of both walks: tokens, physical slots
-  pl->off_holes = take(BH * VATTN_BANDCAP * sizeof(int));
+  pl->off_holes = take(2 * BH * VATTN_BANDCAP * sizeof(int));
   pl->off_dyn = take(3 * BH * pl->npad * sizeof(int));      // tokens, physical slots, score bits
   pl->off_meta = take(BH * sizeof(HeadMeta));
   pl->off_stat = take(BH * 2 * VATTN_STAT_MAXS * (D + 3) * sizeof(double));
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
-  pl->off_gmeta = take(BH * sizeof(int4));
+  pl->off_gmeta = take(2 * BH * sizeof(int4));
   // partial slots (chunks) per head of the gather kernel: 32, except that a handful of heads may use more of
   // the 8 CTAs per SM (64 to 128 chunks each when that many fit the grid at once)
   {

@@ -29,11 +29,13 @@ namespace {
 // lines at 32 heads, and every CTA reads all of it)
 // b: the budget; L: entries to visit (a prefix of the final sample's walk array, members of I_t marked, or the b
 // entries of the head's list when `list` is set); n = 0: an empty row
-struct GMeta { int b, n_s; float m; int n, L, list; };
+// W1: entries of the walk array (the gather computes the ones beyond it)
+struct GMeta { int b, n_s; float m; int n, L, list, W1; };
 __device__ __forceinline__ GMeta ld_gmeta(const int4* g) {
   const int4 v = __ldcg(g);
   GMeta r; r.b = v.x; r.n_s = v.y; r.m = __int_as_float(v.z);
   r.n = v.w < 0 ? 0 : 1; r.L = v.w < 0 ? 0 : (v.w >> 1); r.list = v.w < 0 ? 0 : (v.w & 1);
+  r.W1 = __ldcg(reinterpret_cast<const int*>(g + 1));
   return r;
 }
 
@@ -60,8 +62,14 @@ struct Gather {
       v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
     }
   }
+  // Entries of the final sample's walk beyond its array (budgets of more than about eight base budgets): the token
+  // of such a position is computed here (sigma), its membership in I_t decided from its score like the selection
+  // kernel would.  keys: the walk's round keys, mt: the head's record (both in shared memory).
+  // ident: the budget is the whole residual; every middle token is visited, in token order (no walk needed).
+  struct Far { bool on, ident; int W1, s0, mlen; const unsigned* keys; const HeadMeta* mt; };
   // rows [r_begin, r_end) of head bh -> partial `slot`; the last of `nslots` finishers combines
-  static __device__ void run(const Prob& p, int bh, const GMeta& meta, int r_begin, int r_end, int slot, int nslots,
+  template <bool FAR>
+  static __device__ void run(const Prob& p, int bh, const GMeta& meta, int r_begin, int r_end, const Far& far, int slot, int nslots,
                              float (*part)[NE], int* is_last, float* s_den) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = bh % p.Hq, g = h / p.G;
@@ -94,10 +102,30 @@ struct Gather {
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
+        const bool ok = (FULL || ((k0 + u < iters) && (r < r_end))) && !(FAR && r >= far.W1);
         tok_n[u] = ok ? __ldg(dyn + r) : -1;
         ph_n[u] = ok ? __ldg(dph + r) : 0;
       }
+      if (FAR) {                                        // lane u of a row group computes row u's entry
+        int ctok = -1, cph = 0;
+        if (j < UNROLL) {
+          const int r = r_begin + rg + (k0 + j) * RG;
+          if (r >= far.W1 && (FULL || ((k0 + j < iters) && (r < r_end)))) {
+            ctok = far.s0 + (far.ident ? r : walk_at(make_walk(far.keys, far.mlen), r));
+            cph = page_of(p, bh / p.Hq, ctok >> 4) * VATTN_BLOCK + (ctok & 15);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          const int t = __shfl_sync(0xFFFFFFFFu, ctok, u, LPR), ph = __shfl_sync(0xFFFFFFFFu, cph, u, LPR);
+          if (t >= 0) { tok_n[u] = t; ph_n[u] = ph; }
+        }
+      }
+    };
+    // a computed entry's token may be a member of I_t (nothing marked it): its score decides
+    auto far_member = [&](int k0, int u, int tok) -> bool {
+      if (!FAR || tok < 0 || r_begin + rg + (k0 + u) * RG < far.W1) return false;
+      return in_topk(*far.mt, p.vtab + (long long)bh * VATTN_BANDCAP, p.bitmap + (long long)bh * p.nwords, tok, __ldg(sc + tok));
     };
     auto fetch_next = [&](int k0) {                   // indices of the batch that starts at iteration k0, if any
       if (k0 >= iters) return;
@@ -134,7 +162,7 @@ struct Gather {
           for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kv[e], dot);
 #pragma unroll
           for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
-          if (j == u) { w_mine = p.scale * dot; tok_mine = tok[u]; }
+          if (j == u) { w_mine = p.scale * dot; tok_mine = far_member(k0, u, tok[u]) ? -1 : tok[u]; }
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + off[u]));
         }
@@ -143,7 +171,7 @@ struct Gather {
         for (int u = 0; u < UNROLL; ++u) {
           tok[u] = tok_n[u];
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (j == u) tok_mine = tok[u];
+          if (j == u) tok_mine = far_member(k0, u, tok[u]) ? -1 : tok[u];
           if (FULL || tok[u] >= 0) {
             const int ph = ph_n[u];
             raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL));
@@ -244,16 +272,38 @@ struct Gather {
   }
 };
 
+
+// what a unit needs for entries beyond the walk array (see Gather::Far); uniform over the CTA
+template <typename G>
+__device__ __forceinline__ typename G::Far far_setup(const Prob& p, int bh, const GMeta& meta, int nb, unsigned* s_keys, HeadMeta* s_mt) {
+  typename G::Far far;
+  far.ident = meta.n > 0 && !meta.list && meta.b >= meta.n_s && meta.b > 0;
+  far.W1 = far.ident ? 0 : meta.W1;
+  far.on = meta.n > 0 && !meta.list && nb > far.W1;
+  far.s0 = 0; far.mlen = 1; far.keys = s_keys; far.mt = s_mt;
+  if (far.on) {
+    const int b = bh / p.Hq, h = bh % p.Hq;
+    const Geo geo = head_geometry(p, clamped_len(p, b));
+    far.s0 = geo.s0; far.mlen = geo.l_start - geo.s0;
+    if (threadIdx.x < 2) walk_keys(p, b, p.rng_head_is_kv ? h / p.G : h, 1, threadIdx.x, s_keys);
+    if (threadIdx.x == 32) *s_mt = ld_meta(p.meta + bh);
+    __syncthreads();
+  }
+  return far;
+}
+
 template <typename T, int D, bool KV>
-__global__ void __launch_bounds__(NT, KV ? 8 : 10) k_gather(const Prob p) {
+__global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   using G = Gather<T, D, KV>;
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
+  __shared__ unsigned s_keys[8];
+  __shared__ HeadMeta s_mt;
   TICK_BEGIN(p, VATTN_K_GATHER);
   pdl_wait();
   const int bh = blockIdx.z * p.Hq + blockIdx.y;
-  const GMeta meta = ld_gmeta(p.gat_meta + bh);
+  const GMeta meta = ld_gmeta(p.gat_meta + 2 * bh);
   const int nb = meta.n > 0 ? meta.L : 0;              // entries to visit
   // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
   // (with this many heads the kernel is throughput-bound: 4 batches per row group amortise the fixed hops)
@@ -261,7 +311,9 @@ __global__ void __launch_bounds__(NT, KV ? 8 : 10) k_gather(const Prob p) {
   const int nslots = max(1, (nb + chunk - 1) / chunk);
   if ((int)blockIdx.x >= nslots) return;
   const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
-  G::run(p, bh, meta, r_begin, r_end, blockIdx.x, nslots, part, &is_last, &s_den);
+  const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
+  if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
+  else G::template run<false>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
   TICK_END(p, VATTN_K_GATHER);
 }
 
@@ -271,6 +323,8 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   __shared__ float part[NWARP][G::NE];
   __shared__ int is_last;
   __shared__ float s_den;
+  __shared__ unsigned s_keys[8];
+  __shared__ HeadMeta s_mt;
   __shared__ unsigned s_ready;
   TICK_BEGIN(p, VATTN_K_GATHER);
   const int tid = threadIdx.x;
@@ -300,14 +354,16 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
     __syncthreads();
     if (!waited && s_ready == 0u) { pdl_wait(); waited = true; }      // uniform over the CTA
     DBGT(21);
-    const GMeta meta = ld_gmeta(p.gat_meta + bh);
+    const GMeta meta = ld_gmeta(p.gat_meta + 2 * bh);
     const int nb = meta.n > 0 ? meta.L : 0;            // entries to visit
     const int batches = (nb + BATCH - 1) / BATCH;
     const int rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
     const int nslots = max(1, (nb + rows - 1) / rows); // a head without samples still writes its output
     if (ci < nslots) {
       const int r_begin = min(nb, ci * rows), r_end = min(nb, r_begin + rows);
-      G::run(p, bh, meta, r_begin, r_end, ci, nslots, part, &is_last, &s_den);
+      const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
+      if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);
+      else G::template run<false>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);
     }
     __syncthreads();
   }

@@ -290,7 +290,7 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     pdl_wait();
     pdl_trigger();
     if (tid == 0) {
-      mt.base_J = 0; mt.base_piv = 0; mt.base_list = 0; mt.holes1 = 0;
+      mt.base_J = 0; mt.holes2 = 0; mt.base_list = 0; mt.holes1 = 0;
       p.meta[bh] = mt;
       __threadfence();
       asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(2ull) : "memory");
@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   }
   for (int w = tid; w < ((n + 31) >> 5); w += NT) gbitmap[w] = 0u;     // only the overflow path sets and reads bits
   // the first entries of the head's list of marked positions are read unconditionally by the budget: "none" until set
-  if (tid < 256) p.hole_pos[(long long)bh * VATTN_BANDCAP + tid] = 0x7FFFFFFF;
+  if (tid < 256) p.hole_pos[(long long)bh * 2 * VATTN_BANDCAP + tid] = 0x7FFFFFFF;
 
   pdl_wait();                                          // the score pass is complete: scores, maxima
   pdl_trigger();
@@ -695,14 +695,14 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   const int W0 = walk_region(n_s > 0 ? b0 : 0, n_s, mlen, kk);   // entries the walk kernel wrote
   const int W1 = walk_region(dyn_listed_want(p, n_s, b0), n_s, mlen, kk);
   int* hp0 = sm.hist;                                  // marked positions of the base walk (over the histograms)
-  int* cnts = sm.misc + 8;                             // [0] marked positions of the base walk, [1] of the final walk
-  int base_J = 0, base_list = 0, holes1 = 0, dyn_J = 0, dyn_listed = 0, piv_ph = 0;
+  int* cnts = sm.misc + 8;                             // marked positions: [0] base walk, [1] final walk; [2] members beyond its array
+  int base_J = 0, base_list = 0, holes1 = 0, holes2 = 0, dyn_J = 0, dyn_listed = 0, piv_ph = 0;
   if (n_s > 0 && kk <= NT * 4) {
-    int* hp1 = p.hole_pos + (long long)bh * VATTN_BANDCAP;
+    int* hp1 = p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP;     // positions inside the walk array; + BANDCAP: beyond it
     // physical slots of the first entries of the base walk: one of them is the pivot (the first unmarked entry)
     int pvph = 0;
     if (warp == 0 && lane < 4 && lane < W0) pvph = __ldcg(wa0 + p.npad + lane);
-    if (tid == 0) { cnts[0] = 0; cnts[1] = 0; }
+    if (tid == 0) { cnts[0] = 0; cnts[1] = 0; cnts[2] = 0; }
     const Walk wk0 = make_walk(sm.rkeys + (p.nested_base ? 8 : 0), mlen), wk1 = make_walk(sm.rkeys + 8, mlen);
     __syncthreads();
     DBGT(16);
@@ -719,6 +719,9 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
         wa1[x1] = -1;
         const int i1 = atomicAdd(&cnts[1], 1);
         if (i1 < VATTN_BANDCAP) hp1[i1] = x1;
+      } else {                                         // (budgets that reach beyond the array need these)
+        const int i2 = atomicAdd(&cnts[2], 1);
+        if (i2 < VATTN_BANDCAP) hp1[VATTN_BANDCAP + i2] = x1;
       }
     }
     __syncthreads();
@@ -750,12 +753,15 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     }
     __syncthreads();
     if (!base_list) { base_J = sm.misc[4]; piv_ph = sm.misc[5]; base_list = sm.misc[6]; }
-    if (holes1 <= VATTN_BANDCAP) { dyn_J = W1; dyn_listed = W1 - holes1; }
+    holes2 = cnts[2];
+    // every member's position is known: any budget can be served as "the non-members among the first J positions"
+    // (entries beyond the array are computed by the gather kernel); else only budgets inside the array
+    if (holes1 <= VATTN_BANDCAP) { dyn_J = W1; dyn_listed = holes2 <= VATTN_BANDCAP ? n_s : W1 - holes1; }
   } else if (n_s > 0) {
     base_list = 1;
   }
   if (base_J >= (1 << 22)) base_list = 1;              // the published word has 22 bits for it
-  mt.base_J = base_J; mt.base_piv = 0; mt.base_list = base_list; mt.holes1 = min(holes1, VATTN_BANDCAP);
+  mt.base_J = base_J; mt.holes2 = min(holes2, VATTN_BANDCAP); mt.base_list = base_list; mt.holes1 = min(holes1, VATTN_BANDCAP);
   mt.dyn_J = dyn_J; mt.dyn_listed = dyn_listed;
   DBGT(6);
 

@@ -164,7 +164,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   // (warp 0) the first 256 marked positions of the final sample's walk array, eight per lane; INT_MAX where none
   int hp[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) hp[i] = warp == 0 ? __ldcg(p.hole_pos + (long long)bh * VATTN_BANDCAP + i * 32 + lane) : 0;
+  for (int i = 0; i < 8; ++i) hp[i] = warp == 0 ? __ldcg(p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP + i * 32 + lane) : 0;
   const int n_s = mt.n_s, b0 = mt.b0;
   // what does not depend on the sums, computed while they are on their way
   const double ratio = (b0 > 0) ? (double)n_s / (double)b0 : 0.0;
@@ -242,27 +242,35 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     // positions below J (a fixed point, reached in a few steps); budgets beyond the array take a list (below)
     DBGX(bh, 4);
     const bool listed = bf > mt.dyn_listed;
-    const int nholes = min(max(mt.holes1, 0), VATTN_BANDCAP);
+    const int nholes = min(max(mt.holes1, 0), VATTN_BANDCAP), nholes2 = min(max(mt.holes2, 0), VATTN_BANDCAP);
     int J = bf;
     if (!listed) {
-      const int* hd = p.hole_pos + (long long)bh * VATTN_BANDCAP;
+      const int* hd = p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP;
+      const bool far = bf > mt.dyn_J - nholes;           // reaches beyond the walk array: the members there count too
       for (int it = 0; it < 64; ++it) {
         int c = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) c += __popc(__ballot_sync(FULLMASK, hp[i] < J));
-        for (int i0 = 256; i0 < nholes; i0 += 32) {         // (uniform over the warp)
+        for (int i0 = 256; i0 < nholes; i0 += 32) {            // (uniform over the warp)
           const int v = i0 + lane < nholes ? __ldcg(hd + i0 + lane) : 0x7FFFFFFF;
           c += __popc(__ballot_sync(FULLMASK, v < J));
         }
+        if (far)
+          for (int i0 = 0; i0 < nholes2; i0 += 32) {
+            const int v = i0 + lane < nholes2 ? __ldcg(hd + VATTN_BANDCAP + i0 + lane) : 0x7FFFFFFF;
+            c += __popc(__ballot_sync(FULLMASK, v < J));
+          }
         if (bf + c == J) break;
         J = bf + c;
       }
     }
-    DBGX(bh, 5);
     if (lane == 0) {
       misc[4] = bf; misc[5] = listed ? 1 : 0;
       p.meta[bh].b = bf;
-      p.gat_meta[bh] = make_int4(bf, n_s, __float_as_int(mt.m), (J << 1) | (listed ? 1 : 0));
+      // the whole residual: every middle token is visited (in token order), members of I_t weigh nothing
+      if (!listed && bf >= n_s) J = mt.l_start - mt.s0;
+      p.gat_meta[2 * bh] = make_int4(bf, n_s, __float_as_int(mt.m), (J << 1) | (listed ? 1 : 0));
+      p.gat_meta[2 * bh + 1] = make_int4(mt.dyn_J, 0, 0, 0);
       if (!listed) {                                   // "the budget is known" for the gather kernel's CTAs of this head
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
       }
@@ -347,11 +355,10 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   __shared__ double pivT[D];             // the pivot's w*V, element-major per lane: pivT[e * LPR + j]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // grid (S, Hq, 2 B): the base-row CTAs of every head come first in dispatch order (they have the longer way to
-  // go: pivot, then rows): while the selection kernel holds its SMs not all CTAs of this grid fit the others, and
-  // the ones that start late should be deterministic-row CTAs
-  const bool base_cta = (int)blockIdx.z < p.B;
-  const int h = blockIdx.y, b = base_cta ? blockIdx.z : blockIdx.z - p.B, g = h / p.G;
+  // grid (S, Hq, 2 B): the deterministic-row CTAs of every head come first in dispatch order (their word is
+  // published first), the base-row CTAs follow
+  const bool base_cta = (int)blockIdx.z >= p.B;
+  const int h = blockIdx.y, b = base_cta ? blockIdx.z - p.B : blockIdx.z, g = h / p.G;
   const int bh = b * p.Hq + h;
   const int S = base_cta ? p.stat_splits_base : p.stat_splits;   // CTAs of this kind per head
   const int split = blockIdx.x;
@@ -371,7 +378,13 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   // deterministic-row CTAs wait for "the list of I_t is written" (a 32-bit word, published first), base-row CTAs
   // for the 64-bit word
   const unsigned* fl32 = p.tickets + 4 * p.B * p.Hq + bh;
+#ifdef VATTN_X_NOPOLL
+  pdl_wait();
+  if (tid == 0) s_word = base_cta ? __ldcg(p.flags64 + bh) : 1ull;
+  if (false) {
+#else
   if (tid == 0) {
+#endif
     const unsigned long long* fl = p.flags64 + bh;
     unsigned long long v = 0ull;
     // (relaxed polls, one acquire when the word has arrived: an acquire per poll would cost the SM an L1
@@ -407,7 +420,8 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
     if (base_cta && split == 0) {
       pdl_wait();
       if (tid == 0) {
-        p.gat_meta[bh] = make_int4(0, 0, 0, -1);
+        p.gat_meta[2 * bh] = make_int4(0, 0, 0, -1);
+        p.gat_meta[2 * bh + 1] = make_int4(0, 0, 0, 0);
         __threadfence();
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
         if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = 0;
@@ -459,7 +473,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
         act_n[u] = (k0 + u < iters) && (r < r_end);
         ph_n[u] = ph0;                                       // idle slots re-read the first row
         if (act_n[u])
-          ph_n[u] = r < s0 ? phys_of(p, b, r) : (r < s0 + kk ? __ldcg(tkph + r - s0) : phys_of(p, b, l_start + (r - s0 - kk)));
+          ph_n[u] = r < s0 ? phys_of(p, b, r) : (r < s0 + kk ? __ldg(tkph + r - s0) : phys_of(p, b, l_start + (r - s0 - kk)));
       }
     };
     auto issue = [&](RowRegs<T> (&row)[UN], bool (&act)[UN]) {
@@ -498,20 +512,21 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
     // ---------------------------------------------------------------- base-sample rows, shifted by the pivot
     RowRegs<T> prow;
     const int piv_ph = base_list ? __ldcg(bsph) : word_piv;      // pivot = first base-sample row
-    int ph_n[UN];
-    bool act_n[UN];
+    // (the entries are only requested here and looked at one batch later, when the rows are requested: a marked
+    // entry, token -1, is a member of I_t, not a sample; its slot is valid all the same)
+    int ph_n[UN], tok_n[UN];
     auto fetch = [&](int k0) {
 #pragma unroll
       for (int u = 0; u < UN; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        act_n[u] = (k0 + u < iters) && (r < r_end);
-        ph_n[u] = act_n[u] ? __ldcg(bsph + r) : piv_ph;
-        if (act_n[u]) act_n[u] = __ldcg(bstok + r) >= 0;       // marked entry: a member of I_t, not a sample
+        const bool in = (k0 + u < iters) && (r < r_end);
+        ph_n[u] = in ? __ldg(bsph + r) : piv_ph;
+        tok_n[u] = in ? __ldg(bstok + r) : -1;
       }
     };
     auto issue = [&](RowRegs<T> (&row)[UN], bool (&act)[UN]) {
 #pragma unroll
-      for (int u = 0; u < UN; ++u) { act[u] = act_n[u]; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
+      for (int u = 0; u < UN; ++u) { act[u] = tok_n[u] >= 0; load_row<T, D>(p, g, ph_n[u], j, row[u]); }
     };
     double cw = 0.0;
     auto reduce = [&](const RowRegs<T> (&row)[UN], const bool (&act)[UN]) {
@@ -591,14 +606,22 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   // (the barrier orders every thread's writes before thread 0's fence, which is cumulative; likewise on the way in)
   __syncthreads();
   DBGT(34);
+#ifdef VATTN_X_NOTICKET
+  if (false) {
+#else
   if (tid == 0) {
+#endif
     __threadfence();
     s_flag = (atomicAdd(&p.tickets[3 * p.B * p.Hq + bh], 1u) == (unsigned)(p.stat_splits + p.stat_splits_base - 1));
     __threadfence();
   }
   __syncthreads();
   if (base_cta && split == 0) DBGH(bh, 2);              // (one base CTA's rows are done)
+#ifdef VATTN_X_NOBUDGET
+  if (false) {
+#else
   if (s_flag) {
+#endif
     DBGH(bh, 3);
     DBGX(bh, 8);
     // the rest of the list needs the selection kernel's last words (how far it listed the walk): wait for that

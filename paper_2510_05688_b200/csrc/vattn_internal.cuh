@@ -25,12 +25,13 @@ struct HeadMeta {
   float m;          // largest fp32 score of the head (softmax stabiliser)
   float hi, lo;     // a middle token is in I_t if its score is above hi; scores in [lo, hi] are near-ties
   int run1;         // the list of I_t is two ascending runs: [0, run1) and [run1, kk)
-  int dyn_listed;   // residual tokens among the first dyn_J positions of the final sample's walk: budgets up to
-  int dyn_J;        //   this many are served from the walk arrays (members of I_t marked), larger ones from a list
+  int dyn_listed;   // budgets up to this many are served as "the non-members among the first J positions of the final
+  int dyn_J;        //   sample's walk" (dyn_J positions are in the walk array, members marked), larger ones from a list
   int path;         // code path of the selection (vattn_debug.paths)
   int b;            // final budget |I_dyn| (written by the statistics kernel)
   int base_J;       // the base sample = the unmarked entries among the first base_J of its walk array ...
-  int base_piv;     //   (unused);  base_list = 1: it is in base_idx instead
+  int holes2;       //   members of I_t at positions of the final sample's walk beyond its array (hole_pos + BANDCAP)
+                    //   base_list = 1: the base sample is in base_idx instead
   int base_list;    //   (b0 entries, none marked)
   int holes1;       // marked entries among the first dyn_J of the final sample's walk (their positions in hole_pos)
 };
@@ -68,15 +69,17 @@ struct Prob {
   int* walk_tok;          // [B,Hq,2,2,npad] the first positions of both walks (computed beside the score pass): per
                           //   walk the tokens, then their physical slots.  The selection kernel marks the members
                           //   of I_t (token = -1; the slot stays valid): a sample is the unmarked entries of a prefix
-  int* hole_pos;          // [B,Hq,VATTN_BANDCAP] positions of the marked entries of the final sample's walk array, in
-                          //   no particular order; the first 256 words read INT_MAX where there is none
+  int* hole_pos;          // [B,Hq,2,VATTN_BANDCAP] positions of the marked entries of the final sample's walk array, in
+                          //   no particular order (the first 256 words read INT_MAX where there is none); then the
+                          //   positions of the members of I_t beyond the array
   int* dyn_idx;           // [B,Hq,3,npad] I_dyn as a list (tokens, physical slots) for budgets beyond the walk arrays
                           //               (scratch of the near-tie overflow path while the selection runs)
   HeadMeta* meta;         // [B,Hq]
   double* stat_part;      // [B,Hq,2*16,D+3]  partials of the statistics kernel (deterministic-row CTAs, then base-row CTAs)
   double* stat_piv;       // [B,Hq,D+1] pivot row of the base-sample sums: w*V then w
   double* det_sums;       // [B,Hq,D+1] N_f then D_f
-  int4* gat_meta;         // [B,Hq] what the gather kernel needs of a head: b, n_s, bits of m, n
+  int4* gat_meta;         // [B,Hq,2] what the gather kernel needs of a head: b, n_s, bits of m, entries to visit << 1 |
+                          //   list (-1: an empty row); entries of the final sample's walk array
   float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
   int gat_slots;          // partial slots (chunks) per head: 32; 64 to 128 when at most 18 heads share the grid
   int stat_splits, stat_splits_base;   // statistics CTAs per head: deterministic rows, base-sample rows
