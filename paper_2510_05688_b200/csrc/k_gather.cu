@@ -106,12 +106,21 @@ struct Gather {
         tok_n[u] = ok ? __ldg(dyn + r) : -1;
         ph_n[u] = ok ? __ldg(dph + r) : 0;
       }
-      if (FAR) {                                        // lane u of a row group computes row u's entry
+      if (FAR && far.ident) {                           // the whole residual: entry r is middle token r
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          const int r = r_begin + rg + (k0 + u) * RG;
+          const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
+          const int tok = far.s0 + r;
+          tok_n[u] = ok ? tok : -1;
+          ph_n[u] = ok ? page_of(p, bh / p.Hq, tok >> 4) * VATTN_BLOCK + (tok & 15) : 0;
+        }
+      } else if (FAR) {                                 // lane u of a row group computes row u's entry
         int ctok = -1, cph = 0;
         if (j < UNROLL) {
           const int r = r_begin + rg + (k0 + j) * RG;
           if (r >= far.W1 && (FULL || ((k0 + j < iters) && (r < r_end)))) {
-            ctok = far.s0 + (far.ident ? r : walk_at(make_walk(far.keys, far.mlen), r));
+            ctok = far.s0 + walk_at(make_walk(far.keys, far.mlen), r);
             cph = page_of(p, bh / p.Hq, ctok >> 4) * VATTN_BLOCK + (ctok & 15);
           }
         }
@@ -122,15 +131,15 @@ struct Gather {
         }
       }
     };
-    // a computed entry's token may be a member of I_t (nothing marked it): its score decides
-    auto far_member = [&](int k0, int u, int tok) -> bool {
-      if (!FAR || tok < 0 || r_begin + rg + (k0 + u) * RG < far.W1) return false;
-      return in_topk(*far.mt, p.vtab + (long long)bh * VATTN_BANDCAP, p.bitmap + (long long)bh * p.nwords, tok, __ldg(sc + tok));
-    };
     auto fetch_next = [&](int k0) {                   // indices of the batch that starts at iteration k0, if any
       if (k0 >= iters) return;
       if (k0 + UNROLL <= full_iters) fetch_idx(k0, std::true_type{});
       else fetch_idx(k0, std::false_type{});
+    };
+    // a computed entry's token may be a member of I_t (nothing marked it): its score s decides
+    auto far_member = [&](int k0, int u, int tok, float s) -> bool {
+      if (!FAR || tok < 0 || r_begin + rg + (k0 + u) * RG < far.W1) return false;
+      return in_topk(*far.mt, p.vtab + (long long)bh * VATTN_BANDCAP, p.bitmap + (long long)bh * p.nwords, tok, s);
     };
     // K+V variant: the score of a sampled token is recomputed from its K row (what a selector that leaves no
     // scores for the whole context behind would need); the K slices of a batch come first, then its V slices
@@ -162,7 +171,10 @@ struct Gather {
           for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kv[e], dot);
 #pragma unroll
           for (int mask = LPR / 2; mask >= 1; mask >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, mask);
-          if (j == u) { w_mine = p.scale * dot; tok_mine = far_member(k0, u, tok[u]) ? -1 : tok[u]; }
+          if (j == u) {
+            w_mine = p.scale * dot;
+            tok_mine = (FAR && tok[u] >= 0 && far_member(k0, u, tok[u], __ldg(sc + tok[u]))) ? -1 : tok[u];
+          }
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + off[u]));
         }
@@ -171,14 +183,15 @@ struct Gather {
         for (int u = 0; u < UNROLL; ++u) {
           tok[u] = tok_n[u];
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (j == u) tok_mine = far_member(k0, u, tok[u]) ? -1 : tok[u];
+          if (j == u) tok_mine = tok[u];
           if (FULL || tok[u] >= 0) {
             const int ph = ph_n[u];
             raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL));
           }
         }
         if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);
-        fetch_next(k0 + UNROLL);                        // next batch's indices travel with this batch's rows
+        fetch_next(k0 + UNROLL);
+        if (FAR && j < UNROLL && far_member(k0, j, tok_mine, w_mine)) tok_mine = -1;                        // next batch's indices travel with this batch's rows
       }
       const float e_mine = (tok_mine >= 0) ? expf(w_mine - m) : 0.f;
 #pragma unroll
@@ -285,7 +298,7 @@ __device__ __forceinline__ typename G::Far far_setup(const Prob& p, int bh, cons
     const int b = bh / p.Hq, h = bh % p.Hq;
     const Geo geo = head_geometry(p, clamped_len(p, b));
     far.s0 = geo.s0; far.mlen = geo.l_start - geo.s0;
-    if (threadIdx.x < 2) walk_keys(p, b, p.rng_head_is_kv ? h / p.G : h, 1, threadIdx.x, s_keys);
+    if (threadIdx.x < 2 && !far.ident) walk_keys(p, b, p.rng_head_is_kv ? h / p.G : h, 1, threadIdx.x, s_keys);
     if (threadIdx.x == 32) *s_mt = ld_meta(p.meta + bh);
     __syncthreads();
   }

@@ -385,7 +385,43 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     const int d1 = sm.misc[0];
     const int dlo = max(d1 - 2, 0), dhi = min(d1 + 2, HBINS - 1);           // candidate bins
     kbase = (unsigned)dlo << 21;                       // candidate keys relative to it are below 5 * 2^21 < 2^24
-    const unsigned kend = dhi == HBINS - 1 ? 0xFFFFFFFFu : (((unsigned)dhi + 1u) << 21) - 1u;    // last candidate key
+    unsigned kend = dhi == HBINS - 1 ? 0xFFFFFFFFu : (((unsigned)dhi + 1u) << 21) - 1u;    // last candidate key
+    {
+      // Scores that crowd into a few bins (a near-uniform head: all of them within a factor of two) would make
+      // most of the head a candidate.  The sample says how many keys the five bins hold; when that is more than
+      // the candidate list takes, the candidates are a narrower key range inside the five bins: the sample's keys
+      // of those bins in 5 x 256 finer bins, and the range between the ranks k' - delta and k' + delta of the sample (delta: four
+      // standard deviations of the sample's rank and a little more).  Pass B verifies the range like the bins.
+      int c5 = 0, cb = 0;                              // sample keys in the five bins; in those of them before d1
+      for (int d = dlo; d <= dhi; ++d) { c5 += hA[d]; if (d < d1) cb += hA[d]; }
+      const long long rs = max(1ll, min((long long)ns_tot, ((long long)kk * ns_tot + mlen - 1) / mlen));
+      if ((long long)c5 * mlen > (long long)(ALLCAP * 7 / 8) * ns_tot) {      // (uniform over the CTA)
+        const int before = sm.misc[1] - cb;            // sample keys before bin dlo
+        __syncthreads();                               // (misc is written again below)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int i = ((2 * tid + c) << 4) + (tid & 15);
+          if (i >= s0 && i < l_start) {
+            const unsigned key = keys[key_slot(i)];
+            const int d = (int)(key >> 21);
+            if (d >= dlo && d <= dhi) atomicAdd(&hC[((d - dlo) << 8) | ((key >> 13) & 0xFFu)], 1);     // 5 x 256 finer bins
+          }
+        }
+        __syncthreads();
+        const int r5 = (int)rs - before;               // the rank among the sample keys of the five bins (1-based)
+        const int delta = 4 * (int)sqrtf((float)rs) + 8;
+        block_pick(hC, HBINS, max(1, min(c5, r5 - delta)), sm.misc + 32, sm.misc + 8);
+        __syncthreads();
+        block_pick(hC, HBINS, max(1, min(c5, r5 + delta)), sm.misc + 32, sm.misc + 10);
+        __syncthreads();
+        const unsigned f_lo = (unsigned)sm.misc[8], f_hi = (unsigned)sm.misc[10];
+        if (r5 - delta >= 1) kbase = (((unsigned)dlo + (f_lo >> 8)) << 21) | ((f_lo & 0xFFu) << 13);
+        if (r5 + delta <= c5) kend = (((unsigned)dlo + (f_hi >> 8)) << 21) | ((f_hi & 0xFFu) << 13) | 0x1FFFu;
+        for (int i = tid; i < HBINS; i += NT) hC[i] = 0;       // (the exact selection uses it again)
+        path |= 8;
+        __syncthreads();
+      }
+    }
     DBGT(1);
     {
       // ---- B: upper keys' tokens to the list of I_t, candidates to their list, both ascending by token
@@ -458,8 +494,8 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
       const float Tf = unord_f32(~(kbase + (pref << 12) + (unsigned)sm.misc[5]));
       hi = __fadd_ru(Tf, 2.f * gamma); lo = __fadd_rd(Tf, -2.f * gamma);
       // the band must stay inside the candidate bins: every upper key is then above it, every other key below it
-      const bool up_ok = dlo == 0 || hi <= unord_f32(~((unsigned)dlo << 21));
-      const bool dn_ok = dhi == HBINS - 1 || lo >= unord_f32(~(((unsigned)dhi << 21) | 0x1FFFFFu));
+      const bool up_ok = kbase == 0u || hi <= unord_f32(~kbase);
+      const bool dn_ok = kend == 0xFFFFFFFFu || lo >= unord_f32(~kend);
       // classify the candidates: thread t takes a run of consecutive entries, so ordinals are one prefix sum
       const int per = (ncand + NT - 1) / NT;
       const int c_lo = min(ncand, tid * per), c_hi = min(ncand, c_lo + per);
