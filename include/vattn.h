@@ -199,6 +199,16 @@ int vattn_decode_host(vattn_plan* plan, const void* q_host, const void* k_cache,
  * `stream`; not for the hot path.  Errors: INVALID_ARG, WORKSPACE, CUDA. */
 int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits /* host */);
 
+/* The step's kernels hand work to one another through words in the workspace: a producer CTA publishes a word
+ * (release store), consumer CTAs poll it.  Every such wait is bounded: after a fixed number of polls the CTA falls
+ * back to the grid-level dependency wait, which is always sufficient (the paper has no counterpart: this is how the
+ * implementation overlaps Algorithm 1's stages).  This call runs the wait primitive alone: one thread polls a word
+ * that nothing publishes, `spins` times (1 .. 2^20), and reports through *ran_out (host; 1 = the limit ended the
+ * wait) and *waited_us (host; device-side microseconds).  It synchronises `stream`.  The context stays usable.
+ * Errors: INVALID_ARG (null pointers, spins outside the range), WORKSPACE, CUDA. */
+int vattn_probe_bounded_wait(vattn_plan* plan, uint32_t spins, uint32_t* ran_out /* host */,
+                             uint32_t* waited_us /* host */, void* stream);
+
 /* Number of kernels the last vattn_decode / vattn_dense_decode call on this plan enqueued. */
 int vattn_last_launch_count(const vattn_plan* plan);
 

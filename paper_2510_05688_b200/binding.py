@@ -19,7 +19,7 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
            "vattn_host_staging_bytes", "vattn_decode_host", "vattn_last_status", "vattn_last_launch_count",
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
-           "vattn_dense_decode_noalloc", "vattn_set_stop_after"]
+           "vattn_dense_decode_noalloc", "vattn_set_stop_after", "vattn_probe_bounded_wait"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
 KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_gather"]
 NUM_TICKS = 8
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
     L.vattn_decode_host.restype = i32
     L.vattn_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     L.vattn_last_status.restype = i32
+    L.vattn_probe_bounded_wait.argtypes = [vp, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), vp]
+    L.vattn_probe_bounded_wait.restype = i32
     L.vattn_last_launch_count.argtypes = [vp]
     L.vattn_last_launch_count.restype = i32
     L.vattn_strerror.argtypes = [i32]
@@ -240,6 +242,13 @@ class Plan:
         calls = C.c_int(0)
         _check(lib().vattn_read_profile(self._h, ms, C.byref(calls)), "vattn_read_profile")
         return {n: float(ms[i]) for i, n in enumerate(KERNEL_NAMES)}, int(calls.value)
+
+    def probe_bounded_wait(self, spins: int, stream=None):
+        """Run the bounded wait primitive alone on a word that nothing publishes: (ran_out, waited_us)."""
+        ran, us = C.c_uint32(0), C.c_uint32(0)
+        _check(lib().vattn_probe_bounded_wait(self._h, C.c_uint32(int(spins)), C.byref(ran), C.byref(us),
+                                              C.c_void_p(_stream(stream))), "vattn_probe_bounded_wait")
+        return int(ran.value), int(us.value)
 
     def last_launch_count(self) -> int:
         return int(lib().vattn_last_launch_count(self._h))

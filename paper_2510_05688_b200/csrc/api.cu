@@ -21,7 +21,7 @@ struct vattn_plan {
   // derived
   int G, npad, nwords, dense_splits, stat_splits, stat_splits_base;
   size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_holes, off_dyn, off_meta, off_stat,
-      off_piv, off_det, off_gmeta, off_gat, off_dense, total;
+      off_piv, off_det, off_gmeta, off_probe, off_gat, off_dense, total;
   int gat_slots;
   // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
   struct HostStep {
@@ -116,6 +116,7 @@ void derive(vattn_plan* pl) {
   pl->off_piv = take(BH * (D + 1) * sizeof(double));
   pl->off_det = take(BH * (D + 1) * sizeof(double));
   pl->off_gmeta = take(2 * BH * sizeof(int4));
+  pl->off_probe = take(4 * sizeof(unsigned));
   // partial slots (chunks) per head of the gather kernel: 32, except that a handful of heads may use more of
   // the 8 CTAs per SM (64 to 128 chunks each when that many fit the grid at once)
   {
@@ -574,6 +575,34 @@ int vattn_last_status(vattn_plan* plan, void* stream, uint32_t* bits) {
   CU(cudaMemcpyAsync(bits, dev, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
   CU(cudaMemsetAsync(dev, 0, sizeof(unsigned), st));
   CU(cudaStreamSynchronize(st));
+  return VATTN_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The bounded wait on its own: a kernel polls a word of the workspace that nothing publishes, with the given poll
+// limit, and reports how the wait ended.  No other kernel is involved: what the caller sees is what a CTA of the
+// step sees when its producer never publishes (it then falls back to the grid-level dependency wait).
+__global__ void k_probe_wait(const unsigned* word, unsigned spins, unsigned* result) {
+  if (threadIdx.x == 0) {
+    const unsigned long long t0 = gtime_ns();
+    const unsigned v = wait_word32(word, spins);
+    result[0] = v == 0u ? 1u : 0u;                     // 1: the wait ran out
+    result[1] = (unsigned)((gtime_ns() - t0) / 1000ull);      // microseconds spent waiting
+  }
+}
+
+int vattn_probe_bounded_wait(vattn_plan* plan, uint32_t spins, uint32_t* ran_out, uint32_t* waited_us, void* stream) {
+  if (!plan || !ran_out || !waited_us || spins == 0 || spins > (1u << 20)) return VATTN_ERR_INVALID_ARG;
+  if (!plan->ws) return VATTN_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned* dev = reinterpret_cast<unsigned*>(static_cast<unsigned char*>(plan->ws) + plan->off_probe);
+  CU(cudaMemsetAsync(dev, 0, 4 * sizeof(unsigned), st));
+  k_probe_wait<<<1, 32, 0, st>>>(dev, spins, dev + 2);
+  CU(cudaGetLastError());
+  unsigned host[2] = {0u, 0u};
+  CU(cudaMemcpyAsync(host, dev + 2, 2 * sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  *ran_out = host[0]; *waited_us = host[1];
   return VATTN_OK;
 }
 

@@ -43,7 +43,6 @@ constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
 constexpr int UNROLL = 4;         // rows in flight per row group (16-byte slices kept raw until used); 8 and 2 are slower
 constexpr int MAXS = 32;           // most chunks (partials) per head, per-head decomposition
-constexpr unsigned READY_SPINS = 1u << 16;   // polls of a head's "budget published" word before the grid-level wait takes over
 constexpr int FLAT_MAX_HEADS = VATTN_GATHER_FLAT_HEADS;
 constexpr int MIN_CHUNK = 64;      // rows of a chunk in the per-head decomposition are >= 4 * MIN_CHUNK
 
@@ -352,16 +351,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
   for (int u = blockIdx.x; u < BH * p.gat_slots; u += gridDim.x) {
     const int bh = u % BH, ci = u / BH;
     if (tid == 0) {
-      unsigned v = 0u;
-      if (!waited) {
-        const unsigned* fl = p.tickets + bh;
-        for (unsigned it = 0; it < READY_SPINS; ++it) {     // relaxed polls, one acquire at the end
-          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(fl) : "memory");
-          if (v != 0u) break;
-          __nanosleep(128);
-        }
-        asm volatile("fence.acq_rel.gpu;" ::: "memory");
-      }
+      const unsigned v = waited ? 0u : wait_word32(p.tickets + bh, VATTN_WORD_SPINS);
       s_ready = v;
     }
     __syncthreads();

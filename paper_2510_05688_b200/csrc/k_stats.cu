@@ -30,7 +30,6 @@ constexpr int NT = 128;
 constexpr int NWARP = NT / 32;
 constexpr int UN = 2;            // rows per batch of a row group; two batches are in flight (double buffer)
 constexpr int MAXS = VATTN_STAT_MAXS;   // most split CTAs per head and kind
-constexpr unsigned FLAG_SPINS = 1u << 16;   // polls of a per-head flag (about 10 ms) before the grid-level wait takes over
 
 // 16-byte row slices, fetched with streaming loads: a row is read once, so it should be the first to leave the
 // caches (the scores, index lists and partials that the step re-reads stay in L2)
@@ -134,7 +133,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   // ---- everything this function reads from memory is requested up front (one round trip): the head's record,
   //      the pivot, and the partials: thread e adds element e of both kinds in split order, threads 0..3 the scalar
   //      sums (kind 0 = deterministic rows: [D] = D_f; kind 1 = base-sample rows: [D] = Sw, [D+1] = Sww, [D+2] = Srr)
-  DBGX(bh, 0);
   HeadMeta mt = ld_meta(p.meta + bh);
   const double* src = p.stat_part + (long long)bh * 2 * MAXS * NE;
   const int S0 = p.stat_splits, S1 = p.stat_splits_base;
@@ -178,7 +176,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   if (tid == 0) piv[D] = b0 > 0 ? pvD : 0.0;
   __syncthreads();
   DBGT(30);
-  DBGX(bh, 1);
   double* det = p.det_sums + (long long)bh * (D + 1);
   for (int e = tid; e < D; e += NT) det[e] = tot[e];
   if (warp == 0) {
@@ -205,7 +202,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
     double sigma2 = 0.0, trace = 0.0, Dhat = Dfv;
     int bD = 0, bN = 0, bS = 0, bf = 0;
-    DBGX(bh, 2);
     if (n_s > 0) {
       const double Swv = __shfl_sync(FULLMASK, sv, 1), Swwv = __shfl_sync(FULLMASK, sv, 2), Srrv = __shfl_sync(FULLMASK, sv, 3);
       // lane 0: the denominator chain A = n_s sigma / D_hat, lane 1: the numerator chain B = n_s sqrt(Tr) / |N_hat|,
@@ -217,7 +213,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
       const double den2 = lane == 0 ? Dhat * Dhat : nn;
       const double ab = (double)n_s * sqrt(var / den2);
       const double A = __shfl_sync(FULLMASK, ab, 0), Bn = __shfl_sync(FULLMASK, ab, 1);
-      DBGX(bh, 3);
       sigma2 = __shfl_sync(FULLMASK, var, 0);
       trace = __shfl_sync(FULLMASK, var, 1);
       // lanes 0..14: the split points of b_SDPA; lane 15: b_D; lane 16: b_N (one body: (c1 A + c2 B)^2, the
@@ -240,7 +235,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
     // I_dyn = the unmarked entries among the first J of the final sample's walk array, J = b + the marked
     // positions below J (a fixed point, reached in a few steps); budgets beyond the array take a list (below)
-    DBGX(bh, 4);
     const bool listed = bf > mt.dyn_listed;
     const int nholes = min(max(mt.holes1, 0), VATTN_BANDCAP), nholes2 = min(max(mt.holes2, 0), VATTN_BANDCAP);
     int J = bf;
@@ -287,7 +281,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     }
   }
   DBGT(32);
-  DBGX(bh, 6);
   __syncthreads();
   const int bfin = misc[4];
   int* dl = p.dyn_idx + (long long)bh * 3 * p.npad;
@@ -378,28 +371,9 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   // deterministic-row CTAs wait for "the list of I_t is written" (a 32-bit word, published first), base-row CTAs
   // for the 64-bit word
   const unsigned* fl32 = p.tickets + 4 * p.B * p.Hq + bh;
-#ifdef VATTN_X_NOPOLL
-  pdl_wait();
-  if (tid == 0) s_word = base_cta ? __ldcg(p.flags64 + bh) : 1ull;
-  if (false) {
-#else
   if (tid == 0) {
-#endif
-    const unsigned long long* fl = p.flags64 + bh;
-    unsigned long long v = 0ull;
-    // (relaxed polls, one acquire when the word has arrived: an acquire per poll would cost the SM an L1
-    // invalidation each time, for every waiting CTA)
-    for (unsigned it = 0; it < FLAG_SPINS; ++it) {
-      if (base_cta) asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fl) : "memory");
-      else {
-        unsigned v32;
-        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v32) : "l"(fl32) : "memory");
-        v = v32;
-      }
-      if (v != 0ull) break;
-      __nanosleep(128);
-    }
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    const unsigned long long v = base_cta ? wait_word64(p.flags64 + bh, VATTN_WORD_SPINS)
+                                          : (unsigned long long)wait_word32(fl32, VATTN_WORD_SPINS);
     s_word = v;
   }
   const int n = clamped_len(p, b);
@@ -606,29 +580,19 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   // (the barrier orders every thread's writes before thread 0's fence, which is cumulative; likewise on the way in)
   __syncthreads();
   DBGT(34);
-#ifdef VATTN_X_NOTICKET
-  if (false) {
-#else
   if (tid == 0) {
-#endif
     __threadfence();
     s_flag = (atomicAdd(&p.tickets[3 * p.B * p.Hq + bh], 1u) == (unsigned)(p.stat_splits + p.stat_splits_base - 1));
     __threadfence();
   }
   __syncthreads();
   if (base_cta && split == 0) DBGH(bh, 2);              // (one base CTA's rows are done)
-#ifdef VATTN_X_NOBUDGET
-  if (false) {
-#else
   if (s_flag) {
-#endif
     DBGH(bh, 3);
-    DBGX(bh, 8);
     // the rest of the list needs the selection kernel's last words (how far it listed the walk): wait for that
     // grid as a whole, which also makes "this grid has completed" imply "the selection kernel has" for the gather
     // kernel behind
     pdl_wait();
-    DBGX(bh, 9);
     DBGT(35);
     TICK_BEGIN(p, VATTN_T_BUDGET);
     head_budget(p, b, h, bh, &part[0][0], piv, pivT, s_misc);

@@ -100,12 +100,9 @@ __device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t;
 #define DBGT(k) do { TICK_BEGIN(p, 8 + (k)); TICK_END(p, 8 + (k)); } while (0)
 // per-head stamps: row 64 + 4 * bh + (k >> 1), column k & 1
 #define DBGH(bh, k) do { if ((p).dbg.kernel_ticks && threadIdx.x == 0) (p).dbg.kernel_ticks[2 * (64 + 4 * (bh) + ((k) >> 1)) + ((k) & 1)] = gtime_ns(); } while (0)
-// stamps of one head (the first), slot k < 32: row 200 + (k >> 1), column k & 1; by one thread
-#define DBGX(bh, k) do { if ((p).dbg.kernel_ticks && (bh) == 0 && (threadIdx.x & 31) == 0 && threadIdx.x < 32) (p).dbg.kernel_ticks[2 * (200 + ((k) >> 1)) + ((k) & 1)] = gtime_ns(); } while (0)
 #else
 #define DBGT(k) do { } while (0)
 #define DBGH(bh, k) do { } while (0)
-#define DBGX(bh, k) do { } while (0)
 #endif
 // rows of kernel_ticks
 #define VATTN_K_ZERO 0
@@ -398,6 +395,32 @@ __device__ __forceinline__ HeadMeta ld_meta(const HeadMeta* g) {
   u.v[4] = __ldcg(src + 4);
   return u.m;
 }
+
+// Bounded waits for a word that another kernel's CTA publishes with a release store (zero = not yet).  Relaxed polls
+// (an acquire per poll would cost the SM an L1 invalidation each time, for every waiting CTA), one acquire fence
+// at the end.  Returns the word, or zero when `spins` polls saw nothing: the caller then falls back to the
+// grid-level dependency wait (or reports it); no wait in this library is unbounded.
+__device__ __forceinline__ unsigned wait_word32(const unsigned* w, unsigned spins) {
+  unsigned v = 0u;
+  for (unsigned it = 0; it < spins; ++it) {
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(w) : "memory");
+    if (v != 0u) break;
+    __nanosleep(128);
+  }
+  asm volatile("fence.acq_rel.gpu;" ::: "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned long long wait_word64(const unsigned long long* w, unsigned spins) {
+  unsigned long long v = 0ull;
+  for (unsigned it = 0; it < spins; ++it) {
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(w) : "memory");
+    if (v != 0ull) break;
+    __nanosleep(128);
+  }
+  asm volatile("fence.acq_rel.gpu;" ::: "memory");
+  return v;
+}
+constexpr unsigned VATTN_WORD_SPINS = 1u << 16;   // polls of a published word (about 10 ms) before the fallback
 
 // launchers (one per translation unit)
 cudaError_t launch_zero(unsigned* z, size_t bytes, bool pdl, bool late, unsigned long long* ticks, cudaStream_t s);

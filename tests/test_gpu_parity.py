@@ -472,3 +472,45 @@ def test_non_finite_statistics_fall_back_to_the_whole_residual():
     assert int(dbg["dyn_cnt"][0, 0]) == n_s and int(dbg["budgets"][0, 0, 3]) == n_s
     assert np.array_equal(dbg["dyn_idx"][0, 2], dbg0["dyn_idx"][0, 2])
     assert np.array_equal(dbg["budgets"][0, 2:], dbg0["budgets"][0, 2:])    # KV head 1 does not see the row
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    # The step's kernels wait for one another's published words with a poll limit.  Here the wait primitive runs
+    # alone on a word that nothing publishes: it must give up at its limit (no hang), report that, and leave the
+    # context usable: a whole step afterwards still matches the oracle.
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [700, 333], Hq=4, Hkv=2)
+    plan = vb.plan_for_case(case)
+    plan.set_params(**case.params)
+    ran_out, waited_us = plan.probe_bounded_wait(2000)
+    assert ran_out == 1
+    assert 50 <= waited_us <= 200000, waited_us           # 2,000 polls of at least 128 ns each, far below a second
+    ran_out2, waited_us2 = plan.probe_bounded_wait(20000)
+    assert ran_out2 == 1 and waited_us2 > waited_us
+    with pytest.raises(vb.VattnError):
+        plan.probe_bounded_wait(0)
+    check(case)
+
+
+def test_budgets_beyond_the_walk_array_and_up_to_the_whole_residual():
+    # A small base rate makes the final sample's walk array (about eight base budgets) short, a small eps makes the
+    # budgets long: some heads end between the array's end and the whole residual (their entries beyond the array
+    # are computed by the gather kernel), others take the whole residual (token order).
+    rng = np.random.default_rng(91)
+    lens = [int(x) for x in rng.integers(2500, 6000, size=3)]
+    case = small("bf16", lens, Hq=8, Hkv=2, sink=8, window=16, k=48)
+    case.params = dict(case.params, base_rate=0.01)
+    far, whole = 0, 0
+    for eps in (0.2, 0.08, 0.03, 0.01):
+        case.eps = eps
+        out, dbg, det, plan = check(case)
+        b = np.asarray(dbg["budgets"])[..., 3].reshape(-1).astype(np.int64)
+        b0 = np.asarray(dbg["base_cnt"]).reshape(-1).astype(np.int64)
+        n_s = np.asarray(dbg["stats"])[..., 5].reshape(-1).astype(np.int64)
+        far += int(((b > 9 * b0) & (b < n_s)).sum())
+        whole += int(((b == n_s) & (n_s > 0)).sum())
+    assert far > 0 and whole > 0, (far, whole)
+    case32 = small("fp32", lens[:2], Hq=4, Hkv=2, sink=8, window=16, k=48)
+    case32.params = dict(case32.params, base_rate=0.01)
+    case32.eps = 0.05
+    check(case32)
