@@ -508,12 +508,16 @@ def main():
     es, d, Hq, Hkv = 2, case.head_dim, case.num_q_heads, case.num_kv_heads
     n_tot = int(case.seq_lens.sum())
     n_f = kks.sum() + Hq * (min(case.sink, n_tot) + min(case.window, n_tot))
+    # Entries of a walk that hold c residual tokens: c * |M| / n_s (members of I_t sit among them, marked).
+    mlen_tot = n_tot - Hq * 0 - (min(case.sink, n_tot) + min(case.window, n_tot))        # middle range of the one row
+    infl = mlen_tot / max(1.0, float(mlen_tot - kks.mean()))
+    walk_entries = float((b0s * 1.04 + 8).sum() + np.minimum(8.3 * b0s + 8, mlen_tot).sum())   # both walk arrays, all heads
     alg = {
         "k_score": n_tot * Hkv * d * es + n_tot * Hq * 4,
-        "k_walk": int(5 * b0s.sum()) * 4,
-        "k_select": n_tot * Hq * 4 + int(kks.sum()) * 8 + int(b0s.sum()) * 8 + int(min(8 * b0s.max(), n_tot)) * Hq * 12,
-        "k_stats": int(n_f + b0s.sum()) * d * es * 2,
-        "k_gather": int(b_dyn.sum()) * (d * es + 12),
+        "k_walk": int(walk_entries * 8),                                   # token + physical slot per entry
+        "k_select": n_tot * Hq * 4 + int(kks.sum()) * 16,                  # scores once; I_t written (8 B) and read back, marks
+        "k_stats": int(n_f + b0s.sum() * infl) * (d * es * 2 + 8),         # K and V rows of I_f and the base prefix, entries
+        "k_gather": int(b_dyn.sum() * infl) * (d * es + 12),               # V row, token, slot, score of every entry visited
     }
     rows_bytes = alg["k_stats"] + alg["k_gather"]
     traffic, traffic_note = read_traffic()
@@ -542,9 +546,13 @@ def main():
         g = bytes_ / (us * 1e-6) / 1e9
         return {"us": round(us, 2), "achieved": round(g, 1), "frac": round(g / peak, 4), "frac_of_8TBs_nominal": round(g / 8000.0, 4)}
     # the row kernels (statistics, final sample): device-side spans inside graph-replayed steps
-    rows_span = None
-    if timeline["k_stats"][0] is not None and timeline["k_gather"][1] is not None:
-        rows_span = timeline["k_gather"][1] - timeline["k_stats"][0]
+    # (the row kernels' CTAs are resident, waiting, long before they have work: their spans start when the last head's
+    # I_t is complete, the gather's when the last budget is known)
+    rows_span = stats_span = None
+    if timeline["topk"][1] is not None and timeline["k_gather"][1] is not None:
+        rows_span = timeline["k_gather"][1] - timeline["topk"][1]
+    if timeline["topk"][1] is not None and timeline["budget"][1] is not None:
+        stats_span = timeline["budget"][1] - timeline["topk"][1]
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -587,8 +595,9 @@ def main():
         # the gather / reduce part of the step (rows of I_f, I_bs and I_dyn) and the whole step, against the same peak
         "roofline_rows": dict(frac_of(rows_bytes, rows_span) or {}, kernel="k_stats + k_gather", alg_bytes=int(rows_bytes),
                               traffic=(traffic.get("k_stats", 0) + traffic.get("k_gather", 0)) or None,
-                              timing="first CTA of k_stats to last CTA of k_gather (%globaltimer), graph-replayed steps"),
-        "roofline_k_stats": dict(frac_of(alg["k_stats"], span("k_stats")) or {}, alg_bytes=int(alg["k_stats"])),
+                              timing="last head's I_t complete to last CTA of k_gather (%globaltimer), graph-replayed steps"),
+        "roofline_k_stats": dict(frac_of(alg["k_stats"], stats_span) or {}, alg_bytes=int(alg["k_stats"]),
+                                 timing="last head's I_t complete to last budget known (marking, rows, budget)"),
         "roofline_k_gather": dict(frac_of(alg["k_gather"], (timeline["k_gather"][1] - timeline["budget"][1])
                                           if timeline["k_gather"][1] and timeline["budget"][1] else None) or {},
                                   alg_bytes=int(alg["k_gather"]), timing="last budget known to last CTA of k_gather"),
