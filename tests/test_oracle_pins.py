@@ -309,6 +309,32 @@ def test_p3_eps_delta_definition_over_1000_seeds():
     assert fails / T <= delta + slack
 
 
+def test_p3_nested_base_sample_failure_rate_is_measured():
+    # nested_base = 1: the base sample is the first b0 residual tokens of the final sample's own walk, so the
+    # budget depends on rows that are also in the sample.  The (eps, delta) statement is measured, not assumed:
+    # 1,000 seeds of the same case as above, failure rate within the same statistical slack.  (Measured when this
+    # test was written: independent samples 0 failures, nested 0 failures of 1,000; the bound is delta = 0.1.)
+    eps = delta = 0.1
+    case = synth.make_case("p3", dtype="fp32", B=1, Hq=1, Hkv=1, d=64, seq_lens=[8192], sink=128, window=128,
+                           k=int(0.025 * 8192), eps=eps, delta=delta, seed=0, gen_seed=31337, key_std=0.1,
+                           rho_v=2.0, heavy=None, params=dict(base_rate=0.025, nested_base=1))
+    scale = float(np.float32(1.0 / 8.0))
+    ref = torch_sdpa(case, 0, 0, scale)
+    T, fails, used, nested_ok = 1000, 0, [], 0
+    for seed in range(T):
+        case.seed = seed
+        _, det = run_oracle(case)
+        r = det[(0, 0)]
+        used.append(r["b"] / r["n_s"])
+        nested_ok += set(r["I_bs"].tolist()) <= set(r["I_dyn"].tolist())
+        err = np.linalg.norm(r["out"] - ref) / np.linalg.norm(ref)
+        fails += err > eps
+    assert nested_ok == T
+    assert np.mean(used) < 0.5
+    print("nested P3: failures", fails, "of", T, "mean b/n_s", float(np.mean(used)))
+    assert fails / T <= delta + 3.0 * math.sqrt(delta * (1 - delta) / T)
+
+
 # ----------------------------------------------------------------------------- P4
 def test_p4_normal_quantiles_table():
     for line in open(os.path.join(GOLD, "normal_quantiles.txt")):
