@@ -404,8 +404,13 @@ def main():
         plan.set_params(**dict(case.params, rng_head_is_kv=1))
         grp_graphs = capture(False)
         ms_grp, _, _ = timed(grp_graphs, min(args.steps, 500), args.warmup)
-        plan.set_params(**case.params)
         del grp_graphs
+        # nested samples: the base sample is the head of the final sample's own walk (I_bs inside I_dyn)
+        plan.set_params(**dict(case.params, nested_base=1))
+        nst_graphs = capture(False)
+        ms_nst, _, _ = timed(nst_graphs, min(args.steps, 500), args.warmup)
+        plan.set_params(**case.params)
+        del nst_graphs
 
         # optional external context: a third-party dense paged-decode kernel on the same cache
         fi_us = None
@@ -577,6 +582,7 @@ def main():
                    "mean_budget": float(b_dyn.mean()), "status_bits": status, "step_us_percentiles": step_pct,
                    "kv_gather_variant_us_per_step": round(ms_kv * 1e3, 2),
                    "kv_head_sampling_keys_variant_us_per_step": round(ms_grp * 1e3, 2),
+                   "nested_base_variant_us_per_step": round(ms_nst * 1e3, 2),
                    "value_is": "max-over-ranks step time / n_gpus (each rank runs its own layer)"},
         "e2e": {"value": ms_e2e_max * 1e3 / world, "unit": UNIT,
                 "h2d_bytes_per_step": int(qh.numel() * 2 + bth.numel() * 4 + slh.numel() * 4),

@@ -30,12 +30,14 @@ namespace {
 // b: the budget; L: entries to visit (a prefix of the final sample's walk array, members of I_t marked, or the b
 // entries of the head's list when `list` is set); n = 0: an empty row
 // W1: entries of the walk array (the gather computes the ones beyond it)
-struct GMeta { int b, n_s; float m; int n, L, list, W1; };
+// start: entries before it are accounted for already (nested samples: the base sample's rows)
+struct GMeta { int b, n_s; float m; int n, L, list, W1, start; };
 __device__ __forceinline__ GMeta ld_gmeta(const int4* g) {
   const int4 v = __ldcg(g);
   GMeta r; r.b = v.x; r.n_s = v.y; r.m = __int_as_float(v.z);
   r.n = v.w < 0 ? 0 : 1; r.L = v.w < 0 ? 0 : (v.w >> 1); r.list = v.w < 0 ? 0 : (v.w & 1);
-  r.W1 = __ldcg(reinterpret_cast<const int*>(g + 1));
+  const int2 w = __ldcg(reinterpret_cast<const int2*>(g + 1));
+  r.W1 = w.x; r.start = w.y;
   return r;
 }
 
@@ -291,7 +293,7 @@ __device__ __forceinline__ typename G::Far far_setup(const Prob& p, int bh, cons
   typename G::Far far;
   far.ident = meta.n > 0 && !meta.list && meta.b >= meta.n_s && meta.b > 0;
   far.W1 = far.ident ? 0 : meta.W1;
-  far.on = meta.n > 0 && !meta.list && nb > far.W1;
+  far.on = meta.n > 0 && !meta.list && meta.L > far.W1;
   far.s0 = 0; far.mlen = 1; far.keys = s_keys; far.mt = s_mt;
   if (far.on) {
     const int b = bh / p.Hq, h = bh % p.Hq;
@@ -316,13 +318,13 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   pdl_wait();
   const int bh = blockIdx.z * p.Hq + blockIdx.y;
   const GMeta meta = ld_gmeta(p.gat_meta + 2 * bh);
-  const int nb = meta.n > 0 ? meta.L : 0;              // entries to visit
+  const int nb = meta.n > 0 ? meta.L - meta.start : 0; // entries to visit: [start, L)
   // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
   // (with this many heads the kernel is throughput-bound: 4 batches per row group amortise the fixed hops)
   const int chunk = max(4 * MIN_CHUNK, (nb + MAXS - 1) / MAXS);
   const int nslots = max(1, (nb + chunk - 1) / chunk);
   if ((int)blockIdx.x >= nslots) return;
-  const int r_begin = min(nb, (int)blockIdx.x * chunk), r_end = min(nb, r_begin + chunk);
+  const int r_begin = meta.start + min(nb, (int)blockIdx.x * chunk), r_end = min(meta.L, r_begin + chunk);
   const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
   if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
   else G::template run<false>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
@@ -358,12 +360,12 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
     if (!waited && s_ready == 0u) { pdl_wait(); waited = true; }      // uniform over the CTA
     DBGT(21);
     const GMeta meta = ld_gmeta(p.gat_meta + 2 * bh);
-    const int nb = meta.n > 0 ? meta.L : 0;            // entries to visit
+    const int nb = meta.n > 0 ? meta.L - meta.start : 0;       // entries to visit: [start, L)
     const int batches = (nb + BATCH - 1) / BATCH;
     const int rows = BATCH * max(1, (batches + p.gat_slots - 1) / p.gat_slots);
     const int nslots = max(1, (nb + rows - 1) / rows); // a head without samples still writes its output
     if (ci < nslots) {
-      const int r_begin = min(nb, ci * rows), r_end = min(nb, r_begin + rows);
+      const int r_begin = meta.start + min(nb, ci * rows), r_end = min(meta.L, r_begin + rows);
       const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
       if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);
       else G::template run<false>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);

@@ -34,7 +34,6 @@ constexpr int NT = SEL_THREADS;
 constexpr int NWARP = NT / 32;
 constexpr int HBINS = 2048;            // bins of one radix level
 constexpr int ALLCAP = 4096;           // candidates of a head
-constexpr int WPT = 8;                 // walk positions per thread and round
 constexpr unsigned FULL = 0xFFFFFFFFu;
 
 struct Sm {
@@ -913,7 +912,7 @@ __global__ void __launch_bounds__(256) k_walk(const Prob p) {
 cudaError_t launch_walk(const Prob& p, cudaStream_t s) {
   // positions per head: about 1.03 (b0 + 8 b0), or the whole middle range under a forced budget
   const double b0max = (double)p.base_rate * (double)p.max_seq_len + 2.0;
-  double pos = p.force_budget >= 0 ? (double)p.max_seq_len + 1.1 * b0max : 9.6 * b0max + 64.0;
+  double pos = p.force_budget >= 0 ? (double)p.max_seq_len + 1.1 * b0max : (1.2 + 1.05 * VATTN_WALK_B0S) * b0max + 64.0;
   if (pos > 2.0 * p.max_seq_len) pos = 2.0 * p.max_seq_len;
   int gx = (int)(pos / 256.0) + 1;
   if (gx > 64) gx = 64;

@@ -177,7 +177,6 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   __syncthreads();
   DBGT(30);
   double* det = p.det_sums + (long long)bh * (D + 1);
-  for (int e = tid; e < D; e += NT) det[e] = tot[e];
   if (warp == 0) {
     const double* t0 = tot;
     const double* t1 = tot + NE;
@@ -186,8 +185,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
       const int S = lane == 0 ? S0 : S1;
       for (int sp = 0; sp < S; ++sp) sv += scal[MAXS * lane + sp];
     }
-    const double Dfv = __shfl_sync(FULLMASK, sv, 0);
-    if (lane == 0) det[D] = Dfv;
+    const double Dfv = __shfl_sync(FULLMASK, sv, 0), sv1 = __shfl_sync(FULLMASK, sv, 1);
     double nn = 0.0, sr2 = 0.0;                        // |N_hat|^2 and sum_j (sum_i r'_ij)^2
     for (int e = lane; e < D; e += 32) {
       const double srj = t1[e];
@@ -259,15 +257,15 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
       }
     }
     if (lane == 0) {
-      misc[4] = bf; misc[5] = listed ? 1 : 0;
-      p.meta[bh].b = bf;
       // the whole residual: every middle token is visited (in token order), members of I_t weigh nothing
       if (!listed && bf >= n_s) J = mt.l_start - mt.s0;
-      p.gat_meta[2 * bh] = make_int4(bf, n_s, __float_as_int(mt.m), (J << 1) | (listed ? 1 : 0));
-      p.gat_meta[2 * bh + 1] = make_int4(mt.dyn_J, 0, 0, 0);
-      if (!listed) {                                   // "the budget is known" for the gather kernel's CTAs of this head
-        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
-      }
+      // nested samples: the base sample's rows are the first b0 rows of I_dyn and their sums are known here (in
+      // fp64, from rescored weights): they are folded into the deterministic sums (scaled like the sample), and the
+      // gather kernel starts behind them.  Not for lists, nor when the whole residual is visited in token order.
+      const bool fold = p.nested_base && !listed && !mt.base_list && bf < n_s && b0 > 0 && mt.base_J <= J;
+      misc[4] = bf; misc[5] = listed ? 1 : 0; misc[6] = J; misc[7] = fold ? mt.base_J : 0;
+      tot[D] = Dfv; tot[NE + D] = sv1;                 // D_f and the base sample's shifted sum of weights, for the sums below
+      p.meta[bh].b = bf;
       if (p.dbg.dyn_cnt) p.dbg.dyn_cnt[bh] = bf;
       if (p.dbg.budgets) {
         int* o = p.dbg.budgets + bh * 4;
@@ -283,6 +281,22 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   DBGT(32);
   __syncthreads();
   const int bfin = misc[4];
+  {
+    // N_f and D_f for the gather kernel's last finisher (with the base sample's share when it is folded in), then
+    // the head's record for the gather kernel, then "the budget is known".  The barrier orders every thread's
+    // writes before thread 0's release, which is cumulative.
+    const int start = misc[7];
+    const double f = (start > 0) ? (double)n_s / (double)bfin : 0.0;
+    for (int e = tid; e <= D; e += NT)
+      det[e] = tot[e] + (start > 0 ? f * (tot[NE + e] + (double)b0 * piv[e]) : 0.0);
+    __syncthreads();
+    if (tid == 0) {
+      p.gat_meta[2 * bh] = make_int4(bfin, n_s, __float_as_int(mt.m), (misc[6] << 1) | misc[5]);
+      p.gat_meta[2 * bh + 1] = make_int4(mt.dyn_J, start, 0, 0);
+      if (!misc[5])                                    // (a listed head publishes when its list is complete)
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.tickets + bh), "r"(1u) : "memory");
+    }
+  }
   int* dl = p.dyn_idx + (long long)bh * 3 * p.npad;
   // ---- I_dyn as a list: budgets beyond the walk array (unusual: saturated budgets), and for the debug buffer
   if (bfin > mt.dyn_listed || (p.dbg.dyn_idx && bfin > 0)) {

@@ -8,6 +8,9 @@
 #define VATTN_MAX_SEQ (1 << 18)        // longest sequence a plan accepts
 #define VATTN_BANDCAP 1024             // near-tie top-k candidates ranked from a list (more: exact radix select)
 #define SEL_THREADS 1024               // threads of the selection kernel (one CTA per head)
+#ifndef VATTN_WALK_B0S
+#define VATTN_WALK_B0S 8                 // base budgets of the final walk that the walk kernel lays out ahead
+#endif
 #define VATTN_STAT_MAXS 16             // most split CTAs per head and row kind of the statistics kernel
 #define VATTN_GATHER_FLAT_HEADS 128    // the gather kernel's flat decomposition serves up to this many heads ...
 #define VATTN_GATHER_FLAT_SLOTS 32     // ... with up to this many chunks (partials) each
@@ -293,7 +296,7 @@ __device__ __forceinline__ int walk_region(int want, int n_s, int mlen, int kk) 
 // that make the final-sample kernel walk on), or the forced budget
 __device__ __forceinline__ int dyn_listed_want(const Prob& p, int n_s, int b0) {
   if (n_s <= 0) return 0;
-  return min(n_s, p.force_budget >= 0 ? p.force_budget : 8 * b0);
+  return min(n_s, p.force_budget >= 0 ? p.force_budget : VATTN_WALK_B0S * b0);
 }
 // round keys of one (batch row, head, stream) into keys[0..8): two threads, one Philox call each
 __device__ __forceinline__ void walk_keys(const Prob& p, int b, int hrng, int stream, int half, unsigned* keys) {
