@@ -107,7 +107,8 @@ typedef struct {
 
 /* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG,
  * UNSUPPORTED (head_dim other than 64 / 128, block_size other than 16, more than 64 query heads per KV head,
- * max_seq_len above 262,144, a bf16 batch above 1,536 rows). */
+ * max_seq_len above 262,144, a bf16 batch above 1,536 rows, a batch above 32,767 rows or more than 65,535
+ * (batch row, query head) pairs: the kernels' grid dimensions). */
 int    vattn_plan_create(const vattn_shape* shape, vattn_plan** out);
 void   vattn_plan_destroy(vattn_plan* plan);
 
@@ -138,7 +139,9 @@ int    vattn_set_debug(vattn_plan* plan, const vattn_debug* debug);
  * c = 0, 1, and whose round function is xor with the round key followed by three multiply / xor-shift steps.
  * Degenerate inputs: n = 0 -> out row = 0; sink+window >= n -> exact attention, budget 0;
  * k larger than the middle range is clipped.
- * eps, delta in (0,1).  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ * eps, delta in (0,1).  Errors: INVALID_ARG, WORKSPACE, CUDA.  The step is several kernel launches: after
+ * VATTN_ERR_CUDA some of them may have been enqueued already (they run; `out` is then undefined), and the
+ * first kernel waits for whatever the caller enqueued on `stream` before the call.
  */
 int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
                  const int32_t* block_table, const int32_t* seq_lens,
@@ -169,14 +172,16 @@ int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, con
  *   - All calls, from every thread and stream, share the one array: two calls that overlap on the GPU
  *     race.  Serialise them on one stream or with events.  The part that must start at zero is cleared
  *     on `stream` at the start of every call.
- *   - Block-table entries outside [0, num_blocks) are read as page 0, as in vattn_dense_decode, but there
- *     is no status word to query.
+ *   - Block-table entries outside [0, num_blocks) are read as page 0 and sequence lengths are clamped, as in
+ *     vattn_dense_decode; the status bits of the last call on the current device (also WAIT_TIMEOUT, after
+ *     which `out` is invalid) are read with vattn_noalloc_last_status, which waits for `stream`.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE (too large), CUDA.
  */
 #define VATTN_NOALLOC_SCRATCH_BYTES (4u << 20)
 int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale, const void* q, const void* k_cache,
                                const void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
                                void* out, void* stream);
+int vattn_noalloc_last_status(uint32_t* bits /* host */, void* stream);
 
 /* Same step as vattn_decode with HOST buffers for q, block_table, seq_lens and out (the caches stay on
  * the device): copies the inputs in, runs the step, copies `out` back and waits for it.  `staging` is a

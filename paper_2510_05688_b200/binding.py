@@ -19,7 +19,7 @@ EXPORTS = ["vattn_plan_create", "vattn_plan_destroy", "vattn_workspace_bytes", "
            "vattn_set_params", "vattn_set_debug", "vattn_decode", "vattn_dense_decode",
            "vattn_host_staging_bytes", "vattn_decode_host", "vattn_last_status", "vattn_last_launch_count",
            "vattn_strerror", "vattn_normal_quantile", "vattn_set_profiling", "vattn_read_profile",
-           "vattn_dense_decode_noalloc", "vattn_set_stop_after", "vattn_probe_bounded_wait"]
+           "vattn_dense_decode_noalloc", "vattn_set_stop_after", "vattn_probe_bounded_wait", "vattn_noalloc_last_status"]
 NOALLOC_SCRATCH_BYTES = 4 << 20
 KERNEL_NAMES = ["k_score", "k_walk", "k_select", "k_stats", "k_gather"]
 NUM_TICKS = 8
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
     L.vattn_decode_host.restype = i32
     L.vattn_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     L.vattn_last_status.restype = i32
+    L.vattn_noalloc_last_status.argtypes = [C.POINTER(C.c_uint32), vp]
+    L.vattn_noalloc_last_status.restype = i32
     L.vattn_probe_bounded_wait.argtypes = [vp, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), vp]
     L.vattn_probe_bounded_wait.restype = i32
     L.vattn_last_launch_count.argtypes = [vp]
@@ -268,6 +270,13 @@ def dense_decode_noalloc(shape: Shape, q, k_cache, v_cache, block_table, seq_len
     return int(lib().vattn_dense_decode_noalloc(C.byref(shape), float(scale), _ptr(q), _ptr(k_cache), _ptr(v_cache),
                                                 _ptr(block_table), _ptr(seq_lens), _ptr(out),
                                                 C.c_void_p(_stream(stream))))
+
+
+def noalloc_last_status(stream=None) -> int:
+    """Status bits of the last dense_decode_noalloc call on the current device (waits for the stream)."""
+    bits = C.c_uint32(0)
+    _check(lib().vattn_noalloc_last_status(C.byref(bits), C.c_void_p(_stream(stream))), "vattn_noalloc_last_status")
+    return int(bits.value)
 
 
 def normal_quantile(x: float) -> float:

@@ -232,6 +232,8 @@ int vattn_plan_create(const vattn_shape* shape, vattn_plan** out) {
     return VATTN_ERR_INVALID_ARG;
   if (s.num_q_heads % s.num_kv_heads != 0) return VATTN_ERR_INVALID_ARG;
   if (s.batch > 65535 || s.num_q_heads > 65535) return VATTN_ERR_INVALID_ARG;
+  // grid dimensions y and z hold (batch row, head) pairs and twice the batch
+  if (s.batch > 32767 || (long long)s.batch * s.num_q_heads > 65535) return VATTN_ERR_UNSUPPORTED;
   // the bf16 score kernel keeps two per-row tables of the batch in shared memory beside its page ring
   if (s.dtype == VATTN_DTYPE_BF16 && s.batch > VATTN_MAX_BATCH_BF16) return VATTN_ERR_UNSUPPORTED;
   if (s.head_dim != 64 && s.head_dim != 128) return VATTN_ERR_UNSUPPORTED;

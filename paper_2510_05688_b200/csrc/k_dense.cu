@@ -562,3 +562,15 @@ extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale,
   if (launch_dense(p, st, nullptr) != cudaSuccess) return VATTN_ERR_CUDA;
   return VATTN_OK;
 }
+
+// Status bits (VATTN_STATUS_*) that the kernels of the last vattn_dense_decode_noalloc call on the current device
+// left in the fixed array's first word; waits for `stream`.
+extern "C" int vattn_noalloc_last_status(uint32_t* bits, void* stream) {
+  if (!bits) return VATTN_ERR_INVALID_ARG;
+  void* base = nullptr;
+  if (noalloc_scratch(&base) != cudaSuccess) return VATTN_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(bits, base, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VATTN_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return VATTN_ERR_CUDA;
+  return VATTN_OK;
+}

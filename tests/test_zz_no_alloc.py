@@ -59,3 +59,23 @@ def test_noalloc_rejects_problems_beyond_the_fixed_scratch():
     bad = vb.Shape(1, 8, 2, 96, 16, case.max_blocks_per_seq, case.num_blocks, 64, vb.DTYPE_BF16, 0, 0, 0)
     assert vb.dense_decode_noalloc(bad, dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"],
                                    out) == vb.ERR_UNSUPPORTED
+
+
+def test_noalloc_status_word_reports_a_bad_block_table_entry():
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = _case("bf16", 128, [700, 90], 14)
+    dev = vb.case_to_device(case)
+    plan = vb.plan_for_case(case)
+    out = torch.empty_like(dev["q"])
+    assert vb.dense_decode_noalloc(plan.shape, dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"],
+                                   dev["seq_lens"], out) == vb.OK
+    assert vb.noalloc_last_status() == 0
+    bt = dev["block_table"].clone()
+    bt[0, 3] = case.num_blocks + 5                           # outside the pool: read as page 0, reported
+    assert vb.dense_decode_noalloc(plan.shape, dev["q"], dev["k_cache"], dev["v_cache"], bt, dev["seq_lens"], out) == vb.OK
+    assert vb.noalloc_last_status() & vb.STATUS_BAD_BLOCK
+    # the next call starts from a clean word
+    assert vb.dense_decode_noalloc(plan.shape, dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"],
+                                   dev["seq_lens"], out) == vb.OK
+    assert vb.noalloc_last_status() == 0
