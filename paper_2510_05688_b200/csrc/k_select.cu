@@ -733,36 +733,27 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   int* cnts = sm.misc + 8;                             // marked positions: [0] base walk, [1] final walk; [2] members beyond its array
   int base_J = 0, base_list = 0, holes1 = 0, holes2 = 0, dyn_J = 0, dyn_listed = 0, piv_ph = 0;
   if (n_s > 0 && kk <= NT * 4) {
-    int* hp1 = p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP;     // positions inside the walk array; + BANDCAP: beyond it
     // physical slots of the first entries of the base walk: one of them is the pivot (the first unmarked entry)
     int pvph = 0;
     if (warp == 0 && lane < 4 && lane < W0) pvph = __ldcg(wa0 + p.npad + lane);
     if (tid == 0) { cnts[0] = 0; cnts[1] = 0; cnts[2] = 0; }
-    const Walk wk0 = make_walk(sm.rkeys + (p.nested_base ? 8 : 0), mlen), wk1 = make_walk(sm.rkeys + 8, mlen);
+    const Walk wk0 = make_walk(sm.rkeys + (p.nested_base ? 8 : 0), mlen);
     __syncthreads();
     DBGT(16);
+    // (only the base walk's marks stand between the top-k and the statistics kernel's base rows: the final walk's
+    // marks and member positions follow after the word for the base rows has been published)
     for (int a = tid; a < kk; a += NT) {
       const int t = __ldcg(tk + a) - s0;
-      const int x1 = walk_inv(wk1, t);
-      const int x0 = p.nested_base ? x1 : walk_inv(wk0, t);
+      const int x0 = walk_inv(wk0, t);
       if (x0 < W0) {
         wa0[x0] = -1;
         const int i0 = atomicAdd(&cnts[0], 1);
         if (i0 < HBINS) hp0[i0] = x0;
       }
-      if (x1 < W1) {
-        wa1[x1] = -1;
-        const int i1 = atomicAdd(&cnts[1], 1);
-        if (i1 < VATTN_BANDCAP) hp1[i1] = x1;
-      } else {                                         // (budgets that reach beyond the array need these)
-        const int i2 = atomicAdd(&cnts[2], 1);
-        if (i2 < VATTN_BANDCAP) hp1[VATTN_BANDCAP + i2] = x1;
-      }
     }
     __syncthreads();
     DBGT(17);
     const int H0 = cnts[0];
-    holes1 = cnts[1];
     if (H0 > HBINS) base_list = 1;
     else if (warp == 0) {
       // J = b0 + #{marked positions < J}; the pivot = the first unmarked position
@@ -788,16 +779,12 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     }
     __syncthreads();
     if (!base_list) { base_J = sm.misc[4]; piv_ph = sm.misc[5]; base_list = sm.misc[6]; }
-    holes2 = cnts[2];
-    // every member's position is known: any budget can be served as "the non-members among the first J positions"
-    // (entries beyond the array are computed by the gather kernel); else only budgets inside the array
-    if (holes1 <= VATTN_BANDCAP) { dyn_J = W1; dyn_listed = holes2 <= VATTN_BANDCAP ? n_s : W1 - holes1; }
   } else if (n_s > 0) {
     base_list = 1;
   }
   if (base_J >= (1 << 22)) base_list = 1;              // the published word has 22 bits for it
-  mt.base_J = base_J; mt.holes2 = min(holes2, VATTN_BANDCAP); mt.base_list = base_list; mt.holes1 = min(holes1, VATTN_BANDCAP);
-  mt.dyn_J = dyn_J; mt.dyn_listed = dyn_listed;
+  mt.base_J = base_J; mt.holes2 = 0; mt.base_list = base_list; mt.holes1 = 0;
+  mt.dyn_J = 0; mt.dyn_listed = 0;                     // (the final walk's fields follow below)
   DBGT(6);
 
   // The base sample as a list: for the debug buffer, and for the row kernels when the walk array fell short.
@@ -868,6 +855,33 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
                                     ((unsigned long long)(unsigned)piv_ph << 32);
     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.flags64 + bh), "l"(word) : "memory");
     DBGH(bh, 1);
+  }
+  // ---- the final walk: marks in its array, positions of all members (read by the budget code and the gather
+  //      kernel, which start after this kernel has completed)
+  if (n_s > 0 && kk <= NT * 4) {
+    int* hp1 = p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP;     // positions inside the walk array; + BANDCAP: beyond it
+    const Walk wk1 = make_walk(sm.rkeys + 8, mlen);
+    for (int a = tid; a < kk; a += NT) {
+      const int x1 = walk_inv(wk1, __ldcg(tk + a) - s0);
+      if (x1 < W1) {
+        wa1[x1] = -1;
+        const int i1 = atomicAdd(&cnts[1], 1);
+        if (i1 < VATTN_BANDCAP) hp1[i1] = x1;
+      } else {                                         // (budgets that reach beyond the array need these)
+        const int i2 = atomicAdd(&cnts[2], 1);
+        if (i2 < VATTN_BANDCAP) hp1[VATTN_BANDCAP + i2] = x1;
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      holes1 = cnts[1]; holes2 = cnts[2];
+      // every member's position is known: any budget can be served as "the non-members among the first J
+      // positions" (entries beyond the array are computed by the gather kernel); else only budgets inside the array
+      if (holes1 <= VATTN_BANDCAP) { dyn_J = W1; dyn_listed = holes2 <= VATTN_BANDCAP ? n_s : W1 - holes1; }
+      HeadMeta* gm = p.meta + bh;
+      gm->holes1 = min(holes1, VATTN_BANDCAP); gm->holes2 = min(holes2, VATTN_BANDCAP);
+      gm->dyn_J = dyn_J; gm->dyn_listed = dyn_listed;
+    }
   }
   TICK_END(p, VATTN_K_SELECT);
 }
