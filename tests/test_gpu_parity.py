@@ -514,3 +514,29 @@ def test_budgets_beyond_the_walk_array_and_up_to_the_whole_residual():
     case32.params = dict(case32.params, base_rate=0.01)
     case32.eps = 0.05
     check(case32)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("fp32", 64), ("fp32", 128), ("bf16", 64)])
+def test_sampling_keys_per_kv_head(dtype, d):
+    # rng_head_is_kv = 1: the heads of a KV-head group walk the middle range in one order (their budgets, nested
+    # base samples and top-k members still differ).  Ragged rows, an empty one, group sizes 2, 3, 4 and 8, the nested
+    # variant, budgets beyond the walk array and equal to the whole residual.
+    lens = [2300, 0, 777, 1500, 33]
+    base = dict(base_rate=0.05, rng_head_is_kv=1)
+    check(small(dtype, lens, Hq=8, Hkv=2, d=d, params=base))
+    check(small(dtype, lens, Hq=8, Hkv=2, d=d, params=dict(base, nested_base=1)))
+    check(small(dtype, lens, Hq=8, Hkv=4, d=d, params=base))                      # groups of two heads
+    check(small(dtype, lens, Hq=6, Hkv=2, d=d, params=base))                      # groups of three
+    check(small(dtype, lens, Hq=8, Hkv=1, d=d, params=base))                      # groups of eight
+    case = small(dtype, [4000, 2500], Hq=8, Hkv=2, d=d, sink=8, window=16, k=48, params=dict(base, base_rate=0.01))
+    for eps in (0.2, 0.03, 0.01):
+        case.eps = eps
+        check(case)
+
+
+def test_config2_with_sampling_keys_per_kv_head():
+    case = synth.config2_llama8b()
+    case.params = dict(case.params, rng_head_is_kv=1)
+    out, dbg, det, plan = check(case)
+    case.params = dict(case.params, nested_base=1)
+    check(case)
