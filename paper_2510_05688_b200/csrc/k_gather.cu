@@ -314,21 +314,34 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   __shared__ float s_den;
   __shared__ unsigned s_keys[8];
   __shared__ HeadMeta s_mt;
+  __shared__ unsigned s_ready;
   TICK_BEGIN(p, VATTN_K_GATHER);
-  pdl_wait();
   const int bh = blockIdx.z * p.Hq + blockIdx.y;
+  // A head's CTAs start when that head's budget is published (the statistics kernel's last CTA of the head
+  // releases a word), not when the whole statistics kernel has completed: heads finish over tens of microseconds
+  // at large batch.  Every CTA of the statistics kernel had started before this grid was launched, so the wait
+  // cannot starve; it is bounded and falls back to the grid-level wait.  CTAs leave as soon as they are done (a CTA
+  // that waited for the grid at its end would hold its slot against the CTAs behind it); one CTA does wait, so
+  // that "this grid has completed" implies "the statistics kernel has".
+  const bool anchor = blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
+  if (threadIdx.x == 0) s_ready = wait_word32(p.tickets + bh, VATTN_WORD_SPINS);
+  __syncthreads();
+  const bool waited = s_ready == 0u;
+  if (waited) pdl_wait();                               // uniform over the CTA
   const GMeta meta = ld_gmeta(p.gat_meta + 2 * bh);
   const int nb = meta.n > 0 ? meta.L - meta.start : 0; // entries to visit: [start, L)
   // chunks of at least MIN_CHUNK rows, at most MAXS of them; CTAs beyond the head's chunk count leave at once
   // (with this many heads the kernel is throughput-bound: 4 batches per row group amortise the fixed hops)
   const int chunk = max(4 * MIN_CHUNK, (nb + MAXS - 1) / MAXS);
   const int nslots = max(1, (nb + chunk - 1) / chunk);
-  if ((int)blockIdx.x >= nslots) return;
-  const int r_begin = meta.start + min(nb, (int)blockIdx.x * chunk), r_end = min(meta.L, r_begin + chunk);
-  const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
-  if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
-  else G::template run<false>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
-  TICK_END(p, VATTN_K_GATHER);
+  if ((int)blockIdx.x < nslots) {
+    const int r_begin = meta.start + min(nb, (int)blockIdx.x * chunk), r_end = min(meta.L, r_begin + chunk);
+    const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
+    if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
+    else G::template run<false>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
+    TICK_END(p, VATTN_K_GATHER);
+  }
+  if (anchor && !waited) pdl_wait();
 }
 
 template <typename T, int D, bool KV>
