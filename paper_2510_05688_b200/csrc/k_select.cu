@@ -898,21 +898,42 @@ __global__ void __launch_bounds__(256) k_walk(const Prob p) {
   const int n = clamped_len(p, b);
   const Geo geo = head_geometry(p, n);
   const int mlen = geo.l_start - geo.s0;
-  if (geo.n_s > 0) {
+  const int J0 = walk_region(geo.b0, geo.n_s, mlen, geo.kk);
+  const int J1 = walk_region(dyn_listed_want(p, geo.n_s, geo.b0), geo.n_s, mlen, geo.kk);
+  // (the grid is sized for the longest sequence a plan takes: a CTA without positions leaves before the round keys)
+  // CTA x takes positions [1024 x, 1024 x + 1024) of the two walks laid end to end.  Cycle walking repeats the
+  // network until the value falls below |M|; with |M| just above a power of two that is two passes on average and
+  // four or five for the slowest lane of a warp, so a lane does not wait for its neighbours: it has several
+  // positions to do and goes on to its next one as soon as one is finished (one pass per loop iteration).
+  constexpr int PER = 1024;
+  if (geo.n_s > 0 && (int)blockIdx.x * PER < J0 + J1) {
     const int hrng = p.rng_head_is_kv ? g : h;
     if (tid < 4) walk_keys(p, b, hrng, tid >> 1, tid & 1, keys + (tid >> 1) * 8);
     __syncthreads();
-    const int J0 = walk_region(geo.b0, geo.n_s, mlen, geo.kk);
-    const int J1 = walk_region(dyn_listed_want(p, geo.n_s, geo.b0), geo.n_s, mlen, geo.kk);
-    const Walk w0 = make_walk(keys + (p.nested_base ? 8 : 0), mlen), w1 = make_walk(keys + 8, mlen);
     int* out0 = p.walk_tok + (long long)bh * 4 * p.npad;       // [walk][tokens, physical slots][npad]
-    for (int x = blockIdx.x * 256 + tid; x < J0 + J1; x += gridDim.x * 256) {
-      const bool first = x < J0;
-      const int xx = first ? x : x - J0;
-      const int tok = geo.s0 + walk_at(first ? w0 : w1, xx);
-      int* dst = out0 + (first ? 0 : 2 * p.npad) + xx;
-      dst[0] = tok;
-      dst[p.npad] = page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15);
+#pragma unroll 1
+    for (int x_lo = (int)blockIdx.x * PER; x_lo < J0 + J1; x_lo += (int)gridDim.x * PER) {     // (the grid normally covers the range once)
+    const int x_hi = min(x_lo + PER, J0 + J1);
+#pragma unroll 1
+    for (int which = 0; which < 2; ++which) {          // the part of this CTA's range in the base walk, then in the final walk
+      const int a = which == 0 ? x_lo : max(x_lo, J0), e = which == 0 ? min(x_hi, J0) : x_hi;
+      if (a >= e) continue;
+      const Walk w = make_walk(keys + ((which == 1 || p.nested_base) ? 8 : 0), mlen);
+      const int off = which == 0 ? 0 : J0;
+      int* dst = out0 + (which == 0 ? 0 : 2 * p.npad);
+      int x = a + tid;
+      unsigned cur = (unsigned)(x - off);
+      while (x < e) {
+        cur = walk_pass(w, cur);
+        if (cur < w.mlen) {
+          const int tok = geo.s0 + (int)cur;
+          dst[x - off] = tok;
+          dst[p.npad + x - off] = page_of(p, b, tok >> 4) * VATTN_BLOCK + (tok & 15);
+          x += 256;
+          cur = (unsigned)(x - off);
+        }
+      }
+    }
     }
   }
   TICK_END(p, VATTN_K_WALK);
@@ -928,8 +949,8 @@ cudaError_t launch_walk(const Prob& p, cudaStream_t s) {
   const double b0max = (double)p.base_rate * (double)p.max_seq_len + 2.0;
   double pos = p.force_budget >= 0 ? (double)p.max_seq_len + 1.1 * b0max : (1.2 + 1.05 * VATTN_WALK_B0S) * b0max + 64.0;
   if (pos > 2.0 * p.max_seq_len) pos = 2.0 * p.max_seq_len;
-  int gx = (int)(pos / 256.0) + 1;
-  if (gx > 64) gx = 64;
+  int gx = (int)(pos / 1024.0) + 1;                    // 1024 positions per CTA
+  if (gx > 65535) gx = 65535;
   return launch_pdl(k_walk, dim3((unsigned)gx, (unsigned)(p.B * p.Hq)), dim3(256), 0, s, p);
 }
 

@@ -254,18 +254,20 @@ __device__ __forceinline__ Walk make_walk(const unsigned* keys, int mlen) {
   w.lw = wbits >> 1; w.rw = wbits - w.lw; w.mlen = (unsigned)max(mlen, 1);
   return w;
 }
-__device__ __forceinline__ int walk_at(const Walk& w, int j) {
+// one pass of the network over the domain 2^(lw + rw) (cycle walking repeats it until the value is below mlen)
+__device__ __forceinline__ unsigned walk_pass(const Walk& w, unsigned x) {
   const unsigned ml = (1u << w.lw) - 1u, mr = (1u << w.rw) - 1u;
-  unsigned x = (unsigned)j;
-  do {
-    unsigned L = x >> w.rw, R = x & mr;
+  unsigned L = x >> w.rw, R = x & mr;
 #pragma unroll
-    for (int i = 0; i < 8; i += 2) {
-      L ^= mix32(R, w.k[i]) & ml;
-      R ^= mix32(L, w.k[i + 1]) & mr;
-    }
-    x = (L << w.rw) | R;
-  } while (x >= w.mlen);
+  for (int i = 0; i < 8; i += 2) {
+    L ^= mix32(R, w.k[i]) & ml;
+    R ^= mix32(L, w.k[i + 1]) & mr;
+  }
+  return (L << w.rw) | R;
+}
+__device__ __forceinline__ int walk_at(const Walk& w, int j) {
+  unsigned x = (unsigned)j;
+  do { x = walk_pass(w, x); } while (x >= w.mlen);
   return (int)x;
 }
 // sigma^-1: the walk position at which middle token t (relative to s0) is met
