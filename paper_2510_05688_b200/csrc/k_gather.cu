@@ -103,32 +103,26 @@ struct Gather {
 #pragma unroll
       for (int u = 0; u < UNROLL; ++u) {
         const int r = r_begin + rg + (k0 + u) * RG;
-        const bool ok = (FULL || ((k0 + u < iters) && (r < r_end))) && !(FAR && r >= far.W1);
-        tok_n[u] = ok ? __ldg(dyn + r) : -1;
-        ph_n[u] = ok ? __ldg(dph + r) : 0;
+        const bool ok = (FULL || ((k0 + u < iters) && (r < r_end))) && !(FAR && far.ident);
+        // (FAR, not ident: this CTA has just extended the array over its entries: they are read back through L2)
+        tok_n[u] = ok ? (FAR ? __ldcg(dyn + r) : __ldg(dyn + r)) : -1;
+        ph_n[u] = ok ? (FAR ? __ldcg(dph + r) : __ldg(dph + r)) : 0;
       }
       if (FAR && far.ident) {                           // the whole residual: entry r is middle token r
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const int r = r_begin + rg + (k0 + u) * RG;
-          const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
-          const int tok = far.s0 + r;
-          tok_n[u] = ok ? tok : -1;
-          ph_n[u] = ok ? page_of(p, bh / p.Hq, tok >> 4) * VATTN_BLOCK + (tok & 15) : 0;
-        }
-      } else if (FAR) {                                 // lane u of a row group computes row u's entry
-        int ctok = -1, cph = 0;
+        int cph = 0;                                    // lane u of a row group looks up row u's page
         if (j < UNROLL) {
           const int r = r_begin + rg + (k0 + j) * RG;
-          if (r >= far.W1 && (FULL || ((k0 + j < iters) && (r < r_end)))) {
-            ctok = far.s0 + walk_at(make_walk(far.keys, far.mlen), r);
-            cph = page_of(p, bh / p.Hq, ctok >> 4) * VATTN_BLOCK + (ctok & 15);
+          if (FULL || ((k0 + j < iters) && (r < r_end))) {
+            const int tok = far.s0 + r;
+            cph = page_of(p, bh / p.Hq, tok >> 4) * VATTN_BLOCK + (tok & 15);
           }
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-          const int t = __shfl_sync(0xFFFFFFFFu, ctok, u, LPR), ph = __shfl_sync(0xFFFFFFFFu, cph, u, LPR);
-          if (t >= 0) { tok_n[u] = t; ph_n[u] = ph; }
+          const int r = r_begin + rg + (k0 + u) * RG;
+          const bool ok = FULL || ((k0 + u < iters) && (r < r_end));
+          tok_n[u] = ok ? far.s0 + r : -1;
+          ph_n[u] = __shfl_sync(0xFFFFFFFFu, cph, u, LPR);
         }
       }
     };
@@ -139,7 +133,7 @@ struct Gather {
     };
     // a computed entry's token may be a member of I_t (nothing marked it): its score s decides
     auto far_member = [&](int k0, int u, int tok, float s) -> bool {
-      if (!FAR || tok < 0 || r_begin + rg + (k0 + u) * RG < far.W1) return false;
+      if (!FAR || !far.ident || tok < 0) return false;
       return in_topk(*far.mt, p.vtab + (long long)bh * VATTN_BANDCAP, p.bitmap + (long long)bh * p.nwords, tok, s);
     };
     // K+V variant: the score of a sampled token is recomputed from its K row (what a selector that leaves no
@@ -287,6 +281,50 @@ struct Gather {
 };
 
 
+// Entries [x_lo, x_hi) of head bh's final walk beyond what the walk kernel laid out (budgets of more than about eight
+// base budgets): the CTA that will gather them writes them into the walk array first.  Pass 1: positions -> tokens,
+// a thread going on to its next position as soon as one cycle walk ends; pass 2: the tokens' scores decide membership
+// in I_t as the selection kernel would (marked: token -1), slots from the block table; four entries per thread and
+// round trip.  keys: the walk's round keys, mt: the head's record (both in shared memory).
+__device__ void extend_walk_array(const Prob& p, int bh, const unsigned* keys, const HeadMeta* mt, int x_lo, int x_hi) {
+  const int tid = threadIdx.x, b = bh / p.Hq;
+  int* wt = p.walk_tok + ((long long)bh * 4 + 2) * p.npad;
+  int* wp = wt + p.npad;
+  const Walk wk = make_walk(keys, mt->l_start - mt->s0);
+  {
+    int x = x_lo + tid;
+    unsigned cur = (unsigned)x;
+    while (x < x_hi) {
+      cur = walk_pass(wk, cur);
+      if (cur < wk.mlen) { wt[x] = mt->s0 + (int)cur; x += NT; cur = (unsigned)x; }
+    }
+  }
+  __syncthreads();
+  const int* vt = p.vtab + (long long)bh * VATTN_BANDCAP;
+  const float* sc = p.scores + (long long)bh * p.npad;
+  const unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
+  for (int x0 = x_lo; x0 < x_hi; x0 += 4 * NT) {
+    int tk4[4], pg4[4];
+    float s4[4];
+#pragma unroll
+    for (int q_ = 0; q_ < 4; ++q_) { const int x = x0 + q_ * NT + tid; tk4[q_] = x < x_hi ? __ldcg(wt + x) : -1; }
+#pragma unroll
+    for (int q_ = 0; q_ < 4; ++q_) {
+      s4[q_] = tk4[q_] >= 0 ? __ldg(sc + tk4[q_]) : 0.f;
+      pg4[q_] = tk4[q_] >= 0 ? page_of(p, b, tk4[q_] >> 4) : 0;
+    }
+#pragma unroll
+    for (int q_ = 0; q_ < 4; ++q_) {
+      const int x = x0 + q_ * NT + tid;
+      if (tk4[q_] >= 0) {
+        if (in_topk(*mt, vt, gbitmap, tk4[q_], s4[q_])) wt[x] = -1;
+        wp[x] = pg4[q_] * VATTN_BLOCK + (tk4[q_] & 15);
+      }
+    }
+  }
+  __syncthreads();
+}
+
 // what a unit needs for entries beyond the walk array (see Gather::Far); uniform over the CTA
 template <typename G>
 __device__ __forceinline__ typename G::Far far_setup(const Prob& p, int bh, const GMeta& meta, int nb, unsigned* s_keys, HeadMeta* s_mt) {
@@ -337,6 +375,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather(const Prob p) {
   if ((int)blockIdx.x < nslots) {
     const int r_begin = meta.start + min(nb, (int)blockIdx.x * chunk), r_end = min(meta.L, r_begin + chunk);
     const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
+    if (far.on && !far.ident && r_end > far.W1) extend_walk_array(p, bh, s_keys, &s_mt, max(r_begin, far.W1), r_end);
     if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
     else G::template run<false>(p, bh, meta, r_begin, r_end, far, blockIdx.x, nslots, part, &is_last, &s_den);
     TICK_END(p, VATTN_K_GATHER);
@@ -380,6 +419,7 @@ __global__ void __launch_bounds__(NT, 8) k_gather_flat(const Prob p) {
     if (ci < nslots) {
       const int r_begin = meta.start + min(nb, ci * rows), r_end = min(meta.L, r_begin + rows);
       const typename G::Far far = far_setup<G>(p, bh, meta, nb, s_keys, &s_mt);
+      if (far.on && !far.ident && r_end > far.W1) extend_walk_array(p, bh, s_keys, &s_mt, max(r_begin, far.W1), r_end);
       if (far.on) G::template run<true>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);
       else G::template run<false>(p, bh, meta, r_begin, r_end, far, ci, nslots, part, &is_last, &s_den);
     }
