@@ -20,7 +20,7 @@ struct vattn_plan {
   int prof_calls;           // calls recorded since the last read
   // derived
   int G, npad, nwords, dense_splits, stat_splits, stat_splits_base;
-  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_holes, off_dyn, off_meta, off_stat,
+  size_t off_scores, off_zero, zero_bytes, off_status, off_bitmap, off_vtab, off_topk, off_base, off_walk, off_holes, off_wkeys, off_dyn, off_meta, off_stat,
       off_piv, off_det, off_gmeta, off_probe, off_gat, off_dense, total;
   int gat_slots;
   // vattn_decode_host: CUDA graphs of whole host steps, one per distinct argument set (see there)
@@ -110,6 +110,7 @@ void derive(vattn_plan* pl) {
   pl->off_base = take(2 * BH * pl->npad * sizeof(int));
   pl->off_walk = take(4 * BH * pl->npad * sizeof(int));     // first walk positions of both walks: tokens, physical slots
   pl->off_holes = take(2 * BH * VATTN_BANDCAP * sizeof(int));
+  pl->off_wkeys = take(BH * 8 * sizeof(unsigned));
   pl->off_dyn = take(3 * BH * pl->npad * sizeof(int));      // tokens, physical slots, score bits
   pl->off_meta = take(BH * sizeof(HeadMeta));
   pl->off_stat = take(BH * 2 * VATTN_STAT_MAXS * (D + 3) * sizeof(double));
@@ -164,6 +165,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   p.base_idx = reinterpret_cast<int*>(w + pl->off_base);
   p.walk_tok = reinterpret_cast<int*>(w + pl->off_walk);
   p.hole_pos = reinterpret_cast<int*>(w + pl->off_holes);
+  p.wkeys = reinterpret_cast<unsigned*>(w + pl->off_wkeys);
   p.dyn_idx = reinterpret_cast<int*>(w + pl->off_dyn);
   p.meta = reinterpret_cast<HeadMeta*>(w + pl->off_meta);
   p.stat_part = reinterpret_cast<double*>(w + pl->off_stat);

@@ -333,13 +333,11 @@ __device__ __forceinline__ typename G::Far far_setup(const Prob& p, int bh, cons
   far.W1 = far.ident ? 0 : meta.W1;
   far.on = meta.n > 0 && !meta.list && meta.L > far.W1;
   far.s0 = 0; far.mlen = 1; far.keys = s_keys; far.mt = s_mt;
-  if (far.on) {
-    const int b = bh / p.Hq, h = bh % p.Hq;
-    const Geo geo = head_geometry(p, clamped_len(p, b));
-    far.s0 = geo.s0; far.mlen = geo.l_start - geo.s0;
-    if (threadIdx.x < 2 && !far.ident) walk_keys(p, b, p.rng_head_is_kv ? h / p.G : h, 1, threadIdx.x, s_keys);
+  if (far.on) {                                        // the head's record and its walk's round keys, as the selection kernel left them
+    if (threadIdx.x < 8) s_keys[threadIdx.x] = __ldcg(p.wkeys + (long long)bh * 8 + threadIdx.x);
     if (threadIdx.x == 32) *s_mt = ld_meta(p.meta + bh);
     __syncthreads();
+    far.s0 = s_mt->s0; far.mlen = s_mt->l_start - s_mt->s0;
   }
   return far;
 }

@@ -692,6 +692,8 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   TICK_END(p, VATTN_T_TOPK);
   DBGH(bh, 0);
 
+  // the final walk's round keys for the gather kernel (it extends the walk array for long budgets)
+  if (tid < 8) p.wkeys[(long long)bh * 8 + tid] = sm.rkeys[8 + tid];
   // the near-tie list for the budget's list path
   int* gvtab = p.vtab + (long long)bh * VATTN_BANDCAP;
   for (int c = tid; c < mt.nbt; c += NT) gvtab[c] = sm.vtab[c];

@@ -72,6 +72,7 @@ struct Prob {
   int* walk_tok;          // [B,Hq,2,2,npad] the first positions of both walks (computed beside the score pass): per
                           //   walk the tokens, then their physical slots.  The selection kernel marks the members
                           //   of I_t (token = -1; the slot stays valid): a sample is the unmarked entries of a prefix
+  unsigned* wkeys;        // [B,Hq,8] round keys of the final sample's walk (for the gather kernel's array extension)
   int* hole_pos;          // [B,Hq,2,VATTN_BANDCAP] positions of the marked entries of the final sample's walk array, in
                           //   no particular order (the first 256 words read INT_MAX where there is none); then the
                           //   positions of the members of I_t beyond the array
