@@ -12,6 +12,7 @@ struct vattn_plan {
   void* ws;
   size_t ws_bytes;
   bool status_ready;
+  bool dense_ready;       // the dense kernel's tickets are known to be zero (its last CTAs put them back)
   int last_launches;
   // optional per-kernel timing (events are created on first use; no device memory involved)
   bool profiling;
@@ -79,7 +80,7 @@ void derive(vattn_plan* pl) {
   const int heads = s.batch * s.num_q_heads;
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
-  const int sp = (4 * device_sm_count() + groups - 1) / groups;
+  const int sp = (8 * device_sm_count() + groups - 1) / groups;
   pl->dense_splits = sp < 1 ? 1 : (sp > 128 ? 128 : sp);
   // statistics kernel (128-thread CTAs, 5 per SM): one wave for both kinds of CTA.  The base-sample rows are on
   // the step's critical path (they wait for the sample's list), the deterministic rows start earlier: three fifths
@@ -126,7 +127,7 @@ void derive(vattn_plan* pl) {
     pl->gat_slots = BH <= VATTN_GATHER_FLAT_HEADS ? (int)flat : 32;   // per-head decomposition: up to 32 chunks
   }
   pl->off_gat = take(BH * (size_t)pl->gat_slots * (D + 1) * sizeof(float));
-  pl->off_dense = take(BH * pl->dense_splits * (D + 2) * sizeof(float));
+  pl->off_dense = take(BH * pl->dense_splits * dense_rec((int)D) * sizeof(float));
   pl->total = off;
 }
 
@@ -205,7 +206,12 @@ int prepare_stream(vattn_plan* pl, const Prob& p, cudaStream_t st, bool with_ker
   // The clearing kernel may run ahead of its stream predecessor only when that is this library's own input
   // staging kernel; a caller's kernel (a GEMM, RoPE, a KV append that writes what this step reads) is waited for.
   if (with_kernel) CU(launch_zero(p.m_ord, pl->zero_bytes, pl->inputs_just_staged, pl->inputs_just_staged, p.dbg.kernel_ticks, st));
-  else CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
+  else if (!pl->dense_ready) {
+    // the dense kernel only needs its tickets at zero, and the last CTA of every group puts its ticket back:
+    // one memset after the workspace is bound, none afterwards
+    CU(cudaMemsetAsync(p.m_ord, 0, pl->zero_bytes, st));
+    pl->dense_ready = true;
+  }
   return VATTN_OK;
 }
 
@@ -316,6 +322,7 @@ int vattn_set_workspace(vattn_plan* plan, void* dev_ptr, size_t bytes) {
   plan->ws = dev_ptr;
   plan->ws_bytes = bytes;
   plan->status_ready = false;
+  plan->dense_ready = false;
   plan->gen++;
   return VATTN_OK;
 }

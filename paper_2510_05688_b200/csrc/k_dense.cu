@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
   }
   __syncthreads();
   // CTA partial -> global: [D] unnormalised sum, m, l per head
-  constexpr int NE = D + 2;
+  constexpr int NE = dense_rec(D);
   for (int idx = tid; idx < 4 * NE; idx += NT) {
     const int hh = idx / NE, e = idx % NE;
     const int hl = hc * 4 + hh;
@@ -171,7 +171,11 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
   }
   __threadfence();
   __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.tickets[2 * p.B * p.Hq + b * p.Hq + blockIdx.y], 1u) == (unsigned)(S - 1));
+  if (tid == 0) {
+    unsigned* ticket = &p.tickets[2 * p.B * p.Hq + b * p.Hq + blockIdx.y];
+    is_last = (atomicAdd(ticket, 1u) == (unsigned)(S - 1));
+    if (is_last) *ticket = 0u;                 // every CTA of the group has drawn: ready for the next call
+  }
   __syncthreads();
   if (!is_last) return;
   __threadfence();
@@ -203,14 +207,18 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
 //                                  B = K rows read with 16-byte shared loads (k-slots mapped onto d so
 //                                      that a thread owns 8 consecutive elements of a row)
 //     out[head, dim]  += P V       A = exp(S - m) packed to bf16 straight from the S^T accumulators,
-//                                  B = V through ldmatrix.trans; V rows are copied one by one into rows
-//                                      padded to 272 bytes so the transposing loads are conflict-free
+//                                  B = V read with 16-byte shared loads from the page as it lies in the cache
+//                                      (one copy per page): a thread takes 8 consecutive dims of its four
+//                                      tokens and pairs them up with byte permutes, so column slot (block e,
+//                                      column gr) of a 64-dim half stands for dim 8 gr + e and a thread's
+//                                      accumulators are 16 consecutive dims (no transposing loads, no padding)
 constexpr int DN_WARPS = 6;
 constexpr int DN_NST = 2;
 
-__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], const void* smem_row) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem_row)));
+__device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
+  unsigned r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
 }
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // round to nearest even, lo in bits 0..15
   unsigned r;
@@ -222,10 +230,10 @@ template <int D>
 __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   constexpr int NC = D / 32;                   // 32-element chunks of a K row
   constexpr int ROWB = D * 2, KPAGE = 16 * ROWB;
-  constexpr int VROWB = ROWB + 16, VPAGE = 16 * VROWB;       // padded V rows
-  constexpr int STAGE = KPAGE + VPAGE;
+  constexpr int STAGE = 2 * KPAGE;             // a K page and a V page
+  constexpr int NH = D / 64;                   // 64-dim halves of a V row
   constexpr int NB = D / 8;                    // 8-dim column blocks of the output
-  constexpr int NE = D + 2;
+  constexpr int NE = dense_rec(D);
   extern __shared__ __align__(128) unsigned char smem_dyn[];
   __shared__ float s_m[DN_WARPS][8], s_l[DN_WARPS][8];
   __shared__ int is_last;
@@ -235,12 +243,17 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)DN_WARPS * DN_NST * STAGE) + warp * DN_NST;
   float* s_acc = reinterpret_cast<float*>(smem_dyn);          // [DN_WARPS][8][D], reuses the rings after the main loop
 
-  const int split = blockIdx.x, b = blockIdx.z, S = gridDim.x;
+  const int split = blockIdx.x, b = blockIdx.z, SG = gridDim.x;
   const int GC = (p.G + 7) >> 3;
   const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
   const int h0 = g * p.G + hc * 8, nh = min(8, p.G - hc * 8);
   const int n = clamped_len(p, b);
   const int npages = (n + 15) >> 4;
+  // a sequence takes the share of the SG splits that its length has of the longest possible one, so every
+  // CTA that works gets about the same number of pages whatever the mix of lengths; the others leave
+  const int npages_max = max(1, (p.max_seq_len + 15) >> 4);
+  const int S = min(SG, max(1, (int)(((long long)SG * npages + npages_max - 1) / npages_max)));
+  if (split >= S) return;
   const int wglob = split * DN_WARPS + warp, wtot = S * DN_WARPS;
   const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;
   const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
@@ -257,8 +270,8 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     pg_ids = (k < mine) ? page_of(p, b, wglob + k * wtot) : 0;
   };
   const unsigned long long stream_policy = l2_evict_first_policy();
-  // whole warp: lane 0 arms the barrier, then lanes 0..15 copy one V row each (into padded rows) and
-  // lanes 16..31 the K page (one copy, or one row each when rows are not contiguous)
+  // whole warp: lane 0 arms the barrier, then one copy per page (lanes 0 and 16), or, when the rows of a
+  // page are not contiguous, lanes 0..15 copy one V row each and lanes 16..31 one K row each
   auto issue = [&](int k, int pg) {
     unsigned long long* bar = &bars[k % DN_NST];
     unsigned char* dst = ring + (size_t)(k % DN_NST) * STAGE;
@@ -269,8 +282,10 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     }
     __syncwarp();
     // K and V are read once: evict-first in L2
-    if (lane < 16) bulk_g2s_stream(dst + KPAGE + lane * VROWB, vc + off + (long long)lane * p.st, ROWB, bar, stream_policy);
-    else if (p.st == D) { if (lane == 16) bulk_g2s_stream(dst, kc + off, KPAGE, bar, stream_policy); }
+    if (p.st == D) {
+      if (lane == 0) bulk_g2s_stream(dst + KPAGE, vc + off, KPAGE, bar, stream_policy);
+      else if (lane == 16) bulk_g2s_stream(dst, kc + off, KPAGE, bar, stream_policy);
+    } else if (lane < 16) bulk_g2s_stream(dst + KPAGE + lane * ROWB, vc + off + (long long)lane * p.st, ROWB, bar, stream_policy);
     else bulk_g2s_stream(dst + (lane - 16) * ROWB, kc + off + (long long)(lane - 16) * p.st, ROWB, bar, stream_policy);
   };
   load_ids(0);
@@ -297,7 +312,7 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     const int tok0 = (wglob + k * wtot) << 4;
     if (tok0 + 16 > n) {                       // last page: rows beyond n may hold anything; clear their V
       for (int r = n - tok0; r < 16; ++r)
-        for (int c = lane; c < ROWB / 4; c += 32) reinterpret_cast<unsigned*>(stg + KPAGE + r * VROWB)[c] = 0u;
+        for (int c = lane; c < ROWB / 4; c += 32) reinterpret_cast<unsigned*>(stg + KPAGE + r * ROWB)[c] = 0u;
       __syncwarp();
     }
     // S^T for tokens 0..7 (sa) and 8..15 (sb): only c[0], c[1] (head gr) are meaningful
@@ -330,19 +345,25 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     l_run = l_run * alpha + psum;
     m_run = m_new;
     const unsigned pa0 = pack_bf16x2(pr[0], pr[1]), pa2 = pack_bf16x2(pr[2], pr[3]);
-    // out += P V, 16 dims per ldmatrix.x4.trans (two 8-dim column blocks)
-    const int mj = lane >> 3, mr = lane & 7;   // matrix and row this lane addresses
-    const unsigned char* vrow = stg + KPAGE + ((mj & 1) * 8 + mr) * VROWB + (mj >> 1) * 16;
+    // out += P V: this thread's tokens 2t, 2t+1 (k slots of pa0) and 8+2t, 9+2t (pa2), 8 dims at a time
+    const unsigned char* vrow = stg + KPAGE + (2 * t) * ROWB + gr * 16;
 #pragma unroll
-    for (int nb = 0; nb < NB; nb += 2) {
-      unsigned vb[4];
-      ldmatrix_x4_trans(vb, vrow + nb * 16);
-      float c0[4] = {acc[nb][0] * alpha, acc[nb][1] * alpha, 0.f, 0.f};
-      float c1[4] = {acc[nb + 1][0] * alpha, acc[nb + 1][1] * alpha, 0.f, 0.f};
-      mma_bf16_16816(c0, pa0, 0u, pa2, 0u, vb[0], vb[1]);
-      mma_bf16_16816(c1, pa0, 0u, pa2, 0u, vb[2], vb[3]);
-      acc[nb][0] = c0[0]; acc[nb][1] = c0[1];
-      acc[nb + 1][0] = c1[0]; acc[nb + 1][1] = c1[1];
+    for (int hf = 0; hf < NH; ++hf) {
+      const uint4 v0 = *reinterpret_cast<const uint4*>(vrow + hf * 128);
+      const uint4 v1 = *reinterpret_cast<const uint4*>(vrow + ROWB + hf * 128);
+      const uint4 v2 = *reinterpret_cast<const uint4*>(vrow + 8 * ROWB + hf * 128);
+      const uint4 v3 = *reinterpret_cast<const uint4*>(vrow + 9 * ROWB + hf * 128);
+      const unsigned w0[4] = {v0.x, v0.y, v0.z, v0.w}, w1[4] = {v1.x, v1.y, v1.z, v1.w};
+      const unsigned w2[4] = {v2.x, v2.y, v2.z, v2.w}, w3[4] = {v3.x, v3.y, v3.z, v3.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const unsigned sel = (e & 1) ? 0x7632u : 0x5410u;
+        const unsigned b0 = prmt(w0[e >> 1], w1[e >> 1], sel), b1 = prmt(w2[e >> 1], w3[e >> 1], sel);
+        const int nb = hf * 8 + e;
+        float c0[4] = {acc[nb][0] * alpha, acc[nb][1] * alpha, 0.f, 0.f};
+        mma_bf16_16816(c0, pa0, 0u, pa2, 0u, b0, b1);
+        acc[nb][0] = c0[0]; acc[nb][1] = c0[1];
+      }
     }
     __syncwarp();
     if (k + DN_NST < mine) {
@@ -357,44 +378,64 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
   l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
   __syncthreads();                             // every warp is done with its ring: reuse it for the partials
+  // accumulator (block 8 hf + e, columns 2t and 2t+1) is dim 64 hf + 8 (2t) + e and 64 hf + 8 (2t+1) + e
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
-    s_acc[(warp * 8 + gr) * D + nb * 8 + 2 * t] = acc[nb][0];
-    s_acc[(warp * 8 + gr) * D + nb * 8 + 2 * t + 1] = acc[nb][1];
+    s_acc[(warp * 8 + gr) * D + (nb >> 3) * 64 + 16 * t + (nb & 7)] = acc[nb][0];
+    s_acc[(warp * 8 + gr) * D + (nb >> 3) * 64 + 16 * t + 8 + (nb & 7)] = acc[nb][1];
   }
   if (t == 0) { s_m[warp][gr] = m_run; s_l[warp][gr] = l_run; }
   __syncthreads();
-  // CTA partial -> global: [D] unnormalised sum, m, l per head
-  for (int idx = tid; idx < 8 * NE; idx += DN_WARPS * 32) {
-    const int hh = idx / NE, e = idx % NE;
-    if (hh >= nh) continue;
+  // CTA partial -> global: [D] unnormalised sums, then m and l, per head; warps in a fixed order
+  __shared__ float s_w[DN_WARPS][8];           // weight of warp w's partial inside the CTA's
+  if (tid < 8) {
     float mc = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < DN_WARPS; ++w) mc = fmaxf(mc, s_m[w][hh]);
-    float val;
-    if (e == D) val = mc;
-    else {
-      val = 0.f;
+    for (int w = 0; w < DN_WARPS; ++w) mc = fmaxf(mc, s_m[w][tid]);
+    float lc = 0.f;
 #pragma unroll
-      for (int w = 0; w < DN_WARPS; ++w) {
-        const float sc = (s_m[w][hh] == -INFINITY) ? 0.f : __expf(s_m[w][hh] - mc);
-        val += sc * (e < D ? s_acc[(w * 8 + hh) * D + e] : s_l[w][hh]);
-      }
+    for (int w = 0; w < DN_WARPS; ++w) {
+      const float sc = (s_m[w][tid] == -INFINITY) ? 0.f : __expf(s_m[w][tid] - mc);
+      s_w[w][tid] = sc;
+      lc += sc * s_l[w][tid];
     }
-    p.dense_part[(((long long)b * p.Hq + h0 + hh) * S + split) * NE + e] = val;
+    if (tid < nh)
+      *reinterpret_cast<float4*>(p.dense_part + (((long long)b * p.Hq + h0 + tid) * SG + split) * NE + D) = make_float4(mc, lc, 0.f, 0.f);
   }
-  __threadfence();
   __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.tickets[2 * p.B * p.Hq + b * p.Hq + blockIdx.y], 1u) == (unsigned)(S - 1));
+  for (int idx = tid; idx < nh * (D / 4); idx += DN_WARPS * 32) {
+    const int hh = idx / (D / 4), e = (idx % (D / 4)) * 4;
+    float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < DN_WARPS; ++w) {
+      const float sc = s_w[w][hh];
+      const float4 x = *reinterpret_cast<const float4*>(&s_acc[(w * 8 + hh) * D + e]);
+      val.x += sc * x.x; val.y += sc * x.y; val.z += sc * x.z; val.w += sc * x.w;
+    }
+    *reinterpret_cast<float4*>(p.dense_part + (((long long)b * p.Hq + h0 + hh) * SG + split) * NE + e) = val;
+  }
+  // release: the barrier orders every thread's stores before thread 0's fence (cumulative), which orders
+  // them before the ticket; acquire: the ticket, a fence, and the barrier before anyone reads the partials
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    unsigned* ticket = &p.tickets[2 * p.B * p.Hq + b * p.Hq + blockIdx.y];
+    is_last = (atomicAdd(ticket, 1u) == (unsigned)(S - 1));
+    if (is_last) *ticket = 0u;                 // every CTA of the group has drawn: ready for the next call
+    __threadfence();
+  }
   __syncthreads();
   if (!is_last) return;
-  __threadfence();
-  // last CTA of the group: split maxima and sums first (shared memory), then every output element adds
-  // its S partials with the loads of 8 splits in flight at a time, in split order
+  // last CTA of the group.  Two rounds of loads: every split's (m, l) pair; then, per four output
+  // elements, the S partials with up to MB of them in flight, added in split order
+  constexpr int MB = 20;
   __shared__ float g_m[8][128], g_sc[8][128], g_den[8];
   for (int idx = tid; idx < 8 * S; idx += DN_WARPS * 32) {
     const int hh = idx / S, sp = idx % S;
-    if (hh < nh) g_m[hh][sp] = __ldcg(p.dense_part + (((long long)b * p.Hq + h0 + hh) * S + sp) * NE + D);
+    if (hh < nh) {
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.dense_part + (((long long)b * p.Hq + h0 + hh) * SG + sp) * NE + D));
+      g_m[hh][sp] = ml.x; g_sc[hh][sp] = ml.y;
+    }
   }
   __syncthreads();
   for (int hh = warp; hh < nh; hh += DN_WARPS) {
@@ -405,12 +446,12 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     float den = 0.f;
     for (int sp0 = 0; sp0 < S; sp0 += 32) {          // fixed order: chunks of 32 splits, lanes in a shuffle tree
       const int sp = sp0 + lane;
-      float scv = 0.f, lv = 0.f;
+      float lv = 0.f;
       if (sp < S) {
         const float ms = g_m[hh][sp];
-        scv = (ms == -INFINITY) ? 0.f : __expf(ms - mg);
+        const float scv = (ms == -INFINITY) ? 0.f : __expf(ms - mg);
+        lv = scv * g_sc[hh][sp];
         g_sc[hh][sp] = scv;
-        lv = scv * __ldcg(p.dense_part + (((long long)b * p.Hq + h0 + hh) * S + sp) * NE + D + 1);
       }
 #pragma unroll
       for (int mk = 16; mk >= 1; mk >>= 1) lv += __shfl_xor_sync(0xFFFFFFFFu, lv, mk);
@@ -419,26 +460,34 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     if (lane == 0) g_den[hh] = den;
   }
   __syncthreads();
-  for (int idx = tid; idx < 8 * D; idx += DN_WARPS * 32) {
-    const int hh = idx / D, e = idx % D;
-    if (hh >= nh) continue;
+  for (int idx = tid; idx < nh * (D / 4); idx += DN_WARPS * 32) {
+    const int hh = idx / (D / 4), e = (idx % (D / 4)) * 4;
     const long long bh = (long long)b * p.Hq + h0 + hh;
-    const float* base = p.dense_part + bh * S * NE + e;
-    float num = 0.f;
-    for (int sp0 = 0; sp0 < S; sp0 += 8) {
-      float v[8];
+    const float* base = p.dense_part + bh * SG * NE + e;
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp0 = 0; sp0 < S; sp0 += MB) {
+      float4 v[MB];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = (sp0 + u < S) ? __ldcg(base + (long long)(sp0 + u) * NE) : 0.f;
+      for (int u = 0; u < MB; ++u)
+        v[u] = (sp0 + u < S) ? __ldcg(reinterpret_cast<const float4*>(base + (long long)(sp0 + u) * NE)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) num += (sp0 + u < S) ? g_sc[hh][sp0 + u] * v[u] : 0.f;
+      for (int u = 0; u < MB; ++u) {
+        const float scv = (sp0 + u < S) ? g_sc[hh][sp0 + u] : 0.f;
+        num.x += scv * v[u].x; num.y += scv * v[u].y; num.z += scv * v[u].z; num.w += scv * v[u].w;
+      }
     }
-    reinterpret_cast<bf16_t*>(p.out)[bh * D + e] = Elem<bf16_t>::from_float(n > 0 ? num / g_den[hh] : 0.f);
+    const float den = g_den[hh];
+    bf16_t* o = reinterpret_cast<bf16_t*>(p.out) + bh * D + e;
+    o[0] = Elem<bf16_t>::from_float(n > 0 ? num.x / den : 0.f);
+    o[1] = Elem<bf16_t>::from_float(n > 0 ? num.y / den : 0.f);
+    o[2] = Elem<bf16_t>::from_float(n > 0 ? num.z / den : 0.f);
+    o[3] = Elem<bf16_t>::from_float(n > 0 ? num.w / den : 0.f);
   }
 }
 
 template <int D>
 static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
-  constexpr int STAGE = 16 * D * 2 + 16 * (D * 2 + 16);
+  constexpr int STAGE = 2 * 16 * D * 2;
   const size_t ring = (size_t)DN_WARPS * DN_NST * STAGE;
   const size_t accb = (size_t)DN_WARPS * 8 * D * sizeof(float);
   const size_t smem = (ring > accb ? ring : accb) + DN_WARPS * DN_NST * 8;
@@ -447,7 +496,11 @@ static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const int GC = (p.G + 7) / 8;
   const int groups = p.B * p.Hkv * GC;
-  int S = (2 * device_sm_count() + groups - 1) / groups;               // one wave of two CTAs per SM (registers and shared memory)
+  // Two CTAs fit an SM (registers and shared memory).  With few groups: as many splits as fill one wave, rounded
+  // down (a second, partly filled wave costs a whole CTA's duration).  With many groups (large batches, whose
+  // lengths differ): pieces small enough for four to five waves, so the SMs drain evenly.
+  const int slots = 2 * device_sm_count();
+  int S = slots / groups >= 3 ? slots / groups : (9 * slots / 2 + groups - 1) / groups;
   if (S > p.dense_splits) S = p.dense_splits;
   if (S < 1) S = 1;
   dim3 grid(S, p.Hkv * GC, p.B), block(DN_WARPS * 32);
@@ -457,14 +510,17 @@ static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
 }  // namespace
 
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches) {
-  const int GC = (p.G + 3) / 4;
-  dim3 grid(p.dense_splits, p.Hkv * GC, p.B), block(NT);
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (launches) *launches = 1;
     return p.D == 128 ? launch_dense_mma<128>(p, s) : launch_dense_mma<64>(p, s);
   } else {
-    if (p.D == 128) k_dense<float, 128><<<grid, block, 0, s>>>(p);
-    else k_dense<float, 64><<<grid, block, 0, s>>>(p);
+    const int GC = (p.G + 3) / 4;
+    const int groups = p.B * p.Hkv * GC;
+    Prob pf = p;                                 // about four CTAs per SM
+    pf.dense_splits = min(p.dense_splits, max(1, (4 * device_sm_count() + groups - 1) / groups));
+    dim3 grid(pf.dense_splits, p.Hkv * GC, p.B), block(NT);
+    if (p.D == 128) k_dense<float, 128><<<grid, block, 0, s>>>(pf);
+    else k_dense<float, 64><<<grid, block, 0, s>>>(pf);
   }
   if (launches) *launches = 1;
   return cudaGetLastError();
@@ -529,8 +585,8 @@ extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale,
   const size_t head_bytes = 256 + up256(3 * BH * sizeof(unsigned));
   int splits = (int)((4 * (size_t)device_sm_count() + groups - 1) / groups);
   splits = splits < 1 ? 1 : (splits > 128 ? 128 : splits);
-  while (splits > 1 && head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES) --splits;
-  if (head_bytes + BH * splits * (D + 2) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES)
+  while (splits > 1 && head_bytes + BH * splits * dense_rec((int)D) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES) --splits;
+  if (head_bytes + BH * splits * dense_rec((int)D) * sizeof(float) > VATTN_NOALLOC_SCRATCH_BYTES)
     return VATTN_ERR_WORKSPACE;     // batch * heads too large for the built-in scratch
 
   void* base = nullptr;

@@ -40,6 +40,10 @@ struct HeadMeta {
 };
 
 // Everything a kernel needs, passed by value.
+// floats in one split partial of the dense kernel: D unnormalised sums, the split's maximum, its sum of
+// weights, and two floats of padding (records stay 16-byte aligned)
+__host__ __device__ constexpr int dense_rec(int D) { return D + 4; }
+
 struct Prob {
   int B, Hq, Hkv, G, D, dtype;
   int max_blocks, num_blocks, max_seq_len, npad, nwords;   // npad: max_seq_len rounded up to 32; nwords = npad/32
@@ -87,7 +91,7 @@ struct Prob {
   float* gat_part;        // [B,Hq,gat_slots,D+1]  partials of the gather kernel, one per chunk
   int gat_slots;          // partial slots (chunks) per head: 32; 64 to 128 when at most 18 heads share the grid
   int stat_splits, stat_splits_base;   // statistics CTAs per head: deterministic rows, base-sample rows
-  float* dense_part;      // [B,Hq,dense_splits,D+2]
+  float* dense_part;      // [B,Hq,dense_splits,dense_rec(D)]
   int dense_splits;
   vattn_debug dbg;
 };

@@ -185,6 +185,36 @@ def test_dense_kernel_matches_dense_sdpa():
         tol = 2e-2 if dtype == "bf16" else 2e-5
         assert (np.abs(got - ref) <= tol * np.maximum(1.0, np.abs(ref))).all(), (dtype, d, np.abs(got - ref).max())
         assert plan.last_launch_count() == 1
+        # the kernel leaves its counters ready for the next call: the same again, and after a sparse step
+        out2 = torch.empty_like(out)
+        plan.dense_decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], out2)
+        torch.cuda.synchronize()
+        assert torch.equal(out2.view(torch.int16 if dtype == "bf16" else torch.int32),
+                           out.view(torch.int16 if dtype == "bf16" else torch.int32))
+        plan.decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], case.sink,
+                    case.window, case.k, case.eps, case.delta, case.seed, out2)
+        plan.dense_decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], out2)
+        torch.cuda.synchronize()
+        assert torch.equal(out2.view(torch.int16 if dtype == "bf16" else torch.int32),
+                           out.view(torch.int16 if dtype == "bf16" else torch.int32))
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 8), (8, 1), (12, 1), (6, 2)])
+def test_dense_kernel_group_sizes_and_mixed_lengths(Hq, Hkv):
+    """Query-head groups of 1, 3, 8 and 12 heads (a group larger than the 8 rows of a tile takes two CTAs), and
+    lengths from one page to the longest the cache holds: sequences get splits in proportion to their length."""
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [16, 5000, 333, 4097, 1, 2500], Hq=Hq, Hkv=Hkv)
+    dev = vb.case_to_device(case)
+    plan = vb.plan_for_case(case)
+    out = torch.empty_like(dev["q"])
+    plan.dense_decode(dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], out)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    ref = O.dense_decode(case.q, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype="bf16")
+    assert (np.abs(got - ref) <= 2e-2 * np.maximum(1.0, np.abs(ref))).all(), np.abs(got - ref).max()
+    assert plan.last_status() == 0
 
 
 def test_host_buffer_entry_point_matches_device_entry_point():
