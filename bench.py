@@ -249,6 +249,8 @@ def main():
                          "reasoning-length) and add them to the JSON line as `other_configs`")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
+    ap.add_argument("--profile-dense", action="store_true",
+                    help="with --profile-only: every step is followed by the dense comparison kernel on the same inputs")
     ap.add_argument("--profile-config", default="cfg2", choices=["cfg2", "cfg5", "cfg4"],
                     help="with --profile-only: the workload to run (cfg5: batch 8 at n=32768; cfg4: batch 32, mixed "
                          "lengths; one cache pool each, 1.1 GB and 2.6 GB)")
@@ -310,6 +312,8 @@ def main():
         if args.profile_only:
             for i in range(max(1, args.steps)):
                 step(i)
+                if args.profile_dense:
+                    step(i, dense=True)
             stream.synchronize()
             if rank == 0:
                 print(json.dumps({"profile_only": True, "steps": args.steps, "launches_per_step": plan.last_launch_count()}))
