@@ -55,6 +55,19 @@ typedef struct {
   int32_t max_blocks_per_seq, num_blocks, max_seq_len;    /* max_seq_len <= max_blocks_per_seq * block_size */
   int32_t dtype;                                          /* VATTN_DTYPE_*: element type of q, k_cache, v_cache, out */
   int64_t kv_stride_block, kv_stride_head, kv_stride_token; /* elements; all zero = contiguous HND */
+  int32_t q_len;                                          /* query tokens per sequence in one call; 0 or 1 = one (plain
+                                                             decoding).  With q_len = T > 1 (a question, or speculative
+                                                             tokens: the split-prompt setup of App. C, where everything
+                                                             after the context runs through sparse attention) q and out
+                                                             are [batch, T, num_q_heads, head_dim], the cache already
+                                                             holds the T tokens' K and V rows, seq_lens counts them, and
+                                                             query token t attends to the first seq_len - (T - 1 - t)
+                                                             tokens (causal).  Every (token, head) pair is treated as a
+                                                             head of its own -- own index sets, statistics, budget and
+                                                             samples, drawn as decode step `step + t` -- and the pairs
+                                                             that share a KV head share one pass over its K rows.
+                                                             T * num_q_heads / num_kv_heads <= 64.  Introspection arrays
+                                                             then have the head axis [KV head, t, head within the group] */
 } vattn_shape;
 
 /* Everything Algorithm 1/2 need beyond the short argument list of vattn_decode.  Zero = default. */

@@ -423,3 +423,44 @@ def dense_decode(q, k_cache, v_cache, block_table, seq_lens, *, dtype, scale=Non
             for h in range(g * G, (g + 1) * G):
                 out[b, h] = dense_sdpa(to_f64(q[b, h], dtype), K, V, scale)
     return out
+
+
+# ----------------------------------------------------------------------------- several query tokens per call
+def _visible_lens(seq_lens, Tq, t):
+    """Tokens that query token t of Tq sees: the cache already holds all Tq new rows, attention is causal."""
+    return np.maximum(np.asarray(seq_lens, np.int64) - (Tq - 1 - t), 0)
+
+
+def vattn_decode_multi(q, k_cache, v_cache, block_table, seq_lens, sink, window, k, eps, delta, seed, *,
+                       dtype, step=0, heads=None, **params):
+    """A call that carries Tq query tokens per sequence (a question, speculative tokens: the split-prompt
+    setup of App. C, where everything after the context goes through sparse attention).
+
+    q [B,Tq,Hq,d].  Query token t attends to the first n - (Tq - 1 - t) tokens and is, in every other
+    respect, the decode step `step + t` of Algorithm 1 on that prefix: own index sets, statistics, budget
+    and samples per (token, head).  `heads` optionally restricts the work to (b, t, h) triples.
+    Returns (out [B,Tq,Hq,d] in the storage type, details keyed (b, t, h))."""
+    B, Tq, Hq, d = q.shape
+    out = np.zeros((B, Tq, Hq, d), np.uint16 if dtype == "bf16" else np.float32)
+    details = {}
+    for t in range(Tq):
+        sel = None if heads is None else [(b, h) for (b, tt, h) in heads if tt == t]
+        if sel is not None and not sel:
+            continue
+        o, det = vattn_decode(np.ascontiguousarray(q[:, t]), k_cache, v_cache, block_table,
+                              _visible_lens(seq_lens, Tq, t), sink, window, k, eps, delta, seed, dtype=dtype,
+                              step=step + t, heads=sel, **params)
+        out[:, t] = o
+        for (b, h), r in det.items():
+            details[(b, t, h)] = r
+    return out, details
+
+
+def dense_decode_multi(q, k_cache, v_cache, block_table, seq_lens, *, dtype, scale=None):
+    """Causal dense SDPA for Tq query tokens per sequence, fp64: q [B,Tq,Hq,d] -> [B,Tq,Hq,d]."""
+    B, Tq, Hq, d = q.shape
+    out = np.zeros((B, Tq, Hq, d))
+    for t in range(Tq):
+        out[:, t] = dense_decode(np.ascontiguousarray(q[:, t]), k_cache, v_cache, block_table,
+                                 _visible_lens(seq_lens, Tq, t), dtype=dtype, scale=scale)
+    return out

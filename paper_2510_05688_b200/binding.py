@@ -32,7 +32,8 @@ class Shape(C.Structure):
     _fields_ = [("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("block_size", C.c_int32), ("max_blocks_per_seq", C.c_int32),
                 ("num_blocks", C.c_int32), ("max_seq_len", C.c_int32), ("dtype", C.c_int32),
-                ("kv_stride_block", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64)]
+                ("kv_stride_block", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_stride_token", C.c_int64),
+                ("q_len", C.c_int32)]
 
 
 class Params(C.Structure):
@@ -125,9 +126,9 @@ class Plan:
     """Owner of one vattn_plan plus the torch tensors backing its workspace and debug buffers."""
 
     def __init__(self, *, batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq, num_blocks, max_seq_len,
-                 dtype, block_size=16, kv_strides=(0, 0, 0), device="cuda", alloc_workspace=True):
+                 dtype, block_size=16, kv_strides=(0, 0, 0), q_len=1, device="cuda", alloc_workspace=True):
         self.shape = Shape(batch, num_q_heads, num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks,
-                           max_seq_len, dtype, *kv_strides)
+                           max_seq_len, dtype, *kv_strides, q_len)
         h = C.c_void_p()
         _check(lib().vattn_plan_create(C.byref(self.shape), C.byref(h)), "vattn_plan_create")
         self._h = h
@@ -169,7 +170,8 @@ class Plan:
         """Allocate device buffers for every introspection output and register them."""
         import torch
         s = self.shape
-        BH, cap = (s.batch, s.num_q_heads), s.max_seq_len
+        # with q_len > 1 the head axis is [KV head, query token, head within the group] flattened
+        BH, cap = (s.batch, s.num_q_heads * max(1, s.q_len)), s.max_seq_len
         dev = self.device
         i32 = torch.int32
         self.debug = dict(
@@ -299,8 +301,8 @@ def case_to_device(case, device="cuda"):
                 seq_lens=torch.from_numpy(case.seq_lens).to(device))
 
 
-def plan_for_case(case, device="cuda", max_seq_len=None) -> Plan:
+def plan_for_case(case, device="cuda", max_seq_len=None, q_len=1) -> Plan:
     msl = int(max_seq_len if max_seq_len is not None else case.max_blocks_per_seq * 16)
     return Plan(batch=case.batch, num_q_heads=case.num_q_heads, num_kv_heads=case.num_kv_heads,
                 head_dim=case.head_dim, max_blocks_per_seq=case.max_blocks_per_seq, num_blocks=case.num_blocks,
-                max_seq_len=msl, dtype=DTYPE_BF16 if case.dtype == "bf16" else DTYPE_FP32, device=device)
+                max_seq_len=msl, dtype=DTYPE_BF16 if case.dtype == "bf16" else DTYPE_FP32, q_len=q_len, device=device)

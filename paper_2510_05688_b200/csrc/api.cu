@@ -71,13 +71,17 @@ double upper_quantile(double t) {
   return flip ? -z : z;
 }
 
+// (query token, head) pairs per batch row: the kernels treat each as a head of its own
+inline int q_tokens(const vattn_shape& s) { return s.q_len > 1 ? s.q_len : 1; }
+inline int heads_v(const vattn_shape& s) { return s.num_q_heads * q_tokens(s); }
+
 void derive(vattn_plan* pl) {
   const vattn_shape& s = pl->shape;
-  pl->G = s.num_q_heads / s.num_kv_heads;
+  pl->G = heads_v(s) / s.num_kv_heads;
   pl->npad = (s.max_seq_len + 31) / 32 * 32;
   if (pl->npad == 0) pl->npad = 32;
   pl->nwords = pl->npad / 32;
-  const int heads = s.batch * s.num_q_heads;
+  const int heads = s.batch * heads_v(s);
   const int GC = (pl->G + 3) / 4;
   const int groups = s.batch * s.num_kv_heads * GC;
   const int sp = (8 * device_sm_count() + groups - 1) / groups;
@@ -136,7 +140,8 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   const vattn_shape& s = pl->shape;
   const vattn_params& pr = pl->params;
   memset(&p, 0, sizeof(p));
-  p.B = s.batch; p.Hq = s.num_q_heads; p.Hkv = s.num_kv_heads; p.G = pl->G; p.D = s.head_dim; p.dtype = s.dtype;
+  p.B = s.batch; p.Hq = heads_v(s); p.Hkv = s.num_kv_heads; p.G = pl->G; p.D = s.head_dim; p.dtype = s.dtype;
+  p.Tq = q_tokens(s); p.G1 = s.num_q_heads / s.num_kv_heads;
   p.max_blocks = s.max_blocks_per_seq; p.num_blocks = s.num_blocks; p.max_seq_len = s.max_seq_len;
   p.npad = pl->npad; p.nwords = pl->nwords;
   if (s.kv_stride_block == 0 && s.kv_stride_head == 0 && s.kv_stride_token == 0) {
@@ -155,7 +160,7 @@ int fill_prob(const vattn_plan* pl, Prob& p, const void* q, const void* kc, cons
   unsigned char* w = static_cast<unsigned char*>(pl->ws);
   p.scores = reinterpret_cast<float*>(w + pl->off_scores);
   unsigned* z = reinterpret_cast<unsigned*>(w + pl->off_zero);
-  const size_t BH = (size_t)s.batch * s.num_q_heads;
+  const size_t BH = (size_t)s.batch * heads_v(s);
   p.m_ord = z; p.kabsmax = z + BH; p.tickets = z + BH + (size_t)s.batch * s.num_kv_heads;
   p.unit_ctr = p.tickets + 5 * BH;
   p.flags64 = reinterpret_cast<unsigned long long*>(w + pl->off_zero + pl->zero_bytes - BH * 8);
@@ -236,18 +241,19 @@ int vattn_plan_create(const vattn_shape* shape, vattn_plan** out) {
   if (!shape || !out) return VATTN_ERR_INVALID_ARG;
   const vattn_shape& s = *shape;
   if (s.batch <= 0 || s.num_q_heads <= 0 || s.num_kv_heads <= 0 || s.max_blocks_per_seq <= 0 || s.num_blocks <= 0 ||
-      s.max_seq_len < 0)
+      s.max_seq_len < 0 || s.q_len < 0)
     return VATTN_ERR_INVALID_ARG;
   if (s.num_q_heads % s.num_kv_heads != 0) return VATTN_ERR_INVALID_ARG;
   if (s.batch > 65535 || s.num_q_heads > 65535) return VATTN_ERR_INVALID_ARG;
   // grid dimensions y and z hold (batch row, head) pairs and twice the batch
-  if (s.batch > 32767 || (long long)s.batch * s.num_q_heads > 65535) return VATTN_ERR_UNSUPPORTED;
+  if (s.q_len > 64) return VATTN_ERR_UNSUPPORTED;
+  if (s.batch > 32767 || (long long)s.batch * heads_v(s) > 65535) return VATTN_ERR_UNSUPPORTED;
   // the bf16 score kernel keeps two per-row tables of the batch in shared memory beside its page ring
   if (s.dtype == VATTN_DTYPE_BF16 && s.batch > VATTN_MAX_BATCH_BF16) return VATTN_ERR_UNSUPPORTED;
   if (s.head_dim != 64 && s.head_dim != 128) return VATTN_ERR_UNSUPPORTED;
   if (s.block_size != VATTN_BLOCK) return VATTN_ERR_UNSUPPORTED;
   if (s.dtype != VATTN_DTYPE_FP32 && s.dtype != VATTN_DTYPE_BF16) return VATTN_ERR_UNSUPPORTED;
-  if (s.num_q_heads / s.num_kv_heads > 64) return VATTN_ERR_UNSUPPORTED;
+  if (heads_v(s) / s.num_kv_heads > 64) return VATTN_ERR_UNSUPPORTED;
   if (s.max_seq_len > VATTN_MAX_SEQ) return VATTN_ERR_UNSUPPORTED;
   if ((long long)s.max_seq_len > (long long)s.max_blocks_per_seq * s.block_size) return VATTN_ERR_INVALID_ARG;
   const bool custom = s.kv_stride_block || s.kv_stride_head || s.kv_stride_token;
@@ -428,7 +434,7 @@ size_t vattn_host_staging_bytes(const vattn_plan* plan) {
   if (!plan) return 0;
   const vattn_shape& s = plan->shape;
   const size_t es = s.dtype == VATTN_DTYPE_BF16 ? 2 : 4;
-  const size_t qb = align_up((size_t)s.batch * s.num_q_heads * s.head_dim * es, 256);
+  const size_t qb = align_up((size_t)s.batch * heads_v(s) * s.head_dim * es, 256);
   return 2 * qb + align_up((size_t)s.batch * s.max_blocks_per_seq * 4, 256) + align_up((size_t)s.batch * 4, 256);
 }
 
@@ -450,7 +456,7 @@ static int enqueue_host_step(vattn_plan* plan, const void* q_host, const void* k
                              const vattn_plan::HostStep* mapped) {
   const vattn_shape& s = plan->shape;
   const size_t es = s.dtype == VATTN_DTYPE_BF16 ? 2 : 4;
-  const size_t qbytes = (size_t)s.batch * s.num_q_heads * s.head_dim * es, qb = align_up(qbytes, 256);
+  const size_t qbytes = (size_t)s.batch * heads_v(s) * s.head_dim * es, qb = align_up(qbytes, 256);
   const size_t btbytes = (size_t)s.batch * s.max_blocks_per_seq * 4, slbytes = (size_t)s.batch * 4;
   unsigned char* d = static_cast<unsigned char*>(staging);
   void* dq = d; void* dout = d + qb; int32_t* dbt = reinterpret_cast<int32_t*>(d + 2 * qb);

@@ -33,11 +33,17 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
 #pragma unroll
   for (int hh = 0; hh < 4; ++hh) {
     const int hl = hc * 4 + hh;
-    if (hl < p.G) Elem<T>::load(reinterpret_cast<const T*>(p.q) + ((long long)b * p.Hq + g * p.G + hl) * D + j * EPL, qv[hh]);
+    if (hl < p.G) Elem<T>::load(reinterpret_cast<const T*>(p.q) + q_row(p, b, g * p.G + hl) + j * EPL, qv[hh]);
     else {
 #pragma unroll
       for (int e = 0; e < EPL; ++e) qv[hh][e] = 0.f;
     }
+  }
+  int nh2[2];                                  // tokens that this lane's two heads see (query tokens of one call differ)
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int hl = hc * 4 + 2 * (j & 1) + e;
+    nh2[e] = hl < p.G ? head_len(p, b, g * p.G + hl) : n;
   }
   float m_run[4], l_lane[2] = {0.f, 0.f}, acc[4][EPL];
 #pragma unroll
@@ -80,10 +86,10 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
       width = half;
     }
     // lane (r, j): token (j>>1)*RPI + r, heads 2(j&1)+{0,1}
-    const bool tok_ok = (tok0 + (j >> 1) * RPI + r) < n;
+    const int tok_l = tok0 + (j >> 1) * RPI + r;
     float sv[2], pm[2];
 #pragma unroll
-    for (int e = 0; e < 2; ++e) { sv[e] = tok_ok ? p.scale * sacc[e] : -INFINITY; pm[e] = sv[e]; }
+    for (int e = 0; e < 2; ++e) { sv[e] = tok_l < nh2[e] ? p.scale * sacc[e] : -INFINITY; pm[e] = sv[e]; }
 #pragma unroll
     for (int mask = 2; mask < 32; mask <<= 1) {
       pm[0] = fmaxf(pm[0], __shfl_xor_sync(0xFFFFFFFFu, pm[0], mask));
@@ -106,7 +112,7 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
     float pv[2];
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      pv[e] = __expf(sv[e] - m_new[2 * (j & 1) + e]);
+      pv[e] = sv[e] == -INFINITY ? 0.f : __expf(sv[e] - m_new[2 * (j & 1) + e]);
       l_lane[e] += pv[e];
     }
 #pragma unroll
@@ -194,7 +200,7 @@ __global__ void __launch_bounds__(NT) k_dense(const Prob p) {
       num += sc * __ldcg(base + sp * NE + e);
       den += sc * __ldcg(base + sp * NE + D + 1);
     }
-    reinterpret_cast<T*>(p.out)[bh * D + e] = Elem<T>::from_float(n > 0 ? num / den : 0.f);
+    reinterpret_cast<T*>(p.out)[q_row(p, b, g * p.G + hl) + e] = Elem<T>::from_float(den > 0.f ? num / den : 0.f);
   }
 }
 
@@ -296,9 +302,9 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   for (int c = 0; c < NC; ++c) {
     aq[c] = make_uint4(0u, 0u, 0u, 0u);
     if (gr < nh)
-      aq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
-                                              ((long long)b * p.Hq + h0 + gr) * D + c * 32 + t * 8);
+      aq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) + q_row(p, b, h0 + gr) + c * 32 + t * 8);
   }
+  const int n_h = gr < nh ? head_len(p, b, h0 + gr) : n;   // tokens that head gr sees (query tokens of one call differ)
   float m_run = -INFINITY, l_run = 0.f;        // head gr of this thread's row; l is this lane's share
   float acc[NB][2];
 #pragma unroll
@@ -332,16 +338,16 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     float mx = -INFINITY;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      sc[e] = (tk[e] < n) ? p.scale * sc[e] : -INFINITY;
+      sc[e] = (tk[e] < n_h) ? p.scale * sc[e] : -INFINITY;
       mx = fmaxf(mx, sc[e]);
     }
     mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-    const float m_new = fmaxf(m_run, mx);      // a page has at least one valid token, so m_new is finite
+    const float m_new = fmaxf(m_run, mx);      // (-inf while the head has seen none of its tokens)
     const float alpha = (m_run == -INFINITY) ? 0.f : __expf(m_run - m_new);
     float pr[4], psum = 0.f;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { pr[e] = __expf(sc[e] - m_new); psum += pr[e]; }
+    for (int e = 0; e < 4; ++e) { pr[e] = sc[e] == -INFINITY ? 0.f : __expf(sc[e] - m_new); psum += pr[e]; }
     l_run = l_run * alpha + psum;
     m_run = m_new;
     const unsigned pa0 = pack_bf16x2(pr[0], pr[1]), pa2 = pack_bf16x2(pr[2], pr[3]);
@@ -476,12 +482,12 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
         num.x += scv * v[u].x; num.y += scv * v[u].y; num.z += scv * v[u].z; num.w += scv * v[u].w;
       }
     }
-    const float den = g_den[hh];
-    bf16_t* o = reinterpret_cast<bf16_t*>(p.out) + bh * D + e;
-    o[0] = Elem<bf16_t>::from_float(n > 0 ? num.x / den : 0.f);
-    o[1] = Elem<bf16_t>::from_float(n > 0 ? num.y / den : 0.f);
-    o[2] = Elem<bf16_t>::from_float(n > 0 ? num.z / den : 0.f);
-    o[3] = Elem<bf16_t>::from_float(n > 0 ? num.w / den : 0.f);
+    const float den = g_den[hh];                  // zero: the head sees no token
+    bf16_t* o = reinterpret_cast<bf16_t*>(p.out) + q_row(p, b, h0 + hh) + e;
+    o[0] = Elem<bf16_t>::from_float(den > 0.f ? num.x / den : 0.f);
+    o[1] = Elem<bf16_t>::from_float(den > 0.f ? num.y / den : 0.f);
+    o[2] = Elem<bf16_t>::from_float(den > 0.f ? num.z / den : 0.f);
+    o[3] = Elem<bf16_t>::from_float(den > 0.f ? num.w / den : 0.f);
   }
 }
 
@@ -570,7 +576,7 @@ extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale,
       s.max_seq_len < 0 || s.num_q_heads % s.num_kv_heads != 0 || s.batch > 65535 || s.num_q_heads > 65535)
     return VATTN_ERR_INVALID_ARG;
   if ((s.head_dim != 64 && s.head_dim != 128) || s.block_size != VATTN_BLOCK ||
-      (s.dtype != VATTN_DTYPE_FP32 && s.dtype != VATTN_DTYPE_BF16) || s.num_q_heads / s.num_kv_heads > 64)
+      (s.dtype != VATTN_DTYPE_FP32 && s.dtype != VATTN_DTYPE_BF16) || s.num_q_heads / s.num_kv_heads > 64 || s.q_len > 1)
     return VATTN_ERR_UNSUPPORTED;
   if ((long long)s.max_seq_len > (long long)s.max_blocks_per_seq * s.block_size) return VATTN_ERR_INVALID_ARG;
   const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_cache) |
@@ -597,6 +603,7 @@ extern "C" int vattn_dense_decode_noalloc(const vattn_shape* shape, float scale,
   Prob p;
   memset(&p, 0, sizeof(p));
   p.B = s.batch; p.Hq = s.num_q_heads; p.Hkv = s.num_kv_heads; p.G = G; p.D = s.head_dim; p.dtype = s.dtype;
+  p.Tq = 1; p.G1 = G;
   p.max_blocks = s.max_blocks_per_seq; p.num_blocks = s.num_blocks; p.max_seq_len = s.max_seq_len;
   if (s.kv_stride_block == 0 && s.kv_stride_head == 0 && s.kv_stride_token == 0) {
     p.st = s.head_dim; p.sh = (long long)s.block_size * s.head_dim; p.sb = (long long)s.num_kv_heads * p.sh;

@@ -74,7 +74,7 @@ struct Gather {
                              float (*part)[NE], int* is_last, float* s_den) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = bh % p.Hq, g = h / p.G;
-    T* out = reinterpret_cast<T*>(p.out) + (long long)bh * D;
+    T* out = reinterpret_cast<T*>(p.out) + q_row(p, bh / p.Hq, h);
     if (meta.n == 0) {
       if (slot == 0) for (int e = tid; e < D; e += NT) out[e] = Elem<T>::from_float(0.f);
       return;
@@ -140,7 +140,7 @@ struct Gather {
     // scores for the whole context behind would need); the K slices of a batch come first, then its V slices
     float qf[EPL];
     const T* kcg = reinterpret_cast<const T*>(p.kc) + (long long)g * p.sh;
-    if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+    if (KV) Elem<T>::load(reinterpret_cast<const T*>(p.q) + q_row(p, bh / p.Hq, h) + j * EPL, qf);
     auto batch = [&](int k0, auto full_tag) {
       constexpr bool FULL = decltype(full_tag)::value;
       // lane u of a row group owns row u's weight: one score load and one exp per row instead of LPR

@@ -160,7 +160,13 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
             unsigned char* dst = ring + (size_t)stage * PAGEB;
             const bf16_t* src = kc + (long long)pid * p.sb + (long long)g * p.sh;
             mbar_expect_tx(&full[stage], PAGEB + (with_q ? qbytes : 0u));
-            if (with_q) bulk_g2s(qring + (size_t)stage * qslot_bytes, qsrc, qbytes, &full[stage]);
+            if (with_q) {
+              if (p.Tq == 1) bulk_g2s(qring + (size_t)stage * qslot_bytes, qsrc, qbytes, &full[stage]);
+              else                                    // the rows of different query tokens are apart in memory
+                for (int rr = 0; rr < nh; ++rr)
+                  bulk_g2s(qring + (size_t)stage * qslot_bytes + rr * ROWB,
+                           reinterpret_cast<const bf16_t*>(p.q) + q_row(p, b, h0 + rr), ROWB, &full[stage]);
+            }
             if (p.st == D) bulk_g2s_stream(dst, src, PAGEB, &full[stage], kpolicy);
             else
               for (int rr = 0; rr < VATTN_BLOCK; ++rr) bulk_g2s_stream(dst + rr * ROWB, src + (long long)rr * p.st, ROWB, &full[stage], kpolicy);
@@ -215,6 +221,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
   float runmax[2] = {-INFINITY, -INFINITY};
   unsigned kabs = 0u;
   int cur_unit = -1, cur_bh0 = 0, cur_nh = 0;       // cur_unit holds nh_unit of the unit in progress
+  int hide[2] = {0, 0};                               // tokens at the end of the sequence that this thread's heads do not see
   auto flush = [&]() {                                // running maxima of the unit just finished
     if (cur_unit < 0) return;
 #pragma unroll
@@ -254,6 +261,10 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     if (m.nh_unit != cur_unit) {
       flush();
       cur_unit = m.nh_unit; cur_bh0 = m.bh0; cur_nh = m_nh;
+      if (p.Tq > 1) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) hide[e] = p.Tq - 1 - head_tok(p, (m.bh0 + 2 * t + e) % p.Hq);
+      }
       const unsigned char* qs = qring + (size_t)stage * qslot_bytes;
 #pragma unroll
       for (int c = 0; c < NC; ++c)
@@ -287,8 +298,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
       if (hl < m_nh) {
         float* dst = p.scores + (long long)(m.bh0 + hl) * p.npad;
         const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
-        if (tk_lo < m.n) { dst[tk_lo] = s_lo; runmax[e] = fmaxf(runmax[e], s_lo); }
-        if (tk_hi < m.n) { dst[tk_hi] = s_hi; runmax[e] = fmaxf(runmax[e], s_hi); }
+        if (tk_lo < m.n) { dst[tk_lo] = s_lo; if (tk_lo < m.n - hide[e]) runmax[e] = fmaxf(runmax[e], s_lo); }
+        if (tk_hi < m.n) { dst[tk_hi] = s_hi; if (tk_hi < m.n - hide[e]) runmax[e] = fmaxf(runmax[e], s_hi); }
       }
     }
   }
@@ -319,7 +330,7 @@ __global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
   for (int hh = 0; hh < 4; ++hh) {
     const int hl = hc * 4 + hh;
     if (hl < p.G) {
-      Elem<T>::load(reinterpret_cast<const T*>(p.q) + ((long long)b * p.Hq + g * p.G + hl) * D + j * EPL, qv[hh]);
+      Elem<T>::load(reinterpret_cast<const T*>(p.q) + q_row(p, b, g * p.G + hl) + j * EPL, qv[hh]);
     } else {
 #pragma unroll
       for (int e = 0; e < EPL; ++e) qv[hh][e] = 0.f;
@@ -374,7 +385,7 @@ __global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
       const float sc = p.scale * acc[e];
       if (tok < n && hl < p.G) {
         p.scores[((long long)b * p.Hq + g * p.G + hl) * p.npad + tok] = sc;
-        runmax[e] = fmaxf(runmax[e], sc);
+        if (p.Tq == 1 || tok < n - (p.Tq - 1 - head_tok(p, g * p.G + hl))) runmax[e] = fmaxf(runmax[e], sc);
       }
     }
   }

@@ -273,11 +273,11 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
   TICK_BEGIN(p, VATTN_K_SELECT);
 
   // ------------------------------------------------------------------ before the wait: the step's inputs only
-  const int n = clamped_len(p, b);
+  const int n = head_len(p, b, h);
   const Geo geo = head_geometry(p, n);
   const int s0 = geo.s0, l_start = geo.l_start, kk = geo.kk, n_s = geo.n_s, b0 = geo.b0;
   const int mlen = l_start - s0;
-  const T* qrow = reinterpret_cast<const T*>(p.q) + (long long)bh * D;
+  const T* qrow = reinterpret_cast<const T*>(p.q) + q_row(p, b, h);
   const float* sc = p.scores + (long long)bh * p.npad;
   int* tk = p.topk_idx + (long long)bh * 2 * p.npad;
   unsigned* gbitmap = p.bitmap + (long long)bh * p.nwords;
@@ -300,9 +300,8 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     }
     return;
   }
-  const int hrng = p.rng_head_is_kv ? g : h;
   for (int i = tid; i < 5 * HBINS; i += NT) sm.hist[i] = 0;
-  if (tid < 4) walk_keys(p, b, hrng, tid >> 1, tid & 1, sm.rkeys + (tid >> 1) * 8);
+  if (tid < 4) walk_keys(p, b, h, tid >> 1, tid & 1, sm.rkeys + (tid >> 1) * 8);
   double sa = 0.0;                                     // sum |q_e| (warp 0), for the rounding bound of the scores
   if (warp == 0) {
     for (int e = lane; e < D; e += 32) sa += fabs((double)Elem<T>::to_float(qrow[e]));
@@ -896,8 +895,8 @@ __global__ void __launch_bounds__(256) k_walk(const Prob p) {
   pdl_trigger();
   TICK_BEGIN(p, VATTN_K_WALK);
   const int tid = threadIdx.x, bh = blockIdx.y;
-  const int b = bh / p.Hq, h = bh % p.Hq, g = h / p.G;
-  const int n = clamped_len(p, b);
+  const int b = bh / p.Hq, h = bh % p.Hq;
+  const int n = head_len(p, b, h);
   const Geo geo = head_geometry(p, n);
   const int mlen = geo.l_start - geo.s0;
   const int J0 = walk_region(geo.b0, geo.n_s, mlen, geo.kk);
@@ -909,8 +908,7 @@ __global__ void __launch_bounds__(256) k_walk(const Prob p) {
   // positions to do and goes on to its next one as soon as one is finished (one pass per loop iteration).
   constexpr int PER = 1024;
   if (geo.n_s > 0 && (int)blockIdx.x * PER < J0 + J1) {
-    const int hrng = p.rng_head_is_kv ? g : h;
-    if (tid < 4) walk_keys(p, b, hrng, tid >> 1, tid & 1, keys + (tid >> 1) * 8);
+    if (tid < 4) walk_keys(p, b, h, tid >> 1, tid & 1, keys + (tid >> 1) * 8);
     __syncthreads();
     int* out0 = p.walk_tok + (long long)bh * 4 * p.npad;       // [walk][tokens, physical slots][npad]
 #pragma unroll 1

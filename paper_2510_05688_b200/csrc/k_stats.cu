@@ -301,7 +301,7 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
   // ---- I_dyn as a list: budgets beyond the walk array (unusual: saturated budgets), and for the debug buffer
   if (bfin > mt.dyn_listed || (p.dbg.dyn_idx && bfin > 0)) {
     __shared__ unsigned rkeys[8];
-    if (tid < 2) walk_keys(p, b, p.rng_head_is_kv ? h / p.G : h, 1, tid, rkeys);
+    if (tid < 2) walk_keys(p, b, h, 1, tid, rkeys);
     __syncthreads();
     const int s0 = mt.s0, l_start = mt.l_start;
     const int* vt = p.vtab + (long long)bh * VATTN_BANDCAP;
@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
                                           : (unsigned long long)wait_word32(fl32, VATTN_WORD_SPINS);
     s_word = v;
   }
-  const int n = clamped_len(p, b);
+  const int n = head_len(p, b, h);
   const Geo geo = head_geometry(p, n);
   const int s0 = geo.s0, l_start = geo.l_start, kk = geo.kk, b0 = geo.b0;
   const float m_f = unord_f32(__ldcg(p.m_ord + bh));
@@ -438,7 +438,7 @@ __global__ void __launch_bounds__(NT, 5) k_stats(const __grid_constant__ Prob p)
   __shared__ double qT[D];
   if (warp == 0 && rsub == 0) {
     float qf[EPL];
-    Elem<T>::load(reinterpret_cast<const T*>(p.q) + (long long)bh * D + j * EPL, qf);
+    Elem<T>::load(reinterpret_cast<const T*>(p.q) + q_row(p, b, h) + j * EPL, qf);
 #pragma unroll
     for (int e = 0; e < EPL; ++e) qT[e * LPR + j] = (double)qf[e];
   }

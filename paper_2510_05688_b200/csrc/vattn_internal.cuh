@@ -45,7 +45,8 @@ struct HeadMeta {
 __host__ __device__ constexpr int dense_rec(int D) { return D + 4; }
 
 struct Prob {
-  int B, Hq, Hkv, G, D, dtype;
+  int B, Hq, Hkv, G, D, dtype;   // Hq, G count (query token, head) pairs when a call carries several query tokens
+  int Tq, G1;                    // query tokens per sequence (>= 1) and real query heads per KV head (G = Tq * G1)
   int max_blocks, num_blocks, max_seq_len, npad, nwords;   // npad: max_seq_len rounded up to 32; nwords = npad/32
   long long sb, sh, st;                                      // KV strides in elements
   const void* q; const void* kc; const void* vc; const int* bt; const int* seq_lens; void* out;
@@ -205,6 +206,24 @@ __device__ __forceinline__ int clamped_len(const Prob& p, int b) {
   return n;
 }
 
+// Calls with several query tokens per sequence (a question, speculative tokens).  The cache already holds their
+// K and V rows; query token t of Tq sees the first n - (Tq - 1 - t) tokens (causal).  Inside the kernels every
+// (query token, head) pair is a head of its own: head index hv = g * G + t * G1 + i stands for query token t and
+// real head g * G1 + i, so the heads that share KV head g stay contiguous (one pass over K serves all of them).
+// q and out are [B, Tq, Hkv * G1, D] in memory.
+__device__ __forceinline__ int head_tok(const Prob& p, int hv) { return (hv % p.G) / p.G1; }
+__device__ __forceinline__ int head_real(const Prob& p, int hv) { return (hv / p.G) * p.G1 + (hv % p.G1); }
+// element offset of head hv's row in q and out
+__device__ __forceinline__ long long q_row(const Prob& p, int b, int hv) {
+  if (p.Tq == 1) return ((long long)b * p.Hq + hv) * p.D;
+  return (((long long)b * p.Tq + head_tok(p, hv)) * (p.Hkv * p.G1) + head_real(p, hv)) * p.D;
+}
+// tokens that head hv of batch row b sees
+__device__ __forceinline__ int head_len(const Prob& p, int b, int hv) {
+  const int n = clamped_len(p, b);
+  return p.Tq == 1 ? n : max(0, n - (p.Tq - 1 - head_tok(p, hv)));
+}
+
 // Index-set geometry of one sequence (Algorithm 1 lines 1-5 with absolute sink/window counts):
 // sink range [0,s0), window [l_start,n), middle M = [s0,l_start), kk = |I_t|, n_s = |M| - kk, b0.
 struct Geo { int s0, l_start, kk, n_s, b0; };
@@ -305,10 +324,13 @@ __device__ __forceinline__ int dyn_listed_want(const Prob& p, int n_s, int b0) {
   if (n_s <= 0) return 0;
   return min(n_s, p.force_budget >= 0 ? p.force_budget : VATTN_WALK_B0S * b0);
 }
-// round keys of one (batch row, head, stream) into keys[0..8): two threads, one Philox call each
-__device__ __forceinline__ void walk_keys(const Prob& p, int b, int hrng, int stream, int half, unsigned* keys) {
+// round keys of one (batch row, head, stream) into keys[0..8): two threads, one Philox call each.  The head word is
+// the real query head (or the KV head with rng_head_is_kv); query token t of a call draws as decode step `step + t`
+__device__ __forceinline__ void walk_keys(const Prob& p, int b, int hv, int stream, int half, unsigned* keys) {
+  const int hrng = p.rng_head_is_kv ? hv / p.G : head_real(p, hv);
+  const unsigned step = (unsigned)p.step + (unsigned)head_tok(p, hv);
   const uint4 w4 = philox4x32_10((unsigned)half, ((unsigned)b << 16) | (unsigned)hrng, (unsigned)p.layer,
-                                 ((unsigned)p.step << 1) | (unsigned)stream, p.seed_lo, p.seed_hi);
+                                 (step << 1) | (unsigned)stream, p.seed_lo, p.seed_hi);
   keys[half * 4 + 0] = w4.x; keys[half * 4 + 1] = w4.y; keys[half * 4 + 2] = w4.z; keys[half * 4 + 3] = w4.w;
 }
 // is middle token `tok` (fp32 score s) a member of I_t?  vt: the head's near-tie list (shared or global memory)

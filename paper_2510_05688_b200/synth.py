@@ -168,6 +168,23 @@ C1_CALIBRATED = 9.85   # heavy-hitter strength giving ~10x sparsity on the Llama
                        # oracle's mean density: 0.0999 at this value)
 
 
+def multi_query(case: Case, q_len: int, noise=0.35, gen_seed=9009) -> np.ndarray:
+    """Query rows for a call that carries `q_len` query tokens per sequence: [B, q_len, Hq, d] in the case's
+    storage type.  The last token's rows are the case's own q; earlier tokens are the same rows plus Gaussian
+    noise of `noise` times their standard deviation, so every token keeps the case's attention structure
+    (heavy hitters, near-uniform heads) without repeating its scores."""
+    rng = np.random.default_rng(gen_seed)
+    base = case.values(case.q).astype(np.float32)                  # [B,Hq,d]
+    rows = []
+    for t in range(q_len):
+        if t == q_len - 1:
+            rows.append(base)
+        else:
+            sd = base.std(axis=-1, keepdims=True)
+            rows.append((base + noise * sd * rng.standard_normal(base.shape).astype(np.float32)).astype(np.float32))
+    return np.ascontiguousarray(np.stack([_store(r, case.dtype) for r in rows], axis=1))
+
+
 def config1_tiny(gen_seed=1001, **over) -> Case:
     """Tiny decode: 1 head, d=64, n=1024, fp32, 8 planted heavy hitters of strength 4."""
     kw = dict(dtype="fp32", B=1, Hq=1, Hkv=1, d=64, seq_lens=[1024], sink=4, window=32, k=32,

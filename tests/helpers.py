@@ -39,6 +39,59 @@ def run_gpu(case, debug=True, plan=None, dev=None, **over):
     return out_np, dbg_np, plan
 
 
+def virtual_head(case, q_len, t, h):
+    """Index of (query token t, head h) on the head axis of the introspection arrays of a q_len > 1 plan:
+    [KV head, query token, head within the group] flattened."""
+    G1 = case.num_q_heads // case.num_kv_heads
+    return (h // G1) * (q_len * G1) + t * G1 + (h % G1)
+
+
+def run_oracle_multi(case, q4, heads=None, **over):
+    p = dict(case.params)
+    p.update(over)
+    p.pop("gather_mode", None)
+    return O.vattn_decode_multi(q4, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink, case.window,
+                                case.k, case.eps, case.delta, case.seed, dtype=case.dtype, heads=heads, **p)
+
+
+def run_gpu_multi(case, q4, debug=True, **over):
+    """One call with q4 [B,Tq,Hq,d] through the C ABI.  Returns (out [B,Tq,Hq,d] numpy, debug dict, plan)."""
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    p = dict(case.params)
+    p.update(over)
+    Tq = q4.shape[1]
+    dev = vb.case_to_device(case)
+    if case.dtype == "bf16":
+        qd = torch.from_numpy(np.ascontiguousarray(q4).view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        qd = torch.from_numpy(np.ascontiguousarray(q4)).cuda()
+    plan = vb.plan_for_case(case, q_len=Tq)
+    plan.set_params(**p)
+    dbg = plan.enable_debug() if debug else None
+    out = torch.empty_like(qd)
+    plan.decode(qd, dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], case.sink, case.window,
+                case.k, case.eps, case.delta, case.seed, out)
+    torch.cuda.synchronize()
+    out_np = out.view(torch.int16).cpu().numpy().view(np.uint16) if case.dtype == "bf16" else out.cpu().numpy()
+    dbg_np = {k: v.cpu().numpy() for k, v in dbg.items()} if dbg else None
+    return out_np, dbg_np, plan, dict(dev, q=qd)
+
+
+def assert_parity_multi(case, q_len, out, dbg, det, out_ref, check_scores=True):
+    """assert_parity with (b, t, h) mapped onto the plan's head axis."""
+    B, Hq, d = case.batch, case.num_q_heads, case.head_dim
+    det_v = {(b, virtual_head(case, q_len, t, h)): r for (b, t, h), r in det.items()}
+    out_v = np.zeros((B, q_len * Hq, d), out.dtype)
+    ref_v = np.zeros((B, q_len * Hq, d), out_ref.dtype)
+    for t in range(q_len):
+        for h in range(Hq):
+            hv = virtual_head(case, q_len, t, h)
+            out_v[:, hv] = out[:, t, h]
+            ref_v[:, hv] = out_ref[:, t, h]
+    assert_parity(case, out_v, dbg, det_v, ref_v, check_scores=check_scores)
+
+
 def out_values(case, out):
     if case.dtype == "bf16":
         return (np.asarray(out, np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)

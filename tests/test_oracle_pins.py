@@ -474,3 +474,64 @@ def test_p6_sampler_uniform_over_subsets():
     chi2 = sum((v - exp) ** 2 / exp for v in subsets.values())
     assert len(subsets) == 56 and chi2 < 105.0            # 55 dof: P(chi2 > 105) ~ 5e-5
     assert np.abs(incl[R] / T - c / len(R)).max() < 0.012
+
+
+# ----------------------------------------------------------------------------- several query tokens per call
+def test_multi_query_full_budget_equals_causal_sdpa():
+    """With the whole residual as budget every query token of a call must give causal dense attention: token t
+    of Tq sees the first n - (Tq - 1 - t) rows.  The reference is torch's SDPA over all Tq rows at once with an
+    explicit mask built here, on independently de-paged K and V."""
+    case = small_case("bf16", seq_lens=(70, 33, 2))
+    Tq = 3
+    q4 = synth.multi_query(case, Tq)
+    scale = float(np.float32(1.0 / math.sqrt(case.head_dim)))
+    out, det = O.vattn_decode_multi(q4, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink,
+                                    case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype,
+                                    force_budget=10**9)
+    dense = O.dense_decode_multi(q4, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=case.dtype)
+    G = case.num_q_heads // case.num_kv_heads
+    qv = case.values(q4).astype(np.float64)
+    for b in range(case.batch):
+        n = int(case.seq_lens[b])
+        mask = torch.zeros(Tq, n, dtype=torch.bool)
+        for t in range(Tq):
+            mask[t, :max(0, n - (Tq - 1 - t))] = True
+        for h in range(case.num_q_heads):
+            K = torch.from_numpy(depage_loop(case, case.k_cache, b, h // G))
+            V = torch.from_numpy(depage_loop(case, case.v_cache, b, h // G))
+            Q = torch.from_numpy(qv[b, :, h])
+            ref = torch.nn.functional.scaled_dot_product_attention(Q[None, None], K[None, None], V[None, None],
+                                                                   attn_mask=mask[None, None], scale=scale)[0, 0].numpy()
+            for t in range(Tq):
+                r = det[(b, t, h)]
+                if r["n"] == 0:                              # a query token that sees nothing: zeros by convention
+                    assert not r["out"].any() and not dense[b, t, h].any()
+                    continue
+                assert r["n"] == n - (Tq - 1 - t) and r["b"] == r["n_s"]
+                np.testing.assert_allclose(r["out"], ref[t], rtol=1e-12, atol=1e-13)
+                np.testing.assert_allclose(dense[b, t, h], ref[t], rtol=1e-12, atol=1e-13)
+
+
+def test_multi_query_tokens_are_consecutive_decode_steps():
+    """Query token t of a call is decode step `step + t` on its prefix: the same index sets, budget and output
+    as a single-query call with that step word and that length; one query token is the single-query call."""
+    case = small_case("fp32", seq_lens=(90, 41))
+    Tq = 2
+    q4 = synth.multi_query(case, Tq)
+    _, det = O.vattn_decode_multi(q4, case.k_cache, case.v_cache, case.block_table, case.seq_lens, case.sink,
+                                  case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype, step=5)
+    for t in range(Tq):
+        lens = np.asarray(case.seq_lens) - (Tq - 1 - t)
+        _, one = O.vattn_decode(np.ascontiguousarray(q4[:, t]), case.k_cache, case.v_cache, case.block_table, lens,
+                                case.sink, case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype,
+                                step=5 + t)
+        for (b, h), r in one.items():
+            m = det[(b, t, h)]
+            assert np.array_equal(m["I_dyn"], r["I_dyn"]) and np.array_equal(m["I_bs"], r["I_bs"])
+            assert m["budgets"] == r["budgets"] and np.array_equal(m["out"], r["out"])
+    # samples of consecutive tokens differ (their step words do)
+    assert any(not np.array_equal(det[(0, 0, h)]["I_bs"], det[(0, 1, h)]["I_bs"]) for h in range(case.num_q_heads))
+    out1, det1 = O.vattn_decode_multi(case.q[:, None], case.k_cache, case.v_cache, case.block_table, case.seq_lens,
+                                      case.sink, case.window, case.k, case.eps, case.delta, case.seed, dtype=case.dtype)
+    out0, det0 = run_oracle(case)
+    assert np.array_equal(out1[:, 0], out0)
