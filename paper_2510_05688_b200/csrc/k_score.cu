@@ -36,7 +36,7 @@ struct __align__(16) StageMeta {   // written by the producer before it arms the
   int tok0;             // first token of the page; < 0: no more work for the consumer that owns this stage
   int n;                // tokens of the sequence
   int bh0;              // batch row * Hq + first query head of the group slice
-  int nh_unit;          // query heads in the slice (<= 8) | running unit number of the CTA << 4: a change of
+  int nh_unit;          // query heads in the slice (<= 16) | running unit number of the CTA << 5: a change of
 };                      // the unit tells the consumer to flush its maxima and reload q
 
 // Clears the per-step counters (running maxima, tickets, list lengths, unit counter).  A kernel rather than a
@@ -57,7 +57,9 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-template <int D>
+// WIDE: slices of up to 16 heads (groups of more than 8 heads: calls with several query tokens, or many query heads
+// per KV head); otherwise the second half of the slice and its registers are compiled out
+template <int D, bool WIDE>
 __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p, int qslot_bytes) {
   constexpr int NC = D / 32;
   constexpr int ROWB = D * 2;                 // bytes per row
@@ -76,7 +78,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
   TICK_BEGIN(p, VATTN_K_SCORE);
 
   // ---- units: every CTA derives the same decomposition from the sequence lengths
-  const int GC = (p.G + 7) >> 3;
+  constexpr int SL = WIDE ? 16 : 8;                   // heads per slice: one pass over K serves a slice
+  const int GC = (p.G + SL - 1) / SL;
   const int GPB = p.Hkv * GC;                         // (KV head, head slice) groups per batch row
   int my_pages = 0;
   for (int b = tid; b < p.B; b += SCORE_THREADS) {
@@ -136,7 +139,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
       const int r = u - s_pref[b];
       const int gc = r / chunks, chunk = r % chunks;
       const int g = gc / GC, hc = gc % GC;
-      const int h0 = g * p.G + hc * 8, nh = min(8, p.G - hc * 8);
+      const int h0 = g * p.G + hc * SL, nh = min(SL, p.G - hc * SL);
       const int pA = chunk * CH, cnt = min(CH, np - pA);
       const bf16_t* qsrc = reinterpret_cast<const bf16_t*>(p.q) + ((long long)b * p.Hq + h0) * D;
       // S lanes arm S stages at a time, each lane its own: wait for the stage to be handed back, describe the
@@ -153,17 +156,18 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
           if (ok) {
             const int k = k0 + lane;
             StageMeta m;
-            m.tok0 = (pA + k) << 4; m.n = n; m.bh0 = b * p.Hq + h0; m.nh_unit = nh | (ucount << 4);
+            m.tok0 = (pA + k) << 4; m.n = n; m.bh0 = b * p.Hq + h0; m.nh_unit = nh | (ucount << 5);
             meta[stage] = m;
             const bool with_q = k < CWN;              // every consumer meets q on its first page of the unit
-            const unsigned qbytes = (unsigned)(nh * ROWB);
+            const int nq = min(nh, 8);                // the first 8 heads' rows ride with the page; the others are read by the consumers
+            const unsigned qbytes = (unsigned)(nq * ROWB);
             unsigned char* dst = ring + (size_t)stage * PAGEB;
             const bf16_t* src = kc + (long long)pid * p.sb + (long long)g * p.sh;
             mbar_expect_tx(&full[stage], PAGEB + (with_q ? qbytes : 0u));
             if (with_q) {
               if (p.Tq == 1) bulk_g2s(qring + (size_t)stage * qslot_bytes, qsrc, qbytes, &full[stage]);
               else                                    // the rows of different query tokens are apart in memory
-                for (int rr = 0; rr < nh; ++rr)
+                for (int rr = 0; rr < nq; ++rr)
                   bulk_g2s(qring + (size_t)stage * qslot_bytes + rr * ROWB,
                            reinterpret_cast<const bf16_t*>(p.q) + q_row(p, b, h0 + rr), ROWB, &full[stage]);
             }
@@ -215,26 +219,26 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
 
   // ================================================================= consumer warps
   const int gr = lane >> 2, t = lane & 3;
-  uint4 bq[NC];
+  uint4 bq[NC], bq2[NC];                            // q fragments of heads 0..7 and 8..15 of the slice
 #pragma unroll
-  for (int c = 0; c < NC; ++c) bq[c] = make_uint4(0u, 0u, 0u, 0u);
-  float runmax[2] = {-INFINITY, -INFINITY};
+  for (int c = 0; c < NC; ++c) { bq[c] = make_uint4(0u, 0u, 0u, 0u); bq2[c] = make_uint4(0u, 0u, 0u, 0u); }
+  float runmax[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // heads 2t, 2t+1, 8+2t, 9+2t
   unsigned kabs = 0u;
   int cur_unit = -1, cur_bh0 = 0, cur_nh = 0;       // cur_unit holds nh_unit of the unit in progress
-  int hide[2] = {0, 0};                               // tokens at the end of the sequence that this thread's heads do not see
+  unsigned hide = 0u;                                 // tokens at the end of the sequence that this thread's heads do not see, a byte per head
   auto flush = [&]() {                                // running maxima of the unit just finished
     if (cur_unit < 0) return;
 #pragma unroll
     for (int mask = 4; mask < 32; mask <<= 1) {
-      runmax[0] = fmaxf(runmax[0], __shfl_xor_sync(0xFFFFFFFFu, runmax[0], mask));
-      runmax[1] = fmaxf(runmax[1], __shfl_xor_sync(0xFFFFFFFFu, runmax[1], mask));
+#pragma unroll
+      for (int e = 0; e < (WIDE ? 4 : 2); ++e) runmax[e] = fmaxf(runmax[e], __shfl_xor_sync(0xFFFFFFFFu, runmax[e], mask));
     }
 #pragma unroll
     for (int mask = 1; mask < 32; mask <<= 1) kabs = __vimax3_u16x2(kabs, __shfl_xor_sync(0xFFFFFFFFu, kabs, mask), 0u);
     if (lane < 4) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int hl = 2 * lane + e;
+      for (int e = 0; e < (WIDE ? 4 : 2); ++e) {
+        const int hl = (e >> 1) * 8 + 2 * lane + (e & 1);
         if (hl < cur_nh && runmax[e] > -INFINITY) atomicMax(&p.m_ord[cur_bh0 + hl], ord_f32(runmax[e]));
       }
     }
@@ -243,7 +247,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
       const int b = cur_bh0 / p.Hq, g = (cur_bh0 % p.Hq) / p.G;
       atomicMax(&p.kabsmax[b * p.Hkv + g], mx << 16);
     }
-    runmax[0] = runmax[1] = -INFINITY;
+    runmax[0] = runmax[1] = runmax[2] = runmax[3] = -INFINITY;
     kabs = 0u;
   };
 
@@ -257,13 +261,24 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     }
     const StageMeta m = meta[stage];
     if (m.tok0 < 0) break;
-    const int m_nh = m.nh_unit & 15;
+    const int m_nh = m.nh_unit & 31;
     if (m.nh_unit != cur_unit) {
       flush();
       cur_unit = m.nh_unit; cur_bh0 = m.bh0; cur_nh = m_nh;
       if (p.Tq > 1) {
 #pragma unroll
-        for (int e = 0; e < 2; ++e) hide[e] = p.Tq - 1 - head_tok(p, (m.bh0 + 2 * t + e) % p.Hq);
+        hide = 0u;
+#pragma unroll
+        for (int e = 0; e < (WIDE ? 4 : 2); ++e)
+          hide |= (unsigned)(p.Tq - 1 - head_tok(p, (m.bh0 + (e >> 1) * 8 + 2 * t + (e & 1)) % p.Hq)) << (8 * e);
+      }
+      if (WIDE && m_nh > 8) {                          // heads 8..15 of the slice: their rows come straight from q
+        const int bb = m.bh0 / p.Hq, hv0 = m.bh0 % p.Hq;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+          bq2[c] = (8 + gr < m_nh) ? __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) +
+                                                                         q_row(p, bb, hv0 + 8 + gr) + c * 32 + t * 8))
+                                   : make_uint4(0u, 0u, 0u, 0u);
       }
       const unsigned char* qs = qring + (size_t)stage * qslot_bytes;
 #pragma unroll
@@ -272,6 +287,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     }
     const unsigned char* stg = ring + (size_t)stage * PAGEB;
     float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};   // two independent MMA chains
+    float accB[4] = {0.f, 0.f, 0.f, 0.f}, accB1[4] = {0.f, 0.f, 0.f, 0.f}; // heads 8..15 of the slice, from the same page
+    const bool two = WIDE && m_nh > 8;                 // (uniform over the warp)
     unsigned klo = 0u, khi = 0u;
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
@@ -279,6 +296,10 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
       const uint4 ahi = *reinterpret_cast<const uint4*>(stg + (gr + 8) * ROWB + c * 64 + t * 16);
       mma_bf16_16816(acc, alo.x, ahi.x, alo.y, ahi.y, bq[c].x, bq[c].y);
       mma_bf16_16816(acc1, alo.z, ahi.z, alo.w, ahi.w, bq[c].z, bq[c].w);
+      if (two) {
+        mma_bf16_16816(accB, alo.x, ahi.x, alo.y, ahi.y, bq2[c].x, bq2[c].y);
+        mma_bf16_16816(accB1, alo.z, ahi.z, alo.w, ahi.w, bq2[c].z, bq2[c].w);
+      }
       klo = __vimax3_u16x2(klo, alo.x & 0x7FFF7FFFu, alo.y & 0x7FFF7FFFu);
       klo = __vimax3_u16x2(klo, alo.z & 0x7FFF7FFFu, alo.w & 0x7FFF7FFFu);
       khi = __vimax3_u16x2(khi, ahi.x & 0x7FFF7FFFu, ahi.y & 0x7FFF7FFFu);
@@ -288,18 +309,19 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score_stream(const Prob p,
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty[stage]);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) acc[e] += acc1[e];
+    for (int e = 0; e < 4; ++e) { acc[e] += acc1[e]; accB[e] += accB1[e]; }
     const int tk_lo = m.tok0 + gr, tk_hi = m.tok0 + gr + 8;
     if (tk_lo < m.n) kabs = __vimax3_u16x2(kabs, klo, 0u);
     if (tk_hi < m.n) kabs = __vimax3_u16x2(kabs, khi, 0u);
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int hl = 2 * t + e;
+    for (int e4 = 0; e4 < (WIDE ? 4 : 2); ++e4) {
+      const int e = e4 & 1, hl = (e4 >> 1) * 8 + 2 * t + e;
       if (hl < m_nh) {
         float* dst = p.scores + (long long)(m.bh0 + hl) * p.npad;
-        const float s_lo = p.scale * acc[e], s_hi = p.scale * acc[2 + e];
-        if (tk_lo < m.n) { dst[tk_lo] = s_lo; if (tk_lo < m.n - hide[e]) runmax[e] = fmaxf(runmax[e], s_lo); }
-        if (tk_hi < m.n) { dst[tk_hi] = s_hi; if (tk_hi < m.n - hide[e]) runmax[e] = fmaxf(runmax[e], s_hi); }
+        const float s_lo = p.scale * (e4 < 2 ? acc[e] : accB[e]), s_hi = p.scale * (e4 < 2 ? acc[2 + e] : accB[2 + e]);
+        const int seen = m.n - (int)((hide >> (8 * e4)) & 0xFFu);
+        if (tk_lo < m.n) { dst[tk_lo] = s_lo; if (tk_lo < seen) runmax[e4] = fmaxf(runmax[e4], s_lo); }
+        if (tk_hi < m.n) { dst[tk_hi] = s_hi; if (tk_hi < seen) runmax[e4] = fmaxf(runmax[e4], s_hi); }
       }
     }
   }
@@ -409,23 +431,23 @@ __global__ void __launch_bounds__(WARPS * 32) k_score_fma(const Prob p) {
 
 }  // namespace
 
-template <int D>
+template <int D, bool WIDE>
 static cudaError_t launch_stream(const Prob& p, cudaStream_t s) {
-  constexpr int S = 2048 / D, PAGEB = VATTN_BLOCK * D * 2;
+  constexpr int S = 2048 / D, PAGEB = VATTN_BLOCK * D * 2, SL = WIDE ? 16 : 8;
   const int nh_max = p.G < 8 ? p.G : 8;
   const int qslot_bytes = nh_max * D * 2;
   const size_t smem = (size_t)S * PAGEB + (size_t)S * qslot_bytes + (size_t)S * sizeof(StageMeta) + (size_t)2 * S * 8 +
                       sizeof(int) * ((size_t)2 * p.B + 1 + 16);
   if (smem > 113 * 1024) return cudaErrorInvalidValue;        // two CTAs per SM (plan creation bounds the batch)
   static size_t have[VATTN_MAXDEV];
-  cudaError_t e = optin_smem(k_score_stream<D>, smem, have, true);
+  cudaError_t e = optin_smem(k_score_stream<D, WIDE>, smem, have, true);
   if (e != cudaSuccess) return e;
   // persistent: two CTAs per SM, fewer when the problem cannot have that many units
   const long long pages = (p.max_seq_len + VATTN_BLOCK - 1) / VATTN_BLOCK;
-  const long long units_max = (long long)p.B * p.Hkv * ((p.G + 7) / 8) * ((pages + MIN_UNIT_PAGES - 1) / MIN_UNIT_PAGES);
+  const long long units_max = (long long)p.B * p.Hkv * ((p.G + SL - 1) / SL) * ((pages + MIN_UNIT_PAGES - 1) / MIN_UNIT_PAGES);
   const int slots = 2 * device_sm_count();
   const int grid = (int)(units_max < slots ? (units_max < 1 ? 1 : units_max) : slots);
-  return launch_pdl(k_score_stream<D>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
+  return launch_pdl(k_score_stream<D, WIDE>, dim3(grid), dim3(SCORE_THREADS), smem, s, p, qslot_bytes);
 }
 
 // `pdl`: launch with the programmatic-serialization attribute, i.e. let this grid start while the kernel before it
@@ -447,8 +469,8 @@ cudaError_t launch_score(const Prob& p, cudaStream_t s) {
   const int tiles = (p.max_seq_len + TILE - 1) / TILE;
   if (p.dtype == VATTN_DTYPE_BF16) {
     // rows must be 16-byte aligned for the bulk copies (any stride that is a multiple of 8 elements is)
-    if (p.D == 128) return launch_stream<128>(p, s);
-    return launch_stream<64>(p, s);
+    if (p.G > 8) return p.D == 128 ? launch_stream<128, true>(p, s) : launch_stream<64, true>(p, s);
+    return p.D == 128 ? launch_stream<128, false>(p, s) : launch_stream<64, false>(p, s);
   } else {
     dim3 grid(tiles, p.Hkv * ((p.G + 3) / 4), p.B);
     if (p.D == 128) k_score_fma<float, 128><<<grid, block, 0, s>>>(p);
