@@ -416,6 +416,42 @@ def main():
         plan.set_params(**case.params)
         del nst_graphs
 
+        # four query tokens per call (a question, speculative tokens): 128 (token, head) pairs share one pass over K
+        MQ = 4
+        q4 = torch.from_numpy(np.ascontiguousarray(synth.multi_query(case, MQ)).view(np.int16)).cuda().view(torch.bfloat16)
+        mq_plan = vb.plan_for_case(case, q_len=MQ)
+        mq_plan.set_params(**case.params)
+        mq_out = torch.empty_like(q4)
+
+        def mq_capture(dense):
+            graphs = []
+            for i in range(POOLS):
+                d = pools[i % npools]
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    if dense:
+                        mq_plan.dense_decode(q4, d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], mq_out,
+                                             stream=stream)
+                    else:
+                        mq_plan.decode(q4, d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], case.sink,
+                                       case.window, case.k, case.eps, case.delta, case.seed, mq_out, stream=stream)
+                graphs.append(g)
+            return graphs
+        for dense_ in (False, True):                       # first calls outside a capture (attributes, lazy loading)
+            d = pools[0]
+            if dense_:
+                mq_plan.dense_decode(q4, d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], mq_out, stream=stream)
+            else:
+                mq_plan.decode(q4, d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], case.sink, case.window,
+                               case.k, case.eps, case.delta, case.seed, mq_out, stream=stream)
+        stream.synchronize()
+        mq_graphs = mq_capture(False)
+        ms_mq, _, _ = timed(mq_graphs, min(args.steps, 500), args.warmup)
+        del mq_graphs
+        mq_graphs = mq_capture(True)
+        ms_mq_dense, _, _ = timed(mq_graphs, min(args.steps, 500), args.warmup)
+        del mq_graphs, mq_plan
+
         # optional external context: a third-party dense paged-decode kernel on the same cache
         fi_us = None
         if args.flashinfer:
@@ -587,6 +623,9 @@ def main():
                    "kv_gather_variant_us_per_step": round(ms_kv * 1e3, 2),
                    "kv_head_sampling_keys_variant_us_per_step": round(ms_grp * 1e3, 2),
                    "nested_base_variant_us_per_step": round(ms_nst * 1e3, 2),
+                   "four_query_tokens_per_call": {"sparse_us_per_call": round(ms_mq * 1e3, 2),
+                                                  "dense_us_per_call": round(ms_mq_dense * 1e3, 2),
+                                                  "sparse_us_per_token": round(ms_mq * 1e3 / 4, 2)},
                    "value_is": "max-over-ranks step time / n_gpus (each rank runs its own layer)"},
         "e2e": {"value": ms_e2e_max * 1e3 / world, "unit": UNIT,
                 "h2d_bytes_per_step": int(qh.numel() * 2 + bth.numel() * 4 + slh.numel() * 4),

@@ -9,6 +9,7 @@
  *
  * Tensor layouts
  *   q, out        [batch, num_q_heads, head_dim], contiguous, 16-byte aligned, element type `dtype`
+ *                 ([batch, q_len, num_q_heads, head_dim] for a plan with vattn_shape.q_len > 1)
  *   k_cache,
  *   v_cache       paged: element (block p, kv head g, token t, dim j) at
  *                 p*kv_stride_block + g*kv_stride_head + t*kv_stride_token + j   (element units);
@@ -119,9 +120,9 @@ typedef struct {
 } vattn_debug;
 
 /* Create / destroy a plan for one problem shape.  `out` receives a host object.  Errors: INVALID_ARG,
- * UNSUPPORTED (head_dim other than 64 / 128, block_size other than 16, more than 64 query heads per KV head,
- * max_seq_len above 262,144, a bf16 batch above 1,536 rows, a batch above 32,767 rows or more than 65,535
- * (batch row, query head) pairs: the kernels' grid dimensions). */
+ * UNSUPPORTED (head_dim other than 64 / 128, block_size other than 16, more than 64 (query token, query head)
+ * pairs per KV head, q_len above 64, max_seq_len above 262,144, a bf16 batch above 1,536 rows, a batch above
+ * 32,767 rows or more than 65,535 (batch row, query token, query head) triples: the kernels' grid dimensions). */
 int    vattn_plan_create(const vattn_shape* shape, vattn_plan** out);
 void   vattn_plan_destroy(vattn_plan* plan);
 
@@ -162,7 +163,9 @@ int vattn_decode(vattn_plan* plan, const void* q, const void* k_cache, const voi
                  void* out, void* stream /* cudaStream_t */);
 
 /* Dense attention over the same paged cache (full SDPA of Sec. 3), split over the context with a
- * fixed-order merge: the latency the sparse step is compared with.  Uses the plan's workspace. */
+ * fixed-order merge: the latency the sparse step is compared with.  Uses the plan's workspace (and relies on
+ * the words it leaves there between calls: hand the plan a workspace, then do not write to it).  With
+ * q_len > 1 the query tokens of a call are masked causally like vattn_decode's. */
 int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, const void* v_cache,
                        const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
 
@@ -174,9 +177,10 @@ int vattn_dense_decode(vattn_plan* plan, const void* q, const void* k_cache, con
  * device).  No plan is needed and nothing is allocated, on the host or on the device: the split
  * partials live in a fixed array of VATTN_NOALLOC_SCRATCH_BYTES that is part of the library image, so
  * every GPU that loads the library holds that much memory until the process exits.
- *   - `scale` 0 means 1/sqrt(head_dim).  Arguments and layouts are those of vattn_dense_decode.
+ *   - `scale` 0 means 1/sqrt(head_dim).  Arguments and layouts are those of vattn_dense_decode; one query token
+ *     per sequence only (q_len > 1: VATTN_ERR_UNSUPPORTED).
  *   - The problem must fit: 256 + 12*batch*num_q_heads (rounded up to 256) +
- *     batch*num_q_heads*(head_dim+2)*4 bytes <= VATTN_NOALLOC_SCRATCH_BYTES (about 8,000 (batch row, query
+ *     batch*num_q_heads*(head_dim+4)*4 bytes <= VATTN_NOALLOC_SCRATCH_BYTES (about 8,000 (batch row, query
  *     head) pairs at head_dim 128); larger problems return VATTN_ERR_WORKSPACE.  Fewer context splits are
  *     used when the usual number does not fit, so results can differ from vattn_dense_decode in the
  *     last bits.

@@ -605,6 +605,37 @@ def test_multi_query_variants():
         assert_parity_multi(case, 2, out, dbg, det, out_ref)
 
 
+def test_multi_query_host_buffer_entry_point():
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [900, 350])
+    q4 = synth.multi_query(case, 3)
+    out_dev, _, plan, dev = run_gpu_multi(case, q4, debug=False)
+    qh = dev["q"].cpu().pin_memory()
+    bth = dev["block_table"].cpu().pin_memory()
+    slh = dev["seq_lens"].cpu().pin_memory()
+    outh = torch.empty_like(qh).pin_memory()
+    for _ in range(3):                                   # the third call replays the recorded step
+        outh.zero_()
+        plan.decode_host(qh, dev["k_cache"], dev["v_cache"], bth, slh, case.sink, case.window, case.k, case.eps,
+                         case.delta, case.seed, outh)
+        assert np.array_equal(outh.view(torch.int16).numpy().view(np.uint16), out_dev)
+
+
+def test_multi_query_limits():
+    from paper_2510_05688_b200 import binding as vb
+    case = small("bf16", [64])                           # 4 heads per KV head: 16 tokens fill the 64 rows of a group
+    vb.plan_for_case(case, q_len=16)
+    with pytest.raises(vb.VattnError):
+        vb.plan_for_case(case, q_len=17)
+    shape = vb.plan_for_case(case, q_len=2).shape
+    import torch
+    dev = vb.case_to_device(case)
+    q = torch.zeros(1, 2, 8, 128, dtype=torch.bfloat16, device="cuda")
+    assert vb.dense_decode_noalloc(shape, q, dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"],
+                                   torch.empty_like(q)) == vb.ERR_UNSUPPORTED
+
+
 def test_multi_query_one_token_is_the_plain_call():
     case = small("bf16", [700, 129])
     out1, dbg1, _, _ = run_gpu_multi(case, np.ascontiguousarray(case.q[:, None]))
