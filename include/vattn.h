@@ -127,8 +127,9 @@ int    vattn_plan_create(const vattn_shape* shape, vattn_plan** out);
 void   vattn_plan_destroy(vattn_plan* plan);
 
 /* Bytes of device scratch a plan needs (a pure function of the shape), and handing it over.
- * The pointer must be 256-byte aligned and stay valid while the plan is used.  The library
- * zeroes what it needs on every call; the contents need not be initialised. */
+ * The pointer must be 256-byte aligned and stay valid while the plan is used.  The contents need not
+ * be initialised: the library clears what it needs (vattn_decode on every call, vattn_dense_decode on its
+ * first call after this one); between calls it expects to find the workspace as it left it. */
 size_t vattn_workspace_bytes(const vattn_plan* plan);
 int    vattn_set_workspace(vattn_plan* plan, void* dev_ptr, size_t bytes);
 
