@@ -232,8 +232,14 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // ro
   return r;
 }
 
-template <int D>
-__global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
+// WIDE: up to 16 heads per CTA (rows 8..15 of the tiles carry heads 8..15: groups of more than 8 heads, as calls
+// with several query tokens make them), one CTA per SM with four stages per warp; otherwise 8 heads, two CTAs per
+// SM, two stages
+template <int D, bool WIDE>
+__global__ void __launch_bounds__((WIDE ? 2 : 1) * DN_WARPS * 32) k_dense_mma(const Prob p) {
+  constexpr int HS = WIDE ? 16 : 8;            // heads per CTA
+  constexpr int NW = (WIDE ? 2 : 1) * DN_WARPS; // warps per CTA
+  constexpr int NST = DN_NST;
   constexpr int NC = D / 32;                   // 32-element chunks of a K row
   constexpr int ROWB = D * 2, KPAGE = 16 * ROWB;
   constexpr int STAGE = 2 * KPAGE;             // a K page and a V page
@@ -241,18 +247,21 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   constexpr int NB = D / 8;                    // 8-dim column blocks of the output
   constexpr int NE = dense_rec(D);
   extern __shared__ __align__(128) unsigned char smem_dyn[];
-  __shared__ float s_m[DN_WARPS][8], s_l[DN_WARPS][8];
+  __shared__ float s_m[NW][HS], s_l[NW][HS];
   __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
   const int gr = lane >> 2, t = lane & 3;
-  unsigned char* ring = smem_dyn + (size_t)warp * DN_NST * STAGE;
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)DN_WARPS * DN_NST * STAGE) + warp * DN_NST;
-  float* s_acc = reinterpret_cast<float*>(smem_dyn);          // [DN_WARPS][8][D], reuses the rings after the main loop
+  unsigned char* ring = smem_dyn + (size_t)warp * NST * STAGE;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_dyn + (size_t)NW * NST * STAGE) + warp * NST;
+  float* s_acc = reinterpret_cast<float*>(smem_dyn);          // [NW][HS][D], reuses the rings after the main loop
+  float* g_m = s_acc + NW * HS * D;                     // [HS][128] the merge's split maxima, [HS][128] weights,
+  float* g_sc = g_m + HS * 128;                               // [HS] denominators: behind the partials, also in the rings
+  float* g_den = g_sc + HS * 128;
 
   const int split = blockIdx.x, b = blockIdx.z, SG = gridDim.x;
-  const int GC = (p.G + 7) >> 3;
+  const int GC = (p.G + HS - 1) / HS;
   const int g = blockIdx.y / GC, hc = blockIdx.y % GC;
-  const int h0 = g * p.G + hc * 8, nh = min(8, p.G - hc * 8);
+  const int h0 = g * p.G + hc * HS, nh = min(HS, p.G - hc * HS);
   const int n = clamped_len(p, b);
   const int npages = (n + 15) >> 4;
   // a sequence takes the share of the SG splits that its length has of the longest possible one, so every
@@ -260,12 +269,12 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   const int npages_max = max(1, (p.max_seq_len + 15) >> 4);
   const int S = min(SG, max(1, (int)(((long long)SG * npages + npages_max - 1) / npages_max)));
   if (split >= S) return;
-  const int wglob = split * DN_WARPS + warp, wtot = S * DN_WARPS;
+  const int wglob = split * NW + warp, wtot = S * NW;
   const int mine = wglob < npages ? (npages - 1 - wglob) / wtot + 1 : 0;
   const bf16_t* kc = reinterpret_cast<const bf16_t*>(p.kc);
   const bf16_t* vc = reinterpret_cast<const bf16_t*>(p.vc);
 
-  if (lane < DN_NST) mbar_init(&bars[lane], 1);
+  if (lane < NST) mbar_init(&bars[lane], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncwarp();
@@ -279,8 +288,8 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   // whole warp: lane 0 arms the barrier, then one copy per page (lanes 0 and 16), or, when the rows of a
   // page are not contiguous, lanes 0..15 copy one V row each and lanes 16..31 one K row each
   auto issue = [&](int k, int pg) {
-    unsigned long long* bar = &bars[k % DN_NST];
-    unsigned char* dst = ring + (size_t)(k % DN_NST) * STAGE;
+    unsigned long long* bar = &bars[k % NST];
+    unsigned char* dst = ring + (size_t)(k % NST) * STAGE;
     const long long off = (long long)pg * p.sb + (long long)g * p.sh;
     if (lane == 0) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -295,25 +304,36 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     else bulk_g2s_stream(dst + (lane - 16) * ROWB, kc + off + (long long)(lane - 16) * p.st, ROWB, bar, stream_policy);
   };
   load_ids(0);
-  for (int k = 0; k < min(DN_NST, mine); ++k) issue(k, __shfl_sync(0xFFFFFFFFu, pg_ids, k));
-  // q as the A operand: head (h0 + gr) in rows 0..7, rows 8..15 zero
-  uint4 aq[NC];
+  for (int k = 0; k < min(NST, mine); ++k) issue(k, __shfl_sync(0xFFFFFFFFu, pg_ids, k));
+  // q as the A operand: head (h0 + gr) in rows 0..7; rows 8..15 zero, or heads h0 + 8 + gr (WIDE)
+  uint4 aq[NC], aq2[WIDE ? NC : 1];
 #pragma unroll
   for (int c = 0; c < NC; ++c) {
     aq[c] = make_uint4(0u, 0u, 0u, 0u);
     if (gr < nh)
       aq[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) + q_row(p, b, h0 + gr) + c * 32 + t * 8);
+    if (WIDE) {
+      aq2[c] = make_uint4(0u, 0u, 0u, 0u);
+      if (8 + gr < nh)
+        aq2[c] = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16_t*>(p.q) + q_row(p, b, h0 + 8 + gr) + c * 32 + t * 8);
+    }
   }
-  const int n_h = gr < nh ? head_len(p, b, h0 + gr) : n;   // tokens that head gr sees (query tokens of one call differ)
-  float m_run = -INFINITY, l_run = 0.f;        // head gr of this thread's row; l is this lane's share
-  float acc[NB][2];
+  constexpr int NHT = WIDE ? 2 : 1;            // heads per thread: gr, and 8 + gr
+  int n_h[NHT];                                // tokens that the head sees (query tokens of one call differ)
+  float m_run[NHT], l_run[NHT];                // l is this lane's share
+  float acc[NHT][NB][2];
 #pragma unroll
-  for (int nb = 0; nb < NB; ++nb) { acc[nb][0] = 0.f; acc[nb][1] = 0.f; }
+  for (int x = 0; x < NHT; ++x) {
+    n_h[x] = 8 * x + gr < nh ? head_len(p, b, h0 + 8 * x + gr) : n;
+    m_run[x] = -INFINITY; l_run[x] = 0.f;
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) { acc[x][nb][0] = 0.f; acc[x][nb][1] = 0.f; }
+  }
   bool failed = false;
 
   for (int k = 0; k < mine; ++k) {
-    const int s = k % DN_NST;
-    if (!mbar_wait(&bars[s], (unsigned)(k / DN_NST) & 1u)) { failed = true; break; }
+    const int s = k % NST;
+    if (!mbar_wait(&bars[s], (unsigned)(k / NST) & 1u)) { failed = true; break; }
     unsigned char* stg = ring + (size_t)s * STAGE;
     const int tok0 = (wglob + k * wtot) << 4;
     if (tok0 + 16 > n) {                       // last page: rows beyond n may hold anything; clear their V
@@ -321,37 +341,42 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
         for (int c = lane; c < ROWB / 4; c += 32) reinterpret_cast<unsigned*>(stg + KPAGE + r * ROWB)[c] = 0u;
       __syncwarp();
     }
-    // S^T for tokens 0..7 (sa) and 8..15 (sb): only c[0], c[1] (head gr) are meaningful
+    // S^T for tokens 0..7 (sa) and 8..15 (sb): c[0], c[1] are head gr, c[2], c[3] head 8 + gr (WIDE)
     float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
       const uint4 klo = *reinterpret_cast<const uint4*>(stg + gr * ROWB + c * 64 + t * 16);
       const uint4 khi = *reinterpret_cast<const uint4*>(stg + (gr + 8) * ROWB + c * 64 + t * 16);
-      mma_bf16_16816(sa, aq[c].x, 0u, aq[c].y, 0u, klo.x, klo.y);
-      mma_bf16_16816(sa, aq[c].z, 0u, aq[c].w, 0u, klo.z, klo.w);
-      mma_bf16_16816(sb, aq[c].x, 0u, aq[c].y, 0u, khi.x, khi.y);
-      mma_bf16_16816(sb, aq[c].z, 0u, aq[c].w, 0u, khi.z, khi.w);
+      mma_bf16_16816(sa, aq[c].x, WIDE ? aq2[WIDE ? c : 0].x : 0u, aq[c].y, WIDE ? aq2[WIDE ? c : 0].y : 0u, klo.x, klo.y);
+      mma_bf16_16816(sa, aq[c].z, WIDE ? aq2[WIDE ? c : 0].z : 0u, aq[c].w, WIDE ? aq2[WIDE ? c : 0].w : 0u, klo.z, klo.w);
+      mma_bf16_16816(sb, aq[c].x, WIDE ? aq2[WIDE ? c : 0].x : 0u, aq[c].y, WIDE ? aq2[WIDE ? c : 0].y : 0u, khi.x, khi.y);
+      mma_bf16_16816(sb, aq[c].z, WIDE ? aq2[WIDE ? c : 0].z : 0u, aq[c].w, WIDE ? aq2[WIDE ? c : 0].w : 0u, khi.z, khi.w);
     }
-    // this thread: head gr, tokens tok0 + {2t, 2t+1, 8+2t, 9+2t}
-    float sc[4] = {sa[0], sa[1], sb[0], sb[1]};
+    // this thread: heads gr (and 8 + gr), tokens tok0 + {2t, 2t+1, 8+2t, 9+2t}
     const int tk[4] = {tok0 + 2 * t, tok0 + 2 * t + 1, tok0 + 8 + 2 * t, tok0 + 9 + 2 * t};
-    float mx = -INFINITY;
+    float alpha[NHT];
+    unsigned pa[NHT][2];                       // exp(S - m) of tokens 2t, 2t+1 and of 8+2t, 9+2t, packed
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      sc[e] = (tk[e] < n_h) ? p.scale * sc[e] : -INFINITY;
-      mx = fmaxf(mx, sc[e]);
+    for (int x = 0; x < NHT; ++x) {
+      float sc[4] = {sa[2 * x], sa[2 * x + 1], sb[2 * x], sb[2 * x + 1]};
+      float mx = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        sc[e] = (tk[e] < n_h[x]) ? p.scale * sc[e] : -INFINITY;
+        mx = fmaxf(mx, sc[e]);
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+      const float m_new = fmaxf(m_run[x], mx);   // (-inf while the head has seen none of its tokens)
+      alpha[x] = (m_run[x] == -INFINITY) ? 0.f : __expf(m_run[x] - m_new);
+      float pr[4], psum = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { pr[e] = sc[e] == -INFINITY ? 0.f : __expf(sc[e] - m_new); psum += pr[e]; }
+      l_run[x] = l_run[x] * alpha[x] + psum;
+      m_run[x] = m_new;
+      pa[x][0] = pack_bf16x2(pr[0], pr[1]); pa[x][1] = pack_bf16x2(pr[2], pr[3]);
     }
-    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-    const float m_new = fmaxf(m_run, mx);      // (-inf while the head has seen none of its tokens)
-    const float alpha = (m_run == -INFINITY) ? 0.f : __expf(m_run - m_new);
-    float pr[4], psum = 0.f;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { pr[e] = sc[e] == -INFINITY ? 0.f : __expf(sc[e] - m_new); psum += pr[e]; }
-    l_run = l_run * alpha + psum;
-    m_run = m_new;
-    const unsigned pa0 = pack_bf16x2(pr[0], pr[1]), pa2 = pack_bf16x2(pr[2], pr[3]);
-    // out += P V: this thread's tokens 2t, 2t+1 (k slots of pa0) and 8+2t, 9+2t (pa2), 8 dims at a time
+    // out += P V: this thread's tokens 2t, 2t+1 (k slots of pa[.][0]) and 8+2t, 9+2t (pa[.][1]), 8 dims at a time
     const unsigned char* vrow = stg + KPAGE + (2 * t) * ROWB + gr * 16;
 #pragma unroll
     for (int hf = 0; hf < NH; ++hf) {
@@ -366,41 +391,49 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
         const unsigned sel = (e & 1) ? 0x7632u : 0x5410u;
         const unsigned b0 = prmt(w0[e >> 1], w1[e >> 1], sel), b1 = prmt(w2[e >> 1], w3[e >> 1], sel);
         const int nb = hf * 8 + e;
-        float c0[4] = {acc[nb][0] * alpha, acc[nb][1] * alpha, 0.f, 0.f};
-        mma_bf16_16816(c0, pa0, 0u, pa2, 0u, b0, b1);
-        acc[nb][0] = c0[0]; acc[nb][1] = c0[1];
+        float c0[4] = {acc[0][nb][0] * alpha[0], acc[0][nb][1] * alpha[0], WIDE ? acc[NHT - 1][nb][0] * alpha[NHT - 1] : 0.f,
+                       WIDE ? acc[NHT - 1][nb][1] * alpha[NHT - 1] : 0.f};
+        mma_bf16_16816(c0, pa[0][0], WIDE ? pa[NHT - 1][0] : 0u, pa[0][1], WIDE ? pa[NHT - 1][1] : 0u, b0, b1);
+        acc[0][nb][0] = c0[0]; acc[0][nb][1] = c0[1];
+        if (WIDE) { acc[NHT - 1][nb][0] = c0[2]; acc[NHT - 1][nb][1] = c0[3]; }
       }
     }
     __syncwarp();
-    if (k + DN_NST < mine) {
-      if (((k + DN_NST) & 31) == 0) load_ids(k + DN_NST);
-      issue(k + DN_NST, __shfl_sync(0xFFFFFFFFu, pg_ids, (k + DN_NST) & 31));
+    if (k + NST < mine) {
+      if (((k + NST) & 31) == 0) load_ids(k + NST);
+      issue(k + NST, __shfl_sync(0xFFFFFFFFu, pg_ids, (k + NST) & 31));
     }
   }
   if (failed) {
     if (lane == 0) atomicOr(p.status, VATTN_STATUS_WAIT_TIMEOUT);
-    for (int s = 0; s < DN_NST; ++s) mbar_wait(&bars[s], 0u) || mbar_wait(&bars[s], 1u);
+    for (int s = 0; s < NST; ++s) mbar_wait(&bars[s], 0u) || mbar_wait(&bars[s], 1u);
   }
-  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
-  l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
+#pragma unroll
+  for (int x = 0; x < NHT; ++x) {
+    l_run[x] += __shfl_xor_sync(0xFFFFFFFFu, l_run[x], 1);
+    l_run[x] += __shfl_xor_sync(0xFFFFFFFFu, l_run[x], 2);
+  }
   __syncthreads();                             // every warp is done with its ring: reuse it for the partials
   // accumulator (block 8 hf + e, columns 2t and 2t+1) is dim 64 hf + 8 (2t) + e and 64 hf + 8 (2t+1) + e
 #pragma unroll
-  for (int nb = 0; nb < NB; ++nb) {
-    s_acc[(warp * 8 + gr) * D + (nb >> 3) * 64 + 16 * t + (nb & 7)] = acc[nb][0];
-    s_acc[(warp * 8 + gr) * D + (nb >> 3) * 64 + 16 * t + 8 + (nb & 7)] = acc[nb][1];
+  for (int x = 0; x < NHT; ++x) {
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+      s_acc[(warp * HS + 8 * x + gr) * D + (nb >> 3) * 64 + 16 * t + (nb & 7)] = acc[x][nb][0];
+      s_acc[(warp * HS + 8 * x + gr) * D + (nb >> 3) * 64 + 16 * t + 8 + (nb & 7)] = acc[x][nb][1];
+    }
+    if (t == 0) { s_m[warp][8 * x + gr] = m_run[x]; s_l[warp][8 * x + gr] = l_run[x]; }
   }
-  if (t == 0) { s_m[warp][gr] = m_run; s_l[warp][gr] = l_run; }
   __syncthreads();
   // CTA partial -> global: [D] unnormalised sums, then m and l, per head; warps in a fixed order
-  __shared__ float s_w[DN_WARPS][8];           // weight of warp w's partial inside the CTA's
-  if (tid < 8) {
+  __shared__ float s_w[NW][HS];          // weight of warp w's partial inside the CTA's
+  if (tid < HS) {
     float mc = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < DN_WARPS; ++w) mc = fmaxf(mc, s_m[w][tid]);
+    for (int w = 0; w < NW; ++w) mc = fmaxf(mc, s_m[w][tid]);
     float lc = 0.f;
 #pragma unroll
-    for (int w = 0; w < DN_WARPS; ++w) {
+    for (int w = 0; w < NW; ++w) {
       const float sc = (s_m[w][tid] == -INFINITY) ? 0.f : __expf(s_m[w][tid] - mc);
       s_w[w][tid] = sc;
       lc += sc * s_l[w][tid];
@@ -409,13 +442,13 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
       *reinterpret_cast<float4*>(p.dense_part + (((long long)b * p.Hq + h0 + tid) * SG + split) * NE + D) = make_float4(mc, lc, 0.f, 0.f);
   }
   __syncthreads();
-  for (int idx = tid; idx < nh * (D / 4); idx += DN_WARPS * 32) {
+  for (int idx = tid; idx < nh * (D / 4); idx += NW * 32) {
     const int hh = idx / (D / 4), e = (idx % (D / 4)) * 4;
     float4 val = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int w = 0; w < DN_WARPS; ++w) {
+    for (int w = 0; w < NW; ++w) {
       const float sc = s_w[w][hh];
-      const float4 x = *reinterpret_cast<const float4*>(&s_acc[(w * 8 + hh) * D + e]);
+      const float4 x = *reinterpret_cast<const float4*>(&s_acc[(w * HS + hh) * D + e]);
       val.x += sc * x.x; val.y += sc * x.y; val.z += sc * x.z; val.w += sc * x.w;
     }
     *reinterpret_cast<float4*>(p.dense_part + (((long long)b * p.Hq + h0 + hh) * SG + split) * NE + e) = val;
@@ -435,18 +468,18 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   // last CTA of the group.  Two rounds of loads: every split's (m, l) pair; then, per four output
   // elements, the S partials with up to MB of them in flight, added in split order
   constexpr int MB = 20;
-  __shared__ float g_m[8][128], g_sc[8][128], g_den[8];
-  for (int idx = tid; idx < 8 * S; idx += DN_WARPS * 32) {
+  __syncthreads();                             // (the partials in shared memory have been read)
+  for (int idx = tid; idx < HS * S; idx += NW * 32) {
     const int hh = idx / S, sp = idx % S;
     if (hh < nh) {
       const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.dense_part + (((long long)b * p.Hq + h0 + hh) * SG + sp) * NE + D));
-      g_m[hh][sp] = ml.x; g_sc[hh][sp] = ml.y;
+      g_m[hh * 128 + sp] = ml.x; g_sc[hh * 128 + sp] = ml.y;
     }
   }
   __syncthreads();
-  for (int hh = warp; hh < nh; hh += DN_WARPS) {
+  for (int hh = warp; hh < nh; hh += NW) {
     float mg = -INFINITY;
-    for (int sp = lane; sp < S; sp += 32) mg = fmaxf(mg, g_m[hh][sp]);
+    for (int sp = lane; sp < S; sp += 32) mg = fmaxf(mg, g_m[hh * 128 + sp]);
 #pragma unroll
     for (int mk = 16; mk >= 1; mk >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xFFFFFFFFu, mg, mk));
     float den = 0.f;
@@ -454,10 +487,10 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
       const int sp = sp0 + lane;
       float lv = 0.f;
       if (sp < S) {
-        const float ms = g_m[hh][sp];
+        const float ms = g_m[hh * 128 + sp];
         const float scv = (ms == -INFINITY) ? 0.f : __expf(ms - mg);
-        lv = scv * g_sc[hh][sp];
-        g_sc[hh][sp] = scv;
+        lv = scv * g_sc[hh * 128 + sp];
+        g_sc[hh * 128 + sp] = scv;
       }
 #pragma unroll
       for (int mk = 16; mk >= 1; mk >>= 1) lv += __shfl_xor_sync(0xFFFFFFFFu, lv, mk);
@@ -466,7 +499,7 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
     if (lane == 0) g_den[hh] = den;
   }
   __syncthreads();
-  for (int idx = tid; idx < nh * (D / 4); idx += DN_WARPS * 32) {
+  for (int idx = tid; idx < nh * (D / 4); idx += NW * 32) {
     const int hh = idx / (D / 4), e = (idx % (D / 4)) * 4;
     const long long bh = (long long)b * p.Hq + h0 + hh;
     const float* base = p.dense_part + bh * SG * NE + e;
@@ -478,7 +511,7 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
         v[u] = (sp0 + u < S) ? __ldcg(reinterpret_cast<const float4*>(base + (long long)(sp0 + u) * NE)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int u = 0; u < MB; ++u) {
-        const float scv = (sp0 + u < S) ? g_sc[hh][sp0 + u] : 0.f;
+        const float scv = (sp0 + u < S) ? g_sc[hh * 128 + sp0 + u] : 0.f;
         num.x += scv * v[u].x; num.y += scv * v[u].y; num.z += scv * v[u].z; num.w += scv * v[u].w;
       }
     }
@@ -491,26 +524,26 @@ __global__ void __launch_bounds__(DN_WARPS * 32) k_dense_mma(const Prob p) {
   }
 }
 
-template <int D>
+template <int D, bool WIDE>
 static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
-  constexpr int STAGE = 2 * 16 * D * 2;
-  const size_t ring = (size_t)DN_WARPS * DN_NST * STAGE;
-  const size_t accb = (size_t)DN_WARPS * 8 * D * sizeof(float);
-  const size_t smem = (ring > accb ? ring : accb) + DN_WARPS * DN_NST * 8;
+  constexpr int STAGE = 2 * 16 * D * 2, HS = WIDE ? 16 : 8, NST = DN_NST, NW = (WIDE ? 2 : 1) * DN_WARPS;
+  const size_t ring = (size_t)NW * NST * STAGE;
+  const size_t accb = ((size_t)NW * HS * D + 2 * HS * 128 + HS) * sizeof(float);
+  const size_t smem = (ring > accb ? ring : accb) + NW * NST * 8;
   static size_t have[VATTN_MAXDEV];
-  cudaError_t e = optin_smem(k_dense_mma<D>, smem, have);
+  cudaError_t e = optin_smem(k_dense_mma<D, WIDE>, smem, have);
   if (e != cudaSuccess) return e;
-  const int GC = (p.G + 7) / 8;
+  const int GC = (p.G + HS - 1) / HS;
   const int groups = p.B * p.Hkv * GC;
-  // Two CTAs fit an SM (registers and shared memory).  With few groups: as many splits as fill one wave, rounded
-  // down (a second, partly filled wave costs a whole CTA's duration).  With many groups (large batches, whose
-  // lengths differ): pieces small enough for four to five waves, so the SMs drain evenly.
-  const int slots = 2 * device_sm_count();
+  // Two CTAs fit an SM (registers and shared memory; one of the 16-head kind).  With few groups: as many splits as
+  // fill one wave, rounded down (a second, partly filled wave costs a whole CTA's duration).  With many groups (large
+  // batches, whose lengths differ): pieces small enough for four to five waves, so the SMs drain evenly.
+  const int slots = (WIDE ? 1 : 2) * device_sm_count();
   int S = slots / groups >= 3 ? slots / groups : (9 * slots / 2 + groups - 1) / groups;
   if (S > p.dense_splits) S = p.dense_splits;
   if (S < 1) S = 1;
-  dim3 grid(S, p.Hkv * GC, p.B), block(DN_WARPS * 32);
-  k_dense_mma<D><<<grid, block, smem, s>>>(p);
+  dim3 grid(S, p.Hkv * GC, p.B), block(NW * 32);
+  k_dense_mma<D, WIDE><<<grid, block, smem, s>>>(p);
   return cudaGetLastError();
 }
 }  // namespace
@@ -518,7 +551,8 @@ static cudaError_t launch_dense_mma(const Prob& p, cudaStream_t s) {
 cudaError_t launch_dense(const Prob& p, cudaStream_t s, int* launches) {
   if (p.dtype == VATTN_DTYPE_BF16) {
     if (launches) *launches = 1;
-    return p.D == 128 ? launch_dense_mma<128>(p, s) : launch_dense_mma<64>(p, s);
+    if (p.G > 8) return p.D == 128 ? launch_dense_mma<128, true>(p, s) : launch_dense_mma<64, true>(p, s);
+    return p.D == 128 ? launch_dense_mma<128, false>(p, s) : launch_dense_mma<64, false>(p, s);
   } else {
     const int GC = (p.G + 3) / 4;
     const int groups = p.B * p.Hkv * GC;
