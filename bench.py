@@ -251,6 +251,8 @@ def main():
                     help="run only warm-up + a few plain (non-graph) steps: the command ncu captures")
     ap.add_argument("--profile-dense", action="store_true",
                     help="with --profile-only: every step is followed by the dense comparison kernel on the same inputs")
+    ap.add_argument("--profile-qlen", type=int, default=1,
+                    help="with --profile-only: query tokens per sequence and call (vattn_shape.q_len)")
     ap.add_argument("--profile-config", default="cfg2", choices=["cfg2", "cfg5", "cfg4"],
                     help="with --profile-only: the workload to run (cfg5: batch 8 at n=32768; cfg4: batch 32, mixed "
                          "lengths; one cache pool each, 1.1 GB and 2.6 GB)")
@@ -290,8 +292,12 @@ def main():
         case = {"cfg5": synth.config5_reasoning, "cfg4": synth.config4_serving}[args.profile_config]()
         npools = 1                                         # the cache alone is several times the L2
     dev0 = vb.case_to_device(case)
+    q_len = args.profile_qlen if args.profile_only else 1
+    if q_len > 1:                                          # several query tokens per call: q is [B, q_len, Hq, d]
+        dev0["q"] = torch.from_numpy(np.ascontiguousarray(synth.multi_query(case, q_len)).view(np.int16)).cuda().view(
+            torch.bfloat16)
     pools = [dev0] + [{k: v.clone() for k, v in dev0.items()} for _ in range(npools - 1)]
-    plan = vb.plan_for_case(case)
+    plan = vb.plan_for_case(case, q_len=q_len)
     plan.set_params(**case.params)
     outs = [torch.empty_like(dev0["q"]) for _ in range(POOLS)]
     stream = torch.cuda.Stream()
