@@ -152,7 +152,8 @@ struct Gather {
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
           tok[u] = tok_n[u];
-          const int ph = ph_n[u];
+          int ph = ph_n[u];
+          CHECK_SLOT(p, ph, 2);
           off[u] = (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL;
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (FULL || tok[u] >= 0) raw[u] = __ldcs(reinterpret_cast<const uint4*>(kcg + off[u]));
@@ -180,10 +181,12 @@ struct Gather {
           if (!FULL) raw[u] = make_uint4(0u, 0u, 0u, 0u);
           if (j == u) tok_mine = tok[u];
           if (FULL || tok[u] >= 0) {
-            const int ph = ph_n[u];
+            int ph = ph_n[u];
+            CHECK_SLOT(p, ph, 3);
             raw[u] = __ldcs(reinterpret_cast<const uint4*>(vc + (long long)(ph >> 4) * p.sb + (long long)(ph & 15) * p.st + j * EPL));
           }
         }
+        CHECK_TOK(p, tok_mine, 5);
         if (tok_mine >= 0) w_mine = __ldg(sc + tok_mine);
         fetch_next(k0 + UNROLL);
         if (FAR && j < UNROLL && far_member(k0, j, tok_mine, w_mine)) tok_mine = -1;                        // next batch's indices travel with this batch's rows

@@ -372,6 +372,10 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
       if (i >= s0 && i < l_start) { atomicAdd(&hA[keys[key_slot(i)] >> 21], 1); ++ns_loc; }
     }
     int ns_tot;
+    // A middle range of a few tokens may hold no sampled token at all (a page's sample sits at one offset): the
+    // pick below then finds no bin and writes nothing, so its outputs are preset to bin 0 (the largest scores:
+    // pass B verifies that choice like any other and falls back to the general selection when it is wrong).
+    if (tid == 0) { sm.misc[0] = 0; sm.misc[1] = 0; }
     block_scan_reg(ns_loc, sm.misc + 32, ns_tot);      // (one barrier: the sample histogram is complete behind it)
     __syncthreads();
     {

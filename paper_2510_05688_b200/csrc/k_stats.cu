@@ -55,6 +55,7 @@ struct RowRegs { Raw<T> k, v; };
 template <typename T, int D>
 __device__ __forceinline__ void load_row(const Prob& p, int g, int ph, int j, RowRegs<T>& r) {
   constexpr int EPL = Elem<T>::EPL;
+  CHECK_SLOT(p, ph, 1);
   const long long off = (long long)(ph >> 4) * p.sb + (long long)g * p.sh + (long long)(ph & 15) * p.st + j * EPL;
   r.k.ld(reinterpret_cast<const T*>(p.kc) + off);
   r.v.ld(reinterpret_cast<const T*>(p.vc) + off);

@@ -190,6 +190,21 @@ template <> struct Elem<bf16_t> {
 };
 
 // physical page of logical page `lp` of batch row b (bounds-checked; a bad entry raises a status bit)
+// Diagnosis builds (-DVATTN_CHECK_SLOTS): a physical slot (page * 16 + token % 16) is checked before it becomes an
+// address; a slot outside the cache is recorded (status bit, first offender's value and site) and replaced by slot 0.
+#ifdef VATTN_CHECK_SLOTS
+#define CHECK_SLOT(p, ph, site) do { if ((unsigned)((ph) >> 4) >= (unsigned)(p).num_blocks) { \
+    atomicOr((p).status, VATTN_STATUS_BAD_BLOCK); \
+    if ((p).dbg.paths) { (p).dbg.paths[0] = 0x40000000 | (site); (p).dbg.paths[1] = (ph); (p).dbg.paths[2] = blockIdx.x | (blockIdx.y << 12) | (blockIdx.z << 24); } \
+    (ph) = 0; } } while (0)
+#define CHECK_TOK(p, tok, site) do { if ((tok) >= (p).npad) { \
+    atomicOr((p).status, VATTN_STATUS_BAD_BLOCK); \
+    if ((p).dbg.paths) { (p).dbg.paths[0] = 0x40000000 | (site); (p).dbg.paths[1] = (tok); (p).dbg.paths[2] = blockIdx.x | (blockIdx.y << 12) | (blockIdx.z << 24); } \
+    (tok) = -1; } } while (0)
+#else
+#define CHECK_SLOT(p, ph, site) do { } while (0)
+#define CHECK_TOK(p, tok, site) do { } while (0)
+#endif
 __device__ __forceinline__ int page_of(const Prob& p, int b, int lp) {
   int pg = p.bt[(long long)b * p.max_blocks + lp];
   if ((unsigned)pg >= (unsigned)p.num_blocks) { atomicOr(p.status, VATTN_STATUS_BAD_BLOCK); pg = 0; }

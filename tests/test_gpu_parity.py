@@ -104,6 +104,15 @@ def test_k_zero_and_k_larger_than_middle():
     check(small("bf16", [400, 77], sink=0, window=0, k=7))
 
 
+def test_middle_range_without_a_sampled_token():
+    """Middle ranges of a few tokens that miss the one token per page which the selection samples for its threshold
+    estimate (page 0 is sampled at offset 0, page 1 at offset 0, page 2 at offset 1, ...): the estimate has nothing to
+    go on and the selection must still be exact."""
+    check(small("bf16", [14, 15, 16, 10, 12, 31, 40], sink=4, window=1, k=1))
+    check(small("bf16", [14, 16, 30], sink=4, window=1, k=3, params=dict(base_rate=0.1, nested_base=1)))
+    check(small("fp32", [13, 20, 47], d=64, sink=1, window=2, k=2))
+
+
 def test_topk_fraction_and_kv_head_rng():
     check(small("bf16", [900, 350], k=0, params=dict(base_rate=0.05, topk_frac=0.03)))
     check(small("bf16", [900, 350], params=dict(base_rate=0.1, rng_head_is_kv=1, layer=3, step=77)))
