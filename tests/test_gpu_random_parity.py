@@ -1,0 +1,85 @@
+"""GPU parity on seeded random small problems: shapes, lengths, index-set sizes, (eps, delta), parameter switches
+and the number of query tokens per call drawn at random, each compared with the oracle like the fixed cases.
+
+The fixed tests choose their shapes by hand; this sweep reaches the combinations nobody thought of (the first one
+it found: a middle range of nine tokens that held none of the tokens the selection samples for its threshold
+estimate).  The plans of one sweep are created one after another in one process, so a kernel that reads scratch
+it has not written meets whatever the plan before it left there.
+"""
+import numpy as np
+import pytest
+
+from paper_2510_05688_b200 import synth
+from helpers import (assert_out_close, assert_parity, assert_parity_multi, run_gpu, run_gpu_multi, run_oracle,
+                     run_oracle_multi)
+
+pytestmark = pytest.mark.gpu
+
+LENGTHS = [0, 1, 2, 15, 16, 17, 31, 33, 64, 100, 255, 256, 257, 500, 777, 1024, 1500, 2049, 3000]
+
+
+def draw_case(rng):
+    dtype = str(rng.choice(["bf16", "fp32"]))
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 4]))
+    G = int(rng.choice([1, 2, 3, 4, 5, 8]))
+    B = int(rng.integers(1, 6))
+    lens = [int(x) for x in rng.choice(LENGTHS, size=B)]
+    params = dict(base_rate=float(rng.choice([0.025, 0.05, 0.1, 0.3])))
+    if rng.random() < 0.3:
+        params["topk_frac"] = float(rng.choice([0.01, 0.03, 0.1]))
+    if rng.random() < 0.3:
+        params["mode"] = int(rng.integers(0, 3))
+    if rng.random() < 0.3:
+        params["rng_head_is_kv"] = 1
+    if rng.random() < 0.3:
+        params["nested_base"] = 1
+    if rng.random() < 0.2:
+        params["gather_mode"] = 1
+    if rng.random() < 0.3:
+        params["step"] = int(rng.integers(0, 100000))
+        params["layer"] = int(rng.integers(0, 64))
+    if rng.random() < 0.15:
+        params["force_budget"] = int(rng.choice([0, 5, 100, 10**9]))
+    heavy = None if rng.random() < 0.3 else dict(R=int(rng.integers(1, 20)), c1=float(rng.choice([2.0, 5.0, 9.0])),
+                                                 alpha=(0.75, 1.25))
+    q_len = int(rng.choice([1, 1, 1, 2, 3, 4]))
+    case = synth.make_case("random", dtype=dtype, B=B, Hq=Hkv * G, Hkv=Hkv, d=d, seq_lens=lens,
+                           sink=int(rng.choice([0, 1, 4, 16, 128])), window=int(rng.choice([0, 1, 8, 16, 128])),
+                           k=int(rng.choice([0, 1, 7, 16, 64, 300, 100000])),
+                           eps=float(rng.choice([0.02, 0.05, 0.1, 0.3])), delta=float(rng.choice([0.01, 0.05, 0.2])),
+                           seed=int(rng.integers(0, 2**31)), gen_seed=int(rng.integers(0, 2**31)), key_std=1.0,
+                           rho_v=1.0, heavy=heavy, params=params)
+    return case, q_len
+
+
+@pytest.mark.parametrize("sweep", [1, 2])
+def test_random_problems_with_introspection(sweep):
+    """Index sets, budgets, statistics and outputs (the introspection switches on the list-building paths)."""
+    for it in range(40):
+        case, q_len = draw_case(np.random.default_rng(sweep * 100003 + it))
+        if q_len == 1:
+            out_ref, det = run_oracle(case)
+            out, dbg, plan = run_gpu(case)
+            assert_parity(case, out, dbg, det, out_ref)
+        else:
+            q4 = synth.multi_query(case, q_len)
+            out_ref, det = run_oracle_multi(case, q4)
+            out, dbg, plan, _ = run_gpu_multi(case, q4)
+            assert_parity_multi(case, q_len, out, dbg, det, out_ref)
+        assert plan.last_status() & ~4 == 0, (sweep, it)
+
+
+def test_random_problems_outputs_only():
+    """Without introspection the samples are read off the walk arrays (no lists): outputs against the oracle."""
+    for it in range(40):
+        case, q_len = draw_case(np.random.default_rng(31 * 100003 + it))
+        if q_len == 1:
+            out_ref, _ = run_oracle(case)
+            out, _, plan = run_gpu(case, debug=False)
+        else:
+            q4 = synth.multi_query(case, q_len)
+            out_ref, _ = run_oracle_multi(case, q4)
+            out, _, plan, _ = run_gpu_multi(case, q4, debug=False)
+        assert_out_close(case, out.reshape(out_ref.shape), out_ref, f"outputs only, case {it}")
+        assert plan.last_status() & ~4 == 0, it
