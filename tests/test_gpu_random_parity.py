@@ -83,3 +83,53 @@ def test_random_problems_outputs_only():
             out, _, plan, _ = run_gpu_multi(case, q4, debug=False)
         assert_out_close(case, out.reshape(out_ref.shape), out_ref, f"outputs only, case {it}")
         assert plan.last_status() & ~4 == 0, it
+
+
+def test_random_dense_problems():
+    """The dense comparison kernels on random shapes: group sizes 1..16 (both tile widths), batches up to 19 mixed
+    lengths, one to four query tokens, twice in a row (the kernel puts its counters back), and the entry point that
+    allocates nothing where it applies."""
+    import torch
+    from oracle import vattn_oracle as O
+    from paper_2510_05688_b200 import binding as vb
+    lengths = LENGTHS + [5000, 9001]
+    for it in range(40):
+        rng = np.random.default_rng(7 * 7919 + it)
+        dtype = str(rng.choice(["bf16", "bf16", "fp32"]))
+        d = int(rng.choice([64, 128]))
+        Hkv = int(rng.choice([1, 2, 3, 4, 8]))
+        G = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 12, 16]))
+        B = int(rng.integers(1, 20))
+        lens = [int(x) for x in rng.choice(lengths, size=B)]
+        q_len = int(rng.choice([1, 1, 2, 3, 4]))
+        case = synth.make_case("random_dense", dtype=dtype, B=B, Hq=Hkv * G, Hkv=Hkv, d=d, seq_lens=lens, sink=4,
+                               window=4, k=4, eps=0.1, delta=0.1, seed=1, gen_seed=int(rng.integers(0, 2**31)),
+                               key_std=1.0, rho_v=1.0, heavy=None, params={})
+        q4 = synth.multi_query(case, q_len)
+        dev = vb.case_to_device(case)
+        if dtype == "bf16":
+            qd = torch.from_numpy(np.ascontiguousarray(q4).view(np.int16)).cuda().view(torch.bfloat16)
+        else:
+            qd = torch.from_numpy(np.ascontiguousarray(q4)).cuda()
+        plan = vb.plan_for_case(case, q_len=q_len)
+        ref = O.dense_decode_multi(q4, case.k_cache, case.v_cache, case.block_table, case.seq_lens, dtype=dtype)
+        tol = 2e-2 if dtype == "bf16" else 2e-5
+        bits = torch.int16 if dtype == "bf16" else torch.int32
+        outs = []
+        for _ in range(2):
+            out = torch.empty_like(qd)
+            plan.dense_decode(qd, dev["k_cache"], dev["v_cache"], dev["block_table"], dev["seq_lens"], out)
+            torch.cuda.synchronize()
+            got = out.float().cpu().numpy().astype(np.float64)
+            assert (np.abs(got - ref) <= tol * np.maximum(1.0, np.abs(ref))).all(), (it, np.abs(got - ref).max())
+            outs.append(out)
+        assert torch.equal(outs[0].view(bits), outs[1].view(bits)) and plan.last_status() == 0, it
+        if q_len == 1:
+            out = torch.empty_like(dev["q"])
+            rc = vb.dense_decode_noalloc(plan.shape, dev["q"], dev["k_cache"], dev["v_cache"], dev["block_table"],
+                                         dev["seq_lens"], out)
+            torch.cuda.synchronize()
+            assert rc in (vb.OK, vb.ERR_WORKSPACE), rc
+            if rc == vb.OK:
+                got = out.float().cpu().numpy().astype(np.float64)
+                assert (np.abs(got - ref[:, 0]) <= tol * np.maximum(1.0, np.abs(ref[:, 0]))).all(), it
