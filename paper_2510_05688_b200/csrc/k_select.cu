@@ -761,23 +761,35 @@ __global__ void __launch_bounds__(NT, 1) k_select(const Prob p) {
     const int H0 = cnts[0];
     if (H0 > HBINS) base_list = 1;
     else if (warp == 0) {
-      // J = b0 + #{marked positions < J}; the pivot = the first unmarked position
-      int J = b0;
-      for (int it = 0; it < 64; ++it) {
+      // J = b0 + #{marked positions < J}; the pivot = the first unmarked position.  "The prefix that holds `want`
+      // unmarked entries" is the least fixed point of J -> want + #{marked < J}: a few steps from J = want in the
+      // usual case; when nearly every position is marked (top-k sets that take most of the middle range) the steps
+      // are as short as the runs of marked positions, so after eight of them a bisection takes over (J minus the
+      // marked positions below J never decreases).  W0 + 1: the array holds fewer than `want` unmarked entries.
+      auto below = [&](int J) {
         int c = 0;
         for (int i = lane; i < H0; i += 32) c += hp0[i] < J;
 #pragma unroll
         for (int mk = 16; mk >= 1; mk >>= 1) c += __shfl_xor_sync(FULL, c, mk);
-        if (b0 + c == J) break;
-        J = b0 + c;
-      }
-      int pivx = 0;
-      for (int it = 0; it < 64; ++it) {
-        int hit = 0;
-        for (int i = lane; i < H0; i += 32) hit |= hp0[i] == pivx;
-        if (!__any_sync(FULL, hit)) break;
-        ++pivx;
-      }
+        return c;
+      };
+      auto prefix_for = [&](int want) {
+        int J = want;
+        for (int it = 0; it < 8; ++it) {
+          const int c = below(J);
+          if (want + c == J) return J;
+          J = want + c;
+        }
+        if (W0 - below(W0) < want) return W0 + 1;
+        int lo_ = min(J, W0), hi_ = W0;                  // the steps above never overshoot the fixed point
+        while (lo_ < hi_) {
+          const int mid = (lo_ + hi_) >> 1;
+          if (mid - below(mid) >= want) hi_ = mid; else lo_ = mid + 1;
+        }
+        return lo_;
+      };
+      const int J = prefix_for(b0);
+      const int pivx = prefix_for(1) - 1;
       int ph = __shfl_sync(FULL, pvph, pivx & 3);
       if (pivx >= 4 && pivx < W0) ph = __ldcg(wa0 + p.npad + pivx);
       if (lane == 0) { sm.misc[4] = J; sm.misc[5] = ph; sm.misc[6] = (J > W0 || pivx >= W0) ? 1 : 0; }

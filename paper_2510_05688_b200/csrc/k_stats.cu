@@ -240,21 +240,37 @@ __device__ __noinline__ void head_budget(const Prob& p, int b, int h, int bh, do
     if (!listed) {
       const int* hd = p.hole_pos + (long long)bh * 2 * VATTN_BANDCAP;
       const bool far = bf > mt.dyn_J - nholes;           // reaches beyond the walk array: the members there count too
-      for (int it = 0; it < 64; ++it) {
+      auto marked_below = [&](int Jq) {                   // (uniform over the warp)
         int c = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) c += __popc(__ballot_sync(FULLMASK, hp[i] < J));
-        for (int i0 = 256; i0 < nholes; i0 += 32) {            // (uniform over the warp)
+        for (int i = 0; i < 8; ++i) c += __popc(__ballot_sync(FULLMASK, hp[i] < Jq));
+        for (int i0 = 256; i0 < nholes; i0 += 32) {
           const int v = i0 + lane < nholes ? __ldcg(hd + i0 + lane) : 0x7FFFFFFF;
-          c += __popc(__ballot_sync(FULLMASK, v < J));
+          c += __popc(__ballot_sync(FULLMASK, v < Jq));
         }
         if (far)
           for (int i0 = 0; i0 < nholes2; i0 += 32) {
             const int v = i0 + lane < nholes2 ? __ldcg(hd + VATTN_BANDCAP + i0 + lane) : 0x7FFFFFFF;
-            c += __popc(__ballot_sync(FULLMASK, v < J));
+            c += __popc(__ballot_sync(FULLMASK, v < Jq));
           }
-        if (bf + c == J) break;
+        return c;
+      };
+      // the least fixed point of J -> b + #{marked < J}: a few steps in the usual case; with nearly every position
+      // marked the steps are as short as the runs of marked positions, so after eight a bisection takes over
+      bool conv = false;
+      for (int it = 0; it < 8; ++it) {
+        const int c = marked_below(J);
+        if (bf + c == J) { conv = true; break; }
         J = bf + c;
+      }
+      if (!conv) {
+        int lo_ = J, hi_ = far ? mt.l_start - mt.s0 : mt.dyn_J;
+        lo_ = min(lo_, hi_);
+        while (lo_ < hi_) {
+          const int mid = (lo_ + hi_) >> 1;
+          if (mid - marked_below(mid) >= bf) hi_ = mid; else lo_ = mid + 1;
+        }
+        J = lo_;
       }
     }
     if (lane == 0) {

@@ -113,6 +113,22 @@ def test_middle_range_without_a_sampled_token():
     check(small("fp32", [13, 20, 47], d=64, sink=1, window=2, k=2))
 
 
+def test_topk_takes_almost_the_whole_middle_range():
+    """k within a few tokens of the middle range: nearly every walk position is a member of I_t, so the prefix that
+    holds the base sample (and the pivot, and the final sample) lies behind long runs of marked positions."""
+    case = small("bf16", [202, 300, 150, 1000], sink=0, window=1, k=200, params=dict(base_rate=0.3))
+    check(case)                                        # residuals of 1, 99, 0 and 799 tokens
+    out_ref, _ = run_oracle(case)
+    out, _, _ = run_gpu(case, debug=False)             # (without introspection the samples come off the walk arrays)
+    assert_out_close(case, out, out_ref, "k = middle - 1")
+    for k in (995, 990, 900):
+        case = small("bf16", [1000], sink=2, window=2, k=k, params=dict(base_rate=0.1, nested_base=k % 2))
+        check(case)
+        out_ref, _ = run_oracle(case)
+        out, _, _ = run_gpu(case, debug=False)
+        assert_out_close(case, out, out_ref, f"k = {k} of 996")
+
+
 def test_topk_fraction_and_kv_head_rng():
     check(small("bf16", [900, 350], k=0, params=dict(base_rate=0.05, topk_frac=0.03)))
     check(small("bf16", [900, 350], params=dict(base_rate=0.1, rng_head_is_kv=1, layer=3, step=77)))
