@@ -133,3 +133,52 @@ def test_random_dense_problems():
             if rc == vb.OK:
                 got = out.float().cpu().numpy().astype(np.float64)
                 assert (np.abs(got - ref[:, 0]) <= tol * np.maximum(1.0, np.abs(ref[:, 0]))).all(), it
+
+
+def test_random_calls_on_one_plan():
+    """A decode loop: one plan and one cache, every call with other lengths (empty sequences included), index-set
+    sizes, (eps, delta), seeds and switches.  What a call leaves in the workspace must not reach the next one."""
+    import copy
+    import torch
+    from paper_2510_05688_b200 import binding as vb
+    for it in range(12):
+        rng = np.random.default_rng(1 * 15485863 + 20 + it)          # (session 27 of this stream found the prefix search's step limit)
+        dtype = str(rng.choice(["bf16", "fp32"]))
+        d = int(rng.choice([64, 128]))
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 4, 8]))
+        B = int(rng.integers(1, 6))
+        maxlens = [int(x) for x in rng.choice([64, 300, 1000, 2049, 4000], size=B)]
+        base = synth.make_case("one_plan", dtype=dtype, B=B, Hq=Hkv * G, Hkv=Hkv, d=d, seq_lens=maxlens, sink=4,
+                               window=8, k=16, eps=0.05, delta=0.05, seed=1, gen_seed=int(rng.integers(0, 2**31)),
+                               key_std=1.0, rho_v=1.0, heavy=dict(R=12, c1=5.0, alpha=(0.75, 1.25)),
+                               params=dict(base_rate=0.05))
+        dev = vb.case_to_device(base)
+        plan = vb.plan_for_case(base)
+        for step in range(8):
+            case = copy.copy(base)
+            lens = np.array([int(rng.integers(0, m + 1)) if rng.random() < 0.8 else int(rng.choice([0, 1, 15, 16, 17, m]))
+                             for m in maxlens], np.int32)
+            case.seq_lens = lens
+            case.sink = int(rng.choice([0, 1, 4, 64]))
+            case.window = int(rng.choice([0, 1, 8, 64]))
+            case.k = int(rng.choice([0, 1, 16, 200, 100000]))
+            case.eps = float(rng.choice([0.02, 0.05, 0.3]))
+            case.delta = float(rng.choice([0.01, 0.05, 0.2]))
+            case.seed = int(rng.integers(0, 2**31))
+            params = dict(base_rate=float(rng.choice([0.025, 0.1, 0.3])), step=step)
+            if rng.random() < 0.3:
+                params["nested_base"] = 1
+            if rng.random() < 0.3:
+                params["rng_head_is_kv"] = 1
+            if rng.random() < 0.2:
+                params["gather_mode"] = 1
+            if rng.random() < 0.2:
+                params["force_budget"] = int(rng.choice([0, 7, 10**9]))
+            if rng.random() < 0.3:
+                params["topk_frac"] = float(rng.choice([0.01, 0.1]))
+            case.params = params
+            out_ref, det = run_oracle(case)
+            out, dbg, _ = run_gpu(case, plan=plan, dev=dict(dev, seq_lens=torch.from_numpy(lens).cuda()))
+            assert_parity(case, out, dbg, det, out_ref)
+            assert plan.last_status() & ~4 == 0, (it, step)
