@@ -153,7 +153,8 @@ int    vattn_set_debug(vattn_plan* plan, const vattn_debug* debug);
  * the eight words of Philox4x32-10(key = seed, counter = (c, batch<<16 | head, layer, step<<1 | stream)),
  * c = 0, 1, and whose round function is xor with the round key followed by three multiply / xor-shift steps.
  * Degenerate inputs: n = 0 -> out row = 0; sink+window >= n -> exact attention, budget 0;
- * k larger than the middle range is clipped.
+ * k larger than the middle range is clipped; sink = window = k = 0 with a forced budget of 0 leaves no token at
+ * all and the row is 0/0 (NaN), as the formula gives.
  * eps, delta in (0,1).  Errors: INVALID_ARG, WORKSPACE, CUDA.  The step is several kernel launches: after
  * VATTN_ERR_CUDA some of them may have been enqueued already (they run; `out` is then undefined), and the
  * first kernel waits for whatever the caller enqueued on `stream` before the call.
